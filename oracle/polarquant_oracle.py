@@ -1,0 +1,359 @@
+"""Float64 CPU oracle for the PolarQuant hot path (KV-cache encode + decode attention).
+
+THIS IS TEST INFRASTRUCTURE, NOT PRODUCT CODE.  Only the tests, the smoke check and
+the benchmark's CPU-baseline / reference legs may import it.  It shares nothing with
+the CUDA path: no tables, no constants, no helpers.  It is written to be checked
+against the paper by eye, not to be fast: every function follows one passage of the
+paper, step by step, in float64, vectorised over tokens only (no tiling, no fusion,
+no reordering of the method's steps).
+
+Conventions (the paper is 1-indexed, this file is 0-indexed):
+
+* Row-vector form of Algorithm 1: ``y = x @ S`` and ``x_hat = y_hat @ S.T``.
+* A level-l angle with index j is computed from entries ``2j`` (the cosine side) and
+  ``2j+1`` (the sine side) of the level-(l-1) radius vector; level 0 is ``y`` itself.
+* The recursion runs for ``L`` levels (Section 4.1 uses L = 4), so a d-vector becomes
+  ``d / 2**L`` radii plus ``d/2 + d/4 + ... + d/2**L`` angles.
+* Canonical code order of one vector: all level-1 codes (j = 0 .. d/2-1), then all
+  level-2 codes, ... then level-L codes.  Radii follow in index order.
+* Level 1 angles live in [0, 2*pi), higher levels in [0, pi/2] (Definition 1).
+
+Pins (tests/test_oracle_*.py): exact invertibility of the unquantised transform,
+block radius == block norm, norm preservation under S, Lemma 2 densities against the
+incomplete-beta CDF, Lloyd-Max fixed-point equations against independent quadrature,
+the worked d=4 example under tests/golden/, brute force on d=4 and d=16, closed-form
+expected distortion, and the len=1 / identical-keys attention special cases.
+Parity unpinned: nothing in this file; quality on real model caches is out of scope.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+
+import numpy as np
+
+TWO_PI = 2.0 * math.pi
+HALF_PI = 0.5 * math.pi
+
+DEFAULT_BITS = (4, 2, 2, 2)  # Section 4.1: 4 bits at level 1, 2 bits at levels 2..4
+
+
+# --------------------------------------------------------------------------------------
+# Random preconditioning (Section 3.2 footnote, Section 4.1: "a random rotational matrix")
+# --------------------------------------------------------------------------------------
+def make_rotation(d: int, seed: int) -> np.ndarray:
+    """Haar-distributed orthogonal d x d matrix: QR of a seeded Gaussian, with the
+    signs of R's diagonal folded into Q so that the distribution is uniform."""
+    rng = np.random.default_rng(seed)
+    g = rng.standard_normal((d, d))
+    q, r = np.linalg.qr(g)
+    sign = np.where(np.diag(r) < 0.0, -1.0, 1.0)
+    return q * sign[None, :]
+
+
+def rotate(x: np.ndarray, S: np.ndarray) -> np.ndarray:
+    """Algorithm 1 line 2: y_i = x_i . S for every row."""
+    return np.asarray(x, dtype=np.float64) @ np.asarray(S, dtype=np.float64)
+
+
+# --------------------------------------------------------------------------------------
+# Recursive polar transform (Definition 1, procedure Polar of Algorithm 1)
+# --------------------------------------------------------------------------------------
+def polar(y: np.ndarray, n_levels: int):
+    """Polar(y) for every row of ``y`` (shape [..., d]).
+
+    Returns ``(angles, radii)`` where ``angles[l-1]`` has shape [..., d / 2**l] and
+    ``radii`` (the level-L radius vector) has shape [..., d / 2**L].
+    """
+    r = np.asarray(y, dtype=np.float64)
+    angles = []
+    for level in range(1, n_levels + 1):
+        a = r[..., 0::2]  # entries 2j   : cosine side
+        b = r[..., 1::2]  # entries 2j+1 : sine side
+        psi = np.arctan2(b, a)
+        if level == 1:
+            # Level 1 covers the full circle [0, 2*pi); arctan2 returns (-pi, pi].
+            psi = np.where(psi < 0.0, psi + TWO_PI, psi)
+        psi = psi + 0.0  # turns -0.0 into +0.0
+        angles.append(psi)
+        r = np.hypot(a, b)
+    return angles, r
+
+
+def inverse_polar(angles, radii: np.ndarray) -> np.ndarray:
+    """The reverse map of Definition 1 in the form procedure DeQuant states it:
+    from the top level down, r[2j] = r_parent[j] cos(psi_j), r[2j+1] = r_parent[j] sin(psi_j)."""
+    r = np.asarray(radii, dtype=np.float64)
+    for psi in reversed(list(angles)):
+        child = np.empty(r.shape[:-1] + (2 * r.shape[-1],), dtype=np.float64)
+        child[..., 0::2] = r * np.cos(psi)
+        child[..., 1::2] = r * np.sin(psi)
+        r = child
+    return r
+
+
+# --------------------------------------------------------------------------------------
+# Angle densities (Lemma 2) and codebooks (Eq. 4)
+# --------------------------------------------------------------------------------------
+def level_density(level: int, psi):
+    """Marginal density of one level-``level`` angle of an isotropic Gaussian vector."""
+    psi = np.asarray(psi, dtype=np.float64)
+    if level == 1:
+        return np.full_like(psi, 1.0 / TWO_PI)
+    k = 2 ** (level - 1)  # the two child radii are norms of k-dimensional Gaussians
+    const = math.gamma(k) / (2.0 ** (k - 2) * math.gamma(k / 2.0) ** 2)
+    return const * np.sin(2.0 * psi) ** (k - 1)
+
+
+@dataclass(frozen=True)
+class Codebooks:
+    """Per level: ``centroids[l]`` (2**b_l ascending angles) and ``boundaries[l]``
+    (the 2**b_l - 1 interior cell boundaries)."""
+    bits: tuple
+    centroids: tuple
+    boundaries: tuple
+
+    @property
+    def n_levels(self) -> int:
+        return len(self.bits)
+
+    def flat_centroids(self) -> np.ndarray:
+        return np.concatenate(self.centroids)
+
+    def flat_boundaries(self) -> np.ndarray:
+        return np.concatenate(self.boundaries)
+
+
+_GL_X, _GL_W = np.polynomial.legendre.leggauss(96)
+
+
+def _integrate(fn, lo: float, hi: float) -> float:
+    """Gauss-Legendre quadrature of a smooth function on [lo, hi]."""
+    half = 0.5 * (hi - lo)
+    mid = 0.5 * (hi + lo)
+    return float(half * np.sum(_GL_W * fn(mid + half * _GL_X)))
+
+
+def lloyd_max(level: int, n_bits: int, init=None, tol: float = 1e-15, max_iter: int = 100000):
+    """Minimiser of Eq. 4 for one level: alternate (boundaries = midpoints of adjacent
+    centroids) and (centroid = conditional mean of the density on its cell) to a fixed
+    point.  Returns (centroids, interior boundaries)."""
+    n = 2 ** n_bits
+    lo, hi = (0.0, TWO_PI) if level == 1 else (0.0, HALF_PI)
+    if init is None:
+        theta = lo + (np.arange(n) + 0.5) * (hi - lo) / n
+    else:
+        theta = np.array(init, dtype=np.float64)
+    dens = lambda p: level_density(level, p)
+    mom = lambda p: p * level_density(level, p)
+    for _ in range(max_iter):
+        beta = 0.5 * (theta[:-1] + theta[1:])
+        edges = np.concatenate(([lo], beta, [hi]))
+        new = np.array([
+            _integrate(mom, edges[k], edges[k + 1]) / _integrate(dens, edges[k], edges[k + 1])
+            for k in range(n)
+        ])
+        delta = float(np.max(np.abs(new - theta)))
+        theta = new
+        if delta < tol:
+            break
+    beta = 0.5 * (theta[:-1] + theta[1:])
+    return theta, beta
+
+
+def fit_codebooks(bits=DEFAULT_BITS) -> Codebooks:
+    """Algorithm 1 line 3 with the analytic densities of Lemma 2 ("offline" codebook)."""
+    cents, bounds = [], []
+    for level, b in enumerate(bits, start=1):
+        c, t = lloyd_max(level, b)
+        cents.append(c)
+        bounds.append(t)
+    return Codebooks(tuple(bits), tuple(cents), tuple(bounds))
+
+
+def codebooks_from_arrays(bits, flat_centroids, flat_boundaries=None) -> Codebooks:
+    """Wrap externally supplied centroids (float64, ascending per level).  Boundaries
+    default to the midpoints of adjacent centroids (nearest-centroid rule)."""
+    flat_centroids = np.asarray(flat_centroids, dtype=np.float64)
+    cents, bounds, pos, bpos = [], [], 0, 0
+    for b in bits:
+        n = 2 ** b
+        c = flat_centroids[pos:pos + n].copy()
+        pos += n
+        if flat_boundaries is None:
+            t = 0.5 * (c[:-1] + c[1:])
+        else:
+            t = np.asarray(flat_boundaries, dtype=np.float64)[bpos:bpos + n - 1].copy()
+            bpos += n - 1
+        cents.append(c)
+        bounds.append(t)
+    return Codebooks(tuple(bits), tuple(cents), tuple(bounds))
+
+
+# --------------------------------------------------------------------------------------
+# Quant / DeQuant (Algorithm 1)
+# --------------------------------------------------------------------------------------
+def quantize_angles(psi: np.ndarray, boundaries: np.ndarray) -> np.ndarray:
+    """Procedure Quant: index of the nearest centroid.  With boundaries at the midpoints
+    this is the number of interior boundaries strictly below psi (ties go to the lower
+    index; distance on the line, not on the circle)."""
+    psi = np.asarray(psi, dtype=np.float64)
+    return np.sum(psi[..., None] > boundaries, axis=-1).astype(np.uint8)
+
+
+def quantize_angles_argmin(psi: np.ndarray, centroids: np.ndarray) -> np.ndarray:
+    """Procedure Quant exactly as printed: argmin_k |theta_k - psi| (first minimum)."""
+    psi = np.asarray(psi, dtype=np.float64)
+    return np.argmin(np.abs(psi[..., None] - centroids), axis=-1).astype(np.uint8)
+
+
+def round_radii_fp16(radii: np.ndarray):
+    """b_FPN = 16: one rounding float64 -> binary16, round-to-nearest-even, saturating
+    at the largest finite value.  Returns (fp16 array, number saturated)."""
+    r = np.asarray(radii, dtype=np.float64)
+    sat = r > 65504.0
+    r16 = np.where(sat, 65504.0, r).astype(np.float16)
+    return r16, int(np.count_nonzero(sat))
+
+
+def encode(x: np.ndarray, S: np.ndarray, cb: Codebooks):
+    """PolarQuant (Algorithm 1 lines 2 and 4) for rows of ``x`` ([..., d]).
+
+    Returns ``(codes, radii16, angles)``: uint8 codes in canonical order
+    [..., sum_l d/2**l], float16 radii [..., d/2**L], and the unquantised float64
+    angles per level (for boundary-distance accounting in the parity tests)."""
+    y = rotate(x, S)
+    angles, radii = polar(y, cb.n_levels)
+    codes = [quantize_angles(angles[l], cb.boundaries[l]) for l in range(cb.n_levels)]
+    radii16, _ = round_radii_fp16(radii)
+    return np.concatenate(codes, axis=-1), radii16, angles
+
+
+def split_codes(codes: np.ndarray, d: int, n_levels: int):
+    """Canonical code vector -> list of per-level code arrays."""
+    out, pos = [], 0
+    for level in range(1, n_levels + 1):
+        n = d >> level
+        out.append(codes[..., pos:pos + n])
+        pos += n
+    return out
+
+
+def dequant_rotated(codes: np.ndarray, radii16: np.ndarray, cb: Codebooks, d: int) -> np.ndarray:
+    """Procedure DeQuant without the final multiplication by S^T (the rotated basis)."""
+    per_level = split_codes(np.asarray(codes), d, cb.n_levels)
+    angles = [cb.centroids[l][per_level[l].astype(np.int64)] for l in range(cb.n_levels)]
+    return inverse_polar(angles, np.asarray(radii16).astype(np.float64))
+
+
+def dequant(codes, radii16, cb: Codebooks, S: np.ndarray) -> np.ndarray:
+    """Procedure DeQuant: centroid angles + stored radii -> r^(0) . S^T."""
+    d = S.shape[0]
+    return dequant_rotated(codes, radii16, cb, d) @ np.asarray(S, dtype=np.float64).T
+
+
+# --------------------------------------------------------------------------------------
+# Attention over the dequantised cache (Eq. 2 / Eq. 3)
+# --------------------------------------------------------------------------------------
+def softmax_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, scale: float) -> np.ndarray:
+    """softmax(K q * scale)^T V for one query ``q`` [d], keys/values [n, d]."""
+    s = (K @ q) * scale
+    s = s - np.max(s)
+    p = np.exp(s)
+    p = p / np.sum(p)
+    return p @ V
+
+
+def decode_attention(q, k_codes, k_radii, v_codes, v_radii, lens, cb: Codebooks, S, scale):
+    """Eq. 3 for a batch: one query per (sequence, query head).
+
+    q        [B, Hq, d]                     float64-convertible
+    *_codes  [B, Hkv, capacity, n_codes]    uint8, canonical order
+    *_radii  [B, Hkv, capacity, d/2**L]     float16
+    lens     [B]                            cached tokens per sequence
+    Query head h reads kv-head h // (Hq // Hkv).  Returns float64 [B, Hq, d].
+    """
+    q = np.asarray(q, dtype=np.float64)
+    B, Hq, d = q.shape
+    Hkv = k_codes.shape[1]
+    group = Hq // Hkv
+    out = np.zeros((B, Hq, d), dtype=np.float64)
+    for b in range(B):
+        n = int(lens[b])
+        for hk in range(Hkv):
+            K_hat = dequant(k_codes[b, hk, :n], k_radii[b, hk, :n], cb, S)
+            V_hat = dequant(v_codes[b, hk, :n], v_radii[b, hk, :n], cb, S)
+            for h in range(hk * group, (hk + 1) * group):
+                out[b, h] = softmax_attention(q[b, h], K_hat, V_hat, scale)
+    return out
+
+
+def exact_attention(q, K, V, lens, scale):
+    """Eq. 2 on the unquantised cache (quality information only, never a parity target).
+    K, V: [B, Hkv, capacity, d]."""
+    q = np.asarray(q, dtype=np.float64)
+    B, Hq, d = q.shape
+    Hkv = K.shape[1]
+    group = Hq // Hkv
+    out = np.zeros((B, Hq, d), dtype=np.float64)
+    for b in range(B):
+        n = int(lens[b])
+        for h in range(Hq):
+            hk = h // group
+            out[b, h] = softmax_attention(q[b, h], np.asarray(K[b, hk, :n], dtype=np.float64),
+                                          np.asarray(V[b, hk, :n], dtype=np.float64), scale)
+    return out
+
+
+# --------------------------------------------------------------------------------------
+# A cache that grows (the stream of Section 4: encode a prefill chunk, append one token)
+# --------------------------------------------------------------------------------------
+class OracleCache:
+    """Codes and radii of K and V for B sequences x Hkv heads with per-sequence lengths."""
+
+    def __init__(self, batch: int, n_kv_heads: int, capacity: int, d: int, cb: Codebooks, S):
+        self.cb, self.S, self.d = cb, np.asarray(S, dtype=np.float64), d
+        n_codes = sum(d >> l for l in range(1, cb.n_levels + 1))
+        n_radii = d >> cb.n_levels
+        shape = (batch, n_kv_heads, capacity)
+        self.k_codes = np.zeros(shape + (n_codes,), dtype=np.uint8)
+        self.v_codes = np.zeros(shape + (n_codes,), dtype=np.uint8)
+        self.k_radii = np.zeros(shape + (n_radii,), dtype=np.float16)
+        self.v_radii = np.zeros(shape + (n_radii,), dtype=np.float16)
+        self.lens = np.zeros(batch, dtype=np.int64)
+
+    def encode_chunk(self, b: int, K: np.ndarray, V: np.ndarray):
+        """Append a chunk of ``n`` tokens to sequence ``b``; K, V are [n, Hkv, d]."""
+        n = K.shape[0]
+        pos = int(self.lens[b])
+        for hk in range(K.shape[1]):
+            c, r, _ = encode(K[:, hk], self.S, self.cb)
+            self.k_codes[b, hk, pos:pos + n], self.k_radii[b, hk, pos:pos + n] = c, r
+            c, r, _ = encode(V[:, hk], self.S, self.cb)
+            self.v_codes[b, hk, pos:pos + n], self.v_radii[b, hk, pos:pos + n] = c, r
+        self.lens[b] = pos + n
+
+    def append(self, k_new: np.ndarray, v_new: np.ndarray):
+        """One new token for every sequence; k_new, v_new are [B, Hkv, d]."""
+        for b in range(k_new.shape[0]):
+            self.encode_chunk(b, k_new[b][None], v_new[b][None])
+
+    def attend(self, q: np.ndarray, scale: float) -> np.ndarray:
+        return decode_attention(q, self.k_codes, self.k_radii, self.v_codes, self.v_radii,
+                                self.lens, self.cb, self.S, scale)
+
+
+# --------------------------------------------------------------------------------------
+# Accounting helpers used by the parity tests (not part of the method)
+# --------------------------------------------------------------------------------------
+def boundary_distance(angles, cb: Codebooks):
+    """For every angle, the distance to the nearest decision point of its level: the
+    interior boundaries, plus the wrap point 0 == 2*pi at level 1.  Same layout as the
+    canonical code vector."""
+    out = []
+    for l, psi in enumerate(angles):
+        pts = cb.boundaries[l]
+        if l == 0:
+            pts = np.concatenate(([0.0], pts, [TWO_PI]))
+        out.append(np.min(np.abs(psi[..., None] - pts), axis=-1))
+    return np.concatenate(out, axis=-1)
