@@ -1,0 +1,174 @@
+/*
+ * polarquant.h -- C ABI of the B200 (sm_100a) PolarQuant KV-cache library.
+ *
+ * The library implements the data-parallel hot path of PolarQuant ("Quantizing KV Caches
+ * with Polar Transformation", arXiv 2502.02617): the KV-cache encoder of Algorithm 1
+ * (random preconditioning, recursive polar transform, per-level angle codebooks, bit
+ * packing) and decode attention over the packed cache (Eq. 3).
+ *
+ * General rules
+ *   - Every function returns an int32 status: PQ_OK (0) or a negative PQ_ERR_* value.
+ *     Nothing throws, aborts or traps.
+ *   - "host" pointers are ordinary CPU memory, "dev" pointers are CUDA device memory of
+ *     the current device.  The library allocates no device memory and keeps no state;
+ *     every buffer belongs to the caller.  Device pointers must be 16-byte aligned.
+ *   - Device work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream) and the call returns without synchronising.
+ *   - Problems that only the device can see (a sequence that would exceed `capacity`,
+ *     an empty sequence in attention, non-finite inputs) are written to the caller's
+ *     status words `status_dev` (int32[PQ_STATUS_WORDS], zero it before the first call):
+ *       [0] first error code seen (0 = none)      [1] non-finite input elements seen
+ *       [2] radii that saturated at the fp16 max  [3] 16-coordinate blocks that were
+ *                                                     re-encoded by the float64 path
+ *   - Row-vector convention of Algorithm 1: y = x . S, x_hat = y_hat . S^T; S is stored
+ *     row-major [head_dim][head_dim] in float32.
+ *   - Shapes: head_dim d in {16, 32, 64, 128}; L = 4 levels; bits (4,2,2,2) (Section 4.1);
+ *     a block is 16 consecutive rotated coordinates and owns one fp16 radius.
+ *   - Canonical code order of one vector (used by pq_unpack_codes): level-1 codes
+ *     j = 0..d/2-1, then level 2 (d/4), level 3 (d/8), level 4 (d/16); angle j of level l
+ *     is formed from entries 2j (cosine side) and 2j+1 (sine side) of level l-1.
+ *   - GQA: query head h reads kv head h / (n_q_heads / n_kv_heads).
+ */
+#ifndef POLARQUANT_H_
+#define POLARQUANT_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PQ_OK 0
+#define PQ_ERR_INVALID_ARG (-1)  /* null pointer, non-positive size, bad head ratio */
+#define PQ_ERR_UNSUPPORTED (-2)  /* head_dim / bits / dtype outside the supported set */
+#define PQ_ERR_ALIGNMENT (-3)    /* a device pointer is not 16-byte aligned */
+#define PQ_ERR_CAPACITY (-4)     /* a sequence would grow beyond `capacity` tokens */
+#define PQ_ERR_CUDA (-5)         /* a CUDA runtime call failed (launch error) */
+#define PQ_ERR_TIMEOUT (-6)      /* a bounded device-side wait gave up */
+#define PQ_ERR_NONFINITE (-7)    /* inputs contained NaN or Inf */
+#define PQ_ERR_EMPTY (-8)        /* attention over a sequence of length 0 */
+
+#define PQ_DTYPE_F32 0
+#define PQ_DTYPE_BF16 1
+
+#define PQ_STATUS_WORDS 4
+#define PQ_N_LEVELS 4
+#define PQ_N_CENTROIDS 28  /* 16 + 4 + 4 + 4 */
+#define PQ_N_BOUNDARIES 24 /* 15 + 3 + 3 + 3 */
+
+/* Human-readable name of a status code (static string, never NULL). */
+const char* pq_status_string(int32_t status);
+
+/* Tokens per cache token-block (a compile-time constant of the layout). */
+int32_t pq_token_block(void);
+
+/*
+ * Random preconditioning matrix (Section 3.2 footnote; Section 4.1 "a random rotational
+ * matrix"): a Haar-distributed orthogonal matrix obtained from the Householder QR of a
+ * seeded Gaussian matrix with the signs of diag(R) folded into Q.  Computed in float64 on
+ * the host, written as float32 to S_host[d*d] (row-major, y = x . S).  The same S is meant
+ * to be shared by keys, values, all layers and all heads.
+ */
+int32_t pq_make_rotation(int32_t head_dim, uint64_t seed, float* S_host);
+
+/*
+ * Angle codebooks (Algorithm 1 line 3, Eq. 4) for the analytic densities of Lemma 2:
+ * level 1 uniform on [0, 2pi), level l >= 2 proportional to sin^(2^(l-1)-1)(2 psi) on
+ * [0, pi/2].  Lloyd-Max iteration in float64 on the host.
+ *   bits[4]            bits per level; only {4,2,2,2} is supported
+ *   centroids_host     out, float64[PQ_N_CENTROIDS], ascending per level, levels concatenated
+ *   boundaries_host    out, float64[PQ_N_BOUNDARIES], interior cell boundaries (midpoints)
+ */
+int32_t pq_fit_codebooks(const int32_t* bits, double* centroids_host, double* boundaries_host);
+
+/*
+ * Derived device tables (decision lines of the boundaries, cos/sin of the centroids in the
+ * precisions the kernels use).  The codebook stays the paper's object; this is its compiled
+ * form.  Any ascending centroids are accepted (e.g. a data-fitted codebook); boundaries are
+ * the midpoints passed in.  tables_host must hold pq_tables_bytes() bytes; copy them to the
+ * device unchanged and pass that pointer as `tables_dev`.
+ */
+int64_t pq_tables_bytes(void);
+int32_t pq_build_tables(const double* centroids_host, const double* boundaries_host, void* tables_host);
+
+/* Size in bytes of the packed cache for `batch` sequences x n_kv_heads heads x (K and V),
+ * each with room for `capacity` tokens (rounded up to whole token-blocks).  At d = 128 a
+ * token costs exactly 62 bytes per head for K and 62 for V (Section 4.1: 3.875 bits per
+ * coordinate); d < 64 pads the level-3/4 codes of a token to whole bytes.  Negative on
+ * invalid arguments. */
+int64_t pq_cache_bytes(int32_t head_dim, int32_t batch, int32_t n_kv_heads, int32_t capacity);
+
+/* Scratch bytes pq_decode_attention needs (rotated queries, split partials, tickets). */
+int64_t pq_workspace_bytes(int32_t head_dim, int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
+                           int32_t max_len);
+
+/*
+ * Encode a prefill chunk of every sequence into the cache (Algorithm 1 lines 2 and 4, with
+ * the codebooks fixed): rotate by S, L = 4 polar levels per 16-block, nearest centroid per
+ * angle, fp16 block radii, bit packing.
+ *   K_dev, V_dev       [total_tokens][n_kv_heads][head_dim] elements of `in_dtype`; element
+ *                      (t, h, i) is at t*token_stride + h*head_stride + i (strides in elements)
+ *   cu_seqlens_dev     int32[batch+1]: rows cu[b] .. cu[b+1]-1 belong to sequence b
+ *                      (cu[0] = 0, cu[batch] = total_tokens)
+ *   cache_lens_dev     int32[batch]: tokens already cached; the rows of sequence b are
+ *                      written at positions lens[b] .. and lens[b] grows by its row count
+ *   capacity           token capacity per sequence the cache was sized for; a sequence that
+ *                      would exceed it is left untouched and PQ_ERR_CAPACITY is recorded
+ * Angle decisions are taken in float32 with a certified margin; decisions inside the margin
+ * are re-taken in float64, so codes match a float64 evaluation of Algorithm 1 unless the
+ * angle lies within ~1e-13 rad of a boundary.
+ */
+int32_t pq_encode_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                     const void* K_dev, const void* V_dev, int32_t in_dtype, int64_t token_stride,
+                     int64_t head_stride, const int32_t* cu_seqlens_dev, int32_t batch,
+                     int32_t total_tokens, void* cache_dev, int32_t* cache_lens_dev, int32_t capacity,
+                     int32_t* status_dev, void* stream);
+
+/*
+ * Streaming generation step (Section 4: the stream (q_i, k_i, v_i)): encode one new token per
+ * sequence at position lens[b] and increment lens[b].
+ *   k_new_dev, v_new_dev   [batch][n_kv_heads][head_dim] contiguous, `in_dtype`
+ */
+int32_t pq_append_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                     const void* k_new_dev, const void* v_new_dev, int32_t in_dtype, int32_t batch,
+                     void* cache_dev, int32_t* cache_lens_dev, int32_t capacity, int32_t* status_dev,
+                     void* stream);
+
+/*
+ * Decode attention over the packed cache (Eq. 3): for every sequence b and query head h,
+ * softmax(K_hat q * scale)^T V_hat over the lens[b] cached tokens, K_hat / V_hat being
+ * DeQuant (Algorithm 1) of the stored codes and radii.  The query is rotated once by S and
+ * the result once by S^T; keys and values are decoded in the rotated basis only.
+ *   q_dev          [batch][n_q_heads][head_dim] of `io_dtype` (PQ_DTYPE_BF16 or PQ_DTYPE_F32)
+ *   out_dev        same shape and dtype; accumulation is float32
+ *   max_len        host-side upper bound on lens[b] (used only to size the token splits)
+ *   workspace_dev  pq_workspace_bytes(...) bytes of scratch; contents need not be preserved
+ * A sequence with lens[b] = 0 yields zeros and records PQ_ERR_EMPTY.
+ */
+int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                            const void* tables_dev, const void* q_dev, int32_t io_dtype,
+                            const void* cache_dev, const int32_t* cache_lens_dev, int32_t batch,
+                            int32_t capacity, int32_t max_len, float scale, void* out_dev,
+                            void* workspace_dev, int32_t* status_dev, void* stream);
+
+/*
+ * Inspection (test support, not a hot path): unpack the first n_tokens positions of every
+ * (sequence, kv head, K|V) into canonical order.
+ *   codes_dev   uint8 [batch][n_kv_heads][2][n_tokens][15*d/16]   (index 2: 0 = K, 1 = V)
+ *   radii_dev   fp16  [batch][n_kv_heads][2][n_tokens][d/16]
+ */
+int32_t pq_unpack_codes(int32_t head_dim, int32_t n_kv_heads, const void* cache_dev, int32_t batch,
+                        int32_t capacity, int32_t n_tokens, uint8_t* codes_dev, void* radii_dev,
+                        void* stream);
+
+/* Inspection: DeQuant (Algorithm 1) of the first n_tokens positions, including the final
+ * multiplication by S^T, with the decode arithmetic of the attention kernel.
+ *   x_hat_dev   float32 [batch][n_kv_heads][2][n_tokens][d] */
+int32_t pq_dequant_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                      const void* cache_dev, int32_t batch, int32_t capacity, int32_t n_tokens,
+                      float* x_hat_dev, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* POLARQUANT_H_ */

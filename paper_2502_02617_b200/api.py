@@ -1,0 +1,233 @@
+"""Thin ctypes binding of the C ABI declared in include/polarquant.h.
+
+Argument marshalling only: every step of the path (rotation, polar transform, quantisation,
+packing, decode attention) runs inside the CUDA library.  PyTorch supplies device memory and
+streams.  There is no CPU fallback: if the shared library is missing the import of any entry
+point raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import c_char_p, c_double, c_float, c_int32, c_int64, c_uint64, c_void_p, POINTER
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libpolarquant.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_CAPACITY = -1, -2, -3, -4
+ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE, ERR_EMPTY = -5, -6, -7, -8
+DTYPE_F32, DTYPE_BF16 = 0, 1
+STATUS_WORDS = 4
+N_CENTROIDS, N_BOUNDARIES = 28, 24
+DEFAULT_BITS = (4, 2, 2, 2)
+
+# name -> (restype, argtypes); must list every symbol of include/polarquant.h
+_SIGNATURES = {
+    "pq_status_string": (c_char_p, [c_int32]),
+    "pq_token_block": (c_int32, []),
+    "pq_make_rotation": (c_int32, [c_int32, c_uint64, c_void_p]),
+    "pq_fit_codebooks": (c_int32, [POINTER(c_int32), POINTER(c_double), POINTER(c_double)]),
+    "pq_tables_bytes": (c_int64, []),
+    "pq_build_tables": (c_int32, [POINTER(c_double), POINTER(c_double), c_void_p]),
+    "pq_cache_bytes": (c_int64, [c_int32, c_int32, c_int32, c_int32]),
+    "pq_workspace_bytes": (c_int64, [c_int32, c_int32, c_int32, c_int32, c_int32]),
+    "pq_encode_kv": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int64, c_int64,
+                               c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_int32, c_void_p, c_void_p]),
+    "pq_append_kv": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
+                               c_void_p, c_void_p, c_int32, c_void_p, c_void_p]),
+    "pq_decode_attention": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p,
+                                      c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p,
+                                      c_void_p]),
+    "pq_unpack_codes": (c_int32, [c_int32, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p]),
+    "pq_dequant_kv": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p,
+                                c_void_p]),
+}
+
+_lib = None
+
+
+class PolarQuantError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} ({status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load the CUDA library (built in-tree by __graft_entry__.build()).  Raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} is missing: build it with `python -c 'import __graft_entry__ as g; g.build()'`"
+                              " -- there is no CPU fallback")
+        handle = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(handle, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = handle
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().pq_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != OK:
+        raise PolarQuantError(int(status), where)
+
+
+def _ptr(t) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return DTYPE_F32
+    if t.dtype == torch.bfloat16:
+        return DTYPE_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def token_block() -> int:
+    return int(lib().pq_token_block())
+
+
+def pq_make_rotation(d: int, seed: int) -> torch.Tensor:
+    """Seeded random rotation S (float32 CPU tensor [d, d], y = x @ S)."""
+    S = torch.empty((d, d), dtype=torch.float32)
+    _check(lib().pq_make_rotation(d, seed, S.data_ptr()), "pq_make_rotation")
+    return S
+
+
+def pq_fit_codebooks(bits=DEFAULT_BITS):
+    """Analytic Lloyd-Max codebooks: (centroids float64[28], boundaries float64[24]) CPU tensors."""
+    cen = torch.empty(N_CENTROIDS, dtype=torch.float64)
+    bnd = torch.empty(N_BOUNDARIES, dtype=torch.float64)
+    arr = (c_int32 * 4)(*bits)
+    _check(lib().pq_fit_codebooks(arr, ctypes.cast(cen.data_ptr(), POINTER(c_double)),
+                                  ctypes.cast(bnd.data_ptr(), POINTER(c_double))), "pq_fit_codebooks")
+    return cen, bnd
+
+
+def pq_build_tables(centroids: torch.Tensor, boundaries: torch.Tensor) -> torch.Tensor:
+    """Compiled device tables as a CPU uint8 tensor; move it to the GPU unchanged."""
+    centroids = centroids.to(torch.float64).contiguous()
+    boundaries = boundaries.to(torch.float64).contiguous()
+    out = torch.zeros(int(lib().pq_tables_bytes()), dtype=torch.uint8)
+    _check(lib().pq_build_tables(ctypes.cast(centroids.data_ptr(), POINTER(c_double)),
+                                 ctypes.cast(boundaries.data_ptr(), POINTER(c_double)), out.data_ptr()),
+           "pq_build_tables")
+    return out
+
+
+def pq_cache_bytes(d: int, batch: int, n_kv_heads: int, capacity: int) -> int:
+    n = int(lib().pq_cache_bytes(d, batch, n_kv_heads, capacity))
+    if n < 0:
+        raise PolarQuantError(n, "pq_cache_bytes")
+    return n
+
+
+def pq_workspace_bytes(d: int, batch: int, n_q_heads: int, n_kv_heads: int, max_len: int) -> int:
+    n = int(lib().pq_workspace_bytes(d, batch, n_q_heads, n_kv_heads, max_len))
+    if n < 0:
+        raise PolarQuantError(n, "pq_workspace_bytes")
+    return n
+
+
+def pq_encode_kv(S, tables, K, V, cu_seqlens, cache, cache_lens, capacity, status, stream=None):
+    """Encode packed ragged K, V [total_tokens, Hkv, d] into `cache`; cache_lens advances."""
+    total, n_kv_heads, d = K.shape
+    assert V.shape == K.shape and V.dtype == K.dtype and K.stride(2) == 1 and V.stride() == K.stride()
+    _check(lib().pq_encode_kv(d, n_kv_heads, _ptr(S), _ptr(tables), _ptr(K), _ptr(V), _dtype_code(K), K.stride(0),
+                              K.stride(1), _ptr(cu_seqlens), cu_seqlens.numel() - 1, total, _ptr(cache),
+                              _ptr(cache_lens), capacity, _ptr(status), _stream(stream)), "pq_encode_kv")
+
+
+def pq_append_kv(S, tables, k_new, v_new, cache, cache_lens, capacity, status, stream=None):
+    """Append one token per sequence: k_new, v_new [B, Hkv, d] contiguous."""
+    batch, n_kv_heads, d = k_new.shape
+    assert k_new.is_contiguous() and v_new.is_contiguous() and v_new.shape == k_new.shape
+    _check(lib().pq_append_kv(d, n_kv_heads, _ptr(S), _ptr(tables), _ptr(k_new), _ptr(v_new), _dtype_code(k_new),
+                              batch, _ptr(cache), _ptr(cache_lens), capacity, _ptr(status), _stream(stream)),
+           "pq_append_kv")
+
+
+def pq_decode_attention(S, tables, q, cache, cache_lens, n_kv_heads, capacity, max_len, scale, out, workspace,
+                        status, stream=None):
+    """Eq. 3 for one query per sequence: q, out [B, Hq, d] (bf16 or f32)."""
+    batch, n_q_heads, d = q.shape
+    assert q.is_contiguous() and out.is_contiguous() and out.shape == q.shape and out.dtype == q.dtype
+    _check(lib().pq_decode_attention(d, n_q_heads, n_kv_heads, _ptr(S), _ptr(tables), _ptr(q), _dtype_code(q),
+                                     _ptr(cache), _ptr(cache_lens), batch, capacity, max_len, float(scale),
+                                     _ptr(out), _ptr(workspace), _ptr(status), _stream(stream)),
+           "pq_decode_attention")
+
+
+def pq_unpack_codes(d, n_kv_heads, cache, batch, capacity, n_tokens, stream=None):
+    """Canonical codes uint8 [B, Hkv, 2, n_tokens, 15d/16] and radii fp16 [B, Hkv, 2, n_tokens, d/16]."""
+    codes = torch.empty((batch, n_kv_heads, 2, n_tokens, 15 * d // 16), dtype=torch.uint8, device=cache.device)
+    radii = torch.empty((batch, n_kv_heads, 2, n_tokens, d // 16), dtype=torch.float16, device=cache.device)
+    _check(lib().pq_unpack_codes(d, n_kv_heads, _ptr(cache), batch, capacity, n_tokens, _ptr(codes), _ptr(radii),
+                                 _stream(stream)), "pq_unpack_codes")
+    return codes, radii
+
+
+def pq_dequant_kv(d, n_kv_heads, S, tables, cache, batch, capacity, n_tokens, stream=None):
+    """DeQuant of the first n_tokens positions: float32 [B, Hkv, 2, n_tokens, d] (original basis)."""
+    out = torch.empty((batch, n_kv_heads, 2, n_tokens, d), dtype=torch.float32, device=cache.device)
+    _check(lib().pq_dequant_kv(d, n_kv_heads, _ptr(S), _ptr(tables), _ptr(cache), batch, capacity, n_tokens,
+                               _ptr(out), _stream(stream)), "pq_dequant_kv")
+    return out
+
+
+class PolarQuantCache:
+    """Convenience owner of the device buffers one (layer's) compressed KV cache needs."""
+
+    def __init__(self, batch, n_q_heads, n_kv_heads, d, capacity, seed=0, device="cuda", S=None, codebooks=None):
+        self.batch, self.n_q_heads, self.n_kv_heads, self.d, self.capacity = batch, n_q_heads, n_kv_heads, d, capacity
+        self.device = torch.device(device)
+        self.S_host = pq_make_rotation(d, seed) if S is None else S.to(torch.float32).cpu().contiguous()
+        self.centroids, self.boundaries = pq_fit_codebooks() if codebooks is None else codebooks
+        self.S = self.S_host.to(self.device)
+        self.tables = pq_build_tables(self.centroids, self.boundaries).to(self.device)
+        self.cache = torch.empty(pq_cache_bytes(d, batch, n_kv_heads, capacity), dtype=torch.uint8, device=self.device)
+        self.lens = torch.zeros(batch, dtype=torch.int32, device=self.device)
+        self.status = torch.zeros(STATUS_WORDS, dtype=torch.int32, device=self.device)
+        self.workspace = torch.empty(pq_workspace_bytes(d, batch, n_q_heads, n_kv_heads, capacity), dtype=torch.uint8,
+                                     device=self.device)
+
+    def encode(self, K, V, cu_seqlens, stream=None):
+        pq_encode_kv(self.S, self.tables, K, V, cu_seqlens, self.cache, self.lens, self.capacity, self.status, stream)
+
+    def append(self, k_new, v_new, stream=None):
+        pq_append_kv(self.S, self.tables, k_new, v_new, self.cache, self.lens, self.capacity, self.status, stream)
+
+    def attend(self, q, out=None, scale=None, max_len=None, stream=None):
+        out = torch.empty_like(q) if out is None else out
+        scale = self.d ** -0.5 if scale is None else scale
+        pq_decode_attention(self.S, self.tables, q, self.cache, self.lens, self.n_kv_heads, self.capacity,
+                            self.capacity if max_len is None else max_len, scale, out, self.workspace, self.status,
+                            stream)
+        return out
+
+    def unpack(self, n_tokens):
+        return pq_unpack_codes(self.d, self.n_kv_heads, self.cache, self.batch, self.capacity, n_tokens)
+
+    def dequant(self, n_tokens):
+        return pq_dequant_kv(self.d, self.n_kv_heads, self.S, self.tables, self.cache, self.batch, self.capacity,
+                             n_tokens)
+
+    def check_status(self):
+        st = self.status.cpu().tolist()
+        if st[0] != OK:
+            raise PolarQuantError(st[0], "device status")
+        return st

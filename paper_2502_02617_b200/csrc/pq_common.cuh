@@ -1,0 +1,156 @@
+// Shared definitions of the PolarQuant CUDA library: device tables, packed-cache layout,
+// exact (float64) polar quantiser of one 16-coordinate block.
+#pragma once
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/polarquant.h"
+
+namespace pq {
+
+constexpr int kTokenBlock = 64;  // tokens per cache token-block
+constexpr int kBlockDim = 16;    // coordinates per polar block (L = 4 levels)
+
+// Offsets of each level inside the concatenated centroid / boundary arrays.
+__host__ __device__ constexpr int cen_off(int level) { return level == 1 ? 0 : 16 + 4 * (level - 2); }
+__host__ __device__ constexpr int bnd_off(int level) { return level == 1 ? 0 : 15 + 3 * (level - 2); }
+
+// Compiled form of the codebooks (built on the host by pq_build_tables, copied verbatim to
+// the device by the caller).
+struct Tables {
+  // Decision lines: angle psi = atan2(b, a) is above boundary beta iff
+  // b cos(beta) - a sin(beta) > 0 (given the half-plane bookkeeping at level 1).
+  double bnd[PQ_N_BOUNDARIES];
+  double bnd_cos[PQ_N_BOUNDARIES];
+  double bnd_sin[PQ_N_BOUNDARIES];
+  float bnd_cosf[PQ_N_BOUNDARIES];
+  float bnd_sinf[PQ_N_BOUNDARIES];
+  int32_t bnd_upper[16];  // level 1: boundary k lies in [0, pi]
+  int32_t n_upper;        // number of level-1 boundaries in [0, pi]
+  uint32_t flags;         // bit 0: level-1 boundaries are exactly k*pi/8 (uniform codebook)
+  // cos / sin of the centroids (Algorithm 1, DeQuant).
+  float cen_cos[PQ_N_CENTROIDS];
+  float cen_sin[PQ_N_CENTROIDS];
+  // fp16 decode tables of the attention kernel.
+  //   l1[c]   = (cos, sin) of level-1 centroid c as half2
+  //   l2[c]   = (cos, sin) of level-2 centroid c as half2
+  //   u43[p][c4*4+c3] = t4(c4, side p>>1) * t3(c3, side p&1), p = position of the 4-coordinate
+  //             sub-block inside its 16-block (side 0 = cos, 1 = sin)
+  uint32_t l1_h2[16];
+  uint32_t l2_h2[4];
+  uint16_t u43_h[4][16];
+  uint32_t reserved[32];
+};
+
+constexpr uint32_t kFlagUniformL1 = 1u;
+
+// ------------------------------------------------------------------------------------------
+// Packed cache layout.
+//
+// cache = [sequence b][kv head h][token-block j][K | V] blocks of kTokenBlock tokens.
+// One block holds five planes, each token-major:
+//   L1   : 4*nb bytes per token, byte i = level-1 codes 2i (low nibble) and 2i+1 (high nibble)
+//   L2   : nb bytes per token,   byte i = level-2 codes 4i .. 4i+3, two bits each, LSB first
+//   L3   : max(1, nb/2) bytes,   same packing of the 2*nb level-3 codes
+//   L4   : max(1, nb/4) bytes,   same packing of the nb level-4 codes
+//   radii: nb fp16 values per token
+// nb = head_dim / 16.  At head_dim 128 this is 32 + 8 + 4 + 2 + 16 = 62 bytes per token and
+// every plane starts on a 16-byte boundary.  Each token owns whole bytes in every plane, so
+// tokens can be written independently (append needs no read-modify-write).
+// ------------------------------------------------------------------------------------------
+struct Layout {
+  int nb;                  // 16-blocks per vector
+  int b1, b2, b3, b4, br;  // bytes per token in each plane
+  int o2, o3, o4, orad;    // plane offsets inside a token-block (o1 = 0)
+  int block_bytes;         // bytes of one token-block (K or V)
+  int n_blocks_cap;        // token-blocks per sequence
+  int64_t head_bytes;      // bytes of one (sequence, head): n_blocks_cap * 2 * block_bytes
+};
+
+__host__ __device__ inline Layout make_layout(int head_dim, int capacity) {
+  Layout L;
+  L.nb = head_dim / kBlockDim;
+  L.b1 = 4 * L.nb;
+  L.b2 = L.nb;
+  L.b3 = L.nb >= 2 ? L.nb / 2 : 1;
+  L.b4 = L.nb >= 4 ? L.nb / 4 : 1;
+  L.br = 2 * L.nb;
+  L.o2 = kTokenBlock * L.b1;
+  L.o3 = L.o2 + kTokenBlock * L.b2;
+  L.o4 = L.o3 + kTokenBlock * L.b3;
+  L.orad = L.o4 + kTokenBlock * L.b4;
+  L.block_bytes = L.orad + kTokenBlock * L.br;
+  L.n_blocks_cap = (capacity + kTokenBlock - 1) / kTokenBlock;
+  L.head_bytes = (int64_t)L.n_blocks_cap * 2 * L.block_bytes;
+  return L;
+}
+
+// Start of the token-block that holds position `pos` of (sequence b, head h), K (kv=0) or V (kv=1).
+__host__ __device__ inline int64_t block_offset(const Layout& L, int n_kv_heads, int b, int h, int kv, int pos) {
+  return ((int64_t)b * n_kv_heads + h) * L.head_bytes + ((int64_t)(pos / kTokenBlock) * 2 + kv) * L.block_bytes;
+}
+
+// ------------------------------------------------------------------------------------------
+// Codes of one 16-coordinate block in canonical order.
+// ------------------------------------------------------------------------------------------
+struct BlockCodes {
+  uint32_t l1;  // 8 codes x 4 bits, code j at bits [4j, 4j+4)
+  uint32_t l2;  // 4 codes x 2 bits, LSB first
+  uint32_t l3;  // 2 codes x 2 bits
+  uint32_t l4;  // 1 code  x 2 bits
+};
+
+// Level-1 code of the pair (a, b): number of interior boundaries below atan2(b, a) mod 2pi.
+__device__ inline uint32_t quant_level1_exact(double a, double b, const Tables& tb) {
+  const bool upper = !(b < 0.0);  // psi in [0, pi]; b == -0.0 counts as upper (psi = 0 or pi)
+  uint32_t code = 0;
+#pragma unroll
+  for (int k = 0; k < 15; ++k) {
+    const double cross = b * tb.bnd_cos[k] - a * tb.bnd_sin[k];
+    const bool above = cross > 0.0;
+    const bool bu = tb.bnd_upper[k] != 0;
+    code += bu ? (upper ? above : true) : (upper ? false : above);
+  }
+  return code;
+}
+
+// Level >= 2 code of the pair of radii (a, b), both >= 0.
+__device__ inline uint32_t quant_upper_exact(double a, double b, int level, const Tables& tb) {
+  const int o = bnd_off(level);
+  uint32_t code = 0;
+#pragma unroll
+  for (int k = 0; k < 3; ++k) code += (b * tb.bnd_cos[o + k] - a * tb.bnd_sin[o + k]) > 0.0;
+  return code;
+}
+
+// Polar (Algorithm 1) + Quant of one block in float64.  Returns the level-4 radius.
+__device__ inline double polar_quant_block_exact(const double* y, const Tables& tb, BlockCodes& c) {
+  double r1[8], r2[4], r3[2];
+  c.l1 = c.l2 = c.l3 = 0;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    c.l1 |= quant_level1_exact(y[2 * j], y[2 * j + 1], tb) << (4 * j);
+    r1[j] = hypot(y[2 * j], y[2 * j + 1]);
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    c.l2 |= quant_upper_exact(r1[2 * j], r1[2 * j + 1], 2, tb) << (2 * j);
+    r2[j] = hypot(r1[2 * j], r1[2 * j + 1]);
+  }
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    c.l3 |= quant_upper_exact(r2[2 * j], r2[2 * j + 1], 3, tb) << (2 * j);
+    r3[j] = hypot(r2[2 * j], r2[2 * j + 1]);
+  }
+  c.l4 = quant_upper_exact(r3[0], r3[1], 4, tb);
+  return hypot(r3[0], r3[1]);
+}
+
+// Record the first error seen.
+__device__ inline void set_status(int32_t* status, int32_t code) {
+  if (status != nullptr) atomicCAS(status, 0, code);
+}
+
+}  // namespace pq

@@ -1,0 +1,436 @@
+// Decode attention over the packed cache (Eq. 3) and the inspection kernels.
+#include <math_constants.h>
+
+#include "pq_common.cuh"
+
+namespace pq {
+
+// ---- reading codes of (token, block) from a token-block held in global or shared memory ----
+__device__ inline uint32_t get_l1(const uint8_t* tb, const Layout& L, int tok, int blk) {
+  return *reinterpret_cast<const uint32_t*>(tb + tok * L.b1 + blk * 4);
+}
+__device__ inline uint32_t get_l2(const uint8_t* tb, const Layout& L, int tok, int blk) {
+  return tb[L.o2 + tok * L.b2 + blk];
+}
+__device__ inline uint32_t get_l3(const uint8_t* tb, const Layout& L, int tok, int blk) {
+  return (tb[L.o3 + tok * L.b3 + (blk >> 1)] >> (4 * (blk & 1))) & 0xFu;
+}
+__device__ inline uint32_t get_l4(const uint8_t* tb, const Layout& L, int tok, int blk) {
+  return (tb[L.o4 + tok * L.b4 + (blk >> 2)] >> (2 * (blk & 3))) & 0x3u;
+}
+__device__ inline float get_radius(const uint8_t* tb, const Layout& L, int tok, int blk) {
+  return __half2float(reinterpret_cast<const __half*>(tb + L.orad + tok * L.br)[blk]);
+}
+
+// DeQuant of one block in the rotated basis (Algorithm 1, DeQuant, without the final S^T):
+// from the level-4 radius down, child 2j = parent * cos(theta), child 2j+1 = parent * sin(theta).
+__device__ inline void decode_block(const uint8_t* tb, const Layout& L, int tok, int blk, const float* cen_cos,
+                                    const float* cen_sin, float* y) {
+  const uint32_t l1 = get_l1(tb, L, tok, blk), l2 = get_l2(tb, L, tok, blk);
+  const uint32_t l3 = get_l3(tb, L, tok, blk), l4 = get_l4(tb, L, tok, blk);
+  const float r = get_radius(tb, L, tok, blk);
+  float r3[2], r2[4], r1[8];
+  r3[0] = r * cen_cos[24 + l4];
+  r3[1] = r * cen_sin[24 + l4];
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    const uint32_t c = (l3 >> (2 * j)) & 3u;
+    r2[2 * j] = r3[j] * cen_cos[20 + c];
+    r2[2 * j + 1] = r3[j] * cen_sin[20 + c];
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint32_t c = (l2 >> (2 * j)) & 3u;
+    r1[2 * j] = r2[j] * cen_cos[16 + c];
+    r1[2 * j + 1] = r2[j] * cen_sin[16 + c];
+  }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const uint32_t c = (l1 >> (4 * j)) & 15u;
+    y[2 * j] = r1[j] * cen_cos[c];
+    y[2 * j + 1] = r1[j] * cen_sin[c];
+  }
+}
+
+// One rotated coordinate of one token.
+__device__ inline float decode_coord(const uint8_t* tb, const Layout& L, int tok, int coord, const float* cen_cos,
+                                     const float* cen_sin) {
+  const int blk = coord >> 4, i = coord & 15;
+  const uint32_t c1 = (get_l1(tb, L, tok, blk) >> (4 * (i >> 1))) & 15u;
+  const uint32_t c2 = (get_l2(tb, L, tok, blk) >> (2 * (i >> 2))) & 3u;
+  const uint32_t c3 = (get_l3(tb, L, tok, blk) >> (2 * (i >> 3))) & 3u;
+  const uint32_t c4 = get_l4(tb, L, tok, blk);
+  float v = get_radius(tb, L, tok, blk);
+  v *= (i & 8) ? cen_sin[24 + c4] : cen_cos[24 + c4];
+  v *= (i & 4) ? cen_sin[20 + c3] : cen_cos[20 + c3];
+  v *= (i & 2) ? cen_sin[16 + c2] : cen_cos[16 + c2];
+  v *= (i & 1) ? cen_sin[c1] : cen_cos[c1];
+  return v;
+}
+
+// ---- workspace -----------------------------------------------------------------------------
+struct Workspace {
+  float* qrot;       // [B][Hq][d]      rotated queries times scale*log2(e)
+  int32_t* tickets;  // [B][Hkv]
+  float* ml;         // [B][Hq][splits][2]
+  float* o;          // [B][Hq][splits][d]
+  int n_splits;
+  int64_t bytes;
+};
+
+__host__ inline int choose_splits(int batch, int n_kv_heads, int max_len) {
+  const int units = batch * n_kv_heads;
+  const int max_blocks = (max_len + kTokenBlock - 1) / kTokenBlock;
+  int splits = (148 * 4 + units - 1) / units;
+  if (splits > max_blocks) splits = max_blocks;
+  if (splits < 1) splits = 1;
+  if (splits > 256) splits = 256;
+  return splits;
+}
+
+__host__ inline Workspace carve_workspace(void* base, int d, int batch, int n_q_heads, int n_kv_heads, int max_len) {
+  Workspace w;
+  w.n_splits = choose_splits(batch, n_kv_heads, max_len);
+  auto align = [](int64_t x) { return (x + 255) & ~(int64_t)255; };
+  int64_t off = 0;
+  uint8_t* p = reinterpret_cast<uint8_t*>(base);
+  w.qrot = reinterpret_cast<float*>(p + off);
+  off = align(off + (int64_t)batch * n_q_heads * d * 4);
+  w.tickets = reinterpret_cast<int32_t*>(p + off);
+  off = align(off + (int64_t)batch * n_kv_heads * 4);
+  w.ml = reinterpret_cast<float*>(p + off);
+  off = align(off + (int64_t)batch * n_q_heads * w.n_splits * 2 * 4);
+  w.o = reinterpret_cast<float*>(p + off);
+  off = align(off + (int64_t)batch * n_q_heads * w.n_splits * d * 4);
+  w.bytes = off;
+  return w;
+}
+
+struct DecodeArgs {
+  int d, n_q_heads, n_kv_heads, batch, capacity, io_dtype;
+  float scale;
+  const float* S;
+  const Tables* tables;
+  const void* q;
+  const uint8_t* cache;
+  const int32_t* lens;
+  void* out;
+  int32_t* status;
+  Workspace ws;
+};
+
+// q' = (q . S) * scale * log2(e); also clears the split tickets.
+__global__ void rotate_query_kernel(DecodeArgs a) {
+  extern __shared__ float qs[];
+  const int bh = blockIdx.x, j = threadIdx.x, d = a.d;
+  const int64_t base = (int64_t)bh * d;
+  if (a.io_dtype == PQ_DTYPE_BF16) qs[j] = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.q)[base + j]);
+  else qs[j] = reinterpret_cast<const float*>(a.q)[base + j];
+  __syncthreads();
+  float acc = 0.f;
+  for (int k = 0; k < d; ++k) acc = fmaf(qs[k], a.S[k * d + j], acc);
+  a.ws.qrot[base + j] = acc * a.scale * 1.4426950408889634f;
+  if (bh < a.batch * a.n_kv_heads && j == 0) a.ws.tickets[bh] = 0;
+}
+
+constexpr int kMaxGroup = 8;       // query heads per kv head handled by one CTA
+constexpr int kSimpleThreads = 128;
+
+// Merge the split partials of the `g` query heads of (b, kv head), normalise, rotate back by
+// S^T and store.  Runs in the last CTA that finishes for this (b, kv head).
+__device__ void combine_and_store(const DecodeArgs& a, int b, int hk, int g, float* o_sm /* [d] */) {
+  const int d = a.d, ns = a.ws.n_splits, tid = threadIdx.x;
+  for (int hh = 0; hh < g; ++hh) {
+    const int h = hk * g + hh;
+    const float* ml = a.ws.ml + ((int64_t)b * a.n_q_heads + h) * ns * 2;
+    const float* op = a.ws.o + ((int64_t)b * a.n_q_heads + h) * ns * d;
+    float M = -CUDART_INF_F;
+    for (int s = 0; s < ns; ++s) M = fmaxf(M, ml[2 * s]);
+    float Lsum = 0.f;
+    for (int s = 0; s < ns; ++s) Lsum += ml[2 * s + 1] * (ml[2 * s] == -CUDART_INF_F ? 0.f : exp2f(ml[2 * s] - M));
+    if (tid < d) {
+      float acc = 0.f;
+      for (int s = 0; s < ns; ++s) {
+        const float w = ml[2 * s] == -CUDART_INF_F ? 0.f : exp2f(ml[2 * s] - M);
+        acc += op[(int64_t)s * d + tid] * w;
+      }
+      o_sm[tid] = Lsum > 0.f ? acc / Lsum : 0.f;
+    }
+    __syncthreads();
+    if (tid < d) {
+      // x_hat_i = sum_j y_hat_j S[i][j]
+      float acc = 0.f;
+      const float* srow = a.S + (int64_t)tid * d;
+      for (int j = 0; j < d; ++j) acc = fmaf(o_sm[j], srow[j], acc);
+      const int64_t idx = ((int64_t)b * a.n_q_heads + h) * d + tid;
+      if (a.io_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[idx] = __float2bfloat16(acc);
+      else reinterpret_cast<float*>(a.out)[idx] = acc;
+    }
+    __syncthreads();
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Straightforward float32 kernel: one CTA per (token split, kv head, sequence); per token-block
+// (1) stage the K and V blocks in shared memory, (2) a thread per token decodes the key and
+// forms the scores of the group's query heads, (3) online softmax per head, (4) a thread per
+// coordinate decodes the values and accumulates.  Serves every head_dim and group size.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel(DecodeArgs a) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  const int d = a.d, g = a.n_q_heads / a.n_kv_heads;
+  const Layout L = make_layout(d, a.capacity);
+  const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  uint8_t* kblk = smem;
+  uint8_t* vblk = smem + L.block_bytes;
+  float* qs = reinterpret_cast<float*>(smem + 2 * L.block_bytes);  // [g][d]
+  float* s_part = qs + g * d;                                      // [2][g][64]
+  float* p_sm = s_part + 2 * g * kTokenBlock;                      // [g][64]
+  float* corr_sm = p_sm + g * kTokenBlock;                         // [g]
+  float* m_run = corr_sm + kMaxGroup;                              // [g]
+  float* l_run = m_run + kMaxGroup;                                // [g]
+  float* cen_cos = l_run + kMaxGroup;                              // [28]
+  float* cen_sin = cen_cos + 32;                                   // [28]
+  __shared__ int is_last;
+
+  for (int i = tid; i < g * d; i += kSimpleThreads) qs[i] = a.ws.qrot[((int64_t)b * a.n_q_heads + hk * g) * d + i];
+  if (tid < PQ_N_CENTROIDS) {
+    cen_cos[tid] = a.tables->cen_cos[tid];
+    cen_sin[tid] = a.tables->cen_sin[tid];
+  }
+  if (tid < g) {
+    m_run[tid] = -CUDART_INF_F;
+    l_run[tid] = 0.f;
+  }
+  float o_acc[kMaxGroup];
+#pragma unroll
+  for (int h = 0; h < kMaxGroup; ++h) o_acc[h] = 0.f;
+
+  const int len = a.lens[b];
+  const int nblk_total = len > 0 ? (len + kTokenBlock - 1) / kTokenBlock : 0;
+  const int per = (nblk_total + a.ws.n_splits - 1) / a.ws.n_splits;
+  const int j0 = split * per;
+  const int j1 = min(nblk_total, j0 + per);
+  const uint8_t* head_base = a.cache + ((int64_t)b * a.n_kv_heads + hk) * L.head_bytes;
+  __syncthreads();
+
+  for (int jb = j0; jb < j1; ++jb) {
+    {
+      const uint4* src = reinterpret_cast<const uint4*>(head_base + (int64_t)jb * 2 * L.block_bytes);
+      uint4* dst = reinterpret_cast<uint4*>(smem);
+      for (int i = tid; i < 2 * L.block_bytes / 16; i += kSimpleThreads) dst[i] = src[i];
+    }
+    __syncthreads();
+    {  // scores
+      const int tk = tid & 63, half = tid >> 6;
+      float s[kMaxGroup];
+#pragma unroll
+      for (int h = 0; h < kMaxGroup; ++h) s[h] = 0.f;
+      for (int blk = half; blk < L.nb; blk += 2) {
+        float y[16];
+        decode_block(kblk, L, tk, blk, cen_cos, cen_sin, y);
+#pragma unroll
+        for (int h = 0; h < kMaxGroup; ++h) {
+          if (h < g) {
+            const float* qh = qs + h * d + blk * 16;
+            float acc = s[h];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) acc = fmaf(qh[i], y[i], acc);
+            s[h] = acc;
+          }
+        }
+      }
+#pragma unroll
+      for (int h = 0; h < kMaxGroup; ++h)
+        if (h < g) s_part[(half * g + h) * kTokenBlock + tk] = s[h];
+    }
+    __syncthreads();
+    for (int h = warp; h < g; h += kSimpleThreads / 32) {  // online softmax, one warp per head
+      float sv[2], mx = -CUDART_INF_F;
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        const int tk = lane + 32 * t;
+        const bool ok = jb * kTokenBlock + tk < len;
+        sv[t] = ok ? s_part[h * kTokenBlock + tk] + s_part[(g + h) * kTokenBlock + tk] : -CUDART_INF_F;
+        mx = fmaxf(mx, sv[t]);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      const float m_old = m_run[h], m_new = fmaxf(m_old, mx);
+      float sum = 0.f;
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        const float p = sv[t] == -CUDART_INF_F ? 0.f : exp2f(sv[t] - m_new);
+        p_sm[h * kTokenBlock + lane + 32 * t] = p;
+        sum += p;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      if (lane == 0) {
+        const float corr = m_old == -CUDART_INF_F ? 0.f : exp2f(m_old - m_new);
+        corr_sm[h] = corr;
+        m_run[h] = m_new;
+        l_run[h] = l_run[h] * corr + sum;
+      }
+    }
+    __syncthreads();
+    if (tid < d) {  // values
+#pragma unroll
+      for (int h = 0; h < kMaxGroup; ++h)
+        if (h < g) o_acc[h] *= corr_sm[h];
+      const int n_valid = min(kTokenBlock, len - jb * kTokenBlock);  // stale bytes past len may decode to NaN
+      for (int tk = 0; tk < n_valid; ++tk) {
+        const float v = decode_coord(vblk, L, tk, tid, cen_cos, cen_sin);
+#pragma unroll
+        for (int h = 0; h < kMaxGroup; ++h)
+          if (h < g) o_acc[h] = fmaf(p_sm[h * kTokenBlock + tk], v, o_acc[h]);
+      }
+    }
+    __syncthreads();
+  }
+
+  // partials of this split
+  for (int h = 0; h < g; ++h) {
+    const int64_t idx = ((int64_t)b * a.n_q_heads + hk * g + h) * a.ws.n_splits + split;
+    if (tid == 0) {
+      a.ws.ml[2 * idx] = m_run[h];
+      a.ws.ml[2 * idx + 1] = l_run[h];
+    }
+    if (tid < d) a.ws.o[idx * d + tid] = o_acc[h];
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    const int t = atomicAdd(a.ws.tickets + b * a.n_kv_heads + hk, 1);
+    is_last = (t == a.ws.n_splits - 1);
+    if (is_last && len <= 0) set_status(a.status, PQ_ERR_EMPTY);
+  }
+  __syncthreads();
+  if (is_last) {
+    __threadfence();
+    combine_and_store(a, b, hk, g, reinterpret_cast<float*>(smem));
+  }
+}
+
+// ---- inspection kernels ----------------------------------------------------------------------
+__global__ void unpack_codes_kernel(int d, int n_kv_heads, const uint8_t* cache, int batch, int capacity,
+                                    int n_tokens, uint8_t* codes, __half* radii) {
+  const Layout L = make_layout(d, capacity);
+  const int64_t n = (int64_t)batch * n_kv_heads * 2 * n_tokens;
+  const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (v >= n) return;
+  const int tok = (int)(v % n_tokens);
+  const int kv = (int)((v / n_tokens) & 1);
+  const int h = (int)((v / (2 * (int64_t)n_tokens)) % n_kv_heads);
+  const int b = (int)(v / (2 * (int64_t)n_tokens * n_kv_heads));
+  const uint8_t* tb = cache + block_offset(L, n_kv_heads, b, h, kv, tok);
+  const int t = tok % kTokenBlock;
+  const int n_codes = 15 * L.nb;
+  uint8_t* out = codes + v * n_codes;
+  for (int blk = 0; blk < L.nb; ++blk) {
+    const uint32_t l1 = get_l1(tb, L, t, blk), l2 = get_l2(tb, L, t, blk);
+    const uint32_t l3 = get_l3(tb, L, t, blk), l4 = get_l4(tb, L, t, blk);
+    for (int j = 0; j < 8; ++j) out[blk * 8 + j] = (l1 >> (4 * j)) & 15u;
+    for (int j = 0; j < 4; ++j) out[8 * L.nb + blk * 4 + j] = (l2 >> (2 * j)) & 3u;
+    for (int j = 0; j < 2; ++j) out[12 * L.nb + blk * 2 + j] = (l3 >> (2 * j)) & 3u;
+    out[14 * L.nb + blk] = l4;
+    radii[v * L.nb + blk] = reinterpret_cast<const __half*>(tb + L.orad + t * L.br)[blk];
+  }
+}
+
+__global__ void dequant_kernel(int d, int n_kv_heads, const float* S, const Tables* tables, const uint8_t* cache,
+                               int capacity, int n_tokens, float* x_hat) {
+  extern __shared__ float ysm[];
+  __shared__ float cc[32], cs[32];
+  const Layout L = make_layout(d, capacity);
+  const int64_t v = blockIdx.x;
+  const int j = threadIdx.x;
+  for (int i = j; i < PQ_N_CENTROIDS; i += blockDim.x) {
+    cc[i] = tables->cen_cos[i];
+    cs[i] = tables->cen_sin[i];
+  }
+  __syncthreads();
+  const int tok = (int)(v % n_tokens);
+  const int kv = (int)((v / n_tokens) & 1);
+  const int h = (int)((v / (2 * (int64_t)n_tokens)) % n_kv_heads);
+  const int b = (int)(v / (2 * (int64_t)n_tokens * n_kv_heads));
+  const uint8_t* tb = cache + block_offset(L, n_kv_heads, b, h, kv, tok);
+  ysm[j] = decode_coord(tb, L, tok % kTokenBlock, j, cc, cs);
+  __syncthreads();
+  float acc = 0.f;
+  for (int k = 0; k < d; ++k) acc = fmaf(ysm[k], S[(int64_t)j * d + k], acc);
+  x_hat[v * d + j] = acc;
+}
+
+}  // namespace pq
+
+extern "C" {
+
+int64_t pq_workspace_bytes(int32_t head_dim, int32_t batch, int32_t n_q_heads, int32_t n_kv_heads, int32_t max_len) {
+  if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
+  if (batch <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || max_len <= 0 || n_q_heads % n_kv_heads) return PQ_ERR_INVALID_ARG;
+  return pq::carve_workspace(nullptr, head_dim, batch, n_q_heads, n_kv_heads, max_len).bytes;
+}
+
+int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                            const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
+                            const int32_t* cache_lens_dev, int32_t batch, int32_t capacity, int32_t max_len,
+                            float scale, void* out_dev, void* workspace_dev, int32_t* status_dev, void* stream) {
+  if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
+  if (!S_dev || !tables_dev || !q_dev || !cache_dev || !cache_lens_dev || !out_dev || !workspace_dev || !status_dev)
+    return PQ_ERR_INVALID_ARG;
+  if (batch <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || capacity <= 0 || max_len <= 0) return PQ_ERR_INVALID_ARG;
+  if (n_q_heads % n_kv_heads) return PQ_ERR_INVALID_ARG;
+  if (n_q_heads / n_kv_heads > pq::kMaxGroup) return PQ_ERR_UNSUPPORTED;
+  if (io_dtype != PQ_DTYPE_F32 && io_dtype != PQ_DTYPE_BF16) return PQ_ERR_UNSUPPORTED;
+  const uintptr_t bits = (uintptr_t)S_dev | (uintptr_t)tables_dev | (uintptr_t)q_dev | (uintptr_t)cache_dev |
+                         (uintptr_t)out_dev | (uintptr_t)workspace_dev;
+  if (bits & 15) return PQ_ERR_ALIGNMENT;
+  if (batch > 65535 || n_kv_heads > 65535) return PQ_ERR_UNSUPPORTED;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
+  pq::DecodeArgs a;
+  a.d = head_dim; a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads; a.batch = batch; a.capacity = capacity;
+  a.io_dtype = io_dtype; a.scale = scale; a.S = S_dev; a.tables = reinterpret_cast<const pq::Tables*>(tables_dev);
+  a.q = q_dev; a.cache = reinterpret_cast<const uint8_t*>(cache_dev); a.lens = cache_lens_dev; a.out = out_dev;
+  a.status = status_dev;
+  a.ws = pq::carve_workspace(workspace_dev, head_dim, batch, n_q_heads, n_kv_heads, max_len);
+  const int g = n_q_heads / n_kv_heads;
+  pq::rotate_query_kernel<<<batch * n_q_heads, head_dim, head_dim * sizeof(float), st>>>(a);
+  const pq::Layout L = pq::make_layout(head_dim, capacity);
+  const size_t smem = 2 * L.block_bytes + sizeof(float) * ((size_t)g * head_dim + 3 * g * pq::kTokenBlock +
+                                                           3 * pq::kMaxGroup + 64);
+  dim3 grid(a.ws.n_splits, n_kv_heads, batch);
+  pq::decode_attention_simple_kernel<<<grid, pq::kSimpleThreads, smem, st>>>(a);
+  return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+}
+
+int32_t pq_unpack_codes(int32_t head_dim, int32_t n_kv_heads, const void* cache_dev, int32_t batch, int32_t capacity,
+                        int32_t n_tokens, uint8_t* codes_dev, void* radii_dev, void* stream) {
+  if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
+  if (!cache_dev || !codes_dev || !radii_dev || batch <= 0 || n_kv_heads <= 0 || n_tokens <= 0 || n_tokens > capacity)
+    return PQ_ERR_INVALID_ARG;
+  const int64_t n = (int64_t)batch * n_kv_heads * 2 * n_tokens;
+  pq::unpack_codes_kernel<<<(unsigned)((n + 127) / 128), 128, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      head_dim, n_kv_heads, reinterpret_cast<const uint8_t*>(cache_dev), batch, capacity, n_tokens, codes_dev,
+      reinterpret_cast<__half*>(radii_dev));
+  return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+}
+
+int32_t pq_dequant_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                      const void* cache_dev, int32_t batch, int32_t capacity, int32_t n_tokens, float* x_hat_dev,
+                      void* stream) {
+  if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
+  if (!S_dev || !tables_dev || !cache_dev || !x_hat_dev || batch <= 0 || n_kv_heads <= 0 || n_tokens <= 0 ||
+      n_tokens > capacity)
+    return PQ_ERR_INVALID_ARG;
+  const int64_t n = (int64_t)batch * n_kv_heads * 2 * n_tokens;
+  if (n >= (1ll << 31)) return PQ_ERR_UNSUPPORTED;
+  pq::dequant_kernel<<<(unsigned)n, head_dim, head_dim * sizeof(float), reinterpret_cast<cudaStream_t>(stream)>>>(
+      head_dim, n_kv_heads, S_dev, reinterpret_cast<const pq::Tables*>(tables_dev),
+      reinterpret_cast<const uint8_t*>(cache_dev), capacity, n_tokens, x_hat_dev);
+  return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+}
+
+}  // extern "C"

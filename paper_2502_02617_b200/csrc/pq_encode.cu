@@ -1,0 +1,245 @@
+// KV-cache encoder (Algorithm 1 lines 2 and 4 with fixed codebooks) and the append step.
+#include "pq_common.cuh"
+
+namespace pq {
+
+// Where the vectors of an encode call come from and go to.
+struct EncodeArgs {
+  const void* K;
+  const void* V;
+  int in_dtype;
+  int64_t token_stride, head_stride;
+  const int32_t* cu_seqlens;  // nullptr: one row per sequence (append)
+  int batch;
+  int total_tokens;
+  int n_kv_heads;
+  int head_dim;
+  int capacity;
+  const float* S;
+  const Tables* tables;
+  uint8_t* cache;
+  const int32_t* cache_lens;
+  int32_t* status;
+};
+
+__device__ inline float load_elem(const void* base, int dtype, int64_t idx) {
+  if (dtype == PQ_DTYPE_BF16) return __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(base)[idx]);
+  return reinterpret_cast<const float*>(base)[idx];
+}
+
+// Sequence that owns packed row `row` (largest b with cu[b] <= row).
+__device__ inline int find_sequence(const int32_t* cu, int batch, int row) {
+  int lo = 0, hi = batch - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (cu[mid] <= row) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+// Destination of packed row `row`: sequence and cache position, or pos = -1 if the sequence
+// would overflow the capacity (nothing of it is written).
+__device__ inline void row_destination(const EncodeArgs& a, int row, int* seq, int* pos) {
+  int b, first, count;
+  if (a.cu_seqlens == nullptr) {
+    b = row; first = row; count = 1;
+  } else {
+    b = find_sequence(a.cu_seqlens, a.batch, row);
+    first = a.cu_seqlens[b];
+    count = a.cu_seqlens[b + 1] - first;
+  }
+  const int start = a.cache_lens[b];
+  *seq = b;
+  if (start < 0 || start + count > a.capacity) {
+    set_status(a.status, PQ_ERR_CAPACITY);
+    *pos = -1;
+  } else {
+    *pos = start + (row - first);
+  }
+}
+
+// Store the codes and radius of block `blk` of the token at `pos_in_block` of a token-block.
+// Lanes of a warp that hold the nb blocks of one vector are consecutive and aligned, so the
+// level-3 / level-4 bit fields of a token are merged with shuffles before the byte store.
+__device__ inline void store_block(uint8_t* tb_base, const Layout& L, int tok, int blk, const BlockCodes& c,
+                                   __half radius, bool valid) {
+  const unsigned full = 0xffffffffu;
+  // level 3: 4 bits per block, two blocks per byte
+  uint32_t l3 = c.l3;
+  if (L.nb >= 2) {
+    const uint32_t other = __shfl_down_sync(full, l3, 1);
+    l3 |= other << 4;
+  }
+  // level 4: 2 bits per block, four blocks per byte
+  uint32_t l4 = c.l4;
+  if (L.nb >= 2) l4 |= __shfl_down_sync(full, l4, 1) << 2;
+  if (L.nb >= 4) l4 |= __shfl_down_sync(full, l4, 2) << 4;
+  if (!valid) return;
+  *reinterpret_cast<uint32_t*>(tb_base + tok * L.b1 + blk * 4) = c.l1;
+  tb_base[L.o2 + tok * L.b2 + blk] = (uint8_t)c.l2;
+  if (L.nb < 2 || (blk & 1) == 0) tb_base[L.o3 + tok * L.b3 + (blk >> 1)] = (uint8_t)l3;
+  if (L.nb < 4 || (blk & 3) == 0) tb_base[L.o4 + tok * L.b4 + (blk >> 2)] = (uint8_t)l4;
+  reinterpret_cast<__half*>(tb_base + L.orad + tok * L.br)[blk] = radius;
+}
+
+// ------------------------------------------------------------------------------------------
+// Reference-precision encoder: everything in float64.  One CTA of 128 threads handles
+// 16 * (128 / d) vectors: thread (group, j) forms coordinate j of y = x . S for the 16 vectors
+// of its group, then every thread quantises one 16-coordinate block.
+// A "vector" is (row, kv, head): index v = (row * 2 + kv) * n_kv_heads + head.
+// ------------------------------------------------------------------------------------------
+constexpr int kExactThreads = 128;
+constexpr int kExactVecPerGroup = 16;
+
+__global__ void __launch_bounds__(kExactThreads) encode_exact_kernel(EncodeArgs a) {
+  extern __shared__ double smem_d[];
+  const int d = a.head_dim;
+  const int groups = kExactThreads / d;
+  const int vec_per_cta = kExactVecPerGroup * groups;
+  double* xs = smem_d;                     // [vec_per_cta][d]
+  double* ys = smem_d + vec_per_cta * d;   // [vec_per_cta][d]
+  const int64_t n_vec = (int64_t)a.total_tokens * 2 * a.n_kv_heads;
+  const int64_t v0 = (int64_t)blockIdx.x * vec_per_cta;
+  const int tid = threadIdx.x;
+  const Layout L = make_layout(d, a.capacity);
+
+  int bad = 0;
+  for (int i = tid; i < vec_per_cta * d; i += kExactThreads) {
+    const int64_t v = v0 + i / d;
+    double x = 0.0;
+    if (v < n_vec) {
+      const int head = (int)(v % a.n_kv_heads);
+      const int kv = (int)((v / a.n_kv_heads) & 1);
+      const int64_t row = v / (2 * a.n_kv_heads);
+      const float f = load_elem(kv ? a.V : a.K, a.in_dtype, row * a.token_stride + head * a.head_stride + (i % d));
+      if (!isfinite(f)) ++bad;
+      x = (double)f;
+    }
+    xs[i] = x;
+  }
+  if (bad) {
+    atomicAdd(a.status + 1, bad);
+    set_status(a.status, PQ_ERR_NONFINITE);
+  }
+  __syncthreads();
+
+  {
+    const int grp = tid / d, j = tid % d;
+    double acc[kExactVecPerGroup];
+#pragma unroll
+    for (int i = 0; i < kExactVecPerGroup; ++i) acc[i] = 0.0;
+    const double* xg = xs + grp * kExactVecPerGroup * d;
+    for (int k = 0; k < d; ++k) {
+      const double s = (double)a.S[k * d + j];
+#pragma unroll
+      for (int i = 0; i < kExactVecPerGroup; ++i) acc[i] = fma(xg[i * d + k], s, acc[i]);
+    }
+#pragma unroll
+    for (int i = 0; i < kExactVecPerGroup; ++i) ys[(grp * kExactVecPerGroup + i) * d + j] = acc[i];
+  }
+  __syncthreads();
+
+  {
+    const int nb = L.nb;
+    const int lv = tid / nb, blk = tid % nb;  // local vector, block
+    const int64_t v = v0 + lv;
+    bool valid = v < n_vec;
+    BlockCodes c = {0, 0, 0, 0};
+    double radius = 0.0;
+    int seq = 0, pos = -1, head = 0, kv = 0;
+    if (valid) {
+      head = (int)(v % a.n_kv_heads);
+      kv = (int)((v / a.n_kv_heads) & 1);
+      row_destination(a, (int)(v / (2 * a.n_kv_heads)), &seq, &pos);
+      valid = pos >= 0;
+    }
+    if (valid) {
+      double y[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) y[i] = ys[lv * d + blk * 16 + i];
+      radius = polar_quant_block_exact(y, *a.tables, c);
+      if (radius > 65504.0) {
+        radius = 65504.0;
+        atomicAdd(a.status + 2, 1);
+      }
+    }
+    uint8_t* tb_base = a.cache + (valid ? block_offset(L, a.n_kv_heads, seq, head, kv, pos) : 0);
+    store_block(tb_base, L, valid ? pos % kTokenBlock : 0, blk, c, __double2half(radius), valid);
+  }
+}
+
+// lens[b] += rows of sequence b (skipped for sequences that did not fit).
+__global__ void advance_lens_kernel(const int32_t* cu_seqlens, int batch, int capacity, int32_t* lens) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= batch) return;
+  const int count = cu_seqlens ? cu_seqlens[b + 1] - cu_seqlens[b] : 1;
+  const int start = lens[b];
+  if (start >= 0 && start + count <= capacity) lens[b] = start + count;
+}
+
+static int32_t check_common(int head_dim, int n_kv_heads, const void* S, const void* tables, const void* cache,
+                            const void* lens, const void* status) {
+  if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
+  if (n_kv_heads <= 0 || !S || !tables || !cache || !lens || !status) return PQ_ERR_INVALID_ARG;
+  const uintptr_t bits = (uintptr_t)S | (uintptr_t)tables | (uintptr_t)cache;
+  if (bits & 15) return PQ_ERR_ALIGNMENT;
+  if (((uintptr_t)lens | (uintptr_t)status) & 3) return PQ_ERR_ALIGNMENT;
+  return PQ_OK;
+}
+
+static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
+  if (a.total_tokens == 0) return PQ_OK;
+  const int groups = kExactThreads / a.head_dim;
+  const int vec_per_cta = kExactVecPerGroup * groups;
+  const int64_t n_vec = (int64_t)a.total_tokens * 2 * a.n_kv_heads;
+  const int64_t grid = (n_vec + vec_per_cta - 1) / vec_per_cta;
+  const size_t smem = (size_t)2 * vec_per_cta * a.head_dim * sizeof(double);
+  encode_exact_kernel<<<(unsigned)grid, kExactThreads, smem, stream>>>(a);
+  advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, lens);
+  return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+}
+
+}  // namespace pq
+
+extern "C" {
+
+int32_t pq_encode_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                     const void* K_dev, const void* V_dev, int32_t in_dtype, int64_t token_stride,
+                     int64_t head_stride, const int32_t* cu_seqlens_dev, int32_t batch, int32_t total_tokens,
+                     void* cache_dev, int32_t* cache_lens_dev, int32_t capacity, int32_t* status_dev,
+                     void* stream) {
+  int32_t st = pq::check_common(head_dim, n_kv_heads, S_dev, tables_dev, cache_dev, cache_lens_dev, status_dev);
+  if (st != PQ_OK) return st;
+  if (!K_dev || !V_dev || !cu_seqlens_dev || batch <= 0 || total_tokens < 0 || capacity <= 0) return PQ_ERR_INVALID_ARG;
+  if (in_dtype != PQ_DTYPE_F32 && in_dtype != PQ_DTYPE_BF16) return PQ_ERR_UNSUPPORTED;
+  if (token_stride < 0 || head_stride < 0) return PQ_ERR_INVALID_ARG;
+  if ((int64_t)total_tokens * 2 * n_kv_heads >= (1ll << 31) * 16) return PQ_ERR_UNSUPPORTED;
+  pq::EncodeArgs a;
+  a.K = K_dev; a.V = V_dev; a.in_dtype = in_dtype;
+  a.token_stride = token_stride; a.head_stride = head_stride;
+  a.cu_seqlens = cu_seqlens_dev; a.batch = batch; a.total_tokens = total_tokens;
+  a.n_kv_heads = n_kv_heads; a.head_dim = head_dim; a.capacity = capacity;
+  a.S = S_dev; a.tables = reinterpret_cast<const pq::Tables*>(tables_dev);
+  a.cache = reinterpret_cast<uint8_t*>(cache_dev); a.cache_lens = cache_lens_dev; a.status = status_dev;
+  return pq::launch_encode(a, cache_lens_dev, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int32_t pq_append_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                     const void* k_new_dev, const void* v_new_dev, int32_t in_dtype, int32_t batch,
+                     void* cache_dev, int32_t* cache_lens_dev, int32_t capacity, int32_t* status_dev,
+                     void* stream) {
+  int32_t st = pq::check_common(head_dim, n_kv_heads, S_dev, tables_dev, cache_dev, cache_lens_dev, status_dev);
+  if (st != PQ_OK) return st;
+  if (!k_new_dev || !v_new_dev || batch <= 0 || capacity <= 0) return PQ_ERR_INVALID_ARG;
+  if (in_dtype != PQ_DTYPE_F32 && in_dtype != PQ_DTYPE_BF16) return PQ_ERR_UNSUPPORTED;
+  pq::EncodeArgs a;
+  a.K = k_new_dev; a.V = v_new_dev; a.in_dtype = in_dtype;
+  a.token_stride = (int64_t)n_kv_heads * head_dim; a.head_stride = head_dim;
+  a.cu_seqlens = nullptr; a.batch = batch; a.total_tokens = batch;
+  a.n_kv_heads = n_kv_heads; a.head_dim = head_dim; a.capacity = capacity;
+  a.S = S_dev; a.tables = reinterpret_cast<const pq::Tables*>(tables_dev);
+  a.cache = reinterpret_cast<uint8_t*>(cache_dev); a.cache_lens = cache_lens_dev; a.status = status_dev;
+  return pq::launch_encode(a, cache_lens_dev, reinterpret_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

@@ -1,0 +1,207 @@
+// Host-side entry points: rotation generator, Lloyd-Max codebooks, derived tables, size queries.
+#include <cmath>
+#include <cstring>
+#include <vector>
+
+#include "pq_common.cuh"
+
+namespace {
+
+const double kPi = 3.14159265358979323846264338327950288;
+
+// ---- counter-based Gaussian generator (splitmix64 + Box-Muller) --------------------------
+inline uint64_t splitmix64(uint64_t x) {
+  x += 0x9E3779B97F4A7C15ull;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  return x ^ (x >> 31);
+}
+inline double uniform01(uint64_t seed, uint64_t idx) {  // in (0, 1)
+  const uint64_t bits = splitmix64(splitmix64(seed) ^ (idx * 0xD6E8FEB86659FD93ull + 0x2545F4914F6CDD1Dull));
+  return ((double)(bits >> 11) + 0.5) * (1.0 / 9007199254740992.0);
+}
+inline double gaussian(uint64_t seed, uint64_t idx) {
+  const double u1 = uniform01(seed, 2 * idx), u2 = uniform01(seed, 2 * idx + 1);
+  return std::sqrt(-2.0 * std::log(u1)) * std::cos(2.0 * kPi * u2);
+}
+
+// ---- Lemma 2 densities and Simpson quadrature --------------------------------------------
+inline double density_unnorm(int level, double psi) {
+  if (level == 1) return 1.0;
+  const int k = 1 << (level - 1);
+  return std::pow(std::sin(2.0 * psi), k - 1);
+}
+// Integrals of f and psi*f over [lo, hi] by composite Simpson (the integrand is a polynomial
+// in sin/cos, so 4096 panels are far beyond float64 accuracy).
+inline void cell_moments(int level, double lo, double hi, double* m0, double* m1) {
+  const int n = 4096;
+  const double h = (hi - lo) / n;
+  double s0 = 0.0, s1 = 0.0;
+  for (int i = 0; i <= n; ++i) {
+    const double p = lo + h * i;
+    const double w = (i == 0 || i == n) ? 1.0 : ((i & 1) ? 4.0 : 2.0);
+    const double f = density_unnorm(level, p);
+    s0 += w * f;
+    s1 += w * f * p;
+  }
+  *m0 = s0 * h / 3.0;
+  *m1 = s1 * h / 3.0;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* pq_status_string(int32_t status) {
+  switch (status) {
+    case PQ_OK: return "ok";
+    case PQ_ERR_INVALID_ARG: return "invalid argument";
+    case PQ_ERR_UNSUPPORTED: return "unsupported configuration";
+    case PQ_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
+    case PQ_ERR_CAPACITY: return "cache capacity exceeded";
+    case PQ_ERR_CUDA: return "CUDA runtime error";
+    case PQ_ERR_TIMEOUT: return "bounded device wait timed out";
+    case PQ_ERR_NONFINITE: return "non-finite input";
+    case PQ_ERR_EMPTY: return "attention over an empty sequence";
+    default: return "unknown status";
+  }
+}
+
+int32_t pq_token_block(void) { return pq::kTokenBlock; }
+
+int32_t pq_make_rotation(int32_t d, uint64_t seed, float* S_host) {
+  if (S_host == nullptr || d <= 0) return PQ_ERR_INVALID_ARG;
+  if (d > 4096) return PQ_ERR_UNSUPPORTED;
+  std::vector<double> A((size_t)d * d), Q((size_t)d * d, 0.0), v(d), w(d), rdiag(d);
+  for (int64_t i = 0; i < (int64_t)d * d; ++i) A[i] = gaussian(seed, (uint64_t)i);
+  for (int i = 0; i < d; ++i) Q[(size_t)i * d + i] = 1.0;
+  // Householder QR: A = Q R.  Reflector k zeroes column k below the diagonal.
+  for (int k = 0; k < d; ++k) {
+    double norm = 0.0;
+    for (int i = k; i < d; ++i) norm += A[(size_t)i * d + k] * A[(size_t)i * d + k];
+    norm = std::sqrt(norm);
+    const double x0 = A[(size_t)k * d + k];
+    const double alpha = x0 >= 0.0 ? -norm : norm;
+    rdiag[k] = alpha;
+    double vnorm = 0.0;
+    for (int i = k; i < d; ++i) {
+      v[i] = A[(size_t)i * d + k] - (i == k ? alpha : 0.0);
+      vnorm += v[i] * v[i];
+    }
+    if (vnorm == 0.0) continue;
+    const double beta = 2.0 / vnorm;
+    // A <- (I - beta v v^T) A on rows k..d-1
+    for (int j = k; j < d; ++j) {
+      double s = 0.0;
+      for (int i = k; i < d; ++i) s += v[i] * A[(size_t)i * d + j];
+      w[j] = s * beta;
+    }
+    for (int i = k; i < d; ++i)
+      for (int j = k; j < d; ++j) A[(size_t)i * d + j] -= v[i] * w[j];
+    // Q <- Q (I - beta v v^T) on columns k..d-1
+    for (int i = 0; i < d; ++i) {
+      double s = 0.0;
+      for (int j = k; j < d; ++j) s += Q[(size_t)i * d + j] * v[j];
+      s *= beta;
+      for (int j = k; j < d; ++j) Q[(size_t)i * d + j] -= s * v[j];
+    }
+  }
+  for (int i = 0; i < d; ++i)
+    for (int j = 0; j < d; ++j) S_host[(size_t)i * d + j] = (float)(Q[(size_t)i * d + j] * (rdiag[j] < 0.0 ? -1.0 : 1.0));
+  return PQ_OK;
+}
+
+int32_t pq_fit_codebooks(const int32_t* bits, double* centroids_host, double* boundaries_host) {
+  if (bits == nullptr || centroids_host == nullptr || boundaries_host == nullptr) return PQ_ERR_INVALID_ARG;
+  if (bits[0] != 4 || bits[1] != 2 || bits[2] != 2 || bits[3] != 2) return PQ_ERR_UNSUPPORTED;
+  for (int level = 1; level <= PQ_N_LEVELS; ++level) {
+    const int n = 1 << bits[level - 1];
+    const double lo = 0.0, hi = level == 1 ? 2.0 * kPi : 0.5 * kPi;
+    double* theta = centroids_host + pq::cen_off(level);
+    double* beta = boundaries_host + pq::bnd_off(level);
+    for (int k = 0; k < n; ++k) theta[k] = lo + (k + 0.5) * (hi - lo) / n;
+    for (int it = 0; it < 100000; ++it) {
+      double delta = 0.0;
+      for (int k = 0; k + 1 < n; ++k) beta[k] = 0.5 * (theta[k] + theta[k + 1]);
+      for (int k = 0; k < n; ++k) {
+        const double a = k == 0 ? lo : beta[k - 1], b = k == n - 1 ? hi : beta[k];
+        double m0, m1;
+        cell_moments(level, a, b, &m0, &m1);
+        const double t = m1 / m0;
+        delta = std::fmax(delta, std::fabs(t - theta[k]));
+        theta[k] = t;
+      }
+      if (delta < 1e-15) break;
+    }
+    for (int k = 0; k + 1 < n; ++k) beta[k] = 0.5 * (theta[k] + theta[k + 1]);
+  }
+  return PQ_OK;
+}
+
+int64_t pq_tables_bytes(void) { return (int64_t)sizeof(pq::Tables); }
+
+int32_t pq_build_tables(const double* cen, const double* bnd, void* tables_host) {
+  if (cen == nullptr || bnd == nullptr || tables_host == nullptr) return PQ_ERR_INVALID_ARG;
+  for (int level = 1; level <= PQ_N_LEVELS; ++level) {
+    const int n = level == 1 ? 16 : 4;
+    const double hi = level == 1 ? 2.0 * kPi : 0.5 * kPi;
+    for (int k = 0; k < n; ++k) {
+      const double c = cen[pq::cen_off(level) + k];
+      if (!(c >= 0.0 && c <= hi)) return PQ_ERR_INVALID_ARG;
+      if (k > 0 && !(c > cen[pq::cen_off(level) + k - 1])) return PQ_ERR_INVALID_ARG;
+    }
+    for (int k = 0; k + 1 < n; ++k) {
+      const double b = bnd[pq::bnd_off(level) + k];
+      if (!(b > 0.0 && b < hi)) return PQ_ERR_INVALID_ARG;
+      if (k > 0 && !(b > bnd[pq::bnd_off(level) + k - 1])) return PQ_ERR_INVALID_ARG;
+    }
+  }
+  pq::Tables t;
+  std::memset(&t, 0, sizeof(t));
+  bool uniform = true;
+  for (int k = 0; k < PQ_N_BOUNDARIES; ++k) {
+    t.bnd[k] = bnd[k];
+    t.bnd_cos[k] = std::cos(bnd[k]);
+    t.bnd_sin[k] = std::sin(bnd[k]);
+    t.bnd_cosf[k] = (float)t.bnd_cos[k];
+    t.bnd_sinf[k] = (float)t.bnd_sin[k];
+  }
+  for (int k = 0; k < 15; ++k) {
+    t.bnd_upper[k] = bnd[k] <= kPi ? 1 : 0;
+    t.n_upper += t.bnd_upper[k];
+    if (std::fabs(bnd[k] - (k + 1) * kPi / 8.0) > 1e-12) uniform = false;
+  }
+  t.flags = uniform ? pq::kFlagUniformL1 : 0u;
+  for (int k = 0; k < PQ_N_CENTROIDS; ++k) {
+    t.cen_cos[k] = (float)std::cos(cen[k]);
+    t.cen_sin[k] = (float)std::sin(cen[k]);
+  }
+  auto h2 = [](double lo, double hi) -> uint32_t {
+    const __half a = __double2half(lo), b = __double2half(hi);
+    uint16_t ua, ub;
+    std::memcpy(&ua, &a, 2);
+    std::memcpy(&ub, &b, 2);
+    return (uint32_t)ua | ((uint32_t)ub << 16);
+  };
+  for (int c = 0; c < 16; ++c) t.l1_h2[c] = h2(std::cos(cen[c]), std::sin(cen[c]));
+  for (int c = 0; c < 4; ++c) t.l2_h2[c] = h2(std::cos(cen[16 + c]), std::sin(cen[16 + c]));
+  for (int p = 0; p < 4; ++p)
+    for (int c4 = 0; c4 < 4; ++c4)
+      for (int c3 = 0; c3 < 4; ++c3) {
+        const double a4 = cen[24 + c4], a3 = cen[20 + c3];
+        const double t4 = (p >> 1) ? std::sin(a4) : std::cos(a4);
+        const double t3 = (p & 1) ? std::sin(a3) : std::cos(a3);
+        t.u43_h[p][c4 * 4 + c3] = (uint16_t)(h2(t4 * t3, 0.0) & 0xFFFFu);
+      }
+  std::memcpy(tables_host, &t, sizeof(t));
+  return PQ_OK;
+}
+
+int64_t pq_cache_bytes(int32_t head_dim, int32_t batch, int32_t n_kv_heads, int32_t capacity) {
+  if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
+  if (batch <= 0 || n_kv_heads <= 0 || capacity <= 0) return PQ_ERR_INVALID_ARG;
+  const pq::Layout L = pq::make_layout(head_dim, capacity);
+  return (int64_t)batch * n_kv_heads * L.head_bytes;
+}
+
+}  // extern "C"

@@ -1,0 +1,217 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64 oracle on the same
+seeded bytes.  Codes are compared bit for bit (mismatches are allowed only within 1e-6 rad of a
+decision boundary and must stay below 1e-5 of all codes), decoded keys to 1e-3 and attention
+outputs to 2e-3 relative L2."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2502_02617_b200 as pq
+from paper_2502_02617_b200 import synthetic
+from oracle import polarquant_oracle as orc
+from parity_utils import (TOL_ATTENTION, TOL_DECODED, assert_codes_match, assert_radii_match, code_mismatch_report,
+                          oracle_codebooks, rel_l2, to_f64)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _encode_and_compare(cache, K, V, lens_list, start=None):
+    """Encode ragged K, V ([sum(lens), Hkv, d]) and compare codes / radii with the oracle."""
+    cu = torch.tensor(np.concatenate(([0], np.cumsum(lens_list))), dtype=torch.int32, device=DEV)
+    start = [0] * len(lens_list) if start is None else start
+    cache.encode(K, V, cu)
+    torch.cuda.synchronize()
+    cache.check_status()
+    cb = oracle_codebooks(cache)
+    S = cache.S_host.double().numpy()
+    n_max = max(s + n for s, n in zip(start, lens_list))
+    codes, radii = cache.unpack(n_max)
+    codes, radii = codes.cpu().numpy(), radii.cpu().numpy()
+    Kc, Vc = to_f64(K), to_f64(V)
+    total = dict(total=0, inside=0, outside=0)
+    row = 0
+    for b, n in enumerate(lens_list):
+        for kv, X in ((0, Kc), (1, Vc)):
+            for h in range(cache.n_kv_heads):
+                rep = code_mismatch_report(codes[b, h, kv, start[b]:start[b] + n], X[row:row + n, h], S, cb)
+                assert_radii_match(radii[b, h, kv, start[b]:start[b] + n], rep["radii16"])
+                for key in total:
+                    total[key] += rep[key]
+        row += n
+    assert_codes_match(total)
+    return total
+
+
+def _oracle_cache(cache, K, V, lens_list):
+    cb = oracle_codebooks(cache)
+    ref = orc.OracleCache(cache.batch, cache.n_kv_heads, cache.capacity, cache.d, cb, cache.S_host.double().numpy())
+    Kc, Vc = to_f64(K), to_f64(V)
+    row = 0
+    for b, n in enumerate(lens_list):
+        ref.encode_chunk(b, Kc[row:row + n], Vc[row:row + n])
+        row += n
+    return ref
+
+
+def test_config1_tiny_reference_d16_fp32():
+    """1 sequence, 1 kv head, 1 query head, d = 16, 256 tokens, fp32, full 4-level recursion."""
+    d, n = 16, 256
+    cache = pq.PolarQuantCache(1, 1, 1, d, capacity=n, seed=0, device=DEV)
+    K, V = synthetic.kv_like(0, n, 1, d, torch.float32, DEV, n_outliers=0)
+    rep = _encode_and_compare(cache, K, V, [n])
+    assert rep["inside"] == 0  # the float64 path decides every angle here
+    assert cache.lens.cpu().tolist() == [n]
+    ref = _oracle_cache(cache, K, V, [n])
+    xh = to_f64(cache.dequant(n))
+    S = cache.S_host.double().numpy()
+    assert rel_l2(xh[0, 0, 0], orc.dequant(ref.k_codes[0, 0], ref.k_radii[0, 0], ref.cb, S)) < TOL_DECODED
+    assert rel_l2(xh[0, 0, 1], orc.dequant(ref.v_codes[0, 0], ref.v_radii[0, 0], ref.cb, S)) < TOL_DECODED
+    q = synthetic.queries(0, 1, 1, d, torch.float32, DEV)
+    out = cache.attend(q, scale=0.25)
+    torch.cuda.synchronize()
+    assert rel_l2(to_f64(out), ref.attend(to_f64(q), 0.25)) < TOL_ATTENTION
+
+
+@pytest.mark.parametrize("d,Hq,Hkv", [(128, 8, 2), (64, 4, 4), (32, 2, 1), (16, 8, 1)])
+def test_ragged_batch_encode_dequant_attention(d, Hq, Hkv):
+    """Several token-blocks plus ragged tails; bf16 inputs with outlier key channels."""
+    lens_list = [130, 1, 64, 257]
+    B = len(lens_list)
+    cache = pq.PolarQuantCache(B, Hq, Hkv, d, capacity=300, seed=3, device=DEV)
+    K, V = synthetic.kv_like(7, sum(lens_list), Hkv, d, torch.bfloat16, DEV)
+    _encode_and_compare(cache, K, V, lens_list)
+    assert cache.lens.cpu().tolist() == lens_list
+    ref = _oracle_cache(cache, K, V, lens_list)
+    xh = to_f64(cache.dequant(max(lens_list)))
+    S = cache.S_host.double().numpy()
+    for b, n in enumerate(lens_list):
+        for h in range(Hkv):
+            assert rel_l2(xh[b, h, 0, :n], orc.dequant(ref.k_codes[b, h, :n], ref.k_radii[b, h, :n], ref.cb, S)) < TOL_DECODED
+            assert rel_l2(xh[b, h, 1, :n], orc.dequant(ref.v_codes[b, h, :n], ref.v_radii[b, h, :n], ref.cb, S)) < TOL_DECODED
+    q = synthetic.queries(9, B, Hq, d, torch.bfloat16, DEV)
+    out = cache.attend(q)
+    torch.cuda.synchronize()
+    cache.check_status()
+    want = ref.attend(to_f64(q), d ** -0.5)
+    assert rel_l2(to_f64(out), want) < TOL_ATTENTION
+    for b in range(B):  # per sequence too, so a short sequence cannot hide behind a long one
+        assert rel_l2(to_f64(out)[b], want[b]) < 2 * TOL_ATTENTION
+
+
+def test_chunked_prefill_and_append_equal_one_shot_and_oracle():
+    d, Hq, Hkv = 128, 8, 2
+    lens_list = [100, 37]
+    B = len(lens_list)
+    K, V = synthetic.kv_like(11, sum(lens_list), Hkv, d, torch.bfloat16, DEV)
+    one = pq.PolarQuantCache(B, Hq, Hkv, d, capacity=160, seed=4, device=DEV)
+    _encode_and_compare(one, K, V, lens_list)
+    two = pq.PolarQuantCache(B, Hq, Hkv, d, capacity=160, seed=4, device=DEV)
+    # chunk 1: first 60 / 20 tokens, chunk 2: the rest minus the last token, then append the last token
+    first, rest = [60, 20], [39, 16]
+    idx1 = torch.cat([torch.arange(0, 60), torch.arange(100, 120)]).to(DEV)
+    idx2 = torch.cat([torch.arange(60, 99), torch.arange(120, 136)]).to(DEV)
+    last = torch.tensor([99, 136], device=DEV)
+    for idx, ls in ((idx1, first), (idx2, rest)):
+        cu = torch.tensor(np.concatenate(([0], np.cumsum(ls))), dtype=torch.int32, device=DEV)
+        two.encode(K[idx].contiguous(), V[idx].contiguous(), cu)
+    two.append(K[last].contiguous(), V[last].contiguous())
+    torch.cuda.synchronize()
+    two.check_status()
+    assert two.lens.cpu().tolist() == lens_list
+    c1, r1 = one.unpack(100)
+    c2, r2 = two.unpack(100)
+    for b, n in enumerate(lens_list):
+        assert torch.equal(c1[b, :, :, :n], c2[b, :, :, :n]) and torch.equal(r1[b, :, :, :n], r2[b, :, :, :n])
+    q = synthetic.queries(12, B, Hq, d, torch.bfloat16, DEV)
+    assert torch.equal(one.attend(q), two.attend(q))
+
+
+def test_streaming_decode_steps_follow_the_oracle():
+    """Prefill, then append one token per sequence and attend, several steps; the partial last
+    token-block is exercised because the lengths are not multiples of the block."""
+    d, Hq, Hkv = 128, 8, 2
+    lens_list = [63, 129]
+    B = len(lens_list)
+    cache = pq.PolarQuantCache(B, Hq, Hkv, d, capacity=140, seed=5, device=DEV)
+    K, V = synthetic.kv_like(21, sum(lens_list), Hkv, d, torch.bfloat16, DEV)
+    _encode_and_compare(cache, K, V, lens_list)
+    ref = _oracle_cache(cache, K, V, lens_list)
+    for step in range(4):
+        k1, v1 = synthetic.kv_like(100 + step, B, Hkv, d, torch.bfloat16, DEV)
+        q = synthetic.queries(200 + step, B, Hq, d, torch.bfloat16, DEV)
+        cache.append(k1, v1)
+        out = cache.attend(q)
+        torch.cuda.synchronize()
+        cache.check_status()
+        ref.append(to_f64(k1), to_f64(v1))
+        assert rel_l2(to_f64(out), ref.attend(to_f64(q), d ** -0.5)) < TOL_ATTENTION
+    codes, _ = cache.unpack(133)
+    codes = codes.cpu().numpy()
+    for b, n in enumerate(lens_list):
+        assert np.array_equal(codes[b, :, 0, :n + 4], ref.k_codes[b, :, :n + 4])
+        assert np.array_equal(codes[b, :, 1, :n + 4], ref.v_codes[b, :, :n + 4])
+
+
+def test_attention_special_cases_len1_and_identical_keys():
+    d, Hq, Hkv = 128, 4, 1
+    cache = pq.PolarQuantCache(2, Hq, Hkv, d, capacity=64, seed=6, device=DEV)
+    K, V = synthetic.kv_like(31, 1 + 40, Hkv, d, torch.bfloat16, DEV)
+    K[1:] = K[1]  # sequence 1: forty identical keys
+    cu = torch.tensor([0, 1, 41], dtype=torch.int32, device=DEV)
+    cache.encode(K, V, cu)
+    q = synthetic.queries(32, 2, Hq, d, torch.bfloat16, DEV)
+    out = to_f64(cache.attend(q))
+    xh = to_f64(cache.dequant(40))
+    for h in range(Hq):
+        assert rel_l2(out[0, h], xh[0, 0, 1, 0]) < TOL_ATTENTION          # len 1: the value itself
+        assert rel_l2(out[1, h], xh[1, 0, 1, :40].mean(0)) < 2 * TOL_ATTENTION  # uniform weights: the mean
+
+
+def test_capacity_overflow_and_empty_sequence_are_reported_not_faulted():
+    d, Hq, Hkv = 128, 4, 1
+    cache = pq.PolarQuantCache(2, Hq, Hkv, d, capacity=64, seed=7, device=DEV)
+    K, V = synthetic.kv_like(41, 70 + 10, Hkv, d, torch.bfloat16, DEV)
+    cu = torch.tensor([0, 70, 80], dtype=torch.int32, device=DEV)
+    cache.encode(K, V, cu)  # sequence 0 does not fit: nothing of it is written, lens stays 0
+    torch.cuda.synchronize()
+    assert cache.status.cpu().tolist()[0] == pq.ERR_CAPACITY
+    assert cache.lens.cpu().tolist() == [0, 10]
+    cache.status.zero_()
+    q = synthetic.queries(42, 2, Hq, d, torch.bfloat16, DEV)
+    out = cache.attend(q)
+    torch.cuda.synchronize()
+    assert cache.status.cpu().tolist()[0] == pq.ERR_EMPTY
+    assert torch.all(out[0] == 0) and torch.isfinite(out).all()
+    # append to a full sequence is refused the same way
+    cache.lens.copy_(torch.tensor([64, 10], dtype=torch.int32))
+    cache.status.zero_()
+    cache.append(K[:2].contiguous(), V[:2].contiguous())
+    torch.cuda.synchronize()
+    assert cache.status.cpu().tolist()[0] == pq.ERR_CAPACITY and cache.lens.cpu().tolist() == [64, 11]
+
+
+def test_nonfinite_inputs_are_counted():
+    d = 128
+    cache = pq.PolarQuantCache(1, 1, 1, d, capacity=64, seed=8, device=DEV)
+    K, V = synthetic.kv_like(51, 8, 1, d, torch.bfloat16, DEV)
+    K[3, 0, 5] = float("nan")
+    V[4, 0, 6] = float("inf")
+    cache.encode(K, V, torch.tensor([0, 8], dtype=torch.int32, device=DEV))
+    torch.cuda.synchronize()
+    st = cache.status.cpu().tolist()
+    assert st[0] == pq.ERR_NONFINITE and st[1] == 2
+
+
+def test_mid_size_llama_shape_codes_with_window_accounting():
+    """8 kv heads x 2048 tokens x d = 128 (the encode config's shape, shortened): ~3.9 M codes."""
+    d, Hkv, n = 128, 8, 2048
+    cache = pq.PolarQuantCache(1, 32, Hkv, d, capacity=n, seed=1, device=DEV)
+    K, V = synthetic.kv_like(1, n, Hkv, d, torch.bfloat16, DEV)
+    rep = _encode_and_compare(cache, K, V, [n])
+    assert rep["total"] == 2 * Hkv * n * 120
+    ref = _oracle_cache(cache, K, V, [n])
+    q = synthetic.queries(2, 1, 32, d, torch.bfloat16, DEV)
+    out = cache.attend(q)
+    torch.cuda.synchronize()
+    assert rel_l2(to_f64(out), ref.attend(to_f64(q), d ** -0.5)) < TOL_ATTENTION
