@@ -59,6 +59,9 @@ extern "C" {
 /* Human-readable name of a status code (static string, never NULL). */
 const char* pq_status_string(int32_t status);
 
+/* Text of the CUDA runtime error behind the calling thread's most recent PQ_ERR_CUDA ("" if none). */
+const char* pq_last_cuda_error(void);
+
 /* Tokens per cache token-block (a compile-time constant of the layout). */
 int32_t pq_token_block(void);
 

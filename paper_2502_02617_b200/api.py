@@ -27,6 +27,7 @@ DEFAULT_BITS = (4, 2, 2, 2)
 # name -> (restype, argtypes); must list every symbol of include/polarquant.h
 _SIGNATURES = {
     "pq_status_string": (c_char_p, [c_int32]),
+    "pq_last_cuda_error": (c_char_p, []),
     "pq_token_block": (c_int32, []),
     "pq_make_rotation": (c_int32, [c_int32, c_uint64, c_void_p]),
     "pq_fit_codebooks": (c_int32, [POINTER(c_int32), POINTER(c_double), POINTER(c_double)]),
@@ -52,7 +53,8 @@ _lib = None
 class PolarQuantError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
-        super().__init__(f"{where}: {status_string(status)} ({status})")
+        detail = lib().pq_last_cuda_error().decode() if status == ERR_CUDA else ""
+        super().__init__(f"{where}: {status_string(status)} ({status})" + (f": {detail}" if detail else ""))
 
 
 def lib() -> ctypes.CDLL:

@@ -34,14 +34,15 @@ struct Tables {
   float cen_cos[PQ_N_CENTROIDS];
   float cen_sin[PQ_N_CENTROIDS];
   // fp16 decode tables of the attention kernel.
-  //   l1[c]   = (cos, sin) of level-1 centroid c as half2
-  //   l2[c]   = (cos, sin) of level-2 centroid c as half2
-  //   u43[p][c4*4+c3] = t4(c4, side p>>1) * t3(c3, side p&1), p = position of the 4-coordinate
-  //             sub-block inside its 16-block (side 0 = cos, 1 = sin)
-  uint32_t l1_h2[16];
-  uint32_t l2_h2[4];
-  uint16_t u43_h[4][16];
-  uint32_t reserved[32];
+  //   l1_hi[c], l1_lo[c] : (cos, sin) of level-1 centroid c as half2, split into the fp16 value and
+  //                        the fp16 rounding residual (hi + lo carries ~22 bits)
+  //   u_tab[s][i]        : sub-block s (0..3) of a block, i = c2 | c3 << 2 | c4 << 4: the product of
+  //                        the level-4, level-3 and level-2 factors of the sub-block's two level-1
+  //                        pairs, .x = half2 of the fp16 values, .y = half2 of the residuals
+  uint32_t l1_hi[16];
+  uint32_t l1_lo[16];
+  uint2 u_tab[4][64];
+  uint32_t reserved[30];
 };
 
 constexpr uint32_t kFlagUniformL1 = 1u;
@@ -146,6 +147,15 @@ __device__ inline double polar_quant_block_exact(const double* y, const Tables& 
   }
   c.l4 = quant_upper_exact(r3[0], r3[1], 4, tb);
   return hypot(r3[0], r3[1]);
+}
+
+// Host side: remember the CUDA error behind a PQ_ERR_CUDA return (see pq_last_cuda_error).
+void note_cuda_error(cudaError_t e);
+inline int32_t launch_status() {
+  const cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) return PQ_OK;
+  note_cuda_error(e);
+  return PQ_ERR_CUDA;
 }
 
 // Record the first error seen.

@@ -71,6 +71,8 @@ __device__ inline float decode_coord(const uint8_t* tb, const Layout& L, int tok
 // ---- workspace -----------------------------------------------------------------------------
 struct Workspace {
   float* qrot;       // [B][Hq][d]      rotated queries times scale*log2(e)
+  __half* qrot_h;    // the same rounded to fp16 (tensor-core operand of the fast kernel)
+  __half* qrot_l;    // fp16 residual: qrot - qrot_h
   int32_t* tickets;  // [B][Hkv]
   float* ml;         // [B][Hq][splits][2]
   float* o;          // [B][Hq][splits][d]
@@ -78,8 +80,27 @@ struct Workspace {
   int64_t bytes;
 };
 
-__host__ inline int choose_splits(int batch, int n_kv_heads, int max_len) {
+// Token splits per (sequence, kv head).  The head_dim-128 kernel runs one CTA per SM and works
+// in 128-token stages: pick the split count with the smallest estimated makespan
+// (waves x (stages per CTA + fixed cost)).
+__host__ inline int choose_splits(int d, int batch, int n_kv_heads, int max_len) {
   const int units = batch * n_kv_heads;
+  if (d == 128) {
+    const int nst = (max_len + 127) / 128;
+    int best = 1;
+    double best_cost = 1e30;
+    for (int s = 1; s <= 128 && s <= nst; ++s) {
+      const int per = (nst + s - 1) / s;
+      const long ctas = (long)units * s;
+      const long waves = (ctas + 147) / 148;
+      const double cost = (double)waves * (per + 1.5);
+      if (cost < best_cost - 1e-9) {
+        best_cost = cost;
+        best = s;
+      }
+    }
+    return best;
+  }
   const int max_blocks = (max_len + kTokenBlock - 1) / kTokenBlock;
   int splits = (148 * 4 + units - 1) / units;
   if (splits > max_blocks) splits = max_blocks;
@@ -90,12 +111,16 @@ __host__ inline int choose_splits(int batch, int n_kv_heads, int max_len) {
 
 __host__ inline Workspace carve_workspace(void* base, int d, int batch, int n_q_heads, int n_kv_heads, int max_len) {
   Workspace w;
-  w.n_splits = choose_splits(batch, n_kv_heads, max_len);
+  w.n_splits = choose_splits(d, batch, n_kv_heads, max_len);
   auto align = [](int64_t x) { return (x + 255) & ~(int64_t)255; };
   int64_t off = 0;
   uint8_t* p = reinterpret_cast<uint8_t*>(base);
   w.qrot = reinterpret_cast<float*>(p + off);
   off = align(off + (int64_t)batch * n_q_heads * d * 4);
+  w.qrot_h = reinterpret_cast<__half*>(p + off);
+  off = align(off + (int64_t)batch * n_q_heads * d * 2);
+  w.qrot_l = reinterpret_cast<__half*>(p + off);
+  off = align(off + (int64_t)batch * n_q_heads * d * 2);
   w.tickets = reinterpret_cast<int32_t*>(p + off);
   off = align(off + (int64_t)batch * n_kv_heads * 4);
   w.ml = reinterpret_cast<float*>(p + off);
@@ -129,7 +154,11 @@ __global__ void rotate_query_kernel(DecodeArgs a) {
   __syncthreads();
   float acc = 0.f;
   for (int k = 0; k < d; ++k) acc = fmaf(qs[k], a.S[k * d + j], acc);
-  a.ws.qrot[base + j] = acc * a.scale * 1.4426950408889634f;
+  acc *= a.scale * 1.4426950408889634f;
+  a.ws.qrot[base + j] = acc;
+  const __half qh = __float2half_rn(acc);
+  a.ws.qrot_h[base + j] = qh;
+  a.ws.qrot_l[base + j] = __float2half_rn(acc - __half2float(qh));
   if (bh < a.batch * a.n_kv_heads && j == 0) a.ws.tickets[bh] = 0;
 }
 
@@ -177,7 +206,7 @@ __device__ void combine_and_store(const DecodeArgs& a, int b, int hk, int g, flo
 // coordinate decodes the values and accumulates.  Serves every head_dim and group size.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel(DecodeArgs a) {
-  extern __shared__ __align__(16) uint8_t smem[];
+  extern __shared__ __align__(128) uint8_t smem[];
   const int d = a.d, g = a.n_q_heads / a.n_kv_heads;
   const Layout L = make_layout(d, a.capacity);
   const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
@@ -314,6 +343,10 @@ __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel
   }
 }
 
+}  // namespace pq
+#include "pq_decode_fast.cuh"
+namespace pq {
+
 // ---- inspection kernels ----------------------------------------------------------------------
 __global__ void unpack_codes_kernel(int d, int n_kv_heads, const uint8_t* cache, int batch, int capacity,
                                     int n_tokens, uint8_t* codes, __half* radii) {
@@ -357,7 +390,22 @@ __global__ void dequant_kernel(int d, int n_kv_heads, const float* S, const Tabl
   const int h = (int)((v / (2 * (int64_t)n_tokens)) % n_kv_heads);
   const int b = (int)(v / (2 * (int64_t)n_tokens * n_kv_heads));
   const uint8_t* tb = cache + block_offset(L, n_kv_heads, b, h, kv, tok);
-  ysm[j] = decode_coord(tb, L, tok % kTokenBlock, j, cc, cs);
+  if (d == 128) {
+    // the fp16 arithmetic of the attention kernel's value path: u = rn(r * U), x = rn(u * t1)
+    const int t = tok % kTokenBlock, blk = j >> 4, i = j & 15;
+    const uint32_t c1 = (get_l1(tb, L, t, blk) >> (4 * (i >> 1))) & 15u;
+    const uint32_t c2 = (get_l2(tb, L, t, blk) >> (2 * (i >> 2))) & 3u;
+    const uint32_t c3 = (get_l3(tb, L, t, blk) >> (2 * (i >> 3))) & 3u;
+    const uint32_t c4 = get_l4(tb, L, t, blk);
+    const uint32_t up = tables->u_tab[i >> 2][c2 | (c3 << 2) | (c4 << 4)].x;
+    const __half2 uh = *reinterpret_cast<const __half2*>(&up);
+    const __half r = reinterpret_cast<const __half*>(tb + L.orad + t * L.br)[blk];
+    const __half u = __hmul(r, (i & 2) ? __high2half(uh) : __low2half(uh));
+    const __half2 t1 = *reinterpret_cast<const __half2*>(&tables->l1_hi[c1]);
+    ysm[j] = __half2float(__hmul(u, (i & 1) ? __high2half(t1) : __low2half(t1)));
+  } else {
+    ysm[j] = decode_coord(tb, L, tok % kTokenBlock, j, cc, cs);
+  }
   __syncthreads();
   float acc = 0.f;
   for (int k = 0; k < d; ++k) acc = fmaf(ysm[k], S[(int64_t)j * d + k], acc);
@@ -398,12 +446,27 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
   a.ws = pq::carve_workspace(workspace_dev, head_dim, batch, n_q_heads, n_kv_heads, max_len);
   const int g = n_q_heads / n_kv_heads;
   pq::rotate_query_kernel<<<batch * n_q_heads, head_dim, head_dim * sizeof(float), st>>>(a);
+  if (head_dim == 128) {
+    static bool configured = false;
+    if (!configured) {
+      const cudaError_t e = cudaFuncSetAttribute(pq::decode_attention_fast_kernel,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, pq::kSmTotal);
+      if (e != cudaSuccess) {
+        pq::note_cuda_error(e);
+        return PQ_ERR_CUDA;
+      }
+      configured = true;
+    }
+    dim3 grid(a.ws.n_splits, n_kv_heads, batch);
+    pq::decode_attention_fast_kernel<<<grid, pq::kFastThreads, pq::kSmTotal, st>>>(a);
+    return pq::launch_status();
+  }
   const pq::Layout L = pq::make_layout(head_dim, capacity);
   const size_t smem = 2 * L.block_bytes + sizeof(float) * ((size_t)g * head_dim + 3 * g * pq::kTokenBlock +
                                                            3 * pq::kMaxGroup + 64);
   dim3 grid(a.ws.n_splits, n_kv_heads, batch);
   pq::decode_attention_simple_kernel<<<grid, pq::kSimpleThreads, smem, st>>>(a);
-  return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+  return pq::launch_status();
 }
 
 int32_t pq_unpack_codes(int32_t head_dim, int32_t n_kv_heads, const void* cache_dev, int32_t batch, int32_t capacity,
@@ -415,7 +478,7 @@ int32_t pq_unpack_codes(int32_t head_dim, int32_t n_kv_heads, const void* cache_
   pq::unpack_codes_kernel<<<(unsigned)((n + 127) / 128), 128, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
       head_dim, n_kv_heads, reinterpret_cast<const uint8_t*>(cache_dev), batch, capacity, n_tokens, codes_dev,
       reinterpret_cast<__half*>(radii_dev));
-  return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+  return pq::launch_status();
 }
 
 int32_t pq_dequant_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
@@ -430,7 +493,7 @@ int32_t pq_dequant_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, 
   pq::dequant_kernel<<<(unsigned)n, head_dim, head_dim * sizeof(float), reinterpret_cast<cudaStream_t>(stream)>>>(
       head_dim, n_kv_heads, S_dev, reinterpret_cast<const pq::Tables*>(tables_dev),
       reinterpret_cast<const uint8_t*>(cache_dev), capacity, n_tokens, x_hat_dev);
-  return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+  return pq::launch_status();
 }
 
 }  // extern "C"

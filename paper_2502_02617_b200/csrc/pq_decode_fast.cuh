@@ -1,0 +1,436 @@
+// Fast decode-attention kernel for head_dim 128 (included by pq_decode.cu).
+//
+// One CTA of 16 warps per (token split, kv head, sequence).  128-token stages of the packed cache
+// (K block, V block, K block, V block: one contiguous 15872-byte bulk copy) stream through a
+// shared-memory ring; one elected thread issues the copies three stages ahead, and each warp
+// takes one 8-token tile of every stage.  (16 warps, not 17: the register file is split over four
+// schedulers, and a fifth warp on one of them would cap every thread at 96 registers.)
+//
+// Per tile a warp
+//   * decodes the keys straight into mma.sync B fragments (fp16, rotated basis) with
+//     shared-memory table lookups, and forms S^T = q' K_hat^T (heads x tokens) on tensor cores,
+//   * runs the online softmax on the S^T fragment (log2 domain, fp32),
+//   * decodes the values into A fragments (coordinates x tokens) and accumulates
+//     O^T += V_hat^T P on tensor cores (fp32 accumulators in registers).
+// DeQuant (Algorithm 1) of one 16-coordinate block is a product tree r * t4 * t3 * t2 * t1.
+// Levels 4..2 are folded into one table per 4-coordinate sub-block, level 1 is a half2 multiply:
+//   u    [4][64][16] sub-block s, index c2_s | c3_(s>>1) << 2 | c4 << 4 -> the multipliers of the
+//                    sub-block's two level-1 pairs as (half2 values, half2 rounding residuals)
+//   t1hi [256][16]   index = one byte of level-1 codes (pair 2s | pair 2s+1 << 4) -> (cos, sin) x 2 in fp16
+//   t1lo [256][16]   the fp16 rounding residuals of the same entries
+// All are replicated 16 times so that every lane of a half-warp reads its own banks.
+// Values use the fp16 parts only.  Keys feed the softmax exponent, where an fp16-rounded operand
+// costs ~3x its relative error in the output, so they are decoded as an unevaluated sum hi + lo
+// (error-free fp16 transformations with fused multiply-adds) and contracted with two MMAs.
+#pragma once
+
+namespace pq {
+
+constexpr int kFastConsumerWarps = 16;
+constexpr int kFastThreads = kFastConsumerWarps * 32;
+constexpr int kStageTokens = 2 * kTokenBlock;       // 128
+constexpr int kBlockBytes128 = 62 * kTokenBlock;    // 3968: one K or V token-block at d = 128
+constexpr int kStageBytes = 4 * kBlockBytes128;     // 15872
+constexpr int kStages = 4;
+constexpr int kSpinLimit = 1 << 22;
+
+// shared-memory map (bytes)
+constexpr int kSmT1p = 0;                             // 256 * 16 * 8 = 32768
+constexpr int kSmT1lo = kSmT1p + 256 * 16 * 8;        // 32768
+constexpr int kSmU = kSmT1lo + 256 * 16 * 8;          // 4 * 64 * 16 * 8 = 32768
+constexpr int kSmBar = kSmU + 4 * 64 * 16 * 8;        // full[4], empty[4] : 64
+constexpr int kSmFlags = kSmBar + 64;                 // abort flag, is_last : 16
+constexpr int kSmRing = (kSmFlags + 16 + 127) / 128 * 128;
+// after the main loop the ring is reused for the cross-warp merge: 16 warps x 8 heads x (128 + 2) floats
+constexpr int kMergeBytes = 16 * 8 * 128 * 4 + 16 * 8 * 2 * 4;
+constexpr int kSmTotal = kSmRing + (kStages * kStageBytes > kMergeBytes ? kStages * kStageBytes : kMergeBytes);
+static_assert(kSmRing % 128 == 0, "ring must be 128-byte aligned");
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up after kSpinLimit polls (or as soon as another warp gave up) and raises
+// the CTA's abort flag, so that a lost copy can never hang the GPU.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  for (int i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (i > 64) {
+      __nanosleep(64);
+      if (*abort_flag) return false;
+    }
+  }
+  *abort_flag = 1;
+  return false;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds16(uint32_t addr) {
+  uint16_t v;
+  asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ uint32_t lds8(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
+  return v;
+}
+
+__device__ __forceinline__ __half2 as_h2(uint32_t v) { return *reinterpret_cast<__half2*>(&v); }
+__device__ __forceinline__ uint32_t as_u32(__half2 v) { return *reinterpret_cast<uint32_t*>(&v); }
+
+// D(16x8, f32) += A(16x16, f16, row) * B(16x8, f16, col)
+__device__ __forceinline__ void mma_16816(float* d, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// D(16x8, f32) += A(16x8, f16, row) * B(8x8, f16, col)
+__device__ __forceinline__ void mma_1688(float* d, uint32_t a0, uint32_t a1, uint32_t b0) {
+  asm volatile("mma.sync.aligned.m16n8k8.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+               : "r"(a0), "r"(a1), "r"(b0));
+}
+
+// Byte offsets of the four sub-block entries of a block in the replicated u table
+// (entry idx at idx * 128: c2_s -> bits 7..8, c3 -> bits 9..10, c4 -> bits 11..12).
+__device__ __forceinline__ void u_offsets(uint32_t c2, uint32_t c3n, uint32_t c4, uint32_t* off) {
+  const uint32_t a4 = c4 << 11;
+  const uint32_t hi0 = ((c3n << 9) & 0x600u) | a4, hi1 = ((c3n << 7) & 0x600u) | a4;
+  off[0] = 0 * 8192 + (((c2 << 7) & 0x180u) | hi0);
+  off[1] = 1 * 8192 + (((c2 << 5) & 0x180u) | hi0);
+  off[2] = 2 * 8192 + (((c2 << 3) & 0x180u) | hi1);
+  off[3] = 3 * 8192 + (((c2 << 1) & 0x180u) | hi1);
+}
+
+// DeQuant of one 16-coordinate block in the rotated basis as 8 half2 (coordinates 2i, 2i+1), fp16 path.
+//   l1 : 8 level-1 codes, code j at bits [4j, 4j+4)     c2 : 4 level-2 codes, 2 bits each (clean)
+//   c3n: 2 level-3 codes in a nibble (clean)             c4 : the level-4 code (clean)
+//   r2 : the block radius in both halves                 rep: (lane & 15) * 8
+__device__ __forceinline__ void decode_block_h2(uint32_t l1, uint32_t c2, uint32_t c3n, uint32_t c4, __half2 r2,
+                                                uint32_t sm_base, uint32_t rep, __half2* out) {
+  uint32_t off[4];
+  u_offsets(c2, c3n, c4, off);
+  const uint32_t ub = sm_base + kSmU + rep, t1 = sm_base + kSmT1p + rep;
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    const __half2 u = __hmul2(r2, as_h2(lds32(ub + off[s])));
+    const uint2 e = lds64(t1 + ((s == 0 ? (l1 << 7) : (l1 >> (8 * s - 7))) & 0x7F80u));
+    out[2 * s] = __hmul2(__low2half2(u), as_h2(e.x));
+    out[2 * s + 1] = __hmul2(__high2half2(u), as_h2(e.y));
+  }
+}
+
+// The same block as an unevaluated sum hi + lo of fp16 values (about 21 significant bits):
+//   u = r * (Uhi + Ulo)            u_hi = rn(r Uhi),  u_lo = fma(r, Uhi, -u_hi) + r Ulo
+//   k = (u_hi + u_lo)(thi + tlo)   k_hi = rn(u_hi thi), k_lo = fma(u_hi, thi, -k_hi) + u_lo thi + u_hi tlo
+// (fp16 fused multiply-adds return the exact rounding residual of a product).
+__device__ __forceinline__ void decode_block_hilo(uint32_t l1, uint32_t c2, uint32_t c3n, uint32_t c4, __half2 r2,
+                                                  uint32_t sm_base, uint32_t rep, __half2* hi, __half2* lo) {
+  uint32_t off[4];
+  u_offsets(c2, c3n, c4, off);
+  const uint32_t ub = sm_base + kSmU + rep, t1 = sm_base + kSmT1p + rep;
+#pragma unroll
+  for (int s = 0; s < 4; ++s) {
+    const uint2 uu = lds64(ub + off[s]);
+    const __half2 u_hi = __hmul2(r2, as_h2(uu.x));
+    const __half2 u_lo = __hfma2(r2, as_h2(uu.y), __hfma2(r2, as_h2(uu.x), __hneg2(u_hi)));
+    const uint32_t idx = (s == 0 ? (l1 << 7) : (l1 >> (8 * s - 7))) & 0x7F80u;
+    const uint2 th = lds64(t1 + idx), tl = lds64(t1 + (kSmT1lo - kSmT1p) + idx);
+    const __half2 ua = __low2half2(u_hi), ub2 = __high2half2(u_hi);
+    const __half2 la = __low2half2(u_lo), lb = __high2half2(u_lo);
+    const __half2 ka = __hmul2(ua, as_h2(th.x)), kb = __hmul2(ub2, as_h2(th.y));
+    hi[2 * s] = ka;
+    hi[2 * s + 1] = kb;
+    lo[2 * s] = __hfma2(ua, as_h2(tl.x), __hfma2(la, as_h2(th.x), __hfma2(ua, as_h2(th.x), __hneg2(ka))));
+    lo[2 * s + 1] = __hfma2(ub2, as_h2(tl.y), __hfma2(lb, as_h2(th.y), __hfma2(ub2, as_h2(th.y), __hneg2(kb))));
+  }
+}
+
+// plane offsets of a d = 128 token-block
+constexpr int kO2 = 32 * kTokenBlock, kO3 = kO2 + 8 * kTokenBlock, kO4 = kO3 + 4 * kTokenBlock,
+              kORad = kO4 + 2 * kTokenBlock;
+
+// Build the replicated shared-memory tables from `Tables`.
+__device__ inline void build_fast_tables(uint8_t* smem, const Tables* tb) {
+  const int tid = threadIdx.x;
+  uint2* t1hi = reinterpret_cast<uint2*>(smem + kSmT1p);
+  uint2* t1lo = reinterpret_cast<uint2*>(smem + kSmT1lo);
+  for (int i = tid; i < 256 * 16; i += blockDim.x) {
+    const int e = i >> 4;  // entry; replica = i & 15
+    t1hi[i] = make_uint2(tb->l1_hi[e & 15], tb->l1_hi[e >> 4]);
+    t1lo[i] = make_uint2(tb->l1_lo[e & 15], tb->l1_lo[e >> 4]);
+  }
+  uint2* u = reinterpret_cast<uint2*>(smem + kSmU);
+  for (int i = tid; i < 4 * 64 * 16; i += blockDim.x) u[i] = tb->u_tab[i >> 10][(i >> 4) & 63];
+}
+
+__global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(DecodeArgs a) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  const int g_heads = a.n_q_heads / a.n_kv_heads;
+  const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const uint32_t sm_base = smem_u32(smem);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kSmFlags);
+  int* is_last = reinterpret_cast<int*>(smem + kSmFlags) + 1;
+
+  const int len = a.lens[b];
+  const int nst_total = len > 0 ? (len + kStageTokens - 1) / kStageTokens : 0;
+  const int nblk_total = len > 0 ? (len + kTokenBlock - 1) / kTokenBlock : 0;
+  const int per = (nst_total + a.ws.n_splits - 1) / a.ws.n_splits;
+  const int st0 = split * per;
+  const int st1 = min(nst_total, st0 + per);
+  const uint8_t* head_base = a.cache + ((int64_t)b * a.n_kv_heads + hk) * make_layout(128, a.capacity).head_bytes;
+
+  build_fast_tables(smem, a.tables);
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(sm_base + kSmBar + 8 * s, 1);                                  // full: producer + tx bytes
+      mbar_init(sm_base + kSmBar + 8 * (kStages + s), kFastConsumerWarps);     // empty: one arrive per warp
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  // per-thread attention state (consumer warps)
+  const int g = lane >> 2, c = lane & 3;
+  float o_acc[8][4];  // tile i (pair i of block g): rows 2i / 2i+1 of block g, heads 2c / 2c+1
+#pragma unroll
+  for (int i = 0; i < 8; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
+  float m_run = -CUDART_INF_F, l_run = 0.f;  // of head g (replicated over the 4 lanes of a quad)
+
+  // Copy of iteration `it` (stage st0 + it) into ring slot it % kStages; waits (bounded) until all
+  // 16 warps have released the slot's previous contents.  Called by thread 0 only.
+  int issued = 0;
+  auto issue_copy = [&](int it) -> bool {
+    const int s = it % kStages;
+    if (it >= kStages && !mbar_wait(sm_base + kSmBar + 8 * (kStages + s), ((it / kStages) - 1) & 1, abort_flag))
+      return false;
+    const int st = st0 + it;
+    const int nblk = min(2, nblk_total - 2 * st);
+    const uint32_t bytes = nblk * 2 * kBlockBytes128;
+    mbar_expect_tx(sm_base + kSmBar + 8 * s, bytes);
+    bulk_load(sm_base + kSmRing + s * kStageBytes, head_base + (int64_t)st * kStageBytes, bytes, sm_base + kSmBar + 8 * s);
+    issued = it + 1;
+    return true;
+  };
+  if (tid == 0)
+    for (int it = 0; it < kStages - 1 && st0 + it < st1; ++it) issue_copy(it);
+  __syncwarp();
+  {
+    // ---------------------------------------------------------------- consumers
+    // q' fragments: A operand (16 heads x 16 coords per k-step); rows >= 8 are zero.
+    // k-step ks covers, for thread c, sub-block (ks & 3) of block 2c + (ks >> 2).
+    uint32_t qa[8][2], ql[8][2];  // fp16 value and fp16 residual of q'
+    {
+      const int64_t qoff = ((int64_t)b * a.n_q_heads + hk * g_heads + g) * 128 + 32 * c;
+#pragma unroll
+      for (int ks = 0; ks < 8; ++ks) {
+        uint2 v = make_uint2(0u, 0u), w = make_uint2(0u, 0u);
+        if (g < g_heads) {
+          v = *reinterpret_cast<const uint2*>(a.ws.qrot_h + qoff + 4 * ks);
+          w = *reinterpret_cast<const uint2*>(a.ws.qrot_l + qoff + 4 * ks);
+        }
+        qa[ks][0] = v.x;
+        qa[ks][1] = v.y;
+        ql[ks][0] = w.x;
+        ql[ks][1] = w.y;
+      }
+    }
+    const uint32_t rep = (lane & 15) * 8;
+    // logical token n of a tile (MMA column n) is physical token (n >> 1) + 4 * (n & 1)
+    const int ktok = (g >> 1) + 4 * (g & 1);  // token whose keys this thread decodes
+    for (int st = st0, it = 0; st < st1; ++st, ++it) {
+      const int s = it % kStages;
+      if (tid == 0 && st + kStages - 1 < st1) issue_copy(it + kStages - 1);
+      __syncwarp();
+      if (!mbar_wait(sm_base + kSmBar + 8 * s, (it / kStages) & 1, abort_flag)) break;
+      const int tile_tok0 = st * kStageTokens + warp * 8;  // first token of this warp's tile
+      if (tile_tok0 < len) {
+        const uint32_t kblk = sm_base + kSmRing + s * kStageBytes + (warp >> 3) * 2 * kBlockBytes128;
+        const uint32_t vblk = kblk + kBlockBytes128;
+        const int t0 = (warp & 7) * 8;  // tile's first token inside its token-block
+        // ---- scores: S^T (heads x tokens)
+        float sc[4] = {0.f, 0.f, 0.f, 0.f};
+        {
+          const int tk = t0 + ktok;
+          const uint2 l1 = lds64(kblk + tk * 32 + c * 8);
+          const uint32_t rr = lds32(kblk + kORad + tk * 16 + c * 4);
+          const uint32_t c2 = lds16(kblk + kO2 + tk * 8 + c * 2);
+          const uint32_t c3 = lds8(kblk + kO3 + tk * 4 + c);
+          const uint32_t c4 = lds16(kblk + kO4 + tk * 2) >> (4 * c);
+          __half2 kh[8], kl[8];
+          decode_block_hilo(l1.x, c2 & 0xFFu, c3 & 0xFu, c4 & 3u, __low2half2(as_h2(rr)), sm_base, rep, kh, kl);
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            mma_16816(sc, qa[ks][0], 0u, qa[ks][1], 0u, as_u32(kl[2 * ks]), as_u32(kl[2 * ks + 1]));
+            mma_16816(sc, ql[ks][0], 0u, ql[ks][1], 0u, as_u32(kh[2 * ks]), as_u32(kh[2 * ks + 1]));
+            mma_16816(sc, qa[ks][0], 0u, qa[ks][1], 0u, as_u32(kh[2 * ks]), as_u32(kh[2 * ks + 1]));
+          }
+          decode_block_hilo(l1.y, c2 >> 8, c3 >> 4, (c4 >> 2) & 3u, __high2half2(as_h2(rr)), sm_base, rep, kh, kl);
+#pragma unroll
+          for (int ks = 0; ks < 4; ++ks) {
+            mma_16816(sc, qa[4 + ks][0], 0u, qa[4 + ks][1], 0u, as_u32(kl[2 * ks]), as_u32(kl[2 * ks + 1]));
+            mma_16816(sc, ql[4 + ks][0], 0u, ql[4 + ks][1], 0u, as_u32(kh[2 * ks]), as_u32(kh[2 * ks + 1]));
+            mma_16816(sc, qa[4 + ks][0], 0u, qa[4 + ks][1], 0u, as_u32(kh[2 * ks]), as_u32(kh[2 * ks + 1]));
+          }
+        }
+        // ---- online softmax for head g; this thread holds logical tokens 2c, 2c+1 = physical c, c+4
+        const bool ok0 = tile_tok0 + c < len, ok1 = tile_tok0 + c + 4 < len;
+        const float s0 = ok0 ? sc[0] : -CUDART_INF_F, s1 = ok1 ? sc[1] : -CUDART_INF_F;
+        float mx = fmaxf(s0, s1);
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+        const float m_new = fmaxf(m_run, mx);
+        const float p0 = exp2f(s0 - m_new), p1 = exp2f(s1 - m_new);
+        float psum = p0 + p1;
+        psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+        psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+        const float corr = exp2f(m_run - m_new);  // 0 on the first tile (m_run = -inf)
+        l_run = l_run * corr + psum;
+        if (__any_sync(0xffffffffu, m_new > m_run)) {
+          const float c0 = __shfl_sync(0xffffffffu, corr, (2 * c) << 2);
+          const float c1 = __shfl_sync(0xffffffffu, corr, (2 * c + 1) << 2);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            o_acc[i][0] *= c0;
+            o_acc[i][1] *= c1;
+            o_acc[i][2] *= c0;
+            o_acc[i][3] *= c1;
+          }
+        }
+        m_run = m_new;
+        const uint32_t pb = as_u32(__floats2half2_rn(p0, p1));  // B operand: tokens (2c, 2c+1) x head g
+        // ---- values: block g of physical tokens c and c + 4
+        {
+          __half2 va[8], vb[8];
+          {
+            const int tk = t0 + c;
+            const uint32_t l1 = lds32(vblk + tk * 32 + g * 4);
+            uint32_t rr = lds16(vblk + kORad + tk * 16 + g * 2);
+            const uint32_t c2 = lds8(vblk + kO2 + tk * 8 + g);
+            const uint32_t c3 = lds8(vblk + kO3 + tk * 4 + (g >> 1)) >> (4 * (g & 1));
+            const uint32_t c4 = lds16(vblk + kO4 + tk * 2) >> (2 * g);
+            if (!ok0) rr = 0u;  // stale bytes past the sequence end must not reach the accumulators
+            decode_block_h2(l1, c2, c3 & 0xFu, c4 & 3u, as_h2(rr | (rr << 16)), sm_base, rep, va);
+          }
+          {
+            const int tk = t0 + c + 4;
+            const uint32_t l1 = lds32(vblk + tk * 32 + g * 4);
+            uint32_t rr = lds16(vblk + kORad + tk * 16 + g * 2);
+            const uint32_t c2 = lds8(vblk + kO2 + tk * 8 + g);
+            const uint32_t c3 = lds8(vblk + kO3 + tk * 4 + (g >> 1)) >> (4 * (g & 1));
+            const uint32_t c4 = lds16(vblk + kO4 + tk * 2) >> (2 * g);
+            if (!ok1) rr = 0u;
+            decode_block_h2(l1, c2, c3 & 0xFu, c4 & 3u, as_h2(rr | (rr << 16)), sm_base, rep, vb);
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const uint32_t x = __byte_perm(as_u32(va[i]), as_u32(vb[i]), 0x5410);  // coord 2i   of tokens (A, B)
+            const uint32_t y = __byte_perm(as_u32(va[i]), as_u32(vb[i]), 0x7632);  // coord 2i+1 of tokens (A, B)
+            mma_1688(o_acc[i], x, y, pb);
+          }
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(sm_base + kSmBar + 8 * (kStages + s));
+    }
+  }
+  if (tid == 0 && *abort_flag) {
+    // gave up: let the copies still in flight land (bounded) before the ring is reused
+    for (int it = max(0, issued - kStages); it < issued; ++it)
+      for (int i = 0; i < kSpinLimit && !mbar_try_wait(sm_base + kSmBar + 8 * (it % kStages), (it / kStages) & 1); ++i)
+        __nanosleep(64);
+  }
+  __syncthreads();  // every copy that was issued has been consumed (or the CTA aborted)
+
+  // ---- merge the 16 warps (fixed order), write this split's partial, last CTA combines
+  float* mrg_o = reinterpret_cast<float*>(smem + kSmRing);      // [16 warps][8 heads][128]
+  float* mrg_ml = mrg_o + kFastConsumerWarps * 8 * 128;         // [16 warps][8 heads][2]
+  {
+    if (c == 0) {
+      mrg_ml[(warp * 8 + g) * 2] = m_run;
+      mrg_ml[(warp * 8 + g) * 2 + 1] = l_run;
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      float* o0 = mrg_o + (warp * 8 + 2 * c) * 128 + 16 * g + 2 * i;
+      float* o1 = o0 + 128;
+      o0[0] = o_acc[i][0];
+      o1[0] = o_acc[i][1];
+      o0[1] = o_acc[i][2];
+      o1[1] = o_acc[i][3];
+    }
+  }
+  __syncthreads();
+  for (int idx = tid; idx < g_heads * 128; idx += kFastThreads) {
+    const int h = idx >> 7, j = idx & 127;
+    float M = -CUDART_INF_F;
+#pragma unroll
+    for (int w = 0; w < kFastConsumerWarps; ++w) M = fmaxf(M, mrg_ml[(w * 8 + h) * 2]);
+    float lsum = 0.f, acc = 0.f;
+#pragma unroll
+    for (int w = 0; w < kFastConsumerWarps; ++w) {
+      const float mw = mrg_ml[(w * 8 + h) * 2];
+      const float wgt = mw == -CUDART_INF_F ? 0.f : exp2f(mw - M);
+      lsum += mrg_ml[(w * 8 + h) * 2 + 1] * wgt;
+      acc += mrg_o[(w * 8 + h) * 128 + j] * wgt;
+    }
+    const int64_t pidx = ((int64_t)b * a.n_q_heads + hk * g_heads + h) * a.ws.n_splits + split;
+    a.ws.o[pidx * 128 + j] = acc;
+    if (j == 0) {
+      a.ws.ml[2 * pidx] = M;
+      a.ws.ml[2 * pidx + 1] = lsum;
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) {
+    if (*abort_flag) set_status(a.status, PQ_ERR_TIMEOUT);
+    const int t = atomicAdd(a.ws.tickets + b * a.n_kv_heads + hk, 1);
+    *is_last = (t == a.ws.n_splits - 1);
+    if (*is_last && len <= 0) set_status(a.status, PQ_ERR_EMPTY);
+  }
+  __syncthreads();
+  if (*is_last) {
+    __threadfence();
+    combine_and_store(a, b, hk, g_heads, reinterpret_cast<float*>(smem + kSmRing));
+  }
+}
+
+}  // namespace pq

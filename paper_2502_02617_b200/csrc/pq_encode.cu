@@ -196,7 +196,7 @@ static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
   const size_t smem = (size_t)2 * vec_per_cta * a.head_dim * sizeof(double);
   encode_exact_kernel<<<(unsigned)grid, kExactThreads, smem, stream>>>(a);
   advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, lens);
-  return cudaGetLastError() == cudaSuccess ? PQ_OK : PQ_ERR_CUDA;
+  return pq::launch_status();
 }
 
 }  // namespace pq

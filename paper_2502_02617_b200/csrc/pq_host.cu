@@ -50,7 +50,16 @@ inline void cell_moments(int level, double lo, double hi, double* m0, double* m1
 
 }  // namespace
 
+namespace pq {
+static thread_local cudaError_t g_last_cuda_error = cudaSuccess;
+void note_cuda_error(cudaError_t e) { g_last_cuda_error = e; }
+}  // namespace pq
+
 extern "C" {
+
+const char* pq_last_cuda_error(void) {
+  return pq::g_last_cuda_error == cudaSuccess ? "" : cudaGetErrorString(pq::g_last_cuda_error);
+}
 
 const char* pq_status_string(int32_t status) {
   switch (status) {
@@ -183,16 +192,19 @@ int32_t pq_build_tables(const double* cen, const double* bnd, void* tables_host)
     std::memcpy(&ub, &b, 2);
     return (uint32_t)ua | ((uint32_t)ub << 16);
   };
-  for (int c = 0; c < 16; ++c) t.l1_h2[c] = h2(std::cos(cen[c]), std::sin(cen[c]));
-  for (int c = 0; c < 4; ++c) t.l2_h2[c] = h2(std::cos(cen[16 + c]), std::sin(cen[16 + c]));
-  for (int p = 0; p < 4; ++p)
-    for (int c4 = 0; c4 < 4; ++c4)
-      for (int c3 = 0; c3 < 4; ++c3) {
-        const double a4 = cen[24 + c4], a3 = cen[20 + c3];
-        const double t4 = (p >> 1) ? std::sin(a4) : std::cos(a4);
-        const double t3 = (p & 1) ? std::sin(a3) : std::cos(a3);
-        t.u43_h[p][c4 * 4 + c3] = (uint16_t)(h2(t4 * t3, 0.0) & 0xFFFFu);
-      }
+  auto split = [&](double va, double vb, uint32_t* hi, uint32_t* lo) {
+    const double ha = (double)__half2float(__double2half(va)), hb = (double)__half2float(__double2half(vb));
+    *hi = h2(va, vb);
+    *lo = h2(va - ha, vb - hb);
+  };
+  for (int c = 0; c < 16; ++c) split(std::cos(cen[c]), std::sin(cen[c]), &t.l1_hi[c], &t.l1_lo[c]);
+  for (int s = 0; s < 4; ++s)
+    for (int i = 0; i < 64; ++i) {
+      const double a2 = cen[16 + (i & 3)], a3 = cen[20 + ((i >> 2) & 3)], a4 = cen[24 + (i >> 4)];
+      const double t4 = (s >> 1) ? std::sin(a4) : std::cos(a4);
+      const double t3 = (s & 1) ? std::sin(a3) : std::cos(a3);
+      split(t4 * t3 * std::cos(a2), t4 * t3 * std::sin(a2), &t.u_tab[s][i].x, &t.u_tab[s][i].y);
+    }
   std::memcpy(tables_host, &t, sizeof(t));
   return PQ_OK;
 }
