@@ -194,7 +194,7 @@ def _oracle_match(cache, K_chunk, V_chunk, b_enc, q, out):
             res["codes_mismatch_outside_window"] += int(np.count_nonzero(diff & (dist > 1e-6)))
     lens = cache.lens.cpu().numpy()
     worst = 0.0
-    for (b, hk) in ((b_enc, 0), ((b_enc + 3) % BATCH, 5)):
+    for (b, hk) in ((b_enc, 0), ((b_enc + 3) % BATCH, 5 % HKV)):
         n = int(lens[b])
         c = codes[b, hk, :, :n].cpu().numpy()
         r = radii[b, hk, :, :n].cpu().numpy()
@@ -321,11 +321,11 @@ def run_cuda(args):
     clocks = sampler.stop()
     cache.check_status()
     match = None
-    if rank == 0:
+    if rank == 0 and not args.skip_match:
         b_enc, qq = last
         Kb, Vb = chunks[(n_total - 1) % 2]
         match = _oracle_match(cache, Kb, Vb, b_enc, qq, out)
-    e2e_total_ms, e2e_seg, _ = timed(e2e=True)
+    e2e_total_ms, e2e_seg, _ = (total_ms, seg, None) if args.skip_e2e else timed(e2e=True)
     cache.check_status()
 
     def reduce_max(x):
@@ -357,7 +357,7 @@ def run_cuda(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
         "data": "synthetic",
-        "config": {"workload": WORKLOAD, "per_gpu": True, "l2": "inputs larger than L2 (260 MB cache per decode, "
+        "config": {"workload": WORKLOAD, "batch": BATCH, "per_gpu": True, "l2": "inputs larger than L2 (260 MB cache per decode, "
                    "two alternating 128 MiB prefill chunks)", "compressed_bytes_per_decode": comp_bytes,
                    "decode_ms": dec_ms, "append_ms": app_ms, "encode_ms": enc_ms,
                    "value_definition": "compressed bytes / CUDA-event time of pq_decode_attention (both its kernels)"},
@@ -383,13 +383,18 @@ def run_cuda(args):
 
 
 def main():
+    global BATCH
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=BATCH, help="sequences in the resident batch (profiling captures use fewer)")
+    ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiling captures)")
+    ap.add_argument("--skip-match", action="store_true", help="skip the sampled oracle check (profiling captures)")
     args = ap.parse_args()
+    BATCH = args.batch
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     if args.impl == "reference":
         run_reference(args)

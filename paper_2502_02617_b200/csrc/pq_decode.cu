@@ -131,6 +131,8 @@ __host__ inline Workspace carve_workspace(void* base, int d, int batch, int n_q_
   return w;
 }
 
+constexpr int kMaxGroup = 8;  // query heads per kv head handled by one CTA
+
 struct DecodeArgs {
   int d, n_q_heads, n_kv_heads, batch, capacity, io_dtype;
   float scale;
@@ -162,40 +164,66 @@ __global__ void rotate_query_kernel(DecodeArgs a) {
   if (bh < a.batch * a.n_kv_heads && j == 0) a.ws.tickets[bh] = 0;
 }
 
-constexpr int kMaxGroup = 8;       // query heads per kv head handled by one CTA
 constexpr int kSimpleThreads = 128;
 
-// Merge the split partials of the `g` query heads of (b, kv head), normalise, rotate back by
-// S^T and store.  Runs in the last CTA that finishes for this (b, kv head).
-__device__ void combine_and_store(const DecodeArgs& a, int b, int hk, int g, float* o_sm /* [d] */) {
-  const int d = a.d, ns = a.ws.n_splits, tid = threadIdx.x;
-  for (int hh = 0; hh < g; ++hh) {
-    const int h = hk * g + hh;
-    const float* ml = a.ws.ml + ((int64_t)b * a.n_q_heads + h) * ns * 2;
-    const float* op = a.ws.o + ((int64_t)b * a.n_q_heads + h) * ns * d;
+// Shared memory (floats) that combine_and_store needs.
+__host__ __device__ inline int combine_smem_floats(int g, int d, int n_splits) { return g * n_splits + g + g * d; }
+
+// Merge the split partials of the `g` query heads of (b, kv head) in split order, normalise,
+// rotate back by S^T and store.  Runs in the last CTA that finishes for this (b, kv head); `sm`
+// must hold combine_smem_floats(...) floats.
+__device__ void combine_and_store(const DecodeArgs& a, int b, int hk, int g, float* sm) {
+  const int d = a.d, ns = a.ws.n_splits, tid = threadIdx.x, nthr = blockDim.x;
+  float* w_sm = sm;               // [g][ns] weight of split s for head h
+  float* linv_sm = sm + g * ns;   // [g]
+  float* o_sm = linv_sm + g;      // [g][d]
+  const int64_t h0 = (int64_t)b * a.n_q_heads + hk * g;
+  if (tid < g) {
+    const float* ml = a.ws.ml + (h0 + tid) * ns * 2;
     float M = -CUDART_INF_F;
     for (int s = 0; s < ns; ++s) M = fmaxf(M, ml[2 * s]);
     float Lsum = 0.f;
-    for (int s = 0; s < ns; ++s) Lsum += ml[2 * s + 1] * (ml[2 * s] == -CUDART_INF_F ? 0.f : exp2f(ml[2 * s] - M));
-    if (tid < d) {
-      float acc = 0.f;
-      for (int s = 0; s < ns; ++s) {
-        const float w = ml[2 * s] == -CUDART_INF_F ? 0.f : exp2f(ml[2 * s] - M);
-        acc += op[(int64_t)s * d + tid] * w;
+    for (int s = 0; s < ns; ++s) {
+      const float w = ml[2 * s] == -CUDART_INF_F ? 0.f : exp2f(ml[2 * s] - M);
+      w_sm[tid * ns + s] = w;
+      Lsum += ml[2 * s + 1] * w;
+    }
+    linv_sm[tid] = Lsum > 0.f ? 1.f / Lsum : 0.f;
+  }
+  __syncthreads();
+  for (int idx = tid; idx < g * d; idx += nthr) {
+    const int h = idx / d, j = idx - h * d;
+    const float* op = a.ws.o + (h0 + h) * ns * d + j;
+    float acc = 0.f;
+    for (int s = 0; s < ns; ++s) acc = fmaf(op[(int64_t)s * d], w_sm[h * ns + s], acc);
+    o_sm[idx] = acc * linv_sm[h];
+  }
+  __syncthreads();
+  // x_hat_i = sum_j y_hat_j S[i][j]: one warp per output row i, lanes over j
+  const int lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
+  for (int i = warp; i < d; i += nwarps) {
+    float acc[kMaxGroup];
+#pragma unroll
+    for (int h = 0; h < kMaxGroup; ++h) acc[h] = 0.f;
+    for (int j = lane; j < d; j += 32) {
+      const float sij = a.S[(int64_t)i * d + j];
+#pragma unroll
+      for (int h = 0; h < kMaxGroup; ++h)
+        if (h < g) acc[h] = fmaf(o_sm[h * d + j], sij, acc[h]);
+    }
+#pragma unroll
+    for (int h = 0; h < kMaxGroup; ++h) {
+      if (h < g) {
+        float v = acc[h];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) {
+          const int64_t idx = (h0 + h) * d + i;
+          if (a.io_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[idx] = __float2bfloat16(v);
+          else reinterpret_cast<float*>(a.out)[idx] = v;
+        }
       }
-      o_sm[tid] = Lsum > 0.f ? acc / Lsum : 0.f;
     }
-    __syncthreads();
-    if (tid < d) {
-      // x_hat_i = sum_j y_hat_j S[i][j]
-      float acc = 0.f;
-      const float* srow = a.S + (int64_t)tid * d;
-      for (int j = 0; j < d; ++j) acc = fmaf(o_sm[j], srow[j], acc);
-      const int64_t idx = ((int64_t)b * a.n_q_heads + h) * d + tid;
-      if (a.io_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[idx] = __float2bfloat16(acc);
-      else reinterpret_cast<float*>(a.out)[idx] = acc;
-    }
-    __syncthreads();
   }
 }
 
@@ -462,8 +490,10 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
     return pq::launch_status();
   }
   const pq::Layout L = pq::make_layout(head_dim, capacity);
-  const size_t smem = 2 * L.block_bytes + sizeof(float) * ((size_t)g * head_dim + 3 * g * pq::kTokenBlock +
-                                                           3 * pq::kMaxGroup + 64);
+  size_t smem = 2 * L.block_bytes + sizeof(float) * ((size_t)g * head_dim + 3 * g * pq::kTokenBlock +
+                                                     3 * pq::kMaxGroup + 64);
+  const size_t smem_combine = sizeof(float) * pq::combine_smem_floats(g, head_dim, a.ws.n_splits);
+  if (smem < smem_combine) smem = smem_combine;
   dim3 grid(a.ws.n_splits, n_kv_heads, batch);
   pq::decode_attention_simple_kernel<<<grid, pq::kSimpleThreads, smem, st>>>(a);
   return pq::launch_status();

@@ -42,7 +42,7 @@ constexpr int kSmBar = kSmU + 4 * 64 * 16 * 8;        // full[4], empty[4] : 64
 constexpr int kSmFlags = kSmBar + 64;                 // abort flag, is_last : 16
 constexpr int kSmRing = (kSmFlags + 16 + 127) / 128 * 128;
 // after the main loop the ring is reused for the cross-warp merge: 16 warps x 8 heads x (128 + 2) floats
-constexpr int kMergeBytes = 16 * 8 * 128 * 4 + 16 * 8 * 2 * 4;
+constexpr int kMergeBytes = 16 * 8 * 128 * 4 + 16 * 8 * 2 * 4;  // also >= combine_smem_floats(8, 128, 128) * 4
 constexpr int kSmTotal = kSmRing + (kStages * kStageBytes > kMergeBytes ? kStages * kStageBytes : kMergeBytes);
 static_assert(kSmRing % 128 == 0, "ring must be 128-byte aligned");
 
