@@ -47,6 +47,7 @@ extern "C" {
 #define PQ_ERR_TIMEOUT (-6)      /* a bounded device-side wait gave up */
 #define PQ_ERR_NONFINITE (-7)    /* inputs contained NaN or Inf */
 #define PQ_ERR_EMPTY (-8)        /* attention over a sequence of length 0 */
+#define PQ_ERR_SCRATCH (-9)      /* the problem needs more scratch than the built-in buffer holds */
 
 #define PQ_DTYPE_F32 0
 #define PQ_DTYPE_BF16 1
@@ -153,6 +154,34 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
                             const void* cache_dev, const int32_t* cache_lens_dev, int32_t batch,
                             int32_t capacity, int32_t max_len, float scale, void* out_dev,
                             void* workspace_dev, int32_t* status_dev, void* stream);
+
+/*
+ * pq_decode_attention for callers that cannot hand over scratch memory.  (The paper has no
+ * counterpart; this is a packaging variant of the call above.)
+ *
+ * Some callers are not in a position to allocate device memory when they reach this call: code
+ * running inside a region where the allocator must not be entered (a pre-sized serving loop with
+ * a fixed memory plan, a plugin that is handed its tensors and nothing else, a caller replaying
+ * a fixed sequence of launches).  For them the library carries its own scratch: a file-scope
+ * device array of PQ_STATIC_SCRATCH_BYTES bytes that every GPU which loads the library keeps
+ * until the process exits.  Arguments and results are those of pq_decode_attention without
+ * `workspace_dev`.
+ *   - Returns PQ_ERR_SCRATCH, and launches nothing, if pq_workspace_bytes(...) for these arguments
+ *     exceeds PQ_STATIC_SCRATCH_BYTES (compare pq_static_scratch_bytes()).
+ *   - The first call on each device looks up the device address of the array (a host-side query,
+ *     no allocation); make that first call outside any stream capture.
+ *   - Never calls cudaMalloc, cudaFree or any allocating routine.
+ *   - All calls on a device share the one array.  It keeps the previous call's contents; the part
+ *     that must start at zero (the split tickets) is cleared by the call's own first kernel.
+ *     Calls that may overlap on the GPU (different streams, no ordering) race on it: order them.
+ */
+#define PQ_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+int64_t pq_static_scratch_bytes(void);
+int32_t pq_decode_attention_static(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                                   const void* tables_dev, const void* q_dev, int32_t io_dtype,
+                                   const void* cache_dev, const int32_t* cache_lens_dev, int32_t batch,
+                                   int32_t capacity, int32_t max_len, float scale, void* out_dev,
+                                   int32_t* status_dev, void* stream);
 
 /*
  * Inspection (test support, not a hot path): unpack the first n_tokens positions of every

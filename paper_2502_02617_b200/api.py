@@ -18,7 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libpolarquant.so")
 
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_CAPACITY = -1, -2, -3, -4
-ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE, ERR_EMPTY = -5, -6, -7, -8
+ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE, ERR_EMPTY, ERR_SCRATCH = -5, -6, -7, -8, -9
 DTYPE_F32, DTYPE_BF16 = 0, 1
 STATUS_WORDS = 4
 N_CENTROIDS, N_BOUNDARIES = 28, 24
@@ -42,6 +42,10 @@ _SIGNATURES = {
     "pq_decode_attention": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p,
                                       c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p,
                                       c_void_p]),
+    "pq_static_scratch_bytes": (c_int64, []),
+    "pq_decode_attention_static": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p,
+                                             c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p,
+                                             c_void_p]),
     "pq_unpack_codes": (c_int32, [c_int32, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p]),
     "pq_dequant_kv": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p,
                                 c_void_p]),
@@ -172,6 +176,22 @@ def pq_decode_attention(S, tables, q, cache, cache_lens, n_kv_heads, capacity, m
                                      _ptr(cache), _ptr(cache_lens), batch, capacity, max_len, float(scale),
                                      _ptr(out), _ptr(workspace), _ptr(status), _stream(stream)),
            "pq_decode_attention")
+
+
+def pq_static_scratch_bytes() -> int:
+    return int(lib().pq_static_scratch_bytes())
+
+
+def pq_decode_attention_static(S, tables, q, cache, cache_lens, n_kv_heads, capacity, max_len, scale, out, status,
+                               stream=None):
+    """pq_decode_attention on the library's built-in scratch buffer, for callers that cannot allocate
+    or pass a workspace.  Raises PolarQuantError(ERR_SCRATCH) if the problem needs more scratch than
+    pq_static_scratch_bytes().  Calls on one device share that buffer: keep them stream-ordered."""
+    batch, n_q_heads, d = q.shape
+    assert q.is_contiguous() and out.is_contiguous() and out.shape == q.shape and out.dtype == q.dtype
+    _check(lib().pq_decode_attention_static(d, n_q_heads, n_kv_heads, _ptr(S), _ptr(tables), _ptr(q), _dtype_code(q),
+                                            _ptr(cache), _ptr(cache_lens), batch, capacity, max_len, float(scale),
+                                            _ptr(out), _ptr(status), _stream(stream)), "pq_decode_attention_static")
 
 
 def pq_unpack_codes(d, n_kv_heads, cache, batch, capacity, n_tokens, stream=None):

@@ -499,6 +499,43 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
   return pq::launch_status();
 }
 
+// ---- decode attention on the library's own scratch ---------------------------------------------
+// Scratch for callers that cannot allocate: lives in every GPU context that loads the library.
+// In host code the name below is only a handle; the device address comes from
+// cudaGetSymbolAddress, once per device, and is what the kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[PQ_STATIC_SCRATCH_BYTES];
+
+int64_t pq_static_scratch_bytes(void) { return PQ_STATIC_SCRATCH_BYTES; }
+
+int32_t pq_decode_attention_static(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                                   const void* tables_dev, const void* q_dev, int32_t io_dtype,
+                                   const void* cache_dev, const int32_t* cache_lens_dev, int32_t batch,
+                                   int32_t capacity, int32_t max_len, float scale, void* out_dev,
+                                   int32_t* status_dev, void* stream) {
+  const int64_t need = pq_workspace_bytes(head_dim, batch, n_q_heads, n_kv_heads, max_len);
+  if (need < 0) return (int32_t)need;
+  if (need > PQ_STATIC_SCRATCH_BYTES) return PQ_ERR_SCRATCH;
+  constexpr int kMaxDevices = 64;
+  static void* scratch_of_device[kMaxDevices] = {};
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    pq::note_cuda_error(e == cudaSuccess ? cudaErrorInvalidDevice : e);
+    return PQ_ERR_CUDA;
+  }
+  void* scratch = scratch_of_device[dev];
+  if (scratch == nullptr) {  // first call on this device (which is current): resolve the symbol
+    e = cudaGetSymbolAddress(&scratch, g_static_scratch);
+    if (e != cudaSuccess || scratch == nullptr) {
+      pq::note_cuda_error(e == cudaSuccess ? cudaErrorInvalidSymbol : e);
+      return PQ_ERR_CUDA;
+    }
+    scratch_of_device[dev] = scratch;
+  }
+  return pq_decode_attention(head_dim, n_q_heads, n_kv_heads, S_dev, tables_dev, q_dev, io_dtype, cache_dev,
+                             cache_lens_dev, batch, capacity, max_len, scale, out_dev, scratch, status_dev, stream);
+}
+
 int32_t pq_unpack_codes(int32_t head_dim, int32_t n_kv_heads, const void* cache_dev, int32_t batch, int32_t capacity,
                         int32_t n_tokens, uint8_t* codes_dev, void* radii_dev, void* stream) {
   if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;

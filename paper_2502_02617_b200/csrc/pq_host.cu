@@ -72,6 +72,7 @@ const char* pq_status_string(int32_t status) {
     case PQ_ERR_TIMEOUT: return "bounded device wait timed out";
     case PQ_ERR_NONFINITE: return "non-finite input";
     case PQ_ERR_EMPTY: return "attention over an empty sequence";
+    case PQ_ERR_SCRATCH: return "built-in scratch buffer too small for this problem";
     default: return "unknown status";
   }
 }

@@ -35,7 +35,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_status_strings_and_constants():
     assert pq.status_string(0) == "ok"
-    for code in range(-8, 0):
+    for code in range(-9, 0):
         assert pq.status_string(code) not in ("ok", "unknown status")
     assert pq.status_string(-99) == "unknown status"
     assert pq.token_block() % 8 == 0
