@@ -168,6 +168,147 @@ __global__ void __launch_bounds__(kExactThreads) encode_exact_kernel(EncodeArgs 
   }
 }
 
+}  // namespace pq
+#include "pq_encode_fast.cuh"
+namespace pq {
+
+// ------------------------------------------------------------------------------------------
+// head_dim 128, float32 rotation on the FMA pipe + the fast quantiser.  One CTA = 128 consecutive
+// rows of one (K|V, head); thread (row, half) owns 64 rotated coordinates (4 blocks) of its row.
+// ------------------------------------------------------------------------------------------
+constexpr int kFfmaThreads = 256;
+constexpr int kFfmaSmem = (128 * 129 + 2 * 128) * 4 + 64 + (int)sizeof(FixQueue);
+
+// Write the four blocks [4*half, 4*half+4) of the token at `pos`.
+__device__ __forceinline__ void store_half_token(uint8_t* tb, int tok, int half, const FastBlock* fb, int32_t* status) {
+  constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock, orad = o4 + 2 * kTokenBlock;
+  *reinterpret_cast<uint4*>(tb + tok * 32 + half * 16) = make_uint4(fb[0].l1, fb[1].l1, fb[2].l1, fb[3].l1);
+  *reinterpret_cast<uint32_t*>(tb + o2 + tok * 8 + half * 4) = fb[0].l2 | (fb[1].l2 << 8) | (fb[2].l2 << 16) | (fb[3].l2 << 24);
+  *reinterpret_cast<uint16_t*>(tb + o3 + tok * 4 + half * 2) =
+      (uint16_t)(fb[0].l3 | (fb[1].l3 << 4) | (fb[2].l3 << 8) | (fb[3].l3 << 12));
+  tb[o4 + tok * 2 + half] = (uint8_t)(fb[0].l4 | (fb[1].l4 << 2) | (fb[2].l4 << 4) | (fb[3].l4 << 6));
+  int sat = 0;
+  __half r[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float v = fb[i].radius;
+    if (v > 65504.f) { v = 65504.f; ++sat; }
+    r[i] = __float2half_rn(v);
+  }
+  *reinterpret_cast<uint2*>(tb + orad + tok * 16 + half * 8) = *reinterpret_cast<uint2*>(r);
+  if (sat) atomicAdd(status + 2, sat);
+}
+
+// Quantise and store the 4 blocks of (row, half) whose rotated coordinates are y[64]; ambiguous
+// decisions go to the fix-up queue.  Returns the ambiguity bits that did not fit (4 x 15 bits).
+__device__ __forceinline__ void quantise_and_store(const EncodeArgs& a, const FastQuant& fq, bool uniform_l1, const float* y,
+                                                   float row_norm, int row, int head, int kv, int half, bool valid,
+                                                   FixQueue* q, uint32_t* left, int64_t* xoff_out, uint8_t** tb_out,
+                                                   int* tok_out) {
+  const float dy = kRotErr * row_norm;
+  FastBlock fb[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    polar_quant_block_fast(y + 16 * i, dy, fq, &fb[i]);
+    if (!uniform_l1) fb[i].amb |= 0xFFu;  // other level-1 codebooks: decide every level-1 angle exactly
+    left[i] = 0u;
+  }
+  *tb_out = nullptr;
+  if (!valid) return;
+  int seq, pos;
+  row_destination(a, row, &seq, &pos);
+  if (pos < 0) return;
+  const Layout L = make_layout(128, a.capacity);
+  uint8_t* tb = a.cache + block_offset(L, a.n_kv_heads, seq, head, kv, pos);
+  store_half_token(tb, pos % kTokenBlock, half, fb, a.status);
+  *xoff_out = (int64_t)row * a.token_stride + (int64_t)head * a.head_stride;
+  *tb_out = tb;
+  *tok_out = pos % kTokenBlock;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) left[i] = fb[i].amb;
+}
+
+// Drain the ambiguous decisions of a tile: rounds of (push, barrier, process, barrier).  All
+// `n_threads` threads of the barrier `bar_id` call this together.
+__device__ inline void fixup_rounds(const EncodeArgs& a, FixQueue* q, uint32_t* left, int64_t xoff, uint8_t* tb, int tok,
+                                    int half, int kv, int t, int n_threads, int bar_id) {
+  const void* xbase = kv ? a.V : a.K;
+  for (int round = 0; round < 64; ++round) {
+    if (tb != nullptr) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        if (left[i]) fix_push(q, left[i], xoff, tb, tok, 4 * half + i, &left[i]);
+    }
+    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
+    const int n = min(q->count, kFixCap);
+    if (n == 0) break;  // uniform: every thread reads the same count
+    fix_process(q, n, t, n_threads, xbase, a.in_dtype, a.S, *a.tables, a.status);
+    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
+    if (t == 0) q->count = 0;
+    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
+  }
+}
+
+__global__ void __launch_bounds__(kFfmaThreads) encode_ffma_kernel(EncodeArgs a) {
+  extern __shared__ __align__(16) float smem_f[];
+  float* xT = smem_f;                  // [128 k][129]
+  float* rowsq = smem_f + 128 * 129;   // [2][128]
+  FastQuant* fq = reinterpret_cast<FastQuant*>(rowsq + 256);
+  FixQueue* fixq = reinterpret_cast<FixQueue*>(rowsq + 256 + 16);
+  const int tid = threadIdx.x, head = blockIdx.y, kv = blockIdx.z;
+  const int row0 = blockIdx.x * 128;
+  const void* xbase = kv ? a.V : a.K;
+  int bad = 0;
+  for (int idx = tid; idx < 128 * 128; idx += kFfmaThreads) {
+    const int r = idx >> 7, k = idx & 127;
+    float f = 0.f;
+    if (row0 + r < a.total_tokens) {
+      f = load_elem(xbase, a.in_dtype, (int64_t)(row0 + r) * a.token_stride + (int64_t)head * a.head_stride + k);
+      if (!isfinite(f)) ++bad;
+    }
+    xT[k * 129 + r] = f;
+  }
+  if (bad) {
+    atomicAdd(a.status + 1, bad);
+    set_status(a.status, PQ_ERR_NONFINITE);
+  }
+  if (tid == 0) {
+    load_fast_quant(a.tables, fq);
+    fixq->count = 0;
+  }
+  __syncthreads();
+  const int r = tid & 127, half = tid >> 7;
+  float y[64];
+#pragma unroll
+  for (int i = 0; i < 64; ++i) y[i] = 0.f;
+  const float4* S4 = reinterpret_cast<const float4*>(a.S) + half * 16;
+  for (int k = 0; k < 128; ++k) {
+    const float xv = xT[k * 129 + r];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      const float4 s = __ldg(S4 + k * 32 + i);
+      y[4 * i] = fmaf(xv, s.x, y[4 * i]);
+      y[4 * i + 1] = fmaf(xv, s.y, y[4 * i + 1]);
+      y[4 * i + 2] = fmaf(xv, s.z, y[4 * i + 2]);
+      y[4 * i + 3] = fmaf(xv, s.w, y[4 * i + 3]);
+    }
+  }
+  float sq = 0.f;
+#pragma unroll
+  for (int i = 0; i < 64; ++i) sq = fmaf(y[i], y[i], sq);
+  rowsq[half * 128 + r] = sq;
+  __syncthreads();
+  const float row_norm = sqrtf(rowsq[r] + rowsq[128 + r]) * 1.0001f;
+  const bool uniform = (a.tables->flags & kFlagUniformL1) != 0u;
+  uint32_t left[4];
+  int64_t xoff = 0;
+  uint8_t* tb = nullptr;
+  int tok = 0;
+  quantise_and_store(a, *fq, uniform, y, row_norm, row0 + r, head, kv, half, row0 + r < a.total_tokens, fixq, left, &xoff,
+                     &tb, &tok);
+  fixup_rounds(a, fixq, left, xoff, tb, tok, half, kv, tid, kFfmaThreads, 1);
+}
+
 // lens[b] += rows of sequence b (skipped for sequences that did not fit).
 __global__ void advance_lens_kernel(const int32_t* cu_seqlens, int batch, int capacity, int32_t* lens) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
@@ -189,6 +330,21 @@ static int32_t check_common(int head_dim, int n_kv_heads, const void* S, const v
 
 static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
   if (a.total_tokens == 0) return PQ_OK;
+  if (a.head_dim == 128 && a.total_tokens >= 32) {
+    static bool configured = false;
+    if (!configured) {
+      const cudaError_t e = cudaFuncSetAttribute(encode_ffma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFfmaSmem);
+      if (e != cudaSuccess) {
+        note_cuda_error(e);
+        return PQ_ERR_CUDA;
+      }
+      configured = true;
+    }
+    dim3 grid((a.total_tokens + 127) / 128, a.n_kv_heads, 2);
+    encode_ffma_kernel<<<grid, kFfmaThreads, kFfmaSmem, stream>>>(a);
+    advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, lens);
+    return launch_status();
+  }
   const int groups = kExactThreads / a.head_dim;
   const int vec_per_cta = kExactVecPerGroup * groups;
   const int64_t n_vec = (int64_t)a.total_tokens * 2 * a.n_kv_heads;

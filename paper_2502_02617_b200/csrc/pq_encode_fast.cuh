@@ -1,0 +1,234 @@
+// Fast encoder for head_dim 128 with the uniform level-1 codebook (included by pq_encode.cu).
+//
+// The rotation y = x . S is computed with float32-grade accuracy (tensor cores with S split into
+// two bf16 terms, or float32 FMAs).  Either way |y - y_exact| <= kRotErr * ||x||_2 per coordinate:
+//   two bf16 terms drop at most 2^-17 |S_kj| per entry, so the error is <= 2^-17 sum_k |x_k||S_kj|
+//   <= 2^-17 ||x||_2 (Cauchy-Schwarz, columns of S have unit norm); a float32 dot product of 128
+//   terms has the same bound (129 * 2^-24).
+// Angles are never computed.  Every code is decided by sign tests on the pair (Algorithm 1, Polar +
+// Quant, in the form "which side of the boundary line is the point on"), in float32, together with
+// a certified margin: a decision is trusted only if the point is farther from every boundary than
+// the error bound allows it to move.  The rare decisions inside the margin are taken again in
+// float64 from the original inputs by the whole warp, so the codes equal a float64 evaluation of
+// Algorithm 1 (up to ~1e-15 rad).
+#pragma once
+
+namespace pq {
+
+constexpr float kRotErr = 1.1f * 7.62939453125e-06f;  // 1.1 * 2^-17
+
+// Per-call constants of the fast quantiser (uniform level-1 codebook; levels 2..4 from Tables).
+struct FastQuant {
+  float t2[3][3];   // tan^2 of the three boundaries of levels 2, 3, 4
+};
+
+__device__ inline void load_fast_quant(const Tables* tb, FastQuant* fq) {
+  for (int l = 0; l < 3; ++l)
+    for (int k = 0; k < 3; ++k) {
+      const double t = tb->bnd_sin[15 + 3 * l + k] / tb->bnd_cos[15 + 3 * l + k];
+      fq->t2[l][k] = (float)(t * t);
+    }
+}
+
+// Level >= 2 decision on squared child radii (sa: cosine side, sb: sine side).
+//   code = #{k : sb > T_k sa},  T_k = tan^2(beta_k)  (both sides of r_b cos b > r_a sin b are >= 0).
+// Margin: the radii are norms of n-coordinate sub-vectors, so they move by at most E = sqrt(n) * dy.
+// With D = sb - T sa, |D - D_exact| <= 2E(r_b + T r_a) + E^2 (1 + T) + rho (sb + T sa), and
+// (2E(r_b + T r_a))^2 <= 8 E^2 (sb + T^2 sa), (p+q+z)^2 <= 3(p^2+q^2+z^2), so the decision is
+// certified if D^2 > 24 E^2 (sb + T^2 sa) + 3 E^4 (1+T)^2 + 3 rho^2 (sb + T sa)^2 for every k; the
+// right side grows with T, so the largest T is used with the smallest |D|.
+__device__ __forceinline__ uint32_t quant_upper_fast(float sa, float sb, const float* T, float e2 /* E^2 */,
+                                                     bool* ambiguous) {
+  const float d0 = fmaf(-T[0], sa, sb), d1 = fmaf(-T[1], sa, sb), d2 = fmaf(-T[2], sa, sb);
+  const uint32_t code = (d0 > 0.f) + (d1 > 0.f) + (d2 > 0.f);
+  const float dm = fminf(fminf(fabsf(d0), fabsf(d1)), fabsf(d2));
+  const float tm = T[2];
+  const float w = fmaf(tm * tm, sa, sb);
+  const float u = fmaf(tm, sa, sb);
+  float rhs = fmaf(24.f * e2, w, 3.f * e2 * e2 * (1.f + tm) * (1.f + tm));
+  rhs = fmaf(3e-12f * u, u, rhs);  // rho = 1e-6 covers float32 rounding of the squares and products
+  *ambiguous = !(dm * dm > rhs);   // also true for NaN
+  return code;
+}
+
+// Level-1 decision for the uniform codebook (boundaries k pi/8): fold into the first octant,
+// u = max(|a|,|b|), v = min(|a|,|b|); the boundaries are the axes (v = 0), the diagonals (u = v) and
+// the lines at pi/8 from the axes (v cos(pi/8) = u sin(pi/8)).  The point moves by at most
+// sqrt(2) dy, so the decision is certified if its distance to all three exceeds that.
+__device__ __forceinline__ uint32_t quant_level1_fast(float a, float b, float e1 /* sqrt(2) dy */, bool* ambiguous) {
+  const float ax = fabsf(a), ay = fabsf(b);
+  const float u = fmaxf(ax, ay), v = fminf(ax, ay);
+  const bool swap = ay > ax;
+  const float t = fmaf(v, 0.92387953251128674f, -u * 0.38268343236508977f);  // v cos(pi/8) - u sin(pi/8)
+  const bool hi = t > 0.f;
+  const float dmin = fminf(fminf(v, (u - v) * 0.70710678118654752f), fabsf(t));
+  *ambiguous = !(dmin > fmaf(u, 4.76837158203125e-07f, e1));  // + 2^-21 u for the float32 roundings
+  const uint32_t sector = swap ? (hi ? 2u : 3u) : (hi ? 1u : 0u);  // pi/8 sector inside the quadrant
+  const uint32_t sa = __float_as_uint(a) >> 31, sb = __float_as_uint(b) >> 31;
+  // b >= 0: theta = phi or pi - phi; b < 0: theta = pi + phi or 2 pi - phi
+  return (sb << 3) + (sector ^ ((sa ^ sb) ? 7u : 0u));
+}
+
+// Codes, squared radius and ambiguity mask of one 16-coordinate block.
+// Ambiguity bits: 0..7 level-1 pairs, 8..11 level 2, 12..13 level 3, 14 level 4.
+struct FastBlock {
+  uint32_t l1, l2, l3, l4, amb;
+  float radius;
+};
+
+__device__ __forceinline__ void polar_quant_block_fast(const float* y, float dy, const FastQuant& fq, FastBlock* out) {
+  const float e1 = 1.41421356f * dy;
+  float s1[8], s2[4], s3[2];
+  uint32_t l1 = 0, l2 = 0, l3 = 0, amb = 0;
+  bool am;
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    l1 |= quant_level1_fast(y[2 * j], y[2 * j + 1], e1, &am) << (4 * j);
+    amb |= (am ? 1u : 0u) << j;
+    s1[j] = fmaf(y[2 * j], y[2 * j], y[2 * j + 1] * y[2 * j + 1]);
+  }
+  const float e2 = dy * dy;
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    l2 |= quant_upper_fast(s1[2 * j], s1[2 * j + 1], fq.t2[0], 2.f * e2, &am) << (2 * j);
+    amb |= (am ? 1u : 0u) << (8 + j);
+    s2[j] = s1[2 * j] + s1[2 * j + 1];
+  }
+#pragma unroll
+  for (int j = 0; j < 2; ++j) {
+    l3 |= quant_upper_fast(s2[2 * j], s2[2 * j + 1], fq.t2[1], 4.f * e2, &am) << (2 * j);
+    amb |= (am ? 1u : 0u) << (12 + j);
+    s3[j] = s2[2 * j] + s2[2 * j + 1];
+  }
+  out->l4 = quant_upper_fast(s3[0], s3[1], fq.t2[2], 8.f * e2, &am);
+  amb |= (am ? 1u : 0u) << 14;
+  out->l1 = l1;
+  out->l2 = l2;
+  out->l3 = l3;
+  out->amb = amb;
+  out->radius = sqrtf(s3[0] + s3[1]);
+}
+
+// ---- exact re-decision of the ambiguous angles ------------------------------------------------
+// Threads push their ambiguous decisions into a CTA-wide queue; after a barrier, groups of 8 lanes
+// take one entry each, recompute in float64 the 2^level rotated coordinates under that angle from
+// the original inputs (x in its storage type, S in float32: both exact in float64), decide again
+// and patch the code bits in the cache with 32-bit atomics.  The queue is drained in rounds, so a
+// tile with more ambiguous angles than the queue holds only takes more rounds.
+constexpr int kFixCap = 512;
+
+struct FixQueue {
+  int count;
+  int pad[3];
+  int64_t xoff[kFixCap];   // element offset of the source vector
+  uint8_t* tok[kFixCap];   // token-block base of the destination
+  uint32_t meta[kFixCap];  // token-in-block | blk << 6 | level << 9 | j << 12
+};
+
+// Replace `width` bits at bit offset `bit` of the byte at `addr`.
+__device__ __forceinline__ void patch_bits(uint8_t* addr, int bit, uint32_t mask, uint32_t code) {
+  uint32_t* word = reinterpret_cast<uint32_t*>(reinterpret_cast<uintptr_t>(addr) & ~(uintptr_t)3);
+  const int sh = (int)(reinterpret_cast<uintptr_t>(addr) & 3) * 8 + bit;
+  atomicAnd(word, ~(mask << sh));
+  atomicOr(word, code << sh);
+}
+
+__device__ __forceinline__ void fix_push(FixQueue* q, uint32_t amb, int64_t xoff, uint8_t* tokblock, int tok, int blk,
+                                         uint32_t* left) {
+  while (amb) {
+    const int bit = __ffs(amb) - 1;
+    const int idx = atomicAdd(&q->count, 1);
+    if (idx >= kFixCap) break;  // queue full: keep the rest for the next round
+    amb &= amb - 1;
+    int level, j;
+    if (bit < 8) { level = 1; j = bit; }
+    else if (bit < 12) { level = 2; j = bit - 8; }
+    else if (bit < 14) { level = 3; j = bit - 12; }
+    else { level = 4; j = 0; }
+    q->xoff[idx] = xoff;
+    q->tok[idx] = tokblock;
+    q->meta[idx] = (uint32_t)tok | ((uint32_t)blk << 6) | ((uint32_t)level << 9) | ((uint32_t)j << 12);
+  }
+  *left = amb;
+}
+
+// Process queue entries [0, n): called by `n_threads` threads (a multiple of 32) with linear index `t`.
+__device__ inline void fix_process(const FixQueue* q, int n, int t, int n_threads, const void* xbase, int in_dtype,
+                                   const float* S, const Tables& tb, int32_t* status) {
+  constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock;
+  const int sub = t & 7, group = t >> 3, n_groups = n_threads >> 3;
+  const int rounds = (n + n_groups - 1) / n_groups;
+  int fixed = 0;
+  for (int rd = 0; rd < rounds; ++rd) {
+    const int e = rd * n_groups + group;
+    const bool active = e < n;
+    const uint32_t meta = active ? q->meta[e] : (1u << 9);
+    const int64_t xoff = active ? q->xoff[e] : 0;
+    const int tok = meta & 63, blk = (meta >> 6) & 7, level = (meta >> 9) & 7, j = (meta >> 12) & 7;
+    const int nc = 1 << level, c0 = blk * 16 + j * nc;
+    // this lane's 16 consecutive k
+    double xk[16];
+    if (active) {
+      if (in_dtype == PQ_DTYPE_BF16) {
+        const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(xbase) + xoff + 16 * sub);
+        const uint4 v0 = p[0], v1 = p[1];
+        const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          xk[2 * i] = (double)__uint_as_float(w[i] << 16);
+          xk[2 * i + 1] = (double)__uint_as_float(w[i] & 0xFFFF0000u);
+        }
+      } else {
+        const float* p = reinterpret_cast<const float*>(xbase) + xoff + 16 * sub;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) xk[i] = (double)p[i];
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) xk[i] = 0.0;
+    }
+    int nmax = nc;  // every lane of the warp runs the same number of coordinate steps
+    nmax = max(nmax, __shfl_xor_sync(0xffffffffu, nmax, 8));
+    nmax = max(nmax, __shfl_xor_sync(0xffffffffu, nmax, 16));
+    double y[16];
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+      if (c < nmax) {
+        const int col = c0 + min(c, nc - 1);
+        const float* sp = S + (16 * sub) * 128 + col;
+        double p = 0.0;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) p = fma(xk[i], (double)__ldg(sp + i * 128), p);
+        p += __shfl_xor_sync(0xffffffffu, p, 1);
+        p += __shfl_xor_sync(0xffffffffu, p, 2);
+        p += __shfl_xor_sync(0xffffffffu, p, 4);
+        y[c] = p;
+      } else {
+        y[c] = 0.0;
+      }
+    }
+    if (active && sub == 0) {
+      uint32_t code;
+      if (level == 1) {
+        code = quant_level1_exact(y[0], y[1], tb);
+      } else {
+        // child radii by the same pairwise hypot recursion as Polar
+#pragma unroll
+        for (int m = 16; m > 2; m >>= 1)
+          if (m <= nc)
+#pragma unroll
+            for (int c = 0; c < m / 2; ++c) y[c] = hypot(y[2 * c], y[2 * c + 1]);
+        code = quant_upper_exact(y[0], y[1], level, tb);
+      }
+      uint8_t* tbk = q->tok[e];
+      if (level == 1) patch_bits(tbk + tok * 32 + blk * 4 + (j >> 1), 4 * (j & 1), 0xFu, code);
+      else if (level == 2) patch_bits(tbk + o2 + tok * 8 + blk, 2 * j, 3u, code);
+      else if (level == 3) patch_bits(tbk + o3 + tok * 4 + (blk >> 1), 4 * (blk & 1) + 2 * j, 3u, code);
+      else patch_bits(tbk + o4 + tok * 2 + (blk >> 2), 2 * (blk & 3), 3u, code);
+      ++fixed;
+    }
+  }
+  if (fixed) atomicAdd(status + 3, fixed);
+}
+
+}  // namespace pq

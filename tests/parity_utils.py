@@ -44,8 +44,9 @@ def assert_codes_match(rep):
         f"{rep['inside']} of {rep['total']} codes differ inside the window"
 
 
-def assert_radii_match(gpu_radii: np.ndarray, want16: np.ndarray, max_ulp_fraction=1e-3):
-    """fp16 radii: equal, except that a float32 intermediate may move a value by one fp16 ulp."""
+def assert_radii_match(gpu_radii: np.ndarray, want16: np.ndarray, max_ulp_fraction=5e-3):
+    """fp16 radii: equal, except that the float32-accurate norm of the fast encoder (relative error
+    ~1e-6 against an fp16 spacing of ~7e-4) may round to the neighbouring fp16 value on ~0.2 % of radii."""
     g = gpu_radii.astype(np.float16).view(np.uint16).astype(np.int32)
     w = want16.astype(np.float16).view(np.uint16).astype(np.int32)
     delta = np.abs(g - w)

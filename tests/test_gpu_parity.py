@@ -122,9 +122,12 @@ def test_chunked_prefill_and_append_equal_one_shot_and_oracle():
     c1, r1 = one.unpack(100)
     c2, r2 = two.unpack(100)
     for b, n in enumerate(lens_list):
-        assert torch.equal(c1[b, :, :, :n], c2[b, :, :, :n]) and torch.equal(r1[b, :, :, :n], r2[b, :, :, :n])
+        assert torch.equal(c1[b, :, :, :n], c2[b, :, :, :n])  # codes do not depend on chunking or on the kernel used
+        # radii come from float32-accurate norms whose last rounding may differ between the prefill and
+        # the append kernel: equal, or one fp16 ulp apart on a small fraction
+        assert_radii_match(r1[b, :, :, :n].cpu().numpy(), r2[b, :, :, :n].cpu().numpy())
     q = synthetic.queries(12, B, Hq, d, torch.bfloat16, DEV)
-    assert torch.equal(one.attend(q), two.attend(q))
+    assert rel_l2(to_f64(two.attend(q)), to_f64(one.attend(q))) < 1e-3
 
 
 def test_streaming_decode_steps_follow_the_oracle():
