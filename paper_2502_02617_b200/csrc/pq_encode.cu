@@ -309,6 +309,10 @@ __global__ void __launch_bounds__(kFfmaThreads) encode_ffma_kernel(EncodeArgs a)
   fixup_rounds(a, fixq, left, xoff, tb, tok, half, kv, tid, kFfmaThreads, 1);
 }
 
+}  // namespace pq
+#include "pq_encode_tc.cuh"
+namespace pq {
+
 // lens[b] += rows of sequence b (skipped for sequences that did not fit).
 __global__ void advance_lens_kernel(const int32_t* cu_seqlens, int batch, int capacity, int32_t* lens) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
@@ -330,6 +334,14 @@ static int32_t check_common(int head_dim, int n_kv_heads, const void* S, const v
 
 static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
   if (a.total_tokens == 0) return PQ_OK;
+  {
+    const int32_t tc = try_launch_encode_tc(a, stream);
+    if (tc < 0) return tc;
+    if (tc == 1) {
+      advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, lens);
+      return launch_status();
+    }
+  }
   if (a.head_dim == 128 && a.total_tokens >= 32) {
     static bool configured = false;
     if (!configured) {
