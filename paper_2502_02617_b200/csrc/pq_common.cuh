@@ -42,6 +42,7 @@ struct Tables {
   uint32_t l1_hi[16];
   uint32_t l1_lo[16];
   uint2 u_tab[4][64];
+  double bnd_tan2[9];  // tan^2 of the boundaries of levels 2, 3, 4 (decisions on squared radii)
   uint32_t reserved[30];
 };
 

@@ -228,24 +228,44 @@ __device__ __forceinline__ void quantise_and_store(const EncodeArgs& a, const Fa
   for (int i = 0; i < 4; ++i) left[i] = fb[i].amb;
 }
 
-// Drain the ambiguous decisions of a tile: rounds of (push, barrier, process, barrier).  All
-// `n_threads` threads of the barrier `bar_id` call this together.
-__device__ inline void fixup_rounds(const EncodeArgs& a, FixQueue* q, uint32_t* left, int64_t xoff, uint8_t* tb, int tok,
-                                    int half, int kv, int t, int n_threads, int bar_id) {
-  const void* xbase = kv ? a.V : a.K;
-  for (int round = 0; round < 64; ++round) {
-    if (tb != nullptr) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i)
-        if (left[i]) fix_push(q, left[i], xoff, tb, tok, 4 * half + i, &left[i]);
-    }
+// Named-barrier OR over `n_threads` threads (also a barrier).
+__device__ __forceinline__ bool bar_or(int bar_id, int n_threads, bool v) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, %2, %3, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(out)
+      : "r"((uint32_t)v), "r"(bar_id), "r"(n_threads)
+      : "memory");
+  return out != 0;
+}
+
+// Drain the queue of ambiguous decisions: rounds of (barrier, process, barrier, reset, push what did
+// not fit before).  All `n_threads` threads of named barrier `bar_id` call this together.
+// `leftbits` holds this thread's decisions that found the queue full (15 bits per block, 4 blocks).
+__device__ inline void fix_rounds(const EncodeArgs& a, FixQueue* q, unsigned long long leftbits, int64_t xoff, uint8_t* tb,
+                                  int tok, int half, int kv, int t, int n_threads, int bar_id) {
+  for (int round = 0; round < 256; ++round) {
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
     const int n = min(q->count, kFixCap);
-    if (n == 0) break;  // uniform: every thread reads the same count
-    fix_process(q, n, t, n_threads, xbase, a.in_dtype, a.S, *a.tables, a.status);
+    if (n > 0) fix_process(q, n, t, n_threads, a.K, a.V, a.in_dtype, a.S, *a.tables, a.status);
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
     if (t == 0) q->count = 0;
-    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
+    const bool more = bar_or(bar_id, n_threads, leftbits != 0ull);
+    if (!more) break;
+    if (leftbits != 0ull && tb != nullptr) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const uint32_t bits = (uint32_t)(leftbits >> (15 * i)) & 0x7FFFu;
+        if (bits) {
+          uint32_t left;
+          fix_push(q, bits, xoff, tb, tok, 4 * half + i, kv, &left);
+          leftbits = (leftbits & ~(0x7FFFull << (15 * i))) | ((unsigned long long)left << (15 * i));
+        }
+      }
+    }
   }
 }
 
@@ -306,7 +326,16 @@ __global__ void __launch_bounds__(kFfmaThreads) encode_ffma_kernel(EncodeArgs a)
   int tok = 0;
   quantise_and_store(a, *fq, uniform, y, row_norm, row0 + r, head, kv, half, row0 + r < a.total_tokens, fixq, left, &xoff,
                      &tb, &tok);
-  fixup_rounds(a, fixq, left, xoff, tb, tok, half, kv, tid, kFfmaThreads, 1);
+  unsigned long long leftbits = 0ull;
+  if (tb != nullptr) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      uint32_t rest = 0;
+      if (left[i]) fix_push(fixq, left[i], xoff, tb, tok, 4 * half + i, kv, &rest);
+      leftbits |= (unsigned long long)rest << (15 * i);
+    }
+  }
+  fix_rounds(a, fixq, leftbits, xoff, tb, tok, half, kv, tid, kFfmaThreads, 1);
 }
 
 }  // namespace pq

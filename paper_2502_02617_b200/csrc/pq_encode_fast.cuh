@@ -24,45 +24,45 @@ struct FastQuant {
 
 __device__ inline void load_fast_quant(const Tables* tb, FastQuant* fq) {
   for (int l = 0; l < 3; ++l)
-    for (int k = 0; k < 3; ++k) {
-      const double t = tb->bnd_sin[15 + 3 * l + k] / tb->bnd_cos[15 + 3 * l + k];
-      fq->t2[l][k] = (float)(t * t);
-    }
+    for (int k = 0; k < 3; ++k) fq->t2[l][k] = (float)tb->bnd_tan2[3 * l + k];
 }
 
 // Level >= 2 decision on squared child radii (sa: cosine side, sb: sine side).
 //   code = #{k : sb > T_k sa},  T_k = tan^2(beta_k)  (both sides of r_b cos b > r_a sin b are >= 0).
 // Margin: the radii are norms of n-coordinate sub-vectors, so they move by at most E = sqrt(n) * dy.
 // With D = sb - T sa, |D - D_exact| <= 2E(r_b + T r_a) + E^2 (1 + T) + rho (sb + T sa), and
-// (2E(r_b + T r_a))^2 <= 8 E^2 (sb + T^2 sa), (p+q+z)^2 <= 3(p^2+q^2+z^2), so the decision is
-// certified if D^2 > 24 E^2 (sb + T^2 sa) + 3 E^4 (1+T)^2 + 3 rho^2 (sb + T sa)^2 for every k; the
-// right side grows with T, so the largest T is used with the smallest |D|.
+// (2E(r_b + T r_a))^2 <= 8 E^2 (sb + T^2 sa), (p+q+z)^2 <= 3(p^2+q^2+z^2), so boundary k is
+// certified if D_k^2 > 24 E^2 (sb + T_k^2 sa) + 3 E^4 (1+T_k)^2 + 3 rho^2 (sb + T_k sa)^2.  The last
+// two terms use the largest T (they are tiny; it only saves instructions).
 __device__ __forceinline__ uint32_t quant_upper_fast(float sa, float sb, const float* T, float e2 /* E^2 */,
                                                      bool* ambiguous) {
   const float d0 = fmaf(-T[0], sa, sb), d1 = fmaf(-T[1], sa, sb), d2 = fmaf(-T[2], sa, sb);
   const uint32_t code = (d0 > 0.f) + (d1 > 0.f) + (d2 > 0.f);
-  const float dm = fminf(fminf(fabsf(d0), fabsf(d1)), fabsf(d2));
   const float tm = T[2];
-  const float w = fmaf(tm * tm, sa, sb);
   const float u = fmaf(tm, sa, sb);
-  float rhs = fmaf(24.f * e2, w, 3.f * e2 * e2 * (1.f + tm) * (1.f + tm));
-  rhs = fmaf(3e-12f * u, u, rhs);  // rho = 1e-6 covers float32 rounding of the squares and products
-  *ambiguous = !(dm * dm > rhs);   // also true for NaN
+  const float base = fmaf(3e-12f * u, u, 3.f * e2 * e2 * (1.f + tm) * (1.f + tm));  // rho = 1e-6: float32 roundings
+  const float c = 24.f * e2;
+  const bool ok0 = d0 * d0 > fmaf(c, fmaf(T[0] * T[0], sa, sb), base);
+  const bool ok1 = d1 * d1 > fmaf(c, fmaf(T[1] * T[1], sa, sb), base);
+  const bool ok2 = d2 * d2 > fmaf(c, fmaf(T[2] * T[2], sa, sb), base);
+  *ambiguous = !(ok0 && ok1 && ok2);  // also true for NaN
   return code;
 }
 
 // Level-1 decision for the uniform codebook (boundaries k pi/8): fold into the first octant,
 // u = max(|a|,|b|), v = min(|a|,|b|); the boundaries are the axes (v = 0), the diagonals (u = v) and
-// the lines at pi/8 from the axes (v cos(pi/8) = u sin(pi/8)).  The point moves by at most
-// sqrt(2) dy, so the decision is certified if its distance to all three exceeds that.
-__device__ __forceinline__ uint32_t quant_level1_fast(float a, float b, float e1 /* sqrt(2) dy */, bool* ambiguous) {
+// the lines at pi/8 from the axes (v cos(pi/8) = u sin(pi/8)).  Each coordinate moves by at most
+// dy, so the signed distance to a line with unit normal (n1, n2) moves by at most (|n1| + |n2|) dy:
+// dy for an axis, sqrt(2) dy for a diagonal, (cos + sin)(pi/8) dy = 1.3066 dy for the pi/8 lines.
+// The three distances are scaled so that one comparison against dy serves all.
+__device__ __forceinline__ uint32_t quant_level1_fast(float a, float b, float dy, bool* ambiguous) {
   const float ax = fabsf(a), ay = fabsf(b);
   const float u = fmaxf(ax, ay), v = fminf(ax, ay);
   const bool swap = ay > ax;
   const float t = fmaf(v, 0.92387953251128674f, -u * 0.38268343236508977f);  // v cos(pi/8) - u sin(pi/8)
   const bool hi = t > 0.f;
-  const float dmin = fminf(fminf(v, (u - v) * 0.70710678118654752f), fabsf(t));
-  *ambiguous = !(dmin > fmaf(u, 4.76837158203125e-07f, e1));  // + 2^-21 u for the float32 roundings
+  const float dmin = fminf(fminf(v, (u - v) * 0.5f), fabsf(t) * 0.76536686473017954f);
+  *ambiguous = !(dmin > fmaf(u, 4.76837158203125e-07f, dy));  // + 2^-21 u for the float32 roundings
   const uint32_t sector = swap ? (hi ? 2u : 3u) : (hi ? 1u : 0u);  // pi/8 sector inside the quadrant
   const uint32_t sa = __float_as_uint(a) >> 31, sb = __float_as_uint(b) >> 31;
   // b >= 0: theta = phi or pi - phi; b < 0: theta = pi + phi or 2 pi - phi
@@ -77,13 +77,12 @@ struct FastBlock {
 };
 
 __device__ __forceinline__ void polar_quant_block_fast(const float* y, float dy, const FastQuant& fq, FastBlock* out) {
-  const float e1 = 1.41421356f * dy;
   float s1[8], s2[4], s3[2];
   uint32_t l1 = 0, l2 = 0, l3 = 0, amb = 0;
   bool am;
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    l1 |= quant_level1_fast(y[2 * j], y[2 * j + 1], e1, &am) << (4 * j);
+    l1 |= quant_level1_fast(y[2 * j], y[2 * j + 1], dy, &am) << (4 * j);
     amb |= (am ? 1u : 0u) << j;
     s1[j] = fmaf(y[2 * j], y[2 * j], y[2 * j + 1] * y[2 * j + 1]);
   }
@@ -122,7 +121,7 @@ struct FixQueue {
   int pad[3];
   int64_t xoff[kFixCap];   // element offset of the source vector
   uint8_t* tok[kFixCap];   // token-block base of the destination
-  uint32_t meta[kFixCap];  // token-in-block | blk << 6 | level << 9 | j << 12
+  uint32_t meta[kFixCap];  // token-in-block | blk << 6 | level << 9 | j << 12 | (1 = value, 0 = key) << 15
 };
 
 // Replace `width` bits at bit offset `bit` of the byte at `addr`.
@@ -134,7 +133,7 @@ __device__ __forceinline__ void patch_bits(uint8_t* addr, int bit, uint32_t mask
 }
 
 __device__ __forceinline__ void fix_push(FixQueue* q, uint32_t amb, int64_t xoff, uint8_t* tokblock, int tok, int blk,
-                                         uint32_t* left) {
+                                         int kv, uint32_t* left) {
   while (amb) {
     const int bit = __ffs(amb) - 1;
     const int idx = atomicAdd(&q->count, 1);
@@ -147,79 +146,106 @@ __device__ __forceinline__ void fix_push(FixQueue* q, uint32_t amb, int64_t xoff
     else { level = 4; j = 0; }
     q->xoff[idx] = xoff;
     q->tok[idx] = tokblock;
-    q->meta[idx] = (uint32_t)tok | ((uint32_t)blk << 6) | ((uint32_t)level << 9) | ((uint32_t)j << 12);
+    q->meta[idx] = (uint32_t)tok | ((uint32_t)blk << 6) | ((uint32_t)level << 9) | ((uint32_t)j << 12) | ((uint32_t)kv << 15);
   }
   *left = amb;
 }
 
-// Process queue entries [0, n): called by `n_threads` threads (a multiple of 32) with linear index `t`.
-__device__ inline void fix_process(const FixQueue* q, int n, int t, int n_threads, const void* xbase, int in_dtype,
-                                   const float* S, const Tables& tb, int32_t* status) {
-  constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock;
-  const int sub = t & 7, group = t >> 3, n_groups = n_threads >> 3;
-  const int rounds = (n + n_groups - 1) / n_groups;
-  int fixed = 0;
-  for (int rd = 0; rd < rounds; ++rd) {
-    const int e = rd * n_groups + group;
-    const bool active = e < n;
-    const uint32_t meta = active ? q->meta[e] : (1u << 9);
-    const int64_t xoff = active ? q->xoff[e] : 0;
-    const int tok = meta & 63, blk = (meta >> 6) & 7, level = (meta >> 9) & 7, j = (meta >> 12) & 7;
-    const int nc = 1 << level, c0 = blk * 16 + j * nc;
-    // this lane's 16 consecutive k
-    double xk[16];
-    if (active) {
-      if (in_dtype == PQ_DTYPE_BF16) {
-        const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(xbase) + xoff + 16 * sub);
-        const uint4 v0 = p[0], v1 = p[1];
-        const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+// Exact value of NC consecutive rotated coordinates starting at column c0, for the 8-lane group of
+// this lane: each lane owns 16 consecutive k, NC independent float64 chains, then a 3-step
+// butterfly inside the group.  Every lane of the group returns all NC sums.
+template <int NC>
+__device__ __forceinline__ void exact_coords(const double* xk, const float* S, int sub, int c0, unsigned gmask, double* y) {
+  double acc[NC];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          xk[2 * i] = (double)__uint_as_float(w[i] << 16);
-          xk[2 * i + 1] = (double)__uint_as_float(w[i] & 0xFFFF0000u);
-        }
-      } else {
-        const float* p = reinterpret_cast<const float*>(xbase) + xoff + 16 * sub;
+  for (int c = 0; c < NC; ++c) acc[c] = 0.0;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) xk[i] = (double)p[i];
-      }
+  for (int i = 0; i < 16; ++i) {
+    const float* srow = S + (16 * sub + i) * 128 + c0;
+    if (NC == 2) {
+      const float2 s2 = __ldg(reinterpret_cast<const float2*>(srow));
+      acc[0] = fma(xk[i], (double)s2.x, acc[0]);
+      acc[1] = fma(xk[i], (double)s2.y, acc[1]);
     } else {
 #pragma unroll
-      for (int i = 0; i < 16; ++i) xk[i] = 0.0;
+      for (int c4 = 0; c4 < NC / 4; ++c4) {
+        const float4 s4 = __ldg(reinterpret_cast<const float4*>(srow) + c4);
+        acc[4 * c4] = fma(xk[i], (double)s4.x, acc[4 * c4]);
+        acc[4 * c4 + 1] = fma(xk[i], (double)s4.y, acc[4 * c4 + 1]);
+        acc[4 * c4 + 2] = fma(xk[i], (double)s4.z, acc[4 * c4 + 2]);
+        acc[4 * c4 + 3] = fma(xk[i], (double)s4.w, acc[4 * c4 + 3]);
+      }
     }
-    int nmax = nc;  // every lane of the warp runs the same number of coordinate steps
-    nmax = max(nmax, __shfl_xor_sync(0xffffffffu, nmax, 8));
-    nmax = max(nmax, __shfl_xor_sync(0xffffffffu, nmax, 16));
+  }
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    double p = acc[c];
+    p += __shfl_xor_sync(gmask, p, 1);
+    p += __shfl_xor_sync(gmask, p, 2);
+    p += __shfl_xor_sync(gmask, p, 4);
+    y[c] = p;
+  }
+}
+
+// Decision of one angle of level log2(NC) from the exact coordinates under it.  Levels >= 2 compare
+// the squared child radii, sb > tan^2(beta) sa, which is the same decision as atan2(r_b, r_a) > beta.
+template <int NC>
+__device__ __forceinline__ uint32_t exact_code(const double* y, int level, const Tables& tb) {
+  if (NC == 2) return quant_level1_exact(y[0], y[1], tb);
+  double sa = 0.0, sb = 0.0;
+#pragma unroll
+  for (int c = 0; c < NC / 2; ++c) {
+    sa = fma(y[c], y[c], sa);
+    sb = fma(y[NC / 2 + c], y[NC / 2 + c], sb);
+  }
+  const double* T = tb.bnd_tan2 + 3 * (level - 2);
+  return (uint32_t)(sb > T[0] * sa) + (uint32_t)(sb > T[1] * sa) + (uint32_t)(sb > T[2] * sa);
+}
+
+// Process queue entries [0, n): called by `n_threads` threads (a multiple of 32) with linear index `t`.
+__device__ inline void fix_process(const FixQueue* q, int n, int t, int n_threads, const void* kbase, const void* vbase,
+                                   int in_dtype, const float* S, const Tables& tb, int32_t* status) {
+  constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock;
+  const int sub = t & 7, n_groups = n_threads >> 3;
+  const unsigned gmask = 0xFFu << (t & 24);
+  int fixed = 0;
+  for (int e = t >> 3; e < n; e += n_groups) {  // uniform within a group of 8 lanes
+    const uint32_t meta = q->meta[e];
+    const int64_t xoff = q->xoff[e];
+    const int tok = meta & 63, blk = (meta >> 6) & 7, level = (meta >> 9) & 7, j = (meta >> 12) & 7;
+    const int c0 = blk * 16 + (j << level);
+    const void* xbase = (meta >> 15) & 1 ? vbase : kbase;
+    double xk[16];  // this lane's 16 consecutive k
+    if (in_dtype == PQ_DTYPE_BF16) {
+      const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(xbase) + xoff + 16 * sub);
+      const uint4 v0 = p[0], v1 = p[1];
+      const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        xk[2 * i] = (double)__uint_as_float(w[i] << 16);
+        xk[2 * i + 1] = (double)__uint_as_float(w[i] & 0xFFFF0000u);
+      }
+    } else {
+      const float* p = reinterpret_cast<const float*>(xbase) + xoff + 16 * sub;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) xk[i] = (double)p[i];
+    }
     double y[16];
-#pragma unroll
-    for (int c = 0; c < 16; ++c) {
-      if (c < nmax) {
-        const int col = c0 + min(c, nc - 1);
-        const float* sp = S + (16 * sub) * 128 + col;
-        double p = 0.0;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) p = fma(xk[i], (double)__ldg(sp + i * 128), p);
-        p += __shfl_xor_sync(0xffffffffu, p, 1);
-        p += __shfl_xor_sync(0xffffffffu, p, 2);
-        p += __shfl_xor_sync(0xffffffffu, p, 4);
-        y[c] = p;
-      } else {
-        y[c] = 0.0;
-      }
+    uint32_t code;
+    if (level == 1) {
+      exact_coords<2>(xk, S, sub, c0, gmask, y);
+      code = exact_code<2>(y, level, tb);
+    } else if (level == 2) {
+      exact_coords<4>(xk, S, sub, c0, gmask, y);
+      code = exact_code<4>(y, level, tb);
+    } else if (level == 3) {
+      exact_coords<8>(xk, S, sub, c0, gmask, y);
+      code = exact_code<8>(y, level, tb);
+    } else {
+      exact_coords<16>(xk, S, sub, c0, gmask, y);
+      code = exact_code<16>(y, level, tb);
     }
-    if (active && sub == 0) {
-      uint32_t code;
-      if (level == 1) {
-        code = quant_level1_exact(y[0], y[1], tb);
-      } else {
-        // child radii by the same pairwise hypot recursion as Polar
-#pragma unroll
-        for (int m = 16; m > 2; m >>= 1)
-          if (m <= nc)
-#pragma unroll
-            for (int c = 0; c < m / 2; ++c) y[c] = hypot(y[2 * c], y[2 * c + 1]);
-        code = quant_upper_exact(y[0], y[1], level, tb);
-      }
+    if (sub == 0) {
       uint8_t* tbk = q->tok[e];
       if (level == 1) patch_bits(tbk + tok * 32 + blk * 4 + (j >> 1), 4 * (j & 1), 0xFu, code);
       else if (level == 2) patch_bits(tbk + o2 + tok * 8 + blk, 2 * j, 3u, code);

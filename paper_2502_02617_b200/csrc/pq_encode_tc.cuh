@@ -203,11 +203,13 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     }
   } else {
     // ------------------------------------------------------------------ epilogue (8 warps)
+    constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock, orad = o4 + 2 * kTokenBlock;
     const int et = tid - 64;                       // 0..255
     const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
     const int half = (warp - 2) >> 2;              // columns [64*half, 64*half + 64)
     const int r = quarter * 32 + lane;             // row of the tile
     const bool uniform = (a.tables->flags & kFlagUniformL1) != 0u;
+    const Layout L = make_layout(128, a.capacity);
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
       const int acc = it & 1;
@@ -215,34 +217,79 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
       // A wait that gives up must not leave the loop: the other epilogue warps may be past it and
       // would wait for this one at the named barriers.  The tile is skipped instead (warp-uniform).
       const bool ready = __all_sync(0xffffffffu, tc_mbar_wait(bar_tfull + 8 * acc, (it >> 1) & 1, abort_flag));
-      float y[64];
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 128 + half * 64;
+      // pass 1: squared norm of the row (its two halves are exchanged through shared memory)
+      float sq = 0.f;
       if (ready) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 128 + half * 64;
+#pragma unroll 1
+        for (int i = 0; i < 4; ++i) {
+          float y[16];
+          tc_ld16(taddr + 16 * i, y);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-        for (int i = 0; i < 4; ++i) tc_ld16(taddr + 16 * i, y + 16 * i);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          for (int c = 0; c < 16; ++c) sq = fmaf(y[c], y[c], sq);
+        }
+      }
+      rowsq[half * 128 + r] = sq;
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      const float dy = kRotErr * 1.0001f * sqrtf(rowsq[r] + rowsq[128 + r]);
+      const int row = rt * 128 + r;
+      uint8_t* tb = nullptr;
+      int tok = 0;
+      if (ready && row < a.total_tokens) {
+        int seq, pos;
+        row_destination(a, row, &seq, &pos);
+        if (pos >= 0) {
+          tb = a.cache + block_offset(L, a.n_kv_heads, seq, head, kv, pos);
+          tok = pos % kTokenBlock;
+        }
+      }
+      const int64_t xoff = (int64_t)row * a.token_stride + (int64_t)head * a.head_stride;
+      // pass 2: one block at a time
+      uint32_t l2acc = 0, l3acc = 0, l4acc = 0, sat = 0;
+      unsigned long long racc = 0ull, leftbits = 0ull;
+      if (ready) {
+#pragma unroll 1
+        for (int i = 0; i < 4; ++i) {
+          float y[16];
+          tc_ld16(taddr + 16 * i, y);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          FastBlock fb;
+          polar_quant_block_fast(y, dy, *fq, &fb);
+          if (!uniform) fb.amb |= 0xFFu;  // other level-1 codebooks: decide every level-1 angle exactly
+          if (tb != nullptr) {
+            *reinterpret_cast<uint32_t*>(tb + tok * 32 + half * 16 + 4 * i) = fb.l1;
+            l2acc |= fb.l2 << (8 * i);
+            l3acc |= fb.l3 << (4 * i);
+            l4acc |= fb.l4 << (2 * i);
+            float rv = fb.radius;
+            if (rv > 65504.f) { rv = 65504.f; ++sat; }
+            racc |= (unsigned long long)__half_as_ushort(__float2half_rn(rv)) << (16 * i);
+            if (fb.amb) {
+              uint32_t left;
+              fix_push(fixq, fb.amb, xoff, tb, tok, 4 * half + i, kv, &left);
+              leftbits |= (unsigned long long)left << (15 * i);  // queue full: pushed again by fix_rounds
+            }
+          }
+        }
         asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         __syncwarp();
         if (lane == 0) tc_mbar_arrive(bar_tempty + 8 * acc);  // this accumulator may be overwritten
-      } else {
-#pragma unroll
-        for (int i = 0; i < 64; ++i) y[i] = 0.f;
       }
-      float sq = 0.f;
-#pragma unroll
-      for (int i = 0; i < 64; ++i) sq = fmaf(y[i], y[i], sq);
-      rowsq[half * 128 + r] = sq;
+      if (tb != nullptr) {
+        *reinterpret_cast<uint32_t*>(tb + o2 + tok * 8 + half * 4) = l2acc;
+        *reinterpret_cast<uint16_t*>(tb + o3 + tok * 4 + half * 2) = (uint16_t)l3acc;
+        tb[o4 + tok * 2 + half] = (uint8_t)l4acc;
+        *reinterpret_cast<unsigned long long*>(tb + orad + tok * 16 + half * 8) = racc;
+        if (sat) atomicAdd(a.status + 2, (int)sat);
+      }
+      // Exact re-decisions are batched over tiles: drain the queue when it is half full (a push that
+      // did not fit leaves the counter above the capacity) or after the CTA's last tile.
       asm volatile("bar.sync 1, 256;" ::: "memory");
-      const float row_norm = sqrtf(rowsq[r] + rowsq[128 + r]) * 1.0001f;
-      uint32_t left[4];
-      int64_t xoff = 0;
-      uint8_t* tb = nullptr;
-      int tok = 0;
-      const int row = rt * 128 + r;
-      quantise_and_store(a, *fq, uniform, y, row_norm, row, head, kv, half, ready && row < a.total_tokens, fixq, left,
-                         &xoff, &tb, &tok);
-      fixup_rounds(a, fixq, left, xoff, tb, tok, half, kv, et, kTcEpiThreads, 1);
+      const bool last_tile = tile + (int)gridDim.x >= n_tiles;
+      if (fixq->count > kFixCap / 2 || last_tile)
+        fix_rounds(a, fixq, leftbits, xoff, tb, tok, half, kv, et, kTcEpiThreads, 1);
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");

@@ -176,6 +176,10 @@ int32_t pq_build_tables(const double* cen, const double* bnd, void* tables_host)
     t.bnd_cosf[k] = (float)t.bnd_cos[k];
     t.bnd_sinf[k] = (float)t.bnd_sin[k];
   }
+  for (int k = 0; k < 9; ++k) {
+    const double tn = std::tan(bnd[15 + k]);
+    t.bnd_tan2[k] = tn * tn;
+  }
   for (int k = 0; k < 15; ++k) {
     t.bnd_upper[k] = bnd[k] <= kPi ? 1 : 0;
     t.n_upper += t.bnd_upper[k];
