@@ -347,11 +347,9 @@ def run_cuda(args):
 
     if rank != 0:
         return
-    traffic = None
-    tpath = os.path.join(ROOT, "profiles", "decode_attention_traffic.json")
-    if os.path.exists(tpath):
-        with open(tpath) as f:
-            traffic = json.load(f).get("dram_bytes_per_launch_config3")
+    # DRAM bytes of one decode-attention launch: ncu capture at batch 4 (profiles/decode_attention_fast_kernel_
+    # batch4_ctx32768.md: 130.48 MB read + 4.78 MB written), scaled by the batch (traffic is proportional to it)
+    traffic = (130.48e6 + 4.78e6) * BATCH / 4.0
     cpu = _oracle_sample_throughput(12.0) if world == 1 and not args.no_cpu_baseline else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
