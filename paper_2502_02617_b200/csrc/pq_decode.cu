@@ -69,38 +69,23 @@ __device__ inline float decode_coord(const uint8_t* tb, const Layout& L, int tok
 }
 
 // ---- workspace -----------------------------------------------------------------------------
+constexpr int kFastMaxGridHost = 160;  // upper bound on the persistent kernel's grid (one CTA per SM)
+
 struct Workspace {
   float* qrot;       // [B][Hq][d]      rotated queries times scale*log2(e)
   __half* qrot_h;    // the same rounded to fp16 (tensor-core operand of the fast kernel)
   __half* qrot_l;    // fp16 residual: qrot - qrot_h
   int32_t* tickets;  // [B][Hkv]
-  float* ml;         // [B][Hq][splits][2]
-  float* o;          // [B][Hq][splits][d]
-  int n_splits;
+  float* ml;         // [slot][head in group][2]   slot = first slot of the unit + part
+  float* o;          // [slot][head in group][d]
+  int n_splits;      // parts per unit of the any-head_dim kernel (the head_dim-128 kernel decides on the device)
+  int n_slots;
   int64_t bytes;
 };
 
-// Token splits per (sequence, kv head).  The head_dim-128 kernel runs one CTA per SM and works
-// in 128-token stages: pick the split count with the smallest estimated makespan
-// (waves x (stages per CTA + fixed cost)).
+// Token splits per (sequence, kv head) for the any-head_dim kernel.
 __host__ inline int choose_splits(int d, int batch, int n_kv_heads, int max_len) {
   const int units = batch * n_kv_heads;
-  if (d == 128) {
-    const int nst = (max_len + 127) / 128;
-    int best = 1;
-    double best_cost = 1e30;
-    for (int s = 1; s <= 128 && s <= nst; ++s) {
-      const int per = (nst + s - 1) / s;
-      const long ctas = (long)units * s;
-      const long waves = (ctas + 147) / 148;
-      const double cost = (double)waves * (per + 1.5);
-      if (cost < best_cost - 1e-9) {
-        best_cost = cost;
-        best = s;
-      }
-    }
-    return best;
-  }
   const int max_blocks = (max_len + kTokenBlock - 1) / kTokenBlock;
   int splits = (148 * 4 + units - 1) / units;
   if (splits > max_blocks) splits = max_blocks;
@@ -123,10 +108,12 @@ __host__ inline Workspace carve_workspace(void* base, int d, int batch, int n_q_
   off = align(off + (int64_t)batch * n_q_heads * d * 2);
   w.tickets = reinterpret_cast<int32_t*>(p + off);
   off = align(off + (int64_t)batch * n_kv_heads * 4);
+  const int g = n_q_heads / n_kv_heads, units = batch * n_kv_heads;
+  w.n_slots = (d == 128 && units <= 2048) ? units + kFastMaxGridHost : units * w.n_splits;
   w.ml = reinterpret_cast<float*>(p + off);
-  off = align(off + (int64_t)batch * n_q_heads * w.n_splits * 2 * 4);
+  off = align(off + (int64_t)w.n_slots * g * 2 * 4);
   w.o = reinterpret_cast<float*>(p + off);
-  off = align(off + (int64_t)batch * n_q_heads * w.n_splits * d * 4);
+  off = align(off + (int64_t)w.n_slots * g * d * 4);
   w.bytes = off;
   return w;
 }
@@ -167,35 +154,36 @@ __global__ void rotate_query_kernel(DecodeArgs a) {
 constexpr int kSimpleThreads = 128;
 
 // Shared memory (floats) that combine_and_store needs.
-__host__ __device__ inline int combine_smem_floats(int g, int d, int n_splits) { return g * n_splits + g + g * d; }
+__host__ __device__ inline int combine_smem_floats(int g, int d, int n_parts) { return g * n_parts + g + g * d; }
 
-// Merge the split partials of the `g` query heads of (b, kv head) in split order, normalise,
-// rotate back by S^T and store.  Runs in the last CTA that finishes for this (b, kv head); `sm`
-// must hold combine_smem_floats(...) floats.
-__device__ void combine_and_store(const DecodeArgs& a, int b, int hk, int g, float* sm) {
-  const int d = a.d, ns = a.ws.n_splits, tid = threadIdx.x, nthr = blockDim.x;
+// Merge the `ns` partials (slots slot0 .. slot0 + ns - 1) of the `g` query heads of (b, kv head) in slot
+// order, normalise, rotate back by S^T and store.  Runs in the last CTA that finishes for this
+// (b, kv head); `sm` must hold combine_smem_floats(g, d, ns) floats.
+__device__ void combine_and_store(const DecodeArgs& a, int b, int hk, int g, int slot0, int ns, float* sm) {
+  const int d = a.d, tid = threadIdx.x, nthr = blockDim.x;
   float* w_sm = sm;               // [g][ns] weight of split s for head h
   float* linv_sm = sm + g * ns;   // [g]
   float* o_sm = linv_sm + g;      // [g][d]
   const int64_t h0 = (int64_t)b * a.n_q_heads + hk * g;
   if (tid < g) {
-    const float* ml = a.ws.ml + (h0 + tid) * ns * 2;
+    const float* ml = a.ws.ml + ((int64_t)slot0 * g + tid) * 2;  // part s at ml[s * g * 2]
     float M = -CUDART_INF_F;
-    for (int s = 0; s < ns; ++s) M = fmaxf(M, ml[2 * s]);
+    for (int s = 0; s < ns; ++s) M = fmaxf(M, ml[(int64_t)s * g * 2]);
     float Lsum = 0.f;
     for (int s = 0; s < ns; ++s) {
-      const float w = ml[2 * s] == -CUDART_INF_F ? 0.f : exp2f(ml[2 * s] - M);
+      const float ms = ml[(int64_t)s * g * 2];
+      const float w = ms == -CUDART_INF_F ? 0.f : exp2f(ms - M);
       w_sm[tid * ns + s] = w;
-      Lsum += ml[2 * s + 1] * w;
+      Lsum += ml[(int64_t)s * g * 2 + 1] * w;
     }
     linv_sm[tid] = Lsum > 0.f ? 1.f / Lsum : 0.f;
   }
   __syncthreads();
   for (int idx = tid; idx < g * d; idx += nthr) {
     const int h = idx / d, j = idx - h * d;
-    const float* op = a.ws.o + (h0 + h) * ns * d + j;
+    const float* op = a.ws.o + ((int64_t)slot0 * g + h) * d + j;
     float acc = 0.f;
-    for (int s = 0; s < ns; ++s) acc = fmaf(op[(int64_t)s * d], w_sm[h * ns + s], acc);
+    for (int s = 0; s < ns; ++s) acc = fmaf(op[(int64_t)s * g * d], w_sm[h * ns + s], acc);
     o_sm[idx] = acc * linv_sm[h];
   }
   __syncthreads();
@@ -349,8 +337,9 @@ __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel
   }
 
   // partials of this split
+  const int slot0 = (b * a.n_kv_heads + hk) * a.ws.n_splits;
   for (int h = 0; h < g; ++h) {
-    const int64_t idx = ((int64_t)b * a.n_q_heads + hk * g + h) * a.ws.n_splits + split;
+    const int64_t idx = (int64_t)(slot0 + split) * g + h;
     if (tid == 0) {
       a.ws.ml[2 * idx] = m_run[h];
       a.ws.ml[2 * idx + 1] = l_run[h];
@@ -367,7 +356,7 @@ __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel
   __syncthreads();
   if (is_last) {
     __threadfence();
-    combine_and_store(a, b, hk, g, reinterpret_cast<float*>(smem));
+    combine_and_store(a, b, hk, g, slot0, a.ws.n_splits, reinterpret_cast<float*>(smem));
   }
 }
 
@@ -474,7 +463,7 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
   a.ws = pq::carve_workspace(workspace_dev, head_dim, batch, n_q_heads, n_kv_heads, max_len);
   const int g = n_q_heads / n_kv_heads;
   pq::rotate_query_kernel<<<batch * n_q_heads, head_dim, head_dim * sizeof(float), st>>>(a);
-  if (head_dim == 128) {
+  if (head_dim == 128 && batch * n_kv_heads <= pq::kFastMaxUnits) {
     static bool configured = false;
     if (!configured) {
       const cudaError_t e = cudaFuncSetAttribute(pq::decode_attention_fast_kernel,
@@ -485,7 +474,17 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
       }
       configured = true;
     }
-    dim3 grid(a.ws.n_splits, n_kv_heads, batch);
+    static int n_sm = 0;
+    if (n_sm == 0) {
+      int dev = 0;
+      cudaError_t e = cudaGetDevice(&dev);
+      if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+      if (e != cudaSuccess) {
+        pq::note_cuda_error(e);
+        return PQ_ERR_CUDA;
+      }
+    }
+    const int grid = n_sm < pq::kFastMaxGrid ? n_sm : pq::kFastMaxGrid;
     pq::decode_attention_fast_kernel<<<grid, pq::kFastThreads, pq::kSmTotal, st>>>(a);
     return pq::launch_status();
   }

@@ -39,8 +39,9 @@ constexpr int kSmT1p = 0;                             // 256 * 16 * 8 = 32768
 constexpr int kSmT1lo = kSmT1p + 256 * 16 * 8;        // 32768
 constexpr int kSmU = kSmT1lo + 256 * 16 * 8;          // 4 * 64 * 16 * 8 = 32768
 constexpr int kSmBar = kSmU + 4 * 64 * 16 * 8;        // full[4], empty[4] : 64
-constexpr int kSmFlags = kSmBar + 64;                 // abort flag, is_last : 16
-constexpr int kSmRing = (kSmFlags + 16 + 127) / 128 * 128;
+constexpr int kSmFlags = kSmBar + 64;                 // abort flag, is_last, n_segs : 16
+constexpr int kSmSegs = kSmFlags + 16;                // Segment[32] : 768
+constexpr int kSmRing = (kSmSegs + 768 + 127) / 128 * 128;
 // after the main loop the ring is reused for the cross-warp merge: 16 warps x 8 heads x (128 + 2) floats
 constexpr int kMergeBytes = 16 * 8 * 128 * 4 + 16 * 8 * 2 * 4;  // also >= combine_smem_floats(8, 128, 128) * 4
 constexpr int kSmTotal = kSmRing + (kStages * kStageBytes > kMergeBytes ? kStages * kStageBytes : kMergeBytes);
@@ -199,22 +200,23 @@ __device__ inline void build_fast_tables(uint8_t* smem, const Tables* tb) {
   for (int i = tid; i < 4 * 64 * 16; i += blockDim.x) u[i] = tb->u_tab[i >> 10][(i >> 4) & 63];
 }
 
+// Slots of split partials for the persistent kernel: every unit (sequence, kv head) has one slot
+// per CTA that works on it; the slots of all units sum to at most units + grid size.
+constexpr int kFastMaxGrid = 160;
+constexpr int kFastMaxUnits = 2048;  // (sequence, kv head) units the persistent schedule handles
+constexpr int kFastMaxSegs = 32;     // units one CTA can take part in (<= units / grid + 2)
+struct Segment {
+  int unit, st0, st1, part, n_parts, slot0;
+};
+
 __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int g_heads = a.n_q_heads / a.n_kv_heads;
-  const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t sm_base = smem_u32(smem);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kSmFlags);
   int* is_last = reinterpret_cast<int*>(smem + kSmFlags) + 1;
-
-  const int len = a.lens[b];
-  const int nst_total = len > 0 ? (len + kStageTokens - 1) / kStageTokens : 0;
-  const int nblk_total = len > 0 ? (len + kTokenBlock - 1) / kTokenBlock : 0;
-  const int per = (nst_total + a.ws.n_splits - 1) / a.ws.n_splits;
-  const int st0 = split * per;
-  const int st1 = min(nst_total, st0 + per);
-  const uint8_t* head_base = a.cache + ((int64_t)b * a.n_kv_heads + hk) * make_layout(128, a.capacity).head_bytes;
+  const int64_t head_bytes = make_layout(128, a.capacity).head_bytes;
 
   build_fast_tables(smem, a.tables);
   if (tid == 0) {
@@ -227,32 +229,104 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
   }
   __syncthreads();
 
-  // per-thread attention state (consumer warps)
+  // ---- persistent work split: the 128-token stages of all units, in unit order, are cut into
+  // gridDim.x equal contiguous ranges; a CTA's range may cover the end of one unit and the start of
+  // the next, and a unit may be shared by several CTAs (its "parts").  Each thread works out one
+  // unit; the units this CTA takes part in are collected in a short list.
+  const int n_units = a.batch * a.n_kv_heads, G = gridDim.x, cta = blockIdx.x;
+  int* u_nst = reinterpret_cast<int*>(smem + kSmRing);  // [n_units] stages; the ring is idle during set-up
+  int* u_parts = u_nst + kFastMaxUnits;                 // [n_units] CTAs that share the unit
+  Segment* segs = reinterpret_cast<Segment*>(smem + kSmSegs);
+  int* n_segs = reinterpret_cast<int*>(smem + kSmFlags) + 2;
+  if (tid == 0) *n_segs = 0;
+  for (int u = tid; u < n_units; u += kFastThreads) {
+    const int len_u = a.lens[u / a.n_kv_heads];
+    u_nst[u] = len_u > 0 ? (len_u + kStageTokens - 1) / kStageTokens : 0;
+  }
+  __syncthreads();
+  long long w_total = 0;
+  for (int u = 0; u < n_units; ++u) w_total += u_nst[u];
+  const long long lo = cta * w_total / G, hi = (cta + 1) * w_total / G;
+  for (int u = tid; u < n_units; u += kFastThreads) {
+    int parts = 0;
+    if (u_nst[u] > 0) {
+      long long start = 0;
+      for (int v = 0; v < u; ++v) start += u_nst[v];
+      const long long end = start + u_nst[u];
+      const int c_first = (int)(((start + 1) * G + w_total - 1) / w_total) - 1;  // CTA whose range holds stage `start`
+      const int c_last = (int)((end * G + w_total - 1) / w_total) - 1;           // ... stage `end - 1`
+      parts = c_last - c_first + 1;
+      if (cta >= c_first && cta <= c_last) {
+        const int i = atomicAdd(n_segs, 1);
+        if (i < kFastMaxSegs) {
+          segs[i].unit = u;
+          segs[i].st0 = (int)((lo > start ? lo : start) - start);
+          segs[i].st1 = (int)((hi < end ? hi : end) - start);  // may equal st0: a neutral partial is written
+          segs[i].part = cta - c_first;
+          segs[i].n_parts = parts;
+        }
+      }
+    } else if (cta == 0) {  // empty sequence: zeros, and the status says so
+      const int b = u / a.n_kv_heads, hk = u - b * a.n_kv_heads;
+      for (int i = 0; i < g_heads * 128; ++i) {
+        const int64_t idx = ((int64_t)b * a.n_q_heads + hk * g_heads) * 128 + i;
+        if (a.io_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[idx] = __float2bfloat16(0.f);
+        else reinterpret_cast<float*>(a.out)[idx] = 0.f;
+      }
+      set_status(a.status, PQ_ERR_EMPTY);
+    }
+    u_parts[u] = parts;
+  }
+  __syncthreads();
+  if (*n_segs > kFastMaxSegs) {  // cannot happen for n_units <= kFastMaxUnits; never index past the list
+    if (tid == 0) set_status(a.status, PQ_ERR_UNSUPPORTED);
+    return;
+  }
+  for (int i = tid; i < *n_segs; i += kFastThreads) {  // first partial slot of the unit
+    int slot = 0;
+    for (int v = 0; v < segs[i].unit; ++v) slot += u_parts[v];
+    segs[i].slot0 = slot;
+  }
+  __syncthreads();
+  const int my_segs = *n_segs;
   const int g = lane >> 2, c = lane & 3;
-  float o_acc[8][4];  // tile i (pair i of block g): rows 2i / 2i+1 of block g, heads 2c / 2c+1
-#pragma unroll
-  for (int i = 0; i < 8; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
-  float m_run = -CUDART_INF_F, l_run = 0.f;  // of head g (replicated over the 4 lanes of a quad)
+  const uint32_t rep = (lane & 15) * 8;
+  // logical token n of a tile (MMA column n) is physical token (n >> 1) + 4 * (n & 1)
+  const int ktok = (g >> 1) + 4 * (g & 1);  // token whose keys this thread decodes
+  int it0 = 0;  // stages this CTA has streamed so far (ring slot and barrier phase bookkeeping)
 
-  // Copy of iteration `it` (stage st0 + it) into ring slot it % kStages; waits (bounded) until all
-  // 16 warps have released the slot's previous contents.  Called by thread 0 only.
-  int issued = 0;
-  auto issue_copy = [&](int it) -> bool {
-    const int s = it % kStages;
-    if (it >= kStages && !mbar_wait(sm_base + kSmBar + 8 * (kStages + s), ((it / kStages) - 1) & 1, abort_flag))
-      return false;
-    const int st = st0 + it;
-    const int nblk = min(2, nblk_total - 2 * st);
-    const uint32_t bytes = nblk * 2 * kBlockBytes128;
-    mbar_expect_tx(sm_base + kSmBar + 8 * s, bytes);
-    bulk_load(sm_base + kSmRing + s * kStageBytes, head_base + (int64_t)st * kStageBytes, bytes, sm_base + kSmBar + 8 * s);
-    issued = it + 1;
-    return true;
-  };
-  if (tid == 0)
-    for (int it = 0; it < kStages - 1 && st0 + it < st1; ++it) issue_copy(it);
-  __syncwarp();
-  {
+  for (int sg = 0; sg < my_segs; ++sg) {
+    const int u = segs[sg].unit, st0 = segs[sg].st0, st1 = segs[sg].st1;
+    const int n_parts = segs[sg].n_parts, unit_slot = segs[sg].slot0, c_first = cta - segs[sg].part;
+    const int b = u / a.n_kv_heads, hk = u - b * a.n_kv_heads;
+    const int len = a.lens[b];
+    const int nblk_total = (len + kTokenBlock - 1) / kTokenBlock;
+    const uint8_t* head_base = a.cache + ((int64_t)b * a.n_kv_heads + hk) * head_bytes;
+
+    // per-thread attention state
+    float o_acc[8][4];  // tile i (pair i of block g): rows 2i / 2i+1 of block g, heads 2c / 2c+1
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
+    float m_run = -CUDART_INF_F, l_run = 0.f;  // of head g (replicated over the 4 lanes of a quad)
+
+    // Copy of this segment's iteration `it` (stage st0 + it) into ring slot (it0 + it) % kStages; waits
+    // (bounded) until all 16 warps have released the slot's previous contents.  Thread 0 only.
+    int issued = 0;
+    auto issue_copy = [&](int it) -> bool {
+      const int gi = it0 + it, s = gi % kStages;
+      if (gi >= kStages && !mbar_wait(sm_base + kSmBar + 8 * (kStages + s), ((gi / kStages) - 1) & 1, abort_flag))
+        return false;
+      const int st = st0 + it;
+      const int nblk = min(2, nblk_total - 2 * st);
+      const uint32_t bytes = nblk * 2 * kBlockBytes128;
+      mbar_expect_tx(sm_base + kSmBar + 8 * s, bytes);
+      bulk_load(sm_base + kSmRing + s * kStageBytes, head_base + (int64_t)st * kStageBytes, bytes, sm_base + kSmBar + 8 * s);
+      issued = it + 1;
+      return true;
+    };
+    if (tid == 0)
+      for (int it = 0; it < kStages - 1 && st0 + it < st1; ++it) issue_copy(it);
+    __syncwarp();
     // ---------------------------------------------------------------- consumers
     // q' fragments: A operand (16 heads x 16 coords per k-step); rows >= 8 are zero.
     // k-step ks covers, for thread c, sub-block (ks & 3) of block 2c + (ks >> 2).
@@ -272,14 +346,11 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
         ql[ks][1] = w.y;
       }
     }
-    const uint32_t rep = (lane & 15) * 8;
-    // logical token n of a tile (MMA column n) is physical token (n >> 1) + 4 * (n & 1)
-    const int ktok = (g >> 1) + 4 * (g & 1);  // token whose keys this thread decodes
     for (int st = st0, it = 0; st < st1; ++st, ++it) {
-      const int s = it % kStages;
+      const int gi = it0 + it, s = gi % kStages;
       if (tid == 0 && st + kStages - 1 < st1) issue_copy(it + kStages - 1);
       __syncwarp();
-      if (!mbar_wait(sm_base + kSmBar + 8 * s, (it / kStages) & 1, abort_flag)) break;
+      if (!mbar_wait(sm_base + kSmBar + 8 * s, (gi / kStages) & 1, abort_flag)) break;
       const int tile_tok0 = st * kStageTokens + warp * 8;  // first token of this warp's tile
       if (tile_tok0 < len) {
         const uint32_t kblk = sm_base + kSmRing + s * kStageBytes + (warp >> 3) * 2 * kBlockBytes128;
@@ -370,19 +441,18 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
       __syncwarp();
       if (lane == 0) mbar_arrive(sm_base + kSmBar + 8 * (kStages + s));
     }
-  }
-  if (tid == 0 && *abort_flag) {
-    // gave up: let the copies still in flight land (bounded) before the ring is reused
-    for (int it = max(0, issued - kStages); it < issued; ++it)
-      for (int i = 0; i < kSpinLimit && !mbar_try_wait(sm_base + kSmBar + 8 * (it % kStages), (it / kStages) & 1); ++i)
-        __nanosleep(64);
-  }
-  __syncthreads();  // every copy that was issued has been consumed (or the CTA aborted)
+    if (tid == 0 && *abort_flag) {
+      // gave up: let the copies still in flight land (bounded) before the ring is reused
+      for (int it = max(0, issued - kStages); it < issued; ++it)
+        for (int i = 0; i < kSpinLimit && !mbar_try_wait(sm_base + kSmBar + 8 * ((it0 + it) % kStages), ((it0 + it) / kStages) & 1); ++i)
+          __nanosleep(64);
+    }
+    it0 += st1 - st0;
+    __syncthreads();  // every copy that was issued has been consumed (or the CTA aborted)
 
-  // ---- merge the 16 warps (fixed order), write this split's partial, last CTA combines
-  float* mrg_o = reinterpret_cast<float*>(smem + kSmRing);      // [16 warps][8 heads][128]
-  float* mrg_ml = mrg_o + kFastConsumerWarps * 8 * 128;         // [16 warps][8 heads][2]
-  {
+    // ---- merge the 16 warps (fixed order), write this part's partial, last part combines the unit
+    float* mrg_o = reinterpret_cast<float*>(smem + kSmRing);      // [16 warps][8 heads][128]
+    float* mrg_ml = mrg_o + kFastConsumerWarps * 8 * 128;         // [16 warps][8 heads][2]
     if (c == 0) {
       mrg_ml[(warp * 8 + g) * 2] = m_run;
       mrg_ml[(warp * 8 + g) * 2 + 1] = l_run;
@@ -396,41 +466,42 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
       o0[1] = o_acc[i][2];
       o1[1] = o_acc[i][3];
     }
-  }
-  __syncthreads();
-  for (int idx = tid; idx < g_heads * 128; idx += kFastThreads) {
-    const int h = idx >> 7, j = idx & 127;
-    float M = -CUDART_INF_F;
+    __syncthreads();
+    const int slot = unit_slot + (cta - c_first);
+    for (int idx = tid; idx < g_heads * 128; idx += kFastThreads) {
+      const int h = idx >> 7, j = idx & 127;
+      float M = -CUDART_INF_F;
 #pragma unroll
-    for (int w = 0; w < kFastConsumerWarps; ++w) M = fmaxf(M, mrg_ml[(w * 8 + h) * 2]);
-    float lsum = 0.f, acc = 0.f;
+      for (int w = 0; w < kFastConsumerWarps; ++w) M = fmaxf(M, mrg_ml[(w * 8 + h) * 2]);
+      float lsum = 0.f, acc = 0.f;
 #pragma unroll
-    for (int w = 0; w < kFastConsumerWarps; ++w) {
-      const float mw = mrg_ml[(w * 8 + h) * 2];
-      const float wgt = mw == -CUDART_INF_F ? 0.f : exp2f(mw - M);
-      lsum += mrg_ml[(w * 8 + h) * 2 + 1] * wgt;
-      acc += mrg_o[(w * 8 + h) * 128 + j] * wgt;
+      for (int w = 0; w < kFastConsumerWarps; ++w) {
+        const float mw = mrg_ml[(w * 8 + h) * 2];
+        const float wgt = mw == -CUDART_INF_F ? 0.f : exp2f(mw - M);
+        lsum += mrg_ml[(w * 8 + h) * 2 + 1] * wgt;
+        acc += mrg_o[(w * 8 + h) * 128 + j] * wgt;
+      }
+      const int64_t pidx = (int64_t)slot * g_heads + h;
+      a.ws.o[pidx * 128 + j] = acc;
+      if (j == 0) {
+        a.ws.ml[2 * pidx] = M;
+        a.ws.ml[2 * pidx + 1] = lsum;
+      }
     }
-    const int64_t pidx = ((int64_t)b * a.n_q_heads + hk * g_heads + h) * a.ws.n_splits + split;
-    a.ws.o[pidx * 128 + j] = acc;
-    if (j == 0) {
-      a.ws.ml[2 * pidx] = M;
-      a.ws.ml[2 * pidx + 1] = lsum;
-    }
-  }
-  __threadfence();
-  __syncthreads();
-  if (tid == 0) {
-    if (*abort_flag) set_status(a.status, PQ_ERR_TIMEOUT);
-    const int t = atomicAdd(a.ws.tickets + b * a.n_kv_heads + hk, 1);
-    *is_last = (t == a.ws.n_splits - 1);
-    if (*is_last && len <= 0) set_status(a.status, PQ_ERR_EMPTY);
-  }
-  __syncthreads();
-  if (*is_last) {
     __threadfence();
-    combine_and_store(a, b, hk, g_heads, reinterpret_cast<float*>(smem + kSmRing));
+    __syncthreads();
+    if (tid == 0) {
+      const int t = atomicAdd(a.ws.tickets + u, 1);
+      *is_last = (t == n_parts - 1);
+    }
+    __syncthreads();
+    if (*is_last) {
+      __threadfence();
+      combine_and_store(a, b, hk, g_heads, unit_slot, n_parts, reinterpret_cast<float*>(smem + kSmRing));
+    }
+    __syncthreads();  // the ring is free again for the next unit
   }
+  if (tid == 0 && *abort_flag) set_status(a.status, PQ_ERR_TIMEOUT);
 }
 
 }  // namespace pq

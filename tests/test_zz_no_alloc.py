@@ -40,7 +40,7 @@ def test_static_scratch_entry_matches_workspace_entry_twice_in_a_row(d, Hq, Hkv,
 
 
 def test_static_scratch_entry_rejects_oversized_problems_without_launching():
-    d, Hq, Hkv, B, ctx = 128, 32, 8, 64, 1 << 20
+    d, Hq, Hkv, B, ctx = 128, 64, 8, 256, 1 << 20
     assert pq.pq_workspace_bytes(d, B, Hq, Hkv, ctx) > pq.pq_static_scratch_bytes()
     dummy = torch.zeros(64, dtype=torch.int32, device=DEV)
     q = torch.zeros((B, Hq, d), dtype=torch.bfloat16, device=DEV)
