@@ -142,7 +142,8 @@ __global__ void rotate_query_kernel(DecodeArgs a) {
   else qs[j] = reinterpret_cast<const float*>(a.q)[base + j];
   __syncthreads();
   float acc = 0.f;
-  for (int k = 0; k < d; ++k) acc = fmaf(qs[k], a.S[k * d + j], acc);
+#pragma unroll 16
+  for (int k = 0; k < d; ++k) acc = fmaf(qs[k], __ldg(a.S + k * d + j), acc);
   acc *= a.scale * 1.4426950408889634f;
   a.ws.qrot[base + j] = acc;
   const __half qh = __float2half_rn(acc);

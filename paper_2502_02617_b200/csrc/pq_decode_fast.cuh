@@ -43,7 +43,8 @@ constexpr int kSmFlags = kSmBar + 64;                 // abort flag, is_last, n_
 constexpr int kSmSegs = kSmFlags + 16;                // Segment[32] : 768
 constexpr int kSmRing = (kSmSegs + 768 + 127) / 128 * 128;
 // after the main loop the ring is reused for the cross-warp merge: 16 warps x 8 heads x (128 + 2) floats
-constexpr int kMergeBytes = 16 * 8 * 128 * 4 + 16 * 8 * 2 * 4;  // also >= combine_smem_floats(8, 128, 128) * 4
+constexpr int kMrgStride = 132;  // floats per (warp, head) row of the merge buffer (132 = 128 + 4: bank spread)
+constexpr int kMergeBytes = 16 * 8 * kMrgStride * 4 + 16 * 8 * 2 * 4;  // also >= combine_smem_floats(8, 128, 160) * 4
 constexpr int kSmTotal = kSmRing + (kStages * kStageBytes > kMergeBytes ? kStages * kStageBytes : kMergeBytes);
 static_assert(kSmRing % 128 == 0, "ring must be 128-byte aligned");
 
@@ -186,18 +187,29 @@ __device__ __forceinline__ void decode_block_hilo(uint32_t l1, uint32_t c2, uint
 constexpr int kO2 = 32 * kTokenBlock, kO3 = kO2 + 8 * kTokenBlock, kO4 = kO3 + 4 * kTokenBlock,
               kORad = kO4 + 2 * kTokenBlock;
 
-// Build the replicated shared-memory tables from `Tables`.
+// Build the replicated shared-memory tables from `Tables`: entry e goes to 16 consecutive slots.
+// All loads are issued before the stores so that their latencies overlap.
 __device__ inline void build_fast_tables(uint8_t* smem, const Tables* tb) {
   const int tid = threadIdx.x;
+  static_assert(kFastThreads == 512, "table fill assumes 512 threads");
+  uint2 v[24];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    const int e = (tid + r * kFastThreads) >> 4;  // 0..255
+    v[r] = tb->t1p_hi[e];
+    v[8 + r] = tb->t1p_lo[e];
+    v[16 + r] = tb->u_tab[e >> 6][e & 63];
+  }
   uint2* t1hi = reinterpret_cast<uint2*>(smem + kSmT1p);
   uint2* t1lo = reinterpret_cast<uint2*>(smem + kSmT1lo);
-  for (int i = tid; i < 256 * 16; i += blockDim.x) {
-    const int e = i >> 4;  // entry; replica = i & 15
-    t1hi[i] = make_uint2(tb->l1_hi[e & 15], tb->l1_hi[e >> 4]);
-    t1lo[i] = make_uint2(tb->l1_lo[e & 15], tb->l1_lo[e >> 4]);
-  }
   uint2* u = reinterpret_cast<uint2*>(smem + kSmU);
-  for (int i = tid; i < 4 * 64 * 16; i += blockDim.x) u[i] = tb->u_tab[i >> 10][(i >> 4) & 63];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    const int i = tid + r * kFastThreads;
+    t1hi[i] = v[r];
+    t1lo[i] = v[8 + r];
+    u[i] = v[16 + r];
+  }
 }
 
 // Slots of split partials for the persistent kernel: every unit (sequence, kv head) has one slot
@@ -451,20 +463,24 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     __syncthreads();  // every copy that was issued has been consumed (or the CTA aborted)
 
     // ---- merge the 16 warps (fixed order), write this part's partial, last part combines the unit
-    float* mrg_o = reinterpret_cast<float*>(smem + kSmRing);      // [16 warps][8 heads][128]
-    float* mrg_ml = mrg_o + kFastConsumerWarps * 8 * 128;         // [16 warps][8 heads][2]
+    // Coordinate j of head h of warp w sits at (w * 8 + h) * kMrgStride + (j & 15) * 8 + (j >> 4): for a fixed
+    // accumulator register the 32 lanes (block g, head pair c) then hit 32 different banks.
+    float* mrg_o = reinterpret_cast<float*>(smem + kSmRing);          // [16 warps][8 heads][kMrgStride]
+    float* mrg_ml = mrg_o + kFastConsumerWarps * 8 * kMrgStride;      // [16 warps][8 heads][2]
     if (c == 0) {
       mrg_ml[(warp * 8 + g) * 2] = m_run;
       mrg_ml[(warp * 8 + g) * 2 + 1] = l_run;
     }
+    if (2 * c < g_heads) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      float* o0 = mrg_o + (warp * 8 + 2 * c) * 128 + 16 * g + 2 * i;
-      float* o1 = o0 + 128;
-      o0[0] = o_acc[i][0];
-      o1[0] = o_acc[i][1];
-      o0[1] = o_acc[i][2];
-      o1[1] = o_acc[i][3];
+      for (int i = 0; i < 8; ++i) {
+        float* o0 = mrg_o + (warp * 8 + 2 * c) * kMrgStride + (2 * i) * 8 + g;
+        float* o1 = o0 + kMrgStride;
+        o0[0] = o_acc[i][0];
+        o1[0] = o_acc[i][1];
+        o0[8] = o_acc[i][2];
+        o1[8] = o_acc[i][3];
+      }
     }
     __syncthreads();
     const int slot = unit_slot + (cta - c_first);
@@ -479,7 +495,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
         const float mw = mrg_ml[(w * 8 + h) * 2];
         const float wgt = mw == -CUDART_INF_F ? 0.f : exp2f(mw - M);
         lsum += mrg_ml[(w * 8 + h) * 2 + 1] * wgt;
-        acc += mrg_o[(w * 8 + h) * 128 + j] * wgt;
+        acc += mrg_o[(w * 8 + h) * kMrgStride + (j & 15) * 8 + (j >> 4)] * wgt;
       }
       const int64_t pidx = (int64_t)slot * g_heads + h;
       a.ws.o[pidx * 128 + j] = acc;

@@ -203,6 +203,10 @@ int32_t pq_build_tables(const double* cen, const double* bnd, void* tables_host)
     *lo = h2(va - ha, vb - hb);
   };
   for (int c = 0; c < 16; ++c) split(std::cos(cen[c]), std::sin(cen[c]), &t.l1_hi[c], &t.l1_lo[c]);
+  for (int e = 0; e < 256; ++e) {
+    t.t1p_hi[e] = make_uint2(t.l1_hi[e & 15], t.l1_hi[e >> 4]);
+    t.t1p_lo[e] = make_uint2(t.l1_lo[e & 15], t.l1_lo[e >> 4]);
+  }
   for (int s = 0; s < 4; ++s)
     for (int i = 0; i < 64; ++i) {
       const double a2 = cen[16 + (i & 3)], a3 = cen[20 + ((i >> 2) & 3)], a4 = cen[24 + (i >> 4)];
