@@ -338,6 +338,87 @@ __global__ void __launch_bounds__(kFfmaThreads) encode_ffma_kernel(EncodeArgs a)
   fix_rounds(a, fixq, leftbits, xoff, tb, tok, half, kv, tid, kFfmaThreads, 1);
 }
 
+// ------------------------------------------------------------------------------------------
+// Few vectors (append, short chunks), head_dim 128: one CTA of 128 threads per vector.  Thread j
+// forms y_j in float32; eight threads quantise one block each with the certified sign tests; if
+// any decision of the vector is ambiguous the CTA forms y again in float64 and those blocks are
+// decided exactly.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) encode_vector_kernel(EncodeArgs a) {
+  __shared__ float xs[128];
+  __shared__ float ys[128];
+  __shared__ double yd[128];
+  __shared__ float red[4];
+  __shared__ FastQuant fq;
+  const int j = threadIdx.x;
+  const int64_t v = blockIdx.x;  // vector index: (row * 2 + kv) * n_kv_heads + head
+  const int head = (int)(v % a.n_kv_heads), kv = (int)((v / a.n_kv_heads) & 1);
+  const int row = (int)(v / (2 * a.n_kv_heads));
+  const int64_t xoff = (int64_t)row * a.token_stride + (int64_t)head * a.head_stride;
+  const float xv = load_elem(kv ? a.V : a.K, a.in_dtype, xoff + j);
+  if (!isfinite(xv)) {
+    atomicAdd(a.status + 1, 1);
+    set_status(a.status, PQ_ERR_NONFINITE);
+  }
+  xs[j] = xv;
+  if (j == 0) load_fast_quant(a.tables, &fq);
+  __syncthreads();
+  float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 8
+  for (int k = 0; k < 128; k += 4) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) acc[i] = fmaf(xs[k + i], __ldg(a.S + (k + i) * 128 + j), acc[i]);
+  }
+  const float y = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+  ys[j] = y;
+  float sq = y * y;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+  if ((j & 31) == 0) red[j >> 5] = sq;
+  __syncthreads();
+  // four independent partial sums instead of one chain: the bound of a 128-term float32 dot product still holds
+  const float dy = kRotErr * 1.0001f * sqrtf((red[0] + red[1]) + (red[2] + red[3]));
+  FastBlock fb = {0u, 0u, 0u, 0u, 0u, 0.f};
+  if (j < 8) {
+    float yb[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) yb[i] = ys[16 * j + i];
+    polar_quant_block_fast(yb, dy, fq, &fb);
+    if ((a.tables->flags & kFlagUniformL1) == 0u) fb.amb |= 0xFFu;
+  }
+  if (__syncthreads_or(fb.amb != 0u)) {
+    double accd[4] = {0.0, 0.0, 0.0, 0.0};
+    for (int k = 0; k < 128; k += 4) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) accd[i] = fma((double)xs[k + i], (double)__ldg(a.S + (k + i) * 128 + j), accd[i]);
+    }
+    yd[j] = (accd[0] + accd[1]) + (accd[2] + accd[3]);
+    __syncthreads();
+    if (j < 8 && fb.amb != 0u) {
+      double yb[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) yb[i] = yd[16 * j + i];
+      BlockCodes c;
+      fb.radius = (float)polar_quant_block_exact(yb, *a.tables, c);
+      fb.l1 = c.l1; fb.l2 = c.l2; fb.l3 = c.l3; fb.l4 = c.l4;
+      atomicAdd(a.status + 3, __popc(fb.amb));
+    }
+  }
+  if (j >= 32) return;  // the first warp stores (lanes 0..7 hold the blocks)
+  int seq = 0, pos = -1;
+  if (j < 8) row_destination(a, row, &seq, &pos);
+  const bool valid = j < 8 && pos >= 0;
+  float rv = fb.radius;
+  if (valid && rv > 65504.f) {
+    rv = 65504.f;
+    atomicAdd(a.status + 2, 1);
+  }
+  const Layout L = make_layout(128, a.capacity);
+  BlockCodes c = {fb.l1, fb.l2, fb.l3, fb.l4};
+  uint8_t* tb = a.cache + (valid ? block_offset(L, a.n_kv_heads, seq, head, kv, pos) : 0);
+  store_block(tb, L, valid ? pos % kTokenBlock : 0, j & 7, c, __float2half_rn(rv), valid);
+}
+
 }  // namespace pq
 #include "pq_encode_tc.cuh"
 namespace pq {
@@ -370,6 +451,12 @@ static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
       advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, lens);
       return launch_status();
     }
+  }
+  if (a.head_dim == 128 && a.total_tokens < 32) {
+    const int64_t n_vec = (int64_t)a.total_tokens * 2 * a.n_kv_heads;
+    encode_vector_kernel<<<(unsigned)n_vec, 128, 0, stream>>>(a);
+    advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, lens);
+    return launch_status();
   }
   if (a.head_dim == 128 && a.total_tokens >= 32) {
     static bool configured = false;
