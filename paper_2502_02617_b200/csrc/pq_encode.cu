@@ -205,11 +205,11 @@ __device__ __forceinline__ void quantise_and_store(const EncodeArgs& a, const Fa
                                                    float row_norm, int row, int head, int kv, int half, bool valid,
                                                    FixQueue* q, uint32_t* left, int64_t* xoff_out, uint8_t** tb_out,
                                                    int* tok_out) {
-  const float dy = kRotErr * row_norm;
+  const RowMargins rm = make_row_margins(kRotErr * row_norm, fq);
   FastBlock fb[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    polar_quant_block_fast(y + 16 * i, dy, fq, &fb[i]);
+    polar_quant_block_fast(y + 16 * i, rm, fq, &fb[i]);
     if (!uniform_l1) fb[i].amb |= 0xFFu;  // other level-1 codebooks: decide every level-1 angle exactly
     left[i] = 0u;
   }
@@ -244,9 +244,10 @@ __device__ __forceinline__ bool bar_or(int bar_id, int n_threads, bool v) {
 
 // Drain the queue of ambiguous decisions: rounds of (barrier, process, barrier, reset, push what did
 // not fit before).  All `n_threads` threads of named barrier `bar_id` call this together.
-// `leftbits` holds this thread's decisions that found the queue full (15 bits per block, 4 blocks).
+// `leftbits` holds this thread's decisions that found the queue full (15 bits per block, up to 4 blocks
+// starting at block `blk0`).
 __device__ inline void fix_rounds(const EncodeArgs& a, FixQueue* q, unsigned long long leftbits, int64_t xoff, uint8_t* tb,
-                                  int tok, int half, int kv, int t, int n_threads, int bar_id) {
+                                  int tok, int blk0, int kv, int t, int n_threads, int bar_id) {
   for (int round = 0; round < 256; ++round) {
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
     const int n = min(q->count, kFixCap);
@@ -261,7 +262,7 @@ __device__ inline void fix_rounds(const EncodeArgs& a, FixQueue* q, unsigned lon
         const uint32_t bits = (uint32_t)(leftbits >> (15 * i)) & 0x7FFFu;
         if (bits) {
           uint32_t left;
-          fix_push(q, bits, xoff, tb, tok, 4 * half + i, kv, &left);
+          fix_push(q, bits, xoff, tb, tok, blk0 + i, kv, &left);
           leftbits = (leftbits & ~(0x7FFFull << (15 * i))) | ((unsigned long long)left << (15 * i));
         }
       }
@@ -335,7 +336,7 @@ __global__ void __launch_bounds__(kFfmaThreads) encode_ffma_kernel(EncodeArgs a)
       leftbits |= (unsigned long long)rest << (15 * i);
     }
   }
-  fix_rounds(a, fixq, leftbits, xoff, tb, tok, half, kv, tid, kFfmaThreads, 1);
+  fix_rounds(a, fixq, leftbits, xoff, tb, tok, 4 * half, kv, tid, kFfmaThreads, 1);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -383,7 +384,7 @@ __global__ void __launch_bounds__(128) encode_vector_kernel(EncodeArgs a) {
     float yb[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) yb[i] = ys[16 * j + i];
-    polar_quant_block_fast(yb, dy, fq, &fb);
+    polar_quant_block_fast(yb, make_row_margins(dy, fq), fq, &fb);
     if ((a.tables->flags & kFlagUniformL1) == 0u) fb.amb |= 0xFFu;
   }
   if (__syncthreads_or(fb.amb != 0u)) {

@@ -27,26 +27,52 @@ __device__ inline void load_fast_quant(const Tables* tb, FastQuant* fq) {
     for (int k = 0; k < 3; ++k) fq->t2[l][k] = (float)tb->bnd_tan2[3 * l + k];
 }
 
+// Per-row constants of the margins (dy = bound on the error of one rotated coordinate of the row).
+struct RowMargins {
+  float dy;
+  float c[3];     // 8.4 E^2 for levels 2, 3, 4 (E^2 = 2, 4, 8 dy^2)
+  float base[3];  // 42 E^4 (1 + T_max)^2
+};
+__device__ __forceinline__ RowMargins make_row_margins(float dy, const FastQuant& fq) {
+  RowMargins m;
+  m.dy = dy;
+  const float e2 = dy * dy;
+#pragma unroll
+  for (int l = 0; l < 3; ++l) {
+    const float el = (float)(2 << l) * e2, t1 = 1.f + fq.t2[l][2];
+    m.c[l] = 8.4f * el;
+    m.base[l] = 42.f * el * el * t1 * t1;
+  }
+  return m;
+}
+
 // Level >= 2 decision on squared child radii (sa: cosine side, sb: sine side).
 //   code = #{k : sb > T_k sa},  T_k = tan^2(beta_k)  (both sides of r_b cos b > r_a sin b are >= 0).
 // Margin: the radii are norms of n-coordinate sub-vectors, so they move by at most E = sqrt(n) * dy.
 // With D = sb - T sa, |D - D_exact| <= 2E(r_b + T r_a) + E^2 (1 + T) + rho (sb + T sa), and
-// (2E(r_b + T r_a))^2 <= 8 E^2 (sb + T^2 sa), (p+q+z)^2 <= 3(p^2+q^2+z^2), so boundary k is
-// certified if D_k^2 > 24 E^2 (sb + T_k^2 sa) + 3 E^4 (1+T_k)^2 + 3 rho^2 (sb + T_k sa)^2.  The last
-// two terms use the largest T (they are tiny; it only saves instructions).
-__device__ __forceinline__ uint32_t quant_upper_fast(float sa, float sb, const float* T, float e2 /* E^2 */,
+// (2E(r_b + T r_a))^2 <= 8 E^2 (sb + T^2 sa); with (p+q+z)^2 <= 1.05 p^2 + 21 (q+z)^2 <= 1.05 p^2 + 42 (q^2+z^2)
+// boundary k is certified if D_k^2 > 8.4 E^2 (sb + T_k^2 sa) + 42 E^4 (1+T_k)^2 + 42 rho^2 (sb + T_k sa)^2.
+// A cheap test with the largest T for every k (T_max > 1, so sb + T_max^2 sa bounds both sums)
+// certifies almost all decisions; only its failures run the per-boundary test.
+__device__ __forceinline__ uint32_t quant_upper_fast(float sa, float sb, const float* T, float c, float base,
                                                      bool* ambiguous) {
   const float d0 = fmaf(-T[0], sa, sb), d1 = fmaf(-T[1], sa, sb), d2 = fmaf(-T[2], sa, sb);
-  const uint32_t code = (d0 > 0.f) + (d1 > 0.f) + (d2 > 0.f);
-  const float tm = T[2];
-  const float u = fmaf(tm, sa, sb);
-  const float base = fmaf(3e-12f * u, u, 3.f * e2 * e2 * (1.f + tm) * (1.f + tm));  // rho = 1e-6: float32 roundings
-  const float c = 24.f * e2;
-  const bool ok0 = d0 * d0 > fmaf(c, fmaf(T[0] * T[0], sa, sb), base);
-  const bool ok1 = d1 * d1 > fmaf(c, fmaf(T[1] * T[1], sa, sb), base);
-  const bool ok2 = d2 * d2 > fmaf(c, fmaf(T[2] * T[2], sa, sb), base);
-  *ambiguous = !(ok0 && ok1 && ok2);  // also true for NaN
-  return code;
+  // d0 >= d1 >= d2: the code is the number of positive ones (a zero is ambiguous and decided exactly)
+  const uint32_t neg = (__float_as_uint(d0) >> 31) + (__float_as_uint(d1) >> 31) + (__float_as_uint(d2) >> 31);
+  const float dm = fminf(fminf(fabsf(d0), fabsf(d1)), fabsf(d2));
+  const float w = fmaf(T[2] * T[2], sa, sb);
+  const float rhs = fmaf(4.2e-11f * w, w, fmaf(c, w, base));  // rho = 1e-6 covers the float32 roundings
+  bool amb = !(dm * dm > rhs);  // also true for NaN
+  if (amb) {
+    const float u = fmaf(T[2], sa, sb);
+    const float b2 = fmaf(4.2e-11f * u, u, base);
+    const bool ok0 = d0 * d0 > fmaf(c, fmaf(T[0] * T[0], sa, sb), b2);
+    const bool ok1 = d1 * d1 > fmaf(c, fmaf(T[1] * T[1], sa, sb), b2);
+    const bool ok2 = d2 * d2 > fmaf(c, w, b2);
+    amb = !(ok0 && ok1 && ok2);
+  }
+  *ambiguous = amb;
+  return 3u - neg;
 }
 
 // Level-1 decision for the uniform codebook (boundaries k pi/8): fold into the first octant,
@@ -76,36 +102,42 @@ struct FastBlock {
   float radius;
 };
 
-__device__ __forceinline__ void polar_quant_block_fast(const float* y, float dy, const FastQuant& fq, FastBlock* out) {
+__device__ __forceinline__ float fast_sqrt(float x) {
+  float r;
+  asm("sqrt.approx.f32 %0, %1;" : "=f"(r) : "f"(x));  // 1 ulp-level error: far inside the fp16 rounding of the radius
+  return r;
+}
+
+__device__ __forceinline__ void polar_quant_block_fast(const float* y, const RowMargins& rm, const FastQuant& fq,
+                                                       FastBlock* out) {
   float s1[8], s2[4], s3[2];
   uint32_t l1 = 0, l2 = 0, l3 = 0, amb = 0;
   bool am;
 #pragma unroll
   for (int j = 0; j < 8; ++j) {
-    l1 |= quant_level1_fast(y[2 * j], y[2 * j + 1], dy, &am) << (4 * j);
+    l1 |= quant_level1_fast(y[2 * j], y[2 * j + 1], rm.dy, &am) << (4 * j);
     amb |= (am ? 1u : 0u) << j;
     s1[j] = fmaf(y[2 * j], y[2 * j], y[2 * j + 1] * y[2 * j + 1]);
   }
-  const float e2 = dy * dy;
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    l2 |= quant_upper_fast(s1[2 * j], s1[2 * j + 1], fq.t2[0], 2.f * e2, &am) << (2 * j);
+    l2 |= quant_upper_fast(s1[2 * j], s1[2 * j + 1], fq.t2[0], rm.c[0], rm.base[0], &am) << (2 * j);
     amb |= (am ? 1u : 0u) << (8 + j);
     s2[j] = s1[2 * j] + s1[2 * j + 1];
   }
 #pragma unroll
   for (int j = 0; j < 2; ++j) {
-    l3 |= quant_upper_fast(s2[2 * j], s2[2 * j + 1], fq.t2[1], 4.f * e2, &am) << (2 * j);
+    l3 |= quant_upper_fast(s2[2 * j], s2[2 * j + 1], fq.t2[1], rm.c[1], rm.base[1], &am) << (2 * j);
     amb |= (am ? 1u : 0u) << (12 + j);
     s3[j] = s2[2 * j] + s2[2 * j + 1];
   }
-  out->l4 = quant_upper_fast(s3[0], s3[1], fq.t2[2], 8.f * e2, &am);
+  out->l4 = quant_upper_fast(s3[0], s3[1], fq.t2[2], rm.c[2], rm.base[2], &am);
   amb |= (am ? 1u : 0u) << 14;
   out->l1 = l1;
   out->l2 = l2;
   out->l3 = l3;
   out->amb = amb;
-  out->radius = sqrtf(s3[0] + s3[1]);
+  out->radius = fast_sqrt(s3[0] + s3[1]);
 }
 
 // ---- exact re-decision of the ambiguous angles ------------------------------------------------
@@ -114,7 +146,7 @@ __device__ __forceinline__ void polar_quant_block_fast(const float* y, float dy,
 // the original inputs (x in its storage type, S in float32: both exact in float64), decide again
 // and patch the code bits in the cache with 32-bit atomics.  The queue is drained in rounds, so a
 // tile with more ambiguous angles than the queue holds only takes more rounds.
-constexpr int kFixCap = 512;
+constexpr int kFixCap = 1024;
 
 struct FixQueue {
   int count;

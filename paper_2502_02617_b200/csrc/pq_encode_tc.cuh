@@ -1,31 +1,35 @@
 // Tensor-core encoder for head_dim 128, bf16 inputs (included by pq_encode.cu).
 //
-// Persistent CTAs (one per SM) loop over tiles of 128 rows x one (K|V, head).  Per tile
-//   warp 0   (one lane): TMA loads of the x tile (two 64-column boxes, 128-byte swizzle) into a ring;
-//   warp 1   (one lane): y = x . S on the 5th-generation tensor cores: S is split once per CTA into
-//            two bf16 terms (S = S_hi + S_lo + O(2^-17)) kept in shared memory as the K-major B
-//            operand; 2 terms x 8 k-steps of tcgen05.mma (M = 128 rows, N = 128, K = 16) accumulate
-//            in float32 in tensor memory; two accumulators let the next tile's MMAs overlap the
-//            current tile's epilogue;
-//   warps 2-9: epilogue.  Tensor-memory lane = row, so a thread owns 64 consecutive rotated
-//            coordinates (4 blocks) of one row: tcgen05.ld, sign-test quantiser with certified
-//            margins, packed stores, queued float64 re-decision of the ambiguous angles.
-// Every mbarrier wait is bounded; a wait that gives up raises the CTA's abort flag, all roles leave
-// their loops, tensor memory is released and PQ_ERR_TIMEOUT is recorded.
+// Persistent CTAs (one per SM, 16 warps) loop over tiles of 128 rows x one (K|V, head).  Per tile
+//   * TMA loads of the x tile (two 64-column boxes, 128-byte swizzle) into a 3-deep ring, issued by
+//     one thread two tiles ahead;
+//   * y = x . S on the 5th-generation tensor cores: S is split once per CTA into two bf16 terms
+//     (S = S_hi + S_lo + O(2^-17)) kept in shared memory as the K-major B operand; 2 terms x 8
+//     k-steps of tcgen05.mma (M = 128 rows, N = 128, K = 16) accumulate in float32 in tensor memory;
+//     two accumulators, and the MMAs of tile i+1 are issued (by one thread) when the epilogue of
+//     tile i starts, so they run under it;
+//   * epilogue on all 16 warps.  Tensor-memory lane = row, so a thread owns 32 consecutive rotated
+//     coordinates (2 blocks) of one row: tcgen05.ld, sign-test quantiser with certified margins,
+//     packed stores, queued float64 re-decision of the ambiguous angles.
+// There are no dedicated producer / MMA warps: the register file is split over four schedulers, and
+// a 17th warp would cap every thread at 96 registers (the quantiser then spills).  The issuing
+// threads do not block in practice: what they wait for was completed a tile earlier.
+// Every mbarrier wait is bounded; a wait that gives up raises the CTA's abort flag, the remaining
+// tiles are skipped, tensor memory is released and PQ_ERR_TIMEOUT is recorded.
 #pragma once
 #include <cuda.h>
 
 namespace pq {
 
-constexpr int kTcThreads = 320;
-constexpr int kTcEpiThreads = 256;
+constexpr int kTcThreads = 512;
+constexpr int kTcEpiThreads = 512;
 constexpr int kTcStages = 3;
 constexpr int kTcXBytes = 128 * 128 * 2;   // one x tile: 128 rows x 128 bf16
 constexpr int kTcSBytes = 128 * 128 * 2;   // one bf16 term of S (B operand)
 constexpr int kTcSmS = 0;                  // S_hi, S_lo
 constexpr int kTcSmX = kTcSmS + 2 * kTcSBytes;
-constexpr int kTcSmRowSq = kTcSmX + kTcStages * kTcXBytes;   // [2][128] float
-constexpr int kTcSmFq = kTcSmRowSq + 1024;                   // FastQuant (36 B)
+constexpr int kTcSmRowSq = kTcSmX + kTcStages * kTcXBytes;   // [4][128] float, then [4][128] bytes of level-4 nibbles
+constexpr int kTcSmFq = kTcSmRowSq + 2048 + 512;             // FastQuant (36 B)
 constexpr int kTcSmBar = kTcSmFq + 64;                       // full[3], empty[3], tfull[2], tempty[2]
 constexpr int kTcSmMisc = kTcSmBar + 128;                    // tmem base, abort flag
 constexpr int kTcSmFix = kTcSmMisc + 64;                     // FixQueue
@@ -115,6 +119,7 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   FastQuant* fq = reinterpret_cast<FastQuant*>(smem + kTcSmFq);
   FixQueue* fixq = reinterpret_cast<FixQueue*>(smem + kTcSmFix);
   float* rowsq = reinterpret_cast<float*>(smem + kTcSmRowSq);
+  uint8_t* l4s = reinterpret_cast<uint8_t*>(rowsq + 4 * 128);  // [4][128] level-4 codes of the row's column quarters
   const uint32_t bar_full = sb + kTcSmBar, bar_empty = bar_full + 8 * kTcStages;
   const uint32_t bar_tfull = bar_empty + 8 * kTcStages, bar_tempty = bar_tfull + 16;
   const int n_tiles = n_row_tiles * 2 * a.n_kv_heads;
@@ -139,15 +144,23 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // B operand: B[n][k] = S[k][n]; two halves of 64 k; row n = 128 bytes, 16-byte chunk c stored at c ^ (n & 7).
-  for (int idx = tid; idx < 128 * 128; idx += kTcThreads) {
-    const int k = idx >> 7, n = idx & 127;  // consecutive threads read consecutive n: coalesced
-    const float v = a.S[idx];
-    const __nv_bfloat16 hi = __float2bfloat16_rn(v);
-    const __nv_bfloat16 lo = __float2bfloat16_rn(v - __bfloat162float(hi));
-    const int half = k >> 6, kk = k & 63;
-    const int off = half * 16384 + n * 128 + ((((kk >> 3) ^ (n & 7)) << 4) | ((kk & 7) << 1));
-    *reinterpret_cast<__nv_bfloat16*>(smem + kTcSmS + off) = hi;
-    *reinterpret_cast<__nv_bfloat16*>(smem + kTcSmS + kTcSBytes + off) = lo;
+  // A task is (row n, chunk of 8 consecutive k): 8 coalesced loads (lanes = consecutive n), one 16-byte store per term.
+  for (int task = tid; task < 128 * 16; task += kTcThreads) {
+    const int n = task & 127, oct = task >> 7;  // k = 8 * oct .. 8 * oct + 7
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float v0 = a.S[(8 * oct + 2 * i) * 128 + n], v1 = a.S[(8 * oct + 2 * i + 1) * 128 + n];
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
+      const __nv_bfloat16 l0 = __float2bfloat16_rn(v0 - __bfloat162float(h0));
+      const __nv_bfloat16 l1 = __float2bfloat16_rn(v1 - __bfloat162float(h1));
+      hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+      lo[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+    }
+    const int half = oct >> 3, c = oct & 7;
+    const int off = half * 16384 + n * 128 + ((c ^ (n & 7)) << 4);
+    *reinterpret_cast<uint4*>(smem + kTcSmS + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    *reinterpret_cast<uint4*>(smem + kTcSmS + kTcSBytes + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA unit
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -155,142 +168,156 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
-      int it = 0;
-      for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-        const int s = it % kTcStages;
-        if (it >= kTcStages && !tc_mbar_wait(bar_empty + 8 * s, ((it / kTcStages) - 1) & 1, abort_flag)) break;
-        const int head = tile % a.n_kv_heads, kv = (tile / a.n_kv_heads) & 1, rt = tile / (2 * a.n_kv_heads);
-        const CUtensorMap* map = kv ? &maps.v : &maps.k;
-        const uint32_t dst = sb + kTcSmX + s * kTcXBytes, bar = bar_full + 8 * s;
-        tc_mbar_expect_tx(bar, kTcXBytes);
+  // One thread issues the TMA loads of local tile `it` (tile blockIdx.x + it * gridDim.x).
+  auto issue_tma = [&](int it) {
+    const int tile = blockIdx.x + it * gridDim.x;
+    if (tile >= n_tiles) return;
+    const int s = it % kTcStages;
+    if (it >= kTcStages && !tc_mbar_wait(bar_empty + 8 * s, ((it / kTcStages) - 1) & 1, abort_flag)) return;
+    const int head = tile % a.n_kv_heads, kv = (tile / a.n_kv_heads) & 1, rt = tile / (2 * a.n_kv_heads);
+    const CUtensorMap* map = kv ? &maps.v : &maps.k;
+    const uint32_t dst = sb + kTcSmX + s * kTcXBytes, bar = bar_full + 8 * s;
+    tc_mbar_expect_tx(bar, kTcXBytes);
 #pragma unroll
-        for (int h = 0; h < 2; ++h)
-          asm volatile(
-              "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-              ::"r"(dst + h * 16384), "l"(map), "r"(h * 64), "r"(head), "r"(rt * 128), "r"(bar)
-              : "memory");
-      }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      int it = 0;
-      for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-        const int s = it % kTcStages, acc = it & 1;
-        if (!tc_mbar_wait(bar_full + 8 * s, (it / kTcStages) & 1, abort_flag)) break;
-        if (it >= 2 && !tc_mbar_wait(bar_tempty + 8 * acc, ((it >> 1) - 1) & 1, abort_flag)) break;
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t xa = sb + kTcSmX + s * kTcXBytes;
-        const uint32_t d = tmem_base + acc * 128;
-        uint32_t accumulate = 0;
+    for (int h = 0; h < 2; ++h)
+      asm volatile(
+          "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+          ::"r"(dst + h * 16384), "l"(map), "r"(h * 64), "r"(head), "r"(rt * 128), "r"(bar)
+          : "memory");
+  };
+  // One thread issues the 16 MMAs of local tile `it` into accumulator it & 1.
+  auto issue_mma = [&](int it) {
+    if (blockIdx.x + it * (int)gridDim.x >= n_tiles) return;
+    const int s = it % kTcStages, acc = it & 1;
+    if (!tc_mbar_wait(bar_full + 8 * s, (it / kTcStages) & 1, abort_flag)) return;
+    if (it >= 2 && !tc_mbar_wait(bar_tempty + 8 * acc, ((it >> 1) - 1) & 1, abort_flag)) return;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t xa = sb + kTcSmX + s * kTcXBytes;
+    const uint32_t d = tmem_base + acc * 128;
+    uint32_t accumulate = 0;
 #pragma unroll
-        for (int term = 0; term < 2; ++term)
+    for (int term = 0; term < 2; ++term)
 #pragma unroll
-          for (int h = 0; h < 2; ++h)
+      for (int h = 0; h < 2; ++h)
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-              const uint64_t ad = tc_smem_desc(xa + h * 16384 + ks * 32);
-              const uint64_t bd = tc_smem_desc(sb + kTcSmS + term * kTcSBytes + h * 16384 + ks * 32);
-              tc_mma(d, ad, bd, accumulate);
-              accumulate = 1;
-            }
-        tc_commit(bar_empty + 8 * s);     // the x stage may be refilled once these MMAs have read it
-        tc_commit(bar_tfull + 8 * acc);   // the accumulator is complete
-      }
-    }
-  } else {
-    // ------------------------------------------------------------------ epilogue (8 warps)
-    constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock, orad = o4 + 2 * kTokenBlock;
-    const int et = tid - 64;                       // 0..255
-    const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
-    const int half = (warp - 2) >> 2;              // columns [64*half, 64*half + 64)
-    const int r = quarter * 32 + lane;             // row of the tile
-    const bool uniform = (a.tables->flags & kFlagUniformL1) != 0u;
-    const Layout L = make_layout(128, a.capacity);
-    int it = 0;
-    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-      const int acc = it & 1;
-      const int head = tile % a.n_kv_heads, kv = (tile / a.n_kv_heads) & 1, rt = tile / (2 * a.n_kv_heads);
-      // A wait that gives up must not leave the loop: the other epilogue warps may be past it and
-      // would wait for this one at the named barriers.  The tile is skipped instead (warp-uniform).
-      const bool ready = __all_sync(0xffffffffu, tc_mbar_wait(bar_tfull + 8 * acc, (it >> 1) & 1, abort_flag));
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 128 + half * 64;
-      // pass 1: squared norm of the row (its two halves are exchanged through shared memory)
-      float sq = 0.f;
-      if (ready) {
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll 1
-        for (int i = 0; i < 4; ++i) {
-          float y[16];
-          tc_ld16(taddr + 16 * i, y);
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-          for (int c = 0; c < 16; ++c) sq = fmaf(y[c], y[c], sq);
+        for (int ks = 0; ks < 4; ++ks) {
+          const uint64_t ad = tc_smem_desc(xa + h * 16384 + ks * 32);
+          const uint64_t bd = tc_smem_desc(sb + kTcSmS + term * kTcSBytes + h * 16384 + ks * 32);
+          tc_mma(d, ad, bd, accumulate);
+          accumulate = 1;
         }
-      }
-      rowsq[half * 128 + r] = sq;
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      const float dy = kRotErr * 1.0001f * sqrtf(rowsq[r] + rowsq[128 + r]);
-      const int row = rt * 128 + r;
-      uint8_t* tb = nullptr;
-      int tok = 0;
-      if (ready && row < a.total_tokens) {
-        int seq, pos;
+    tc_commit(bar_empty + 8 * s);     // the x stage may be refilled once these MMAs have read it
+    tc_commit(bar_tfull + 8 * acc);   // the accumulator is complete
+  };
+  if (tid == 0) {
+    issue_tma(0);
+    issue_tma(1);
+  }
+  if (tid == 32) issue_mma(0);
+  __syncwarp();
+
+  // ---- tile loop: all 16 warps are epilogue warps
+  constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock, orad = o4 + 2 * kTokenBlock;
+  const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
+  const int cq = warp >> 2;                      // columns [32*cq, 32*cq + 32): blocks 2cq, 2cq+1
+  const int r = quarter * 32 + lane;             // row of the tile
+  const bool uniform = (a.tables->flags & kFlagUniformL1) != 0u;
+  const Layout L = make_layout(128, a.capacity);
+  int rd_seq = 0, rd_first = 0, rd_count = 0, rd_start = -1;   // destination of the last row looked up
+  int it = 0;
+  for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+    const int acc = it & 1;
+    const int head = tile % a.n_kv_heads, kv = (tile / a.n_kv_heads) & 1, rt = tile / (2 * a.n_kv_heads);
+    // A wait that gives up must not leave the loop: the other warps may be past it and would wait
+    // for this one at the named barriers.  The tile is skipped instead (warp-uniform).
+    const bool ready = __all_sync(0xffffffffu, tc_mbar_wait(bar_tfull + 8 * acc, (it >> 1) & 1, abort_flag));
+    // keep the pipeline fed: loads two tiles ahead, the next tile's MMAs under this tile's epilogue
+    if (tid == 0) issue_tma(it + 2);
+    if (tid == 32) issue_mma(it + 1);
+    __syncwarp();
+    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 128 + cq * 32;
+    // pass 1: squared norm of the row (its four column quarters are exchanged through shared memory)
+    float sq = 0.f;
+    if (ready) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      float y[32];
+      tc_ld16(taddr, y);
+      tc_ld16(taddr + 16, y + 16);
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+      for (int c = 0; c < 32; ++c) sq = fmaf(y[c], y[c], sq);
+    }
+    rowsq[cq * 128 + r] = sq;
+    asm volatile("bar.sync 1, 512;" ::: "memory");
+    const RowMargins rm = make_row_margins(
+        kRotErr * 1.0001f * sqrtf((rowsq[r] + rowsq[128 + r]) + (rowsq[256 + r] + rowsq[384 + r])), *fq);
+    const int row = rt * 128 + r;
+    uint8_t* tb = nullptr;
+    int tok = 0;
+    if (ready && row < a.total_tokens) {
+      int seq, pos;
+      if (row >= rd_first && row < rd_first + rd_count) {  // same sequence as this thread's previous row
+        seq = rd_seq;
+        pos = rd_start < 0 ? -1 : rd_start + (row - rd_first);
+      } else {
         row_destination(a, row, &seq, &pos);
-        if (pos >= 0) {
-          tb = a.cache + block_offset(L, a.n_kv_heads, seq, head, kv, pos);
-          tok = pos % kTokenBlock;
-        }
+        rd_seq = seq;
+        rd_first = a.cu_seqlens ? a.cu_seqlens[seq] : row;
+        rd_count = a.cu_seqlens ? a.cu_seqlens[seq + 1] - rd_first : 1;
+        rd_start = pos < 0 ? -1 : pos - (row - rd_first);
       }
-      const int64_t xoff = (int64_t)row * a.token_stride + (int64_t)head * a.head_stride;
-      // pass 2: one block at a time
-      uint32_t l2acc = 0, l3acc = 0, l4acc = 0, sat = 0;
-      unsigned long long racc = 0ull, leftbits = 0ull;
-      if (ready) {
+      if (pos >= 0) {
+        tb = a.cache + block_offset(L, a.n_kv_heads, seq, head, kv, pos);
+        tok = pos % kTokenBlock;
+      }
+    }
+    const int64_t xoff = (int64_t)row * a.token_stride + (int64_t)head * a.head_stride;
+    // pass 2: one block at a time
+    uint32_t l2acc = 0, l3acc = 0, l4acc = 0, racc = 0, sat = 0;
+    unsigned long long leftbits = 0ull;
+    if (ready) {
 #pragma unroll 1
-        for (int i = 0; i < 4; ++i) {
-          float y[16];
-          tc_ld16(taddr + 16 * i, y);
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-          FastBlock fb;
-          polar_quant_block_fast(y, dy, *fq, &fb);
-          if (!uniform) fb.amb |= 0xFFu;  // other level-1 codebooks: decide every level-1 angle exactly
-          if (tb != nullptr) {
-            *reinterpret_cast<uint32_t*>(tb + tok * 32 + half * 16 + 4 * i) = fb.l1;
-            l2acc |= fb.l2 << (8 * i);
-            l3acc |= fb.l3 << (4 * i);
-            l4acc |= fb.l4 << (2 * i);
-            float rv = fb.radius;
-            if (rv > 65504.f) { rv = 65504.f; ++sat; }
-            racc |= (unsigned long long)__half_as_ushort(__float2half_rn(rv)) << (16 * i);
-            if (fb.amb) {
-              uint32_t left;
-              fix_push(fixq, fb.amb, xoff, tb, tok, 4 * half + i, kv, &left);
-              leftbits |= (unsigned long long)left << (15 * i);  // queue full: pushed again by fix_rounds
-            }
+      for (int i = 0; i < 2; ++i) {
+        float y[16];
+        tc_ld16(taddr + 16 * i, y);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        FastBlock fb;
+        polar_quant_block_fast(y, rm, *fq, &fb);
+        if (!uniform) fb.amb |= 0xFFu;  // other level-1 codebooks: decide every level-1 angle exactly
+        if (tb != nullptr) {
+          *reinterpret_cast<uint32_t*>(tb + tok * 32 + cq * 8 + 4 * i) = fb.l1;
+          l2acc |= fb.l2 << (8 * i);
+          l3acc |= fb.l3 << (4 * i);
+          l4acc |= fb.l4 << (2 * i);
+          float rv = fb.radius;
+          if (rv > 65504.f) { rv = 65504.f; ++sat; }
+          racc |= (uint32_t)__half_as_ushort(__float2half_rn(rv)) << (16 * i);
+          if (fb.amb) {
+            uint32_t left;
+            fix_push(fixq, fb.amb, xoff, tb, tok, 2 * cq + i, kv, &left);
+            leftbits |= (unsigned long long)left << (15 * i);  // queue full: pushed again by fix_rounds
           }
         }
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) tc_mbar_arrive(bar_tempty + 8 * acc);  // this accumulator may be overwritten
       }
-      if (tb != nullptr) {
-        *reinterpret_cast<uint32_t*>(tb + o2 + tok * 8 + half * 4) = l2acc;
-        *reinterpret_cast<uint16_t*>(tb + o3 + tok * 4 + half * 2) = (uint16_t)l3acc;
-        tb[o4 + tok * 2 + half] = (uint8_t)l4acc;
-        *reinterpret_cast<unsigned long long*>(tb + orad + tok * 16 + half * 8) = racc;
-        if (sat) atomicAdd(a.status + 2, (int)sat);
-      }
-      // Exact re-decisions are batched over tiles: drain the queue when it is half full (a push that
-      // did not fit leaves the counter above the capacity) or after the CTA's last tile.
-      asm volatile("bar.sync 1, 256;" ::: "memory");
-      const bool last_tile = tile + (int)gridDim.x >= n_tiles;
-      if (fixq->count > kFixCap / 2 || last_tile)
-        fix_rounds(a, fixq, leftbits, xoff, tb, tok, half, kv, et, kTcEpiThreads, 1);
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) tc_mbar_arrive(bar_tempty + 8 * acc);  // this accumulator may be overwritten
     }
+    l4s[cq * 128 + r] = (uint8_t)l4acc;
+    if (tb != nullptr) {
+      *reinterpret_cast<uint16_t*>(tb + o2 + tok * 8 + cq * 2) = (uint16_t)l2acc;
+      tb[o3 + tok * 4 + cq] = (uint8_t)l3acc;
+      *reinterpret_cast<uint32_t*>(tb + orad + tok * 16 + cq * 4) = racc;
+      if (sat) atomicAdd(a.status + 2, (int)sat);
+    }
+    asm volatile("bar.sync 1, 512;" ::: "memory");
+    if (tb != nullptr && (cq & 1) == 0)  // level-4 codes of four blocks share a byte: two column quarters
+      tb[o4 + tok * 2 + (cq >> 1)] = (uint8_t)(l4s[cq * 128 + r] | (l4s[(cq + 1) * 128 + r] << 4));
+    // Exact re-decisions are batched over tiles: drain the queue when it is 3/4 full (a push that
+    // did not fit leaves the counter above the capacity) or after the CTA's last tile.
+    const bool last_tile = tile + (int)gridDim.x >= n_tiles;
+    if (fixq->count > (3 * kFixCap) / 4 || last_tile)
+      fix_rounds(a, fixq, leftbits, xoff, tb, tok, 2 * cq, kv, tid, kTcEpiThreads, 1);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
