@@ -2,9 +2,12 @@
 //
 // The rotation y = x . S is computed with float32-grade accuracy (tensor cores with S split into
 // two bf16 terms, or float32 FMAs).  Either way |y - y_exact| <= kRotErr * ||x||_2 per coordinate:
-//   two bf16 terms drop at most 2^-17 |S_kj| per entry, so the error is <= 2^-17 sum_k |x_k||S_kj|
-//   <= 2^-17 ||x||_2 (Cauchy-Schwarz, columns of S have unit norm); a float32 dot product of 128
-//   terms has the same bound (129 * 2^-24).
+//   * two bf16 terms (round to nearest, 8 significant bits each) leave |S - hi - lo| <= 2^-18 |S|, so
+//     the representation error is <= 2^-18 sum_k |x_k||S_kj| <= 2^-18 ||x||_2 (Cauchy-Schwarz,
+//     columns of S have unit norm); the products of bf16 inputs are exact in float32 and the 16
+//     accumulating MMAs may add up to 2^-19 sum_k |x_k||S_kj| more (2 ulp of the running sum each);
+//   * a float32 dot product of 128 terms is off by at most 128 * 2^-24 = 2^-17 of the same sum.
+// kRotErr = 1.1 * 2^-17 covers both.
 // Angles are never computed.  Every code is decided by sign tests on the pair (Algorithm 1, Polar +
 // Quant, in the form "which side of the boundary line is the point on"), in float32, together with
 // a certified margin: a decision is trusted only if the point is farther from every boundary than
