@@ -340,7 +340,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
       for (int it = 0; it < kStages - 1 && st0 + it < st1; ++it) issue_copy(it);
     __syncwarp();
     // ---------------------------------------------------------------- consumers
-    // q' fragments: A operand (16 heads x 16 coords per k-step); rows >= 8 are zero.
+    // q' fragments: A operand (16 rows x 16 coords per k-step): rows 0..7 the fp16 values, rows 8..15 the residuals.
     // k-step ks covers, for thread c, sub-block (ks & 3) of block 2c + (ks >> 2).
     uint32_t qa[8][2], ql[8][2];  // fp16 value and fp16 residual of q'
     {
@@ -369,7 +369,10 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
         const uint32_t vblk = kblk + kBlockBytes128;
         const int t0 = (warp & 7) * 8;  // tile's first token inside its token-block
         // ---- scores: S^T (heads x tokens)
-        float sc[4] = {0.f, 0.f, 0.f, 0.f};
+        // A operand: rows 0..7 = q_hi of the group's heads, rows 8..15 = q_lo of the same heads, so one MMA
+        // with k_hi yields q_hi k_hi (row g) and q_lo k_hi (row g + 8), and one with k_lo the two small
+        // terms; both rows of a head land in the same thread.  Two accumulators: two chains of 8 MMAs.
+        float sc[4] = {0.f, 0.f, 0.f, 0.f}, sc_lo[4] = {0.f, 0.f, 0.f, 0.f};
         {
           const int tk = t0 + ktok;
           const uint2 l1 = lds64(kblk + tk * 32 + c * 8);
@@ -381,17 +384,19 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
           decode_block_hilo(l1.x, c2 & 0xFFu, c3 & 0xFu, c4 & 3u, __low2half2(as_h2(rr)), sm_base, rep, kh, kl);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
-            mma_16816(sc, qa[ks][0], 0u, qa[ks][1], 0u, as_u32(kl[2 * ks]), as_u32(kl[2 * ks + 1]));
-            mma_16816(sc, ql[ks][0], 0u, ql[ks][1], 0u, as_u32(kh[2 * ks]), as_u32(kh[2 * ks + 1]));
-            mma_16816(sc, qa[ks][0], 0u, qa[ks][1], 0u, as_u32(kh[2 * ks]), as_u32(kh[2 * ks + 1]));
+            mma_16816(sc_lo, qa[ks][0], ql[ks][0], qa[ks][1], ql[ks][1], as_u32(kl[2 * ks]), as_u32(kl[2 * ks + 1]));
+            mma_16816(sc, qa[ks][0], ql[ks][0], qa[ks][1], ql[ks][1], as_u32(kh[2 * ks]), as_u32(kh[2 * ks + 1]));
           }
           decode_block_hilo(l1.y, c2 >> 8, c3 >> 4, (c4 >> 2) & 3u, __high2half2(as_h2(rr)), sm_base, rep, kh, kl);
 #pragma unroll
           for (int ks = 0; ks < 4; ++ks) {
-            mma_16816(sc, qa[4 + ks][0], 0u, qa[4 + ks][1], 0u, as_u32(kl[2 * ks]), as_u32(kl[2 * ks + 1]));
-            mma_16816(sc, ql[4 + ks][0], 0u, ql[4 + ks][1], 0u, as_u32(kh[2 * ks]), as_u32(kh[2 * ks + 1]));
-            mma_16816(sc, qa[4 + ks][0], 0u, qa[4 + ks][1], 0u, as_u32(kh[2 * ks]), as_u32(kh[2 * ks + 1]));
+            mma_16816(sc_lo, qa[4 + ks][0], ql[4 + ks][0], qa[4 + ks][1], ql[4 + ks][1], as_u32(kl[2 * ks]),
+                      as_u32(kl[2 * ks + 1]));
+            mma_16816(sc, qa[4 + ks][0], ql[4 + ks][0], qa[4 + ks][1], ql[4 + ks][1], as_u32(kh[2 * ks]),
+                      as_u32(kh[2 * ks + 1]));
           }
+          sc[0] += (sc_lo[0] + sc_lo[2]) + sc[2];  // small terms first
+          sc[1] += (sc_lo[1] + sc_lo[3]) + sc[3];
         }
         // ---- online softmax for head g; this thread holds logical tokens 2c, 2c+1 = physical c, c+4
         const bool ok0 = tile_tok0 + c < len, ok1 = tile_tok0 + c + 4 < len;
