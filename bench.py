@@ -48,21 +48,53 @@ def _peaks():
 
 
 class ClockSampler:
-    """nvidia-smi clock / throttle-reason samples taken while the timed region runs."""
+    """SM clock and throttle-reason samples taken while the timed region runs: an NVML polling thread
+    (about every 2 ms, the timed region lasts tens of milliseconds); nvidia-smi as a fallback."""
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
              "clocks_event_reasons.sw_power_cap")
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, gpu_index: int):
         self.gpu_index = gpu_index
         self.proc = None
         self.path = None
+        self.thread = None
+        self.stop_flag = False
+        self.sm, self.reason_bits, self.smax = [], 0, None
+
+    def _poll(self, nvml, handle):
+        while not self.stop_flag:
+            try:
+                self.sm.append(nvml.nvmlDeviceGetClockInfo(handle, nvml.NVML_CLOCK_SM))
+                self.reason_bits |= int(nvml.nvmlDeviceGetCurrentClocksEventReasons(handle))
+            except Exception:
+                break
+            time.sleep(0.002)
 
     def start(self):
         try:
+            import threading
+            import pynvml as nvml
+            nvml.nvmlInit()
+            # NVML enumerates all GPUs of the host; CUDA_VISIBLE_DEVICES may renumber them
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            idx = self.gpu_index
+            if vis:
+                entry = vis.split(",")[self.gpu_index].strip()
+                handle = nvml.nvmlDeviceGetHandleByIndex(int(entry)) if entry.isdigit() else nvml.nvmlDeviceGetHandleByUUID(entry)
+            else:
+                handle = nvml.nvmlDeviceGetHandleByIndex(idx)
+            self.smax = nvml.nvmlDeviceGetMaxClockInfo(handle, nvml.NVML_CLOCK_SM)
+            self.thread = threading.Thread(target=self._poll, args=(nvml, handle), daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.thread = None
+        try:
             fd, self.path = tempfile.mkstemp(suffix=".csv")
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"], stdout=fd,
+                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=fd,
                                          stderr=subprocess.DEVNULL)
             os.close(fd)
         except OSError:
@@ -70,6 +102,14 @@ class ClockSampler:
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.thread is not None:
+            self.stop_flag = True
+            self.thread.join(timeout=2)
+            if self.sm:
+                out.update(sm_mhz=float(statistics.median(self.sm)), sm_max_mhz=float(self.smax),
+                           reasons=sorted(n for bit, n in self.REASONS.items() if self.reason_bits & bit),
+                           samples=len(self.sm), source="nvml")
+            return out
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -97,7 +137,8 @@ class ClockSampler:
         except OSError:
             pass
         if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm))
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm),
+                       source="nvidia-smi")
         return out
 
 
@@ -384,7 +425,7 @@ def main():
     global BATCH
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")

@@ -43,7 +43,8 @@ struct Tables {
   uint32_t l1_lo[16];
   uint2 u_tab[4][64];
   double bnd_tan2[9];  // tan^2 of the boundaries of levels 2, 3, 4 (decisions on squared radii)
-  //   t1p_hi[e], t1p_lo[e] : e = one byte of level-1 codes (pair a | pair b << 4): .x = entry of a, .y = entry of b
+  //   t1p_hi[e], t1p_lo[e] : e = one byte of level-1 codes (pair a | pair b << 4): .x = (cos a, cos b), .y = (sin a, sin b)
+  //                          so that a half2 of the two pairs' multipliers multiplies element-wise
   uint2 t1p_hi[256];
   uint2 t1p_lo[256];
   uint32_t reserved[30];

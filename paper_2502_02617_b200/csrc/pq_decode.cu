@@ -419,7 +419,7 @@ __global__ void dequant_kernel(int d, int n_kv_heads, const float* S, const Tabl
     const __half2 uh = *reinterpret_cast<const __half2*>(&up);
     const __half r = reinterpret_cast<const __half*>(tb + L.orad + t * L.br)[blk];
     const __half u = __hmul(r, (i & 2) ? __high2half(uh) : __low2half(uh));
-    const __half2 t1 = *reinterpret_cast<const __half2*>(&tables->l1_hi[c1]);
+    const __half2 t1 = *reinterpret_cast<const __half2*>(&tables->l1_hi[c1]);  // (cos, sin) of the centroid
     ysm[j] = __half2float(__hmul(u, (i & 1) ? __high2half(t1) : __low2half(t1)));
   } else {
     ysm[j] = decode_coord(tb, L, tok % kTokenBlock, j, cc, cs);

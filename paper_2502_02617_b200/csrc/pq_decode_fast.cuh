@@ -16,7 +16,8 @@
 // Levels 4..2 are folded into one table per 4-coordinate sub-block, level 1 is a half2 multiply:
 //   u    [4][64][16] sub-block s, index c2_s | c3_(s>>1) << 2 | c4 << 4 -> the multipliers of the
 //                    sub-block's two level-1 pairs as (half2 values, half2 rounding residuals)
-//   t1hi [256][16]   index = one byte of level-1 codes (pair 2s | pair 2s+1 << 4) -> (cos, sin) x 2 in fp16
+//   t1hi [256][16]   index = one byte of level-1 codes (pair a = 2s | pair b = 2s+1 << 4) -> (cos a, cos b), (sin a, sin b)
+//                    in fp16: the half2 (u_a, u_b) of the table above multiplies them element-wise
 //   t1lo [256][16]   the fp16 rounding residuals of the same entries
 // All are replicated 16 times so that every lane of a half-warp reads its own banks.
 // Values use the fp16 parts only.  Keys feed the softmax exponent, where an fp16-rounded operand
@@ -139,7 +140,9 @@ __device__ __forceinline__ void u_offsets(uint32_t c2, uint32_t c3n, uint32_t c4
   off[3] = 3 * 8192 + (((c2 << 1) & 0x180u) | hi1);
 }
 
-// DeQuant of one 16-coordinate block in the rotated basis as 8 half2 (coordinates 2i, 2i+1), fp16 path.
+// DeQuant of one 16-coordinate block in the rotated basis, fp16 path.  For sub-block s (coordinates
+// 4s .. 4s+3, level-1 pairs a = 2s and b = 2s+1) the result is two half2:
+//   out[2s]   = (x_a, x_b) = coordinates (4s, 4s+2)        out[2s+1] = (y_a, y_b) = coordinates (4s+1, 4s+3)
 //   l1 : 8 level-1 codes, code j at bits [4j, 4j+4)     c2 : 4 level-2 codes, 2 bits each (clean)
 //   c3n: 2 level-3 codes in a nibble (clean)             c4 : the level-4 code (clean)
 //   r2 : the block radius in both halves                 rep: (lane & 15) * 8
@@ -152,8 +155,8 @@ __device__ __forceinline__ void decode_block_h2(uint32_t l1, uint32_t c2, uint32
   for (int s = 0; s < 4; ++s) {
     const __half2 u = __hmul2(r2, as_h2(lds32(ub + off[s])));
     const uint2 e = lds64(t1 + ((s == 0 ? (l1 << 7) : (l1 >> (8 * s - 7))) & 0x7F80u));
-    out[2 * s] = __hmul2(__low2half2(u), as_h2(e.x));
-    out[2 * s + 1] = __hmul2(__high2half2(u), as_h2(e.y));
+    out[2 * s] = __hmul2(u, as_h2(e.x));
+    out[2 * s + 1] = __hmul2(u, as_h2(e.y));
   }
 }
 
@@ -173,13 +176,11 @@ __device__ __forceinline__ void decode_block_hilo(uint32_t l1, uint32_t c2, uint
     const __half2 u_lo = __hfma2(r2, as_h2(uu.y), __hfma2(r2, as_h2(uu.x), __hneg2(u_hi)));
     const uint32_t idx = (s == 0 ? (l1 << 7) : (l1 >> (8 * s - 7))) & 0x7F80u;
     const uint2 th = lds64(t1 + idx), tl = lds64(t1 + (kSmT1lo - kSmT1p) + idx);
-    const __half2 ua = __low2half2(u_hi), ub2 = __high2half2(u_hi);
-    const __half2 la = __low2half2(u_lo), lb = __high2half2(u_lo);
-    const __half2 ka = __hmul2(ua, as_h2(th.x)), kb = __hmul2(ub2, as_h2(th.y));
-    hi[2 * s] = ka;
-    hi[2 * s + 1] = kb;
-    lo[2 * s] = __hfma2(ua, as_h2(tl.x), __hfma2(la, as_h2(th.x), __hfma2(ua, as_h2(th.x), __hneg2(ka))));
-    lo[2 * s + 1] = __hfma2(ub2, as_h2(tl.y), __hfma2(lb, as_h2(th.y), __hfma2(ub2, as_h2(th.y), __hneg2(kb))));
+    const __half2 kx = __hmul2(u_hi, as_h2(th.x)), ky = __hmul2(u_hi, as_h2(th.y));
+    hi[2 * s] = kx;
+    hi[2 * s + 1] = ky;
+    lo[2 * s] = __hfma2(u_hi, as_h2(tl.x), __hfma2(u_lo, as_h2(th.x), __hfma2(u_hi, as_h2(th.x), __hneg2(kx))));
+    lo[2 * s + 1] = __hfma2(u_hi, as_h2(tl.y), __hfma2(u_lo, as_h2(th.y), __hfma2(u_hi, as_h2(th.y), __hneg2(ky))));
   }
 }
 
@@ -352,10 +353,11 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
           v = *reinterpret_cast<const uint2*>(a.ws.qrot_h + qoff + 4 * ks);
           w = *reinterpret_cast<const uint2*>(a.ws.qrot_l + qoff + 4 * ks);
         }
-        qa[ks][0] = v.x;
-        qa[ks][1] = v.y;
-        ql[ks][0] = w.x;
-        ql[ks][1] = w.y;
+        // decoded keys come as (coord 0, coord 2), (coord 1, coord 3) of each sub-block: permute q' to match
+        qa[ks][0] = __byte_perm(v.x, v.y, 0x5410);
+        qa[ks][1] = __byte_perm(v.x, v.y, 0x7632);
+        ql[ks][0] = __byte_perm(w.x, w.y, 0x5410);
+        ql[ks][1] = __byte_perm(w.x, w.y, 0x7632);
       }
     }
     for (int st = st0, it = 0; st < st1; ++st, ++it) {
@@ -447,10 +449,13 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
             if (!ok1) rr = 0u;
             decode_block_h2(l1, c2, c3 & 0xFu, c4 & 3u, as_h2(rr | (rr << 16)), sm_base, rep, vb);
           }
+          // va[2s] = (x_a, x_b), va[2s+1] = (y_a, y_b) of sub-block s: pair i = 2s + h takes half h of both
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
-            const uint32_t x = __byte_perm(as_u32(va[i]), as_u32(vb[i]), 0x5410);  // coord 2i   of tokens (A, B)
-            const uint32_t y = __byte_perm(as_u32(va[i]), as_u32(vb[i]), 0x7632);  // coord 2i+1 of tokens (A, B)
+            const int s2 = 2 * (i >> 1);
+            const uint32_t sel = (i & 1) ? 0x7632 : 0x5410;
+            const uint32_t x = __byte_perm(as_u32(va[s2]), as_u32(vb[s2]), sel);          // coord 2i   of tokens (A, B)
+            const uint32_t y = __byte_perm(as_u32(va[s2 + 1]), as_u32(vb[s2 + 1]), sel);  // coord 2i+1 of tokens (A, B)
             mma_1688(o_acc[i], x, y, pb);
           }
         }

@@ -204,8 +204,9 @@ int32_t pq_build_tables(const double* cen, const double* bnd, void* tables_host)
   };
   for (int c = 0; c < 16; ++c) split(std::cos(cen[c]), std::sin(cen[c]), &t.l1_hi[c], &t.l1_lo[c]);
   for (int e = 0; e < 256; ++e) {
-    t.t1p_hi[e] = make_uint2(t.l1_hi[e & 15], t.l1_hi[e >> 4]);
-    t.t1p_lo[e] = make_uint2(t.l1_lo[e & 15], t.l1_lo[e >> 4]);
+    const uint32_t ha = t.l1_hi[e & 15], hb = t.l1_hi[e >> 4], la = t.l1_lo[e & 15], lb = t.l1_lo[e >> 4];
+    t.t1p_hi[e] = make_uint2((ha & 0xFFFFu) | (hb << 16), (ha >> 16) | (hb & 0xFFFF0000u));
+    t.t1p_lo[e] = make_uint2((la & 0xFFFFu) | (lb << 16), (la >> 16) | (lb & 0xFFFF0000u));
   }
   for (int s = 0; s < 4; ++s)
     for (int i = 0; i < 64; ++i) {
