@@ -47,69 +47,47 @@ def _peaks():
     return 6650.0, "fallback (earlier pool measurement)"
 
 
+_POLLER = r"""
+import sys, time, os
+import pynvml as nvml
+nvml.nvmlInit()
+sel = sys.argv[1]
+h = nvml.nvmlDeviceGetHandleByIndex(int(sel)) if sel.isdigit() else nvml.nvmlDeviceGetHandleByUUID(sel)
+smax = nvml.nvmlDeviceGetMaxClockInfo(h, nvml.NVML_CLOCK_SM)
+out = open(sys.argv[2], "w", buffering=1)
+while True:
+    out.write("%.6f %d %d %d\n" % (time.time(), nvml.nvmlDeviceGetClockInfo(h, nvml.NVML_CLOCK_SM), smax,
+                                     nvml.nvmlDeviceGetCurrentClocksEventReasons(h)))
+    time.sleep(0.001)
+"""
+
+
 class ClockSampler:
-    """SM clock and throttle-reason samples taken while the timed region runs: an NVML polling thread
-    (about every 2 ms, the timed region lasts tens of milliseconds); nvidia-smi as a fallback."""
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-             "clocks_event_reasons.sw_power_cap")
+    """SM clock and throttle-reason samples taken while the timed region runs, by a separate NVML
+    polling process (about one sample per millisecond; the samples are cut to the timed window)."""
     REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, gpu_index: int):
         self.gpu_index = gpu_index
         self.proc = None
         self.path = None
-        self.thread = None
-        self.stop_flag = False
-        self.sm, self.reason_bits, self.smax = [], 0, None
-
-    def _poll(self, nvml, handle):
-        while not self.stop_flag:
-            try:
-                self.sm.append(nvml.nvmlDeviceGetClockInfo(handle, nvml.NVML_CLOCK_SM))
-                self.reason_bits |= int(nvml.nvmlDeviceGetCurrentClocksEventReasons(handle))
-            except Exception:
-                break
-            time.sleep(0.002)
 
     def start(self):
         try:
-            import threading
-            import pynvml as nvml
-            nvml.nvmlInit()
-            # NVML enumerates all GPUs of the host; CUDA_VISIBLE_DEVICES may renumber them
             vis = os.environ.get("CUDA_VISIBLE_DEVICES")
-            idx = self.gpu_index
-            if vis:
-                entry = vis.split(",")[self.gpu_index].strip()
-                handle = nvml.nvmlDeviceGetHandleByIndex(int(entry)) if entry.isdigit() else nvml.nvmlDeviceGetHandleByUUID(entry)
-            else:
-                handle = nvml.nvmlDeviceGetHandleByIndex(idx)
-            self.smax = nvml.nvmlDeviceGetMaxClockInfo(handle, nvml.NVML_CLOCK_SM)
-            self.thread = threading.Thread(target=self._poll, args=(nvml, handle), daemon=True)
-            self.thread.start()
-            return
-        except Exception:
-            self.thread = None
-        try:
-            fd, self.path = tempfile.mkstemp(suffix=".csv")
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "20"], stdout=fd,
-                                         stderr=subprocess.DEVNULL)
+            sel = vis.split(",")[self.gpu_index].strip() if vis else str(self.gpu_index)
+            fd, self.path = tempfile.mkstemp(suffix=".clk")
             os.close(fd)
+            self.proc = subprocess.Popen([sys.executable, "-c", _POLLER, sel, self.path], stdout=subprocess.DEVNULL,
+                                         stderr=subprocess.DEVNULL)
+            deadline = time.time() + 10.0
+            while time.time() < deadline and os.path.getsize(self.path) == 0 and self.proc.poll() is None:
+                time.sleep(0.01)  # first sample written: the poller is running
         except OSError:
             self.proc = None
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.thread is not None:
-            self.stop_flag = True
-            self.thread.join(timeout=2)
-            if self.sm:
-                out.update(sm_mhz=float(statistics.median(self.sm)), sm_max_mhz=float(self.smax),
-                           reasons=sorted(n for bit, n in self.REASONS.items() if self.reason_bits & bit),
-                           samples=len(self.sm), source="nvml")
-            return out
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -117,28 +95,25 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, smax, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        sm, smax, bits = [], None, 0
         try:
             with open(self.path) as f:
                 for line in f:
-                    parts = [p.strip() for p in line.split(",")]
-                    if len(parts) < 9:
+                    parts = line.split()
+                    if len(parts) != 4:
                         continue
-                    try:
-                        sm.append(float(parts[1]))
-                        smax.append(float(parts[2]))
-                    except ValueError:
+                    ts = float(parts[0])
+                    if t_begin is not None and not (t_begin <= ts <= t_end):
                         continue
-                    for name, val in zip(names, parts[5:9]):
-                        if val.lower().startswith("active"):
-                            reasons.add(name)
+                    sm.append(int(parts[1]))
+                    smax = int(parts[2])
+                    bits |= int(parts[3])
             os.unlink(self.path)
-        except OSError:
+        except (OSError, ValueError):
             pass
         if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons), samples=len(sm),
-                       source="nvidia-smi")
+            out.update(sm_mhz=float(statistics.median(sm)), sm_max_mhz=float(smax), samples=len(sm),
+                       reasons=sorted(n for bit, n in self.REASONS.items() if bits & bit))
         return out
 
 
@@ -345,6 +320,7 @@ def run_cuda(args):
         for i in range(args.warmup):
             step(i, None, e2e)
         barrier()
+        wall = [time.time(), None]
         t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t_start.record(stream)
         last = None
@@ -352,21 +328,22 @@ def run_cuda(args):
             last = step(args.warmup + i, evs[i], e2e)
         t_end.record(stream)
         barrier()
+        wall[1] = time.time()
         total_ms = t_start.elapsed_time(t_end)
         seg = np.array([[e[k].elapsed_time(e[k + 1]) for k in range(3)] for e in evs])  # encode, append, decode
-        return total_ms, seg, last
+        return total_ms, seg, last, wall
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    total_ms, seg, last = timed(e2e=False)
-    clocks = sampler.stop()
+    total_ms, seg, last, wall = timed(e2e=False)
+    clocks = sampler.stop(wall[0], wall[1])
     cache.check_status()
     match = None
     if rank == 0 and not args.skip_match:
         b_enc, qq = last
         Kb, Vb = chunks[(n_total - 1) % 2]
         match = _oracle_match(cache, Kb, Vb, b_enc, qq, out)
-    e2e_total_ms, e2e_seg, _ = (total_ms, seg, None) if args.skip_e2e else timed(e2e=True)
+    e2e_total_ms, e2e_seg, _, _ = (total_ms, seg, None, None) if args.skip_e2e else timed(e2e=True)
     cache.check_status()
 
     def reduce_max(x):
