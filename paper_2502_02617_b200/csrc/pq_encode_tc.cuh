@@ -6,8 +6,10 @@
 //   * y = x . S on the 5th-generation tensor cores: S is split once per CTA into two bf16 terms
 //     (S = S_hi + S_lo + O(2^-17)) kept in shared memory as the K-major B operand; 2 terms x 8
 //     k-steps of tcgen05.mma (M = 128 rows, N = 128, K = 16) accumulate in float32 in tensor memory;
-//     two accumulators, and the MMAs of tile i+1 are issued (by one thread) when the epilogue of
-//     tile i starts, so they run under it;
+//     two accumulators, and the MMAs of tile i+1 are issued when the epilogue of tile i starts, so
+//     they run under it.  Four threads (one per scheduler) issue four MMAs each, so that no warp is
+//     held up by the whole batch; since their order is then free, every MMA accumulates and the
+//     epilogue clears the accumulator after reading it;
 //   * epilogue on all 16 warps.  Tensor-memory lane = row, so a thread owns 32 consecutive rotated
 //     coordinates (2 blocks) of one row: tcgen05.ld, sign-test quantiser with certified margins,
 //     packed stores, queued float64 re-decision of the ambiguous angles.
@@ -104,6 +106,13 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
   for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+__device__ __forceinline__ void tc_st16_zero(uint32_t taddr) {
+  const uint32_t z = 0u;
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};" ::"r"(taddr), "r"(z)
+      : "memory");
+}
+
 struct TcMaps {
   CUtensorMap k, v;
 };
@@ -128,10 +137,10 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
       tc_mbar_init(bar_full + 8 * s, 1);
-      tc_mbar_init(bar_empty + 8 * s, 1);
+      tc_mbar_init(bar_empty + 8 * s, 4);   // one commit per issuing thread
     }
     for (int i = 0; i < 2; ++i) {
-      tc_mbar_init(bar_tfull + 8 * i, 1);
+      tc_mbar_init(bar_tfull + 8 * i, 4);   // one commit per issuing thread
       tc_mbar_init(bar_tempty + 8 * i, kTcEpiThreads / 32);
     }
     *abort_flag = 0;
@@ -185,35 +194,39 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
           ::"r"(dst + h * 16384), "l"(map), "r"(h * 64), "r"(head), "r"(rt * 128), "r"(bar)
           : "memory");
   };
-  // One thread issues the 16 MMAs of local tile `it` into accumulator it & 1.
-  auto issue_mma = [&](int it) {
+  // Lane 0 of warps 0..3 each issue 4 of the 16 MMAs of local tile `it` into accumulator it & 1:
+  // issuer q takes term q >> 1 of S and k-half q & 1.  All MMAs accumulate (the accumulator is zero).
+  auto issue_mma = [&](int it, int q) {
     if (blockIdx.x + it * (int)gridDim.x >= n_tiles) return;
     const int s = it % kTcStages, acc = it & 1;
     if (!tc_mbar_wait(bar_full + 8 * s, (it / kTcStages) & 1, abort_flag)) return;
     if (it >= 2 && !tc_mbar_wait(bar_tempty + 8 * acc, ((it >> 1) - 1) & 1, abort_flag)) return;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t xa = sb + kTcSmX + s * kTcXBytes;
+    const uint32_t xa = sb + kTcSmX + s * kTcXBytes + (q & 1) * 16384;
+    const uint32_t sa = sb + kTcSmS + (q >> 1) * kTcSBytes + (q & 1) * 16384;
     const uint32_t d = tmem_base + acc * 128;
-    uint32_t accumulate = 0;
 #pragma unroll
-    for (int term = 0; term < 2; ++term)
-#pragma unroll
-      for (int h = 0; h < 2; ++h)
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks) {
-          const uint64_t ad = tc_smem_desc(xa + h * 16384 + ks * 32);
-          const uint64_t bd = tc_smem_desc(sb + kTcSmS + term * kTcSBytes + h * 16384 + ks * 32);
-          tc_mma(d, ad, bd, accumulate);
-          accumulate = 1;
-        }
+    for (int ks = 0; ks < 4; ++ks) tc_mma(d, tc_smem_desc(xa + ks * 32), tc_smem_desc(sa + ks * 32), 1u);
     tc_commit(bar_empty + 8 * s);     // the x stage may be refilled once these MMAs have read it
-    tc_commit(bar_tfull + 8 * acc);   // the accumulator is complete
+    tc_commit(bar_tfull + 8 * acc);   // this issuer's share of the accumulator is complete
   };
+  // both accumulators start at zero
+  {
+    const uint32_t z = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (warp >> 2) * 32;
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+      for (int j = 0; j < 2; ++j) tc_st16_zero(z + i * 128 + 16 * j);
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  }
   if (tid == 0) {
     issue_tma(0);
     issue_tma(1);
   }
-  if (tid == 32) issue_mma(0);
+  if (lane == 0 && warp < 4) issue_mma(0, warp);
   __syncwarp();
 
   // ---- tile loop: all 16 warps are epilogue warps
@@ -233,7 +246,7 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     const bool ready = __all_sync(0xffffffffu, tc_mbar_wait(bar_tfull + 8 * acc, (it >> 1) & 1, abort_flag));
     // keep the pipeline fed: loads two tiles ahead, the next tile's MMAs under this tile's epilogue
     if (tid == 0) issue_tma(it + 2);
-    if (tid == 32) issue_mma(it + 1);
+    if (lane == 0 && warp < 4) issue_mma(it + 1, warp);
     __syncwarp();
     const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 128 + cq * 32;
     // pass 1: squared norm of the row (its four column quarters are exchanged through shared memory)
@@ -299,9 +312,12 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
           }
         }
       }
+      tc_st16_zero(taddr);  // leave the accumulator cleared for the next tile that uses it
+      tc_st16_zero(taddr + 16);
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
-      if (lane == 0) tc_mbar_arrive(bar_tempty + 8 * acc);  // this accumulator may be overwritten
+      if (lane == 0) tc_mbar_arrive(bar_tempty + 8 * acc);  // this accumulator may be written again
     }
     l4s[cq * 128 + r] = (uint8_t)l4acc;
     if (tb != nullptr) {
