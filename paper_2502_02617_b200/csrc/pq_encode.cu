@@ -250,10 +250,9 @@ __device__ inline void fix_rounds(const EncodeArgs& a, FixQueue* q, unsigned lon
                                   int tok, int blk0, int kv, int t, int n_threads, int bar_id) {
   for (int round = 0; round < 256; ++round) {
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
-    const int n = min(q->count, kFixCap);
-    if (n > 0) fix_process(q, n, t, n_threads, a.K, a.V, a.in_dtype, a.S, *a.tables, a.status);
+    fix_process(q, t, n_threads, a.K, a.V, a.in_dtype, a.S, *a.tables, a.status);
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
-    if (t == 0) q->count = 0;
+    if (t < 4) q->count[t] = 0;
     const bool more = bar_or(bar_id, n_threads, leftbits != 0ull);
     if (!more) break;
     if (leftbits != 0ull && tb != nullptr) {
@@ -295,7 +294,7 @@ __global__ void __launch_bounds__(kFfmaThreads) encode_ffma_kernel(EncodeArgs a)
   }
   if (tid == 0) {
     load_fast_quant(a.tables, fq);
-    fixq->count = 0;
+    fixq->count[0] = fixq->count[1] = fixq->count[2] = fixq->count[3] = 0;
   }
   __syncthreads();
   const int r = tid & 127, half = tid >> 7;

@@ -150,14 +150,22 @@ __device__ __forceinline__ void polar_quant_block_fast(const float* y, const Row
 // and patch the code bits in the cache with 32-bit atomics.  The queue is drained in rounds, so a
 // tile with more ambiguous angles than the queue holds only takes more rounds.
 constexpr int kFixCap = 1024;
+// The queue is kept sorted by level (one region per level), so that the four 8-lane groups of a warp,
+// which take consecutive entries, almost always run the same code path.
+__host__ __device__ constexpr int fix_off(int level) { return level == 1 ? 0 : level == 2 ? 512 : level == 3 ? 768 : 896; }
+__host__ __device__ constexpr int fix_cap(int level) { return level == 1 ? 512 : level == 2 ? 256 : 128; }
 
 struct FixQueue {
-  int count;
-  int pad[3];
+  int count[4];            // entries pushed per level (may exceed the capacity: the excess was not stored)
   int64_t xoff[kFixCap];   // element offset of the source vector
   uint8_t* tok[kFixCap];   // token-block base of the destination
   uint32_t meta[kFixCap];  // token-in-block | blk << 6 | level << 9 | j << 12 | (1 = value, 0 = key) << 15
 };
+
+// True if some region is 3/4 full (or has overflowed).
+__device__ __forceinline__ bool fix_should_drain(const FixQueue* q) {
+  return q->count[0] > 384 || q->count[1] > 192 || q->count[2] > 96 || q->count[3] > 96;
+}
 
 // Replace `width` bits at bit offset `bit` of the byte at `addr`.
 __device__ __forceinline__ void patch_bits(uint8_t* addr, int bit, uint32_t mask, uint32_t code) {
@@ -169,21 +177,26 @@ __device__ __forceinline__ void patch_bits(uint8_t* addr, int bit, uint32_t mask
 
 __device__ __forceinline__ void fix_push(FixQueue* q, uint32_t amb, int64_t xoff, uint8_t* tokblock, int tok, int blk,
                                          int kv, uint32_t* left) {
+  uint32_t rest = 0;
   while (amb) {
     const int bit = __ffs(amb) - 1;
-    const int idx = atomicAdd(&q->count, 1);
-    if (idx >= kFixCap) break;  // queue full: keep the rest for the next round
     amb &= amb - 1;
     int level, j;
     if (bit < 8) { level = 1; j = bit; }
     else if (bit < 12) { level = 2; j = bit - 8; }
     else if (bit < 14) { level = 3; j = bit - 12; }
     else { level = 4; j = 0; }
-    q->xoff[idx] = xoff;
-    q->tok[idx] = tokblock;
-    q->meta[idx] = (uint32_t)tok | ((uint32_t)blk << 6) | ((uint32_t)level << 9) | ((uint32_t)j << 12) | ((uint32_t)kv << 15);
+    const int idx = atomicAdd(&q->count[level - 1], 1);
+    if (idx >= fix_cap(level)) {  // this level's region is full: keep the decision for the next round
+      rest |= 1u << bit;
+      continue;
+    }
+    const int e = fix_off(level) + idx;
+    q->xoff[e] = xoff;
+    q->tok[e] = tokblock;
+    q->meta[e] = (uint32_t)tok | ((uint32_t)blk << 6) | ((uint32_t)level << 9) | ((uint32_t)j << 12) | ((uint32_t)kv << 15);
   }
-  *left = amb;
+  *left = rest;
 }
 
 // Exact value of NC consecutive rotated coordinates starting at column c0, for the 8-lane group of
@@ -237,14 +250,17 @@ __device__ __forceinline__ uint32_t exact_code(const double* y, int level, const
   return (uint32_t)(sb > T[0] * sa) + (uint32_t)(sb > T[1] * sa) + (uint32_t)(sb > T[2] * sa);
 }
 
-// Process queue entries [0, n): called by `n_threads` threads (a multiple of 32) with linear index `t`.
-__device__ inline void fix_process(const FixQueue* q, int n, int t, int n_threads, const void* kbase, const void* vbase,
+// Process everything queued, in level order: called by `n_threads` threads (a multiple of 32) with linear index `t`.
+__device__ inline void fix_process(const FixQueue* q, int t, int n_threads, const void* kbase, const void* vbase,
                                    int in_dtype, const float* S, const Tables& tb, int32_t* status) {
   constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock;
   const int sub = t & 7, n_groups = n_threads >> 3;
   const unsigned gmask = 0xFFu << (t & 24);
+  const int n1 = min(q->count[0], fix_cap(1)), n2 = n1 + min(q->count[1], fix_cap(2));
+  const int n3 = n2 + min(q->count[2], fix_cap(3)), n = n3 + min(q->count[3], fix_cap(4));
   int fixed = 0;
-  for (int e = t >> 3; e < n; e += n_groups) {  // uniform within a group of 8 lanes
+  for (int i = t >> 3; i < n; i += n_groups) {  // uniform within a group of 8 lanes
+    const int e = i < n1 ? i : i < n2 ? fix_off(2) + (i - n1) : i < n3 ? fix_off(3) + (i - n2) : fix_off(4) + (i - n3);
     const uint32_t meta = q->meta[e];
     const int64_t xoff = q->xoff[e];
     const int tok = meta & 63, blk = (meta >> 6) & 7, level = (meta >> 9) & 7, j = (meta >> 12) & 7;

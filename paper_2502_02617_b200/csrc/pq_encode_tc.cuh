@@ -144,7 +144,7 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
       tc_mbar_init(bar_tempty + 8 * i, kTcEpiThreads / 32);
     }
     *abort_flag = 0;
-    fixq->count = 0;
+    fixq->count[0] = fixq->count[1] = fixq->count[2] = fixq->count[3] = 0;
     load_fast_quant(a.tables, fq);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -332,7 +332,7 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     // Exact re-decisions are batched over tiles: drain the queue when it is 3/4 full (a push that
     // did not fit leaves the counter above the capacity) or after the CTA's last tile.
     const bool last_tile = tile + (int)gridDim.x >= n_tiles;
-    if (fixq->count > (3 * kFixCap) / 4 || last_tile)
+    if (fix_should_drain(fixq) || last_tile)
       fix_rounds(a, fixq, leftbits, xoff, tb, tok, 2 * cq, kv, tid, kTcEpiThreads, 1);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
