@@ -163,6 +163,33 @@ inline int32_t launch_status() {
   return PQ_ERR_CUDA;
 }
 
+// One-time, per-device launch configuration of a kernel that needs more than 48 KB of dynamic shared
+// memory: the attribute belongs to the (kernel, device) pair, so the memo is indexed by the current
+// device. `state` is a zero-initialised array the caller keeps per kernel; an entry holds the device's
+// SM count once the kernel is configured there. Returns the SM count, or 0 with the CUDA error noted.
+constexpr int kMaxDevices = 64;
+template <typename Kernel>
+inline int configure_for_device(Kernel kernel, int smem_bytes, int (&state)[kMaxDevices]) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess && (dev < 0 || dev >= kMaxDevices)) e = cudaErrorInvalidDevice;
+  if (e != cudaSuccess) {
+    note_cuda_error(e);
+    return 0;
+  }
+  if (state[dev] > 0) return state[dev];
+  int n_sm = 0;
+  e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
+  if (e == cudaSuccess && n_sm <= 0) e = cudaErrorInvalidDevice;
+  if (e != cudaSuccess) {
+    note_cuda_error(e);
+    return 0;
+  }
+  state[dev] = n_sm;
+  return n_sm;
+}
+
 // Record the first error seen.
 __device__ inline void set_status(int32_t* status, int32_t code) {
   if (status != nullptr) atomicCAS(status, 0, code);

@@ -465,26 +465,9 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
   const int g = n_q_heads / n_kv_heads;
   pq::rotate_query_kernel<<<batch * n_q_heads, head_dim, head_dim * sizeof(float), st>>>(a);
   if (head_dim == 128 && batch * n_kv_heads <= pq::kFastMaxUnits) {
-    static bool configured = false;
-    if (!configured) {
-      const cudaError_t e = cudaFuncSetAttribute(pq::decode_attention_fast_kernel,
-                                                 cudaFuncAttributeMaxDynamicSharedMemorySize, pq::kSmTotal);
-      if (e != cudaSuccess) {
-        pq::note_cuda_error(e);
-        return PQ_ERR_CUDA;
-      }
-      configured = true;
-    }
-    static int n_sm = 0;
-    if (n_sm == 0) {
-      int dev = 0;
-      cudaError_t e = cudaGetDevice(&dev);
-      if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-      if (e != cudaSuccess) {
-        pq::note_cuda_error(e);
-        return PQ_ERR_CUDA;
-      }
-    }
+    static int configured[pq::kMaxDevices] = {};
+    const int n_sm = pq::configure_for_device(pq::decode_attention_fast_kernel, pq::kSmTotal, configured);
+    if (n_sm == 0) return PQ_ERR_CUDA;
     const int grid = n_sm < pq::kFastMaxGrid ? n_sm : pq::kFastMaxGrid;
     pq::decode_attention_fast_kernel<<<grid, pq::kFastThreads, pq::kSmTotal, st>>>(a);
     return pq::launch_status();
@@ -515,11 +498,10 @@ int32_t pq_decode_attention_static(int32_t head_dim, int32_t n_q_heads, int32_t 
   const int64_t need = pq_workspace_bytes(head_dim, batch, n_q_heads, n_kv_heads, max_len);
   if (need < 0) return (int32_t)need;
   if (need > PQ_STATIC_SCRATCH_BYTES) return PQ_ERR_SCRATCH;
-  constexpr int kMaxDevices = 64;
-  static void* scratch_of_device[kMaxDevices] = {};
+  static void* scratch_of_device[pq::kMaxDevices] = {};
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
-  if (e != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+  if (e != cudaSuccess || dev < 0 || dev >= pq::kMaxDevices) {
     pq::note_cuda_error(e == cudaSuccess ? cudaErrorInvalidDevice : e);
     return PQ_ERR_CUDA;
   }

@@ -459,15 +459,8 @@ static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
     return launch_status();
   }
   if (a.head_dim == 128 && a.total_tokens >= 32) {
-    static bool configured = false;
-    if (!configured) {
-      const cudaError_t e = cudaFuncSetAttribute(encode_ffma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kFfmaSmem);
-      if (e != cudaSuccess) {
-        note_cuda_error(e);
-        return PQ_ERR_CUDA;
-      }
-      configured = true;
-    }
+    static int configured[kMaxDevices] = {};
+    if (configure_for_device(encode_ffma_kernel, kFfmaSmem, configured) == 0) return PQ_ERR_CUDA;
     dim3 grid((a.total_tokens + 127) / 128, a.n_kv_heads, 2);
     encode_ffma_kernel<<<grid, kFfmaThreads, kFfmaSmem, stream>>>(a);
     advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, lens);

@@ -386,20 +386,9 @@ static int32_t try_launch_encode_tc(const EncodeArgs& a, cudaStream_t stream) {
   TcMaps maps;
   if (!make_x_map(fn, &maps.k, a.K, a.n_kv_heads, a.total_tokens, a.token_stride, a.head_stride)) return 0;
   if (!make_x_map(fn, &maps.v, a.V, a.n_kv_heads, a.total_tokens, a.token_stride, a.head_stride)) return 0;
-  static int n_sm = 0;
-  static bool configured = false;
-  if (!configured) {
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(encode_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmTotal);
-    if (e != cudaSuccess) {
-      note_cuda_error(e);
-      return PQ_ERR_CUDA;
-    }
-    configured = true;
-  }
+  static int configured[kMaxDevices] = {};
+  const int n_sm = configure_for_device(encode_tc_kernel, kTcSmTotal, configured);
+  if (n_sm == 0) return PQ_ERR_CUDA;
   const int n_row_tiles = (a.total_tokens + 127) / 128;
   const int n_tiles = n_row_tiles * 2 * a.n_kv_heads;
   const int grid = n_tiles < n_sm ? n_tiles : n_sm;

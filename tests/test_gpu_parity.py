@@ -218,3 +218,35 @@ def test_mid_size_llama_shape_codes_with_window_accounting():
     out = cache.attend(q)
     torch.cuda.synchronize()
     assert rel_l2(to_f64(out), ref.attend(to_f64(q), d ** -0.5)) < TOL_ATTENTION
+
+
+def _perturbed_codebooks(seed):
+    """A data-fitted-like codebook: the analytic centroids moved a little (still ascending), with
+    midpoint boundaries.  Level 1 is no longer the uniform k*pi/8 grid."""
+    cen, _ = pq.pq_fit_codebooks()
+    rng = np.random.default_rng(seed)
+    c = cen.numpy().copy()
+    c[:16] += rng.uniform(-0.05, 0.05, 16)
+    c[16:] += rng.uniform(-0.02, 0.02, 12)
+    bnd = np.concatenate([0.5 * (c[o:o + n - 1] + c[o + 1:o + n]) for o, n in ((0, 16), (16, 4), (20, 4), (24, 4))])
+    return torch.from_numpy(c), torch.from_numpy(bnd)
+
+
+@pytest.mark.parametrize("n", [5, 40, 300])
+def test_other_codebooks_fp32_inputs_and_strided_views(n):
+    """Paths beside the bf16 tensor-core encoder: a non-uniform level-1 codebook (every level-1 decision is
+    then taken in float64), float32 inputs (FMA rotation), strided K/V views, and chunks of every size class
+    (per-vector kernel < 32 rows, FMA kernel < 128 rows, tensor-core kernel above)."""
+    d, Hq, Hkv = 128, 8, 2
+    for dtype, cbk in ((torch.bfloat16, _perturbed_codebooks(3)), (torch.float32, None), (torch.bfloat16, None)):
+        cache = pq.PolarQuantCache(1, Hq, Hkv, d, capacity=n + 3, seed=9, device=DEV, codebooks=cbk)
+        big_k, big_v = synthetic.kv_like(70 + n, n, Hkv + 1, d + 64, dtype, DEV)
+        K, V = big_k[:, 1:, 32:32 + d], big_v[:, 1:, 32:32 + d]  # views: token stride 3*(d+64), head stride d+64
+        assert not K.is_contiguous()
+        _encode_and_compare(cache, K, V, [n])
+        ref = _oracle_cache(cache, K, V, [n])
+        q = synthetic.queries(n, 1, Hq, d, torch.bfloat16, DEV)
+        out = cache.attend(q)
+        torch.cuda.synchronize()
+        cache.check_status()
+        assert rel_l2(to_f64(out), ref.attend(to_f64(q), d ** -0.5)) < TOL_ATTENTION
