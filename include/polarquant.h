@@ -146,7 +146,9 @@ int32_t pq_append_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, c
  *   q_dev          [batch][n_q_heads][head_dim] of `io_dtype` (PQ_DTYPE_BF16 or PQ_DTYPE_F32)
  *   out_dev        same shape and dtype; accumulation is float32
  *   max_len        host-side upper bound on lens[b] (used only to size the token splits)
- *   workspace_dev  pq_workspace_bytes(...) bytes of scratch; contents need not be preserved
+ *   workspace_dev  pq_workspace_bytes(...) bytes of scratch; it need not be initialised (the split
+ *                  counters inside are tagged with a per-call number) and need not be preserved;
+ *                  two calls that overlap in time must not share it
  * A sequence with lens[b] = 0 yields zeros and records PQ_ERR_EMPTY.
  */
 int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,

@@ -1,4 +1,5 @@
 // Decode attention over the packed cache (Eq. 3) and the inspection kernels.
+#include <atomic>
 #include <math_constants.h>
 
 #include "pq_common.cuh"
@@ -107,7 +108,7 @@ __host__ inline Workspace carve_workspace(void* base, int d, int batch, int n_q_
   w.qrot_l = reinterpret_cast<__half*>(p + off);
   off = align(off + (int64_t)batch * n_q_heads * d * 2);
   w.tickets = reinterpret_cast<int32_t*>(p + off);
-  off = align(off + (int64_t)batch * n_kv_heads * 4);
+  off = align(off + (int64_t)batch * n_kv_heads * 8);  // 8 bytes per unit (the persistent kernel's tagged tickets)
   const int g = n_q_heads / n_kv_heads, units = batch * n_kv_heads;
   w.n_slots = (d == 128 && units <= 2048) ? units + kFastMaxGridHost : units * w.n_splits;
   w.ml = reinterpret_cast<float*>(p + off);
@@ -123,6 +124,7 @@ constexpr int kMaxGroup = 8;  // query heads per kv head handled by one CTA
 struct DecodeArgs {
   int d, n_q_heads, n_kv_heads, batch, capacity, io_dtype;
   float scale;
+  uint32_t epoch;  // differs from call to call (never 0): tags the split tickets of the persistent kernel
   const float* S;
   const Tables* tables;
   const void* q;
@@ -155,27 +157,35 @@ __global__ void rotate_query_kernel(DecodeArgs a) {
 constexpr int kSimpleThreads = 128;
 
 // Shared memory (floats) that combine_and_store needs.
-__host__ __device__ inline int combine_smem_floats(int g, int d, int n_parts) { return g * n_parts + g + g * d; }
+__host__ __device__ inline int combine_smem_floats(int g, int d, int n_parts) { return ((2 * g * n_parts + g + 3) & ~3) + g * d; }
 
 // Merge the `ns` partials (slots slot0 .. slot0 + ns - 1) of the `g` query heads of (b, kv head) in slot
 // order, normalise, rotate back by S^T and store.  Runs in the last CTA that finishes for this
-// (b, kv head); `sm` must hold combine_smem_floats(g, d, ns) floats.
+// (b, kv head); `sm` must hold combine_smem_floats(g, d, ns) floats.  Every phase issues its global
+// loads side by side (the CTA that runs this is the last one still working on the unit).
 __device__ void combine_and_store(const DecodeArgs& a, int b, int hk, int g, int slot0, int ns, float* sm) {
   const int d = a.d, tid = threadIdx.x, nthr = blockDim.x;
-  float* w_sm = sm;               // [g][ns] weight of split s for head h
-  float* linv_sm = sm + g * ns;   // [g]
-  float* o_sm = linv_sm + g;      // [g][d]
+  float* w_sm = sm;                  // [g][ns] running maximum of split s for head h, then its weight
+  float* l_sm = sm + g * ns;         // [g][ns] denominator of split s for head h
+  float* linv_sm = l_sm + g * ns;    // [g]
+  float* o_sm = sm + ((2 * g * ns + g + 3) & ~3);  // [g][d], 16-byte aligned
   const int64_t h0 = (int64_t)b * a.n_q_heads + hk * g;
+  for (int idx = tid; idx < g * ns; idx += nthr) {
+    const int h = idx / ns, s = idx - h * ns;
+    const float2 ml = *reinterpret_cast<const float2*>(a.ws.ml + ((int64_t)(slot0 + s) * g + h) * 2);
+    w_sm[idx] = ml.x;
+    l_sm[idx] = ml.y;
+  }
+  __syncthreads();
   if (tid < g) {
-    const float* ml = a.ws.ml + ((int64_t)slot0 * g + tid) * 2;  // part s at ml[s * g * 2]
     float M = -CUDART_INF_F;
-    for (int s = 0; s < ns; ++s) M = fmaxf(M, ml[(int64_t)s * g * 2]);
+    for (int s = 0; s < ns; ++s) M = fmaxf(M, w_sm[tid * ns + s]);
     float Lsum = 0.f;
-    for (int s = 0; s < ns; ++s) {
-      const float ms = ml[(int64_t)s * g * 2];
+    for (int s = 0; s < ns; ++s) {  // slot order
+      const float ms = w_sm[tid * ns + s];
       const float w = ms == -CUDART_INF_F ? 0.f : exp2f(ms - M);
       w_sm[tid * ns + s] = w;
-      Lsum += ml[(int64_t)s * g * 2 + 1] * w;
+      Lsum += l_sm[tid * ns + s] * w;
     }
     linv_sm[tid] = Lsum > 0.f ? 1.f / Lsum : 0.f;
   }
@@ -184,33 +194,50 @@ __device__ void combine_and_store(const DecodeArgs& a, int b, int hk, int g, int
     const int h = idx / d, j = idx - h * d;
     const float* op = a.ws.o + ((int64_t)slot0 * g + h) * d + j;
     float acc = 0.f;
+#pragma unroll 4
     for (int s = 0; s < ns; ++s) acc = fmaf(op[(int64_t)s * g * d], w_sm[h * ns + s], acc);
     o_sm[idx] = acc * linv_sm[h];
   }
   __syncthreads();
-  // x_hat_i = sum_j y_hat_j S[i][j]: one warp per output row i, lanes over j
+  // x_hat_i = sum_j y_hat_j S[i][j]: a warp takes eight rows i at a time, lanes over j (coalesced), and
+  // has the loads of all eight rows in flight before the first is used.
   const int lane = tid & 31, warp = tid >> 5, nwarps = nthr >> 5;
-  for (int i = warp; i < d; i += nwarps) {
-    float acc[kMaxGroup];
+  constexpr int kRows = 8;
+  for (int i0 = warp * kRows; i0 < d; i0 += nwarps * kRows) {
+    float sv[kRows][4];
 #pragma unroll
-    for (int h = 0; h < kMaxGroup; ++h) acc[h] = 0.f;
-    for (int j = lane; j < d; j += 32) {
-      const float sij = a.S[(int64_t)i * d + j];
+    for (int r = 0; r < kRows; ++r)
 #pragma unroll
-      for (int h = 0; h < kMaxGroup; ++h)
-        if (h < g) acc[h] = fmaf(o_sm[h * d + j], sij, acc[h]);
-    }
+      for (int q = 0; q < 4; ++q) {
+        const int j = lane + 32 * q;
+        sv[r][q] = (i0 + r < d && j < d) ? __ldg(a.S + (int64_t)(i0 + r) * d + j) : 0.f;
+      }
+    for (int h = 0; h < g; ++h) {
+      float ov[4];
 #pragma unroll
-    for (int h = 0; h < kMaxGroup; ++h) {
-      if (h < g) {
-        float v = acc[h];
+      for (int q = 0; q < 4; ++q) ov[q] = lane + 32 * q < d ? o_sm[h * d + lane + 32 * q] : 0.f;
+      float v[kRows];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0) {
-          const int64_t idx = (h0 + h) * d + i;
-          if (a.io_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[idx] = __float2bfloat16(v);
-          else reinterpret_cast<float*>(a.out)[idx] = v;
-        }
+      for (int r = 0; r < kRows; ++r)
+        v[r] = fmaf(ov[3], sv[r][3], fmaf(ov[2], sv[r][2], fmaf(ov[1], sv[r][1], ov[0] * sv[r][0])));
+      // Sum over the 32 lanes: three halving exchanges leave lane L with row L >> 2 (summed over eight
+      // lanes), two more finish it.  9 shuffles per head instead of 40; the order is fixed.
+      float w4[4], w2[2];
+      const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4;
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        w4[k] = (b4 ? v[k + 4] : v[k]) + __shfl_xor_sync(0xffffffffu, b4 ? v[k] : v[k + 4], 16);
+#pragma unroll
+      for (int k = 0; k < 2; ++k)
+        w2[k] = (b3 ? w4[k + 2] : w4[k]) + __shfl_xor_sync(0xffffffffu, b3 ? w4[k] : w4[k + 2], 8);
+      float t = (b2 ? w2[1] : w2[0]) + __shfl_xor_sync(0xffffffffu, b2 ? w2[0] : w2[1], 4);
+      t += __shfl_xor_sync(0xffffffffu, t, 2);
+      t += __shfl_xor_sync(0xffffffffu, t, 1);
+      const int row = i0 + (lane >> 2);
+      if ((lane & 3) == 0 && row < d) {
+        const int64_t oidx = (h0 + h) * d + row;
+        if (a.io_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[oidx] = __float2bfloat16(t);
+        else reinterpret_cast<float*>(a.out)[oidx] = t;
       }
     }
   }
@@ -463,8 +490,11 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
   a.status = status_dev;
   a.ws = pq::carve_workspace(workspace_dev, head_dim, batch, n_q_heads, n_kv_heads, max_len);
   const int g = n_q_heads / n_kv_heads;
-  pq::rotate_query_kernel<<<batch * n_q_heads, head_dim, head_dim * sizeof(float), st>>>(a);
   if (head_dim == 128 && batch * n_kv_heads <= pq::kFastMaxUnits) {
+    // One launch: the persistent kernel rotates the queries itself and needs no cleared tickets.
+    static std::atomic<uint32_t> call_epoch{0};
+    do a.epoch = call_epoch.fetch_add(1u, std::memory_order_relaxed) + 1u;
+    while (a.epoch == 0u);
     static int configured[pq::kMaxDevices] = {};
     const int n_sm = pq::configure_for_device(pq::decode_attention_fast_kernel, pq::kSmTotal, configured);
     if (n_sm == 0) return PQ_ERR_CUDA;
@@ -472,6 +502,8 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
     pq::decode_attention_fast_kernel<<<grid, pq::kFastThreads, pq::kSmTotal, st>>>(a);
     return pq::launch_status();
   }
+  a.epoch = 0u;
+  pq::rotate_query_kernel<<<batch * n_q_heads, head_dim, head_dim * sizeof(float), st>>>(a);
   const pq::Layout L = pq::make_layout(head_dim, capacity);
   size_t smem = 2 * L.block_bytes + sizeof(float) * ((size_t)g * head_dim + 3 * g * pq::kTokenBlock +
                                                      3 * pq::kMaxGroup + 64);

@@ -42,7 +42,8 @@ constexpr int kSmU = kSmT1lo + 256 * 16 * 8;          // 4 * 64 * 16 * 8 = 32768
 constexpr int kSmBar = kSmU + 4 * 64 * 16 * 8;        // full[4], empty[4] : 64
 constexpr int kSmFlags = kSmBar + 64;                 // abort flag, is_last, n_segs : 16
 constexpr int kSmSegs = kSmFlags + 16;                // Segment[32] : 768
-constexpr int kSmRing = (kSmSegs + 768 + 127) / 128 * 128;
+constexpr int kSmQ = kSmSegs + 768;                   // q (fp32) [8][128], q' fp16 value [8][128], q' fp16 residual [8][128] : 8192
+constexpr int kSmRing = (kSmQ + 8192 + 127) / 128 * 128;
 // after the main loop the ring is reused for the cross-warp merge: 16 warps x 8 heads x (128 + 2) floats
 constexpr int kMrgStride = 132;  // floats per (warp, head) row of the merge buffer (132 = 128 + 4: bank spread)
 constexpr int kMergeBytes = 16 * 8 * kMrgStride * 4 + 16 * 8 * 2 * 4;  // also >= combine_smem_floats(8, 128, 160) * 4
@@ -217,6 +218,7 @@ __device__ inline void build_fast_tables(uint8_t* smem, const Tables* tb) {
 // per CTA that works on it; the slots of all units sum to at most units + grid size.
 constexpr int kFastMaxGrid = 160;
 constexpr int kFastMaxUnits = 2048;  // (sequence, kv head) units the persistent schedule handles
+constexpr int kSegmentCost = 5;      // stages' worth of time a CTA spends on starting and finishing a unit
 constexpr int kFastMaxSegs = 32;     // units one CTA can take part in (<= units / grid + 2)
 struct Segment {
   int unit, st0, st1, part, n_parts, slot0;
@@ -243,9 +245,11 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
   __syncthreads();
 
   // ---- persistent work split: the 128-token stages of all units, in unit order, are cut into
-  // gridDim.x equal contiguous ranges; a CTA's range may cover the end of one unit and the start of
-  // the next, and a unit may be shared by several CTAs (its "parts").  Each thread works out one
-  // unit; the units this CTA takes part in are collected in a short list.
+  // gridDim.x contiguous ranges of equal cost; a CTA's range may cover the end of one unit and the
+  // start of the next, and a unit may be shared by several CTAs (its "parts").  Starting on another
+  // unit costs a CTA about kSegmentCost stages (query rotation, refilling the ring, the merge), so
+  // every unit is preceded by that many empty positions on the line that is cut.  Each thread works
+  // out one unit; the units this CTA takes part in are collected in a short list.
   const int n_units = a.batch * a.n_kv_heads, G = gridDim.x, cta = blockIdx.x;
   int* u_nst = reinterpret_cast<int*>(smem + kSmRing);  // [n_units] stages; the ring is idle during set-up
   int* u_parts = u_nst + kFastMaxUnits;                 // [n_units] CTAs that share the unit
@@ -258,13 +262,13 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
   }
   __syncthreads();
   long long w_total = 0;
-  for (int u = 0; u < n_units; ++u) w_total += u_nst[u];
+  for (int u = 0; u < n_units; ++u) w_total += u_nst[u] > 0 ? u_nst[u] + kSegmentCost : 0;
   const long long lo = cta * w_total / G, hi = (cta + 1) * w_total / G;
   for (int u = tid; u < n_units; u += kFastThreads) {
     int parts = 0;
     if (u_nst[u] > 0) {
-      long long start = 0;
-      for (int v = 0; v < u; ++v) start += u_nst[v];
+      long long start = kSegmentCost;  // position of the unit's first stage
+      for (int v = 0; v < u; ++v) start += u_nst[v] > 0 ? u_nst[v] + kSegmentCost : 0;
       const long long end = start + u_nst[u];
       const int c_first = (int)(((start + 1) * G + w_total - 1) / w_total) - 1;  // CTA whose range holds stage `start`
       const int c_last = (int)((end * G + w_total - 1) / w_total) - 1;           // ... stage `end - 1`
@@ -274,7 +278,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
         if (i < kFastMaxSegs) {
           segs[i].unit = u;
           segs[i].st0 = (int)((lo > start ? lo : start) - start);
-          segs[i].st1 = (int)((hi < end ? hi : end) - start);  // may equal st0: a neutral partial is written
+          segs[i].st1 = (int)((hi < end ? hi : end) - start);  // > st0: the CTA's range holds a stage of the unit
           segs[i].part = cta - c_first;
           segs[i].n_parts = parts;
         }
@@ -341,17 +345,42 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
       for (int it = 0; it < kStages - 1 && st0 + it < st1; ++it) issue_copy(it);
     __syncwarp();
     // ---------------------------------------------------------------- consumers
+    // q' = (q S) * scale * log2(e) for the unit's query heads, as an fp16 value plus an fp16 residual.
+    // The first stages of the segment are already on their way while this runs.
+    {
+      float* q_in = reinterpret_cast<float*>(smem + kSmQ);
+      __half* q_hi = reinterpret_cast<__half*>(smem + kSmQ + 4096);
+      __half* q_lo = q_hi + 8 * 128;
+      const int64_t q0 = ((int64_t)b * a.n_q_heads + hk * g_heads) * 128;
+      for (int i = tid; i < g_heads * 128; i += kFastThreads)
+        q_in[i] = a.io_dtype == PQ_DTYPE_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.q)[q0 + i])
+                                              : reinterpret_cast<const float*>(a.q)[q0 + i];
+      __syncthreads();
+      for (int i = tid; i < g_heads * 128; i += kFastThreads) {
+        const float* qrow = q_in + (i & ~127);
+        const float* scol = a.S + (i & 127);
+        float acc = 0.f;
+#pragma unroll 16
+        for (int k = 0; k < 128; ++k) acc = fmaf(qrow[k], __ldg(scol + k * 128), acc);
+        acc *= a.scale * 1.4426950408889634f;
+        const __half qh = __float2half_rn(acc);
+        q_hi[i] = qh;
+        q_lo[i] = __float2half_rn(acc - __half2float(qh));
+      }
+      __syncthreads();
+    }
     // q' fragments: A operand (16 rows x 16 coords per k-step): rows 0..7 the fp16 values, rows 8..15 the residuals.
     // k-step ks covers, for thread c, sub-block (ks & 3) of block 2c + (ks >> 2).
     uint32_t qa[8][2], ql[8][2];  // fp16 value and fp16 residual of q'
     {
-      const int64_t qoff = ((int64_t)b * a.n_q_heads + hk * g_heads + g) * 128 + 32 * c;
+      const uint2* q_hi = reinterpret_cast<const uint2*>(smem + kSmQ + 4096) + (g * 128 + 32 * c) / 4;
+      const uint2* q_lo = q_hi + 8 * 128 / 4;
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
         uint2 v = make_uint2(0u, 0u), w = make_uint2(0u, 0u);
         if (g < g_heads) {
-          v = *reinterpret_cast<const uint2*>(a.ws.qrot_h + qoff + 4 * ks);
-          w = *reinterpret_cast<const uint2*>(a.ws.qrot_l + qoff + 4 * ks);
+          v = q_hi[ks];
+          w = q_lo[ks];
         }
         // decoded keys come as (coord 0, coord 2), (coord 1, coord 3) of each sub-block: permute q' to match
         qa[ks][0] = __byte_perm(v.x, v.y, 0x5410);
@@ -517,8 +546,24 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-      const int t = atomicAdd(a.ws.tickets + u, 1);
-      *is_last = (t == n_parts - 1);
+      // Arrival count of the unit's parts.  The workspace is not assumed to start at zero: a ticket
+      // holds (call epoch << 32 | arrivals), and a ticket of another epoch counts as zero arrivals.
+      bool last = true;
+      if (n_parts > 1) {
+        unsigned long long* tk = reinterpret_cast<unsigned long long*>(a.ws.tickets) + u;
+        unsigned long long cur = *reinterpret_cast<volatile unsigned long long*>(tk), want = 0ull;
+        bool done = false;
+        for (int i = 0; i < 4096 && !done; ++i) {  // every failed attempt is another part's success: <= n_parts rounds
+          want = (uint32_t)(cur >> 32) == a.epoch ? cur + 1ull : ((unsigned long long)a.epoch << 32) | 1ull;
+          const unsigned long long prev = atomicCAS(tk, cur, want);
+          done = prev == cur;
+          cur = prev;
+        }
+        if (!done) set_status(a.status, PQ_ERR_TIMEOUT);
+        last = done && (int)(want & 0xffffffffull) == n_parts;
+        if (last) *tk = 0ull;  // no other part of this call touches it any more
+      }
+      *is_last = last;
     }
     __syncthreads();
     if (*is_last) {
