@@ -247,10 +247,11 @@ __device__ __forceinline__ bool bar_or(int bar_id, int n_threads, bool v) {
 // `leftbits` holds this thread's decisions that found the queue full (15 bits per block, up to 4 blocks
 // starting at block `blk0`).
 __device__ inline void fix_rounds(const EncodeArgs& a, FixQueue* q, unsigned long long leftbits, int64_t xoff, uint8_t* tb,
-                                  int tok, int blk0, int kv, int t, int n_threads, int bar_id) {
+                                  int tok, int blk0, int kv, int t, int n_threads, int bar_id,
+                                  const double* Sd = nullptr) {
   for (int round = 0; round < 256; ++round) {
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
-    fix_process(q, t, n_threads, a.K, a.V, a.in_dtype, a.S, *a.tables, a.status);
+    fix_process(q, t, n_threads, a.K, a.V, a.in_dtype, a.S, Sd, *a.tables, a.status);
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
     if (t < 4) q->count[t] = 0;
     const bool more = bar_or(bar_id, n_threads, leftbits != 0ull);

@@ -235,6 +235,37 @@ __device__ __forceinline__ void exact_coords(const double* xk, const float* S, i
   }
 }
 
+// The same sums with S staged in shared memory as float64 (no conversions, no L2 latency in the loop).
+// Row k of S sits at row (k & 15) * 8 + (k >> 4) of `Sd`, rows kFixSdStride doubles apart, so the eight
+// lanes of a group (k = 16 * sub + i) read eight consecutive rows: 16-byte loads without bank conflicts.
+constexpr int kFixSdStride = 130;
+constexpr int kFixSdBytes = 128 * kFixSdStride * 8;
+template <int NC>
+__device__ __forceinline__ void exact_coords_sm(const double* xk, const double* Sd, int sub, int c0, unsigned gmask,
+                                                double* y) {
+  double acc[NC];
+#pragma unroll
+  for (int c = 0; c < NC; ++c) acc[c] = 0.0;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const double2* srow = reinterpret_cast<const double2*>(Sd + (i * 8 + sub) * kFixSdStride + c0);
+#pragma unroll
+    for (int c2 = 0; c2 < NC / 2; ++c2) {
+      const double2 s2 = srow[c2];
+      acc[2 * c2] = fma(xk[i], s2.x, acc[2 * c2]);
+      acc[2 * c2 + 1] = fma(xk[i], s2.y, acc[2 * c2 + 1]);
+    }
+  }
+#pragma unroll
+  for (int c = 0; c < NC; ++c) {
+    double p = acc[c];
+    p += __shfl_xor_sync(gmask, p, 1);
+    p += __shfl_xor_sync(gmask, p, 2);
+    p += __shfl_xor_sync(gmask, p, 4);
+    y[c] = p;
+  }
+}
+
 // Decision of one angle of level log2(NC) from the exact coordinates under it.  Levels >= 2 compare
 // the squared child radii, sb > tan^2(beta) sa, which is the same decision as atan2(r_b, r_a) > beta.
 template <int NC>
@@ -251,39 +282,66 @@ __device__ __forceinline__ uint32_t exact_code(const double* y, int level, const
 }
 
 // Process everything queued, in level order: called by `n_threads` threads (a multiple of 32) with linear index `t`.
+// `Sd` (may be null) is S staged in shared memory for exact_coords_sm.
 __device__ inline void fix_process(const FixQueue* q, int t, int n_threads, const void* kbase, const void* vbase,
-                                   int in_dtype, const float* S, const Tables& tb, int32_t* status) {
+                                   int in_dtype, const float* S, const double* Sd, const Tables& tb, int32_t* status) {
   constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock;
   const int sub = t & 7, n_groups = n_threads >> 3;
   const unsigned gmask = 0xFFu << (t & 24);
   const int n1 = min(q->count[0], fix_cap(1)), n2 = n1 + min(q->count[1], fix_cap(2));
   const int n3 = n2 + min(q->count[2], fix_cap(3)), n = n3 + min(q->count[3], fix_cap(4));
   int fixed = 0;
+  auto entry_of = [&](int i) {
+    return i < n1 ? i : i < n2 ? fix_off(2) + (i - n1) : i < n3 ? fix_off(3) + (i - n2) : fix_off(4) + (i - n3);
+  };
+  // The source vector of the group's next entry is fetched while the current one is decided.
+  auto fetch = [&](int i, uint4* raw) {
+    if (i >= n || in_dtype != PQ_DTYPE_BF16) return;
+    const int e = entry_of(i);
+    const void* xbase = (q->meta[e] >> 15) & 1 ? vbase : kbase;
+    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(xbase) + q->xoff[e] + 16 * sub);
+    raw[0] = __ldg(p);
+    raw[1] = __ldg(p + 1);
+  };
+  uint4 raw[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
+  fetch(t >> 3, raw);
   for (int i = t >> 3; i < n; i += n_groups) {  // uniform within a group of 8 lanes
-    const int e = i < n1 ? i : i < n2 ? fix_off(2) + (i - n1) : i < n3 ? fix_off(3) + (i - n2) : fix_off(4) + (i - n3);
+    const int e = entry_of(i);
     const uint32_t meta = q->meta[e];
-    const int64_t xoff = q->xoff[e];
     const int tok = meta & 63, blk = (meta >> 6) & 7, level = (meta >> 9) & 7, j = (meta >> 12) & 7;
     const int c0 = blk * 16 + (j << level);
-    const void* xbase = (meta >> 15) & 1 ? vbase : kbase;
     double xk[16];  // this lane's 16 consecutive k
     if (in_dtype == PQ_DTYPE_BF16) {
-      const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(xbase) + xoff + 16 * sub);
-      const uint4 v0 = p[0], v1 = p[1];
-      const uint32_t w[8] = {v0.x, v0.y, v0.z, v0.w, v1.x, v1.y, v1.z, v1.w};
+      const uint32_t w[8] = {raw[0].x, raw[0].y, raw[0].z, raw[0].w, raw[1].x, raw[1].y, raw[1].z, raw[1].w};
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        xk[2 * i] = (double)__uint_as_float(w[i] << 16);
-        xk[2 * i + 1] = (double)__uint_as_float(w[i] & 0xFFFF0000u);
+      for (int i2 = 0; i2 < 8; ++i2) {
+        xk[2 * i2] = (double)__uint_as_float(w[i2] << 16);
+        xk[2 * i2 + 1] = (double)__uint_as_float(w[i2] & 0xFFFF0000u);
       }
+      fetch(i + n_groups, raw);
     } else {
-      const float* p = reinterpret_cast<const float*>(xbase) + xoff + 16 * sub;
+      const void* xbase = (meta >> 15) & 1 ? vbase : kbase;
+      const float* p = reinterpret_cast<const float*>(xbase) + q->xoff[e] + 16 * sub;
 #pragma unroll
-      for (int i = 0; i < 16; ++i) xk[i] = (double)p[i];
+      for (int i2 = 0; i2 < 16; ++i2) xk[i2] = (double)p[i2];
     }
     double y[16];
     uint32_t code;
-    if (level == 1) {
+    if (Sd != nullptr) {  // uniform over the CTA
+      if (level == 1) {
+        exact_coords_sm<2>(xk, Sd, sub, c0, gmask, y);
+        code = exact_code<2>(y, level, tb);
+      } else if (level == 2) {
+        exact_coords_sm<4>(xk, Sd, sub, c0, gmask, y);
+        code = exact_code<4>(y, level, tb);
+      } else if (level == 3) {
+        exact_coords_sm<8>(xk, Sd, sub, c0, gmask, y);
+        code = exact_code<8>(y, level, tb);
+      } else {
+        exact_coords_sm<16>(xk, Sd, sub, c0, gmask, y);
+        code = exact_code<16>(y, level, tb);
+      }
+    } else if (level == 1) {
       exact_coords<2>(xk, S, sub, c0, gmask, y);
       code = exact_code<2>(y, level, tb);
     } else if (level == 2) {

@@ -37,6 +37,7 @@ constexpr int kTcSmMisc = kTcSmBar + 128;                    // tmem base, abort
 constexpr int kTcSmFix = kTcSmMisc + 64;                     // FixQueue
 constexpr int kTcSmTotal = kTcSmFix + (int)sizeof(FixQueue) + 1024;  // + slack for 1024-byte alignment
 constexpr int kTcSpin = 1 << 22;
+static_assert(kFixSdBytes <= kTcSmRowSq, "the float64 copy of S must fit in the operand buffers");
 
 __device__ __forceinline__ uint32_t tc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void tc_mbar_init(uint32_t bar, uint32_t count) {
@@ -261,7 +262,8 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
       for (int c = 0; c < 32; ++c) sq = fmaf(y[c], y[c], sq);
     }
     rowsq[cq * 128 + r] = sq;
-    asm volatile("bar.sync 1, 512;" ::: "memory");
+    // only the four warps that share these 32 rows exchange their parts of the norm
+    asm volatile("bar.sync %0, 128;" ::"r"(2 + quarter) : "memory");
     const RowMargins rm = make_row_margins(
         kRotErr * 1.0001f * sqrtf((rowsq[r] + rowsq[128 + r]) + (rowsq[256 + r] + rowsq[384 + r])), *fq);
     const int row = rt * 128 + r;
@@ -332,8 +334,19 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     // Exact re-decisions are batched over tiles: drain the queue when it is 3/4 full (a push that
     // did not fit leaves the counter above the capacity) or after the CTA's last tile.
     const bool last_tile = tile + (int)gridDim.x >= n_tiles;
-    if (fix_should_drain(fixq) || last_tile)
+    if (last_tile) {
+      // The operand buffers are idle now (every MMA and copy of this CTA has completed): stage S there as
+      // float64 so that the last, largest batch of re-decisions reads it from shared memory.
+      asm volatile("bar.sync 1, 512;" ::: "memory");
+      double* Sd = reinterpret_cast<double*>(smem + kTcSmS);
+      for (int idx = tid; idx < 128 * 128; idx += kTcThreads) {
+        const int k = idx >> 7, n = idx & 127;
+        Sd[((k & 15) * 8 + (k >> 4)) * kFixSdStride + n] = (double)__ldg(a.S + idx);
+      }
+      fix_rounds(a, fixq, leftbits, xoff, tb, tok, 2 * cq, kv, tid, kTcEpiThreads, 1, Sd);
+    } else if (fix_should_drain(fixq)) {
       fix_rounds(a, fixq, leftbits, xoff, tb, tok, 2 * cq, kv, tid, kTcEpiThreads, 1);
+    }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
