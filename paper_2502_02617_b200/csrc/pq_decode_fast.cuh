@@ -47,7 +47,13 @@ constexpr int kSmRing = (kSmQ + 8192 + 127) / 128 * 128;
 // after the main loop the ring is reused for the cross-warp merge: 16 warps x 8 heads x (128 + 2) floats
 constexpr int kMrgStride = 132;  // floats per (warp, head) row of the merge buffer (132 = 128 + 4: bank spread)
 constexpr int kMergeBytes = 16 * 8 * kMrgStride * 4 + 16 * 8 * 2 * 4;  // also >= combine_smem_floats(8, 128, 160) * 4
-constexpr int kSmTotal = kSmRing + (kStages * kStageBytes > kMergeBytes ? kStages * kStageBytes : kMergeBytes);
+constexpr int kSmUsed = kSmRing + (kStages * kStageBytes > kMergeBytes ? kStages * kStageBytes : kMergeBytes);
+// The tables start on a 32 KB boundary of the shared window, so that a table address is the OR of
+// disjoint bit fields (base | lane replica | index) and needs no addition; the launch asks for 32 KB
+// of slack to place them.
+constexpr int kSmAlign = 32768;
+constexpr int kSmTotal = kSmUsed + kSmAlign;
+static_assert(kSmT1p == 0 && kSmT1lo == 32768 && kSmU == 65536, "table addresses are formed with OR");
 static_assert(kSmRing % 128 == 0, "ring must be 128-byte aligned");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -101,6 +107,18 @@ __device__ __forceinline__ uint2 lds64(uint32_t addr) {
   asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
   return v;
 }
+template <int kOff>
+__device__ __forceinline__ uint32_t lds32i(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(kOff));
+  return v;
+}
+template <int kOff>
+__device__ __forceinline__ uint2 lds64i(uint32_t addr) {
+  uint2 v;
+  asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+%3];" : "=r"(v.x), "=r"(v.y) : "r"(addr), "n"(kOff));
+  return v;
+}
 __device__ __forceinline__ uint32_t lds16(uint32_t addr) {
   uint16_t v;
   asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
@@ -130,15 +148,20 @@ __device__ __forceinline__ void mma_1688(float* d, uint32_t a0, uint32_t a1, uin
                : "r"(a0), "r"(a1), "r"(b0));
 }
 
-// Byte offsets of the four sub-block entries of a block in the replicated u table
-// (entry idx at idx * 128: c2_s -> bits 7..8, c3 -> bits 9..10, c4 -> bits 11..12).
-__device__ __forceinline__ void u_offsets(uint32_t c2, uint32_t c3n, uint32_t c4, uint32_t* off) {
-  const uint32_t a4 = c4 << 11;
+// Addresses of the four sub-block entries of a block in the replicated u table, less s * 8192 (the
+// loads add that as an immediate).  Entry idx sits at idx * 128: c2_s -> bits 7..8, c3 -> bits 9..10,
+// c4 -> bits 11..12; `ub` = table base | lane replica has none of these bits set.
+__device__ __forceinline__ void u_offsets(uint32_t c2, uint32_t c3n, uint32_t c4, uint32_t ub, uint32_t* off) {
+  const uint32_t a4 = c4 * 2048u + ub;
   const uint32_t hi0 = ((c3n << 9) & 0x600u) | a4, hi1 = ((c3n << 7) & 0x600u) | a4;
-  off[0] = 0 * 8192 + (((c2 << 7) & 0x180u) | hi0);
-  off[1] = 1 * 8192 + (((c2 << 5) & 0x180u) | hi0);
-  off[2] = 2 * 8192 + (((c2 << 3) & 0x180u) | hi1);
-  off[3] = 3 * 8192 + (((c2 << 1) & 0x180u) | hi1);
+  off[0] = ((c2 << 7) & 0x180u) | hi0;
+  off[1] = ((c2 << 5) & 0x180u) | hi0;
+  off[2] = ((c2 << 3) & 0x180u) | hi1;
+  off[3] = ((c2 << 1) & 0x180u) | hi1;
+}
+template <int kS>
+__device__ __forceinline__ uint32_t t1_address(uint32_t l1, uint32_t t1) {  // byte kS of l1 -> bits 7..14
+  return ((kS == 0 ? (l1 << 7) : (l1 >> (8 * kS - 7))) & 0x7F80u) | t1;
 }
 
 // DeQuant of one 16-coordinate block in the rotated basis, fp16 path.  For sub-block s (coordinates
@@ -150,15 +173,17 @@ __device__ __forceinline__ void u_offsets(uint32_t c2, uint32_t c3n, uint32_t c4
 __device__ __forceinline__ void decode_block_h2(uint32_t l1, uint32_t c2, uint32_t c3n, uint32_t c4, __half2 r2,
                                                 uint32_t sm_base, uint32_t rep, __half2* out) {
   uint32_t off[4];
-  u_offsets(c2, c3n, c4, off);
-  const uint32_t ub = sm_base + kSmU + rep, t1 = sm_base + kSmT1p + rep;
-#pragma unroll
-  for (int s = 0; s < 4; ++s) {
-    const __half2 u = __hmul2(r2, as_h2(lds32(ub + off[s])));
-    const uint2 e = lds64(t1 + ((s == 0 ? (l1 << 7) : (l1 >> (8 * s - 7))) & 0x7F80u));
-    out[2 * s] = __hmul2(u, as_h2(e.x));
-    out[2 * s + 1] = __hmul2(u, as_h2(e.y));
+  const uint32_t t1 = sm_base + kSmT1p + rep;
+  u_offsets(c2, c3n, c4, sm_base + kSmU + rep, off);
+#define PQ_SUB(S)                                                               \
+  {                                                                             \
+    const __half2 u = __hmul2(r2, as_h2(lds32i<(S) * 8192>(off[S])));           \
+    const uint2 e = lds64i<0>(t1_address<S>(l1, t1));                           \
+    out[2 * (S)] = __hmul2(u, as_h2(e.x));                                      \
+    out[2 * (S) + 1] = __hmul2(u, as_h2(e.y));                                  \
   }
+  PQ_SUB(0) PQ_SUB(1) PQ_SUB(2) PQ_SUB(3)
+#undef PQ_SUB
 }
 
 // The same block as an unevaluated sum hi + lo of fp16 values (about 21 significant bits):
@@ -168,21 +193,25 @@ __device__ __forceinline__ void decode_block_h2(uint32_t l1, uint32_t c2, uint32
 __device__ __forceinline__ void decode_block_hilo(uint32_t l1, uint32_t c2, uint32_t c3n, uint32_t c4, __half2 r2,
                                                   uint32_t sm_base, uint32_t rep, __half2* hi, __half2* lo) {
   uint32_t off[4];
-  u_offsets(c2, c3n, c4, off);
-  const uint32_t ub = sm_base + kSmU + rep, t1 = sm_base + kSmT1p + rep;
-#pragma unroll
-  for (int s = 0; s < 4; ++s) {
-    const uint2 uu = lds64(ub + off[s]);
-    const __half2 u_hi = __hmul2(r2, as_h2(uu.x));
-    const __half2 u_lo = __hfma2(r2, as_h2(uu.y), __hfma2(r2, as_h2(uu.x), __hneg2(u_hi)));
-    const uint32_t idx = (s == 0 ? (l1 << 7) : (l1 >> (8 * s - 7))) & 0x7F80u;
-    const uint2 th = lds64(t1 + idx), tl = lds64(t1 + (kSmT1lo - kSmT1p) + idx);
-    const __half2 kx = __hmul2(u_hi, as_h2(th.x)), ky = __hmul2(u_hi, as_h2(th.y));
-    hi[2 * s] = kx;
-    hi[2 * s + 1] = ky;
-    lo[2 * s] = __hfma2(u_hi, as_h2(tl.x), __hfma2(u_lo, as_h2(th.x), __hfma2(u_hi, as_h2(th.x), __hneg2(kx))));
-    lo[2 * s + 1] = __hfma2(u_hi, as_h2(tl.y), __hfma2(u_lo, as_h2(th.y), __hfma2(u_hi, as_h2(th.y), __hneg2(ky))));
+  const uint32_t t1 = sm_base + kSmT1p + rep;
+  u_offsets(c2, c3n, c4, sm_base + kSmU + rep, off);
+#define PQ_SUB(S)                                                                                                  \
+  {                                                                                                                \
+    const uint2 uu = lds64i<(S) * 8192>(off[S]);                                                                   \
+    const __half2 u_hi = __hmul2(r2, as_h2(uu.x));                                                                 \
+    const __half2 u_lo = __hfma2(r2, as_h2(uu.y), __hfma2(r2, as_h2(uu.x), __hneg2(u_hi)));                        \
+    const uint32_t ta = t1_address<S>(l1, t1);                                                                     \
+    const uint2 th = lds64i<0>(ta), tl = lds64i<kSmT1lo - kSmT1p>(ta);                                             \
+    const __half2 kx = __hmul2(u_hi, as_h2(th.x)), ky = __hmul2(u_hi, as_h2(th.y));                                \
+    hi[2 * (S)] = kx;                                                                                              \
+    hi[2 * (S) + 1] = ky;                                                                                          \
+    lo[2 * (S)] =                                                                                                  \
+        __hfma2(u_hi, as_h2(tl.x), __hfma2(u_lo, as_h2(th.x), __hfma2(u_hi, as_h2(th.x), __hneg2(kx))));           \
+    lo[2 * (S) + 1] =                                                                                              \
+        __hfma2(u_hi, as_h2(tl.y), __hfma2(u_lo, as_h2(th.y), __hfma2(u_hi, as_h2(th.y), __hneg2(ky))));           \
   }
+  PQ_SUB(0) PQ_SUB(1) PQ_SUB(2) PQ_SUB(3)
+#undef PQ_SUB
 }
 
 // plane offsets of a d = 128 token-block
@@ -225,7 +254,8 @@ struct Segment {
 };
 
 __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(DecodeArgs a) {
-  extern __shared__ __align__(128) uint8_t smem[];
+  extern __shared__ __align__(128) uint8_t smem_raw[];
+  uint8_t* smem = smem_raw + ((kSmAlign - (smem_u32(smem_raw) & (kSmAlign - 1))) & (kSmAlign - 1));
   const int g_heads = a.n_q_heads / a.n_kv_heads;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const uint32_t sm_base = smem_u32(smem);
