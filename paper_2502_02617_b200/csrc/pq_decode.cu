@@ -495,11 +495,13 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
     static std::atomic<uint32_t> call_epoch{0};
     do a.epoch = call_epoch.fetch_add(1u, std::memory_order_relaxed) + 1u;
     while (a.epoch == 0u);
-    static int configured[pq::kMaxDevices] = {};
-    const int n_sm = pq::configure_for_device(pq::decode_attention_fast_kernel, pq::kSmTotal, configured);
+    static int configured4[pq::kMaxDevices] = {}, configured8[pq::kMaxDevices] = {};
+    const int n_sm = g <= 4 ? pq::configure_for_device(pq::decode_attention_fast_kernel<1>, pq::kSmTotal, configured4)
+                            : pq::configure_for_device(pq::decode_attention_fast_kernel<2>, pq::kSmTotal, configured8);
     if (n_sm == 0) return PQ_ERR_CUDA;
     const int grid = n_sm < pq::kFastMaxGrid ? n_sm : pq::kFastMaxGrid;
-    pq::decode_attention_fast_kernel<<<grid, pq::kFastThreads, pq::kSmTotal, st>>>(a);
+    if (g <= 4) pq::decode_attention_fast_kernel<1><<<grid, pq::kFastThreads, pq::kSmTotal, st>>>(a);
+    else pq::decode_attention_fast_kernel<2><<<grid, pq::kFastThreads, pq::kSmTotal, st>>>(a);
     return pq::launch_status();
   }
   a.epoch = 0u;

@@ -1,15 +1,16 @@
 // Fast decode-attention kernel for head_dim 128 (included by pq_decode.cu).
 //
-// One CTA of 16 warps per (token split, kv head, sequence).  128-token stages of the packed cache
-// (K block, V block, K block, V block: one contiguous 15872-byte bulk copy) stream through a
-// shared-memory ring; one elected thread issues the copies three stages ahead, and each warp
-// takes one 8-token tile of every stage.  (16 warps, not 17: the register file is split over four
-// schedulers, and a fifth warp on one of them would cap every thread at 96 registers.)
+// Persistent CTAs of 16 warps, each with a contiguous share of the (sequence, kv head) token streams.
+// 128-token stages of the packed cache (K block, V block, K block, V block: one contiguous 15872-byte
+// bulk copy) stream through a shared-memory ring.  The warps form two groups of 8 that take alternate
+// stages; each group has two ring slots and one thread that issues its copies a stage ahead; each warp
+// takes one 16-token tile of its group's stage.  (16 warps, not 17: the register file is split over
+// four schedulers, and a fifth warp on one of them would cap every thread at 96 registers.)
 //
 // Per tile a warp
-//   * decodes the keys straight into mma.sync B fragments (fp16, rotated basis) with
-//     shared-memory table lookups, and forms S^T = q' K_hat^T (heads x tokens) on tensor cores,
-//   * runs the online softmax on the S^T fragment (log2 domain, fp32),
+//   * decodes the keys of 16 tokens straight into mma.sync A fragments (fp16, rotated basis) with
+//     shared-memory table lookups, and forms S = K_hat q'^T (tokens x heads) on tensor cores,
+//   * runs the online softmax on the S fragment (log2 domain, fp32),
 //   * decodes the values into A fragments (coordinates x tokens) and accumulates
 //     O^T += V_hat^T P on tensor cores (fp32 accumulators in registers).
 // DeQuant (Algorithm 1) of one 16-coordinate block is a product tree r * t4 * t3 * t2 * t1.
@@ -32,7 +33,7 @@ constexpr int kFastThreads = kFastConsumerWarps * 32;
 constexpr int kStageTokens = 2 * kTokenBlock;       // 128
 constexpr int kBlockBytes128 = 62 * kTokenBlock;    // 3968: one K or V token-block at d = 128
 constexpr int kStageBytes = 4 * kBlockBytes128;     // 15872
-constexpr int kStages = 4;
+constexpr int kStages = 4;                          // two per group of 8 warps
 constexpr int kSpinLimit = 1 << 22;
 
 // shared-memory map (bytes)
@@ -148,70 +149,62 @@ __device__ __forceinline__ void mma_1688(float* d, uint32_t a0, uint32_t a1, uin
                : "r"(a0), "r"(a1), "r"(b0));
 }
 
-// Addresses of the four sub-block entries of a block in the replicated u table, less s * 8192 (the
-// loads add that as an immediate).  Entry idx sits at idx * 128: c2_s -> bits 7..8, c3 -> bits 9..10,
-// c4 -> bits 11..12; `ub` = table base | lane replica has none of these bits set.
-__device__ __forceinline__ void u_offsets(uint32_t c2, uint32_t c3n, uint32_t c4, uint32_t ub, uint32_t* off) {
-  const uint32_t a4 = c4 * 2048u + ub;
-  const uint32_t hi0 = ((c3n << 9) & 0x600u) | a4, hi1 = ((c3n << 7) & 0x600u) | a4;
-  off[0] = ((c2 << 7) & 0x180u) | hi0;
-  off[1] = ((c2 << 5) & 0x180u) | hi0;
-  off[2] = ((c2 << 3) & 0x180u) | hi1;
-  off[3] = ((c2 << 1) & 0x180u) | hi1;
+// Codes of one 16-coordinate block of one token, prepared for the table lookups.  Entry idx of the
+// replicated u table of sub-block s sits at s * 8192 + idx * 128 with idx = c2_s | c3 << 2 | c4 << 4, i.e.
+// c2_s -> address bits 7..8, c3 -> bits 9..10, c4 -> bits 11..12; `ub` = table base | lane replica has
+// none of these bits set, so the address is an OR (the loads add s * 8192 as an immediate).
+struct BlockRef {
+  uint32_t l1;        // 8 level-1 codes, code j at bits [4j, 4j+4)
+  uint32_t c2;        // 4 level-2 codes in bits 0..7 (higher bits are ignored)
+  uint32_t hi0, hi1;  // ub | c4 | level-3 code of sub-blocks 0-1 / 2-3, in address position
+  __half2 r2;         // the block radius in both halves
+};
+__device__ __forceinline__ BlockRef make_block_ref(uint32_t l1, uint32_t c2, uint32_t c3n, uint32_t c4_clean, __half2 r2,
+                                                   uint32_t ub) {
+  BlockRef b;
+  const uint32_t a4 = c4_clean * 2048u + ub;
+  b.l1 = l1;
+  b.c2 = c2;
+  b.hi0 = ((c3n << 9) & 0x600u) | a4;
+  b.hi1 = ((c3n << 7) & 0x600u) | a4;
+  b.r2 = r2;
+  return b;
+}
+template <int kS>
+__device__ __forceinline__ uint32_t u_address(const BlockRef& b) {
+  return ((kS == 3 ? (b.c2 << 1) : (b.c2 << (7 - 2 * kS))) & 0x180u) | (kS < 2 ? b.hi0 : b.hi1);
 }
 template <int kS>
 __device__ __forceinline__ uint32_t t1_address(uint32_t l1, uint32_t t1) {  // byte kS of l1 -> bits 7..14
   return ((kS == 0 ? (l1 << 7) : (l1 >> (8 * kS - 7))) & 0x7F80u) | t1;
 }
 
-// DeQuant of one 16-coordinate block in the rotated basis, fp16 path.  For sub-block s (coordinates
-// 4s .. 4s+3, level-1 pairs a = 2s and b = 2s+1) the result is two half2:
-//   out[2s]   = (x_a, x_b) = coordinates (4s, 4s+2)        out[2s+1] = (y_a, y_b) = coordinates (4s+1, 4s+3)
-//   l1 : 8 level-1 codes, code j at bits [4j, 4j+4)     c2 : 4 level-2 codes, 2 bits each (clean)
-//   c3n: 2 level-3 codes in a nibble (clean)             c4 : the level-4 code (clean)
-//   r2 : the block radius in both halves                 rep: (lane & 15) * 8
-__device__ __forceinline__ void decode_block_h2(uint32_t l1, uint32_t c2, uint32_t c3n, uint32_t c4, __half2 r2,
-                                                uint32_t sm_base, uint32_t rep, __half2* out) {
-  uint32_t off[4];
-  const uint32_t t1 = sm_base + kSmT1p + rep;
-  u_offsets(c2, c3n, c4, sm_base + kSmU + rep, off);
-#define PQ_SUB(S)                                                               \
-  {                                                                             \
-    const __half2 u = __hmul2(r2, as_h2(lds32i<(S) * 8192>(off[S])));           \
-    const uint2 e = lds64i<0>(t1_address<S>(l1, t1));                           \
-    out[2 * (S)] = __hmul2(u, as_h2(e.x));                                      \
-    out[2 * (S) + 1] = __hmul2(u, as_h2(e.y));                                  \
-  }
-  PQ_SUB(0) PQ_SUB(1) PQ_SUB(2) PQ_SUB(3)
-#undef PQ_SUB
+// DeQuant (Algorithm 1) of sub-block kS (coordinates 4 kS .. 4 kS + 3, level-1 pairs a = 2 kS and
+// b = 2 kS + 1) of a block in the rotated basis, fp16:  x = (x_a, x_b) = coordinates (4 kS, 4 kS + 2),
+// y = (y_a, y_b) = coordinates (4 kS + 1, 4 kS + 3).  `t1` = level-1 table base | lane replica.
+template <int kS>
+__device__ __forceinline__ void sub_block_h2(const BlockRef& b, uint32_t t1, __half2& x, __half2& y) {
+  const __half2 u = __hmul2(b.r2, as_h2(lds32i<kS * 8192>(u_address<kS>(b))));
+  const uint2 e = lds64i<0>(t1_address<kS>(b.l1, t1));
+  x = __hmul2(u, as_h2(e.x));
+  y = __hmul2(u, as_h2(e.y));
 }
-
-// The same block as an unevaluated sum hi + lo of fp16 values (about 21 significant bits):
+// The same sub-block as an unevaluated sum hi + lo of fp16 values (about 21 significant bits):
 //   u = r * (Uhi + Ulo)            u_hi = rn(r Uhi),  u_lo = fma(r, Uhi, -u_hi) + r Ulo
 //   k = (u_hi + u_lo)(thi + tlo)   k_hi = rn(u_hi thi), k_lo = fma(u_hi, thi, -k_hi) + u_lo thi + u_hi tlo
 // (fp16 fused multiply-adds return the exact rounding residual of a product).
-__device__ __forceinline__ void decode_block_hilo(uint32_t l1, uint32_t c2, uint32_t c3n, uint32_t c4, __half2 r2,
-                                                  uint32_t sm_base, uint32_t rep, __half2* hi, __half2* lo) {
-  uint32_t off[4];
-  const uint32_t t1 = sm_base + kSmT1p + rep;
-  u_offsets(c2, c3n, c4, sm_base + kSmU + rep, off);
-#define PQ_SUB(S)                                                                                                  \
-  {                                                                                                                \
-    const uint2 uu = lds64i<(S) * 8192>(off[S]);                                                                   \
-    const __half2 u_hi = __hmul2(r2, as_h2(uu.x));                                                                 \
-    const __half2 u_lo = __hfma2(r2, as_h2(uu.y), __hfma2(r2, as_h2(uu.x), __hneg2(u_hi)));                        \
-    const uint32_t ta = t1_address<S>(l1, t1);                                                                     \
-    const uint2 th = lds64i<0>(ta), tl = lds64i<kSmT1lo - kSmT1p>(ta);                                             \
-    const __half2 kx = __hmul2(u_hi, as_h2(th.x)), ky = __hmul2(u_hi, as_h2(th.y));                                \
-    hi[2 * (S)] = kx;                                                                                              \
-    hi[2 * (S) + 1] = ky;                                                                                          \
-    lo[2 * (S)] =                                                                                                  \
-        __hfma2(u_hi, as_h2(tl.x), __hfma2(u_lo, as_h2(th.x), __hfma2(u_hi, as_h2(th.x), __hneg2(kx))));           \
-    lo[2 * (S) + 1] =                                                                                              \
-        __hfma2(u_hi, as_h2(tl.y), __hfma2(u_lo, as_h2(th.y), __hfma2(u_hi, as_h2(th.y), __hneg2(ky))));           \
-  }
-  PQ_SUB(0) PQ_SUB(1) PQ_SUB(2) PQ_SUB(3)
-#undef PQ_SUB
+template <int kS>
+__device__ __forceinline__ void sub_block_hilo(const BlockRef& b, uint32_t t1, __half2& xh, __half2& yh, __half2& xl,
+                                               __half2& yl) {
+  const uint2 uu = lds64i<kS * 8192>(u_address<kS>(b));
+  const __half2 u_hi = __hmul2(b.r2, as_h2(uu.x));
+  const __half2 u_lo = __hfma2(b.r2, as_h2(uu.y), __hfma2(b.r2, as_h2(uu.x), __hneg2(u_hi)));
+  const uint32_t ta = t1_address<kS>(b.l1, t1);
+  const uint2 th = lds64i<0>(ta), tl = lds64i<kSmT1lo - kSmT1p>(ta);
+  xh = __hmul2(u_hi, as_h2(th.x));
+  yh = __hmul2(u_hi, as_h2(th.y));
+  xl = __hfma2(u_hi, as_h2(tl.x), __hfma2(u_lo, as_h2(th.x), __hfma2(u_hi, as_h2(th.x), __hneg2(xh))));
+  yl = __hfma2(u_hi, as_h2(tl.y), __hfma2(u_lo, as_h2(th.y), __hfma2(u_hi, as_h2(th.y), __hneg2(yh))));
 }
 
 // plane offsets of a d = 128 token-block
@@ -253,6 +246,8 @@ struct Segment {
   int unit, st0, st1, part, n_parts, slot0;
 };
 
+// kHG = groups of four query heads per kv head (1: up to 4 heads, 2: up to 8).
+template <int kHG>
 __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((kSmAlign - (smem_u32(smem_raw) & (kSmAlign - 1))) & (kSmAlign - 1));
@@ -267,7 +262,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(sm_base + kSmBar + 8 * s, 1);                                  // full: producer + tx bytes
-      mbar_init(sm_base + kSmBar + 8 * (kStages + s), kFastConsumerWarps);     // empty: one arrive per warp
+      mbar_init(sm_base + kSmBar + 8 * (kStages + s), kFastConsumerWarps / 2);  // empty: one arrive per warp of the group
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -338,9 +333,9 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
   const int my_segs = *n_segs;
   const int g = lane >> 2, c = lane & 3;
   const uint32_t rep = (lane & 15) * 8;
-  // logical token n of a tile (MMA column n) is physical token (n >> 1) + 4 * (n & 1)
-  const int ktok = (g >> 1) + 4 * (g & 1);  // token whose keys this thread decodes
-  int it0 = 0;  // stages this CTA has streamed so far (ring slot and barrier phase bookkeeping)
+  const uint32_t ua = sm_base + kSmU + rep, t1a = sm_base + kSmT1p + rep;  // table base | lane replica
+  const int wg = warp >> 3;  // group of 8 warps
+  int gl0 = 0;               // stages this group has streamed so far (ring slot and barrier phase bookkeeping)
 
   for (int sg = 0; sg < my_segs; ++sg) {
     const int u = segs[sg].unit, st0 = segs[sg].st0, st1 = segs[sg].st1;
@@ -354,27 +349,32 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     float o_acc[8][4];  // tile i (pair i of block g): rows 2i / 2i+1 of block g, heads 2c / 2c+1
 #pragma unroll
     for (int i = 0; i < 8; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
-    float m_run = -CUDART_INF_F, l_run = 0.f;  // of head g (replicated over the 4 lanes of a quad)
+    float m_run[kHG], l_run[kHG];  // of head c + 4 hg (replicated over the 8 lanes with the same c)
+#pragma unroll
+    for (int hg = 0; hg < kHG; ++hg) {
+      m_run[hg] = -CUDART_INF_F;
+      l_run[hg] = 0.f;
+    }
 
-    // Copy of this segment's iteration `it` (stage st0 + it) into ring slot (it0 + it) % kStages; waits
-    // (bounded) until all 16 warps have released the slot's previous contents.  Thread 0 only.
+    // The two groups of 8 warps take alternate stages: group wg handles stages st0 + wg + 2 li and owns
+    // ring slots 2 wg and 2 wg + 1.  Lane 0 of the group's first warp issues the group's copies, one
+    // stage of its own ahead; it waits (bounded) until the group's 8 warps have released the slot.
+    const int n_li = st1 - st0 > wg ? (st1 - st0 - wg + 1) >> 1 : 0;
     int issued = 0;
-    auto issue_copy = [&](int it) -> bool {
-      const int gi = it0 + it, s = gi % kStages;
-      if (gi >= kStages && !mbar_wait(sm_base + kSmBar + 8 * (kStages + s), ((gi / kStages) - 1) & 1, abort_flag))
-        return false;
-      const int st = st0 + it;
+    auto issue_copy = [&](int li) -> bool {
+      const int gl = gl0 + li, s = 2 * wg + (gl & 1);
+      if (gl >= 2 && !mbar_wait(sm_base + kSmBar + 8 * (kStages + s), ((gl >> 1) - 1) & 1, abort_flag)) return false;
+      const int st = st0 + wg + 2 * li;
       const int nblk = min(2, nblk_total - 2 * st);
       const uint32_t bytes = nblk * 2 * kBlockBytes128;
       mbar_expect_tx(sm_base + kSmBar + 8 * s, bytes);
       bulk_load(sm_base + kSmRing + s * kStageBytes, head_base + (int64_t)st * kStageBytes, bytes, sm_base + kSmBar + 8 * s);
-      issued = it + 1;
+      issued = li + 1;
       return true;
     };
-    if (tid == 0)
-      for (int it = 0; it < kStages - 1 && st0 + it < st1; ++it) issue_copy(it);
+    const bool producer = (tid & 255) == 0;
+    if (producer && n_li > 0) issue_copy(0);
     __syncwarp();
-    // ---------------------------------------------------------------- consumers
     // q' = (q S) * scale * log2(e) for the unit's query heads, as an fp16 value plus an fp16 residual.
     // The first stages of the segment are already on their way while this runs.
     {
@@ -399,82 +399,110 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
       }
       __syncthreads();
     }
-    // q' fragments: A operand (16 rows x 16 coords per k-step): rows 0..7 the fp16 values, rows 8..15 the residuals.
-    // k-step ks covers, for thread c, sub-block (ks & 3) of block 2c + (ks >> 2).
-    uint32_t qa[8][2], ql[8][2];  // fp16 value and fp16 residual of q'
-    {
-      const uint2* q_hi = reinterpret_cast<const uint2*>(smem + kSmQ + 4096) + (g * 128 + 32 * c) / 4;
-      const uint2* q_lo = q_hi + 8 * 128 / 4;
+    // q' fragments, B operand (16 coords x 8 columns per k-step): column n = 2 h + part holds the fp16 value
+    // (part 0) or the fp16 residual (part 1) of head h (+ 4 hg).  k-step ks covers, for thread c, sub-block
+    // (ks & 3) of block 2c + (ks >> 2).
+    uint32_t qb[kHG][8][2];
+#pragma unroll
+    for (int hg = 0; hg < kHG; ++hg) {
+      const int h = (g >> 1) + 4 * hg;
+      const uint2* qsrc = reinterpret_cast<const uint2*>(smem + kSmQ + 4096 + (g & 1) * 2048) + (h * 128 + 32 * c) / 4;
 #pragma unroll
       for (int ks = 0; ks < 8; ++ks) {
-        uint2 v = make_uint2(0u, 0u), w = make_uint2(0u, 0u);
-        if (g < g_heads) {
-          v = q_hi[ks];
-          w = q_lo[ks];
-        }
+        uint2 v = make_uint2(0u, 0u);
+        if (h < g_heads) v = qsrc[ks];
         // decoded keys come as (coord 0, coord 2), (coord 1, coord 3) of each sub-block: permute q' to match
-        qa[ks][0] = __byte_perm(v.x, v.y, 0x5410);
-        qa[ks][1] = __byte_perm(v.x, v.y, 0x7632);
-        ql[ks][0] = __byte_perm(w.x, w.y, 0x5410);
-        ql[ks][1] = __byte_perm(w.x, w.y, 0x7632);
+        qb[hg][ks][0] = __byte_perm(v.x, v.y, 0x5410);
+        qb[hg][ks][1] = __byte_perm(v.x, v.y, 0x7632);
       }
     }
-    for (int st = st0, it = 0; st < st1; ++st, ++it) {
-      const int gi = it0 + it, s = gi % kStages;
-      if (tid == 0 && st + kStages - 1 < st1) issue_copy(it + kStages - 1);
+    for (int li = 0; li < n_li; ++li) {
+      const int gl = gl0 + li, s = 2 * wg + (gl & 1);
+      const int st = st0 + wg + 2 * li;
+      if (producer && li + 1 < n_li) issue_copy(li + 1);
       __syncwarp();
-      if (!mbar_wait(sm_base + kSmBar + 8 * s, (gi / kStages) & 1, abort_flag)) break;
-      const int tile_tok0 = st * kStageTokens + warp * 8;  // first token of this warp's tile
+      if (!mbar_wait(sm_base + kSmBar + 8 * s, (gl >> 1) & 1, abort_flag)) break;
+      const int tile_tok0 = st * kStageTokens + (warp & 7) * 16;  // first token of this warp's 16-token tile
       if (tile_tok0 < len) {
-        const uint32_t kblk = sm_base + kSmRing + s * kStageBytes + (warp >> 3) * 2 * kBlockBytes128;
+        const uint32_t kblk = sm_base + kSmRing + s * kStageBytes + ((warp >> 2) & 1) * 2 * kBlockBytes128;
         const uint32_t vblk = kblk + kBlockBytes128;
-        const int t0 = (warp & 7) * 8;  // tile's first token inside its token-block
-        // ---- scores: S^T (heads x tokens)
-        // A operand: rows 0..7 = q_hi of the group's heads, rows 8..15 = q_lo of the same heads, so one MMA
-        // with k_hi yields q_hi k_hi (row g) and q_lo k_hi (row g + 8), and one with k_lo the two small
-        // terms; both rows of a head land in the same thread.  Two accumulators: two chains of 8 MMAs.
-        float sc[4] = {0.f, 0.f, 0.f, 0.f}, sc_lo[4] = {0.f, 0.f, 0.f, 0.f};
+        const int t0 = (warp & 3) * 16;  // tile's first token inside its token-block
+        // ---- scores S (tokens x columns): A operand = keys of tokens g (rows 0..7) and g + 8 (rows 8..15),
+        // decoded as hi + lo; one MMA with the hi parts and one with the lo parts per k-step.  Column 2c is
+        // q_hi of head c, column 2c+1 its q_lo, so all four products of a (token, head) land in this thread.
+        float sc[kHG][4], scl[kHG][4];
+#pragma unroll
+        for (int hg = 0; hg < kHG; ++hg)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) sc[hg][i] = scl[hg][i] = 0.f;
         {
-          const int tk = t0 + ktok;
-          const uint2 l1 = lds64(kblk + tk * 32 + c * 8);
-          const uint32_t rr = lds32(kblk + kORad + tk * 16 + c * 4);
-          const uint32_t c2 = lds16(kblk + kO2 + tk * 8 + c * 2);
-          const uint32_t c3 = lds8(kblk + kO3 + tk * 4 + c);
-          const uint32_t c4 = lds16(kblk + kO4 + tk * 2) >> (4 * c);
-          __half2 kh[8], kl[8];
-          decode_block_hilo(l1.x, c2 & 0xFFu, c3 & 0xFu, c4 & 3u, __low2half2(as_h2(rr)), sm_base, rep, kh, kl);
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks) {
-            mma_16816(sc_lo, qa[ks][0], ql[ks][0], qa[ks][1], ql[ks][1], as_u32(kl[2 * ks]), as_u32(kl[2 * ks + 1]));
-            mma_16816(sc, qa[ks][0], ql[ks][0], qa[ks][1], ql[ks][1], as_u32(kh[2 * ks]), as_u32(kh[2 * ks + 1]));
+          const int tkA = t0 + g, tkB = tkA + 8;
+          const uint2 l1A = lds64(kblk + tkA * 32 + c * 8), l1B = lds64(kblk + tkB * 32 + c * 8);
+          const uint32_t rrA = lds32(kblk + kORad + tkA * 16 + c * 4), rrB = lds32(kblk + kORad + tkB * 16 + c * 4);
+          const uint32_t c2A = lds16(kblk + kO2 + tkA * 8 + c * 2), c2B = lds16(kblk + kO2 + tkB * 8 + c * 2);
+          const uint32_t c3A = lds8(kblk + kO3 + tkA * 4 + c), c3B = lds8(kblk + kO3 + tkB * 4 + c);
+          const uint32_t c4A = lds16(kblk + kO4 + tkA * 2) >> (4 * c), c4B = lds16(kblk + kO4 + tkB * 2) >> (4 * c);
+#define PQ_KSTEP(H, S)                                                                                    \
+  {                                                                                                       \
+    __half2 xhA, yhA, xlA, ylA, xhB, yhB, xlB, ylB;                                                       \
+    sub_block_hilo<S>(bA, t1a, xhA, yhA, xlA, ylA);                                                       \
+    sub_block_hilo<S>(bB, t1a, xhB, yhB, xlB, ylB);                                                       \
+    _Pragma("unroll") for (int hg = 0; hg < kHG; ++hg) {                                                  \
+      mma_16816(scl[hg], as_u32(xlA), as_u32(xlB), as_u32(ylA), as_u32(ylB), qb[hg][4 * (H) + (S)][0],    \
+                qb[hg][4 * (H) + (S)][1]);                                                                \
+      mma_16816(sc[hg], as_u32(xhA), as_u32(xhB), as_u32(yhA), as_u32(yhB), qb[hg][4 * (H) + (S)][0],     \
+                qb[hg][4 * (H) + (S)][1]);                                                                \
+    }                                                                                                     \
+  }
+          {
+            const BlockRef bA = make_block_ref(l1A.x, c2A, c3A, c4A & 3u, __low2half2(as_h2(rrA)), ua);
+            const BlockRef bB = make_block_ref(l1B.x, c2B, c3B, c4B & 3u, __low2half2(as_h2(rrB)), ua);
+            PQ_KSTEP(0, 0) PQ_KSTEP(0, 1) PQ_KSTEP(0, 2) PQ_KSTEP(0, 3)
           }
-          decode_block_hilo(l1.y, c2 >> 8, c3 >> 4, (c4 >> 2) & 3u, __high2half2(as_h2(rr)), sm_base, rep, kh, kl);
-#pragma unroll
-          for (int ks = 0; ks < 4; ++ks) {
-            mma_16816(sc_lo, qa[4 + ks][0], ql[4 + ks][0], qa[4 + ks][1], ql[4 + ks][1], as_u32(kl[2 * ks]),
-                      as_u32(kl[2 * ks + 1]));
-            mma_16816(sc, qa[4 + ks][0], ql[4 + ks][0], qa[4 + ks][1], ql[4 + ks][1], as_u32(kh[2 * ks]),
-                      as_u32(kh[2 * ks + 1]));
+          {
+            const BlockRef bA = make_block_ref(l1A.y, c2A >> 8, c3A >> 4, (c4A >> 2) & 3u, __high2half2(as_h2(rrA)), ua);
+            const BlockRef bB = make_block_ref(l1B.y, c2B >> 8, c3B >> 4, (c4B >> 2) & 3u, __high2half2(as_h2(rrB)), ua);
+            PQ_KSTEP(1, 0) PQ_KSTEP(1, 1) PQ_KSTEP(1, 2) PQ_KSTEP(1, 3)
           }
-          sc[0] += (sc_lo[0] + sc_lo[2]) + sc[2];  // small terms first
-          sc[1] += (sc_lo[1] + sc_lo[3]) + sc[3];
+#undef PQ_KSTEP
         }
-        // ---- online softmax for head g; this thread holds logical tokens 2c, 2c+1 = physical c, c+4
-        const bool ok0 = tile_tok0 + c < len, ok1 = tile_tok0 + c + 4 < len;
-        const float s0 = ok0 ? sc[0] : -CUDART_INF_F, s1 = ok1 ? sc[1] : -CUDART_INF_F;
-        float mx = fmaxf(s0, s1);
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
-        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
-        const float m_new = fmaxf(m_run, mx);
-        const float p0 = exp2f(s0 - m_new), p1 = exp2f(s1 - m_new);
-        float psum = p0 + p1;
-        psum += __shfl_xor_sync(0xffffffffu, psum, 1);
-        psum += __shfl_xor_sync(0xffffffffu, psum, 2);
-        const float corr = exp2f(m_run - m_new);  // 0 on the first tile (m_run = -inf)
-        l_run = l_run * corr + psum;
-        if (__any_sync(0xffffffffu, m_new > m_run)) {
-          const float c0 = __shfl_sync(0xffffffffu, corr, (2 * c) << 2);
-          const float c1 = __shfl_sync(0xffffffffu, corr, (2 * c + 1) << 2);
+        // ---- online softmax: this thread holds head c (+ 4 hg) of tokens g and g + 8
+        const bool ok0 = tile_tok0 + g < len, ok1 = tile_tok0 + g + 8 < len;
+        uint32_t ph[kHG];   // (p of token g, p of token g + 8) in fp16
+        float corr[kHG];
+        bool grew = false;
+#pragma unroll
+        for (int hg = 0; hg < kHG; ++hg) {
+          const float s0 = ok0 ? (scl[hg][0] + scl[hg][1]) + sc[hg][1] + sc[hg][0] : -CUDART_INF_F;  // small terms first
+          const float s1 = ok1 ? (scl[hg][2] + scl[hg][3]) + sc[hg][3] + sc[hg][2] : -CUDART_INF_F;
+          float mx = fmaxf(s0, s1);
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+          const float m_new = fmaxf(m_run[hg], mx);  // finite: token 0 of the tile is inside the sequence
+          const float p0 = exp2f(s0 - m_new), p1 = exp2f(s1 - m_new);
+          float psum = p0 + p1;
+          psum += __shfl_xor_sync(0xffffffffu, psum, 4);
+          psum += __shfl_xor_sync(0xffffffffu, psum, 8);
+          psum += __shfl_xor_sync(0xffffffffu, psum, 16);
+          corr[hg] = exp2f(m_run[hg] - m_new);  // 0 on the first tile (m_run = -inf)
+          l_run[hg] = l_run[hg] * corr[hg] + psum;
+          grew = grew || m_new > m_run[hg];
+          m_run[hg] = m_new;
+          ph[hg] = as_u32(__floats2half2_rn(p0, p1));
+        }
+        if (__any_sync(0xffffffffu, grew)) {
+          // accumulator columns 2c, 2c+1 are heads 2c, 2c+1: their factors live in lanes (2c) & 3, (2c+1) & 3
+          float c0 = __shfl_sync(0xffffffffu, corr[0], (2 * c) & 3);
+          float c1 = __shfl_sync(0xffffffffu, corr[0], (2 * c + 1) & 3);
+          if (kHG == 2) {
+            const float d0 = __shfl_sync(0xffffffffu, corr[kHG - 1], (2 * c) & 3);
+            const float d1 = __shfl_sync(0xffffffffu, corr[kHG - 1], (2 * c + 1) & 3);
+            if (c >= 2) {
+              c0 = d0;
+              c1 = d1;
+            }
+          }
 #pragma unroll
           for (int i = 0; i < 8; ++i) {
             o_acc[i][0] *= c0;
@@ -483,62 +511,85 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
             o_acc[i][3] *= c1;
           }
         }
-        m_run = m_new;
-        const uint32_t pb = as_u32(__floats2half2_rn(p0, p1));  // B operand: tokens (2c, 2c+1) x head g
-        // ---- values: block g of physical tokens c and c + 4
+        // B operand of the value MMAs: column n = g is head g, rows = tokens 2c, 2c+1 | 2c+8, 2c+9
+        uint32_t pb0, pb1;
         {
-          __half2 va[8], vb[8];
-          {
-            const int tk = t0 + c;
-            const uint32_t l1 = lds32(vblk + tk * 32 + g * 4);
-            uint32_t rr = lds16(vblk + kORad + tk * 16 + g * 2);
-            const uint32_t c2 = lds8(vblk + kO2 + tk * 8 + g);
-            const uint32_t c3 = lds8(vblk + kO3 + tk * 4 + (g >> 1)) >> (4 * (g & 1));
-            const uint32_t c4 = lds16(vblk + kO4 + tk * 2) >> (2 * g);
-            if (!ok0) rr = 0u;  // stale bytes past the sequence end must not reach the accumulators
-            decode_block_h2(l1, c2, c3 & 0xFu, c4 & 3u, as_h2(rr | (rr << 16)), sm_base, rep, va);
+          const int srcA = (2 * c) * 4 + (g & 3), srcB = srcA + 4;
+          uint32_t uA = __shfl_sync(0xffffffffu, ph[0], srcA), uB = __shfl_sync(0xffffffffu, ph[0], srcB);
+          if (kHG == 2) {
+            const uint32_t wA = __shfl_sync(0xffffffffu, ph[kHG - 1], srcA), wB = __shfl_sync(0xffffffffu, ph[kHG - 1], srcB);
+            if (g >= 4) {
+              uA = wA;
+              uB = wB;
+            }
           }
-          {
-            const int tk = t0 + c + 4;
-            const uint32_t l1 = lds32(vblk + tk * 32 + g * 4);
-            uint32_t rr = lds16(vblk + kORad + tk * 16 + g * 2);
-            const uint32_t c2 = lds8(vblk + kO2 + tk * 8 + g);
-            const uint32_t c3 = lds8(vblk + kO3 + tk * 4 + (g >> 1)) >> (4 * (g & 1));
-            const uint32_t c4 = lds16(vblk + kO4 + tk * 2) >> (2 * g);
-            if (!ok1) rr = 0u;
-            decode_block_h2(l1, c2, c3 & 0xFu, c4 & 3u, as_h2(rr | (rr << 16)), sm_base, rep, vb);
-          }
-          // va[2s] = (x_a, x_b), va[2s+1] = (y_a, y_b) of sub-block s: pair i = 2s + h takes half h of both
+          pb0 = __byte_perm(uA, uB, 0x5410);
+          pb1 = __byte_perm(uA, uB, 0x7632);
+        }
+        // ---- values: block g of tokens 2c, 2c+1, 2c+8, 2c+9 -> O^T (coordinates x heads) += V_hat^T P
+        {
+          BlockRef bv[4];
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int s2 = 2 * (i >> 1);
-            const uint32_t sel = (i & 1) ? 0x7632 : 0x5410;
-            const uint32_t x = __byte_perm(as_u32(va[s2]), as_u32(vb[s2]), sel);          // coord 2i   of tokens (A, B)
-            const uint32_t y = __byte_perm(as_u32(va[s2 + 1]), as_u32(vb[s2 + 1]), sel);  // coord 2i+1 of tokens (A, B)
-            mma_1688(o_acc[i], x, y, pb);
+          for (int j = 0; j < 4; ++j) {
+            const int tt = 2 * c + (j & 1) + 8 * (j >> 1);
+            const int tk = t0 + tt;
+            const uint32_t l1 = lds32(vblk + tk * 32 + g * 4);
+            uint32_t rr = lds16(vblk + kORad + tk * 16 + g * 2);
+            const uint32_t c2 = lds8(vblk + kO2 + tk * 8 + g);
+            const uint32_t c3 = lds8(vblk + kO3 + tk * 4 + (g >> 1)) >> (4 * (g & 1));
+            const uint32_t c4 = lds16(vblk + kO4 + tk * 2) >> (2 * g);
+            if (tile_tok0 + tt >= len) rr = 0u;  // stale bytes past the sequence end must not reach the accumulators
+            bv[j] = make_block_ref(l1, c2, c3, c4 & 3u, as_h2(rr | (rr << 16)), ua);
           }
+#define PQ_VSTEP(S)                                                                                      \
+  {                                                                                                      \
+    __half2 x0, y0, x1, y1, x2, y2, x3, y3;                                                              \
+    sub_block_h2<S>(bv[0], t1a, x0, y0);                                                                 \
+    sub_block_h2<S>(bv[1], t1a, x1, y1);                                                                 \
+    sub_block_h2<S>(bv[2], t1a, x2, y2);                                                                 \
+    sub_block_h2<S>(bv[3], t1a, x3, y3);                                                                 \
+    mma_16816(o_acc[2 * (S)], __byte_perm(as_u32(x0), as_u32(x1), 0x5410),                               \
+              __byte_perm(as_u32(y0), as_u32(y1), 0x5410), __byte_perm(as_u32(x2), as_u32(x3), 0x5410),  \
+              __byte_perm(as_u32(y2), as_u32(y3), 0x5410), pb0, pb1);                                    \
+    mma_16816(o_acc[2 * (S) + 1], __byte_perm(as_u32(x0), as_u32(x1), 0x7632),                           \
+              __byte_perm(as_u32(y0), as_u32(y1), 0x7632), __byte_perm(as_u32(x2), as_u32(x3), 0x7632),  \
+              __byte_perm(as_u32(y2), as_u32(y3), 0x7632), pb0, pb1);                                    \
+  }
+          PQ_VSTEP(0) PQ_VSTEP(1) PQ_VSTEP(2) PQ_VSTEP(3)
+#undef PQ_VSTEP
         }
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(sm_base + kSmBar + 8 * (kStages + s));
     }
-    if (tid == 0 && *abort_flag) {
+    gl0 += n_li;
+    __syncthreads();  // every copy that was consumed is done with; the rest is waited for below
+    if (*abort_flag) {
       // gave up: let the copies still in flight land (bounded) before the ring is reused
-      for (int it = max(0, issued - kStages); it < issued; ++it)
-        for (int i = 0; i < kSpinLimit && !mbar_try_wait(sm_base + kSmBar + 8 * ((it0 + it) % kStages), ((it0 + it) / kStages) & 1); ++i)
-          __nanosleep(64);
+      if (producer)
+        for (int li = max(0, issued - 2); li < issued; ++li) {
+          const int gl = gl0 - n_li + li;
+          for (int i = 0; i < kSpinLimit && !mbar_try_wait(sm_base + kSmBar + 8 * (2 * wg + (gl & 1)), (gl >> 1) & 1); ++i)
+            __nanosleep(64);
+        }
+      __syncthreads();
     }
-    it0 += st1 - st0;
-    __syncthreads();  // every copy that was issued has been consumed (or the CTA aborted)
 
     // ---- merge the 16 warps (fixed order), write this part's partial, last part combines the unit
     // Coordinate j of head h of warp w sits at (w * 8 + h) * kMrgStride + (j & 15) * 8 + (j >> 4): for a fixed
     // accumulator register the 32 lanes (block g, head pair c) then hit 32 different banks.
     float* mrg_o = reinterpret_cast<float*>(smem + kSmRing);          // [16 warps][8 heads][kMrgStride]
     float* mrg_ml = mrg_o + kFastConsumerWarps * 8 * kMrgStride;      // [16 warps][8 heads][2]
-    if (c == 0) {
-      mrg_ml[(warp * 8 + g) * 2] = m_run;
-      mrg_ml[(warp * 8 + g) * 2 + 1] = l_run;
+    if (g == 0) {
+#pragma unroll
+      for (int hg = 0; hg < kHG; ++hg) {
+        mrg_ml[(warp * 8 + c + 4 * hg) * 2] = m_run[hg];
+        mrg_ml[(warp * 8 + c + 4 * hg) * 2 + 1] = l_run[hg];
+      }
+      if (kHG == 1) {  // heads 4..7 do not exist: neutral entries
+        mrg_ml[(warp * 8 + c + 4) * 2] = -CUDART_INF_F;
+        mrg_ml[(warp * 8 + c + 4) * 2 + 1] = 0.f;
+      }
     }
     if (2 * c < g_heads) {
 #pragma unroll

@@ -73,7 +73,7 @@ def test_config1_tiny_reference_d16_fp32():
     assert rel_l2(to_f64(out), ref.attend(to_f64(q), 0.25)) < TOL_ATTENTION
 
 
-@pytest.mark.parametrize("d,Hq,Hkv", [(128, 8, 2), (64, 4, 4), (32, 2, 1), (16, 8, 1)])
+@pytest.mark.parametrize("d,Hq,Hkv", [(128, 8, 2), (128, 16, 2), (128, 6, 2), (64, 4, 4), (32, 2, 1), (16, 8, 1)])
 def test_ragged_batch_encode_dequant_attention(d, Hq, Hkv):
     """Several token-blocks plus ragged tails; bf16 inputs with outlier key channels."""
     lens_list = [130, 1, 64, 257]
