@@ -366,8 +366,8 @@ def run_cuda(args):
     if rank != 0:
         return
     # DRAM bytes of one decode-attention launch: ncu capture at batch 4 (profiles/decode_attention_fast_kernel_
-    # batch4_ctx32768.md: 130.48 MB read + 4.78 MB written), scaled by the batch (traffic is proportional to it)
-    traffic = (130.48e6 + 4.78e6) * BATCH / 4.0
+    # batch4_ctx32768.md: 130.50 MB read + 4.10 MB written), scaled by the batch (traffic is proportional to it)
+    traffic = (130.50e6 + 4.10e6) * BATCH / 4.0
     cpu = _oracle_sample_throughput(12.0) if world == 1 and not args.no_cpu_baseline else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -376,7 +376,7 @@ def run_cuda(args):
         "config": {"workload": WORKLOAD, "batch": BATCH, "per_gpu": True, "l2": "inputs larger than L2 (260 MB cache per decode, "
                    "two alternating 128 MiB prefill chunks)", "compressed_bytes_per_decode": comp_bytes,
                    "decode_ms": dec_ms, "append_ms": app_ms, "encode_ms": enc_ms,
-                   "value_definition": "compressed bytes / CUDA-event time of pq_decode_attention (both its kernels)"},
+                   "value_definition": "compressed bytes / CUDA-event time of pq_decode_attention (one persistent kernel)"},
         "encode": {"tokens_per_s": world * CTX / (enc_ms * 1e-3), "vectors_per_s": world * CTX * HKV * 2 / (enc_ms * 1e-3),
                    "gbs": enc_bytes / (enc_ms * 1e-3) / 1e9, "hbm_frac_measured": enc_bytes / (enc_ms * 1e-3) / 1e9 / peak,
                    "e2e_tokens_per_s": world * CTX / (e_enc_ms * 1e-3)},
@@ -389,7 +389,7 @@ def run_cuda(args):
                 "definition": "compressed bytes / (H2D of new k,v and q + append + decode attention + D2H of the output); "
                               "the 128 MiB prefill chunk's H2D is charged to encode.e2e_tokens_per_s",
                 "ms_per_step": float(reduce_max(e2e_total_ms)) / args.steps},
-        "gpu_launches": 6 * args.steps,
+        "gpu_launches": 5 * args.steps,  # encode + lens, append + lens, decode attention
         "clocks": clocks,
         "oracle_match": match,
     }

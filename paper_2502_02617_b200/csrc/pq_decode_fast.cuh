@@ -120,6 +120,18 @@ __device__ __forceinline__ uint2 lds64i(uint32_t addr) {
   asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+%3];" : "=r"(v.x), "=r"(v.y) : "r"(addr), "n"(kOff));
   return v;
 }
+template <int kOff>
+__device__ __forceinline__ uint32_t lds16i(uint32_t addr) {
+  uint16_t v;
+  asm volatile("ld.shared.u16 %0, [%1+%2];" : "=h"(v) : "r"(addr), "n"(kOff));
+  return v;
+}
+template <int kOff>
+__device__ __forceinline__ uint32_t lds8i(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared.u8 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(kOff));
+  return v;
+}
 __device__ __forceinline__ uint32_t lds16(uint32_t addr) {
   uint16_t v;
   asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
@@ -335,6 +347,15 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
   const uint32_t rep = (lane & 15) * 8;
   const uint32_t ua = sm_base + kSmU + rep, t1a = sm_base + kSmT1p + rep;  // table base | lane replica
   const int wg = warp >> 3;  // group of 8 warps
+  // Offsets, inside a token-block, of what this thread reads of its tile (16 tokens from token (warp & 3) * 16).
+  // Keys: tokens g and g + 8, blocks 2c and 2c + 1.  Values: block g of tokens c, c + 4, c + 8, c + 12 (these are
+  // rows 2c, 2c + 1, 2c + 8, 2c + 9 of the value MMA: with this order the four lanes of a quad read four
+  // consecutive tokens and the loads are free of bank conflicts).
+  const int tk_k = (warp & 3) * 16 + (lane >> 2), tk_v = (warp & 3) * 16 + (lane & 3);
+  const uint32_t ok_l1 = tk_k * 32 + (lane & 3) * 8, ok_r = kORad + tk_k * 16 + (lane & 3) * 4;
+  const uint32_t ok_c2 = kO2 + tk_k * 8 + (lane & 3) * 2, ok_c3 = kO3 + tk_k * 4 + (lane & 3), ok_c4 = kO4 + tk_k * 2;
+  const uint32_t ov_l1 = tk_v * 32 + (lane >> 2) * 4, ov_r = kORad + tk_v * 16 + (lane >> 2) * 2;
+  const uint32_t ov_c2 = kO2 + tk_v * 8 + (lane >> 2), ov_c3 = kO3 + tk_v * 4 + (lane >> 3), ov_c4 = kO4 + tk_v * 2;
   int gl0 = 0;               // stages this group has streamed so far (ring slot and barrier phase bookkeeping)
 
   for (int sg = 0; sg < my_segs; ++sg) {
@@ -436,12 +457,11 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
 #pragma unroll
           for (int i = 0; i < 4; ++i) sc[hg][i] = scl[hg][i] = 0.f;
         {
-          const int tkA = t0 + g, tkB = tkA + 8;
-          const uint2 l1A = lds64(kblk + tkA * 32 + c * 8), l1B = lds64(kblk + tkB * 32 + c * 8);
-          const uint32_t rrA = lds32(kblk + kORad + tkA * 16 + c * 4), rrB = lds32(kblk + kORad + tkB * 16 + c * 4);
-          const uint32_t c2A = lds16(kblk + kO2 + tkA * 8 + c * 2), c2B = lds16(kblk + kO2 + tkB * 8 + c * 2);
-          const uint32_t c3A = lds8(kblk + kO3 + tkA * 4 + c), c3B = lds8(kblk + kO3 + tkB * 4 + c);
-          const uint32_t c4A = lds16(kblk + kO4 + tkA * 2) >> (4 * c), c4B = lds16(kblk + kO4 + tkB * 2) >> (4 * c);
+          const uint2 l1A = lds64i<0>(kblk + ok_l1), l1B = lds64i<8 * 32>(kblk + ok_l1);
+          const uint32_t rrA = lds32i<0>(kblk + ok_r), rrB = lds32i<8 * 16>(kblk + ok_r);
+          const uint32_t c2A = lds16i<0>(kblk + ok_c2), c2B = lds16i<8 * 8>(kblk + ok_c2);
+          const uint32_t c3A = lds8i<0>(kblk + ok_c3), c3B = lds8i<8 * 4>(kblk + ok_c3);
+          const uint32_t c4A = lds16i<0>(kblk + ok_c4) >> (4 * c), c4B = lds16i<8 * 2>(kblk + ok_c4) >> (4 * c);
 #define PQ_KSTEP(H, S)                                                                                    \
   {                                                                                                       \
     __half2 xhA, yhA, xlA, ylA, xhB, yhB, xlB, ylB;                                                       \
@@ -511,10 +531,10 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
             o_acc[i][3] *= c1;
           }
         }
-        // B operand of the value MMAs: column n = g is head g, rows = tokens 2c, 2c+1 | 2c+8, 2c+9
+        // B operand of the value MMAs: column n = g is head g, rows 2c, 2c+1 | 2c+8, 2c+9 = tokens c, c+4 | c+8, c+12
         uint32_t pb0, pb1;
         {
-          const int srcA = (2 * c) * 4 + (g & 3), srcB = srcA + 4;
+          const int srcA = c * 4 + (g & 3), srcB = srcA + 16;
           uint32_t uA = __shfl_sync(0xffffffffu, ph[0], srcA), uB = __shfl_sync(0xffffffffu, ph[0], srcB);
           if (kHG == 2) {
             const uint32_t wA = __shfl_sync(0xffffffffu, ph[kHG - 1], srcA), wB = __shfl_sync(0xffffffffu, ph[kHG - 1], srcB);
@@ -529,18 +549,18 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
         // ---- values: block g of tokens 2c, 2c+1, 2c+8, 2c+9 -> O^T (coordinates x heads) += V_hat^T P
         {
           BlockRef bv[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            const int tt = 2 * c + (j & 1) + 8 * (j >> 1);
-            const int tk = t0 + tt;
-            const uint32_t l1 = lds32(vblk + tk * 32 + g * 4);
-            uint32_t rr = lds16(vblk + kORad + tk * 16 + g * 2);
-            const uint32_t c2 = lds8(vblk + kO2 + tk * 8 + g);
-            const uint32_t c3 = lds8(vblk + kO3 + tk * 4 + (g >> 1)) >> (4 * (g & 1));
-            const uint32_t c4 = lds16(vblk + kO4 + tk * 2) >> (2 * g);
-            if (tile_tok0 + tt >= len) rr = 0u;  // stale bytes past the sequence end must not reach the accumulators
-            bv[j] = make_block_ref(l1, c2, c3, c4 & 3u, as_h2(rr | (rr << 16)), ua);
-          }
+#define PQ_VLOAD(J)                                                                                          \
+  {                                                                                                          \
+    const uint32_t l1 = lds32i<4 * (J) * 32>(vblk + ov_l1);                                                  \
+    uint32_t rr = lds16i<4 * (J) * 16>(vblk + ov_r);                                                         \
+    const uint32_t c2 = lds8i<4 * (J) * 8>(vblk + ov_c2);                                                    \
+    const uint32_t c3 = lds8i<4 * (J) * 4>(vblk + ov_c3) >> (4 * (g & 1));                                   \
+    const uint32_t c4 = lds16i<4 * (J) * 2>(vblk + ov_c4) >> (2 * g);                                        \
+    if (tile_tok0 + c + 4 * (J) >= len) rr = 0u; /* stale bytes past the sequence end stay out of the sums */ \
+    bv[J] = make_block_ref(l1, c2, c3, c4 & 3u, as_h2(rr | (rr << 16)), ua);                                 \
+  }
+          PQ_VLOAD(0) PQ_VLOAD(1) PQ_VLOAD(2) PQ_VLOAD(3)
+#undef PQ_VLOAD
 #define PQ_VSTEP(S)                                                                                      \
   {                                                                                                      \
     __half2 x0, y0, x1, y1, x2, y2, x3, y3;                                                              \
