@@ -51,6 +51,9 @@ struct Tables {
 };
 
 constexpr uint32_t kFlagUniformL1 = 1u;
+// bit 1: at every level >= 2 the boundaries are b, pi/4, pi/2 - b (tan^2: T, 1, 1/T to 1e-9 relative), as for
+// every Lloyd-Max codebook of the symmetric densities of Lemma 2
+constexpr uint32_t kFlagSymmetricUpper = 2u;
 
 // ------------------------------------------------------------------------------------------
 // Packed cache layout.

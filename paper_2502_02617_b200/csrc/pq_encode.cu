@@ -209,7 +209,8 @@ __device__ __forceinline__ void quantise_and_store(const EncodeArgs& a, const Fa
   FastBlock fb[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    polar_quant_block_fast(y + 16 * i, rm, fq, &fb[i]);
+    if (fq.sym) polar_quant_block_fast<true>(y + 16 * i, rm, fq, &fb[i]);
+    else polar_quant_block_fast<false>(y + 16 * i, rm, fq, &fb[i]);
     if (!uniform_l1) fb[i].amb |= 0xFFu;  // other level-1 codebooks: decide every level-1 angle exactly
     left[i] = 0u;
   }
@@ -384,7 +385,8 @@ __global__ void __launch_bounds__(128) encode_vector_kernel(EncodeArgs a) {
     float yb[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) yb[i] = ys[16 * j + i];
-    polar_quant_block_fast(yb, make_row_margins(dy, fq), fq, &fb);
+    if (fq.sym) polar_quant_block_fast<true>(yb, make_row_margins(dy, fq), fq, &fb);
+    else polar_quant_block_fast<false>(yb, make_row_margins(dy, fq), fq, &fb);
     if ((a.tables->flags & kFlagUniformL1) == 0u) fb.amb |= 0xFFu;
   }
   if (__syncthreads_or(fb.amb != 0u)) {

@@ -23,11 +23,13 @@ constexpr float kRotErr = 1.1f * 7.62939453125e-06f;  // 1.1 * 2^-17
 // Per-call constants of the fast quantiser (uniform level-1 codebook; levels 2..4 from Tables).
 struct FastQuant {
   float t2[3][3];   // tan^2 of the three boundaries of levels 2, 3, 4
+  uint32_t sym;     // the boundaries of every level >= 2 are b, pi/4, pi/2 - b (kFlagSymmetricUpper)
 };
 
 __device__ inline void load_fast_quant(const Tables* tb, FastQuant* fq) {
   for (int l = 0; l < 3; ++l)
     for (int k = 0; k < 3; ++k) fq->t2[l][k] = (float)tb->bnd_tan2[3 * l + k];
+  fq->sym = (tb->flags & kFlagSymmetricUpper) != 0u;
 }
 
 // Per-row constants of the margins (dy = bound on the error of one rotated coordinate of the row).
@@ -42,7 +44,7 @@ __device__ __forceinline__ RowMargins make_row_margins(float dy, const FastQuant
   const float e2 = dy * dy;
 #pragma unroll
   for (int l = 0; l < 3; ++l) {
-    const float el = (float)(2 << l) * e2, t1 = 1.f + fq.t2[l][2];
+    const float el = (float)(2 << l) * e2, t1 = fq.sym ? 2.f : 1.f + fq.t2[l][2];  // 1 + largest T that is tested
     m.c[l] = 8.4f * el;
     m.base[l] = 42.f * el * el * t1 * t1;
   }
@@ -78,6 +80,28 @@ __device__ __forceinline__ uint32_t quant_upper_fast(float sa, float sb, const f
   return 3u - neg;
 }
 
+// The same decision for symmetric boundaries (T0, 1, 1/T0), folded onto m = min(sa, sb), M = max(sa, sb):
+// only the diagonal (M - m) and the boundary m = T0 M of the point's own side can be the nearest ones, and the
+// margin of the boundary sb = sa / T0 is the one of m = T0 M after multiplying both sides by T0^2.  Every T
+// that is tested is <= 1, so sb + T^2 sa <= sa + sb and the caller's `base` uses (1 + T)^2 <= 4.
+__device__ __forceinline__ uint32_t quant_upper_sym(float sa, float sb, float T0, float c, float base, bool* ambiguous) {
+  const float m = fminf(sa, sb), M = fmaxf(sa, sb);
+  const bool hi = sb > sa;
+  const float dout = fmaf(-T0, M, m), ddiag = M - m;
+  const bool lo = dout > 0.f;
+  const float w = sa + sb;
+  const float dm = fminf(fabsf(dout), ddiag);
+  const float b2 = fmaf(4.2e-11f * w, w, base);  // rho = 1e-6 covers the float32 roundings
+  bool amb = !(dm * dm > fmaf(c, w, b2));        // also true for NaN margins
+  if (amb) {
+    const bool ok_d = ddiag * ddiag > fmaf(c, w, b2);
+    const bool ok_o = dout * dout > fmaf(c, fmaf(T0 * T0, M, m), b2);
+    amb = !(ok_d && ok_o);
+  }
+  *ambiguous = amb;
+  return (hi ? 3u : 0u) ^ (lo ? 1u : 0u);
+}
+
 // Level-1 decision for the uniform codebook (boundaries k pi/8): fold into the first octant,
 // u = max(|a|,|b|), v = min(|a|,|b|); the boundaries are the axes (v = 0), the diagonals (u = v) and
 // the lines at pi/8 from the axes (v cos(pi/8) = u sin(pi/8)).  Each coordinate moves by at most
@@ -111,6 +135,12 @@ __device__ __forceinline__ float fast_sqrt(float x) {
   return r;
 }
 
+template <bool kSym>
+__device__ __forceinline__ uint32_t quant_upper_any(float sa, float sb, const float* T, float c, float base, bool* am) {
+  return kSym ? quant_upper_sym(sa, sb, T[0], c, base, am) : quant_upper_fast(sa, sb, T, c, base, am);
+}
+
+template <bool kSym>
 __device__ __forceinline__ void polar_quant_block_fast(const float* y, const RowMargins& rm, const FastQuant& fq,
                                                        FastBlock* out) {
   float s1[8], s2[4], s3[2];
@@ -124,17 +154,17 @@ __device__ __forceinline__ void polar_quant_block_fast(const float* y, const Row
   }
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    l2 |= quant_upper_fast(s1[2 * j], s1[2 * j + 1], fq.t2[0], rm.c[0], rm.base[0], &am) << (2 * j);
+    l2 |= quant_upper_any<kSym>(s1[2 * j], s1[2 * j + 1], fq.t2[0], rm.c[0], rm.base[0], &am) << (2 * j);
     amb |= (am ? 1u : 0u) << (8 + j);
     s2[j] = s1[2 * j] + s1[2 * j + 1];
   }
 #pragma unroll
   for (int j = 0; j < 2; ++j) {
-    l3 |= quant_upper_fast(s2[2 * j], s2[2 * j + 1], fq.t2[1], rm.c[1], rm.base[1], &am) << (2 * j);
+    l3 |= quant_upper_any<kSym>(s2[2 * j], s2[2 * j + 1], fq.t2[1], rm.c[1], rm.base[1], &am) << (2 * j);
     amb |= (am ? 1u : 0u) << (12 + j);
     s3[j] = s2[2 * j] + s2[2 * j + 1];
   }
-  out->l4 = quant_upper_fast(s3[0], s3[1], fq.t2[2], rm.c[2], rm.base[2], &am);
+  out->l4 = quant_upper_any<kSym>(s3[0], s3[1], fq.t2[2], rm.c[2], rm.base[2], &am);
   amb |= (am ? 1u : 0u) << 14;
   out->l1 = l1;
   out->l2 = l2;

@@ -7,9 +7,9 @@
 //     (S = S_hi + S_lo + O(2^-17)) kept in shared memory as the K-major B operand; 2 terms x 8
 //     k-steps of tcgen05.mma (M = 128 rows, N = 128, K = 16) accumulate in float32 in tensor memory;
 //     two accumulators, and the MMAs of tile i+1 are issued when the epilogue of tile i starts, so
-//     they run under it.  Four threads (one per scheduler) issue four MMAs each, so that no warp is
-//     held up by the whole batch; since their order is then free, every MMA accumulates and the
-//     epilogue clears the accumulator after reading it;
+//     they run under it.  Lane 0 of every warp issues one of the 16 MMAs, so that no warp is held up
+//     by the batch (a warp that is late delays all 16 at the next barrier); since their order is then
+//     free, every MMA accumulates and the epilogue clears the accumulator after reading it;
 //   * epilogue on all 16 warps.  Tensor-memory lane = row, so a thread owns 32 consecutive rotated
 //     coordinates (2 blocks) of one row: tcgen05.ld, sign-test quantiser with certified margins,
 //     packed stores, queued float64 re-decision of the ambiguous angles.
@@ -31,8 +31,8 @@ constexpr int kTcSBytes = 128 * 128 * 2;   // one bf16 term of S (B operand)
 constexpr int kTcSmS = 0;                  // S_hi, S_lo
 constexpr int kTcSmX = kTcSmS + 2 * kTcSBytes;
 constexpr int kTcSmRowSq = kTcSmX + kTcStages * kTcXBytes;   // [4][128] float, then [4][128] bytes of level-4 nibbles
-constexpr int kTcSmFq = kTcSmRowSq + 2048 + 512;             // FastQuant (36 B)
-constexpr int kTcSmBar = kTcSmFq + 64;                       // full[3], empty[3], tfull[2], tempty[2]
+constexpr int kTcSmFq = kTcSmRowSq + 2048 + 512;             // FastQuant (40 B)
+constexpr int kTcSmBar = kTcSmFq + 64;                       // full[3], empty[3], tfull[2]
 constexpr int kTcSmMisc = kTcSmBar + 128;                    // tmem base, abort flag
 constexpr int kTcSmFix = kTcSmMisc + 64;                     // FixQueue
 constexpr int kTcSmTotal = kTcSmFix + (int)sizeof(FixQueue) + 1024;  // + slack for 1024-byte alignment
@@ -131,18 +131,17 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   float* rowsq = reinterpret_cast<float*>(smem + kTcSmRowSq);
   uint8_t* l4s = reinterpret_cast<uint8_t*>(rowsq + 4 * 128);  // [4][128] level-4 codes of the row's column quarters
   const uint32_t bar_full = sb + kTcSmBar, bar_empty = bar_full + 8 * kTcStages;
-  const uint32_t bar_tfull = bar_empty + 8 * kTcStages, bar_tempty = bar_tfull + 16;
+  const uint32_t bar_tfull = bar_empty + 8 * kTcStages;
   const int n_tiles = n_row_tiles * 2 * a.n_kv_heads;
 
   // ---- set-up: barriers, tensor memory, S split into two bf16 terms in the B-operand layout
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
       tc_mbar_init(bar_full + 8 * s, 1);
-      tc_mbar_init(bar_empty + 8 * s, 4);   // one commit per issuing thread
+      tc_mbar_init(bar_empty + 8 * s, kTcThreads / 32);   // one commit per warp
     }
     for (int i = 0; i < 2; ++i) {
-      tc_mbar_init(bar_tfull + 8 * i, 4);   // one commit per issuing thread
-      tc_mbar_init(bar_tempty + 8 * i, kTcEpiThreads / 32);
+      tc_mbar_init(bar_tfull + 8 * i, kTcThreads / 32);   // one commit per warp
     }
     *abort_flag = 0;
     fixq->count[0] = fixq->count[1] = fixq->count[2] = fixq->count[3] = 0;
@@ -178,13 +177,24 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
-  // One thread issues the TMA loads of local tile `it` (tile blockIdx.x + it * gridDim.x).
-  auto issue_tma = [&](int it) {
+  // Tile t = (row tile, K|V, head) with head fastest: t = head + n_kv_heads * hq, hq = 2 * row tile + kv.  A CTA's
+  // tiles are gridDim.x apart; their coordinates are advanced without divisions.
+  const int step_h = (int)gridDim.x % a.n_kv_heads, step_q = (int)gridDim.x / a.n_kv_heads;
+  auto advance = [&](int& head, int& hq) {
+    head += step_h;
+    hq += step_q;
+    if (head >= a.n_kv_heads) {
+      head -= a.n_kv_heads;
+      ++hq;
+    }
+  };
+  // One thread issues the TMA loads of local tile `it` (tile blockIdx.x + it * gridDim.x = head + n_kv_heads * hq).
+  auto issue_tma = [&](int it, int head, int hq) {
     const int tile = blockIdx.x + it * gridDim.x;
     if (tile >= n_tiles) return;
     const int s = it % kTcStages;
     if (it >= kTcStages && !tc_mbar_wait(bar_empty + 8 * s, ((it / kTcStages) - 1) & 1, abort_flag)) return;
-    const int head = tile % a.n_kv_heads, kv = (tile / a.n_kv_heads) & 1, rt = tile / (2 * a.n_kv_heads);
+    const int kv = hq & 1, rt = hq >> 1;
     const CUtensorMap* map = kv ? &maps.v : &maps.k;
     const uint32_t dst = sb + kTcSmX + s * kTcXBytes, bar = bar_full + 8 * s;
     tc_mbar_expect_tx(bar, kTcXBytes);
@@ -195,19 +205,18 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
           ::"r"(dst + h * 16384), "l"(map), "r"(h * 64), "r"(head), "r"(rt * 128), "r"(bar)
           : "memory");
   };
-  // Lane 0 of warps 0..3 each issue 4 of the 16 MMAs of local tile `it` into accumulator it & 1:
-  // issuer q takes term q >> 1 of S and k-half q & 1.  All MMAs accumulate (the accumulator is zero).
+  // Lane 0 of every warp issues one of the 16 MMAs of local tile `it` into accumulator it & 1: issuer q takes
+  // term q >> 3 of S, k-half (q >> 2) & 1 and k-step q & 3.  All MMAs accumulate (the accumulator is zero).
+  // The accumulator is free: its previous tile was read and cleared by every warp before the CTA-wide barrier
+  // that ended that tile, which this thread has passed.
   auto issue_mma = [&](int it, int q) {
     if (blockIdx.x + it * (int)gridDim.x >= n_tiles) return;
     const int s = it % kTcStages, acc = it & 1;
     if (!tc_mbar_wait(bar_full + 8 * s, (it / kTcStages) & 1, abort_flag)) return;
-    if (it >= 2 && !tc_mbar_wait(bar_tempty + 8 * acc, ((it >> 1) - 1) & 1, abort_flag)) return;
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t xa = sb + kTcSmX + s * kTcXBytes + (q & 1) * 16384;
-    const uint32_t sa = sb + kTcSmS + (q >> 1) * kTcSBytes + (q & 1) * 16384;
-    const uint32_t d = tmem_base + acc * 128;
-#pragma unroll
-    for (int ks = 0; ks < 4; ++ks) tc_mma(d, tc_smem_desc(xa + ks * 32), tc_smem_desc(sa + ks * 32), 1u);
+    const uint32_t off = ((q >> 2) & 1) * 16384 + (q & 3) * 32;
+    tc_mma(tmem_base + acc * 128, tc_smem_desc(sb + kTcSmX + s * kTcXBytes + off),
+           tc_smem_desc(sb + kTcSmS + (q >> 3) * kTcSBytes + off), 1u);
     tc_commit(bar_empty + 8 * s);     // the x stage may be refilled once these MMAs have read it
     tc_commit(bar_tfull + 8 * acc);   // this issuer's share of the accumulator is complete
   };
@@ -223,11 +232,13 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   }
-  if (tid == 0) {
-    issue_tma(0);
-    issue_tma(1);
-  }
-  if (lane == 0 && warp < 4) issue_mma(0, warp);
+  int head = (int)blockIdx.x % a.n_kv_heads, hq = (int)blockIdx.x / a.n_kv_heads;  // this tile
+  int head2 = head, hq2 = hq;                                                      // the tile two ahead
+  if (tid == 0) issue_tma(0, head2, hq2);
+  advance(head2, hq2);
+  if (tid == 0) issue_tma(1, head2, hq2);
+  advance(head2, hq2);
+  if (lane == 0) issue_mma(0, warp);
   __syncwarp();
 
   // ---- tile loop: all 16 warps are epilogue warps
@@ -236,30 +247,36 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   const int cq = warp >> 2;                      // columns [32*cq, 32*cq + 32): blocks 2cq, 2cq+1
   const int r = quarter * 32 + lane;             // row of the tile
   const bool uniform = (a.tables->flags & kFlagUniformL1) != 0u;
+  const bool sym = fq->sym != 0u;  // uniform over the grid
   const Layout L = make_layout(128, a.capacity);
   int rd_seq = 0, rd_first = 0, rd_count = 0, rd_start = -1;   // destination of the last row looked up
   int it = 0;
-  for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+  for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it, advance(head, hq)) {
     const int acc = it & 1;
-    const int head = tile % a.n_kv_heads, kv = (tile / a.n_kv_heads) & 1, rt = tile / (2 * a.n_kv_heads);
+    const int kv = hq & 1, rt = hq >> 1;
     // A wait that gives up must not leave the loop: the other warps may be past it and would wait
     // for this one at the named barriers.  The tile is skipped instead (warp-uniform).
     const bool ready = __all_sync(0xffffffffu, tc_mbar_wait(bar_tfull + 8 * acc, (it >> 1) & 1, abort_flag));
     // keep the pipeline fed: loads two tiles ahead, the next tile's MMAs under this tile's epilogue
-    if (tid == 0) issue_tma(it + 2);
-    if (lane == 0 && warp < 4) issue_mma(it + 1, warp);
+    if (tid == 0) issue_tma(it + 2, head2, hq2);
+    advance(head2, hq2);
+    if (lane == 0) issue_mma(it + 1, warp);
     __syncwarp();
     const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 128 + cq * 32;
-    // pass 1: squared norm of the row (its four column quarters are exchanged through shared memory)
+    // pass 1: the thread's 32 coordinates and their share of the row's squared norm (the four column
+    // quarters of a row are exchanged through shared memory)
     float sq = 0.f;
+    float y[32];
     if (ready) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      float y[32];
       tc_ld16(taddr, y);
       tc_ld16(taddr + 16, y + 16);
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
       for (int c = 0; c < 32; ++c) sq = fmaf(y[c], y[c], sq);
+    } else {
+#pragma unroll
+      for (int c = 0; c < 32; ++c) y[c] = 0.f;
     }
     rowsq[cq * 128 + r] = sq;
     // only the four warps that share these 32 rows exchange their parts of the norm
@@ -291,13 +308,11 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     uint32_t l2acc = 0, l3acc = 0, l4acc = 0, racc = 0, sat = 0;
     unsigned long long leftbits = 0ull;
     if (ready) {
-#pragma unroll 1
+#pragma unroll
       for (int i = 0; i < 2; ++i) {
-        float y[16];
-        tc_ld16(taddr + 16 * i, y);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         FastBlock fb;
-        polar_quant_block_fast(y, rm, *fq, &fb);
+        if (sym) polar_quant_block_fast<true>(y + 16 * i, rm, *fq, &fb);
+        else polar_quant_block_fast<false>(y + 16 * i, rm, *fq, &fb);
         if (!uniform) fb.amb |= 0xFFu;  // other level-1 codebooks: decide every level-1 angle exactly
         if (tb != nullptr) {
           *reinterpret_cast<uint32_t*>(tb + tok * 32 + cq * 8 + 4 * i) = fb.l1;
@@ -318,8 +333,6 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
       tc_st16_zero(taddr + 16);
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) tc_mbar_arrive(bar_tempty + 8 * acc);  // this accumulator may be written again
     }
     l4s[cq * 128 + r] = (uint8_t)l4acc;
     if (tb != nullptr) {

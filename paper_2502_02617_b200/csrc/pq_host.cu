@@ -185,7 +185,11 @@ int32_t pq_build_tables(const double* cen, const double* bnd, void* tables_host)
     t.n_upper += t.bnd_upper[k];
     if (std::fabs(bnd[k] - (k + 1) * kPi / 8.0) > 1e-12) uniform = false;
   }
-  t.flags = uniform ? pq::kFlagUniformL1 : 0u;
+  bool symmetric = true;
+  for (int l = 0; l < 3; ++l)
+    if (std::fabs(t.bnd_tan2[3 * l + 1] - 1.0) > 1e-9 || std::fabs(t.bnd_tan2[3 * l] * t.bnd_tan2[3 * l + 2] - 1.0) > 1e-9)
+      symmetric = false;
+  t.flags = (uniform ? pq::kFlagUniformL1 : 0u) | (symmetric ? pq::kFlagSymmetricUpper : 0u);
   for (int k = 0; k < PQ_N_CENTROIDS; ++k) {
     t.cen_cos[k] = (float)std::cos(cen[k]);
     t.cen_sin[k] = (float)std::sin(cen[k]);
