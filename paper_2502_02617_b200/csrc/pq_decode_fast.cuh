@@ -252,7 +252,7 @@ __device__ inline void build_fast_tables(uint8_t* smem, const Tables* tb) {
 // per CTA that works on it; the slots of all units sum to at most units + grid size.
 constexpr int kFastMaxGrid = 160;
 constexpr int kFastMaxUnits = 2048;  // (sequence, kv head) units the persistent schedule handles
-constexpr int kSegmentCost = 5;      // stages' worth of time a CTA spends on starting and finishing a unit
+constexpr int kSegmentCost = 7;     // stages' worth of time a CTA spends on starting and finishing a unit
 constexpr int kFastMaxSegs = 32;     // units one CTA can take part in (<= units / grid + 2)
 struct Segment {
   int unit, st0, st1, part, n_parts, slot0;
@@ -411,7 +411,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
         const float* qrow = q_in + (i & ~127);
         const float* scol = a.S + (i & 127);
         float acc = 0.f;
-#pragma unroll 16
+#pragma unroll 32
         for (int k = 0; k < 128; ++k) acc = fmaf(qrow[k], __ldg(scol + k * 128), acc);
         acc *= a.scale * 1.4426950408889634f;
         const __half qh = __float2half_rn(acc);
