@@ -270,7 +270,6 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
   int* is_last = reinterpret_cast<int*>(smem + kSmFlags) + 1;
   const int64_t head_bytes = make_layout(128, a.capacity).head_bytes;
 
-  build_fast_tables(smem, a.tables);
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
       mbar_init(sm_base + kSmBar + 8 * s, 1);                                  // full: producer + tx bytes
@@ -396,6 +395,9 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     const bool producer = (tid & 255) == 0;
     if (producer && n_li > 0) issue_copy(0);
     __syncwarp();
+    // The lookup tables are filled once, with the CTA's first copies already on their way (the barriers
+    // of the query rotation below order the fill before the first lookup).
+    if (sg == 0) build_fast_tables(smem, a.tables);
     // q' = (q S) * scale * log2(e) for the unit's query heads, as an fp16 value plus an fp16 residual.
     // The first stages of the segment are already on their way while this runs.
     {
