@@ -59,3 +59,59 @@ def test_random_shapes_against_oracle(seed):
             want = orc.decode_attention(to_f64(q[b, hk * g:(hk + 1) * g])[None], c[0][None, None], r[0][None, None],
                                         c[1][None, None], r[1][None, None], [n], cb, S, 128 ** -0.5)[0]
             assert rel_l2(got, want) < TOL_F32_IO, (seed, trial, B, Hq, Hkv, b, hk, n)
+
+
+@pytest.mark.parametrize("seed", [21, 22])
+def test_random_encode_chunks_against_oracle(seed):
+    """Encoder on randomly drawn chunk patterns: every sequence receives 1-4 chunks whose row counts sit around
+    the kernels' dispatch limits (per-vector kernel < 32 rows, float32-FMA kernel < 128 rows or float32 input or
+    odd strides, tensor-core kernel otherwise), from strided views; codes and radii of every stored vector are
+    compared with the oracle."""
+    from parity_utils import assert_codes_match, assert_radii_match, code_mismatch_report
+    rng = np.random.default_rng(seed)
+    total = dict(total=0, inside=0, outside=0)
+    for trial in range(8):
+        Hkv = int(rng.choice([1, 2, 3, 8]))
+        B = int(rng.choice([1, 2, 4, 7]))
+        dt = torch.bfloat16 if rng.integers(3) else torch.float32
+        cap = int(rng.integers(200, 1500))
+        cache = pq.PolarQuantCache(B, Hkv, Hkv, 128, capacity=cap, seed=int(rng.integers(1000)), device=DEV)
+        S, cb = cache.S_host.double().numpy(), oracle_codebooks(cache)
+        done = [0] * B
+        hist = [[] for _ in range(B)]
+        for _chunk in range(int(rng.integers(1, 5))):
+            take = [int(min(cap - done[b], rng.choice([0, 1, 3, 31, 32, 33, 100, 127, 128, 129, 300]))) for b in range(B)]
+            n = sum(take)
+            if n == 0:
+                continue
+            pad_h, pad_d = int(rng.integers(0, 2)), int(rng.choice([0, 8, 64]))
+            if dt == torch.float32 and rng.integers(2):
+                pad_d = 3
+            big_k, big_v = synthetic.kv_like(int(rng.integers(100000)), n, Hkv + pad_h, 128 + pad_d, dt, DEV)
+            off = 8 if pad_d and pad_d % 8 == 0 and rng.integers(2) else 0
+            K, V = big_k[:, pad_h:, off:off + 128], big_v[:, pad_h:, off:off + 128]
+            cu = torch.tensor(np.concatenate(([0], np.cumsum(take))), dtype=torch.int32, device=DEV)
+            cache.encode(K, V, cu)
+            r0 = 0
+            for b in range(B):
+                if take[b]:
+                    hist[b].append((K[r0:r0 + take[b]].clone(), V[r0:r0 + take[b]].clone()))
+                r0 += take[b]
+                done[b] += take[b]
+        torch.cuda.synchronize()
+        cache.check_status()
+        assert cache.lens.cpu().tolist() == done
+        if max(done) == 0:
+            continue
+        codes, radii = cache.unpack(max(done))
+        for b in range(B):
+            if not done[b]:
+                continue
+            for kv in (0, 1):
+                X = torch.cat([h[kv] for h in hist[b]])
+                for h in range(Hkv):
+                    rep = code_mismatch_report(codes[b, h, kv, :done[b]].cpu().numpy(), to_f64(X[:, h]), S, cb)
+                    assert_radii_match(radii[b, h, kv, :done[b]].cpu().numpy(), rep["radii16"])
+                    for key in total:
+                        total[key] += rep[key]
+    assert_codes_match(total)
