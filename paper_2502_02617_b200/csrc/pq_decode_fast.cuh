@@ -143,6 +143,14 @@ __device__ __forceinline__ uint32_t lds8(uint32_t addr) {
   return v;
 }
 
+// 2^x, x <= 0 or slightly above (ex2.approx: relative error 2^-22; 2^-inf = 0)
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+constexpr float kLazyMax = 8.f;
+
 __device__ __forceinline__ __half2 as_h2(uint32_t v) { return *reinterpret_cast<__half2*>(&v); }
 __device__ __forceinline__ uint32_t as_u32(__half2 v) { return *reinterpret_cast<uint32_t*>(&v); }
 
@@ -369,7 +377,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     float o_acc[8][4];  // tile i (pair i of block g): rows 2i / 2i+1 of block g, heads 2c / 2c+1
 #pragma unroll
     for (int i = 0; i < 8; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
-    float m_run[kHG], l_run[kHG];  // of head c + 4 hg (replicated over the 8 lanes with the same c)
+    float m_run[kHG], l_run[kHG];  // of head c + 4 hg: reference (the same in the 8 lanes with this c), own share of the sum
 #pragma unroll
     for (int hg = 0; hg < kHG; ++hg) {
       m_run[hg] = -CUDART_INF_F;
@@ -488,32 +496,33 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
           }
 #undef PQ_KSTEP
         }
-        // ---- online softmax: this thread holds head c (+ 4 hg) of tokens g and g + 8
+        // ---- online softmax: this thread holds head c (+ 4 hg) of tokens g and g + 8.  The reference m_run of a
+        // head moves only when a score exceeds it by more than kLazyMax (log2 units), so p = 2^(s - m_run) stays
+        // below 2^kLazyMax (fp16 holds it with its full relative precision) and the common tile needs neither
+        // the reductions over tokens nor a rescaling; l_run is this thread's share of the denominator (its own
+        // tokens), summed over the eight lanes of the head when the segment ends.
         const bool ok0 = tile_tok0 + g < len, ok1 = tile_tok0 + g + 8 < len;
-        uint32_t ph[kHG];   // (p of token g, p of token g + 8) in fp16
-        float corr[kHG];
-        bool grew = false;
+        float s0[kHG], s1[kHG];
+        bool over = false;
 #pragma unroll
         for (int hg = 0; hg < kHG; ++hg) {
-          const float s0 = ok0 ? (scl[hg][0] + scl[hg][1]) + sc[hg][1] + sc[hg][0] : -CUDART_INF_F;  // small terms first
-          const float s1 = ok1 ? (scl[hg][2] + scl[hg][3]) + sc[hg][3] + sc[hg][2] : -CUDART_INF_F;
-          float mx = fmaxf(s0, s1);
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
-          mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
-          const float m_new = fmaxf(m_run[hg], mx);  // finite: token 0 of the tile is inside the sequence
-          const float p0 = exp2f(s0 - m_new), p1 = exp2f(s1 - m_new);
-          float psum = p0 + p1;
-          psum += __shfl_xor_sync(0xffffffffu, psum, 4);
-          psum += __shfl_xor_sync(0xffffffffu, psum, 8);
-          psum += __shfl_xor_sync(0xffffffffu, psum, 16);
-          corr[hg] = exp2f(m_run[hg] - m_new);  // 0 on the first tile (m_run = -inf)
-          l_run[hg] = l_run[hg] * corr[hg] + psum;
-          grew = grew || m_new > m_run[hg];
-          m_run[hg] = m_new;
-          ph[hg] = as_u32(__floats2half2_rn(p0, p1));
+          s0[hg] = ok0 ? (scl[hg][0] + scl[hg][1]) + sc[hg][1] + sc[hg][0] : -CUDART_INF_F;  // small terms first
+          s1[hg] = ok1 ? (scl[hg][2] + scl[hg][3]) + sc[hg][3] + sc[hg][2] : -CUDART_INF_F;
+          over = over || fmaxf(s0[hg], s1[hg]) > m_run[hg] + kLazyMax;  // always on the first tile (m_run = -inf)
         }
-        if (__any_sync(0xffffffffu, grew)) {
+        if (__any_sync(0xffffffffu, over)) {
+          float corr[kHG];
+#pragma unroll
+          for (int hg = 0; hg < kHG; ++hg) {
+            float mx = fmaxf(s0[hg], s1[hg]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+            const float m_new = fmaxf(m_run[hg], mx);  // finite: token 0 of the tile is inside the sequence
+            corr[hg] = fast_exp2(m_run[hg] - m_new);   // 0 on the first tile
+            l_run[hg] *= corr[hg];
+            m_run[hg] = m_new;
+          }
           // accumulator columns 2c, 2c+1 are heads 2c, 2c+1: their factors live in lanes (2c) & 3, (2c+1) & 3
           float c0 = __shfl_sync(0xffffffffu, corr[0], (2 * c) & 3);
           float c1 = __shfl_sync(0xffffffffu, corr[0], (2 * c + 1) & 3);
@@ -532,6 +541,13 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
             o_acc[i][2] *= c0;
             o_acc[i][3] *= c1;
           }
+        }
+        uint32_t ph[kHG];   // (p of token g, p of token g + 8) in fp16
+#pragma unroll
+        for (int hg = 0; hg < kHG; ++hg) {
+          const float p0 = fast_exp2(s0[hg] - m_run[hg]), p1 = fast_exp2(s1[hg] - m_run[hg]);
+          l_run[hg] += p0 + p1;
+          ph[hg] = as_u32(__floats2half2_rn(p0, p1));
         }
         // B operand of the value MMAs: column n = g is head g, rows 2c, 2c+1 | 2c+8, 2c+9 = tokens c, c+4 | c+8, c+12
         uint32_t pb0, pb1;
@@ -602,6 +618,12 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     // accumulator register the 32 lanes (block g, head pair c) then hit 32 different banks.
     float* mrg_o = reinterpret_cast<float*>(smem + kSmRing);          // [16 warps][8 heads][kMrgStride]
     float* mrg_ml = mrg_o + kFastConsumerWarps * 8 * kMrgStride;      // [16 warps][8 heads][2]
+#pragma unroll
+    for (int hg = 0; hg < kHG; ++hg) {  // the head's denominator: sum of the shares of its eight lanes
+      l_run[hg] += __shfl_xor_sync(0xffffffffu, l_run[hg], 4);
+      l_run[hg] += __shfl_xor_sync(0xffffffffu, l_run[hg], 8);
+      l_run[hg] += __shfl_xor_sync(0xffffffffu, l_run[hg], 16);
+    }
     if (g == 0) {
 #pragma unroll
       for (int hg = 0; hg < kHG; ++hg) {
