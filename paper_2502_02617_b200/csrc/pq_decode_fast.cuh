@@ -46,7 +46,7 @@ constexpr int kSmSegs = kSmFlags + 16;                // Segment[32] : 768
 constexpr int kSmQ = kSmSegs + 768;                   // q (fp32) [8][128], q' fp16 value [8][128], q' fp16 residual [8][128] : 8192
 constexpr int kSmRing = (kSmQ + 8192 + 127) / 128 * 128;
 // after the main loop the ring is reused for the cross-warp merge: 16 warps x 8 heads x (128 + 2) floats
-constexpr int kMrgStride = 132;  // floats per (warp, head) row of the merge buffer (132 = 128 + 4: bank spread)
+constexpr int kMrgStride = 136;  // floats per (warp, head) row of the merge buffer (136 = 128 + 8: heads 8 banks apart)
 constexpr int kMergeBytes = 16 * 8 * kMrgStride * 4 + 16 * 8 * 2 * 4;  // also >= combine_smem_floats(8, 128, 160) * 4
 constexpr int kSmUsed = kSmRing + (kStages * kStageBytes > kMergeBytes ? kStages * kStageBytes : kMergeBytes);
 // The tables start on a 32 KB boundary of the shared window, so that a table address is the OR of
@@ -374,9 +374,12 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     const uint8_t* head_base = a.cache + ((int64_t)b * a.n_kv_heads + hk) * head_bytes;
 
     // per-thread attention state
-    float o_acc[8][4];  // tile i (pair i of block g): rows 2i / 2i+1 of block g, heads 2c / 2c+1
+    // o_acc[hg][S][.]: head c + 4 hg, block g, coordinates 4S, 4S + 2, 4S + 1, 4S + 3 (see the value MMAs)
+    float o_acc[kHG][4][4];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) o_acc[i][0] = o_acc[i][1] = o_acc[i][2] = o_acc[i][3] = 0.f;
+    for (int hg = 0; hg < kHG; ++hg)
+#pragma unroll
+      for (int i = 0; i < 4; ++i) o_acc[hg][i][0] = o_acc[hg][i][1] = o_acc[hg][i][2] = o_acc[hg][i][3] = 0.f;
     float m_run[kHG], l_run[kHG];  // of head c + 4 hg: reference (the same in the 8 lanes with this c), own share of the sum
 #pragma unroll
     for (int hg = 0; hg < kHG; ++hg) {
@@ -523,24 +526,15 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
             l_run[hg] *= corr[hg];
             m_run[hg] = m_new;
           }
-          // accumulator columns 2c, 2c+1 are heads 2c, 2c+1: their factors live in lanes (2c) & 3, (2c+1) & 3
-          float c0 = __shfl_sync(0xffffffffu, corr[0], (2 * c) & 3);
-          float c1 = __shfl_sync(0xffffffffu, corr[0], (2 * c + 1) & 3);
-          if (kHG == 2) {
-            const float d0 = __shfl_sync(0xffffffffu, corr[kHG - 1], (2 * c) & 3);
-            const float d1 = __shfl_sync(0xffffffffu, corr[kHG - 1], (2 * c + 1) & 3);
-            if (c >= 2) {
-              c0 = d0;
-              c1 = d1;
-            }
-          }
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            o_acc[i][0] *= c0;
-            o_acc[i][1] *= c1;
-            o_acc[i][2] *= c0;
-            o_acc[i][3] *= c1;
-          }
+          for (int hg = 0; hg < kHG; ++hg)  // the accumulators of this thread belong to its own head
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              o_acc[hg][i][0] *= corr[hg];
+              o_acc[hg][i][1] *= corr[hg];
+              o_acc[hg][i][2] *= corr[hg];
+              o_acc[hg][i][3] *= corr[hg];
+            }
         }
         uint32_t ph[kHG];   // (p of token g, p of token g + 8) in fp16
 #pragma unroll
@@ -549,22 +543,22 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
           l_run[hg] += p0 + p1;
           ph[hg] = as_u32(__floats2half2_rn(p0, p1));
         }
-        // B operand of the value MMAs: column n = g is head g, rows 2c, 2c+1 | 2c+8, 2c+9 = tokens c, c+4 | c+8, c+12
-        uint32_t pb0, pb1;
-        {
-          const int srcA = c * 4 + (g & 3), srcB = srcA + 16;
-          uint32_t uA = __shfl_sync(0xffffffffu, ph[0], srcA), uB = __shfl_sync(0xffffffffu, ph[0], srcB);
-          if (kHG == 2) {
-            const uint32_t wA = __shfl_sync(0xffffffffu, ph[kHG - 1], srcA), wB = __shfl_sync(0xffffffffu, ph[kHG - 1], srcB);
-            if (g >= 4) {
-              uA = wA;
-              uB = wB;
-            }
-          }
-          pb0 = __byte_perm(uA, uB, 0x5410);
-          pb1 = __byte_perm(uA, uB, 0x7632);
+        // B operand of the value MMAs.  The contraction index is (token, which element of a decoded half2): rows
+        // 2c, 2c+1 = token c (first MMA) or c + 8 (second), rows 2c+8, 2c+9 = token c + 4 or c + 12.  Column
+        // n = 2h + e is head h restricted to element e: its entry is p in half e and zero in the other, so a
+        // decoded half2 is an A register as it is and no column of the MMA is idle (4 heads x 2 elements).
+        uint32_t pb[kHG][2][2];
+#pragma unroll
+        for (int hg = 0; hg < kHG; ++hg) {
+          const int srcA = c * 4 + (g >> 1);  // lane that holds tokens c and c + 8 of head g >> 1
+          const uint32_t uA = __shfl_sync(0xffffffffu, ph[hg], srcA), uB = __shfl_sync(0xffffffffu, ph[hg], srcA + 16);
+          const uint32_t sel_lo = (g & 1) ? 0x1044u : 0x4410u, sel_hi = (g & 1) ? 0x3244u : 0x4432u;
+          pb[hg][0][0] = __byte_perm(uA, 0u, sel_lo);
+          pb[hg][0][1] = __byte_perm(uB, 0u, sel_lo);
+          pb[hg][1][0] = __byte_perm(uA, 0u, sel_hi);
+          pb[hg][1][1] = __byte_perm(uB, 0u, sel_hi);
         }
-        // ---- values: block g of tokens 2c, 2c+1, 2c+8, 2c+9 -> O^T (coordinates x heads) += V_hat^T P
+        // ---- values: block g of tokens c, c+4, c+8, c+12 -> O^T (coordinates x (head, element)) += V_hat^T P
         {
           BlockRef bv[4];
 #define PQ_VLOAD(J)                                                                                          \
@@ -586,12 +580,10 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     sub_block_h2<S>(bv[1], t1a, x1, y1);                                                                 \
     sub_block_h2<S>(bv[2], t1a, x2, y2);                                                                 \
     sub_block_h2<S>(bv[3], t1a, x3, y3);                                                                 \
-    mma_16816(o_acc[2 * (S)], __byte_perm(as_u32(x0), as_u32(x1), 0x5410),                               \
-              __byte_perm(as_u32(y0), as_u32(y1), 0x5410), __byte_perm(as_u32(x2), as_u32(x3), 0x5410),  \
-              __byte_perm(as_u32(y2), as_u32(y3), 0x5410), pb0, pb1);                                    \
-    mma_16816(o_acc[2 * (S) + 1], __byte_perm(as_u32(x0), as_u32(x1), 0x7632),                           \
-              __byte_perm(as_u32(y0), as_u32(y1), 0x7632), __byte_perm(as_u32(x2), as_u32(x3), 0x7632),  \
-              __byte_perm(as_u32(y2), as_u32(y3), 0x7632), pb0, pb1);                                    \
+    _Pragma("unroll") for (int hg = 0; hg < kHG; ++hg) {                                                 \
+      mma_16816(o_acc[hg][S], as_u32(x0), as_u32(y0), as_u32(x1), as_u32(y1), pb[hg][0][0], pb[hg][0][1]); \
+      mma_16816(o_acc[hg][S], as_u32(x2), as_u32(y2), as_u32(x3), as_u32(y3), pb[hg][1][0], pb[hg][1][1]); \
+    }                                                                                                    \
   }
           PQ_VSTEP(0) PQ_VSTEP(1) PQ_VSTEP(2) PQ_VSTEP(3)
 #undef PQ_VSTEP
@@ -615,7 +607,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
 
     // ---- merge the 16 warps (fixed order), write this part's partial, last part combines the unit
     // Coordinate j of head h of warp w sits at (w * 8 + h) * kMrgStride + (j & 15) * 8 + (j >> 4): for a fixed
-    // accumulator register the 32 lanes (block g, head pair c) then hit 32 different banks.
+    // accumulator register the 32 lanes (block g, head c) then hit 32 different banks.
     float* mrg_o = reinterpret_cast<float*>(smem + kSmRing);          // [16 warps][8 heads][kMrgStride]
     float* mrg_ml = mrg_o + kFastConsumerWarps * 8 * kMrgStride;      // [16 warps][8 heads][2]
 #pragma unroll
@@ -635,17 +627,18 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
         mrg_ml[(warp * 8 + c + 4) * 2 + 1] = 0.f;
       }
     }
-    if (2 * c < g_heads) {
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        float* o0 = mrg_o + (warp * 8 + 2 * c) * kMrgStride + (2 * i) * 8 + g;
-        float* o1 = o0 + kMrgStride;
-        o0[0] = o_acc[i][0];
-        o1[0] = o_acc[i][1];
-        o0[8] = o_acc[i][2];
-        o1[8] = o_acc[i][3];
+    for (int hg = 0; hg < kHG; ++hg)
+      if (c + 4 * hg < g_heads) {
+        float* o0 = mrg_o + (warp * 8 + c + 4 * hg) * kMrgStride + g;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          o0[(4 * i) * 8] = o_acc[hg][i][0];
+          o0[(4 * i + 2) * 8] = o_acc[hg][i][1];
+          o0[(4 * i + 1) * 8] = o_acc[hg][i][2];
+          o0[(4 * i + 3) * 8] = o_acc[hg][i][3];
+        }
       }
-    }
     __syncthreads();
     const int slot = unit_slot + (cta - c_first);
     for (int idx = tid; idx < g_heads * 128; idx += kFastThreads) {
