@@ -366,8 +366,8 @@ def run_cuda(args):
     if rank != 0:
         return
     # DRAM bytes of one decode-attention launch: ncu capture at batch 4 (profiles/decode_attention_fast_kernel_
-    # batch4_ctx32768.md: 130.50 MB read + 4.10 MB written), scaled by the batch (traffic is proportional to it)
-    traffic = (130.50e6 + 4.10e6) * BATCH / 4.0
+    # batch4_ctx32768.md: 130.47 MB read + 3.45 MB written), scaled by the batch (traffic is proportional to it)
+    traffic = (130.47e6 + 3.45e6) * BATCH / 4.0
     cpu = _oracle_sample_throughput(12.0) if world == 1 and not args.no_cpu_baseline else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
