@@ -460,7 +460,6 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
       if (tile_tok0 < len) {
         const uint32_t kblk = sm_base + kSmRing + s * kStageBytes + ((warp >> 2) & 1) * 2 * kBlockBytes128;
         const uint32_t vblk = kblk + kBlockBytes128;
-        const int t0 = (warp & 3) * 16;  // tile's first token inside its token-block
         // ---- scores S (tokens x columns): A operand = keys of tokens g (rows 0..7) and g + 8 (rows 8..15),
         // decoded as hi + lo; one MMA with the hi parts and one with the lo parts per k-step.  Column 2c is
         // q_hi of head c, column 2c+1 its q_lo, so all four products of a (token, head) land in this thread.

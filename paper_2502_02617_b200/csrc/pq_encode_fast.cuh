@@ -80,48 +80,6 @@ __device__ __forceinline__ uint32_t quant_upper_fast(float sa, float sb, const f
   return 3u - neg;
 }
 
-// The same decision for symmetric boundaries (T0, 1, 1/T0), folded onto m = min(sa, sb), M = max(sa, sb):
-// only the diagonal (M - m) and the boundary m = T0 M of the point's own side can be the nearest ones, and the
-// margin of the boundary sb = sa / T0 is the one of m = T0 M after multiplying both sides by T0^2.  Every T
-// that is tested is <= 1, so sb + T^2 sa <= sa + sb and the caller's `base` uses (1 + T)^2 <= 4.
-__device__ __forceinline__ uint32_t quant_upper_sym(float sa, float sb, float T0, float c, float base, bool* ambiguous) {
-  const float m = fminf(sa, sb), M = fmaxf(sa, sb);
-  const bool hi = sb > sa;
-  const float dout = fmaf(-T0, M, m), ddiag = M - m;
-  const bool lo = dout > 0.f;
-  const float w = sa + sb;
-  const float dm = fminf(fabsf(dout), ddiag);
-  const float b2 = fmaf(4.2e-11f * w, w, base);  // rho = 1e-6 covers the float32 roundings
-  bool amb = !(dm * dm > fmaf(c, w, b2));        // also true for NaN margins
-  if (amb) {
-    const bool ok_d = ddiag * ddiag > fmaf(c, w, b2);
-    const bool ok_o = dout * dout > fmaf(c, fmaf(T0 * T0, M, m), b2);
-    amb = !(ok_d && ok_o);
-  }
-  *ambiguous = amb;
-  return (hi ? 3u : 0u) ^ (lo ? 1u : 0u);
-}
-
-// Level-1 decision for the uniform codebook (boundaries k pi/8): fold into the first octant,
-// u = max(|a|,|b|), v = min(|a|,|b|); the boundaries are the axes (v = 0), the diagonals (u = v) and
-// the lines at pi/8 from the axes (v cos(pi/8) = u sin(pi/8)).  Each coordinate moves by at most
-// dy, so the signed distance to a line with unit normal (n1, n2) moves by at most (|n1| + |n2|) dy:
-// dy for an axis, sqrt(2) dy for a diagonal, (cos + sin)(pi/8) dy = 1.3066 dy for the pi/8 lines.
-// The three distances are scaled so that one comparison against dy serves all.
-__device__ __forceinline__ uint32_t quant_level1_fast(float a, float b, float dy, bool* ambiguous) {
-  const float ax = fabsf(a), ay = fabsf(b);
-  const float u = fmaxf(ax, ay), v = fminf(ax, ay);
-  const bool swap = ay > ax;
-  const float t = fmaf(v, 0.92387953251128674f, -u * 0.38268343236508977f);  // v cos(pi/8) - u sin(pi/8)
-  const bool hi = t > 0.f;
-  const float dmin = fminf(fminf(v, (u - v) * 0.5f), fabsf(t) * 0.76536686473017954f);
-  *ambiguous = !(dmin > fmaf(u, 4.76837158203125e-07f, dy));  // + 2^-21 u for the float32 roundings
-  const uint32_t sector = swap ? (hi ? 2u : 3u) : (hi ? 1u : 0u);  // pi/8 sector inside the quadrant
-  const uint32_t sa = __float_as_uint(a) >> 31, sb = __float_as_uint(b) >> 31;
-  // b >= 0: theta = phi or pi - phi; b < 0: theta = pi + phi or 2 pi - phi
-  return (sb << 3) + (sector ^ ((sa ^ sb) ? 7u : 0u));
-}
-
 // Codes, squared radius and ambiguity mask of one 16-coordinate block.
 // Ambiguity bits: 0..7 level-1 pairs, 8..11 level 2, 12..13 level 3, 14 level 4.
 struct FastBlock {
@@ -135,41 +93,106 @@ __device__ __forceinline__ float fast_sqrt(float x) {
   return r;
 }
 
-template <bool kSym>
-__device__ __forceinline__ uint32_t quant_upper_any(float sa, float sb, const float* T, float c, float base, bool* am) {
-  return kSym ? quant_upper_sym(sa, sb, T[0], c, base, am) : quant_upper_fast(sa, sb, T, c, base, am);
+// ---- decisions whose code bits are read off sign bits ------------------------------------------
+// (acc << 1) | sign bit of v: one funnel shift collects a decision bit.
+__device__ __forceinline__ uint32_t push_sign(uint32_t acc, uint32_t v) { return __funnelshift_l(v, acc, 1); }
+
+// Level-1 decision for the uniform codebook (boundaries k pi/8): fold into the first octant,
+// u = max(|a|,|b|), v = min(|a|,|b|); the boundaries are the axes (v = 0), the diagonals (u = v) and
+// the lines at pi/8 from the axes (v cos(pi/8) = u sin(pi/8)).  Each coordinate moves by at most
+// dy, so the signed distance to a line with unit normal (n1, n2) moves by at most (|n1| + |n2|) dy:
+// dy for an axis, sqrt(2) dy for a diagonal, (cos + sin)(pi/8) dy = 1.3066 dy for the pi/8 lines.
+// The three distances are scaled so that one comparison against dy serves all.
+// The function appends the 4 code bits to `l1` and one "certified" bit to
+// `ok`.  With x = sign(a) ^ sign(b), w = (|b| > |a|), hi = (past the pi/8 line of the folded octant) the code
+// is sign(b) << 3 | x << 2 | (w ^ x) << 1 | (w ^ hi ^ x); w is the sign of |a| - |b| and hi the complement of
+// the sign of t.  A zero (or NaN) anywhere leaves the pair uncertified, so the sign conventions at exact
+// zeros do not matter.
+__device__ __forceinline__ void quant_level1_push(float a, float b, float dy, uint32_t& l1, uint32_t& ok) {
+  const float ax = fabsf(a), ay = fabsf(b);
+  const float u = fmaxf(ax, ay), v = fminf(ax, ay);
+  const float d = ax - ay;
+  const float t = fmaf(v, 0.92387953251128674f, -u * 0.38268343236508977f);  // v cos(pi/8) - u sin(pi/8)
+  const float dmin = fminf(fminf(v, fabsf(d) * 0.5f), fabsf(t) * 0.76536686473017954f);
+  const float slack = fmaf(u, 4.76837158203125e-07f, dy) - dmin;  // < 0: certified (+ 2^-21 u for the float32 roundings)
+  const uint32_t bb = __float_as_uint(b), x = __float_as_uint(a) ^ bb;
+  const uint32_t e1 = __float_as_uint(d) ^ x;
+  const uint32_t e0 = ~(__float_as_uint(t) ^ e1);
+  l1 = push_sign(push_sign(push_sign(push_sign(l1, bb), x), e1), e0);
+  ok = push_sign(ok, __float_as_uint(slack));
 }
 
+// The level >= 2 decision (see quant_upper_fast) for symmetric boundaries (T0, 1, 1/T0), folded onto m = min(sa, sb), M = max(sa, sb):
+// only the diagonal (M - m) and the boundary m = T0 M of the point's own side can be the nearest ones, and the
+// margin of the boundary sb = sa / T0 is the one of m = T0 M after multiplying both sides by T0^2.  Every T
+// that is tested is <= 1, so sb + T^2 sa <= sa + sb and the caller's `base` uses (1 + T)^2 <= 4.
+// The function appends the 2 code bits to `lv` and one "certified" bit to `ok`: the code is
+// hi << 1 | (hi ^ lo) with hi = (sb > sa) = sign of sa - sb and lo = (m > T0 M) = complement of the sign of dout.
+__device__ __forceinline__ void quant_upper_sym_push(float sa, float sb, float T0, float c, float base, uint32_t& lv,
+                                                     uint32_t& ok) {
+  const float m = fminf(sa, sb), M = fmaxf(sa, sb);
+  const float h = sa - sb, dout = fmaf(-T0, M, m);
+  const float w = sa + sb;
+  const float dm = fminf(fabsf(dout), fabsf(h));
+  const float b2 = fmaf(4.2e-11f * w, w, base);  // rho = 1e-6 covers the float32 roundings
+  float slack = fmaf(-dm, dm, fmaf(c, w, b2));   // < 0: certified by the cheap test
+  if (!(slack < 0.f)) {                          // rare; also taken for NaN
+    const bool ok_d = h * h > fmaf(c, w, b2);
+    const bool ok_o = dout * dout > fmaf(c, fmaf(T0 * T0, M, m), b2);
+    slack = (ok_d && ok_o) ? -1.f : 1.f;
+  }
+  const uint32_t hb = __float_as_uint(h);
+  lv = push_sign(push_sign(lv, hb), ~(hb ^ __float_as_uint(dout)));
+  ok = push_sign(ok, __float_as_uint(slack));
+}
+
+// Codes, squared radius and ambiguity mask of one block.  Pairs and nodes are visited from the last to the
+// first, so that the bits that are appended end up in canonical order.
 template <bool kSym>
 __device__ __forceinline__ void polar_quant_block_fast(const float* y, const RowMargins& rm, const FastQuant& fq,
                                                        FastBlock* out) {
   float s1[8], s2[4], s3[2];
-  uint32_t l1 = 0, l2 = 0, l3 = 0, amb = 0;
-  bool am;
+  uint32_t l1 = 0, l2 = 0, l3 = 0, l4 = 0, ok1 = 0, ok2 = 0, ok3 = 0, ok4 = 0;
 #pragma unroll
-  for (int j = 0; j < 8; ++j) {
-    l1 |= quant_level1_fast(y[2 * j], y[2 * j + 1], rm.dy, &am) << (4 * j);
-    amb |= (am ? 1u : 0u) << j;
+  for (int j = 7; j >= 0; --j) {
+    quant_level1_push(y[2 * j], y[2 * j + 1], rm.dy, l1, ok1);
     s1[j] = fmaf(y[2 * j], y[2 * j], y[2 * j + 1] * y[2 * j + 1]);
   }
+  if (kSym) {
 #pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    l2 |= quant_upper_any<kSym>(s1[2 * j], s1[2 * j + 1], fq.t2[0], rm.c[0], rm.base[0], &am) << (2 * j);
-    amb |= (am ? 1u : 0u) << (8 + j);
-    s2[j] = s1[2 * j] + s1[2 * j + 1];
-  }
+    for (int j = 3; j >= 0; --j) {
+      quant_upper_sym_push(s1[2 * j], s1[2 * j + 1], fq.t2[0][0], rm.c[0], rm.base[0], l2, ok2);
+      s2[j] = s1[2 * j] + s1[2 * j + 1];
+    }
 #pragma unroll
-  for (int j = 0; j < 2; ++j) {
-    l3 |= quant_upper_any<kSym>(s2[2 * j], s2[2 * j + 1], fq.t2[1], rm.c[1], rm.base[1], &am) << (2 * j);
-    amb |= (am ? 1u : 0u) << (12 + j);
-    s3[j] = s2[2 * j] + s2[2 * j + 1];
+    for (int j = 1; j >= 0; --j) {
+      quant_upper_sym_push(s2[2 * j], s2[2 * j + 1], fq.t2[1][0], rm.c[1], rm.base[1], l3, ok3);
+      s3[j] = s2[2 * j] + s2[2 * j + 1];
+    }
+    quant_upper_sym_push(s3[0], s3[1], fq.t2[2][0], rm.c[2], rm.base[2], l4, ok4);
+  } else {
+    bool am;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      l2 |= quant_upper_fast(s1[2 * j], s1[2 * j + 1], fq.t2[0], rm.c[0], rm.base[0], &am) << (2 * j);
+      ok2 |= (am ? 0u : 1u) << j;
+      s2[j] = s1[2 * j] + s1[2 * j + 1];
+    }
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+      l3 |= quant_upper_fast(s2[2 * j], s2[2 * j + 1], fq.t2[1], rm.c[1], rm.base[1], &am) << (2 * j);
+      ok3 |= (am ? 0u : 1u) << j;
+      s3[j] = s2[2 * j] + s2[2 * j + 1];
+    }
+    l4 = quant_upper_fast(s3[0], s3[1], fq.t2[2], rm.c[2], rm.base[2], &am);
+    ok4 = am ? 0u : 1u;
   }
-  out->l4 = quant_upper_any<kSym>(s3[0], s3[1], fq.t2[2], rm.c[2], rm.base[2], &am);
-  amb |= (am ? 1u : 0u) << 14;
   out->l1 = l1;
   out->l2 = l2;
   out->l3 = l3;
-  out->amb = amb;
+  out->l4 = l4;
+  // ambiguity bits: 0..7 level-1 pairs, 8..11 level 2, 12..13 level 3, 14 level 4
+  out->amb = ~(ok1 | (ok2 << 8) | (ok3 << 12) | (ok4 << 14)) & 0x7FFFu;
   out->radius = fast_sqrt(s3[0] + s3[1]);
 }
 
