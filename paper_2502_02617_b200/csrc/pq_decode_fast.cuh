@@ -10,9 +10,9 @@
 // Per tile a warp
 //   * decodes the keys of 16 tokens straight into mma.sync A fragments (fp16, rotated basis) with
 //     shared-memory table lookups, and forms S = K_hat q'^T (tokens x heads) on tensor cores,
-//   * runs the online softmax on the S fragment (log2 domain, fp32),
-//   * decodes the values into A fragments (coordinates x tokens) and accumulates
-//     O^T += V_hat^T P on tensor cores (fp32 accumulators in registers).
+//   * runs the online softmax on the S fragment (log2 domain, fp32, lazily updated reference),
+//   * decodes the values into A fragments (coordinates x (token, element of a decoded pair)) and
+//     accumulates O^T += V_hat^T P on tensor cores (fp32 accumulators in registers).
 // DeQuant (Algorithm 1) of one 16-coordinate block is a product tree r * t4 * t3 * t2 * t1.
 // Levels 4..2 are folded into one table per 4-coordinate sub-block, level 1 is a half2 multiply:
 //   u    [4][64][16] sub-block s, index c2_s | c3_(s>>1) << 2 | c4 << 4 -> the multipliers of the
@@ -45,7 +45,7 @@ constexpr int kSmFlags = kSmBar + 64;                 // abort flag, is_last, n_
 constexpr int kSmSegs = kSmFlags + 16;                // Segment[32] : 768
 constexpr int kSmQ = kSmSegs + 768;                   // q (fp32) [8][128], q' fp16 value [8][128], q' fp16 residual [8][128] : 8192
 constexpr int kSmRing = (kSmQ + 8192 + 127) / 128 * 128;
-// after the main loop the ring is reused for the cross-warp merge: 16 warps x 8 heads x (128 + 2) floats
+// after the main loop the ring is reused for the cross-warp merge: 16 warps x 8 heads x (kMrgStride + 2) floats
 constexpr int kMrgStride = 136;  // floats per (warp, head) row of the merge buffer (136 = 128 + 8: heads 8 banks apart)
 constexpr int kMergeBytes = 16 * 8 * kMrgStride * 4 + 16 * 8 * 2 * 4;  // also >= combine_smem_floats(8, 128, 160) * 4
 constexpr int kSmUsed = kSmRing + (kStages * kStageBytes > kMergeBytes ? kStages * kStageBytes : kMergeBytes);
