@@ -32,7 +32,7 @@ constexpr int kTcSmS = 0;                  // S_hi, S_lo
 constexpr int kTcSmX = kTcSmS + 2 * kTcSBytes;
 constexpr int kTcSmRowSq = kTcSmX + kTcStages * kTcXBytes;   // [4][128] float, then [4][128] bytes of level-4 nibbles
 constexpr int kTcSmFq = kTcSmRowSq + 2048 + 512;             // FastQuant (40 B)
-constexpr int kTcSmBar = kTcSmFq + 64;                       // full[3], empty[3], tfull[2]
+constexpr int kTcSmBar = kTcSmFq + 64;                       // full[3], tfull[2]
 constexpr int kTcSmMisc = kTcSmBar + 128;                    // tmem base, abort flag
 constexpr int kTcSmFix = kTcSmMisc + 64;                     // FixQueue
 constexpr int kTcSmTotal = kTcSmFix + (int)sizeof(FixQueue) + 1024;  // + slack for 1024-byte alignment
@@ -60,7 +60,19 @@ __device__ __forceinline__ bool tc_mbar_try(uint32_t bar, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ bool tc_mbar_test(uint32_t bar, uint32_t parity) {  // non-blocking probe
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ bool tc_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (tc_mbar_test(bar, parity)) return true;  // the usual case: completed a tile ago
   for (int i = 0; i < kTcSpin; ++i) {
     if (tc_mbar_try(bar, parity)) return true;
     if (i > 32) {
@@ -130,16 +142,12 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   FixQueue* fixq = reinterpret_cast<FixQueue*>(smem + kTcSmFix);
   float* rowsq = reinterpret_cast<float*>(smem + kTcSmRowSq);
   uint8_t* l4s = reinterpret_cast<uint8_t*>(rowsq + 4 * 128);  // [4][128] level-4 codes of the row's column quarters
-  const uint32_t bar_full = sb + kTcSmBar, bar_empty = bar_full + 8 * kTcStages;
-  const uint32_t bar_tfull = bar_empty + 8 * kTcStages;
+  const uint32_t bar_full = sb + kTcSmBar, bar_tfull = bar_full + 8 * kTcStages;
   const int n_tiles = n_row_tiles * 2 * a.n_kv_heads;
 
   // ---- set-up: barriers, tensor memory, S split into two bf16 terms in the B-operand layout
   if (tid == 0) {
-    for (int s = 0; s < kTcStages; ++s) {
-      tc_mbar_init(bar_full + 8 * s, 1);
-      tc_mbar_init(bar_empty + 8 * s, kTcThreads / 32);   // one commit per warp
-    }
+    for (int s = 0; s < kTcStages; ++s) tc_mbar_init(bar_full + 8 * s, 1);
     for (int i = 0; i < 2; ++i) {
       tc_mbar_init(bar_tfull + 8 * i, kTcThreads / 32);   // one commit per warp
     }
@@ -193,7 +201,8 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     const int tile = blockIdx.x + it * gridDim.x;
     if (tile >= n_tiles) return;
     const int s = it % kTcStages;
-    if (it >= kTcStages && !tc_mbar_wait(bar_empty + 8 * s, ((it / kTcStages) - 1) & 1, abort_flag)) return;
+    // The stage is free: its previous tile (local tile it - 3) was multiplied before this thread passed the
+    // wait for that tile's accumulator, two tiles ago.
     const int kv = hq & 1, rt = hq >> 1;
     const CUtensorMap* map = kv ? &maps.v : &maps.k;
     const uint32_t dst = sb + kTcSmX + s * kTcXBytes, bar = bar_full + 8 * s;
@@ -217,8 +226,7 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     const uint32_t off = ((q >> 2) & 1) * 16384 + (q & 3) * 32;
     tc_mma(tmem_base + acc * 128, tc_smem_desc(sb + kTcSmX + s * kTcXBytes + off),
            tc_smem_desc(sb + kTcSmS + (q >> 3) * kTcSBytes + off), 1u);
-    tc_commit(bar_empty + 8 * s);     // the x stage may be refilled once these MMAs have read it
-    tc_commit(bar_tfull + 8 * acc);   // this issuer's share of the accumulator is complete
+    tc_commit(bar_tfull + 8 * acc);   // this issuer's share of the accumulator is complete (and of the reads of the x stage)
   };
   // both accumulators start at zero
   {
