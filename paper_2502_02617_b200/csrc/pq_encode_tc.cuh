@@ -197,9 +197,11 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     }
   };
   // One thread issues the TMA loads of local tile `it` (tile blockIdx.x + it * gridDim.x = head + n_kv_heads * hq).
+  int tma_issued = 0;  // local tiles whose copies this thread has issued (thread 0 only)
   auto issue_tma = [&](int it, int head, int hq) {
     const int tile = blockIdx.x + it * gridDim.x;
-    if (tile >= n_tiles) return;
+    if (tile >= n_tiles || *abort_flag) return;  // after a wait gave up nothing new is put in flight
+    tma_issued = it + 1;
     const int s = it % kTcStages;
     // The stage is free: its previous tile (local tile it - 3) was multiplied before this thread passed the
     // wait for that tile's accumulator, two tiles ago.
@@ -368,6 +370,13 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     } else if (fix_should_drain(fixq)) {
       fix_rounds(a, fixq, leftbits, xoff, tb, tok, 2 * cq, kv, tid, kTcEpiThreads, 1);
     }
+  }
+  if (*abort_flag && tid == 0) {
+    // gave up somewhere: let the copies that are still in flight land (bounded) before the CTA and its
+    // shared memory go away
+    for (int t = max(0, tma_issued - kTcStages); t < tma_issued; ++t)
+      for (int i = 0; i < (1 << 16) && !tc_mbar_try(bar_full + 8 * (t % kTcStages), (t / kTcStages) & 1); ++i)
+        __nanosleep(64);
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
