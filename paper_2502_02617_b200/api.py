@@ -46,6 +46,7 @@ _SIGNATURES = {
     "pq_decode_attention_static": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p,
                                              c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p,
                                              c_void_p]),
+    "pq_debug_fail_next_wait": (c_int32, [c_int32]),
     "pq_unpack_codes": (c_int32, [c_int32, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p]),
     "pq_dequant_kv": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p,
                                 c_void_p]),
@@ -192,6 +193,12 @@ def pq_decode_attention_static(S, tables, q, cache, cache_lens, n_kv_heads, capa
     _check(lib().pq_decode_attention_static(d, n_q_heads, n_kv_heads, _ptr(S), _ptr(tables), _ptr(q), _dtype_code(q),
                                             _ptr(cache), _ptr(cache_lens), batch, capacity, max_len, float(scale),
                                             _ptr(out), _ptr(status), _stream(stream)), "pq_decode_attention_static")
+
+
+def pq_debug_fail_next_wait(which: int) -> None:
+    """Test support: 1 = the next tensor-core encode launch, 2 = the next head_dim-128 decode-attention
+    launch runs its give-up path (PQ_ERR_TIMEOUT in status word 0); 0 disarms."""
+    _check(lib().pq_debug_fail_next_wait(int(which)), "pq_debug_fail_next_wait")
 
 
 def pq_unpack_codes(d, n_kv_heads, cache, batch, capacity, n_tokens, stream=None):

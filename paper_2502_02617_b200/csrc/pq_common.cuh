@@ -159,6 +159,9 @@ __device__ inline double polar_quant_block_exact(const double* y, const Tables& 
 
 // Host side: remember the CUDA error behind a PQ_ERR_CUDA return (see pq_last_cuda_error).
 void note_cuda_error(cudaError_t e);
+// Test hook (pq_debug_fail_next_wait): returns true once after the hook was armed for `which`
+// (1 = tensor-core encoder, 2 = head_dim-128 decode attention) and disarms it.
+bool take_debug_wait_failure(int which);
 inline int32_t launch_status() {
   const cudaError_t e = cudaGetLastError();
   if (e == cudaSuccess) return PQ_OK;

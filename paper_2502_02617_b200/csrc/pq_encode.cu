@@ -1,4 +1,6 @@
 // KV-cache encoder (Algorithm 1 lines 2 and 4 with fixed codebooks) and the append step.
+#include <math_constants.h>
+
 #include "pq_common.cuh"
 
 namespace pq {
@@ -20,6 +22,7 @@ struct EncodeArgs {
   uint8_t* cache;
   const int32_t* cache_lens;
   int32_t* status;
+  uint32_t debug;  // bit 0: test hook, the first bounded wait of CTA 0 of the tensor-core kernel reports failure
 };
 
 __device__ inline float load_elem(const void* base, int dtype, int64_t idx) {
@@ -245,28 +248,34 @@ __device__ __forceinline__ bool bar_or(int bar_id, int n_threads, bool v) {
 
 // Drain the queue of ambiguous decisions: rounds of (barrier, process, barrier, reset, push what did
 // not fit before).  All `n_threads` threads of named barrier `bar_id` call this together.
-// `leftbits` holds this thread's decisions that found the queue full (15 bits per block, up to 4 blocks
-// starting at block `blk0`).
-__device__ inline void fix_rounds(const EncodeArgs& a, FixQueue* q, unsigned long long leftbits, int64_t xoff, uint8_t* tb,
+// `left` holds this thread's decisions that found the queue full: 15 bits per block, four blocks per
+// word, starting at block `blk0`; it is all zero on return.
+template <class Q, int kWords>
+__device__ inline void fix_rounds(const EncodeArgs& a, Q* q, unsigned long long (&left)[kWords], int64_t xoff, uint8_t* tb,
                                   int tok, int blk0, int kv, int t, int n_threads, int bar_id,
                                   const double* Sd = nullptr) {
-  for (int round = 0; round < 256; ++round) {
+  for (int round = 0; round < 4096; ++round) {
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
     fix_process(q, t, n_threads, a.K, a.V, a.in_dtype, a.S, Sd, *a.tables, a.status);
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
     if (t < 4) q->count[t] = 0;
-    const bool more = bar_or(bar_id, n_threads, leftbits != 0ull);
-    if (!more) break;
-    if (leftbits != 0ull && tb != nullptr) {
+    bool mine = false;
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t bits = (uint32_t)(leftbits >> (15 * i)) & 0x7FFFu;
-        if (bits) {
-          uint32_t left;
-          fix_push(q, bits, xoff, tb, tok, blk0 + i, kv, &left);
-          leftbits = (leftbits & ~(0x7FFFull << (15 * i))) | ((unsigned long long)left << (15 * i));
+    for (int w = 0; w < kWords; ++w) mine = mine || left[w] != 0ull;
+    const bool more = bar_or(bar_id, n_threads, mine);
+    if (!more) break;
+    if (mine && tb != nullptr) {
+#pragma unroll
+      for (int w = 0; w < kWords; ++w)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t bits = (uint32_t)(left[w] >> (15 * i)) & 0x7FFFu;
+          if (bits) {
+            uint32_t rest;
+            fix_push(q, bits, xoff, tb, tok, blk0 + 4 * w + i, kv, &rest);
+            left[w] = (left[w] & ~(0x7FFFull << (15 * i))) | ((unsigned long long)rest << (15 * i));
+          }
         }
-      }
     }
   }
 }
@@ -328,13 +337,13 @@ __global__ void __launch_bounds__(kFfmaThreads) encode_ffma_kernel(EncodeArgs a)
   int tok = 0;
   quantise_and_store(a, *fq, uniform, y, row_norm, row0 + r, head, kv, half, row0 + r < a.total_tokens, fixq, left, &xoff,
                      &tb, &tok);
-  unsigned long long leftbits = 0ull;
+  unsigned long long leftbits[1] = {0ull};
   if (tb != nullptr) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       uint32_t rest = 0;
       if (left[i]) fix_push(fixq, left[i], xoff, tb, tok, 4 * half + i, kv, &rest);
-      leftbits |= (unsigned long long)rest << (15 * i);
+      leftbits[0] |= (unsigned long long)rest << (15 * i);
     }
   }
   fix_rounds(a, fixq, leftbits, xoff, tb, tok, 4 * half, kv, tid, kFfmaThreads, 1);
@@ -501,6 +510,7 @@ int32_t pq_encode_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, c
   a.n_kv_heads = n_kv_heads; a.head_dim = head_dim; a.capacity = capacity;
   a.S = S_dev; a.tables = reinterpret_cast<const pq::Tables*>(tables_dev);
   a.cache = reinterpret_cast<uint8_t*>(cache_dev); a.cache_lens = cache_lens_dev; a.status = status_dev;
+  a.debug = 0u;
   return pq::launch_encode(a, cache_lens_dev, reinterpret_cast<cudaStream_t>(stream));
 }
 
@@ -519,6 +529,7 @@ int32_t pq_append_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, c
   a.n_kv_heads = n_kv_heads; a.head_dim = head_dim; a.capacity = capacity;
   a.S = S_dev; a.tables = reinterpret_cast<const pq::Tables*>(tables_dev);
   a.cache = reinterpret_cast<uint8_t*>(cache_dev); a.cache_lens = cache_lens_dev; a.status = status_dev;
+  a.debug = 0u;
   return pq::launch_encode(a, cache_lens_dev, reinterpret_cast<cudaStream_t>(stream));
 }
 

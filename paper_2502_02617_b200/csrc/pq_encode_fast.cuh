@@ -202,22 +202,27 @@ __device__ __forceinline__ void polar_quant_block_fast(const float* y, const Row
 // the original inputs (x in its storage type, S in float32: both exact in float64), decide again
 // and patch the code bits in the cache with 32-bit atomics.  The queue is drained in rounds, so a
 // tile with more ambiguous angles than the queue holds only takes more rounds.
-constexpr int kFixCap = 1024;
-// The queue is kept sorted by level (one region per level), so that the four 8-lane groups of a warp,
-// which take consecutive entries, almost always run the same code path.
-__host__ __device__ constexpr int fix_off(int level) { return level == 1 ? 0 : level == 2 ? 512 : level == 3 ? 768 : 896; }
-__host__ __device__ constexpr int fix_cap(int level) { return level == 1 ? 512 : level == 2 ? 256 : 128; }
-
-struct FixQueue {
-  int count[4];            // entries pushed per level (may exceed the capacity: the excess was not stored)
-  int64_t xoff[kFixCap];   // element offset of the source vector
-  uint8_t* tok[kFixCap];   // token-block base of the destination
-  uint32_t meta[kFixCap];  // token-in-block | blk << 6 | level << 9 | j << 12 | (1 = value, 0 = key) << 15
+// The queue is kept sorted by level (one region per level: 1/2, 1/4, 1/8 and 1/8 of the capacity), so that
+// the four 8-lane groups of a warp, which take consecutive entries, almost always run the same code path.
+template <int kCap>
+struct FixQueueT {
+  static constexpr int kCapacity = kCap;
+  __host__ __device__ static constexpr int off(int level) {
+    return level == 1 ? 0 : level == 2 ? kCap / 2 : level == 3 ? 3 * kCap / 4 : 7 * kCap / 8;
+  }
+  __host__ __device__ static constexpr int cap(int level) { return level == 1 ? kCap / 2 : level == 2 ? kCap / 4 : kCap / 8; }
+  int count[4];         // entries pushed per level (may exceed the capacity: the excess was not stored)
+  int64_t xoff[kCap];   // element offset of the source vector
+  uint8_t* tok[kCap];   // token-block base of the destination
+  uint32_t meta[kCap];  // token-in-block | blk << 6 | level << 9 | j << 12 | (1 = value, 0 = key) << 15
 };
+using FixQueue = FixQueueT<1024>;
 
 // True if some region is 3/4 full (or has overflowed).
-__device__ __forceinline__ bool fix_should_drain(const FixQueue* q) {
-  return q->count[0] > 384 || q->count[1] > 192 || q->count[2] > 96 || q->count[3] > 96;
+template <class Q>
+__device__ __forceinline__ bool fix_should_drain(const Q* q) {
+  return q->count[0] > 3 * Q::cap(1) / 4 || q->count[1] > 3 * Q::cap(2) / 4 || q->count[2] > 3 * Q::cap(3) / 4 ||
+         q->count[3] > 3 * Q::cap(4) / 4;
 }
 
 // Replace `width` bits at bit offset `bit` of the byte at `addr`.
@@ -228,7 +233,8 @@ __device__ __forceinline__ void patch_bits(uint8_t* addr, int bit, uint32_t mask
   atomicOr(word, code << sh);
 }
 
-__device__ __forceinline__ void fix_push(FixQueue* q, uint32_t amb, int64_t xoff, uint8_t* tokblock, int tok, int blk,
+template <class Q>
+__device__ __forceinline__ void fix_push(Q* q, uint32_t amb, int64_t xoff, uint8_t* tokblock, int tok, int blk,
                                          int kv, uint32_t* left) {
   uint32_t rest = 0;
   while (amb) {
@@ -240,11 +246,11 @@ __device__ __forceinline__ void fix_push(FixQueue* q, uint32_t amb, int64_t xoff
     else if (bit < 14) { level = 3; j = bit - 12; }
     else { level = 4; j = 0; }
     const int idx = atomicAdd(&q->count[level - 1], 1);
-    if (idx >= fix_cap(level)) {  // this level's region is full: keep the decision for the next round
+    if (idx >= Q::cap(level)) {  // this level's region is full: keep the decision for the next round
       rest |= 1u << bit;
       continue;
     }
-    const int e = fix_off(level) + idx;
+    const int e = Q::off(level) + idx;
     q->xoff[e] = xoff;
     q->tok[e] = tokblock;
     q->meta[e] = (uint32_t)tok | ((uint32_t)blk << 6) | ((uint32_t)level << 9) | ((uint32_t)j << 12) | ((uint32_t)kv << 15);
@@ -336,16 +342,17 @@ __device__ __forceinline__ uint32_t exact_code(const double* y, int level, const
 
 // Process everything queued, in level order: called by `n_threads` threads (a multiple of 32) with linear index `t`.
 // `Sd` (may be null) is S staged in shared memory for exact_coords_sm.
-__device__ inline void fix_process(const FixQueue* q, int t, int n_threads, const void* kbase, const void* vbase,
+template <class Q>
+__device__ inline void fix_process(const Q* q, int t, int n_threads, const void* kbase, const void* vbase,
                                    int in_dtype, const float* S, const double* Sd, const Tables& tb, int32_t* status) {
   constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock;
   const int sub = t & 7, n_groups = n_threads >> 3;
   const unsigned gmask = 0xFFu << (t & 24);
-  const int n1 = min(q->count[0], fix_cap(1)), n2 = n1 + min(q->count[1], fix_cap(2));
-  const int n3 = n2 + min(q->count[2], fix_cap(3)), n = n3 + min(q->count[3], fix_cap(4));
+  const int n1 = min(q->count[0], Q::cap(1)), n2 = n1 + min(q->count[1], Q::cap(2));
+  const int n3 = n2 + min(q->count[2], Q::cap(3)), n = n3 + min(q->count[3], Q::cap(4));
   int fixed = 0;
   auto entry_of = [&](int i) {
-    return i < n1 ? i : i < n2 ? fix_off(2) + (i - n1) : i < n3 ? fix_off(3) + (i - n2) : fix_off(4) + (i - n3);
+    return i < n1 ? i : i < n2 ? Q::off(2) + (i - n1) : i < n3 ? Q::off(3) + (i - n2) : Q::off(4) + (i - n3);
   };
   // The source vector of the group's next entry is fetched while the current one is decided.
   auto fetch = [&](int i, uint4* raw) {

@@ -1,43 +1,51 @@
 // Tensor-core encoder for head_dim 128, bf16 inputs (included by pq_encode.cu).
 //
-// Persistent CTAs (one per SM, 16 warps) loop over tiles of 128 rows x one (K|V, head).  Per tile
-//   * TMA loads of the x tile (two 64-column boxes, 128-byte swizzle) into a 3-deep ring, issued by
-//     one thread two tiles ahead;
-//   * y = x . S on the 5th-generation tensor cores: S is split once per CTA into two bf16 terms
-//     (S = S_hi + S_lo + O(2^-17)) kept in shared memory as the K-major B operand; 2 terms x 8
-//     k-steps of tcgen05.mma (M = 128 rows, N = 128, K = 16) accumulate in float32 in tensor memory;
-//     two accumulators, and the MMAs of tile i+1 are issued when the epilogue of tile i starts, so
-//     they run under it.  Lane 0 of every warp issues one of the 16 MMAs, so that no warp is held up
-//     by the batch (a warp that is late delays all 16 at the next barrier); since their order is then
-//     free, every MMA accumulates and the epilogue clears the accumulator after reading it;
-//   * epilogue on all 16 warps.  Tensor-memory lane = row, so a thread owns 32 consecutive rotated
-//     coordinates (2 blocks) of one row: tcgen05.ld, sign-test quantiser with certified margins,
-//     packed stores, queued float64 re-decision of the ambiguous angles.
+// Persistent CTAs (one per SM, 16 warps) loop over tiles of 128 rows x one (K|V, head).  The 16 warps form
+// four groups ("slots") of four warps; a slot owns one of four 128-column accumulators in tensor memory
+// and takes every fourth tile of the CTA.  Per tile
+//   * TMA loads of the x tile (two 64-column boxes, 128-byte swizzle) into a 3-deep ring; the copy of
+//     tile i+3 is issued as soon as the MMAs of tile i, which read the same ring stage, have completed;
+//   * y = x . S on the 5th-generation tensor cores: S is split once per CTA into bf16 terms
+//     (S = S_hi + S_lo + O(2^-17)) kept in shared memory as the K-major B operand; terms x 8 k-steps of
+//     tcgen05.mma (M = 128 rows, N = 128, K = 16) accumulate in float32 in the slot's accumulator.  One
+//     thread of the slot issues them when the slot's previous tile has been read out; the other three
+//     slots are in their epilogues meanwhile, so the tensor work hides under ALU work;
+//   * epilogue on the slot's four warps.  Tensor-memory lane = row and a warp may read its own quarter of
+//     the lanes, so a thread owns one whole row (8 blocks): one pass over the accumulator for the row norm
+//     (the certified margins need it), a second pass of tcgen05.ld of 32 coordinates at a time through the
+//     sign-test quantiser, packed stores of whole plane entries of the token, queued float64 re-decision of
+//     the ambiguous angles (one queue per slot, drained by the slot; the rest after the last tile by the CTA).
+// Per-row work (norm, margins, cache destination, stores) is paid once per 8 blocks, and the only
+// synchronisation in the loop is one named barrier of the slot's 128 threads per tile.
 // There are no dedicated producer / MMA warps: the register file is split over four schedulers, and
-// a 17th warp would cap every thread at 96 registers (the quantiser then spills).  The issuing
-// threads do not block in practice: what they wait for was completed a tile earlier.
+// a 17th warp would cap every thread at 96 registers (the quantiser then spills).
 // Every mbarrier wait is bounded; a wait that gives up raises the CTA's abort flag, the remaining
-// tiles are skipped, tensor memory is released and PQ_ERR_TIMEOUT is recorded.
+// tiles are skipped (the loops keep their shape, so the named barriers stay consistent), copies in
+// flight are drained, tensor memory is released and PQ_ERR_TIMEOUT is recorded.
 #pragma once
 #include <cuda.h>
 
 namespace pq {
 
 constexpr int kTcThreads = 512;
-constexpr int kTcEpiThreads = 512;
-constexpr int kTcStages = 3;
+constexpr int kTcSlots = 4;                // accumulators in tensor memory = groups of four warps
+constexpr int kTcSlotThreads = kTcThreads / kTcSlots;
+constexpr int kTcStages = 3;               // x tiles in flight
+constexpr int kTcTerms = 2;                // bf16 terms of S
 constexpr int kTcXBytes = 128 * 128 * 2;   // one x tile: 128 rows x 128 bf16
 constexpr int kTcSBytes = 128 * 128 * 2;   // one bf16 term of S (B operand)
-constexpr int kTcSmS = 0;                  // S_hi, S_lo
-constexpr int kTcSmX = kTcSmS + 2 * kTcSBytes;
-constexpr int kTcSmRowSq = kTcSmX + kTcStages * kTcXBytes;   // [4][128] float, then [4][128] bytes of level-4 nibbles
-constexpr int kTcSmFq = kTcSmRowSq + 2048 + 512;             // FastQuant (40 B)
-constexpr int kTcSmBar = kTcSmFq + 64;                       // full[3], tfull[2]
-constexpr int kTcSmMisc = kTcSmBar + 128;                    // tmem base, abort flag
-constexpr int kTcSmFix = kTcSmMisc + 64;                     // FixQueue
-constexpr int kTcSmTotal = kTcSmFix + (int)sizeof(FixQueue) + 1024;  // + slack for 1024-byte alignment
+using TcFixQueue = FixQueueT<256>;
+constexpr int kTcSmS = 0;
+constexpr int kTcSmX = kTcSmS + kTcTerms * kTcSBytes;
+constexpr int kTcSmOperandEnd = kTcSmX + kTcStages * kTcXBytes;
+constexpr int kTcSmFq = kTcSmOperandEnd;                     // FastQuant (40 B)
+constexpr int kTcSmBar = kTcSmFq + 64;                       // x_full[3], acc_full[4]
+constexpr int kTcSmMisc = kTcSmBar + 64;                     // tmem base, abort flag, copies issued per stage [3], debug
+constexpr int kTcSmFix = kTcSmMisc + 64;                     // one TcFixQueue per slot
+constexpr int kTcSmTotal = kTcSmFix + kTcSlots * (int)sizeof(TcFixQueue) + 1024;  // + slack for 1024-byte alignment
 constexpr int kTcSpin = 1 << 22;
-static_assert(kFixSdBytes <= kTcSmRowSq, "the float64 copy of S must fit in the operand buffers");
+static_assert(kFixSdBytes <= kTcSmOperandEnd, "the float64 copy of S must fit in the operand buffers");
+static_assert(sizeof(TcFixQueue) % 16 == 0, "queues are laid out back to back");
 
 __device__ __forceinline__ uint32_t tc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void tc_mbar_init(uint32_t bar, uint32_t count) {
@@ -108,27 +116,42 @@ __device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, float* v) {
-  uint32_t r[16];
+// 32 consecutive columns of this thread's tensor-memory lane (issue only; follow with tc_wait_ld).
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
+  uint32_t r[32];
   asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
       : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
       : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-  for (int i = 0; i < 16; ++i) v[i] = __uint_as_float(r[i]);
-}
-
-__device__ __forceinline__ void tc_st16_zero(uint32_t taddr) {
-  const uint32_t z = 0u;
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1,%1};" ::"r"(taddr), "r"(z)
-      : "memory");
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 struct TcMaps {
   CUtensorMap k, v;
 };
+
+// Non-finite elements among the 128 bf16 inputs of one vector (read again from global memory: only
+// rows whose rotated norm is not finite get here).
+__device__ inline int count_nonfinite_bf16(const void* base, int64_t xoff) {
+  const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(base) + xoff);
+  int bad = 0;
+  for (int i = 0; i < 16; ++i) {
+    const uint4 w = __ldg(p + i);
+    const uint32_t v[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      bad += ((v[k] & 0x7F80u) == 0x7F80u);          // exponent all ones: Inf or NaN
+      bad += ((v[k] & 0x7F800000u) == 0x7F800000u);
+    }
+  }
+  return bad;
+}
 
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_tiles) {
@@ -136,48 +159,56 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sb = tc_smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int quarter = warp & 3;            // tensor-memory lanes this warp may read: rows 32 * quarter ..
+  const int slot = warp >> 2;              // accumulator and tile sequence of this group of four warps
+  const int st = quarter * 32 + lane;      // thread index inside the slot = row of the tile
+  const bool leader = st == 0;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kTcSmMisc + 4);
+  volatile int* copies_issued = reinterpret_cast<volatile int*>(smem + kTcSmMisc + 8);  // [kTcStages]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kTcSmMisc);
   FastQuant* fq = reinterpret_cast<FastQuant*>(smem + kTcSmFq);
-  FixQueue* fixq = reinterpret_cast<FixQueue*>(smem + kTcSmFix);
-  float* rowsq = reinterpret_cast<float*>(smem + kTcSmRowSq);
-  uint8_t* l4s = reinterpret_cast<uint8_t*>(rowsq + 4 * 128);  // [4][128] level-4 codes of the row's column quarters
-  const uint32_t bar_full = sb + kTcSmBar, bar_tfull = bar_full + 8 * kTcStages;
+  TcFixQueue* queues = reinterpret_cast<TcFixQueue*>(smem + kTcSmFix);
+  TcFixQueue* fixq = queues + slot;
+  const uint32_t bar_xfull = sb + kTcSmBar, bar_acc = bar_xfull + 8 * kTcStages;
   const int n_tiles = n_row_tiles * 2 * a.n_kv_heads;
 
-  // ---- set-up: barriers, tensor memory, S split into two bf16 terms in the B-operand layout
+  // ---- set-up: barriers, tensor memory, S split into bf16 terms in the B-operand layout
   if (tid == 0) {
-    for (int s = 0; s < kTcStages; ++s) tc_mbar_init(bar_full + 8 * s, 1);
-    for (int i = 0; i < 2; ++i) {
-      tc_mbar_init(bar_tfull + 8 * i, kTcThreads / 32);   // one commit per warp
+    for (int s = 0; s < kTcStages; ++s) {
+      tc_mbar_init(bar_xfull + 8 * s, 1);
+      copies_issued[s] = 0;
     }
+    for (int i = 0; i < kTcSlots; ++i) tc_mbar_init(bar_acc + 8 * i, 1);   // one commit by the slot's issuing thread
     *abort_flag = 0;
-    fixq->count[0] = fixq->count[1] = fixq->count[2] = fixq->count[3] = 0;
     load_fast_quant(a.tables, fq);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (st < 4) fixq->count[st] = 0;
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(sb + kTcSmMisc) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(sb + kTcSmMisc) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // B operand: B[n][k] = S[k][n]; two halves of 64 k; row n = 128 bytes, 16-byte chunk c stored at c ^ (n & 7).
   // A task is (row n, chunk of 8 consecutive k): 8 coalesced loads (lanes = consecutive n), one 16-byte store per term.
   for (int task = tid; task < 128 * 16; task += kTcThreads) {
     const int n = task & 127, oct = task >> 7;  // k = 8 * oct .. 8 * oct + 7
-    uint32_t hi[4], lo[4];
+    uint32_t term[kTcTerms][4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      const float v0 = a.S[(8 * oct + 2 * i) * 128 + n], v1 = a.S[(8 * oct + 2 * i + 1) * 128 + n];
-      const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
-      const __nv_bfloat16 l0 = __float2bfloat16_rn(v0 - __bfloat162float(h0));
-      const __nv_bfloat16 l1 = __float2bfloat16_rn(v1 - __bfloat162float(h1));
-      hi[i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-      lo[i] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+      float v0 = a.S[(8 * oct + 2 * i) * 128 + n], v1 = a.S[(8 * oct + 2 * i + 1) * 128 + n];
+#pragma unroll
+      for (int t = 0; t < kTcTerms; ++t) {
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
+        term[t][i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+        v0 -= __bfloat162float(h0);  // exact: the residual of a bf16 rounding fits float32
+        v1 -= __bfloat162float(h1);
+      }
     }
     const int half = oct >> 3, c = oct & 7;
     const int off = half * 16384 + n * 128 + ((c ^ (n & 7)) << 4);
-    *reinterpret_cast<uint4*>(smem + kTcSmS + off) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-    *reinterpret_cast<uint4*>(smem + kTcSmS + kTcSBytes + off) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+#pragma unroll
+    for (int t = 0; t < kTcTerms; ++t)
+      *reinterpret_cast<uint4*>(smem + kTcSmS + t * kTcSBytes + off) = make_uint4(term[t][0], term[t][1], term[t][2], term[t][3]);
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA unit
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -185,29 +216,19 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
-  // Tile t = (row tile, K|V, head) with head fastest: t = head + n_kv_heads * hq, hq = 2 * row tile + kv.  A CTA's
-  // tiles are gridDim.x apart; their coordinates are advanced without divisions.
-  const int step_h = (int)gridDim.x % a.n_kv_heads, step_q = (int)gridDim.x / a.n_kv_heads;
-  auto advance = [&](int& head, int& hq) {
-    head += step_h;
-    hq += step_q;
-    if (head >= a.n_kv_heads) {
-      head -= a.n_kv_heads;
-      ++hq;
-    }
-  };
-  // One thread issues the TMA loads of local tile `it` (tile blockIdx.x + it * gridDim.x = head + n_kv_heads * hq).
-  int tma_issued = 0;  // local tiles whose copies this thread has issued (thread 0 only)
-  auto issue_tma = [&](int it, int head, int hq) {
+  // Local tile `it` of this CTA is tile blockIdx.x + it * gridDim.x = head + n_kv_heads * (2 * row tile + kv); it
+  // uses ring stage it % kTcStages and belongs to slot it % kTcSlots.
+  // One thread issues the TMA loads of local tile `it`.  The caller knows that the stage is free: the MMAs of
+  // local tile it - kTcStages, which read it, have completed.
+  auto issue_tma = [&](int it) {
     const int tile = blockIdx.x + it * gridDim.x;
     if (tile >= n_tiles || *abort_flag) return;  // after a wait gave up nothing new is put in flight
-    tma_issued = it + 1;
     const int s = it % kTcStages;
-    // The stage is free: its previous tile (local tile it - 3) was multiplied before this thread passed the
-    // wait for that tile's accumulator, two tiles ago.
+    const int head = tile % a.n_kv_heads, hq = tile / a.n_kv_heads;
     const int kv = hq & 1, rt = hq >> 1;
     const CUtensorMap* map = kv ? &maps.v : &maps.k;
-    const uint32_t dst = sb + kTcSmX + s * kTcXBytes, bar = bar_full + 8 * s;
+    const uint32_t dst = sb + kTcSmX + s * kTcXBytes, bar = bar_xfull + 8 * s;
+    copies_issued[s] = copies_issued[s] + 1;
     tc_mbar_expect_tx(bar, kTcXBytes);
 #pragma unroll
     for (int h = 0; h < 2; ++h)
@@ -216,173 +237,174 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
           ::"r"(dst + h * 16384), "l"(map), "r"(h * 64), "r"(head), "r"(rt * 128), "r"(bar)
           : "memory");
   };
-  // Lane 0 of every warp issues one of the 16 MMAs of local tile `it` into accumulator it & 1: issuer q takes
-  // term q >> 3 of S, k-half (q >> 2) & 1 and k-step q & 3.  All MMAs accumulate (the accumulator is zero).
-  // The accumulator is free: its previous tile was read and cleared by every warp before the CTA-wide barrier
-  // that ended that tile, which this thread has passed.
-  auto issue_mma = [&](int it, int q) {
-    if (blockIdx.x + it * (int)gridDim.x >= n_tiles) return;
-    const int s = it % kTcStages, acc = it & 1;
-    if (!tc_mbar_wait(bar_full + 8 * s, (it / kTcStages) & 1, abort_flag)) return;
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const uint32_t off = ((q >> 2) & 1) * 16384 + (q & 3) * 32;
-    tc_mma(tmem_base + acc * 128, tc_smem_desc(sb + kTcSmX + s * kTcXBytes + off),
-           tc_smem_desc(sb + kTcSmS + (q >> 3) * kTcSBytes + off), 1u);
-    tc_commit(bar_tfull + 8 * acc);   // this issuer's share of the accumulator is complete (and of the reads of the x stage)
-  };
-  // both accumulators start at zero
-  {
-    const uint32_t z = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (warp >> 2) * 32;
-#pragma unroll
-    for (int i = 0; i < 2; ++i)
-#pragma unroll
-      for (int j = 0; j < 2; ++j) tc_st16_zero(z + i * 128 + 16 * j);
-    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  }
-  int head = (int)blockIdx.x % a.n_kv_heads, hq = (int)blockIdx.x / a.n_kv_heads;  // this tile
-  int head2 = head, hq2 = hq;                                                      // the tile two ahead
-  if (tid == 0) issue_tma(0, head2, hq2);
-  advance(head2, hq2);
-  if (tid == 0) issue_tma(1, head2, hq2);
-  advance(head2, hq2);
-  if (lane == 0) issue_mma(0, warp);
-  __syncwarp();
+  if (tid == 0)
+    for (int it = 0; it < kTcStages; ++it) issue_tma(it);
 
-  // ---- tile loop: all 16 warps are epilogue warps
+  // ---- tile loop of this slot
   constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock, orad = o4 + 2 * kTokenBlock;
-  const int quarter = warp & 3;                  // tensor-memory lanes this warp may read
-  const int cq = warp >> 2;                      // columns [32*cq, 32*cq + 32): blocks 2cq, 2cq+1
-  const int r = quarter * 32 + lane;             // row of the tile
   const bool uniform = (a.tables->flags & kFlagUniformL1) != 0u;
   const bool sym = fq->sym != 0u;  // uniform over the grid
   const Layout L = make_layout(128, a.capacity);
+  const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + slot * 128;
+  const int slot_bar = 1 + slot;
   int rd_seq = 0, rd_first = 0, rd_count = 0, rd_start = -1;   // destination of the last row looked up
-  int it = 0;
-  for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it, advance(head, hq)) {
-    const int acc = it & 1;
+  for (int it = slot; blockIdx.x + it * (int)gridDim.x < n_tiles; it += kTcSlots) {
+    const int tile = blockIdx.x + it * gridDim.x;
+    const int head = tile % a.n_kv_heads, hq = tile / a.n_kv_heads;
     const int kv = hq & 1, rt = hq >> 1;
-    // A wait that gives up must not leave the loop: the other warps may be past it and would wait
-    // for this one at the named barriers.  The tile is skipped instead (warp-uniform).
-    const bool ready = __all_sync(0xffffffffu, tc_mbar_wait(bar_tfull + 8 * acc, (it >> 1) & 1, abort_flag));
-    // keep the pipeline fed: loads two tiles ahead, the next tile's MMAs under this tile's epilogue
-    if (tid == 0) issue_tma(it + 2, head2, hq2);
-    advance(head2, hq2);
-    if (lane == 0) issue_mma(it + 1, warp);
-    __syncwarp();
-    const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * 128 + cq * 32;
-    // pass 1: the thread's 32 coordinates and their share of the row's squared norm (the four column
-    // quarters of a row are exchanged through shared memory)
-    float sq = 0.f;
-    float y[32];
-    if (ready) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      tc_ld16(taddr, y);
-      tc_ld16(taddr + 16, y + 16);
-      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+    const int s = it % kTcStages;
+    if (leader) {
+      // The accumulator is free: the slot's four warps read the previous tile out of it before the barrier
+      // that ended that tile.  All MMAs of the tile come from this thread, in order: the first overwrites.
+      // The copy of this tile is issued by another slot's thread (when the tile three back has been
+      // multiplied).  A parity wait taken before that would be satisfied by the stage's previous phase, so
+      // first wait (bounded) until the copy has been issued: the previous phase is complete by then.
+      bool ok = false;
+      for (int i = 0; i < kTcSpin && !ok; ++i) {
+        ok = copies_issued[s] > it / kTcStages;
+        if (!ok && i > 32) {
+          __nanosleep(64);
+          if (*abort_flag) break;
+        }
+      }
+      if (!ok) *abort_flag = 1;
+      ok = ok && tc_mbar_wait(bar_xfull + 8 * s, (it / kTcStages) & 1, abort_flag);
+      if (ok && (a.debug & 1u) && blockIdx.x == 0 && it == 0) {  // test hook: report this wait as failed
+        *abort_flag = 1;
+        ok = false;
+      }
+      if (ok) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll
-      for (int c = 0; c < 32; ++c) sq = fmaf(y[c], y[c], sq);
-    } else {
-#pragma unroll
-      for (int c = 0; c < 32; ++c) y[c] = 0.f;
+        for (int q = 0; q < 8 * kTcTerms; ++q) {
+          const uint32_t off = ((q >> 2) & 1) * 16384 + (q & 3) * 32;
+          tc_mma(tmem_base + slot * 128, tc_smem_desc(sb + kTcSmX + s * kTcXBytes + off),
+                 tc_smem_desc(sb + kTcSmS + (q >> 3) * kTcSBytes + off), q ? 1u : 0u);
+        }
+        tc_commit(bar_acc + 8 * slot);  // the accumulator is complete and the x stage has been read
+      }
     }
-    rowsq[cq * 128 + r] = sq;
-    // only the four warps that share these 32 rows exchange their parts of the norm
-    asm volatile("bar.sync %0, 128;" ::"r"(2 + quarter) : "memory");
-    const RowMargins rm = make_row_margins(
-        kRotErr * 1.0001f * sqrtf((rowsq[r] + rowsq[128 + r]) + (rowsq[256 + r] + rowsq[384 + r])), *fq);
-    const int row = rt * 128 + r;
+    __syncwarp();
+    // A wait that gives up must not leave the loop: the other warps of the slot would wait for this one at the
+    // slot's barrier.  The tile is skipped instead (warp-uniform).
+    const bool ready = __all_sync(0xffffffffu, tc_mbar_wait(bar_acc + 8 * slot, (it / kTcSlots) & 1, abort_flag));
+    if (leader && ready) issue_tma(it + kTcStages);  // the stage of this tile is free again
+    const int row = rt * 128 + st;
+    const int64_t xoff = (int64_t)row * a.token_stride + (int64_t)head * a.head_stride;
     uint8_t* tb = nullptr;
     int tok = 0;
-    if (ready && row < a.total_tokens) {
-      int seq, pos;
-      if (row >= rd_first && row < rd_first + rd_count) {  // same sequence as this thread's previous row
-        seq = rd_seq;
-        pos = rd_start < 0 ? -1 : rd_start + (row - rd_first);
-      } else {
-        row_destination(a, row, &seq, &pos);
-        rd_seq = seq;
-        rd_first = a.cu_seqlens ? a.cu_seqlens[seq] : row;
-        rd_count = a.cu_seqlens ? a.cu_seqlens[seq + 1] - rd_first : 1;
-        rd_start = pos < 0 ? -1 : pos - (row - rd_first);
-      }
-      if (pos >= 0) {
-        tb = a.cache + block_offset(L, a.n_kv_heads, seq, head, kv, pos);
-        tok = pos % kTokenBlock;
-      }
-    }
-    const int64_t xoff = (int64_t)row * a.token_stride + (int64_t)head * a.head_stride;
-    // pass 2: one block at a time
-    uint32_t l2acc = 0, l3acc = 0, l4acc = 0, racc = 0, sat = 0;
-    unsigned long long leftbits = 0ull;
+    unsigned long long left[2] = {0ull, 0ull};
     if (ready) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      float y[32];
+      // pass 1: squared norm of the row (four partial sums)
+      float sq[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        tc_ld32(taddr + 32 * c, y);
 #pragma unroll
-      for (int i = 0; i < 2; ++i) {
-        FastBlock fb;
-        if (sym) polar_quant_block_fast<true>(y + 16 * i, rm, *fq, &fb);
-        else polar_quant_block_fast<false>(y + 16 * i, rm, *fq, &fb);
-        if (!uniform) fb.amb |= 0xFFu;  // other level-1 codebooks: decide every level-1 angle exactly
-        if (tb != nullptr) {
-          *reinterpret_cast<uint32_t*>(tb + tok * 32 + cq * 8 + 4 * i) = fb.l1;
-          l2acc |= fb.l2 << (8 * i);
-          l3acc |= fb.l3 << (4 * i);
-          l4acc |= fb.l4 << (2 * i);
+        for (int i = 0; i < 32; ++i) sq[i & 3] = fmaf(y[i], y[i], sq[i & 3]);
+      }
+      const float sqsum = (sq[0] + sq[1]) + (sq[2] + sq[3]);
+      bool bad_row = false;
+      if (!(sqsum < CUDART_INF_F) && row < a.total_tokens) {  // NaN or overflow: look at the inputs
+        const int bad = count_nonfinite_bf16(kv ? a.V : a.K, xoff);
+        if (bad) {
+          atomicAdd(a.status + 1, bad);
+          set_status(a.status, PQ_ERR_NONFINITE);
+          bad_row = true;
+        }
+      }
+      const RowMargins rm = make_row_margins(kRotErr * 1.0001f * sqrtf(sqsum), *fq);
+      if (row < a.total_tokens) {
+        int seq, pos;
+        if (row >= rd_first && row < rd_first + rd_count) {  // same sequence as this thread's previous row
+          seq = rd_seq;
+          pos = rd_start < 0 ? -1 : rd_start + (row - rd_first);
+        } else {
+          row_destination(a, row, &seq, &pos);
+          rd_seq = seq;
+          rd_first = a.cu_seqlens ? a.cu_seqlens[seq] : row;
+          rd_count = a.cu_seqlens ? a.cu_seqlens[seq + 1] - rd_first : 1;
+          rd_start = pos < 0 ? -1 : pos - (row - rd_first);
+        }
+        if (pos >= 0) {
+          tb = a.cache + block_offset(L, a.n_kv_heads, seq, head, kv, pos);
+          tok = pos % kTokenBlock;
+        }
+      }
+      // pass 2: 32 coordinates (two blocks) at a time
+      uint32_t l2lo = 0, l2hi = 0, l3acc = 0, l4acc = 0, sat = 0;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        tc_ld32(taddr + 32 * c, y);
+        uint32_t l1w[2], racc = 0, l2c = 0;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+          FastBlock fb;
+          if (sym) polar_quant_block_fast<true>(y + 16 * i, rm, *fq, &fb);
+          else polar_quant_block_fast<false>(y + 16 * i, rm, *fq, &fb);
+          if (!uniform) fb.amb |= 0xFFu;  // other level-1 codebooks: decide every level-1 angle exactly
+          l1w[i] = fb.l1;
+          l2c |= fb.l2 << (8 * i);
+          l3acc |= fb.l3 << (8 * c + 4 * i);
+          l4acc |= fb.l4 << (4 * c + 2 * i);
           float rv = fb.radius;
           if (rv > 65504.f) { rv = 65504.f; ++sat; }
           racc |= (uint32_t)__half_as_ushort(__float2half_rn(rv)) << (16 * i);
-          if (fb.amb) {
-            uint32_t left;
-            fix_push(fixq, fb.amb, xoff, tb, tok, 2 * cq + i, kv, &left);
-            leftbits |= (unsigned long long)left << (15 * i);  // queue full: pushed again by fix_rounds
+          if (tb != nullptr && fb.amb && !bad_row) {
+            uint32_t rest;
+            fix_push(fixq, fb.amb, xoff, tb, tok, 2 * c + i, kv, &rest);
+            left[c >> 1] |= (unsigned long long)rest << (15 * (2 * (c & 1) + i));  // queue full: pushed again by fix_rounds
           }
         }
+        if (c < 2) l2lo |= l2c << (16 * c);
+        else l2hi |= l2c << (16 * (c - 2));
+        if (tb != nullptr) {
+          if (bad_row) l1w[0] = l1w[1] = racc = 0u;
+          *reinterpret_cast<uint2*>(tb + tok * 32 + c * 8) = make_uint2(l1w[0], l1w[1]);
+          *reinterpret_cast<uint32_t*>(tb + orad + tok * 16 + c * 4) = racc;
+        }
       }
-      tc_st16_zero(taddr);  // leave the accumulator cleared for the next tile that uses it
-      tc_st16_zero(taddr + 16);
-      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      if (tb != nullptr) {
+        if (bad_row) l2lo = l2hi = l3acc = l4acc = sat = 0u;  // a row with non-finite inputs is stored as the zero vector
+        *reinterpret_cast<uint2*>(tb + o2 + tok * 8) = make_uint2(l2lo, l2hi);
+        *reinterpret_cast<uint32_t*>(tb + o3 + tok * 4) = l3acc;
+        *reinterpret_cast<uint16_t*>(tb + o4 + tok * 2) = (uint16_t)l4acc;
+        if (sat) atomicAdd(a.status + 2, (int)sat);
+      }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
-    l4s[cq * 128 + r] = (uint8_t)l4acc;
-    if (tb != nullptr) {
-      *reinterpret_cast<uint16_t*>(tb + o2 + tok * 8 + cq * 2) = (uint16_t)l2acc;
-      tb[o3 + tok * 4 + cq] = (uint8_t)l3acc;
-      *reinterpret_cast<uint32_t*>(tb + orad + tok * 16 + cq * 4) = racc;
-      if (sat) atomicAdd(a.status + 2, (int)sat);
-    }
-    asm volatile("bar.sync 1, 512;" ::: "memory");
-    if (tb != nullptr && (cq & 1) == 0)  // level-4 codes of four blocks share a byte: two column quarters
-      tb[o4 + tok * 2 + (cq >> 1)] = (uint8_t)(l4s[cq * 128 + r] | (l4s[(cq + 1) * 128 + r] << 4));
-    // Exact re-decisions are batched over tiles: drain the queue when it is 3/4 full (a push that
-    // did not fit leaves the counter above the capacity) or after the CTA's last tile.
-    const bool last_tile = tile + (int)gridDim.x >= n_tiles;
-    if (last_tile) {
-      // The operand buffers are idle now (every MMA and copy of this CTA has completed): stage S there as
-      // float64 so that the last, largest batch of re-decisions reads it from shared memory.
-      asm volatile("bar.sync 1, 512;" ::: "memory");
-      double* Sd = reinterpret_cast<double*>(smem + kTcSmS);
-      for (int idx = tid; idx < 128 * 128; idx += kTcThreads) {
-        const int k = idx >> 7, n = idx & 127;
-        Sd[((k & 15) * 8 + (k >> 4)) * kFixSdStride + n] = (double)__ldg(a.S + idx);
-      }
-      fix_rounds(a, fixq, leftbits, xoff, tb, tok, 2 * cq, kv, tid, kTcEpiThreads, 1, Sd);
-    } else if (fix_should_drain(fixq)) {
-      fix_rounds(a, fixq, leftbits, xoff, tb, tok, 2 * cq, kv, tid, kTcEpiThreads, 1);
-    }
+    // End of the tile for the slot (the accumulator may be overwritten after this barrier).  The same barrier
+    // decides, for all 128 threads alike, whether the slot drains its queue of exact re-decisions now: when a
+    // region is 3/4 full or a push did not fit.
+    const bool drain = bar_or(slot_bar, kTcSlotThreads, (left[0] | left[1]) != 0ull || fix_should_drain(fixq));
+    if (drain) fix_rounds(a, fixq, left, xoff, tb, tok, 0, kv, st, kTcSlotThreads, slot_bar);
   }
-  if (*abort_flag && tid == 0) {
-    // gave up somewhere: let the copies that are still in flight land (bounded) before the CTA and its
-    // shared memory go away
-    for (int t = max(0, tma_issued - kTcStages); t < tma_issued; ++t)
-      for (int i = 0; i < (1 << 16) && !tc_mbar_try(bar_full + 8 * (t % kTcStages), (t / kTcStages) & 1); ++i)
-        __nanosleep(64);
-  }
+  // ---- after the last tile: every MMA and copy of this CTA has completed (each was waited for by its slot), so
+  // the operand buffers are idle: stage S there as float64 and let all 16 warps take the queued re-decisions.
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (*abort_flag) {
+    // gave up somewhere: let the copies that are still in flight land (bounded) before the CTA and its
+    // shared memory go away; nothing is staged over the ring in that case
+    if (tid < kTcStages && copies_issued[tid] > 0)
+      for (int i = 0; i < (1 << 16) && !tc_mbar_try(bar_xfull + 8 * tid, (copies_issued[tid] - 1) & 1); ++i) __nanosleep(64);
+    __syncthreads();
+    for (int i = 0; i < kTcSlots; ++i) fix_process(queues + i, tid, kTcThreads, a.K, a.V, a.in_dtype, a.S, (const double*)nullptr, *a.tables, a.status);
+  } else {
+    double* Sd = reinterpret_cast<double*>(smem + kTcSmS);
+    for (int idx = tid; idx < 128 * 128; idx += kTcThreads) {
+      const int k = idx >> 7, n = idx & 127;
+      Sd[((k & 15) * 8 + (k >> 4)) * kFixSdStride + n] = (double)__ldg(a.S + idx);
+    }
+    __syncthreads();
+    for (int i = 0; i < kTcSlots; ++i) fix_process(queues + i, tid, kTcThreads, a.K, a.V, a.in_dtype, a.S, Sd, *a.tables, a.status);
+  }
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem_base) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
   }
   if (tid == 0 && *abort_flag) set_status(a.status, PQ_ERR_TIMEOUT);
 }
@@ -435,7 +457,9 @@ static int32_t try_launch_encode_tc(const EncodeArgs& a, cudaStream_t stream) {
   const int n_row_tiles = (a.total_tokens + 127) / 128;
   const int n_tiles = n_row_tiles * 2 * a.n_kv_heads;
   const int grid = n_tiles < n_sm ? n_tiles : n_sm;
-  encode_tc_kernel<<<grid, kTcThreads, kTcSmTotal, stream>>>(a, maps, n_row_tiles);
+  EncodeArgs args = a;
+  if (take_debug_wait_failure(1)) args.debug |= 1u;
+  encode_tc_kernel<<<grid, kTcThreads, kTcSmTotal, stream>>>(args, maps, n_row_tiles);
   return 1;
 }
 

@@ -1,4 +1,5 @@
 // Host-side entry points: rotation generator, Lloyd-Max codebooks, derived tables, size queries.
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <vector>
@@ -53,6 +54,11 @@ inline void cell_moments(int level, double lo, double hi, double* m0, double* m1
 namespace pq {
 static thread_local cudaError_t g_last_cuda_error = cudaSuccess;
 void note_cuda_error(cudaError_t e) { g_last_cuda_error = e; }
+static std::atomic<int> g_debug_wait_failure{0};
+bool take_debug_wait_failure(int which) {
+  int armed = which;
+  return g_debug_wait_failure.compare_exchange_strong(armed, 0);
+}
 }  // namespace pq
 
 extern "C" {
@@ -78,6 +84,12 @@ const char* pq_status_string(int32_t status) {
 }
 
 int32_t pq_token_block(void) { return pq::kTokenBlock; }
+
+int32_t pq_debug_fail_next_wait(int32_t which) {
+  if (which < 0 || which > 2) return PQ_ERR_INVALID_ARG;
+  pq::g_debug_wait_failure.store(which);
+  return PQ_OK;
+}
 
 int32_t pq_make_rotation(int32_t d, uint64_t seed, float* S_host) {
   if (S_host == nullptr || d <= 0) return PQ_ERR_INVALID_ARG;
