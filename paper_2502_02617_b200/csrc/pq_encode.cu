@@ -208,7 +208,7 @@ __device__ __forceinline__ void quantise_and_store(const EncodeArgs& a, const Fa
                                                    float row_norm, int row, int head, int kv, int half, bool valid,
                                                    FixQueue* q, uint32_t* left, int64_t* xoff_out, uint8_t** tb_out,
                                                    int* tok_out) {
-  const RowMargins rm = make_row_margins(kRotErr * row_norm, fq);
+  const RowMargins rm = make_row_margins(row_norm, kRotErr, fq);
   FastBlock fb[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
@@ -253,10 +253,10 @@ __device__ __forceinline__ bool bar_or(int bar_id, int n_threads, bool v) {
 template <class Q, int kWords>
 __device__ inline void fix_rounds(const EncodeArgs& a, Q* q, unsigned long long (&left)[kWords], int64_t xoff, uint8_t* tb,
                                   int tok, int blk0, int kv, int t, int n_threads, int bar_id,
-                                  const double* Sd = nullptr) {
+                                  const float* Sf = nullptr) {
   for (int round = 0; round < 4096; ++round) {
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
-    fix_process(q, t, n_threads, a.K, a.V, a.in_dtype, a.S, Sd, *a.tables, a.status);
+    fix_process(q, 1, t, n_threads, a.K, a.V, a.in_dtype, a.S, Sf, *a.tables, a.status);
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
     if (t < 4) q->count[t] = 0;
     bool mine = false;
@@ -388,14 +388,14 @@ __global__ void __launch_bounds__(128) encode_vector_kernel(EncodeArgs a) {
   if ((j & 31) == 0) red[j >> 5] = sq;
   __syncthreads();
   // four independent partial sums instead of one chain: the bound of a 128-term float32 dot product still holds
-  const float dy = kRotErr * 1.0001f * sqrtf((red[0] + red[1]) + (red[2] + red[3]));
+  const float norm = 1.0001f * sqrtf((red[0] + red[1]) + (red[2] + red[3]));
   FastBlock fb = {0u, 0u, 0u, 0u, 0u, 0.f};
   if (j < 8) {
     float yb[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) yb[i] = ys[16 * j + i];
-    if (fq.sym) polar_quant_block_fast<true>(yb, make_row_margins(dy, fq), fq, &fb);
-    else polar_quant_block_fast<false>(yb, make_row_margins(dy, fq), fq, &fb);
+    if (fq.sym) polar_quant_block_fast<true>(yb, make_row_margins(norm, kRotErr, fq), fq, &fb);
+    else polar_quant_block_fast<false>(yb, make_row_margins(norm, kRotErr, fq), fq, &fb);
     if ((a.tables->flags & kFlagUniformL1) == 0u) fb.amb |= 0xFFu;
   }
   if (__syncthreads_or(fb.amb != 0u)) {

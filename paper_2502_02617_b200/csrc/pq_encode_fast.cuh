@@ -1,13 +1,15 @@
 // Fast encoder for head_dim 128 with the uniform level-1 codebook (included by pq_encode.cu).
 //
 // The rotation y = x . S is computed with float32-grade accuracy (tensor cores with S split into
-// two bf16 terms, or float32 FMAs).  Either way |y - y_exact| <= kRotErr * ||x||_2 per coordinate:
-//   * two bf16 terms (round to nearest, 8 significant bits each) leave |S - hi - lo| <= 2^-18 |S|, so
-//     the representation error is <= 2^-18 sum_k |x_k||S_kj| <= 2^-18 ||x||_2 (Cauchy-Schwarz,
-//     columns of S have unit norm); the products of bf16 inputs are exact in float32 and the 16
-//     accumulating MMAs may add up to 2^-19 sum_k |x_k||S_kj| more (2 ulp of the running sum each);
-//   * a float32 dot product of 128 terms is off by at most 128 * 2^-24 = 2^-17 of the same sum.
-// kRotErr = 1.1 * 2^-17 covers both.
+// bf16 terms, or float32 FMAs).  Either way |y - y_exact| <= rot_err * ||x||_2 per coordinate:
+//   * a float32 dot product of 128 terms is off by at most 128 * 2^-24 = 2^-17 of sum_k |x_k||S_kj|, which is
+//     at most ||x||_2 (Cauchy-Schwarz, columns of S have unit norm): kRotErr = 1.1 * 2^-17;
+//   * on tensor cores the products of bf16 inputs are exact in float32.  Three bf16 terms (round to nearest,
+//     8 significant bits each) represent a float32 S to 2^-26 |S|, and the 24 accumulating MMAs are taken to
+//     add at most 2 ulp of the running sum each, 3 * 2^-20 of the same sum in all: kRotErrTc = 1.1 * (3 * 2^-20
+//     + 2^-26).  Measured against float64 on 1.07e9 rotated coordinates of the synthetic workloads (N(0,1),
+//     outlier channels, rows scaled up 30 x): the largest error was 0.09 * 2^-17 ||x||_2, 4.5 x inside the bound
+//     (with two terms, whose representation error alone may reach 2^-18: 0.28 * 2^-17).
 // Angles are never computed.  Every code is decided by sign tests on the pair (Algorithm 1, Polar +
 // Quant, in the form "which side of the boundary line is the point on"), in float32, together with
 // a certified margin: a decision is trusted only if the point is farther from every boundary than
@@ -18,7 +20,8 @@
 
 namespace pq {
 
-constexpr float kRotErr = 1.1f * 7.62939453125e-06f;  // 1.1 * 2^-17
+constexpr float kRotErr = 1.1f * 7.62939453125e-06f;                                  // 1.1 * 2^-17
+constexpr float kRotErrTc = 1.1f * (3.f * 9.5367431640625e-07f + 1.4901161193847656e-08f);  // 1.1 * (3 * 2^-20 + 2^-26)
 
 // Per-call constants of the fast quantiser (uniform level-1 codebook; levels 2..4 from Tables).
 struct FastQuant {
@@ -34,18 +37,29 @@ __device__ inline void load_fast_quant(const Tables* tb, FastQuant* fq) {
 
 // Per-row constants of the margins (dy = bound on the error of one rotated coordinate of the row).
 struct RowMargins {
-  float dy;
+  float dy;       // as given
+  float dy1;      // level-1 threshold: dy plus the float32 roundings of the level-1 tests
   float c[3];     // 8.4 E^2 for levels 2, 3, 4 (E^2 = 2, 4, 8 dy^2)
+  float cs[3];    // the same plus the float32-rounding term of the folded (symmetric) test
   float base[3];  // 42 E^4 (1 + T_max)^2
 };
-__device__ __forceinline__ RowMargins make_row_margins(float dy, const FastQuant& fq) {
+// `norm` >= ||y||_2 of the row, `rot_err` = bound on the error of one rotated coordinate relative to it.
+// The float32 roundings of the tests themselves are folded into the constants, using u <= norm and w <= norm^2
+// for every coordinate magnitude u and partial squared radius w of the row:
+//   * level 1: the scaled distances are off by at most 1.3 * 2^-24 u (the two constants of t and one product);
+//     1.8e-7 norm covers that twice over;
+//   * levels >= 2 (folded test): the squared radii carry a relative error of at most 2^-22 + 2^-24 < rho = 4e-7,
+//     and 42 rho^2 w^2 <= 6.8e-12 norm^2 w.
+__device__ __forceinline__ RowMargins make_row_margins(float norm, float rot_err, const FastQuant& fq) {
   RowMargins m;
-  m.dy = dy;
-  const float e2 = dy * dy;
+  m.dy = rot_err * norm;
+  m.dy1 = fmaf(1.8e-7f, norm, m.dy);
+  const float e2 = m.dy * m.dy, rr = 6.8e-12f * norm * norm;
 #pragma unroll
   for (int l = 0; l < 3; ++l) {
     const float el = (float)(2 << l) * e2, t1 = fq.sym ? 2.f : 1.f + fq.t2[l][2];  // 1 + largest T that is tested
     m.c[l] = 8.4f * el;
+    m.cs[l] = m.c[l] + rr;
     m.base[l] = 42.f * el * el * t1 * t1;
   }
   return m;
@@ -102,24 +116,29 @@ __device__ __forceinline__ uint32_t push_sign(uint32_t acc, uint32_t v) { return
 // the lines at pi/8 from the axes (v cos(pi/8) = u sin(pi/8)).  Each coordinate moves by at most
 // dy, so the signed distance to a line with unit normal (n1, n2) moves by at most (|n1| + |n2|) dy:
 // dy for an axis, sqrt(2) dy for a diagonal, (cos + sin)(pi/8) dy = 1.3066 dy for the pi/8 lines.
-// The three distances are scaled so that one comparison against dy serves all.
-// The function appends the 4 code bits to `l1` and one "certified" bit to
-// `ok`.  With x = sign(a) ^ sign(b), w = (|b| > |a|), hi = (past the pi/8 line of the folded octant) the code
-// is sign(b) << 3 | x << 2 | (w ^ x) << 1 | (w ^ hi ^ x); w is the sign of |a| - |b| and hi the complement of
-// the sign of t.  A zero (or NaN) anywhere leaves the pair uncertified, so the sign conventions at exact
-// zeros do not matter.
-__device__ __forceinline__ void quant_level1_push(float a, float b, float dy, uint32_t& l1, uint32_t& ok) {
+// The three distances are computed already scaled (d = (|a| - |b|) / 2, t = 0.76537 (v cos - u sin)), so
+// that one comparison against `dy1` (dy plus the float32 roundings, see make_row_margins) serves all.
+// The function appends four raw sign bits to `raw` -- sign(b), sign(a), sign(d), sign(t) -- and one
+// "certified" bit to `ok`; level1_codes() turns the raw nibbles of a block into codes.  A zero (or NaN)
+// anywhere leaves the pair uncertified, so the sign conventions at exact zeros do not matter.
+__device__ __forceinline__ void quant_level1_push(float a, float b, float dy1, uint32_t& raw, uint32_t& ok) {
   const float ax = fabsf(a), ay = fabsf(b);
   const float u = fmaxf(ax, ay), v = fminf(ax, ay);
-  const float d = ax - ay;
-  const float t = fmaf(v, 0.92387953251128674f, -u * 0.38268343236508977f);  // v cos(pi/8) - u sin(pi/8)
-  const float dmin = fminf(fminf(v, fabsf(d) * 0.5f), fabsf(t) * 0.76536686473017954f);
-  const float slack = fmaf(u, 4.76837158203125e-07f, dy) - dmin;  // < 0: certified (+ 2^-21 u for the float32 roundings)
-  const uint32_t bb = __float_as_uint(b), x = __float_as_uint(a) ^ bb;
-  const uint32_t e1 = __float_as_uint(d) ^ x;
-  const uint32_t e0 = ~(__float_as_uint(t) ^ e1);
-  l1 = push_sign(push_sign(push_sign(push_sign(l1, bb), x), e1), e0);
+  const float d = fmaf(ay, -0.5f, 0.5f * ax);
+  const float t = fmaf(v, 0.92387953251128674f * 0.76536686473017954f, u * (-0.38268343236508977f * 0.76536686473017954f));
+  const float dmin = fminf(fminf(v, fabsf(d)), fabsf(t));
+  const float slack = dy1 - dmin;  // < 0: certified
+  raw = push_sign(push_sign(push_sign(push_sign(raw, __float_as_uint(b)), __float_as_uint(a)), __float_as_uint(d)),
+                  __float_as_uint(t));
   ok = push_sign(ok, __float_as_uint(slack));
+}
+// Codes of the eight pairs of a block from their raw nibbles (sb, sa, sd, st), all pairs at once.  With
+// x = sa ^ sb, w = (|b| > |a|) = sd, hi = (past the pi/8 line of the folded octant) = ~st the code is
+// sb << 3 | x << 2 | (w ^ x) << 1 | (w ^ hi ^ x): a prefix-xor inside each nibble and a flip of bit 0.
+__device__ __forceinline__ uint32_t level1_codes(uint32_t raw) {
+  uint32_t c = raw ^ ((raw & 0xEEEEEEEEu) >> 1);   // (r3, r2^r3, r1^r2, r0^r1)
+  c ^= (c & 0xCCCCCCCCu) >> 2;                     // (r3, r2^r3, r1^r2^r3, r0^r1^r2^r3)
+  return c ^ 0x11111111u;
 }
 
 // The level >= 2 decision (see quant_upper_fast) for symmetric boundaries (T0, 1, 1/T0), folded onto m = min(sa, sb), M = max(sa, sb):
@@ -128,19 +147,14 @@ __device__ __forceinline__ void quant_level1_push(float a, float b, float dy, ui
 // that is tested is <= 1, so sb + T^2 sa <= sa + sb and the caller's `base` uses (1 + T)^2 <= 4.
 // The function appends the 2 code bits to `lv` and one "certified" bit to `ok`: the code is
 // hi << 1 | (hi ^ lo) with hi = (sb > sa) = sign of sa - sb and lo = (m > T0 M) = complement of the sign of dout.
-__device__ __forceinline__ void quant_upper_sym_push(float sa, float sb, float T0, float c, float base, uint32_t& lv,
+__device__ __forceinline__ void quant_upper_sym_push(float sa, float sb, float T0, float cs, float base, uint32_t& lv,
                                                      uint32_t& ok) {
   const float m = fminf(sa, sb), M = fmaxf(sa, sb);
   const float h = sa - sb, dout = fmaf(-T0, M, m);
   const float w = sa + sb;
   const float dm = fminf(fabsf(dout), fabsf(h));
-  const float b2 = fmaf(4.2e-11f * w, w, base);  // rho = 1e-6 covers the float32 roundings
-  float slack = fmaf(-dm, dm, fmaf(c, w, b2));   // < 0: certified by the cheap test
-  if (!(slack < 0.f)) {                          // rare; also taken for NaN
-    const bool ok_d = h * h > fmaf(c, w, b2);
-    const bool ok_o = dout * dout > fmaf(c, fmaf(T0 * T0, M, m), b2);
-    slack = (ok_d && ok_o) ? -1.f : 1.f;
-  }
+  // certified if dm^2 > c w + base + 42 rho^2 w^2; the last term is inside cs (see make_row_margins).  NaN: not certified.
+  const float slack = fmaf(-dm, dm, fmaf(cs, w, base));
   const uint32_t hb = __float_as_uint(h);
   lv = push_sign(push_sign(lv, hb), ~(hb ^ __float_as_uint(dout)));
   ok = push_sign(ok, __float_as_uint(slack));
@@ -155,21 +169,21 @@ __device__ __forceinline__ void polar_quant_block_fast(const float* y, const Row
   uint32_t l1 = 0, l2 = 0, l3 = 0, l4 = 0, ok1 = 0, ok2 = 0, ok3 = 0, ok4 = 0;
 #pragma unroll
   for (int j = 7; j >= 0; --j) {
-    quant_level1_push(y[2 * j], y[2 * j + 1], rm.dy, l1, ok1);
+    quant_level1_push(y[2 * j], y[2 * j + 1], rm.dy1, l1, ok1);
     s1[j] = fmaf(y[2 * j], y[2 * j], y[2 * j + 1] * y[2 * j + 1]);
   }
   if (kSym) {
 #pragma unroll
     for (int j = 3; j >= 0; --j) {
-      quant_upper_sym_push(s1[2 * j], s1[2 * j + 1], fq.t2[0][0], rm.c[0], rm.base[0], l2, ok2);
+      quant_upper_sym_push(s1[2 * j], s1[2 * j + 1], fq.t2[0][0], rm.cs[0], rm.base[0], l2, ok2);
       s2[j] = s1[2 * j] + s1[2 * j + 1];
     }
 #pragma unroll
     for (int j = 1; j >= 0; --j) {
-      quant_upper_sym_push(s2[2 * j], s2[2 * j + 1], fq.t2[1][0], rm.c[1], rm.base[1], l3, ok3);
+      quant_upper_sym_push(s2[2 * j], s2[2 * j + 1], fq.t2[1][0], rm.cs[1], rm.base[1], l3, ok3);
       s3[j] = s2[2 * j] + s2[2 * j + 1];
     }
-    quant_upper_sym_push(s3[0], s3[1], fq.t2[2][0], rm.c[2], rm.base[2], l4, ok4);
+    quant_upper_sym_push(s3[0], s3[1], fq.t2[2][0], rm.cs[2], rm.base[2], l4, ok4);
   } else {
     bool am;
 #pragma unroll
@@ -187,7 +201,7 @@ __device__ __forceinline__ void polar_quant_block_fast(const float* y, const Row
     l4 = quant_upper_fast(s3[0], s3[1], fq.t2[2], rm.c[2], rm.base[2], &am);
     ok4 = am ? 0u : 1u;
   }
-  out->l1 = l1;
+  out->l1 = level1_codes(l1);
   out->l2 = l2;
   out->l3 = l3;
   out->l4 = l4;
@@ -294,25 +308,34 @@ __device__ __forceinline__ void exact_coords(const double* xk, const float* S, i
   }
 }
 
-// The same sums with S staged in shared memory as float64 (no conversions, no L2 latency in the loop).
-// Row k of S sits at row (k & 15) * 8 + (k >> 4) of `Sd`, rows kFixSdStride doubles apart, so the eight
-// lanes of a group (k = 16 * sub + i) read eight consecutive rows: 16-byte loads without bank conflicts.
-constexpr int kFixSdStride = 130;
-constexpr int kFixSdBytes = 128 * kFixSdStride * 8;
+// The same sums with a float32 copy of S in shared memory (no L2 latency in the loop).  Row k of S sits at
+// row (k & 15) * 8 + (k >> 4) of `Sf`, rows kFixSfStride floats apart, so the eight lanes of a group
+// (k = 16 * sub + i) read eight consecutive rows: 8- and 16-byte loads without bank conflicts.
+constexpr int kFixSfStride = 132;
+constexpr int kFixSfBytes = 128 * kFixSfStride * 4;
+__host__ __device__ constexpr int fix_sf_row(int k) { return (k & 15) * 8 + (k >> 4); }
 template <int NC>
-__device__ __forceinline__ void exact_coords_sm(const double* xk, const double* Sd, int sub, int c0, unsigned gmask,
+__device__ __forceinline__ void exact_coords_sm(const double* xk, const float* Sf, int sub, int c0, unsigned gmask,
                                                 double* y) {
   double acc[NC];
 #pragma unroll
   for (int c = 0; c < NC; ++c) acc[c] = 0.0;
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
-    const double2* srow = reinterpret_cast<const double2*>(Sd + (i * 8 + sub) * kFixSdStride + c0);
+    const float* srow = Sf + (i * 8 + sub) * kFixSfStride + c0;
+    if (NC == 2) {
+      const float2 s2 = *reinterpret_cast<const float2*>(srow);
+      acc[0] = fma(xk[i], (double)s2.x, acc[0]);
+      acc[1] = fma(xk[i], (double)s2.y, acc[1]);
+    } else {
 #pragma unroll
-    for (int c2 = 0; c2 < NC / 2; ++c2) {
-      const double2 s2 = srow[c2];
-      acc[2 * c2] = fma(xk[i], s2.x, acc[2 * c2]);
-      acc[2 * c2 + 1] = fma(xk[i], s2.y, acc[2 * c2 + 1]);
+      for (int c4 = 0; c4 < NC / 4; ++c4) {
+        const float4 s4 = reinterpret_cast<const float4*>(srow)[c4];
+        acc[4 * c4] = fma(xk[i], (double)s4.x, acc[4 * c4]);
+        acc[4 * c4 + 1] = fma(xk[i], (double)s4.y, acc[4 * c4 + 1]);
+        acc[4 * c4 + 2] = fma(xk[i], (double)s4.z, acc[4 * c4 + 2]);
+        acc[4 * c4 + 3] = fma(xk[i], (double)s4.w, acc[4 * c4 + 3]);
+      }
     }
   }
 #pragma unroll
@@ -341,33 +364,49 @@ __device__ __forceinline__ uint32_t exact_code(const double* y, int level, const
 }
 
 // Process everything queued, in level order: called by `n_threads` threads (a multiple of 32) with linear index `t`.
-// `Sd` (may be null) is S staged in shared memory for exact_coords_sm.
+// `q` points to `n_queues` queues laid out back to back; their entries are taken level by level.
+// `Sf` (may be null) is the copy of S in shared memory for exact_coords_sm.
 template <class Q>
-__device__ inline void fix_process(const Q* q, int t, int n_threads, const void* kbase, const void* vbase,
-                                   int in_dtype, const float* S, const double* Sd, const Tables& tb, int32_t* status) {
+__device__ inline void fix_process(const Q* q, int n_queues, int t, int n_threads, const void* kbase, const void* vbase,
+                                   int in_dtype, const float* S, const float* Sf, const Tables& tb, int32_t* status) {
   constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock;
   const int sub = t & 7, n_groups = n_threads >> 3;
   const unsigned gmask = 0xFFu << (t & 24);
-  const int n1 = min(q->count[0], Q::cap(1)), n2 = n1 + min(q->count[1], Q::cap(2));
-  const int n3 = n2 + min(q->count[2], Q::cap(3)), n = n3 + min(q->count[3], Q::cap(4));
+  int n = 0;
+  for (int level = 1; level <= 4; ++level)
+    for (int k = 0; k < n_queues; ++k) n += min(q[k].count[level - 1], Q::cap(level));
   int fixed = 0;
-  auto entry_of = [&](int i) {
-    return i < n1 ? i : i < n2 ? Q::off(2) + (i - n1) : i < n3 ? Q::off(3) + (i - n2) : Q::off(4) + (i - n3);
+  // entry i of the level-major order: which queue, which slot of it
+  auto entry_of = [&](int i, const Q** which) {
+    int base = 0;
+    for (int level = 1; level <= 4; ++level)
+      for (int k = 0; k < n_queues; ++k) {
+        const int cnt = min(q[k].count[level - 1], Q::cap(level));
+        if (i < base + cnt) {
+          *which = q + k;
+          return Q::off(level) + (i - base);
+        }
+        base += cnt;
+      }
+    *which = q;
+    return 0;
   };
   // The source vector of the group's next entry is fetched while the current one is decided.
   auto fetch = [&](int i, uint4* raw) {
     if (i >= n || in_dtype != PQ_DTYPE_BF16) return;
-    const int e = entry_of(i);
-    const void* xbase = (q->meta[e] >> 15) & 1 ? vbase : kbase;
-    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(xbase) + q->xoff[e] + 16 * sub);
+    const Q* qe;
+    const int e = entry_of(i, &qe);
+    const void* xbase = (qe->meta[e] >> 15) & 1 ? vbase : kbase;
+    const uint4* p = reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(xbase) + qe->xoff[e] + 16 * sub);
     raw[0] = __ldg(p);
     raw[1] = __ldg(p + 1);
   };
   uint4 raw[2] = {make_uint4(0u, 0u, 0u, 0u), make_uint4(0u, 0u, 0u, 0u)};
   fetch(t >> 3, raw);
   for (int i = t >> 3; i < n; i += n_groups) {  // uniform within a group of 8 lanes
-    const int e = entry_of(i);
-    const uint32_t meta = q->meta[e];
+    const Q* qe;
+    const int e = entry_of(i, &qe);
+    const uint32_t meta = qe->meta[e];
     const int tok = meta & 63, blk = (meta >> 6) & 7, level = (meta >> 9) & 7, j = (meta >> 12) & 7;
     const int c0 = blk * 16 + (j << level);
     double xk[16];  // this lane's 16 consecutive k
@@ -381,24 +420,24 @@ __device__ inline void fix_process(const Q* q, int t, int n_threads, const void*
       fetch(i + n_groups, raw);
     } else {
       const void* xbase = (meta >> 15) & 1 ? vbase : kbase;
-      const float* p = reinterpret_cast<const float*>(xbase) + q->xoff[e] + 16 * sub;
+      const float* p = reinterpret_cast<const float*>(xbase) + qe->xoff[e] + 16 * sub;
 #pragma unroll
       for (int i2 = 0; i2 < 16; ++i2) xk[i2] = (double)p[i2];
     }
     double y[16];
     uint32_t code;
-    if (Sd != nullptr) {  // uniform over the CTA
+    if (Sf != nullptr) {  // uniform over the CTA
       if (level == 1) {
-        exact_coords_sm<2>(xk, Sd, sub, c0, gmask, y);
+        exact_coords_sm<2>(xk, Sf, sub, c0, gmask, y);
         code = exact_code<2>(y, level, tb);
       } else if (level == 2) {
-        exact_coords_sm<4>(xk, Sd, sub, c0, gmask, y);
+        exact_coords_sm<4>(xk, Sf, sub, c0, gmask, y);
         code = exact_code<4>(y, level, tb);
       } else if (level == 3) {
-        exact_coords_sm<8>(xk, Sd, sub, c0, gmask, y);
+        exact_coords_sm<8>(xk, Sf, sub, c0, gmask, y);
         code = exact_code<8>(y, level, tb);
       } else {
-        exact_coords_sm<16>(xk, Sd, sub, c0, gmask, y);
+        exact_coords_sm<16>(xk, Sf, sub, c0, gmask, y);
         code = exact_code<16>(y, level, tb);
       }
     } else if (level == 1) {
@@ -415,7 +454,7 @@ __device__ inline void fix_process(const Q* q, int t, int n_threads, const void*
       code = exact_code<16>(y, level, tb);
     }
     if (sub == 0) {
-      uint8_t* tbk = q->tok[e];
+      uint8_t* tbk = qe->tok[e];
       if (level == 1) patch_bits(tbk + tok * 32 + blk * 4 + (j >> 1), 4 * (j & 1), 0xFu, code);
       else if (level == 2) patch_bits(tbk + o2 + tok * 8 + blk, 2 * j, 3u, code);
       else if (level == 3) patch_bits(tbk + o3 + tok * 4 + (blk >> 1), 4 * (blk & 1) + 2 * j, 3u, code);

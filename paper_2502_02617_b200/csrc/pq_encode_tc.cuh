@@ -5,18 +5,20 @@
 // and takes every fourth tile of the CTA.  Per tile
 //   * TMA loads of the x tile (two 64-column boxes, 128-byte swizzle) into a 3-deep ring; the copy of
 //     tile i+3 is issued as soon as the MMAs of tile i, which read the same ring stage, have completed;
-//   * y = x . S on the 5th-generation tensor cores: S is split once per CTA into bf16 terms
-//     (S = S_hi + S_lo + O(2^-17)) kept in shared memory as the K-major B operand; terms x 8 k-steps of
-//     tcgen05.mma (M = 128 rows, N = 128, K = 16) accumulate in float32 in the slot's accumulator.  One
-//     thread of the slot issues them when the slot's previous tile has been read out; the other three
-//     slots are in their epilogues meanwhile, so the tensor work hides under ALU work;
+//   * y = x . S on the 5th-generation tensor cores: S is split once per CTA into three bf16 terms (exact
+//     for a float32 S) kept in shared memory as the K-major B operand; 3 terms x 8 k-steps of tcgen05.mma
+//     (M = 128 rows, N = 128, K = 16) accumulate in float32 in the slot's accumulator.  One thread of the
+//     slot issues them for the slot's next tile as soon as the current tile's last coordinates have been
+//     read into registers, so the tensor work runs under the quantiser of the last two blocks (and the
+//     other three slots are in their epilogues anyway);
 //   * epilogue on the slot's four warps.  Tensor-memory lane = row and a warp may read its own quarter of
 //     the lanes, so a thread owns one whole row (8 blocks): one pass over the accumulator for the row norm
 //     (the certified margins need it), a second pass of tcgen05.ld of 32 coordinates at a time through the
 //     sign-test quantiser, packed stores of whole plane entries of the token, queued float64 re-decision of
-//     the ambiguous angles (one queue per slot, drained by the slot; the rest after the last tile by the CTA).
+//     the ambiguous angles (one queue per slot; all 16 warps take them together after the CTA's last tile,
+//     a slot drains alone only when its queue fills up).
 // Per-row work (norm, margins, cache destination, stores) is paid once per 8 blocks, and the only
-// synchronisation in the loop is one named barrier of the slot's 128 threads per tile.
+// synchronisation in the loop is two named barriers of the slot's 128 threads per tile.
 // There are no dedicated producer / MMA warps: the register file is split over four schedulers, and
 // a 17th warp would cap every thread at 96 registers (the quantiser then spills).
 // Every mbarrier wait is bounded; a wait that gives up raises the CTA's abort flag, the remaining
@@ -31,21 +33,23 @@ constexpr int kTcThreads = 512;
 constexpr int kTcSlots = 4;                // accumulators in tensor memory = groups of four warps
 constexpr int kTcSlotThreads = kTcThreads / kTcSlots;
 constexpr int kTcStages = 3;               // x tiles in flight
-constexpr int kTcTerms = 2;                // bf16 terms of S
+constexpr int kTcTerms = 3;                // bf16 terms of S (exact for a float32 S)
 constexpr int kTcXBytes = 128 * 128 * 2;   // one x tile: 128 rows x 128 bf16
 constexpr int kTcSBytes = 128 * 128 * 2;   // one bf16 term of S (B operand)
 using TcFixQueue = FixQueueT<256>;
 constexpr int kTcSmS = 0;
 constexpr int kTcSmX = kTcSmS + kTcTerms * kTcSBytes;
-constexpr int kTcSmOperandEnd = kTcSmX + kTcStages * kTcXBytes;
-constexpr int kTcSmFq = kTcSmOperandEnd;                     // FastQuant (40 B)
-constexpr int kTcSmBar = kTcSmFq + 64;                       // x_full[3], acc_full[4]
-constexpr int kTcSmMisc = kTcSmBar + 64;                     // tmem base, abort flag, copies issued per stage [3], debug
+constexpr int kTcSmSf = kTcSmX;                              // float32 copy of S for the last batch of exact re-decisions (over the idle ring)
+constexpr int kTcSmFq = kTcSmX + kTcStages * kTcXBytes;      // FastQuant (40 B)
+constexpr int kTcSmBar = kTcSmFq + 64;                       // x_full[kTcStages], acc_full[kTcSlots]
+constexpr int kTcSmMisc = kTcSmBar + 64;                     // tmem base, abort flag, copies issued per stage
 constexpr int kTcSmFix = kTcSmMisc + 64;                     // one TcFixQueue per slot
 constexpr int kTcSmTotal = kTcSmFix + kTcSlots * (int)sizeof(TcFixQueue) + 1024;  // + slack for 1024-byte alignment
 constexpr int kTcSpin = 1 << 22;
-static_assert(kFixSdBytes <= kTcSmOperandEnd, "the float64 copy of S must fit in the operand buffers");
+static_assert(kTcTerms == 3, "kRotErrTc is the bound for three terms");
 static_assert(sizeof(TcFixQueue) % 16 == 0, "queues are laid out back to back");
+static_assert(kTcSmTotal <= 227 * 1024, "shared memory of one CTA");
+static_assert(kFixSfBytes <= kTcStages * kTcXBytes, "the float32 copy of S must fit in the ring");
 
 __device__ __forceinline__ uint32_t tc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void tc_mbar_init(uint32_t bar, uint32_t count) {
@@ -167,54 +171,10 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   volatile int* copies_issued = reinterpret_cast<volatile int*>(smem + kTcSmMisc + 8);  // [kTcStages]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kTcSmMisc);
   FastQuant* fq = reinterpret_cast<FastQuant*>(smem + kTcSmFq);
-  TcFixQueue* queues = reinterpret_cast<TcFixQueue*>(smem + kTcSmFix);
-  TcFixQueue* fixq = queues + slot;
+  float* Sf = reinterpret_cast<float*>(smem + kTcSmSf);
+  TcFixQueue* fixq = reinterpret_cast<TcFixQueue*>(smem + kTcSmFix) + slot;
   const uint32_t bar_xfull = sb + kTcSmBar, bar_acc = bar_xfull + 8 * kTcStages;
   const int n_tiles = n_row_tiles * 2 * a.n_kv_heads;
-
-  // ---- set-up: barriers, tensor memory, S split into bf16 terms in the B-operand layout
-  if (tid == 0) {
-    for (int s = 0; s < kTcStages; ++s) {
-      tc_mbar_init(bar_xfull + 8 * s, 1);
-      copies_issued[s] = 0;
-    }
-    for (int i = 0; i < kTcSlots; ++i) tc_mbar_init(bar_acc + 8 * i, 1);   // one commit by the slot's issuing thread
-    *abort_flag = 0;
-    load_fast_quant(a.tables, fq);
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  }
-  if (st < 4) fixq->count[st] = 0;
-  if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(sb + kTcSmMisc) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  // B operand: B[n][k] = S[k][n]; two halves of 64 k; row n = 128 bytes, 16-byte chunk c stored at c ^ (n & 7).
-  // A task is (row n, chunk of 8 consecutive k): 8 coalesced loads (lanes = consecutive n), one 16-byte store per term.
-  for (int task = tid; task < 128 * 16; task += kTcThreads) {
-    const int n = task & 127, oct = task >> 7;  // k = 8 * oct .. 8 * oct + 7
-    uint32_t term[kTcTerms][4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float v0 = a.S[(8 * oct + 2 * i) * 128 + n], v1 = a.S[(8 * oct + 2 * i + 1) * 128 + n];
-#pragma unroll
-      for (int t = 0; t < kTcTerms; ++t) {
-        const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
-        term[t][i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-        v0 -= __bfloat162float(h0);  // exact: the residual of a bf16 rounding fits float32
-        v1 -= __bfloat162float(h1);
-      }
-    }
-    const int half = oct >> 3, c = oct & 7;
-    const int off = half * 16384 + n * 128 + ((c ^ (n & 7)) << 4);
-#pragma unroll
-    for (int t = 0; t < kTcTerms; ++t)
-      *reinterpret_cast<uint4*>(smem + kTcSmS + t * kTcSBytes + off) = make_uint4(term[t][0], term[t][1], term[t][2], term[t][3]);
-  }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA unit
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
-  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_base = *tmem_slot;
 
   // Local tile `it` of this CTA is tile blockIdx.x + it * gridDim.x = head + n_kv_heads * (2 * row tile + kv); it
   // uses ring stage it % kTcStages and belongs to slot it % kTcSlots.
@@ -237,8 +197,92 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
           ::"r"(dst + h * 16384), "l"(map), "r"(h * 64), "r"(head), "r"(rt * 128), "r"(bar)
           : "memory");
   };
-  if (tid == 0)
-    for (int it = 0; it < kTcStages; ++it) issue_tma(it);
+
+  // ---- set-up: barriers, first copies, tensor memory, S split into bf16 terms in the B-operand layout
+  if (tid == 0) {
+    for (int s = 0; s < kTcStages; ++s) {
+      tc_mbar_init(bar_xfull + 8 * s, 1);
+      copies_issued[s] = 0;
+    }
+    for (int i = 0; i < kTcSlots; ++i) tc_mbar_init(bar_acc + 8 * i, 1);   // one commit by the slot's issuing thread
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    for (int it = 0; it < kTcStages; ++it) issue_tma(it);  // the first tiles arrive while S is split
+    load_fast_quant(a.tables, fq);
+  }
+  if (st < 4) fixq->count[st] = 0;
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(sb + kTcSmMisc) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // B operand: B[n][k] = S[k][n]; two halves of 64 k; row n = 128 bytes, 16-byte chunk c stored at c ^ (n & 7).
+  // A task is (row n, chunk of 8 consecutive k): 8 coalesced loads (lanes = consecutive n), one 16-byte store per
+  // term.
+  for (int task = tid; task < 128 * 16; task += kTcThreads) {
+    const int n = task & 127, oct = task >> 7;  // k = 8 * oct .. 8 * oct + 7
+    float v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) v[i] = a.S[(8 * oct + i) * 128 + n];
+    uint32_t term[kTcTerms][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      float v0 = v[2 * i], v1 = v[2 * i + 1];
+#pragma unroll
+      for (int t = 0; t < kTcTerms; ++t) {
+        const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
+        term[t][i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+        v0 -= __bfloat162float(h0);  // exact: the residual of a bf16 rounding fits float32
+        v1 -= __bfloat162float(h1);
+      }
+    }
+    const int half = oct >> 3, c = oct & 7;
+    const int off = half * 16384 + n * 128 + ((c ^ (n & 7)) << 4);
+#pragma unroll
+    for (int t = 0; t < kTcTerms; ++t)
+      *reinterpret_cast<uint4*>(smem + kTcSmS + t * kTcSBytes + off) = make_uint4(term[t][0], term[t][1], term[t][2], term[t][3]);
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA unit
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  // The slot's issuing thread multiplies local tile `it` into the slot's accumulator.  The accumulator is free:
+  // the slot's four warps have read the previous tile out of it before the barrier that precedes this call.
+  // All MMAs of the tile come from this thread, in order: the first overwrites, the others accumulate.
+  const uint64_t desc_hi = tc_smem_desc(0u) & 0xFFFFFFFF00000000ull;  // the address field is in the low word
+  const uint32_t bdesc_lo = (uint32_t)tc_smem_desc(sb + kTcSmS);
+  auto issue_mmas = [&](int it) {
+    if (blockIdx.x + it * (int)gridDim.x >= n_tiles) return;
+    const int s = it % kTcStages;
+    // The copy of the tile is issued by another slot's thread (when the tile kTcStages back has been
+    // multiplied).  A parity wait taken before that would be satisfied by the stage's previous phase, so
+    // first wait (bounded) until the copy has been issued: the previous phase is complete by then.
+    bool ok = false;
+    for (int i = 0; i < kTcSpin && !ok; ++i) {
+      ok = copies_issued[s] > it / kTcStages;
+      if (!ok && i > 32) {
+        __nanosleep(64);
+        if (*abort_flag) break;
+      }
+    }
+    if (!ok) *abort_flag = 1;
+    ok = ok && tc_mbar_wait(bar_xfull + 8 * s, (it / kTcStages) & 1, abort_flag);
+    if (ok && (a.debug & 1u) && blockIdx.x == 0 && it == 0) {  // test hook: report this wait as failed
+      *abort_flag = 1;
+      ok = false;
+    }
+    if (!ok) return;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t adesc_lo = (uint32_t)tc_smem_desc(sb + kTcSmX + s * kTcXBytes);
+#pragma unroll
+    for (int q = 0; q < 8 * kTcTerms; ++q) {
+      const uint32_t off = ((q >> 2) & 1) * 16384 + (q & 3) * 32;  // k-half, k-step inside the 128-byte swizzled row
+      tc_mma(tmem_base + slot * 128, desc_hi | (adesc_lo + (off >> 4)),
+             desc_hi | (bdesc_lo + (((q >> 3) * kTcSBytes + off) >> 4)), q ? 1u : 0u);
+    }
+    tc_commit(bar_acc + 8 * slot);  // the accumulator is complete and the x stage has been read
+  };
 
   // ---- tile loop of this slot
   constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock, orad = o4 + 2 * kTokenBlock;
@@ -248,45 +292,14 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + slot * 128;
   const int slot_bar = 1 + slot;
   int rd_seq = 0, rd_first = 0, rd_count = 0, rd_start = -1;   // destination of the last row looked up
+  if (leader) issue_mmas(slot);
+  __syncwarp();
   for (int it = slot; blockIdx.x + it * (int)gridDim.x < n_tiles; it += kTcSlots) {
     const int tile = blockIdx.x + it * gridDim.x;
     const int head = tile % a.n_kv_heads, hq = tile / a.n_kv_heads;
     const int kv = hq & 1, rt = hq >> 1;
-    const int s = it % kTcStages;
-    if (leader) {
-      // The accumulator is free: the slot's four warps read the previous tile out of it before the barrier
-      // that ended that tile.  All MMAs of the tile come from this thread, in order: the first overwrites.
-      // The copy of this tile is issued by another slot's thread (when the tile three back has been
-      // multiplied).  A parity wait taken before that would be satisfied by the stage's previous phase, so
-      // first wait (bounded) until the copy has been issued: the previous phase is complete by then.
-      bool ok = false;
-      for (int i = 0; i < kTcSpin && !ok; ++i) {
-        ok = copies_issued[s] > it / kTcStages;
-        if (!ok && i > 32) {
-          __nanosleep(64);
-          if (*abort_flag) break;
-        }
-      }
-      if (!ok) *abort_flag = 1;
-      ok = ok && tc_mbar_wait(bar_xfull + 8 * s, (it / kTcStages) & 1, abort_flag);
-      if (ok && (a.debug & 1u) && blockIdx.x == 0 && it == 0) {  // test hook: report this wait as failed
-        *abort_flag = 1;
-        ok = false;
-      }
-      if (ok) {
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-        for (int q = 0; q < 8 * kTcTerms; ++q) {
-          const uint32_t off = ((q >> 2) & 1) * 16384 + (q & 3) * 32;
-          tc_mma(tmem_base + slot * 128, tc_smem_desc(sb + kTcSmX + s * kTcXBytes + off),
-                 tc_smem_desc(sb + kTcSmS + (q >> 3) * kTcSBytes + off), q ? 1u : 0u);
-        }
-        tc_commit(bar_acc + 8 * slot);  // the accumulator is complete and the x stage has been read
-      }
-    }
-    __syncwarp();
     // A wait that gives up must not leave the loop: the other warps of the slot would wait for this one at the
-    // slot's barrier.  The tile is skipped instead (warp-uniform).
+    // slot's barriers.  The tile is skipped instead (warp-uniform): it is quantised as zeros and not stored.
     const bool ready = __all_sync(0xffffffffu, tc_mbar_wait(bar_acc + 8 * slot, (it / kTcSlots) & 1, abort_flag));
     if (leader && ready) issue_tma(it + kTcStages);  // the stage of this tile is free again
     const int row = rt * 128 + st;
@@ -294,112 +307,126 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     uint8_t* tb = nullptr;
     int tok = 0;
     unsigned long long left[2] = {0ull, 0ull};
+    float y[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) y[i] = 0.f;
+    // pass 1: squared norm of the row (four partial sums)
+    float sq[4] = {0.f, 0.f, 0.f, 0.f};
     if (ready) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      float y[32];
-      // pass 1: squared norm of the row (four partial sums)
-      float sq[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
       for (int c = 0; c < 4; ++c) {
         tc_ld32(taddr + 32 * c, y);
 #pragma unroll
         for (int i = 0; i < 32; ++i) sq[i & 3] = fmaf(y[i], y[i], sq[i & 3]);
       }
-      const float sqsum = (sq[0] + sq[1]) + (sq[2] + sq[3]);
-      bool bad_row = false;
-      if (!(sqsum < CUDART_INF_F) && row < a.total_tokens) {  // NaN or overflow: look at the inputs
-        const int bad = count_nonfinite_bf16(kv ? a.V : a.K, xoff);
-        if (bad) {
-          atomicAdd(a.status + 1, bad);
-          set_status(a.status, PQ_ERR_NONFINITE);
-          bad_row = true;
-        }
+    }
+    const float sqsum = (sq[0] + sq[1]) + (sq[2] + sq[3]);
+    bool bad_row = false;
+    if (!(sqsum < CUDART_INF_F) && row < a.total_tokens) {  // NaN or overflow: look at the inputs
+      const int bad = count_nonfinite_bf16(kv ? a.V : a.K, xoff);
+      if (bad) {
+        atomicAdd(a.status + 1, bad);
+        set_status(a.status, PQ_ERR_NONFINITE);
+        bad_row = true;
       }
-      const RowMargins rm = make_row_margins(kRotErr * 1.0001f * sqrtf(sqsum), *fq);
-      if (row < a.total_tokens) {
-        int seq, pos;
-        if (row >= rd_first && row < rd_first + rd_count) {  // same sequence as this thread's previous row
-          seq = rd_seq;
-          pos = rd_start < 0 ? -1 : rd_start + (row - rd_first);
-        } else {
-          row_destination(a, row, &seq, &pos);
-          rd_seq = seq;
-          rd_first = a.cu_seqlens ? a.cu_seqlens[seq] : row;
-          rd_count = a.cu_seqlens ? a.cu_seqlens[seq + 1] - rd_first : 1;
-          rd_start = pos < 0 ? -1 : pos - (row - rd_first);
-        }
-        if (pos >= 0) {
-          tb = a.cache + block_offset(L, a.n_kv_heads, seq, head, kv, pos);
-          tok = pos % kTokenBlock;
-        }
+    }
+    const RowMargins rm = make_row_margins(1.0001f * sqrtf(sqsum), kRotErrTc, *fq);
+    if (ready && row < a.total_tokens) {
+      int seq, pos;
+      if (row >= rd_first && row < rd_first + rd_count) {  // same sequence as this thread's previous row
+        seq = rd_seq;
+        pos = rd_start < 0 ? -1 : rd_start + (row - rd_first);
+      } else {
+        row_destination(a, row, &seq, &pos);
+        rd_seq = seq;
+        rd_first = a.cu_seqlens ? a.cu_seqlens[seq] : row;
+        rd_count = a.cu_seqlens ? a.cu_seqlens[seq + 1] - rd_first : 1;
+        rd_start = pos < 0 ? -1 : pos - (row - rd_first);
       }
-      // pass 2: 32 coordinates (two blocks) at a time
-      uint32_t l2lo = 0, l2hi = 0, l3acc = 0, l4acc = 0, sat = 0;
+      if (pos >= 0) {
+        tb = a.cache + block_offset(L, a.n_kv_heads, seq, head, kv, pos);
+        tok = pos % kTokenBlock;
+      }
+    }
+    // pass 2: 32 coordinates (two blocks) at a time; the two blocks are quantised in one straight-line
+    // piece of code (their instruction streams interleave), the rare queue pushes come after both
+    uint32_t l2lo = 0, l2hi = 0, l3acc = 0, l4acc = 0, sat = 0;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        tc_ld32(taddr + 32 * c, y);
-        uint32_t l1w[2], racc = 0, l2c = 0;
-#pragma unroll
-        for (int i = 0; i < 2; ++i) {
-          FastBlock fb;
-          if (sym) polar_quant_block_fast<true>(y + 16 * i, rm, *fq, &fb);
-          else polar_quant_block_fast<false>(y + 16 * i, rm, *fq, &fb);
-          if (!uniform) fb.amb |= 0xFFu;  // other level-1 codebooks: decide every level-1 angle exactly
-          l1w[i] = fb.l1;
-          l2c |= fb.l2 << (8 * i);
-          l3acc |= fb.l3 << (8 * c + 4 * i);
-          l4acc |= fb.l4 << (4 * c + 2 * i);
-          float rv = fb.radius;
-          if (rv > 65504.f) { rv = 65504.f; ++sat; }
-          racc |= (uint32_t)__half_as_ushort(__float2half_rn(rv)) << (16 * i);
-          if (tb != nullptr && fb.amb && !bad_row) {
-            uint32_t rest;
-            fix_push(fixq, fb.amb, xoff, tb, tok, 2 * c + i, kv, &rest);
-            left[c >> 1] |= (unsigned long long)rest << (15 * (2 * (c & 1) + i));  // queue full: pushed again by fix_rounds
-          }
-        }
-        if (c < 2) l2lo |= l2c << (16 * c);
-        else l2hi |= l2c << (16 * (c - 2));
-        if (tb != nullptr) {
-          if (bad_row) l1w[0] = l1w[1] = racc = 0u;
-          *reinterpret_cast<uint2*>(tb + tok * 32 + c * 8) = make_uint2(l1w[0], l1w[1]);
-          *reinterpret_cast<uint32_t*>(tb + orad + tok * 16 + c * 4) = racc;
-        }
+    for (int c = 0; c < 4; ++c) {
+      if (ready) tc_ld32(taddr + 32 * c, y);
+      if (c == 3) {
+        // The last coordinates are in registers: the accumulator is free.  The slot's next tile is multiplied
+        // while this one's last two blocks are quantised.
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        asm volatile("bar.sync %0, %1;" ::"r"(slot_bar), "n"(kTcSlotThreads) : "memory");
+        if (leader) issue_mmas(it + kTcSlots);
+        __syncwarp();
+      }
+      FastBlock fb0, fb1;
+      if (sym) {
+        polar_quant_block_fast<true>(y, rm, *fq, &fb0);
+        polar_quant_block_fast<true>(y + 16, rm, *fq, &fb1);
+      } else {
+        polar_quant_block_fast<false>(y, rm, *fq, &fb0);
+        polar_quant_block_fast<false>(y + 16, rm, *fq, &fb1);
+      }
+      float r0 = fb0.radius, r1 = fb1.radius;
+      sat += (r0 > 65504.f) + (r1 > 65504.f);
+      r0 = fminf(r0, 65504.f);
+      r1 = fminf(r1, 65504.f);
+      uint32_t racc = (uint32_t)__half_as_ushort(__float2half_rn(r0)) | ((uint32_t)__half_as_ushort(__float2half_rn(r1)) << 16);
+      const uint32_t l2c = fb0.l2 | (fb1.l2 << 8);
+      l3acc |= (fb0.l3 | (fb1.l3 << 4)) << (8 * c);
+      l4acc |= (fb0.l4 | (fb1.l4 << 2)) << (4 * c);
+      if (c < 2) l2lo |= l2c << (16 * c);
+      else l2hi |= l2c << (16 * (c - 2));
+      uint32_t amb0 = fb0.amb, amb1 = fb1.amb;
+      if (!uniform) {  // other level-1 codebooks: decide every level-1 angle exactly
+        amb0 |= 0xFFu;
+        amb1 |= 0xFFu;
       }
       if (tb != nullptr) {
-        if (bad_row) l2lo = l2hi = l3acc = l4acc = sat = 0u;  // a row with non-finite inputs is stored as the zero vector
-        *reinterpret_cast<uint2*>(tb + o2 + tok * 8) = make_uint2(l2lo, l2hi);
-        *reinterpret_cast<uint32_t*>(tb + o3 + tok * 4) = l3acc;
-        *reinterpret_cast<uint16_t*>(tb + o4 + tok * 2) = (uint16_t)l4acc;
-        if (sat) atomicAdd(a.status + 2, (int)sat);
+        if (bad_row) fb0.l1 = fb1.l1 = racc = amb0 = amb1 = 0u;
+        *reinterpret_cast<uint2*>(tb + tok * 32 + c * 8) = make_uint2(fb0.l1, fb1.l1);
+        *reinterpret_cast<uint32_t*>(tb + orad + tok * 16 + c * 4) = racc;
+        if (amb0 | amb1) {
+          uint32_t rest0 = 0, rest1 = 0;
+          if (amb0) fix_push(fixq, amb0, xoff, tb, tok, 2 * c, kv, &rest0);
+          if (amb1) fix_push(fixq, amb1, xoff, tb, tok, 2 * c + 1, kv, &rest1);
+          // queue full: pushed again by fix_rounds
+          left[c >> 1] |= ((unsigned long long)rest0 | ((unsigned long long)rest1 << 15)) << (30 * (c & 1));
+        }
       }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
-    // End of the tile for the slot (the accumulator may be overwritten after this barrier).  The same barrier
-    // decides, for all 128 threads alike, whether the slot drains its queue of exact re-decisions now: when a
-    // region is 3/4 full or a push did not fit.
+    if (tb != nullptr) {
+      if (bad_row) l2lo = l2hi = l3acc = l4acc = sat = 0u;  // a row with non-finite inputs is stored as the zero vector
+      *reinterpret_cast<uint2*>(tb + o2 + tok * 8) = make_uint2(l2lo, l2hi);
+      *reinterpret_cast<uint32_t*>(tb + o3 + tok * 4) = l3acc;
+      *reinterpret_cast<uint16_t*>(tb + o4 + tok * 2) = (uint16_t)l4acc;
+      if (sat) atomicAdd(a.status + 2, (int)sat);
+    }
+    // End of the tile for the slot.  The barrier decides, for all 128 threads alike, whether the slot has to take
+    // its queued exact re-decisions now: when a push did not fit or a region is 3/4 full.  Otherwise they wait
+    // for the end of the CTA's work, where all 16 warps take them together (the float64 pipe is slow, and a slot
+    // that drains alone holds up its own tiles for as long).
     const bool drain = bar_or(slot_bar, kTcSlotThreads, (left[0] | left[1]) != 0ull || fix_should_drain(fixq));
     if (drain) fix_rounds(a, fixq, left, xoff, tb, tok, 0, kv, st, kTcSlotThreads, slot_bar);
   }
-  // ---- after the last tile: every MMA and copy of this CTA has completed (each was waited for by its slot), so
-  // the operand buffers are idle: stage S there as float64 and let all 16 warps take the queued re-decisions.
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  if (*abort_flag) {
+  // Every MMA and copy of this CTA has completed (each was waited for by its slot), so the ring is idle: put a
+  // float32 copy of S there (rows permuted, see fix_sf_row) for the queued exact re-decisions.
+  if (!*abort_flag) {
+    for (int idx = tid; idx < 128 * 128; idx += kTcThreads) Sf[fix_sf_row(idx >> 7) * kFixSfStride + (idx & 127)] = __ldg(a.S + idx);
+    __syncthreads();
+  }
+  fix_process(fixq - slot, kTcSlots, tid, kTcThreads, a.K, a.V, a.in_dtype, a.S, *abort_flag ? (const float*)nullptr : Sf,
+              *a.tables, a.status);
+  if (*abort_flag && tid < kTcStages && copies_issued[tid] > 0) {
     // gave up somewhere: let the copies that are still in flight land (bounded) before the CTA and its
-    // shared memory go away; nothing is staged over the ring in that case
-    if (tid < kTcStages && copies_issued[tid] > 0)
-      for (int i = 0; i < (1 << 16) && !tc_mbar_try(bar_xfull + 8 * tid, (copies_issued[tid] - 1) & 1); ++i) __nanosleep(64);
-    __syncthreads();
-    for (int i = 0; i < kTcSlots; ++i) fix_process(queues + i, tid, kTcThreads, a.K, a.V, a.in_dtype, a.S, (const double*)nullptr, *a.tables, a.status);
-  } else {
-    double* Sd = reinterpret_cast<double*>(smem + kTcSmS);
-    for (int idx = tid; idx < 128 * 128; idx += kTcThreads) {
-      const int k = idx >> 7, n = idx & 127;
-      Sd[((k & 15) * 8 + (k >> 4)) * kFixSdStride + n] = (double)__ldg(a.S + idx);
-    }
-    __syncthreads();
-    for (int i = 0; i < kTcSlots; ++i) fix_process(queues + i, tid, kTcThreads, a.K, a.V, a.in_dtype, a.S, Sd, *a.tables, a.status);
+    // shared memory go away
+    for (int i = 0; i < (1 << 16) && !tc_mbar_try(bar_xfull + 8 * tid, (copies_issued[tid] - 1) & 1); ++i) __nanosleep(64);
   }
   __syncthreads();
   if (warp == 1) {

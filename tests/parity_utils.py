@@ -44,11 +44,23 @@ def assert_codes_match(rep):
         f"{rep['inside']} of {rep['total']} codes differ inside the window"
 
 
-def assert_radii_match(gpu_radii: np.ndarray, want16: np.ndarray, max_ulp_fraction=5e-3):
-    """fp16 radii: equal, except that the float32-accurate norm of the fast encoder (relative error
-    ~1e-6 against an fp16 spacing of ~7e-4) may round to the neighbouring fp16 value on ~0.2 % of radii."""
-    g = gpu_radii.astype(np.float16).view(np.uint16).astype(np.int32)
-    w = want16.astype(np.float16).view(np.uint16).astype(np.int32)
+MAX_RADIUS_ULP_FRACTION = 2.5e-3  # of radii one fp16 ulp off (measured: 0.9e-3 tensor-core encoder, 0.2e-3 the others)
+
+
+def radii_ulp_report(gpu_radii: np.ndarray, want16: np.ndarray):
+    """(radii that differ from the oracle's fp16 value, radii compared); a difference of more than one fp16
+    ulp fails at once."""
+    g = np.asarray(gpu_radii).astype(np.float16).view(np.uint16).astype(np.int32)
+    w = np.asarray(want16).astype(np.float16).view(np.uint16).astype(np.int32)
     delta = np.abs(g - w)
     assert delta.max() <= 1, f"radius differs by {delta.max()} fp16 ulps"
-    assert np.count_nonzero(delta) <= max_ulp_fraction * delta.size + 1
+    return int(np.count_nonzero(delta)), int(delta.size)
+
+
+def assert_radii_match(gpu_radii: np.ndarray = None, want16: np.ndarray = None, counts=None):
+    """fp16 radii equal the oracle's single rounding of the float64 block norm, except that the encoder's
+    float32-accurate norm (relative error ~2e-7 against an fp16 spacing of 5e-4 .. 1e-3) lands on the neighbouring
+    fp16 value for a small fraction of them.  `counts` = (off by one, compared) summed by the caller over many small
+    samples (a sample of a few hundred radii cannot be held to a fraction of 1e-3 by itself)."""
+    off, n = counts if counts is not None else radii_ulp_report(gpu_radii, want16)
+    assert off <= MAX_RADIUS_ULP_FRACTION * n + 3, f"{off} of {n} radii are one fp16 ulp off"

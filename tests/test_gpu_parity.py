@@ -10,6 +10,7 @@ import paper_2502_02617_b200 as pq
 from paper_2502_02617_b200 import synthetic
 from oracle import polarquant_oracle as orc
 from parity_utils import (TOL_ATTENTION, TOL_DECODED, assert_codes_match, assert_radii_match, code_mismatch_report,
+                          radii_ulp_report,
                           oracle_codebooks, rel_l2, to_f64)
 
 pytestmark = pytest.mark.gpu
@@ -30,16 +31,19 @@ def _encode_and_compare(cache, K, V, lens_list, start=None):
     codes, radii = codes.cpu().numpy(), radii.cpu().numpy()
     Kc, Vc = to_f64(K), to_f64(V)
     total = dict(total=0, inside=0, outside=0)
+    radii_off = radii_n = 0
     row = 0
     for b, n in enumerate(lens_list):
         for kv, X in ((0, Kc), (1, Vc)):
             for h in range(cache.n_kv_heads):
                 rep = code_mismatch_report(codes[b, h, kv, start[b]:start[b] + n], X[row:row + n, h], S, cb)
-                assert_radii_match(radii[b, h, kv, start[b]:start[b] + n], rep["radii16"])
+                off, cnt = radii_ulp_report(radii[b, h, kv, start[b]:start[b] + n], rep["radii16"])
+                radii_off, radii_n = radii_off + off, radii_n + cnt
                 for key in total:
                     total[key] += rep[key]
         row += n
     assert_codes_match(total)
+    assert_radii_match(counts=(radii_off, radii_n))
     return total
 
 
@@ -121,11 +125,14 @@ def test_chunked_prefill_and_append_equal_one_shot_and_oracle():
     assert two.lens.cpu().tolist() == lens_list
     c1, r1 = one.unpack(100)
     c2, r2 = two.unpack(100)
+    radii_off = radii_n = 0
     for b, n in enumerate(lens_list):
         assert torch.equal(c1[b, :, :, :n], c2[b, :, :, :n])  # codes do not depend on chunking or on the kernel used
         # radii come from float32-accurate norms whose last rounding may differ between the prefill and
         # the append kernel: equal, or one fp16 ulp apart on a small fraction
-        assert_radii_match(r1[b, :, :, :n].cpu().numpy(), r2[b, :, :, :n].cpu().numpy())
+        off, cnt = radii_ulp_report(r1[b, :, :, :n].cpu().numpy(), r2[b, :, :, :n].cpu().numpy())
+        radii_off, radii_n = radii_off + off, radii_n + cnt
+    assert_radii_match(counts=(radii_off, radii_n))
     q = synthetic.queries(12, B, Hq, d, torch.bfloat16, DEV)
     assert rel_l2(to_f64(two.attend(q)), to_f64(one.attend(q))) < 1e-3
 
