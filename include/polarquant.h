@@ -188,8 +188,9 @@ int32_t pq_decode_attention_static(int32_t head_dim, int32_t n_q_heads, int32_t 
 /*
  * Test support: make the next launch of one kernel run its give-up path.  `which` = 1 arms the
  * tensor-core encoder behind pq_encode_kv (head_dim 128, bf16, >= 128 rows), 2 arms the head_dim-128
- * kernel behind pq_decode_attention, 0 disarms.  In the armed launch the first bounded wait of CTA 0
- * is reported as failed although what it waited for arrived: the CTA abandons its share of the work,
+ * kernel behind pq_decode_attention, 0 disarms.  In the armed launch the first bounded wait of one CTA
+ * (the one that starts the first tile / the first non-empty sequence) is reported as failed although
+ * what it waited for arrived: the CTA abandons its share of the work,
  * waits for its copies in flight, releases what it holds and records PQ_ERR_TIMEOUT in status word 0;
  * nothing on the device is left waiting and the next call runs normally.  (The paper has no
  * counterpart: it exercises the error handling of Section "General rules" without losing a copy.)

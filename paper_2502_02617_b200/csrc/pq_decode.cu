@@ -1,5 +1,6 @@
 // Decode attention over the packed cache (Eq. 3) and the inspection kernels.
 #include <atomic>
+#include <chrono>
 #include <math_constants.h>
 
 #include "pq_common.cuh"
@@ -124,7 +125,8 @@ constexpr int kMaxGroup = 8;  // query heads per kv head handled by one CTA
 struct DecodeArgs {
   int d, n_q_heads, n_kv_heads, batch, capacity, io_dtype;
   float scale;
-  uint32_t epoch;  // differs from call to call (never 0): tags the split tickets of the persistent kernel
+  uint32_t epoch;  // differs from call to call (top bit set): tags the split tickets of the persistent kernel
+  uint32_t debug;  // bit 0: test hook, the first bounded wait of CTA 0 of the persistent kernel reports failure
   const float* S;
   const Tables* tables;
   const void* q;
@@ -379,6 +381,7 @@ __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel
   if (tid == 0) {
     const int t = atomicAdd(a.ws.tickets + b * a.n_kv_heads + hk, 1);
     is_last = (t == a.ws.n_splits - 1);
+    if (is_last) a.ws.tickets[b * a.n_kv_heads + hk] = 0;  // leave no small counts behind in scratch that other calls reuse
     if (is_last && len <= 0) set_status(a.status, PQ_ERR_EMPTY);
   }
   __syncthreads();
@@ -492,9 +495,17 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
   const int g = n_q_heads / n_kv_heads;
   if (head_dim == 128 && batch * n_kv_heads <= pq::kFastMaxUnits) {
     // One launch: the persistent kernel rotates the queries itself and needs no cleared tickets.
-    static std::atomic<uint32_t> call_epoch{0};
-    do a.epoch = call_epoch.fetch_add(1u, std::memory_order_relaxed) + 1u;
-    while (a.epoch == 0u);
+    // The tickets in the (uninitialised, possibly shared) scratch are tagged with a per-call number.  It starts
+    // at a value drawn from the clock and the address space of this process, advances by an odd constant and
+    // always has its top bit set, so it cannot equal a small integer that another kernel left in the same bytes.
+    static std::atomic<uint32_t> call_epoch{[] {
+      uint64_t x = (uint64_t)std::chrono::steady_clock::now().time_since_epoch().count() ^ (uint64_t)(uintptr_t)&pq_decode_attention;
+      x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+      x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+      return (uint32_t)(x ^ (x >> 31));
+    }()};
+    a.epoch = call_epoch.fetch_add(0x9E3779B1u, std::memory_order_relaxed) | 0x80000000u;
+    a.debug = pq::take_debug_wait_failure(2) ? 1u : 0u;
     static int configured4[pq::kMaxDevices] = {}, configured8[pq::kMaxDevices] = {};
     const int n_sm = g <= 4 ? pq::configure_for_device(pq::decode_attention_fast_kernel<1>, pq::kSmTotal, configured4)
                             : pq::configure_for_device(pq::decode_attention_fast_kernel<2>, pq::kSmTotal, configured8);
@@ -505,6 +516,7 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
     return pq::launch_status();
   }
   a.epoch = 0u;
+  a.debug = 0u;
   pq::rotate_query_kernel<<<batch * n_q_heads, head_dim, head_dim * sizeof(float), st>>>(a);
   const pq::Layout L = pq::make_layout(head_dim, capacity);
   size_t smem = 2 * L.block_bytes + sizeof(float) * ((size_t)g * head_dim + 3 * g * pq::kTokenBlock +

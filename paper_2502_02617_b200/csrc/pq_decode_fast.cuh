@@ -41,7 +41,7 @@ constexpr int kSmT1p = 0;                             // 256 * 16 * 8 = 32768
 constexpr int kSmT1lo = kSmT1p + 256 * 16 * 8;        // 32768
 constexpr int kSmU = kSmT1lo + 256 * 16 * 8;          // 4 * 64 * 16 * 8 = 32768
 constexpr int kSmBar = kSmU + 4 * 64 * 16 * 8;        // full[4], empty[4] : 64
-constexpr int kSmFlags = kSmBar + 64;                 // abort flag, is_last, n_segs : 16
+constexpr int kSmFlags = kSmBar + 64;                 // abort flag, is_last, n_segs, first_rank : 16
 constexpr int kSmSegs = kSmFlags + 16;                // Segment[32] : 768
 constexpr int kSmQ = kSmSegs + 768;                   // q (fp32) [8][128], q' fp16 value [8][128], q' fp16 residual [8][128] : 8192
 constexpr int kSmRing = (kSmQ + 8192 + 127) / 128 * 128;
@@ -261,7 +261,7 @@ __device__ inline void build_fast_tables(uint8_t* smem, const Tables* tb) {
 constexpr int kFastMaxGrid = 160;
 constexpr int kFastMaxUnits = 2048;  // (sequence, kv head) units the persistent schedule handles
 constexpr int kSegmentCost = 7;     // stages' worth of time a CTA spends on starting and finishing a unit
-constexpr int kFastMaxSegs = 32;     // units one CTA can take part in (<= units / grid + 2)
+constexpr int kFastMaxSegs = 16;     // units of one CTA that are listed at a time
 struct Segment {
   int unit, st0, st1, part, n_parts, slot0;
 };
@@ -293,63 +293,88 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
   // start of the next, and a unit may be shared by several CTAs (its "parts").  Starting on another
   // unit costs a CTA about kSegmentCost stages (query rotation, refilling the ring, the merge), so
   // every unit is preceded by that many empty positions on the line that is cut.  Each thread works
-  // out one unit; the units this CTA takes part in are collected in a short list.
+  // out one unit; the units this CTA takes part in are consecutive among the non-empty ones and are
+  // listed kFastMaxSegs at a time (a ragged batch -- one very long sequence and many short ones --
+  // can give a CTA more than that; the split is then worked out again for the next batch of the list,
+  // because its scratch lies in the ring).
   const int n_units = a.batch * a.n_kv_heads, G = gridDim.x, cta = blockIdx.x;
-  int* u_nst = reinterpret_cast<int*>(smem + kSmRing);  // [n_units] stages; the ring is idle during set-up
+  int* u_nst = reinterpret_cast<int*>(smem + kSmRing);  // [n_units] stages; the ring is idle while the split is worked out
   int* u_parts = u_nst + kFastMaxUnits;                 // [n_units] CTAs that share the unit
   Segment* segs = reinterpret_cast<Segment*>(smem + kSmSegs);
-  int* n_segs = reinterpret_cast<int*>(smem + kSmFlags) + 2;
-  if (tid == 0) *n_segs = 0;
-  for (int u = tid; u < n_units; u += kFastThreads) {
-    const int len_u = a.lens[u / a.n_kv_heads];
-    u_nst[u] = len_u > 0 ? (len_u + kStageTokens - 1) / kStageTokens : 0;
-  }
-  __syncthreads();
-  long long w_total = 0;
-  for (int u = 0; u < n_units; ++u) w_total += u_nst[u] > 0 ? u_nst[u] + kSegmentCost : 0;
-  const long long lo = cta * w_total / G, hi = (cta + 1) * w_total / G;
-  for (int u = tid; u < n_units; u += kFastThreads) {
-    int parts = 0;
-    if (u_nst[u] > 0) {
-      long long start = kSegmentCost;  // position of the unit's first stage
-      for (int v = 0; v < u; ++v) start += u_nst[v] > 0 ? u_nst[v] + kSegmentCost : 0;
-      const long long end = start + u_nst[u];
-      const int c_first = (int)(((start + 1) * G + w_total - 1) / w_total) - 1;  // CTA whose range holds stage `start`
-      const int c_last = (int)((end * G + w_total - 1) / w_total) - 1;           // ... stage `end - 1`
-      parts = c_last - c_first + 1;
-      if (cta >= c_first && cta <= c_last) {
-        const int i = atomicAdd(n_segs, 1);
-        if (i < kFastMaxSegs) {
-          segs[i].unit = u;
-          segs[i].st0 = (int)((lo > start ? lo : start) - start);
-          segs[i].st1 = (int)((hi < end ? hi : end) - start);  // > st0: the CTA's range holds a stage of the unit
-          segs[i].part = cta - c_first;
-          segs[i].n_parts = parts;
-        }
-      }
-    } else if (cta == 0) {  // empty sequence: zeros, and the status says so
-      const int b = u / a.n_kv_heads, hk = u - b * a.n_kv_heads;
-      for (int i = 0; i < g_heads * 128; ++i) {
-        const int64_t idx = ((int64_t)b * a.n_q_heads + hk * g_heads) * 128 + i;
-        if (a.io_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[idx] = __float2bfloat16(0.f);
-        else reinterpret_cast<float*>(a.out)[idx] = 0.f;
-      }
-      set_status(a.status, PQ_ERR_EMPTY);
+  int* n_segs = reinterpret_cast<int*>(smem + kSmFlags) + 2;   // units of this CTA (all batches of the list)
+  int* first_rank = reinterpret_cast<int*>(smem + kSmFlags) + 3;
+  // Fills `segs` with the CTA's units number kFastMaxSegs * batch_no .. (counted among the CTA's own) and returns how many
+  // units the CTA has in all.  Called by all threads.
+  auto build_segments = [&](int batch_no) -> int {
+    if (tid == 0) {
+      *n_segs = 0;
+      *first_rank = 0x7fffffff;
     }
-    u_parts[u] = parts;
-  }
-  __syncthreads();
-  if (*n_segs > kFastMaxSegs) {  // cannot happen for n_units <= kFastMaxUnits; never index past the list
-    if (tid == 0) set_status(a.status, PQ_ERR_UNSUPPORTED);
-    return;
-  }
-  for (int i = tid; i < *n_segs; i += kFastThreads) {  // first partial slot of the unit
-    int slot = 0;
-    for (int v = 0; v < segs[i].unit; ++v) slot += u_parts[v];
-    segs[i].slot0 = slot;
-  }
-  __syncthreads();
-  const int my_segs = *n_segs;
+    for (int u = tid; u < n_units; u += kFastThreads) {
+      const int len_u = a.lens[u / a.n_kv_heads];
+      u_nst[u] = len_u > 0 ? (len_u + kStageTokens - 1) / kStageTokens : 0;
+    }
+    __syncthreads();
+    long long w_total = 0;
+    for (int u = 0; u < n_units; ++u) w_total += u_nst[u] > 0 ? u_nst[u] + kSegmentCost : 0;
+    const long long lo = cta * w_total / G, hi = (cta + 1) * w_total / G;
+    // pass 1: parts of every unit; rank (among non-empty units) of the first unit of this CTA
+    for (int u = tid; u < n_units; u += kFastThreads) {
+      int parts = 0;
+      if (u_nst[u] > 0) {
+        long long start = kSegmentCost;  // position of the unit's first stage
+        int rank = 0;
+        for (int v = 0; v < u; ++v) {
+          start += u_nst[v] > 0 ? u_nst[v] + kSegmentCost : 0;
+          rank += u_nst[v] > 0;
+        }
+        const long long end = start + u_nst[u];
+        const int c_first = (int)(((start + 1) * G + w_total - 1) / w_total) - 1;  // CTA whose range holds stage `start`
+        const int c_last = (int)((end * G + w_total - 1) / w_total) - 1;           // ... stage `end - 1`
+        parts = c_last - c_first + 1;
+        if (cta >= c_first && cta <= c_last) {
+          atomicAdd(n_segs, 1);
+          atomicMin(first_rank, rank);
+        }
+      } else if (cta == 0 && batch_no == 0) {  // empty sequence: zeros, and the status says so
+        const int b = u / a.n_kv_heads, hk = u - b * a.n_kv_heads;
+        for (int i = 0; i < g_heads * 128; ++i) {
+          const int64_t idx = ((int64_t)b * a.n_q_heads + hk * g_heads) * 128 + i;
+          if (a.io_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[idx] = __float2bfloat16(0.f);
+          else reinterpret_cast<float*>(a.out)[idx] = 0.f;
+        }
+        set_status(a.status, PQ_ERR_EMPTY);
+      }
+      u_parts[u] = parts;
+    }
+    __syncthreads();
+    const int r0 = *first_rank + batch_no * kFastMaxSegs;  // this batch: ranks r0 .. r0 + kFastMaxSegs - 1
+    // pass 2: the units of this batch, in unit order
+    for (int u = tid; u < n_units; u += kFastThreads) {
+      if (u_nst[u] == 0) continue;
+      long long start = kSegmentCost;
+      int rank = 0, slot = 0;
+      for (int v = 0; v < u; ++v) {
+        start += u_nst[v] > 0 ? u_nst[v] + kSegmentCost : 0;
+        rank += u_nst[v] > 0;
+        slot += u_parts[v];
+      }
+      const long long end = start + u_nst[u];
+      const int c_first = (int)(((start + 1) * G + w_total - 1) / w_total) - 1;
+      const int c_last = (int)((end * G + w_total - 1) / w_total) - 1;
+      if (cta >= c_first && cta <= c_last && rank >= r0 && rank < r0 + kFastMaxSegs) {
+        Segment& sgm = segs[rank - r0];
+        sgm.unit = u;
+        sgm.st0 = (int)((lo > start ? lo : start) - start);
+        sgm.st1 = (int)((hi < end ? hi : end) - start);  // > st0: the CTA's range holds a stage of the unit
+        sgm.part = cta - c_first;
+        sgm.n_parts = u_parts[u];
+        sgm.slot0 = slot;  // first partial slot of the unit
+      }
+    }
+    __syncthreads();
+    return *n_segs;
+  };
   const int g = lane >> 2, c = lane & 3;
   const uint32_t rep = (lane & 15) * 8;
   const uint32_t ua = sm_base + kSmU + rep, t1a = sm_base + kSmT1p + rep;  // table base | lane replica
@@ -365,6 +390,10 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
   const uint32_t ov_c2 = kO2 + tk_v * 8 + (lane >> 2), ov_c3 = kO3 + tk_v * 4 + (lane >> 3), ov_c4 = kO4 + tk_v * 2;
   int gl0 = 0;               // stages this group has streamed so far (ring slot and barrier phase bookkeeping)
 
+  int my_units = build_segments(0);
+  for (int batch_no = 0; batch_no * kFastMaxSegs < my_units; ++batch_no) {
+  if (batch_no > 0) my_units = build_segments(batch_no);
+  const int my_segs = min(kFastMaxSegs, my_units - batch_no * kFastMaxSegs);
   for (int sg = 0; sg < my_segs; ++sg) {
     const int u = segs[sg].unit, st0 = segs[sg].st0, st1 = segs[sg].st1;
     const int n_parts = segs[sg].n_parts, unit_slot = segs[sg].slot0, c_first = cta - segs[sg].part;
@@ -408,7 +437,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     __syncwarp();
     // The lookup tables are filled once, with the CTA's first copies already on their way (the barriers
     // of the query rotation below order the fill before the first lookup).
-    if (sg == 0) build_fast_tables(smem, a.tables);
+    if (sg == 0 && batch_no == 0) build_fast_tables(smem, a.tables);
     // q' = (q S) * scale * log2(e) for the unit's query heads, as an fp16 value plus an fp16 residual.
     // The first stages of the segment are already on their way while this runs.
     {
@@ -456,6 +485,11 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
       if (producer && li + 1 < n_li) issue_copy(li + 1);
       __syncwarp();
       if (!mbar_wait(sm_base + kSmBar + 8 * s, (gl >> 1) & 1, abort_flag)) break;
+      if ((a.debug & 1u) && unit_slot == 0 && cta == c_first && li == 0 && warp == 0) {  // test hook: the first wait of the CTA
+        // that starts the first non-empty unit is reported as failed
+        *abort_flag = 1;
+        break;
+      }
       const int tile_tok0 = st * kStageTokens + (warp & 7) * 16;  // first token of this warp's 16-token tile
       if (tile_tok0 < len) {
         const uint32_t kblk = sm_base + kSmRing + s * kStageBytes + ((warp >> 2) & 1) * 2 * kBlockBytes128;
@@ -688,6 +722,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
       combine_and_store(a, b, hk, g_heads, unit_slot, n_parts, reinterpret_cast<float*>(smem + kSmRing));
     }
     __syncthreads();  // the ring is free again for the next unit
+  }
   }
   if (tid == 0 && *abort_flag) set_status(a.status, PQ_ERR_TIMEOUT);
 }

@@ -201,16 +201,66 @@ def test_capacity_overflow_and_empty_sequence_are_reported_not_faulted():
     assert cache.status.cpu().tolist()[0] == pq.ERR_CAPACITY and cache.lens.cpu().tolist() == [64, 11]
 
 
-def test_nonfinite_inputs_are_counted():
+@pytest.mark.parametrize("n", [8, 40, 300])
+def test_nonfinite_inputs_are_counted(n):
+    """8 rows go through the per-vector kernel, 40 through the float32-FMA kernel, 300 through the tensor-core
+    kernel: each records the error and counts the non-finite input elements; the other rows are encoded as usual."""
     d = 128
-    cache = pq.PolarQuantCache(1, 1, 1, d, capacity=64, seed=8, device=DEV)
-    K, V = synthetic.kv_like(51, 8, 1, d, torch.bfloat16, DEV)
+    cache = pq.PolarQuantCache(1, 2, 2, d, capacity=n, seed=8, device=DEV)
+    K, V = synthetic.kv_like(51, n, 2, d, torch.bfloat16, DEV)
     K[3, 0, 5] = float("nan")
-    V[4, 0, 6] = float("inf")
-    cache.encode(K, V, torch.tensor([0, 8], dtype=torch.int32, device=DEV))
+    V[n - 4, 1, 6] = float("inf")
+    V[n - 4, 1, 7] = float("-inf")
+    cache.encode(K, V, torch.tensor([0, n], dtype=torch.int32, device=DEV))
     torch.cuda.synchronize()
     st = cache.status.cpu().tolist()
-    assert st[0] == pq.ERR_NONFINITE and st[1] == 2
+    assert st[0] == pq.ERR_NONFINITE and st[1] == 3
+    codes, _ = cache.unpack(n)
+    cb, S = oracle_codebooks(cache), cache.S_host.double().numpy()
+    keep = np.array([t for t in range(n) if t not in (3, n - 4)])
+    for kv, X in ((0, K), (1, V)):
+        for h in range(2):
+            rep = code_mismatch_report(codes[0, h, kv].cpu().numpy()[keep], to_f64(X[:, h])[keep], S, cb)
+            assert_codes_match(rep)
+
+
+def test_wait_that_gives_up_in_the_encoder_is_reported_and_the_next_call_is_clean():
+    """The armed launch treats the first bounded wait of its CTA 0 as failed (the copy it waited for did arrive):
+    that CTA abandons its tiles, lets its copies land, releases tensor memory and records PQ_ERR_TIMEOUT.  Nothing
+    is left waiting on the device, and the same call repeated afterwards encodes everything."""
+    d, Hkv, n = 128, 2, 1024
+    cache = pq.PolarQuantCache(1, 2, Hkv, d, capacity=n, seed=3, device=DEV)
+    K, V = synthetic.kv_like(5, n, Hkv, d, torch.bfloat16, DEV)
+    cu = torch.tensor([0, n], dtype=torch.int32, device=DEV)
+    pq.pq_debug_fail_next_wait(1)
+    cache.encode(K, V, cu)
+    torch.cuda.synchronize()
+    assert cache.status.cpu().tolist()[0] == pq.ERR_TIMEOUT
+    cache.status.zero_()
+    cache.lens.zero_()
+    _encode_and_compare(cache, K, V, [n])   # the hook is disarmed: a normal call, checked against the oracle
+    pq.pq_debug_fail_next_wait(0)
+
+
+def test_wait_that_gives_up_in_decode_attention_is_reported_and_the_next_call_is_clean():
+    d, Hq, Hkv, n = 128, 8, 2, 3000
+    cache = pq.PolarQuantCache(1, Hq, Hkv, d, capacity=n, seed=4, device=DEV)
+    K, V = synthetic.kv_like(6, n, Hkv, d, torch.bfloat16, DEV)
+    cache.encode(K, V, torch.tensor([0, n], dtype=torch.int32, device=DEV))
+    q = synthetic.queries(7, 1, Hq, d, torch.bfloat16, DEV)
+    want = cache.attend(q)
+    torch.cuda.synchronize()
+    cache.check_status()
+    pq.pq_debug_fail_next_wait(2)
+    cache.attend(q)
+    torch.cuda.synchronize()
+    assert cache.status.cpu().tolist()[0] == pq.ERR_TIMEOUT
+    cache.status.zero_()
+    got = cache.attend(q)
+    torch.cuda.synchronize()
+    cache.check_status()
+    assert torch.equal(got, want)
+    pq.pq_debug_fail_next_wait(0)
 
 
 def test_mid_size_llama_shape_codes_with_window_accounting():

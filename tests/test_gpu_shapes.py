@@ -61,6 +61,39 @@ def test_random_shapes_against_oracle(seed):
             assert rel_l2(got, want) < TOL_F32_IO, (seed, trial, B, Hq, Hkv, b, hk, n)
 
 
+def test_one_long_sequence_and_many_short_ones():
+    """A ragged batch in which the equal-cost split hands single CTAs more (sequence, kv head) units than they list
+    at a time: one sequence of 61 000 tokens and 255 of 100 tokens, 8 kv heads (2048 units; the CTAs that hold only
+    short units take about 17 each).  Outputs of sampled short units, of the units next to the long sequence and
+    of the long sequence itself are compared with the oracle."""
+    B, Hkv, Hq, d, long_len, short_len = 256, 8, 8, 128, 61000, 100
+    lens = [short_len] * B
+    lens[37] = long_len
+    cache = pq.PolarQuantCache(B, Hq, Hkv, d, capacity=long_len, seed=77, device=DEV)
+    K, V = synthetic.kv_like(78, sum(lens), Hkv, d, torch.bfloat16, DEV)
+    cu = torch.tensor(np.concatenate(([0], np.cumsum(lens))), dtype=torch.int32, device=DEV)
+    cache.encode(K, V, cu)
+    q = synthetic.queries(79, B, Hq, d, torch.float32, DEV)
+    out = cache.attend(q)
+    again = cache.attend(q)
+    torch.cuda.synchronize()
+    cache.check_status()
+    assert torch.equal(out, again)
+    cb, S = oracle_codebooks(cache), cache.S_host.double().numpy()
+    rng = np.random.default_rng(5)
+    units = [(37, 0), (37, 7), (36, 7), (38, 0), (0, 0), (255, 7)] + [(int(rng.integers(B)), int(rng.integers(Hkv))) for _ in range(40)]
+    for b, hk in units:
+        n = lens[b]
+        codes, radii = pq.pq_unpack_codes(d, Hkv, cache.cache[b * (cache.cache.numel() // B):(b + 1) * (cache.cache.numel() // B)],
+                                          1, cache.capacity, n)
+        c, r = codes[0, hk].cpu().numpy(), radii[0, hk].cpu().numpy()
+        want = orc.decode_attention(to_f64(q[b, hk:hk + 1])[None], c[0][None, None], r[0][None, None], c[1][None, None],
+                                    r[1][None, None], [n], cb, S, d ** -0.5)[0]
+        assert rel_l2(to_f64(out[b, hk:hk + 1]), want) < TOL_F32_IO, (b, hk)
+    # every short unit was written: none of the outputs is left at the fill value
+    assert torch.isfinite(out).all() and (out.abs().amax(dim=(1, 2)) > 0).all()
+
+
 @pytest.mark.parametrize("seed", [21, 22])
 def test_random_encode_chunks_against_oracle(seed):
     """Encoder on randomly drawn chunk patterns: every sequence receives 1-4 chunks whose row counts sit around

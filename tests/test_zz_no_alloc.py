@@ -39,6 +39,30 @@ def test_static_scratch_entry_matches_workspace_entry_twice_in_a_row(d, Hq, Hkv,
         assert torch.equal(got, want)  # same kernels, same split order: bit-identical
 
 
+def test_static_scratch_entry_after_a_call_of_the_other_kernel_family():
+    """The head_dim-16 path counts its splits with small integers in the shared array; the head_dim-128 path that
+    runs next on the same bytes (units shared by several CTAs) must not take them for arrivals of its own call.  Device
+    memory in use is the same before and after: the entry allocates nothing."""
+    small = _filled_cache(16, 2, 1, [100, 37], seed=62)
+    big = _filled_cache(128, 8, 2, [9000, 5000], seed=63)   # few units, many CTAs per unit
+    q16 = synthetic.queries(80, 2, 2, 16, torch.bfloat16, DEV)
+    q128 = synthetic.queries(81, 2, 8, 128, torch.bfloat16, DEV)
+    want = big.attend(q128)
+    got16, got = torch.empty_like(q16), torch.empty_like(q128)
+    torch.cuda.synchronize()
+    free_before, allocated_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
+    for _ in range(2):
+        pq.pq_decode_attention_static(small.S, small.tables, q16, small.cache, small.lens, 1, small.capacity,
+                                      small.capacity, 0.25, got16, small.status)
+        pq.pq_decode_attention_static(big.S, big.tables, q128, big.cache, big.lens, 2, big.capacity, big.capacity,
+                                      128 ** -0.5, got, big.status)
+        torch.cuda.synchronize()
+        big.check_status()
+        small.check_status()
+        assert torch.equal(got, want)
+    assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_allocated() == allocated_before
+
+
 def test_static_scratch_entry_rejects_oversized_problems_without_launching():
     d, Hq, Hkv, B, ctx = 128, 64, 8, 256, 1 << 20
     assert pq.pq_workspace_bytes(d, B, Hq, Hkv, ctx) > pq.pq_static_scratch_bytes()
