@@ -10,8 +10,14 @@
  *   - Every function returns an int32 status: PQ_OK (0) or a negative PQ_ERR_* value.
  *     Nothing throws, aborts or traps.
  *   - "host" pointers are ordinary CPU memory, "dev" pointers are CUDA device memory of
- *     the current device.  The library allocates no device memory and keeps no state;
- *     every buffer belongs to the caller.  Device pointers must be 16-byte aligned.
+ *     the current device.  The library allocates no device memory; every buffer belongs to
+ *     the caller.  Device pointers must be 16-byte aligned.
+ *   - State the library keeps, all of it per process: a call counter that tags the scratch of
+ *     pq_decode_attention, a per-device note of which kernels have been configured (and, for
+ *     pq_decode_attention_static, the device address of its built-in array, which every GPU
+ *     that loads the library carries), the last CUDA error of each host thread, and the test
+ *     hook of pq_debug_fail_next_wait.  All of it is updated atomically: host threads may call
+ *     into the library concurrently as long as they do not share output buffers or scratch.
  *   - Device work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
  *     legacy default stream) and the call returns without synchronising.
  *   - Problems that only the device can see (a sequence that would exceed `capacity`,
@@ -173,9 +179,11 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
  *   - The first call on each device looks up the device address of the array (a host-side query,
  *     no allocation); make that first call outside any stream capture.
  *   - Never calls cudaMalloc, cudaFree or any allocating routine.
- *   - All calls on a device share the one array.  It keeps the previous call's contents; the part
- *     that must start at zero (the split tickets) is cleared by the call's own first kernel.
- *     Calls that may overlap on the GPU (different streams, no ordering) race on it: order them.
+ *   - All calls on a device share the one array.  It keeps the previous call's contents; nothing in
+ *     it has to start at zero: the head_dim-128 kernel tags its split counters with the call's
+ *     number and ignores counters of other calls, the other head_dims clear theirs in the call's
+ *     first kernel.  Calls that may overlap on the GPU (different streams, no ordering) race on
+ *     it: order them.
  */
 #define PQ_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
 int64_t pq_static_scratch_bytes(void);

@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/polarquant.h"
 
 namespace pq {
@@ -172,10 +174,13 @@ inline int32_t launch_status() {
 // One-time, per-device launch configuration of a kernel that needs more than 48 KB of dynamic shared
 // memory: the attribute belongs to the (kernel, device) pair, so the memo is indexed by the current
 // device. `state` is a zero-initialised array the caller keeps per kernel; an entry holds the device's
-// SM count once the kernel is configured there. Returns the SM count, or 0 with the CUDA error noted.
+// SM count once the kernel is configured there (atomic: host threads may call into the library
+// concurrently; two that race on a device both set the same attribute). Returns the SM count, or 0 with
+// the CUDA error noted.
 constexpr int kMaxDevices = 64;
+using DeviceMemo = std::atomic<int>[kMaxDevices];
 template <typename Kernel>
-inline int configure_for_device(Kernel kernel, int smem_bytes, int (&state)[kMaxDevices]) {
+inline int configure_for_device(Kernel kernel, int smem_bytes, DeviceMemo& state) {
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e == cudaSuccess && (dev < 0 || dev >= kMaxDevices)) e = cudaErrorInvalidDevice;
@@ -183,7 +188,8 @@ inline int configure_for_device(Kernel kernel, int smem_bytes, int (&state)[kMax
     note_cuda_error(e);
     return 0;
   }
-  if (state[dev] > 0) return state[dev];
+  const int known = state[dev].load(std::memory_order_acquire);
+  if (known > 0) return known;
   int n_sm = 0;
   e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev);
   if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes);
@@ -192,7 +198,7 @@ inline int configure_for_device(Kernel kernel, int smem_bytes, int (&state)[kMax
     note_cuda_error(e);
     return 0;
   }
-  state[dev] = n_sm;
+  state[dev].store(n_sm, std::memory_order_release);
   return n_sm;
 }
 

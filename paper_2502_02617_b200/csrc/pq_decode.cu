@@ -506,7 +506,7 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
     }()};
     a.epoch = call_epoch.fetch_add(0x9E3779B1u, std::memory_order_relaxed) | 0x80000000u;
     a.debug = pq::take_debug_wait_failure(2) ? 1u : 0u;
-    static int configured4[pq::kMaxDevices] = {}, configured8[pq::kMaxDevices] = {};
+    static pq::DeviceMemo configured4, configured8;
     const int n_sm = g <= 4 ? pq::configure_for_device(pq::decode_attention_fast_kernel<1>, pq::kSmTotal, configured4)
                             : pq::configure_for_device(pq::decode_attention_fast_kernel<2>, pq::kSmTotal, configured8);
     if (n_sm == 0) return PQ_ERR_CUDA;
@@ -544,21 +544,21 @@ int32_t pq_decode_attention_static(int32_t head_dim, int32_t n_q_heads, int32_t 
   const int64_t need = pq_workspace_bytes(head_dim, batch, n_q_heads, n_kv_heads, max_len);
   if (need < 0) return (int32_t)need;
   if (need > PQ_STATIC_SCRATCH_BYTES) return PQ_ERR_SCRATCH;
-  static void* scratch_of_device[pq::kMaxDevices] = {};
+  static std::atomic<void*> scratch_of_device[pq::kMaxDevices];
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess || dev < 0 || dev >= pq::kMaxDevices) {
     pq::note_cuda_error(e == cudaSuccess ? cudaErrorInvalidDevice : e);
     return PQ_ERR_CUDA;
   }
-  void* scratch = scratch_of_device[dev];
+  void* scratch = scratch_of_device[dev].load(std::memory_order_acquire);
   if (scratch == nullptr) {  // first call on this device (which is current): resolve the symbol
     e = cudaGetSymbolAddress(&scratch, g_static_scratch);
     if (e != cudaSuccess || scratch == nullptr) {
       pq::note_cuda_error(e == cudaSuccess ? cudaErrorInvalidSymbol : e);
       return PQ_ERR_CUDA;
     }
-    scratch_of_device[dev] = scratch;
+    scratch_of_device[dev].store(scratch, std::memory_order_release);
   }
   return pq_decode_attention(head_dim, n_q_heads, n_kv_heads, S_dev, tables_dev, q_dev, io_dtype, cache_dev,
                              cache_lens_dev, batch, capacity, max_len, scale, out_dev, scratch, status_dev, stream);

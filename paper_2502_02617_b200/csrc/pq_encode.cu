@@ -471,7 +471,7 @@ static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
     return launch_status();
   }
   if (a.head_dim == 128 && a.total_tokens >= 32) {
-    static int configured[kMaxDevices] = {};
+    static DeviceMemo configured;
     if (configure_for_device(encode_ffma_kernel, kFfmaSmem, configured) == 0) return PQ_ERR_CUDA;
     dim3 grid((a.total_tokens + 127) / 128, a.n_kv_heads, 2);
     encode_ffma_kernel<<<grid, kFfmaThreads, kFfmaSmem, stream>>>(a);

@@ -442,16 +442,14 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
 static EncodeTiledFn get_encode_tiled() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
+  static const EncodeTiledFn fn = [] {  // looked up once per process (thread-safe initialisation)
     void* p = nullptr;
     cudaDriverEntryPointQueryResult qres;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(p);
-  }
+      return reinterpret_cast<EncodeTiledFn>(p);
+    return static_cast<EncodeTiledFn>(nullptr);
+  }();
   return fn;
 }
 
@@ -478,7 +476,7 @@ static int32_t try_launch_encode_tc(const EncodeArgs& a, cudaStream_t stream) {
   TcMaps maps;
   if (!make_x_map(fn, &maps.k, a.K, a.n_kv_heads, a.total_tokens, a.token_stride, a.head_stride)) return 0;
   if (!make_x_map(fn, &maps.v, a.V, a.n_kv_heads, a.total_tokens, a.token_stride, a.head_stride)) return 0;
-  static int configured[kMaxDevices] = {};
+  static DeviceMemo configured;
   const int n_sm = configure_for_device(encode_tc_kernel, kTcSmTotal, configured);
   if (n_sm == 0) return PQ_ERR_CUDA;
   const int n_row_tiles = (a.total_tokens + 127) / 128;

@@ -79,6 +79,32 @@ def test_config2_and_config3_full_size():
     assert torch.equal(out, again)
 
 
+def test_config2_every_code_against_the_oracle():
+    """All 62.9 M codes and 4.2 M radii of one full config-2 encode (32768 tokens x 8 kv heads x K, V): none may
+    differ outside the 1e-6 rad window around a boundary, fewer than 1e-5 of them inside it."""
+    n = 32768
+    cache = pq.PolarQuantCache(1, HQ, HKV, D, capacity=n, seed=1, device=DEV)
+    K, V = synthetic.kv_like(1, n, HKV, D, torch.bfloat16, DEV)
+    cache.encode(K, V, torch.tensor([0, n], dtype=torch.int32, device=DEV))
+    torch.cuda.synchronize()
+    cache.check_status()
+    codes, radii = cache.unpack(n)
+    cb, S = oracle_codebooks(cache), cache.S_host.double().numpy()
+    total = dict(total=0, inside=0, outside=0)
+    radii_off = radii_n = 0
+    for kv, X in ((0, K), (1, V)):
+        for h in range(HKV):
+            rep = code_mismatch_report(codes[0, h, kv].cpu().numpy(), to_f64(X[:, h]), S, cb)
+            off, cnt = radii_ulp_report(radii[0, h, kv].cpu().numpy(), rep["radii16"])
+            radii_off, radii_n = radii_off + off, radii_n + cnt
+            for key in total:
+                total[key] += rep[key]
+    print(f"config 2, all codes: {total}; radii one fp16 ulp off: {radii_off} of {radii_n}")
+    assert total["total"] == 2 * HKV * n * 120
+    assert total["outside"] == 0 and total["inside"] < 1e-5 * total["total"]
+    assert_radii_match(counts=(radii_off, radii_n))
+
+
 def test_config4_long_context_layer():
     """One layer of the long-context shape: batch 1, 131072 tokens, 32 q / 8 kv heads."""
     n = 131072

@@ -158,12 +158,45 @@ def test_codebook_minimises_eq4_and_is_unique(cb, level):
     assert np.allclose(skew, theta, atol=1e-12)
 
 
+def test_codebooks_match_the_tabulated_multiprecision_values(cb):
+    """Centroids, outer boundaries and Eq. 4 cost of levels 2-4 against values tabulated from an independent
+    40-digit computation (tests/golden/codebooks_levels_2_to_4.txt)."""
+    rows = [ln.split() for ln in (GOLDEN / "codebooks_levels_2_to_4.txt").read_text().splitlines()
+            if ln and not ln.startswith("#")]
+    assert [int(r[0]) for r in rows] == [2, 3, 4]
+    for r in rows:
+        level, vals = int(r[0]), [float(v) for v in r[1:]]
+        c, b = cb.centroids[level - 1], cb.boundaries[level - 1]
+        assert np.allclose(c, vals[0:4], atol=1e-11, rtol=0)
+        assert abs(b[0] - vals[4]) < 1e-11 and abs(b[1] - math.pi / 4) < 1e-13 and abs(b[2] - vals[5]) < 1e-11
+        edges = np.concatenate(([0.0], b, [math.pi / 2]))
+        k = 2 ** (level - 1)  # Lemma 2: Gamma(k) / (2^(k-2) Gamma(k/2)^2) sin^(k-1)(2 psi)
+        const = math.gamma(k) / (2.0 ** (k - 2) * math.gamma(k / 2) ** 2)
+        mse = sum(integrate.quad(lambda p: (p - c[i]) ** 2 * const * math.sin(2 * p) ** (k - 1), edges[i], edges[i + 1],
+                                 epsabs=1e-14)[0] for i in range(4))
+        assert abs(mse - vals[6]) < 2e-11
+
+
 def test_level1_cost_closed_form(cb):
     # uniform density, 16 equal cells of width pi/8: mean squared error (pi/8)^2 / 12
     c = cb.centroids[0]
     b = np.concatenate(([0.0], cb.boundaries[0], [2 * math.pi]))
     mse = sum(integrate.quad(lambda p: (p - c[i]) ** 2 / (2 * math.pi), b[i], b[i + 1])[0] for i in range(16))
     assert abs(mse - (math.pi / 8) ** 2 / 12) < 1e-14
+
+
+# ---------------------------------------------------------------- radii (b_FPN = 16)
+def test_radius_rounding_is_round_to_nearest_even_and_saturates():
+    """binary16 spacing in [1, 2) is 2^-10: a value 3/4 of the way up rounds up (truncation would not), exact ties
+    go to the even significand, 65504 is the largest finite value; anything above it saturates and is counted."""
+    ulp = 2.0 ** -10
+    r16, sat = orc.round_radii_fp16(np.array([1 + 0.75 * ulp, 1 + 0.5 * ulp, 1 + 1.5 * ulp, 1 + 0.25 * ulp, 2048.0 + 1.0,
+                                              2048.0 + 3.0, 65504.0, 0.0]))
+    assert sat == 0
+    assert r16.dtype == np.float16
+    assert r16.astype(np.float64).tolist() == [1 + ulp, 1.0, 1 + 2 * ulp, 1.0, 2048.0, 2052.0, 65504.0, 0.0]
+    r16, sat = orc.round_radii_fp16(np.array([70000.0, 65504.0, 65519.0, 1e9, 3.0]))
+    assert sat == 3 and r16.astype(np.float64).tolist() == [65504.0, 65504.0, 65504.0, 65504.0, 3.0]
 
 
 # ---------------------------------------------------------------- Quant
@@ -337,6 +370,26 @@ def test_attention_equals_rotated_basis_evaluation_and_gqa_mapping(cb):
             s = yk @ (q[b, h] @ S) * 0.25  # <q, y S^T> = <q S, y>
             p = special.softmax(s)
             assert np.allclose(out[b, h], (p @ yv) @ S.T, atol=1e-13)
+
+
+def test_exact_attention_special_cases_and_brute_force():
+    """Eq. 2 on the unquantised cache (reported as information only): one token returns its value, identical keys
+    average the values, and a small case equals the definition written out with Python loops."""
+    rng = np.random.default_rng(3)
+    B, Hq, Hkv, n, d = 2, 4, 2, 5, 8
+    K, V, q = rng.normal(size=(B, Hkv, n, d)), rng.normal(size=(B, Hkv, n, d)), rng.normal(size=(B, Hq, d))
+    one = orc.exact_attention(q, K, V, [1, 1], 0.3)
+    for h in range(Hq):
+        assert np.allclose(one[:, h], V[:, h // 2, 0], atol=1e-15)
+    same = orc.exact_attention(q, np.repeat(K[:, :, :1], n, axis=2), V, [n, n], 0.3)
+    for h in range(Hq):
+        assert np.allclose(same[:, h], V[:, h // 2].mean(axis=1), atol=1e-14)
+    got = orc.exact_attention(q, K, V, [n, 3], 0.3)
+    for b, nb in enumerate([n, 3]):
+        for h in range(Hq):
+            w = [math.exp(0.3 * sum(q[b, h, i] * K[b, h // 2, t, i] for i in range(d))) for t in range(nb)]
+            want = [sum(w[t] * V[b, h // 2, t, i] for t in range(nb)) / sum(w) for i in range(d)]
+            assert np.allclose(got[b, h], want, atol=1e-13)
 
 
 def test_attention_without_quantisation_does_not_depend_on_S():
