@@ -1,15 +1,19 @@
 #!/usr/bin/env python
 """Benchmark of the PolarQuant hot path on B200.
 
-One step = one pass of the whole path on synthetic Llama-3.1-8B-shaped data:
-  (1) pq_encode_kv   : a prefill chunk of 32768 tokens x 8 KV heads x d=128, bf16 K and V
-                       (re-encodes one sequence of the resident batch),
+One pass = the whole path once on synthetic Llama-3.1-8B-shaped data:
+  (1) pq_encode_kv   : a prefill chunk of 32768 tokens x 8 KV heads x d=128, bf16 K and V (config 2; it
+                       re-encodes one sequence of a resident batch),
   (2) pq_append_kv   : one new token for each of the 8 sequences,
-  (3) pq_decode_attention : 32 query heads / 8 KV heads over batch 8 x ~32769 cached tokens.
-The headline `value` is the decode-attention throughput on compressed bytes (62 B per token per
-KV head for K and again for V), from CUDA events around call (3); the encoder's tokens/s and the
-whole-step time are reported beside it.  With --gpus N every rank runs the same per-GPU workload
-on its own sequences (no data-path collective; weak scaling) and the slowest rank's time counts.
+  (3) pq_decode_attention : 32 query heads / 8 KV heads over batch 8 x ~32769 cached tokens (config 3).
+Two resident caches alternate: a pass writes (1), (2) into one and reads (3) from the other, so that the
+decode never finds in L2 what the encoder of the same pass just wrote.  A step is `inner` consecutive
+passes (chosen so that the timed region lasts about two seconds; see `config.inner`); times are per pass.
+The headline `value` is the decode-attention throughput on compressed bytes (62 B per token per KV head
+for K and again for V), from CUDA events around call (3); the encoder's tokens/s, the long-context step
+(config 4: 36 layers x 131072 tokens) and the streaming loop (config 5: ragged batch 16, 128 steps) are
+reported beside it.  With --gpus N every rank runs the same per-GPU workload on its own sequences (no
+data-path collective; weak scaling) and the slowest rank's time counts.
 
 `--impl reference` times the float64 CPU oracle on a bounded sample of the same workload.
 """
@@ -17,6 +21,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -33,10 +38,13 @@ import torch
 
 D, HQ, HKV, BATCH, CTX = 128, 32, 8, 8, 32768
 BYTES_PER_TOKEN_HEAD = 124  # 62 B of K + 62 B of V
+ENCODE_BYTES_PER_VECTOR = 256 + 62
 METRIC = "decode_attention_compressed_kv_throughput"
 UNIT = "GB/s"
 WORKLOAD = ("decode attention: batch 8 x ctx 32768, 32 q / 8 kv heads, d=128 (config 3); encode chunk 32768 tokens x "
             "8 kv heads (config 2); append 1 token/sequence")
+TARGET_REGION_S = 2.2
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "decode_attention_fast_kernel_batch4_ctx32768.json")
 
 
 def _peaks():
@@ -45,6 +53,17 @@ def _peaks():
         with open(path) as f:
             return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     return 6650.0, "fallback (earlier pool measurement)"
+
+
+def _decode_traffic(batch):
+    """DRAM bytes of one decode-attention launch, from the ncu capture recorded beside the profile summary
+    (taken at a smaller batch; the traffic is proportional to the batch)."""
+    try:
+        with open(TRAFFIC_FILE) as f:
+            t = json.load(f)
+        return (t["dram_bytes_read"] + t["dram_bytes_write"]) * batch / t["batch"]
+    except (OSError, KeyError, ValueError):
+        return None
 
 
 _POLLER = r"""
@@ -87,7 +106,7 @@ class ClockSampler:
             self.proc = None
 
     def stop(self, t_begin=None, t_end=None):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "samples_under_load": 0}
         if self.proc is None:
             return out
         self.proc.terminate()
@@ -112,19 +131,25 @@ class ClockSampler:
         except (OSError, ValueError):
             pass
         if sm:
-            out.update(sm_mhz=float(statistics.median(sm)), sm_max_mhz=float(smax), samples=len(sm),
+            out.update(sm_mhz=float(statistics.median(sm)), sm_min_mhz=float(min(sm)), sm_max_mhz=float(smax),
+                       samples=len(sm), samples_under_load=len(sm),
                        reasons=sorted(n for bit, n in self.REASONS.items() if bits & bit))
         return out
 
 
-def _dist_setup(n_gpus):
+def dist_setup(backend="nccl"):
+    """(dist or None, rank, world, local_rank) from the torchrun environment."""
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if world > 1:
         import torch.distributed as dist
-        torch.cuda.set_device(local_rank)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        if not dist.is_initialized():
+            if backend == "nccl":
+                torch.cuda.set_device(local_rank)
+                dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+            else:
+                dist.init_process_group(backend)
         return dist, rank, world, local_rank
     return None, 0, 1, 0
 
@@ -187,84 +212,91 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def _oracle_match(cache, K_chunk, V_chunk, b_enc, q, out):
-    """Sampled parity at the benchmark's full size: codes of sampled vectors of the chunk just
-    encoded, and the attention output of two (sequence, kv head) units."""
+def _oracle_setup(cache):
     from oracle import polarquant_oracle as orc
-    rng = np.random.default_rng(0)
     cb = orc.codebooks_from_arrays((4, 2, 2, 2), cache.centroids.numpy(), cache.boundaries.numpy())
-    S = cache.S_host.double().numpy()
-    n_tok = CTX + 1
-    codes, radii = cache.unpack(n_tok)
+    return orc, cb, cache.S_host.double().numpy()
+
+
+def _attention_unit_error(pq, cache, cache_buf, batch, capacity, lens, q, out, b, hk):
+    """Relative L2 error of one (sequence, kv head) unit of `out` against the oracle run on the codes that the GPU
+    stored in `cache_buf` (a packed cache of `batch` sequences with room for `capacity` tokens each)."""
+    orc, cb, S = _oracle_setup(cache)
+    n = int(lens[b])
+    per_seq = cache_buf.numel() // batch
+    codes, radii = pq.pq_unpack_codes(D, HKV, cache_buf[b * per_seq:(b + 1) * per_seq], 1, capacity, n)
+    c, r = codes[0, hk].cpu().numpy(), radii[0, hk].cpu().numpy()
+    g = HQ // HKV
+    qq = q[b, hk * g:(hk + 1) * g].float().cpu().double().numpy()[None]
+    want = orc.decode_attention(qq, c[0][None, None], r[0][None, None], c[1][None, None], r[1][None, None], [n], cb, S,
+                                D ** -0.5)[0]
+    got = out[b, hk * g:(hk + 1) * g].float().cpu().double().numpy()
+    return float(np.linalg.norm(got - want) / np.linalg.norm(want))
+
+
+def _oracle_match(pq, cache, enc_buf, b_enc, K_chunk, V_chunk, dec_buf, dec_lens, q, out, units):
+    """Sampled parity at the benchmark's full size: codes of sampled vectors of the chunk just encoded as sequence
+    `b_enc` of `enc_buf`, and the attention output of sampled (sequence, kv head) units of the cache that was decoded."""
+    orc, cb, S = _oracle_setup(cache)
+    rng = np.random.default_rng(0)
+    per_seq = enc_buf.numel() // BATCH
+    codes, _ = pq.pq_unpack_codes(D, HKV, enc_buf[b_enc * per_seq:(b_enc + 1) * per_seq], 1, cache.capacity, CTX)
     toks = np.sort(rng.choice(CTX, 512, replace=False))
     res = {"codes_checked": 0, "codes_mismatch_inside_window": 0, "codes_mismatch_outside_window": 0}
     for kv, X in ((0, K_chunk), (1, V_chunk)):
         for h in range(HKV):
             x = X[torch.as_tensor(toks, device=X.device), h].float().cpu().double().numpy()
             want, _, angles = orc.encode(x, S, cb)
-            got = codes[b_enc, h, kv][torch.as_tensor(toks, device=codes.device)].cpu().numpy()
+            got = codes[0, h, kv][torch.as_tensor(toks, device=codes.device)].cpu().numpy()
             diff = got != want
             dist = orc.boundary_distance(angles, cb)
             res["codes_checked"] += int(want.size)
             res["codes_mismatch_inside_window"] += int(np.count_nonzero(diff & (dist <= 1e-6)))
             res["codes_mismatch_outside_window"] += int(np.count_nonzero(diff & (dist > 1e-6)))
-    lens = cache.lens.cpu().numpy()
-    worst = 0.0
-    for (b, hk) in ((b_enc, 0), ((b_enc + 3) % BATCH, 5 % HKV)):
-        n = int(lens[b])
-        c = codes[b, hk, :, :n].cpu().numpy()
-        r = radii[b, hk, :, :n].cpu().numpy()
-        g = HQ // HKV
-        qq = q[b, hk * g:(hk + 1) * g].float().cpu().double().numpy()[None]
-        want = orc.decode_attention(qq, c[0][None, None], r[0][None, None], c[1][None, None], r[1][None, None], [n],
-                                    cb, S, D ** -0.5)[0]
-        got = out[b, hk * g:(hk + 1) * g].float().cpu().double().numpy()
-        worst = max(worst, float(np.linalg.norm(got - want) / np.linalg.norm(want)))
-    res["attention_rel_l2_worst_of_2_units"] = worst
+    worst = max(_attention_unit_error(pq, cache, dec_buf, BATCH, cache.capacity, dec_lens, q, out, b, hk) for b, hk in units)
+    res["attention_rel_l2_worst_of_%d_units" % len(units)] = worst
     res["ok"] = bool(res["codes_mismatch_outside_window"] == 0 and worst < 2e-3)
     return res
 
 
 # --------------------------------------------------------------------------------------------
-# The CUDA arm
+# The CUDA arm: local measurements of one rank
 # --------------------------------------------------------------------------------------------
-def run_cuda(args):
-    import paper_2502_02617_b200 as pq
-    from paper_2502_02617_b200 import synthetic
-    dist, rank, world, local_rank = _dist_setup(args.gpus)
-    dev = torch.device("cuda", local_rank)
-    torch.cuda.set_device(dev)
-    pq.lib()
+def _event():
+    return torch.cuda.Event(enable_timing=True)
+
+
+def measure_headline(args, pq, synthetic, dev, rank, barrier):
+    """Configs 2 + 3 (+ append): returns the local timings of this rank."""
     capacity = CTX + 256
     cache = pq.PolarQuantCache(BATCH, HQ, HKV, D, capacity, seed=0, device=dev)
     stream = torch.cuda.current_stream()
+    bufs = [cache.cache, torch.empty_like(cache.cache)]      # two resident caches
+    lens = [cache.lens, torch.zeros_like(cache.lens)]
 
-    # Resident state: the batch's cache, filled by the encoder itself (2 distinct prefill chunks,
-    # each 128 MiB of bf16 K+V, so successive encode steps never find their input in L2).
+    # Resident state: both caches filled by the encoder itself (2 distinct prefill chunks, each 128 MiB of bf16
+    # K+V, so successive encode passes never find their input in L2).
     chunks = [synthetic.kv_like(1000 * rank + 10 + i, CTX, HKV, D, torch.bfloat16, dev) for i in range(2)]
-    cu = torch.tensor([0, CTX], dtype=torch.int32, device=dev)
     cu_all = torch.zeros(BATCH + 1, dtype=torch.int32, device=dev)
-    for b in range(BATCH):
-        cu_all.zero_()
-        cu_all[b + 1:] = CTX
-        Kb, Vb = chunks[b % 2]
-        pq.pq_encode_kv(cache.S, cache.tables, Kb, Vb, cu_all, cache.cache, cache.lens, capacity, cache.status)
+    for w in range(2):
+        for b in range(BATCH):
+            cu_all.zero_()
+            cu_all[b + 1:] = CTX
+            Kb, Vb = chunks[(b + w) % 2]
+            pq.pq_encode_kv(cache.S, cache.tables, Kb, Vb, cu_all, bufs[w], lens[w], capacity, cache.status)
     torch.cuda.synchronize()
     cache.check_status()
-    assert cache.lens.cpu().tolist() == [CTX] * BATCH
+    assert lens[0].cpu().tolist() == [CTX] * BATCH and lens[1].cpu().tolist() == [CTX] * BATCH
 
-    n_total = args.warmup + args.steps
     q_all = [synthetic.queries(77 + i + 1000 * rank, BATCH, HQ, D, torch.bfloat16, dev) for i in range(4)]
     new_all = [synthetic.kv_like(99 + i + 1000 * rank, BATCH, HKV, D, torch.bfloat16, dev) for i in range(4)]
     out = torch.empty_like(q_all[0])
-    lens_base = torch.full((BATCH,), CTX, dtype=torch.int32, device=dev)
-    cu_step = []
-    lens_step = []
+    cu_step, lens_step = [], []
     for b in range(BATCH):
         c = torch.zeros(BATCH + 1, dtype=torch.int32, device=dev)
         c[b + 1:] = CTX
         cu_step.append(c)
-        l = lens_base.clone()
+        l = torch.full((BATCH,), CTX, dtype=torch.int32, device=dev)
         l[b] = 0
         lens_step.append(l)
 
@@ -276,18 +308,18 @@ def run_cuda(args):
     dK, dV = torch.empty_like(chunks[0][0]), torch.empty_like(chunks[0][1])
     dq, dk1, dv1 = torch.empty_like(q_all[0]), torch.empty_like(new_all[0][0]), torch.empty_like(new_all[0][1])
 
-    def step(i, ev=None, e2e=False):
-        b_enc = i % BATCH
-        cache.lens.copy_(lens_step[b_enc])
+    def one_pass(i, ev=None, e2e=False):
+        """ev: four events -> [encode incl. its H2D | append incl. its H2D | decode incl. H2D of q and D2H of out]."""
+        b_enc, w = (i // 2) % BATCH, i % 2      # write cache w, read cache 1 - w
+        lens[w].copy_(lens_step[b_enc])
+        if ev: ev[0].record(stream)
         if e2e:
-            if ev: ev[0].record(stream)
             dK.copy_(host_chunks[i % 2][0], non_blocking=True)
             dV.copy_(host_chunks[i % 2][1], non_blocking=True)
             Kb, Vb = dK, dV
         else:
             Kb, Vb = chunks[i % 2]
-            if ev: ev[0].record(stream)
-        pq.pq_encode_kv(cache.S, cache.tables, Kb, Vb, cu_step[b_enc], cache.cache, cache.lens, capacity, cache.status)
+        pq.pq_encode_kv(cache.S, cache.tables, Kb, Vb, cu_step[b_enc], bufs[w], lens[w], capacity, cache.status)
         if ev: ev[1].record(stream)
         if e2e:
             dk1.copy_(host_new[i % 4][0], non_blocking=True)
@@ -295,19 +327,271 @@ def run_cuda(args):
             k1, v1 = dk1, dv1
         else:
             k1, v1 = new_all[i % 4]
-        pq.pq_append_kv(cache.S, cache.tables, k1, v1, cache.cache, cache.lens, capacity, cache.status)
+        pq.pq_append_kv(cache.S, cache.tables, k1, v1, bufs[w], lens[w], capacity, cache.status)
         if ev: ev[2].record(stream)
         if e2e:
             dq.copy_(host_q[i % 4], non_blocking=True)
             qq = dq
         else:
             qq = q_all[i % 4]
-        pq.pq_decode_attention(cache.S, cache.tables, qq, cache.cache, cache.lens, HKV, capacity, CTX + 1,
+        pq.pq_decode_attention(cache.S, cache.tables, qq, bufs[1 - w], lens[1 - w], HKV, capacity, CTX + 1,
                                D ** -0.5, out, cache.workspace, cache.status)
         if e2e:
             host_out.copy_(out, non_blocking=True)
         if ev: ev[3].record(stream)
-        return b_enc, qq
+        return b_enc, w, qq
+
+    def timed(e2e, inner, max_samples=400):
+        n_pass = args.steps * inner
+        stride = max(1, n_pass // max_samples)
+        evs = {}
+        for i in range(args.warmup * min(inner, 8)):
+            one_pass(i, None, e2e)
+        barrier()
+        wall0 = time.time()
+        t_start, t_end = _event(), _event()
+        t_start.record(stream)
+        last = None
+        for i in range(n_pass):
+            ev = None
+            if i % stride == 0:
+                ev = evs[i] = [_event() for _ in range(4)]
+            last = one_pass(i, ev, e2e)
+        t_end.record(stream)
+        barrier()
+        wall1 = time.time()
+        seg = np.array([[e[k].elapsed_time(e[k + 1]) for k in range(3)] for e in evs.values()])  # encode, append, decode
+        return t_start.elapsed_time(t_end), seg, last, (wall0, wall1)
+
+    # size the timed region: about TARGET_REGION_S seconds
+    probe = [_event() for _ in range(2)]
+    for i in range(4):
+        one_pass(i)
+    torch.cuda.synchronize()
+    probe[0].record(stream)
+    for i in range(16):
+        one_pass(i)
+    probe[1].record(stream)
+    torch.cuda.synchronize()
+    pass_ms = probe[0].elapsed_time(probe[1]) / 16
+    inner = args.inner if args.inner > 0 else max(1, math.ceil(TARGET_REGION_S * 1e3 / (args.steps * pass_ms)))
+
+    sampler = ClockSampler(dev.index or 0)
+    sampler.start()
+    total_ms, seg, last, wall = timed(False, inner)
+    clocks = sampler.stop(wall[0], wall[1])
+    cache.check_status()
+    match = None
+    if rank == 0 and not args.skip_match:
+        b_enc, w, qq = last
+        n_pass = args.steps * inner
+        Kb, Vb = chunks[(n_pass - 1) % 2]
+        dec_lens = lens[1 - w].cpu().tolist()
+        match = _oracle_match(pq, cache, bufs[w], b_enc, Kb, Vb, bufs[1 - w], dec_lens, qq, out,
+                              [(b_enc, 0), ((b_enc + 3) % BATCH, 5 % HKV)])
+    if args.skip_e2e:
+        e2e_total_ms, e2e_seg, e2e_inner = total_ms, seg, inner
+    else:
+        e2e_inner = max(1, math.ceil(1.0e3 / (args.steps * 3.0)))   # a pass with its 128 MiB of H2D takes about 3 ms
+        e2e_total_ms, e2e_seg, _, _ = timed(True, e2e_inner, 200)
+    cache.check_status()
+    return {
+        "inner": inner, "e2e_inner": e2e_inner, "total_ms": total_ms, "e2e_total_ms": e2e_total_ms,
+        "seg_ms": seg.mean(0).tolist(), "seg_best_ms": seg.min(0).tolist(), "e2e_seg_ms": e2e_seg.mean(0).tolist(),
+        "seg_samples": int(seg.shape[0]), "clocks": clocks, "match": match,
+        "h2d_decode_bytes": int(2 * new_all[0][0].numel() * 2 + q_all[0].numel() * 2),
+        "h2d_encode_bytes": int(2 * chunks[0][0].numel() * 2), "d2h_bytes": int(out.numel() * 2),
+    }
+
+
+def measure_config4(args, pq, synthetic, dev, rank):
+    """Config 4: 36 layers x (batch 1, 131072 tokens), every layer encoded on the device from its own seed and kept
+    packed (4.68 GB); one decode step = 36 sequential pq_decode_attention launches."""
+    layers, n = 36, 131072
+    base = pq.PolarQuantCache(1, HQ, HKV, D, n, seed=4, device=dev)
+    caches = [base.cache] + [torch.empty_like(base.cache) for _ in range(layers - 1)]
+    lens = [torch.zeros(1, dtype=torch.int32, device=dev) for _ in range(layers)]
+    cu = torch.tensor([0, n], dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+    enc_ev = []
+    for l in range(layers):
+        K, V = synthetic.kv_like(4000 + 100 * rank + l, n, HKV, D, torch.bfloat16, dev)
+        e = (_event(), _event())
+        e[0].record(stream)
+        pq.pq_encode_kv(base.S, base.tables, K, V, cu, caches[l], lens[l], n, base.status)
+        e[1].record(stream)
+        enc_ev.append(e)
+        del K, V
+    torch.cuda.synchronize()
+    base.check_status()
+    qs = [synthetic.queries(4500 + l, 1, HQ, D, torch.bfloat16, dev) for l in range(layers)]
+    outs = [torch.empty_like(qs[0]) for _ in range(layers)]
+
+    def step():
+        for l in range(layers):
+            pq.pq_decode_attention(base.S, base.tables, qs[l], caches[l], lens[l], HKV, n, n, D ** -0.5, outs[l],
+                                   base.workspace, base.status)
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    reps = 30
+    evs = [(_event(), _event()) for _ in range(reps)]
+    for a, b in evs:
+        a.record(stream)
+        step()
+        b.record(stream)
+    torch.cuda.synchronize()
+    base.check_status()
+    t = [a.elapsed_time(b) for a, b in evs]
+    res = {"layers": layers, "ctx": n, "batch": 1, "decode_step_ms": float(np.mean(t)), "decode_step_best_ms": float(min(t)),
+           "launches_per_step": layers, "compressed_bytes_per_step": layers * n * HKV * BYTES_PER_TOKEN_HEAD,
+           "encode_ms_per_layer": float(np.mean([a.elapsed_time(b) for a, b in enc_ev[1:]]))}
+    if rank == 0 and not args.skip_match:
+        res["attention_rel_l2_layer17_unit"] = _attention_unit_error(pq, base, caches[17], 1, n, [n], qs[17], outs[17], 0, 3)
+    return res
+
+
+def measure_config5(args, pq, synthetic, dev, rank):
+    """Config 5: batch 16, ragged contexts in [4096, 65536], prefill in 4096-token chunks, then 128 steps of
+    (append one token per sequence, decode attention)."""
+    B, steps, chunk = 16, 128, 4096
+    lens0 = synthetic.ragged_lengths(5, B, 4096, 65536)
+    cap = max(lens0) + steps
+    cache = pq.PolarQuantCache(B, HQ, HKV, D, cap, seed=5, device=dev)
+    stream = torch.cuda.current_stream()
+    done, c_idx, prefill_ms, pre_ev = [0] * B, 0, 0.0, []
+    while any(d < n for d, n in zip(done, lens0)):
+        take = [min(chunk, n - d) for d, n in zip(done, lens0)]
+        K, V = synthetic.kv_like(500 + c_idx + 1000 * rank, sum(take), HKV, D, torch.bfloat16, dev)
+        cu = torch.tensor(np.concatenate(([0], np.cumsum(take))), dtype=torch.int32, device=dev)
+        e = (_event(), _event())
+        e[0].record(stream)
+        cache.encode(K, V, cu)
+        e[1].record(stream)
+        pre_ev.append((e, sum(take)))
+        done = [d + t for d, t in zip(done, take)]
+        c_idx += 1
+    torch.cuda.synchronize()
+    cache.check_status()
+    prefill_ms = sum(e[0].elapsed_time(e[1]) for e, _ in pre_ev[1:])
+    prefill_tokens = sum(t for _, t in pre_ev[1:])
+    lens_base = cache.lens.clone()
+    new = [synthetic.kv_like(9000 + s, B, HKV, D, torch.bfloat16, dev) for s in range(8)]
+    qs = [synthetic.queries(9500 + s, B, HQ, D, torch.bfloat16, dev) for s in range(8)]
+    out = torch.empty_like(qs[0])
+    totals, app, dec = [], [], []
+    for rep in range(3):          # the first repetition warms up
+        cache.lens.copy_(lens_base)
+        evs = [[_event() for _ in range(3)] for _ in range(steps)]
+        for s in range(steps):
+            evs[s][0].record(stream)
+            cache.append(*new[s % 8])
+            evs[s][1].record(stream)
+            cache.attend(qs[s % 8], out=out, max_len=cap)
+            evs[s][2].record(stream)
+        torch.cuda.synchronize()
+        cache.check_status()
+        if rep:
+            totals.append(evs[0][0].elapsed_time(evs[-1][2]))
+            app.append(np.mean([e[0].elapsed_time(e[1]) for e in evs]))
+            dec.append(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
+    mean_tokens = sum(lens0) + B * (steps + 1) / 2
+    return {"batch": B, "steps": steps, "context_lengths": [min(lens0), max(lens0)], "cached_tokens_at_start": sum(lens0),
+            "total_ms_128_steps": float(np.mean(totals)), "ms_per_step": float(np.mean(totals)) / steps,
+            "append_ms": float(np.mean(app)), "decode_ms": float(np.mean(dec)),
+            "compressed_bytes_per_step": int(mean_tokens * HKV * BYTES_PER_TOKEN_HEAD),
+            "prefill_chunk_tokens": chunk, "prefill_tokens_per_s": prefill_tokens / (prefill_ms * 1e-3)}
+
+
+# --------------------------------------------------------------------------------------------
+# Reduction over ranks and the JSON line (no CUDA calls: covered by a two-rank gloo test)
+# --------------------------------------------------------------------------------------------
+def reduce_and_format(local, steps, warmup, rank, world, dist=None, device="cpu", cpu_baseline=None):
+    """Max over ranks of every timing of `local` (the slowest rank's time counts), then the JSON line (rank 0
+    returns it, the other ranks return None)."""
+    from paper_2502_02617_b200 import sharding
+    head = local["headline"]
+    keys = ["total_ms", "e2e_total_ms"]
+    flat = [head[k] for k in keys] + head["seg_ms"] + head["seg_best_ms"] + head["e2e_seg_ms"]
+    c4, c5 = local.get("cfg4"), local.get("cfg5")
+    if c4:
+        flat += [c4["decode_step_ms"], c4["decode_step_best_ms"], c4["encode_ms_per_layer"]]
+    if c5:
+        flat += [c5["total_ms_128_steps"], c5["append_ms"], c5["decode_ms"]]
+    red = sharding.max_over_ranks(flat, dist, device)
+    total_ms, e2e_total_ms = red[0], red[1]
+    enc_ms, app_ms, dec_ms = red[2:5]
+    enc_best, app_best, dec_best = red[5:8]
+    e_enc_ms, e_app_ms, e_dec_ms = red[8:11]
+    pos = 11
+    if rank != 0:
+        return None
+    inner, batch = head["inner"], local["batch"]
+    n_pass = steps * inner
+    comp_bytes = batch * HKV * (CTX + 1) * BYTES_PER_TOKEN_HEAD
+    peak, peak_src = _peaks()
+    achieved = comp_bytes / (dec_ms * 1e-3) / 1e9
+    value = world * achieved
+    e2e_region_ms = e_app_ms + e_dec_ms
+    enc_bytes = CTX * HKV * 2 * ENCODE_BYTES_PER_VECTOR
+    clocks = head["clocks"]
+    mhz = clocks.get("sm_mhz") or 0.0
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "batch": batch, "per_gpu": True, "inner": inner,
+                   "step_definition": f"{inner} consecutive passes of (encode chunk, append, decode attention); times below are per pass",
+                   "ms_per_pass": total_ms / n_pass, "timed_region_s": total_ms * 1e-3,
+                   "l2": "inputs larger than L2 and rotated: two resident 260 MB caches alternate (a pass encodes and appends into one "
+                         "and decodes the other, which was last written two passes earlier), two alternating 128 MiB prefill chunks",
+                   "compressed_bytes_per_decode": comp_bytes, "decode_ms": dec_ms, "append_ms": app_ms, "encode_ms": enc_ms,
+                   "decode_best_ms": dec_best, "encode_best_ms": enc_best, "event_samples": head["seg_samples"],
+                   "decode_ms_x_sm_mhz": dec_ms * mhz, "encode_ms_x_sm_mhz": enc_ms * mhz,
+                   "value_definition": "compressed bytes / mean CUDA-event time of pq_decode_attention (one persistent kernel)"},
+        "encode": {"tokens_per_s": world * CTX / (enc_ms * 1e-3), "vectors_per_s": world * CTX * HKV * 2 / (enc_ms * 1e-3),
+                   "gbs": enc_bytes / (enc_ms * 1e-3) / 1e9, "hbm_frac_measured": enc_bytes / (enc_ms * 1e-3) / 1e9 / peak,
+                   "frac_of_nominal_8TBs": enc_bytes / (enc_ms * 1e-3) / 1e9 / 8000.0,
+                   "e2e_tokens_per_s": world * CTX / (e_enc_ms * 1e-3), "e2e_h2d_bytes_per_chunk": head["h2d_encode_bytes"]},
+        "roofline": {"kernel": "decode_attention_fast_kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "peak_source": peak_src, "traffic": _decode_traffic(batch)},
+        "e2e": {"value": world * comp_bytes / (e2e_region_ms * 1e-3) / 1e9, "unit": UNIT,
+                "h2d_bytes_per_step": head["h2d_decode_bytes"], "d2h_bytes_per_step": head["d2h_bytes"],
+                "region_ms": e2e_region_ms,
+                "definition": "compressed bytes / time of [H2D of the new k, v from pinned memory, pq_append_kv, H2D of q, "
+                              "pq_decode_attention, D2H of the output]; the byte counts are the copies inside that region.  "
+                              "The prefill chunk's own H2D (e2e_h2d_bytes_per_chunk) and encode are timed as encode.e2e_tokens_per_s",
+                "ms_per_pass_with_prefill_h2d": e2e_total_ms / (steps * head["e2e_inner"])},
+        "gpu_launches": 5 * n_pass,  # encode + lens, append + lens, decode attention
+        "clocks": clocks,
+        "oracle_match": head["match"],
+        "configs": {},
+    }
+    if c4:
+        t, tb, te = red[pos:pos + 3]
+        pos += 3
+        gbs = c4["compressed_bytes_per_step"] / (t * 1e-3) / 1e9
+        line["configs"]["cfg4"] = dict(c4, decode_step_ms=t, decode_step_best_ms=tb, encode_ms_per_layer=te,
+                                       per_layer_us=t / c4["layers"] * 1e3, gbs=gbs, hbm_frac_measured=gbs / peak,
+                                       frac_of_nominal_8TBs=gbs / 8000.0)
+    if c5:
+        t, ta, td = red[pos:pos + 3]
+        gbs = c5["compressed_bytes_per_step"] / (td * 1e-3) / 1e9
+        line["configs"]["cfg5"] = dict(c5, total_ms_128_steps=t, ms_per_step=t / c5["steps"], append_ms=ta, decode_ms=td,
+                                       decode_gbs=gbs, hbm_frac_measured=gbs / peak, frac_of_nominal_8TBs=gbs / 8000.0)
+    if cpu_baseline is not None:
+        line["cpu_baseline"] = cpu_baseline
+    return line
+
+
+def run_cuda(args):
+    import paper_2502_02617_b200 as pq
+    from paper_2502_02617_b200 import synthetic
+    dist, rank, world, local_rank = dist_setup("nccl")
+    dev = torch.device("cuda", local_rank)
+    torch.cuda.set_device(dev)
+    pq.lib()
 
     def barrier():
         torch.cuda.synchronize()
@@ -315,87 +599,17 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(e2e):
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-        for i in range(args.warmup):
-            step(i, None, e2e)
-        barrier()
-        wall = [time.time(), None]
-        t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        t_start.record(stream)
-        last = None
-        for i in range(args.steps):
-            last = step(args.warmup + i, evs[i], e2e)
-        t_end.record(stream)
-        barrier()
-        wall[1] = time.time()
-        total_ms = t_start.elapsed_time(t_end)
-        seg = np.array([[e[k].elapsed_time(e[k + 1]) for k in range(3)] for e in evs])  # encode, append, decode
-        return total_ms, seg, last, wall
-
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    total_ms, seg, last, wall = timed(e2e=False)
-    clocks = sampler.stop(wall[0], wall[1])
-    cache.check_status()
-    match = None
-    if rank == 0 and not args.skip_match:
-        b_enc, qq = last
-        Kb, Vb = chunks[(n_total - 1) % 2]
-        match = _oracle_match(cache, Kb, Vb, b_enc, qq, out)
-    e2e_total_ms, e2e_seg, _, _ = (total_ms, seg, None, None) if args.skip_e2e else timed(e2e=True)
-    cache.check_status()
-
-    def reduce_max(x):
-        if dist is None:
-            return x
-        t = torch.tensor(x, dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return t.cpu().numpy() if t.ndim else float(t)
-
-    enc_ms, app_ms, dec_ms = (float(v) for v in reduce_max(seg.mean(0)))
-    e_enc_ms, e_app_ms, e_dec_ms = (float(v) for v in reduce_max(e2e_seg.mean(0)))
-    step_ms = float(reduce_max(total_ms)) / args.steps
-    comp_bytes = BATCH * HKV * (CTX + 1) * BYTES_PER_TOKEN_HEAD
-    value = world * comp_bytes / (dec_ms * 1e-3) / 1e9
-    e2e_value = world * comp_bytes / ((e_app_ms + e_dec_ms) * 1e-3) / 1e9
-    peak, peak_src = _peaks()
-    achieved = comp_bytes / (dec_ms * 1e-3) / 1e9
-    enc_bytes = CTX * HKV * 2 * (256 + 62)
-
-    if rank != 0:
-        return
-    # DRAM bytes of one decode-attention launch: ncu capture at batch 4 (profiles/decode_attention_fast_kernel_
-    # batch4_ctx32768.md: 130.47 MB read + 3.45 MB written), scaled by the batch (traffic is proportional to it)
-    traffic = (130.47e6 + 3.45e6) * BATCH / 4.0
-    cpu = _oracle_sample_throughput(12.0) if world == 1 and not args.no_cpu_baseline else None
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f16",
-        "data": "synthetic",
-        "config": {"workload": WORKLOAD, "batch": BATCH, "per_gpu": True, "l2": "inputs larger than L2 (260 MB cache per decode, "
-                   "two alternating 128 MiB prefill chunks)", "compressed_bytes_per_decode": comp_bytes,
-                   "decode_ms": dec_ms, "append_ms": app_ms, "encode_ms": enc_ms,
-                   "value_definition": "compressed bytes / CUDA-event time of pq_decode_attention (one persistent kernel)"},
-        "encode": {"tokens_per_s": world * CTX / (enc_ms * 1e-3), "vectors_per_s": world * CTX * HKV * 2 / (enc_ms * 1e-3),
-                   "gbs": enc_bytes / (enc_ms * 1e-3) / 1e9, "hbm_frac_measured": enc_bytes / (enc_ms * 1e-3) / 1e9 / peak,
-                   "e2e_tokens_per_s": world * CTX / (e_enc_ms * 1e-3)},
-        "roofline": {"kernel": "decode attention main kernel", "bound": "hbm", "achieved": achieved, "peak": peak,
-                     "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8TBs": achieved / 8000.0,
-                     "peak_source": peak_src, "traffic": traffic},
-        "e2e": {"value": e2e_value, "unit": UNIT,
-                "h2d_bytes_per_step": int(2 * chunks[0][0].numel() * 2 + 2 * new_all[0][0].numel() * 2 + q_all[0].numel() * 2),
-                "d2h_bytes_per_step": int(out.numel() * 2),
-                "definition": "compressed bytes / (H2D of new k,v and q + append + decode attention + D2H of the output); "
-                              "the 128 MiB prefill chunk's H2D is charged to encode.e2e_tokens_per_s",
-                "ms_per_step": float(reduce_max(e2e_total_ms)) / args.steps},
-        "gpu_launches": 5 * args.steps,  # encode + lens, append + lens, decode attention
-        "clocks": clocks,
-        "oracle_match": match,
-    }
-    if cpu is not None:
-        line["cpu_baseline"] = cpu
-    print(json.dumps(line))
+    local = {"batch": BATCH, "headline": measure_headline(args, pq, synthetic, dev, rank, barrier)}
+    torch.cuda.empty_cache()
+    if not args.skip_configs:
+        local["cfg4"] = measure_config4(args, pq, synthetic, dev, rank)
+        torch.cuda.empty_cache()
+        local["cfg5"] = measure_config5(args, pq, synthetic, dev, rank)
+        torch.cuda.empty_cache()
+    cpu = _oracle_sample_throughput(12.0) if rank == 0 and world == 1 and not args.no_cpu_baseline else None
+    line = reduce_and_format(local, args.steps, args.warmup, rank, world, dist, dev, cpu)
+    if line is not None:
+        print(json.dumps(line))
 
 
 def main():
@@ -405,10 +619,12 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--inner", type=int, default=0, help="passes per step (0: sized for a timed region of about two seconds)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=BATCH, help="sequences in the resident batch (profiling captures use fewer)")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiling captures)")
-    ap.add_argument("--skip-match", action="store_true", help="skip the sampled oracle check (profiling captures)")
+    ap.add_argument("--skip-match", action="store_true", help="skip the sampled oracle checks (profiling captures)")
+    ap.add_argument("--skip-configs", action="store_true", help="skip configs 4 and 5 (profiling captures)")
     args = ap.parse_args()
     BATCH = args.batch
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup

@@ -44,6 +44,63 @@ def _worker(rank, world, port, results):
         dist.destroy_process_group()
 
 
+def _fake_local(rank):
+    """What bench.py measures on one rank, with made-up numbers (no CUDA on this machine): rank 1 is the slower one."""
+    slow = 1.0 + 0.5 * rank
+    head = {"inner": 3, "e2e_inner": 2, "total_ms": 60.0 * slow, "e2e_total_ms": 90.0 * slow,
+            "seg_ms": [0.1 * slow, 0.02 * slow, 0.15 * slow], "seg_best_ms": [0.09, 0.02, 0.14],
+            "e2e_seg_ms": [2.0 * slow, 0.03 * slow, 0.2 * slow], "seg_samples": 60,
+            "clocks": {"sm_mhz": 1965.0, "sm_max_mhz": 1965.0, "reasons": [], "samples": 10, "samples_under_load": 10},
+            "match": None, "h2d_decode_bytes": 98304, "h2d_encode_bytes": 134217728, "d2h_bytes": 65536}
+    cfg4 = {"layers": 36, "ctx": 131072, "batch": 1, "decode_step_ms": 3.0 * slow, "decode_step_best_ms": 2.9,
+            "launches_per_step": 36, "compressed_bytes_per_step": 4680843264, "encode_ms_per_layer": 0.4 * slow}
+    cfg5 = {"batch": 16, "steps": 128, "context_lengths": [4096, 65536], "cached_tokens_at_start": 600000,
+            "total_ms_128_steps": 40.0 * slow, "ms_per_step": 0.3, "append_ms": 0.02 * slow, "decode_ms": 0.3 * slow,
+            "compressed_bytes_per_step": 600000000, "prefill_chunk_tokens": 4096, "prefill_tokens_per_s": 2.5e8}
+    return {"batch": 8, "headline": head, "cfg4": cfg4, "cfg5": cfg5}
+
+
+def _bench_worker(rank, world, port, results):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world),
+                      LOCAL_RANK=str(rank))
+    import bench
+    d, r, w, _ = bench.dist_setup("gloo")
+    try:
+        line = bench.reduce_and_format(_fake_local(rank), steps=20, warmup=3, rank=r, world=w, dist=d, device="cpu")
+        if rank == 0:
+            results.put(line)
+        else:
+            assert line is None
+    finally:
+        d.destroy_process_group()
+
+
+def test_bench_rank_logic_takes_the_slowest_rank_and_sums_the_job():
+    """bench.py's own reduction and JSON line under two gloo ranks (the CUDA measurements are replaced by made-up
+    numbers): every time is the maximum over ranks, `value` is the whole job's throughput."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    results = ctx.Queue()
+    procs = [ctx.Process(target=_bench_worker, args=(r, 2, port, results)) for r in range(2)]
+    for p in procs:
+        p.start()
+    line = results.get(timeout=180)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    comp = 8 * 8 * 32769 * 124
+    assert line["n_gpus"] == 2 and line["scaling"] == "weak" and line["steps"] == 20
+    assert abs(line["config"]["decode_ms"] - 0.15 * 1.5) < 1e-12           # the slower rank's time
+    assert abs(line["value"] - 2 * comp / (0.15 * 1.5 * 1e-3) / 1e9) < 1e-6  # both ranks' bytes over that time
+    assert abs(line["ms_per_step"] - 60.0 * 1.5 / 20) < 1e-9
+    assert abs(line["e2e"]["region_ms"] - (0.03 + 0.2) * 1.5) < 1e-12
+    assert line["e2e"]["h2d_bytes_per_step"] == 98304 and line["gpu_launches"] == 5 * 20 * 3
+    assert abs(line["configs"]["cfg4"]["decode_step_ms"] - 4.5) < 1e-12 and abs(line["configs"]["cfg5"]["decode_ms"] - 0.45) < 1e-12
+    assert line["roofline"]["bound"] == "hbm" and abs(line["roofline"]["frac"] * line["roofline"]["peak"] - line["roofline"]["achieved"]) < 1e-6
+
+
 def test_two_ranks_shard_sequences_without_data_path_collectives():
     assert [list(sharding.shard_range(5, r, 2)) for r in range(2)] == [[0, 1, 2], [3, 4]]
     assert [len(sharding.shard_range(8, r, 3)) for r in range(3)] == [3, 3, 2]
