@@ -253,10 +253,10 @@ __device__ __forceinline__ bool bar_or(int bar_id, int n_threads, bool v) {
 template <class Q, int kWords>
 __device__ inline void fix_rounds(const EncodeArgs& a, Q* q, unsigned long long (&left)[kWords], int64_t xoff, uint8_t* tb,
                                   int tok, int blk0, int kv, int t, int n_threads, int bar_id,
-                                  const float* Sf = nullptr) {
+                                  const double* Sd = nullptr) {
   for (int round = 0; round < 4096; ++round) {
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
-    fix_process(q, 1, t, n_threads, a.K, a.V, a.in_dtype, a.S, Sf, *a.tables, a.status);
+    fix_process(q, 1, t, n_threads, a.K, a.V, a.in_dtype, a.S, Sd, *a.tables, a.status);
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(n_threads) : "memory");
     if (t < 4) q->count[t] = 0;
     bool mine = false;

@@ -308,34 +308,27 @@ __device__ __forceinline__ void exact_coords(const double* xk, const float* S, i
   }
 }
 
-// The same sums with a float32 copy of S in shared memory (no L2 latency in the loop).  Row k of S sits at
-// row (k & 15) * 8 + (k >> 4) of `Sf`, rows kFixSfStride floats apart, so the eight lanes of a group
-// (k = 16 * sub + i) read eight consecutive rows: 8- and 16-byte loads without bank conflicts.
-constexpr int kFixSfStride = 132;
-constexpr int kFixSfBytes = 128 * kFixSfStride * 4;
-__host__ __device__ constexpr int fix_sf_row(int k) { return (k & 15) * 8 + (k >> 4); }
+// The same sums with S staged in shared memory as float64 (no conversions, no L2 latency in the loop; on this
+// GPU a warp-wide float64 FMA occupies its pipe for 16 cycles, so the loop should hold nothing else that is slow).
+// Row k of S sits at row (k & 15) * 8 + (k >> 4) of `Sd`, rows kFixSdStride doubles apart, so the eight lanes of a
+// group (k = 16 * sub + i) read eight consecutive rows: 16-byte loads without bank conflicts.
+constexpr int kFixSdStride = 130;
+constexpr int kFixSdBytes = 128 * kFixSdStride * 8;
+__host__ __device__ constexpr int fix_sd_row(int k) { return (k & 15) * 8 + (k >> 4); }
 template <int NC>
-__device__ __forceinline__ void exact_coords_sm(const double* xk, const float* Sf, int sub, int c0, unsigned gmask,
+__device__ __forceinline__ void exact_coords_sm(const double* xk, const double* Sd, int sub, int c0, unsigned gmask,
                                                 double* y) {
   double acc[NC];
 #pragma unroll
   for (int c = 0; c < NC; ++c) acc[c] = 0.0;
 #pragma unroll
   for (int i = 0; i < 16; ++i) {
-    const float* srow = Sf + (i * 8 + sub) * kFixSfStride + c0;
-    if (NC == 2) {
-      const float2 s2 = *reinterpret_cast<const float2*>(srow);
-      acc[0] = fma(xk[i], (double)s2.x, acc[0]);
-      acc[1] = fma(xk[i], (double)s2.y, acc[1]);
-    } else {
+    const double2* srow = reinterpret_cast<const double2*>(Sd + (i * 8 + sub) * kFixSdStride + c0);
 #pragma unroll
-      for (int c4 = 0; c4 < NC / 4; ++c4) {
-        const float4 s4 = reinterpret_cast<const float4*>(srow)[c4];
-        acc[4 * c4] = fma(xk[i], (double)s4.x, acc[4 * c4]);
-        acc[4 * c4 + 1] = fma(xk[i], (double)s4.y, acc[4 * c4 + 1]);
-        acc[4 * c4 + 2] = fma(xk[i], (double)s4.z, acc[4 * c4 + 2]);
-        acc[4 * c4 + 3] = fma(xk[i], (double)s4.w, acc[4 * c4 + 3]);
-      }
+    for (int c2 = 0; c2 < NC / 2; ++c2) {
+      const double2 s2 = srow[c2];
+      acc[2 * c2] = fma(xk[i], s2.x, acc[2 * c2]);
+      acc[2 * c2 + 1] = fma(xk[i], s2.y, acc[2 * c2 + 1]);
     }
   }
 #pragma unroll
@@ -365,10 +358,10 @@ __device__ __forceinline__ uint32_t exact_code(const double* y, int level, const
 
 // Process everything queued, in level order: called by `n_threads` threads (a multiple of 32) with linear index `t`.
 // `q` points to `n_queues` queues laid out back to back; their entries are taken level by level.
-// `Sf` (may be null) is the copy of S in shared memory for exact_coords_sm.
+// `Sd` (may be null) is the float64 copy of S in shared memory for exact_coords_sm.
 template <class Q>
 __device__ inline void fix_process(const Q* q, int n_queues, int t, int n_threads, const void* kbase, const void* vbase,
-                                   int in_dtype, const float* S, const float* Sf, const Tables& tb, int32_t* status) {
+                                   int in_dtype, const float* S, const double* Sd, const Tables& tb, int32_t* status) {
   constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock;
   const int sub = t & 7, n_groups = n_threads >> 3;
   const unsigned gmask = 0xFFu << (t & 24);
@@ -426,18 +419,18 @@ __device__ inline void fix_process(const Q* q, int n_queues, int t, int n_thread
     }
     double y[16];
     uint32_t code;
-    if (Sf != nullptr) {  // uniform over the CTA
+    if (Sd != nullptr) {  // uniform over the CTA
       if (level == 1) {
-        exact_coords_sm<2>(xk, Sf, sub, c0, gmask, y);
+        exact_coords_sm<2>(xk, Sd, sub, c0, gmask, y);
         code = exact_code<2>(y, level, tb);
       } else if (level == 2) {
-        exact_coords_sm<4>(xk, Sf, sub, c0, gmask, y);
+        exact_coords_sm<4>(xk, Sd, sub, c0, gmask, y);
         code = exact_code<4>(y, level, tb);
       } else if (level == 3) {
-        exact_coords_sm<8>(xk, Sf, sub, c0, gmask, y);
+        exact_coords_sm<8>(xk, Sd, sub, c0, gmask, y);
         code = exact_code<8>(y, level, tb);
       } else {
-        exact_coords_sm<16>(xk, Sf, sub, c0, gmask, y);
+        exact_coords_sm<16>(xk, Sd, sub, c0, gmask, y);
         code = exact_code<16>(y, level, tb);
       }
     } else if (level == 1) {

@@ -39,7 +39,6 @@ constexpr int kTcSBytes = 128 * 128 * 2;   // one bf16 term of S (B operand)
 using TcFixQueue = FixQueueT<256>;
 constexpr int kTcSmS = 0;
 constexpr int kTcSmX = kTcSmS + kTcTerms * kTcSBytes;
-constexpr int kTcSmSf = kTcSmX;                              // float32 copy of S for the last batch of exact re-decisions (over the idle ring)
 constexpr int kTcSmFq = kTcSmX + kTcStages * kTcXBytes;      // FastQuant (40 B)
 constexpr int kTcSmBar = kTcSmFq + 64;                       // x_full[kTcStages], acc_full[kTcSlots]
 constexpr int kTcSmMisc = kTcSmBar + 64;                     // tmem base, abort flag, copies issued per stage
@@ -49,7 +48,7 @@ constexpr int kTcSpin = 1 << 22;
 static_assert(kTcTerms == 3, "kRotErrTc is the bound for three terms");
 static_assert(sizeof(TcFixQueue) % 16 == 0, "queues are laid out back to back");
 static_assert(kTcSmTotal <= 227 * 1024, "shared memory of one CTA");
-static_assert(kFixSfBytes <= kTcStages * kTcXBytes, "the float32 copy of S must fit in the ring");
+static_assert(kFixSdBytes <= kTcSmFq, "the float64 copy of S must fit in the operand buffers");
 
 __device__ __forceinline__ uint32_t tc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void tc_mbar_init(uint32_t bar, uint32_t count) {
@@ -171,7 +170,6 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   volatile int* copies_issued = reinterpret_cast<volatile int*>(smem + kTcSmMisc + 8);  // [kTcStages]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kTcSmMisc);
   FastQuant* fq = reinterpret_cast<FastQuant*>(smem + kTcSmFq);
-  float* Sf = reinterpret_cast<float*>(smem + kTcSmSf);
   TcFixQueue* fixq = reinterpret_cast<TcFixQueue*>(smem + kTcSmFix) + slot;
   const uint32_t bar_xfull = sb + kTcSmBar, bar_acc = bar_xfull + 8 * kTcStages;
   const int n_tiles = n_row_tiles * 2 * a.n_kv_heads;
@@ -218,28 +216,36 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   // B operand: B[n][k] = S[k][n]; two halves of 64 k; row n = 128 bytes, 16-byte chunk c stored at c ^ (n & 7).
   // A task is (row n, chunk of 8 consecutive k): 8 coalesced loads (lanes = consecutive n), one 16-byte store per
   // term.
-  for (int task = tid; task < 128 * 16; task += kTcThreads) {
-    const int n = task & 127, oct = task >> 7;  // k = 8 * oct .. 8 * oct + 7
-    float v[8];
+  {
+    constexpr int kTasks = 128 * 16 / kTcThreads;  // per thread
+    float v[kTasks][8];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = a.S[(8 * oct + i) * 128 + n];
-    uint32_t term[kTcTerms][4];
+    for (int j = 0; j < kTasks; ++j) {             // all loads first: one round trip to L2 instead of kTasks
+      const int task = tid + j * kTcThreads, n = task & 127, oct = task >> 7;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      float v0 = v[2 * i], v1 = v[2 * i + 1];
-#pragma unroll
-      for (int t = 0; t < kTcTerms; ++t) {
-        const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
-        term[t][i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-        v0 -= __bfloat162float(h0);  // exact: the residual of a bf16 rounding fits float32
-        v1 -= __bfloat162float(h1);
-      }
+      for (int i = 0; i < 8; ++i) v[j][i] = __ldg(a.S + (8 * oct + i) * 128 + n);
     }
-    const int half = oct >> 3, c = oct & 7;
-    const int off = half * 16384 + n * 128 + ((c ^ (n & 7)) << 4);
 #pragma unroll
-    for (int t = 0; t < kTcTerms; ++t)
-      *reinterpret_cast<uint4*>(smem + kTcSmS + t * kTcSBytes + off) = make_uint4(term[t][0], term[t][1], term[t][2], term[t][3]);
+    for (int j = 0; j < kTasks; ++j) {
+      const int task = tid + j * kTcThreads, n = task & 127, oct = task >> 7;  // k = 8 * oct .. 8 * oct + 7
+      uint32_t term[kTcTerms][4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float v0 = v[j][2 * i], v1 = v[j][2 * i + 1];
+#pragma unroll
+        for (int t = 0; t < kTcTerms; ++t) {
+          const __nv_bfloat16 h0 = __float2bfloat16_rn(v0), h1 = __float2bfloat16_rn(v1);
+          term[t][i] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+          v0 -= __bfloat162float(h0);  // exact: the residual of a bf16 rounding fits float32
+          v1 -= __bfloat162float(h1);
+        }
+      }
+      const int half = oct >> 3, c = oct & 7;
+      const int off = half * 16384 + n * 128 + ((c ^ (n & 7)) << 4);
+#pragma unroll
+      for (int t = 0; t < kTcTerms; ++t)
+        *reinterpret_cast<uint4*>(smem + kTcSmS + t * kTcSBytes + off) = make_uint4(term[t][0], term[t][1], term[t][2], term[t][3]);
+    }
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA unit
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -415,13 +421,22 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
-  // Every MMA and copy of this CTA has completed (each was waited for by its slot), so the ring is idle: put a
-  // float32 copy of S there (rows permuted, see fix_sf_row) for the queued exact re-decisions.
+  // Every MMA and copy of this CTA has completed (each was waited for by its slot), so the operand buffers are
+  // idle: put a float64 copy of S there (rows permuted, see fix_sd_row) for the queued exact re-decisions.
+  double* Sd = reinterpret_cast<double*>(smem + kTcSmS);
   if (!*abort_flag) {
-    for (int idx = tid; idx < 128 * 128; idx += kTcThreads) Sf[fix_sf_row(idx >> 7) * kFixSfStride + (idx & 127)] = __ldg(a.S + idx);
+    constexpr int kPer = 128 * 128 / kTcThreads;
+    float sv[kPer];
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) sv[j] = __ldg(a.S + tid + j * kTcThreads);
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) {
+      const int idx = tid + j * kTcThreads;
+      Sd[fix_sd_row(idx >> 7) * kFixSdStride + (idx & 127)] = (double)sv[j];
+    }
     __syncthreads();
   }
-  fix_process(fixq - slot, kTcSlots, tid, kTcThreads, a.K, a.V, a.in_dtype, a.S, *abort_flag ? (const float*)nullptr : Sf,
+  fix_process(fixq - slot, kTcSlots, tid, kTcThreads, a.K, a.V, a.in_dtype, a.S, *abort_flag ? (const double*)nullptr : Sd,
               *a.tables, a.status);
   if (*abort_flag && tid < kTcStages && copies_issued[tid] > 0) {
     // gave up somewhere: let the copies that are still in flight land (bounded) before the CTA and its

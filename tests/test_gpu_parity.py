@@ -9,7 +9,7 @@ import torch
 import paper_2502_02617_b200 as pq
 from paper_2502_02617_b200 import synthetic
 from oracle import polarquant_oracle as orc
-from parity_utils import (TOL_ATTENTION, TOL_DECODED, assert_codes_match, assert_radii_match, code_mismatch_report,
+from parity_utils import (TOL_ATTENTION, TOL_ATTENTION_F32_IO, TOL_DECODED, assert_codes_match, assert_radii_match, code_mismatch_report,
                           radii_ulp_report,
                           oracle_codebooks, rel_l2, to_f64)
 
@@ -99,8 +99,12 @@ def test_ragged_batch_encode_dequant_attention(d, Hq, Hkv):
     cache.check_status()
     want = ref.attend(to_f64(q), d ** -0.5)
     assert rel_l2(to_f64(out), want) < TOL_ATTENTION
-    for b in range(B):  # per sequence too, so a short sequence cannot hide behind a long one
-        assert rel_l2(to_f64(out)[b], want[b]) < 2 * TOL_ATTENTION
+    # per sequence too, so that a short sequence cannot hide behind a long one: with float32 I/O
+    q32 = q.float()
+    out32 = to_f64(cache.attend(q32))
+    want32 = ref.attend(to_f64(q32), d ** -0.5)
+    for b in range(B):
+        assert rel_l2(out32[b], want32[b]) < TOL_ATTENTION_F32_IO
 
 
 def test_chunked_prefill_and_append_equal_one_shot_and_oracle():
@@ -170,12 +174,12 @@ def test_attention_special_cases_len1_and_identical_keys():
     K[1:] = K[1]  # sequence 1: forty identical keys
     cu = torch.tensor([0, 1, 41], dtype=torch.int32, device=DEV)
     cache.encode(K, V, cu)
-    q = synthetic.queries(32, 2, Hq, d, torch.bfloat16, DEV)
+    q = synthetic.queries(32, 2, Hq, d, torch.float32, DEV)   # float32 I/O: single heads are looked at
     out = to_f64(cache.attend(q))
     xh = to_f64(cache.dequant(40))
     for h in range(Hq):
-        assert rel_l2(out[0, h], xh[0, 0, 1, 0]) < TOL_ATTENTION          # len 1: the value itself
-        assert rel_l2(out[1, h], xh[1, 0, 1, :40].mean(0)) < 2 * TOL_ATTENTION  # uniform weights: the mean
+        assert rel_l2(out[0, h], xh[0, 0, 1, 0]) < TOL_ATTENTION_F32_IO          # len 1: the value itself
+        assert rel_l2(out[1, h], xh[1, 0, 1, :40].mean(0)) < TOL_ATTENTION_F32_IO  # uniform weights: the mean
 
 
 def test_capacity_overflow_and_empty_sequence_are_reported_not_faulted():
