@@ -165,7 +165,10 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   const int quarter = warp & 3;            // tensor-memory lanes this warp may read: rows 32 * quarter ..
   const int slot = warp >> 2;              // accumulator and tile sequence of this group of four warps
   const int st = quarter * 32 + lane;      // thread index inside the slot = row of the tile
-  const bool leader = st == 0;
+  // The slot's issuing thread (TMA, MMAs).  The four warps of a slot sit on the four schedulers; the issuing threads
+  // of the four slots are spread over them too, so that no scheduler carries all of that extra work (the other
+  // warps of a slot would wait for the slow one at every barrier).
+  const bool leader = quarter == slot && lane == 0;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kTcSmMisc + 4);
   volatile int* copies_issued = reinterpret_cast<volatile int*>(smem + kTcSmMisc + 8);  // [kTcStages]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kTcSmMisc);
