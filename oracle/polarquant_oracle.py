@@ -288,6 +288,34 @@ def decode_attention(q, k_codes, k_radii, v_codes, v_radii, lens, cb: Codebooks,
     return out
 
 
+def multi_query_attention(q, k_codes, k_radii, v_codes, v_radii, lens, cb: Codebooks, S, scale):
+    """Eq. 2 / Eq. 3 for the last ``n_q`` positions of every sequence at once (a chunk of a prefill, or the
+    drafted tokens of a speculative step): in the stream of Section 4 the i-th query attends to the first i
+    tokens, so query ``j`` (0-based) of the chunk sees the cached tokens ``t < lens[b] - (n_q - 1 - j)``; the
+    last query sees all of them.  The keys and values of the chunk itself are already in the cache.
+
+    q  [B, n_q, Hq, d];  the other arguments as in decode_attention.  Returns float64 [B, n_q, Hq, d]
+    (a query that would see no token returns zeros).
+    """
+    q = np.asarray(q, dtype=np.float64)
+    B, n_q, Hq, d = q.shape
+    Hkv = k_codes.shape[1]
+    group = Hq // Hkv
+    out = np.zeros((B, n_q, Hq, d), dtype=np.float64)
+    for b in range(B):
+        n = int(lens[b])
+        for hk in range(Hkv):
+            K_hat = dequant(k_codes[b, hk, :n], k_radii[b, hk, :n], cb, S)
+            V_hat = dequant(v_codes[b, hk, :n], v_radii[b, hk, :n], cb, S)
+            for j in range(n_q):
+                visible = n - (n_q - 1 - j)
+                if visible <= 0:
+                    continue
+                for h in range(hk * group, (hk + 1) * group):
+                    out[b, j, h] = softmax_attention(q[b, j, h], K_hat[:visible], V_hat[:visible], scale)
+    return out
+
+
 def exact_attention(q, K, V, lens, scale):
     """Eq. 2 on the unquantised cache (quality information only, never a parity target).
     K, V: [B, Hkv, capacity, d]."""

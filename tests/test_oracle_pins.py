@@ -392,6 +392,33 @@ def test_exact_attention_special_cases_and_brute_force():
             assert np.allclose(got[b, h], want, atol=1e-13)
 
 
+def test_multi_query_attention_is_the_causal_stream(cb):
+    """The chunk of n_q queries at the end of a sequence: one query reduces to decode attention; in general the
+    result equals a masked softmax over all cached tokens (scores of the tokens a query must not see set to -inf),
+    written here with explicit loops on the dequantised cache."""
+    rng = np.random.default_rng(9)
+    B, Hq, Hkv, d, n_q = 2, 4, 2, 16, 3
+    S = orc.make_rotation(d, 4)
+    cache = orc.OracleCache(B, Hkv, 12, d, cb, S)
+    for b, n in enumerate((9, 2)):
+        cache.encode_chunk(b, rng.normal(size=(n, Hkv, d)), rng.normal(size=(n, Hkv, d)))
+    q = rng.normal(size=(B, n_q, Hq, d))
+    args = (cache.k_codes, cache.k_radii, cache.v_codes, cache.v_radii, cache.lens, cb, S, 0.3)
+    got = orc.multi_query_attention(q, *args)
+    assert np.allclose(orc.multi_query_attention(q[:, -1:], *args)[:, 0], orc.decode_attention(q[:, -1], *args), atol=1e-15)
+    for b in range(B):
+        n = int(cache.lens[b])
+        for h in range(Hq):
+            K = orc.dequant(cache.k_codes[b, h // 2, :n], cache.k_radii[b, h // 2, :n], cb, S)
+            V = orc.dequant(cache.v_codes[b, h // 2, :n], cache.v_radii[b, h // 2, :n], cb, S)
+            for j in range(n_q):
+                last_visible = n - n_q + j           # position of the query's own token
+                w = [math.exp(0.3 * float(K[t] @ q[b, j, h])) if t <= last_visible else 0.0 for t in range(n)]
+                want = sum(w[t] * V[t] for t in range(n)) / sum(w) if sum(w) > 0 else np.zeros(d)
+                assert np.allclose(got[b, j, h], want, atol=1e-13)
+    assert np.all(got[1, 0] == 0)  # sequence 1 holds 2 tokens: the first of 3 queries precedes them all
+
+
 def test_attention_without_quantisation_does_not_depend_on_S():
     d, n = 16, 50
     K, V, q = RNG.standard_normal((n, d)), RNG.standard_normal((n, d)), RNG.standard_normal(d)
