@@ -164,6 +164,23 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
                             void* workspace_dev, int32_t* status_dev, void* stream);
 
 /*
+ * Attention of the last n_q positions of every sequence over the packed cache (Eq. 2 / Eq. 3 for a chunk of a
+ * prefill or the drafted tokens of a speculative step).  The keys and values of those positions are already in
+ * the cache (pq_encode_kv / pq_append_kv ran first); in the stream of Section 4 the i-th query attends to the
+ * first i tokens, so query j (0-based) of a sequence sees the cached tokens t < lens[b] - (n_q - 1 - j), and
+ * the last query sees all lens[b] of them.  n_q = 1 is pq_decode_attention.
+ *   q_dev, out_dev   [batch][n_q][n_q_heads][head_dim] of `io_dtype`
+ *   workspace_dev    pq_workspace_bytes(head_dim, batch * n_q, n_q_heads, n_kv_heads, max_len) bytes
+ * A query that sees no token (lens[b] < n_q - j) yields zeros and records PQ_ERR_EMPTY.  Every query decodes the
+ * cache for itself (the cost is n_q decode attentions); batch * n_q must not exceed 65535.
+ */
+int32_t pq_multi_query_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                                 const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
+                                 const int32_t* cache_lens_dev, int32_t batch, int32_t n_q, int32_t capacity,
+                                 int32_t max_len, float scale, void* out_dev, void* workspace_dev, int32_t* status_dev,
+                                 void* stream);
+
+/*
  * pq_decode_attention for callers that cannot hand over scratch memory.  (The paper has no
  * counterpart; this is a packaging variant of the call above.)
  *

@@ -42,6 +42,9 @@ _SIGNATURES = {
     "pq_decode_attention": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p,
                                       c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p,
                                       c_void_p]),
+    "pq_multi_query_attention": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p,
+                                           c_void_p, c_int32, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p,
+                                           c_void_p, c_void_p]),
     "pq_static_scratch_bytes": (c_int64, []),
     "pq_decode_attention_static": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p,
                                              c_void_p, c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p,
@@ -179,6 +182,18 @@ def pq_decode_attention(S, tables, q, cache, cache_lens, n_kv_heads, capacity, m
            "pq_decode_attention")
 
 
+def pq_multi_query_attention(S, tables, q, cache, cache_lens, n_kv_heads, capacity, max_len, scale, out, workspace,
+                             status, stream=None):
+    """Eq. 2 / 3 for the last n_q positions of every sequence: q, out [B, n_q, Hq, d]; query j sees the cached
+    tokens before and at its own position.  `workspace` must hold pq_workspace_bytes(d, B * n_q, Hq, Hkv, max_len)."""
+    batch, n_q, n_q_heads, d = q.shape
+    assert q.is_contiguous() and out.is_contiguous() and out.shape == q.shape and out.dtype == q.dtype
+    _check(lib().pq_multi_query_attention(d, n_q_heads, n_kv_heads, _ptr(S), _ptr(tables), _ptr(q), _dtype_code(q),
+                                          _ptr(cache), _ptr(cache_lens), batch, n_q, capacity, max_len, float(scale),
+                                          _ptr(out), _ptr(workspace), _ptr(status), _stream(stream)),
+           "pq_multi_query_attention")
+
+
 def pq_static_scratch_bytes() -> int:
     return int(lib().pq_static_scratch_bytes())
 
@@ -246,6 +261,18 @@ class PolarQuantCache:
         pq_decode_attention(self.S, self.tables, q, self.cache, self.lens, self.n_kv_heads, self.capacity,
                             self.capacity if max_len is None else max_len, scale, out, self.workspace, self.status,
                             stream)
+        return out
+
+    def attend_multi(self, q, out=None, scale=None, max_len=None, stream=None):
+        """q [B, n_q, Hq, d]: the last n_q positions of every sequence (already in the cache), causal."""
+        out = torch.empty_like(q) if out is None else out
+        scale = self.d ** -0.5 if scale is None else scale
+        need = pq_workspace_bytes(self.d, self.batch * q.shape[1], self.n_q_heads, self.n_kv_heads, self.capacity)
+        if getattr(self, "_multi_ws", None) is None or self._multi_ws.numel() < need:
+            self._multi_ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        pq_multi_query_attention(self.S, self.tables, q, self.cache, self.lens, self.n_kv_heads, self.capacity,
+                                 self.capacity if max_len is None else max_len, scale, out, self._multi_ws, self.status,
+                                 stream)
         return out
 
     def unpack(self, n_tokens):

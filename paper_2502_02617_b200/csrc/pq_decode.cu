@@ -124,6 +124,8 @@ constexpr int kMaxGroup = 8;  // query heads per kv head handled by one CTA
 
 struct DecodeArgs {
   int d, n_q_heads, n_kv_heads, batch, capacity, io_dtype;
+  int n_q;  // queries per sequence (1: decode).  `batch` counts (sequence, query) pairs: q and out are
+            // [batch][n_q_heads][d] with pair p = sequence * n_q + query; `lens` and the cache are per sequence.
   float scale;
   uint32_t epoch;  // differs from call to call (top bit set): tags the split tickets of the persistent kernel
   uint32_t debug;  // bit 0: test hook, the first bounded wait of CTA 0 of the persistent kernel reports failure
@@ -135,6 +137,14 @@ struct DecodeArgs {
   void* out;
   int32_t* status;
   Workspace ws;
+  // Sequence of (sequence, query) pair p, and the cached tokens its query sees: query j of the n_q last positions of
+  // a sequence attends to the tokens before and at its own position (Section 4: the i-th query sees i tokens).
+  __device__ __forceinline__ int seq_of(int p) const { return n_q == 1 ? p : p / n_q; }
+  __device__ __forceinline__ int visible_len(int p) const {
+    if (n_q == 1) return lens[p];
+    const int b = p / n_q, v = lens[b] - (n_q - 1 - (p - b * n_q));
+    return v > 0 ? v : 0;
+  }
 };
 
 // q' = (q . S) * scale * log2(e); also clears the split tickets.
@@ -283,12 +293,12 @@ __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel
 #pragma unroll
   for (int h = 0; h < kMaxGroup; ++h) o_acc[h] = 0.f;
 
-  const int len = a.lens[b];
+  const int len = a.visible_len(b);
   const int nblk_total = len > 0 ? (len + kTokenBlock - 1) / kTokenBlock : 0;
   const int per = (nblk_total + a.ws.n_splits - 1) / a.ws.n_splits;
   const int j0 = split * per;
   const int j1 = min(nblk_total, j0 + per);
-  const uint8_t* head_base = a.cache + ((int64_t)b * a.n_kv_heads + hk) * L.head_bytes;
+  const uint8_t* head_base = a.cache + ((int64_t)a.seq_of(b) * a.n_kv_heads + hk) * L.head_bytes;
   __syncthreads();
 
   for (int jb = j0; jb < j1; ++jb) {
@@ -470,36 +480,37 @@ int64_t pq_workspace_bytes(int32_t head_dim, int32_t batch, int32_t n_q_heads, i
   return pq::carve_workspace(nullptr, head_dim, batch, n_q_heads, n_kv_heads, max_len).bytes;
 }
 
-int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
-                            const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
-                            const int32_t* cache_lens_dev, int32_t batch, int32_t capacity, int32_t max_len,
-                            float scale, void* out_dev, void* workspace_dev, int32_t* status_dev, void* stream) {
+static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                                const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
+                                const int32_t* cache_lens_dev, int32_t batch, int32_t n_q, int32_t capacity, int32_t max_len,
+                                float scale, void* out_dev, void* workspace_dev, int32_t* status_dev, void* stream) {
   if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
   if (!S_dev || !tables_dev || !q_dev || !cache_dev || !cache_lens_dev || !out_dev || !workspace_dev || !status_dev)
     return PQ_ERR_INVALID_ARG;
-  if (batch <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || capacity <= 0 || max_len <= 0) return PQ_ERR_INVALID_ARG;
+  if (batch <= 0 || n_q <= 0 || n_q_heads <= 0 || n_kv_heads <= 0 || capacity <= 0 || max_len <= 0) return PQ_ERR_INVALID_ARG;
   if (n_q_heads % n_kv_heads) return PQ_ERR_INVALID_ARG;
   if (n_q_heads / n_kv_heads > pq::kMaxGroup) return PQ_ERR_UNSUPPORTED;
   if (io_dtype != PQ_DTYPE_F32 && io_dtype != PQ_DTYPE_BF16) return PQ_ERR_UNSUPPORTED;
   const uintptr_t bits = (uintptr_t)S_dev | (uintptr_t)tables_dev | (uintptr_t)q_dev | (uintptr_t)cache_dev |
                          (uintptr_t)out_dev | (uintptr_t)workspace_dev;
   if (bits & 15) return PQ_ERR_ALIGNMENT;
-  if (batch > 65535 || n_kv_heads > 65535) return PQ_ERR_UNSUPPORTED;
+  const int64_t pairs = (int64_t)batch * n_q;  // (sequence, query) pairs: the kernels' batch
+  if (pairs > 65535 || n_kv_heads > 65535) return PQ_ERR_UNSUPPORTED;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(stream);
   pq::DecodeArgs a;
-  a.d = head_dim; a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads; a.batch = batch; a.capacity = capacity;
+  a.d = head_dim; a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads; a.batch = (int)pairs; a.n_q = n_q; a.capacity = capacity;
   a.io_dtype = io_dtype; a.scale = scale; a.S = S_dev; a.tables = reinterpret_cast<const pq::Tables*>(tables_dev);
   a.q = q_dev; a.cache = reinterpret_cast<const uint8_t*>(cache_dev); a.lens = cache_lens_dev; a.out = out_dev;
   a.status = status_dev;
-  a.ws = pq::carve_workspace(workspace_dev, head_dim, batch, n_q_heads, n_kv_heads, max_len);
+  a.ws = pq::carve_workspace(workspace_dev, head_dim, (int)pairs, n_q_heads, n_kv_heads, max_len);
   const int g = n_q_heads / n_kv_heads;
-  if (head_dim == 128 && batch * n_kv_heads <= pq::kFastMaxUnits) {
+  if (head_dim == 128 && pairs * n_kv_heads <= pq::kFastMaxUnits) {
     // One launch: the persistent kernel rotates the queries itself and needs no cleared tickets.
     // The tickets in the (uninitialised, possibly shared) scratch are tagged with a per-call number.  It starts
     // at a value drawn from the clock and the address space of this process, advances by an odd constant and
     // always has its top bit set, so it cannot equal a small integer that another kernel left in the same bytes.
     static std::atomic<uint32_t> call_epoch{[] {
-      uint64_t x = (uint64_t)std::chrono::steady_clock::now().time_since_epoch().count() ^ (uint64_t)(uintptr_t)&pq_decode_attention;
+      uint64_t x = (uint64_t)std::chrono::steady_clock::now().time_since_epoch().count() ^ (uint64_t)(uintptr_t)&launch_attention;
       x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
       x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
       return (uint32_t)(x ^ (x >> 31));
@@ -517,15 +528,32 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
   }
   a.epoch = 0u;
   a.debug = 0u;
-  pq::rotate_query_kernel<<<batch * n_q_heads, head_dim, head_dim * sizeof(float), st>>>(a);
+  pq::rotate_query_kernel<<<(unsigned)pairs * n_q_heads, head_dim, head_dim * sizeof(float), st>>>(a);
   const pq::Layout L = pq::make_layout(head_dim, capacity);
   size_t smem = 2 * L.block_bytes + sizeof(float) * ((size_t)g * head_dim + 3 * g * pq::kTokenBlock +
                                                      3 * pq::kMaxGroup + 64);
   const size_t smem_combine = sizeof(float) * pq::combine_smem_floats(g, head_dim, a.ws.n_splits);
   if (smem < smem_combine) smem = smem_combine;
-  dim3 grid(a.ws.n_splits, n_kv_heads, batch);
+  dim3 grid(a.ws.n_splits, n_kv_heads, (unsigned)pairs);
   pq::decode_attention_simple_kernel<<<grid, pq::kSimpleThreads, smem, st>>>(a);
   return pq::launch_status();
+}
+
+int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                            const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
+                            const int32_t* cache_lens_dev, int32_t batch, int32_t capacity, int32_t max_len,
+                            float scale, void* out_dev, void* workspace_dev, int32_t* status_dev, void* stream) {
+  return launch_attention(head_dim, n_q_heads, n_kv_heads, S_dev, tables_dev, q_dev, io_dtype, cache_dev, cache_lens_dev,
+                          batch, 1, capacity, max_len, scale, out_dev, workspace_dev, status_dev, stream);
+}
+
+int32_t pq_multi_query_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                                 const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
+                                 const int32_t* cache_lens_dev, int32_t batch, int32_t n_q, int32_t capacity,
+                                 int32_t max_len, float scale, void* out_dev, void* workspace_dev, int32_t* status_dev,
+                                 void* stream) {
+  return launch_attention(head_dim, n_q_heads, n_kv_heads, S_dev, tables_dev, q_dev, io_dtype, cache_dev, cache_lens_dev,
+                          batch, n_q, capacity, max_len, scale, out_dev, workspace_dev, status_dev, stream);
 }
 
 // ---- decode attention on the library's own scratch ---------------------------------------------

@@ -311,7 +311,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
       *first_rank = 0x7fffffff;
     }
     for (int u = tid; u < n_units; u += kFastThreads) {
-      const int len_u = a.lens[u / a.n_kv_heads];
+      const int len_u = a.visible_len(u / a.n_kv_heads);
       u_nst[u] = len_u > 0 ? (len_u + kStageTokens - 1) / kStageTokens : 0;
     }
     __syncthreads();
@@ -398,9 +398,9 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     const int u = segs[sg].unit, st0 = segs[sg].st0, st1 = segs[sg].st1;
     const int n_parts = segs[sg].n_parts, unit_slot = segs[sg].slot0, c_first = cta - segs[sg].part;
     const int b = u / a.n_kv_heads, hk = u - b * a.n_kv_heads;
-    const int len = a.lens[b];
+    const int len = a.visible_len(b);   // b counts (sequence, query) pairs: see DecodeArgs
     const int nblk_total = (len + kTokenBlock - 1) / kTokenBlock;
-    const uint8_t* head_base = a.cache + ((int64_t)b * a.n_kv_heads + hk) * head_bytes;
+    const uint8_t* head_base = a.cache + ((int64_t)a.seq_of(b) * a.n_kv_heads + hk) * head_bytes;
 
     // per-thread attention state
     // o_acc[hg][S][.]: head c + 4 hg, block g, coordinates 4S, 4S + 2, 4S + 1, 4S + 3 (see the value MMAs)

@@ -182,6 +182,43 @@ def test_attention_special_cases_len1_and_identical_keys():
         assert rel_l2(out[1, h], xh[1, 0, 1, :40].mean(0)) < TOL_ATTENTION_F32_IO  # uniform weights: the mean
 
 
+@pytest.mark.parametrize("d,Hq,Hkv,n_q", [(128, 8, 2, 5), (128, 8, 1, 3), (16, 4, 2, 4)])
+def test_multi_query_attention_is_causal_over_the_last_positions(d, Hq, Hkv, n_q):
+    """The last n_q positions of every sequence attend at once; query j sees the tokens up to its own position.
+    Float32 I/O against the oracle per query, and n_q = 1 equals decode attention bit for bit."""
+    lens_list = [300, 70, 3]   # the last sequence is shorter than the chunk: its first queries see nothing
+    B = len(lens_list)
+    cache = pq.PolarQuantCache(B, Hq, Hkv, d, capacity=320, seed=21, device=DEV)
+    K, V = synthetic.kv_like(22, sum(lens_list), Hkv, d, torch.bfloat16, DEV)
+    _encode_and_compare(cache, K, V, lens_list)
+    ref = _oracle_cache(cache, K, V, lens_list)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(23)
+    q = torch.randn((B, n_q, Hq, d), generator=g, device=DEV, dtype=torch.float32)
+    out = cache.attend_multi(q)
+    torch.cuda.synchronize()
+    want = orc.multi_query_attention(to_f64(q), ref.k_codes, ref.k_radii, ref.v_codes, ref.v_radii, ref.lens, ref.cb,
+                                     ref.S, d ** -0.5)
+    got = to_f64(out)
+    for b in range(B):
+        for j in range(n_q):
+            if lens_list[b] - (n_q - 1 - j) <= 0:
+                assert np.all(got[b, j] == 0)
+            else:
+                assert rel_l2(got[b, j], want[b, j]) < TOL_ATTENTION_F32_IO, (b, j)
+    assert cache.status.cpu().tolist()[0] in (pq.OK, pq.ERR_EMPTY)
+    cache.status.zero_()
+    one = cache.attend_multi(q[:, -1:].contiguous())
+    assert torch.equal(one[:, 0], cache.attend(q[:, -1].contiguous()))
+    qb = q.to(torch.bfloat16)
+    assert rel_l2(to_f64(cache.attend_multi(qb))[:2], want_bf16(orc, ref, qb, d)[:2]) < TOL_ATTENTION
+
+
+def want_bf16(orc, ref, qb, d):
+    return orc.multi_query_attention(to_f64(qb), ref.k_codes, ref.k_radii, ref.v_codes, ref.v_radii, ref.lens, ref.cb, ref.S,
+                                     d ** -0.5)
+
+
 def test_capacity_overflow_and_empty_sequence_are_reported_not_faulted():
     d, Hq, Hkv = 128, 4, 1
     cache = pq.PolarQuantCache(2, Hq, Hkv, d, capacity=64, seed=7, device=DEV)
