@@ -171,8 +171,10 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
  * the last query sees all lens[b] of them.  n_q = 1 is pq_decode_attention.
  *   q_dev, out_dev   [batch][n_q][n_q_heads][head_dim] of `io_dtype`
  *   workspace_dev    pq_workspace_bytes(head_dim, batch * n_q, n_q_heads, n_kv_heads, max_len) bytes
- * A query that sees no token (lens[b] < n_q - j) yields zeros and records PQ_ERR_EMPTY.  Every query decodes the
- * cache for itself (the cost is n_q decode attentions); batch * n_q must not exceed 65535.
+ * A query that sees no token (lens[b] < n_q - j) yields zeros and records PQ_ERR_EMPTY.  At head_dim 128, chunks
+ * of at least 64 / (n_q_heads / n_kv_heads) queries run on a kernel that decodes every block of the cache once for 64
+ * (query, head) rows and contracts on tensor cores (no workspace is touched); shorter chunks and other head_dims
+ * decode the cache once per query (the cost is n_q decode attentions).  batch * n_q must not exceed 65535.
  */
 int32_t pq_multi_query_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
                                  const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,

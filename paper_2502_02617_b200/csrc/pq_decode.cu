@@ -403,6 +403,7 @@ __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel
 
 }  // namespace pq
 #include "pq_decode_fast.cuh"
+#include "pq_prefill.cuh"
 namespace pq {
 
 // ---- inspection kernels ----------------------------------------------------------------------
@@ -504,6 +505,15 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
   a.status = status_dev;
   a.ws = pq::carve_workspace(workspace_dev, head_dim, (int)pairs, n_q_heads, n_kv_heads, max_len);
   const int g = n_q_heads / n_kv_heads;
+  if (head_dim == 128 && n_q * g >= pq::kPfRows) {
+    // Many queries per sequence: decode each block of the cache once for 64 (query, head) rows on tensor cores.
+    static pq::DeviceMemo configured_pf;
+    if (pq::configure_for_device(pq::prefill_attention_kernel, pq::kPfTotal, configured_pf) == 0) return PQ_ERR_CUDA;
+    const int qb_rows = pq::kPfRows / g;
+    dim3 grid((n_q + qb_rows - 1) / qb_rows, n_kv_heads, batch);
+    pq::prefill_attention_kernel<<<grid, pq::kPfThreads, pq::kPfTotal, st>>>(a, n_q);
+    return pq::launch_status();
+  }
   if (head_dim == 128 && pairs * n_kv_heads <= pq::kFastMaxUnits) {
     // One launch: the persistent kernel rotates the queries itself and needs no cleared tickets.
     // The tickets in the (uninitialised, possibly shared) scratch are tagged with a per-call number.  It starts

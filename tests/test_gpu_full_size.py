@@ -109,6 +109,33 @@ def test_config2_every_code_against_the_oracle():
     assert_radii_match(counts=(radii_off, radii_n))
 
 
+def test_chunk_of_64_queries_over_a_config3_cache():
+    """Multi-query attention at full size: the last 64 positions of two 32768-token sequences (32 q / 8 kv heads)
+    attend causally; all 64 queries of sampled (sequence, kv head) units against the oracle."""
+    B, n, n_q = 2, 32768, 64
+    cache = pq.PolarQuantCache(B, HQ, HKV, D, capacity=n, seed=1, device=DEV)
+    for b in range(B):
+        K, V = synthetic.kv_like(10 + b, n, HKV, D, torch.bfloat16, DEV)
+        cu = torch.zeros(B + 1, dtype=torch.int32, device=DEV)
+        cu[b + 1:] = n
+        cache.encode(K, V, cu)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(64)
+    q = torch.randn((B, n_q, HQ, D), generator=g, device=DEV, dtype=torch.float32).to(torch.bfloat16)
+    out = cache.attend_multi(q)
+    torch.cuda.synchronize()
+    cache.check_status()
+    assert torch.equal(out, cache.attend_multi(q))
+    codes, radii = cache.unpack(n)
+    cb, S = oracle_codebooks(cache), cache.S_host.double().numpy()
+    grp = HQ // HKV
+    for b, hk in ((0, 2), (1, 7)):
+        c, r = codes[b, hk].cpu().numpy(), radii[b, hk].cpu().numpy()
+        want = orc.multi_query_attention(to_f64(q[b:b + 1, :, hk * grp:(hk + 1) * grp]), c[0][None, None], r[0][None, None],
+                                         c[1][None, None], r[1][None, None], [n], cb, S, D ** -0.5)[0]
+        assert rel_l2(to_f64(out[b, :, hk * grp:(hk + 1) * grp]), want) < TOL_ATTENTION, (b, hk)
+
+
 def test_config4_long_context_layers():
     """Three layers of the long-context shape (batch 1, 131072 tokens, 32 q / 8 kv heads), each from its own seed,
     sharing S and the codebooks as the layers of a model do; the benchmark runs 36 of them back to back."""

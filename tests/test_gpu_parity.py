@@ -182,7 +182,8 @@ def test_attention_special_cases_len1_and_identical_keys():
         assert rel_l2(out[1, h], xh[1, 0, 1, :40].mean(0)) < TOL_ATTENTION_F32_IO  # uniform weights: the mean
 
 
-@pytest.mark.parametrize("d,Hq,Hkv,n_q", [(128, 8, 2, 5), (128, 8, 1, 3), (16, 4, 2, 4)])
+@pytest.mark.parametrize("d,Hq,Hkv,n_q", [(128, 8, 2, 5), (128, 8, 1, 3), (16, 4, 2, 4),            # one decode per query
+                                           (128, 8, 2, 40), (128, 8, 1, 9), (128, 6, 2, 22), (128, 2, 2, 70)])  # tensor-core kernel
 def test_multi_query_attention_is_causal_over_the_last_positions(d, Hq, Hkv, n_q):
     """The last n_q positions of every sequence attend at once; query j sees the tokens up to its own position.
     Float32 I/O against the oracle per query, and n_q = 1 equals decode attention bit for bit."""
