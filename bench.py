@@ -455,6 +455,37 @@ def measure_config4(args, pq, synthetic, dev, rank):
     return res
 
 
+def measure_multi_query(args, pq, synthetic, dev, rank):
+    """A chunk of 64 queries per sequence over a config-3 cache (batch 8 x 32768 tokens): multi-query attention."""
+    n_q = 64
+    cache = pq.PolarQuantCache(BATCH, HQ, HKV, D, CTX, seed=0, device=dev)
+    for b in range(BATCH):
+        K, V = synthetic.kv_like(1000 * rank + 10 + b % 2, CTX, HKV, D, torch.bfloat16, dev)
+        cu = torch.zeros(BATCH + 1, dtype=torch.int32, device=dev)
+        cu[b + 1:] = CTX
+        cache.encode(K, V, cu)
+    g = torch.Generator(device=dev)
+    g.manual_seed(640 + rank)
+    q = torch.randn((BATCH, n_q, HQ, D), generator=g, device=dev, dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty_like(q)
+    stream = torch.cuda.current_stream()
+    for _ in range(2):
+        cache.attend_multi(q, out=out)
+    evs = [(_event(), _event()) for _ in range(8)]
+    for a, b in evs:
+        a.record(stream)
+        cache.attend_multi(q, out=out)
+        b.record(stream)
+    torch.cuda.synchronize()
+    cache.check_status()
+    t = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    pairs = BATCH * n_q * HQ * (CTX - (n_q - 1) / 2.0)          # (query head, visible token) pairs
+    return {"batch": BATCH, "ctx": CTX, "n_q": n_q, "ms": t, "us_per_query": t / n_q * 1e3,
+            "mma_tflops": pairs * 512 * 2 / (t * 1e-3) / 1e12,
+            "mma_flops_definition": "4 x 128 multiply-adds per (query head, visible token): Q'K^T with the key as fp16 value + "
+                                    "residual and the query likewise (3 products), and PV"}
+
+
 def measure_config5(args, pq, synthetic, dev, rank):
     """Config 5: batch 16, ragged contexts in [4096, 65536], prefill in 4096-token chunks, then 128 steps of
     (append one token per sequence, decode attention)."""
@@ -517,11 +548,13 @@ def reduce_and_format(local, steps, warmup, rank, world, dist=None, device="cpu"
     head = local["headline"]
     keys = ["total_ms", "e2e_total_ms"]
     flat = [head[k] for k in keys] + head["seg_ms"] + head["seg_best_ms"] + head["e2e_seg_ms"]
-    c4, c5 = local.get("cfg4"), local.get("cfg5")
+    c4, c5, mq = local.get("cfg4"), local.get("cfg5"), local.get("multi_query")
     if c4:
         flat += [c4["decode_step_ms"], c4["decode_step_best_ms"], c4["encode_ms_per_layer"]]
     if c5:
         flat += [c5["total_ms_128_steps"], c5["append_ms"], c5["decode_ms"]]
+    if mq:
+        flat += [mq["ms"]]
     red = sharding.max_over_ranks(flat, dist, device)
     total_ms, e2e_total_ms = red[0], red[1]
     enc_ms, app_ms, dec_ms = red[2:5]
@@ -581,9 +614,14 @@ def reduce_and_format(local, steps, warmup, rank, world, dist=None, device="cpu"
                                        frac_of_nominal_8TBs=gbs / 8000.0)
     if c5:
         t, ta, td = red[pos:pos + 3]
+        pos_mq = pos + 3
         gbs = c5["compressed_bytes_per_step"] / (td * 1e-3) / 1e9
         line["configs"]["cfg5"] = dict(c5, total_ms_128_steps=t, ms_per_step=t / c5["steps"], append_ms=ta, decode_ms=td,
                                        decode_gbs=gbs, hbm_frac_measured=gbs / peak, frac_of_nominal_8TBs=gbs / 8000.0)
+    if mq:
+        t = red[pos_mq if c5 else pos]
+        line["configs"]["multi_query_chunk"] = dict(mq, ms=t, us_per_query=t / mq["n_q"] * 1e3,
+                                                    mma_tflops=mq["mma_tflops"] * mq["ms"] / t)
     if cpu_baseline is not None:
         line["cpu_baseline"] = cpu_baseline
     return line
@@ -609,6 +647,8 @@ def run_cuda(args):
         local["cfg4"] = measure_config4(args, pq, synthetic, dev, rank)
         torch.cuda.empty_cache()
         local["cfg5"] = measure_config5(args, pq, synthetic, dev, rank)
+        torch.cuda.empty_cache()
+        local["multi_query"] = measure_multi_query(args, pq, synthetic, dev, rank)
         torch.cuda.empty_cache()
     cpu = _oracle_sample_throughput(12.0) if rank == 0 and world == 1 and not args.no_cpu_baseline else None
     line = reduce_and_format(local, args.steps, args.warmup, rank, world, dist, dev, cpu)
