@@ -22,7 +22,9 @@ Pins (tests/test_oracle_*.py): exact invertibility of the unquantised transform,
 block radius == block norm, norm preservation under S, Lemma 2 densities against the
 incomplete-beta CDF, Lloyd-Max fixed-point equations against independent quadrature,
 the worked d=4 example under tests/golden/, brute force on d=4 and d=16, closed-form
-expected distortion, and the len=1 / identical-keys attention special cases.
+expected distortion, the len=1 / identical-keys attention special cases, multi-query attention against a
+masked softmax, and the online codebook (histogram counts, k-means fixed point, two-cluster toy, convergence to the
+analytic codebook on samples of the analytic density).
 Parity unpinned: nothing in this file; quality on real model caches is out of scope.
 """
 from __future__ import annotations
@@ -166,6 +168,62 @@ def fit_codebooks(bits=DEFAULT_BITS) -> Codebooks:
     cents, bounds = [], []
     for level, b in enumerate(bits, start=1):
         c, t = lloyd_max(level, b)
+        cents.append(c)
+        bounds.append(t)
+    return Codebooks(tuple(bits), tuple(cents), tuple(bounds))
+
+
+# --------------------------------------------------------------------------------------
+# "Online" codebook (Section 4.1): clustering of the observed angles of one prompt and layer
+# --------------------------------------------------------------------------------------
+def angle_histograms(x: np.ndarray, S: np.ndarray, n_levels: int, n_bins: int) -> np.ndarray:
+    """The angles that Polar (Algorithm 1) produces for the rows of ``x`` ([n, d]; keys and values of the
+    prompt stacked), counted per level in ``n_bins`` bins of equal width over the level's range ([0, 2 pi) at level
+    1, [0, pi/2] above).  The histogram is the sample the clustering runs on: an angle stands for the centre of
+    its bin.  Returns int64 [n_levels, n_bins]."""
+    angles, _ = polar(rotate(x, S), n_levels)
+    hist = np.zeros((n_levels, n_bins), dtype=np.int64)
+    for level in range(1, n_levels + 1):
+        width = (TWO_PI if level == 1 else HALF_PI) / n_bins
+        idx = np.minimum((angles[level - 1].ravel() / width).astype(np.int64), n_bins - 1)
+        hist[level - 1] = np.bincount(idx, minlength=n_bins)
+    return hist
+
+
+def kmeans_on_histogram(counts: np.ndarray, level: int, init: np.ndarray, max_iter: int = 10000):
+    """1-D k-means (Lloyd's iteration) on binned samples: the discrete form of Eq. 4, with the bin centres as
+    sample values and the counts as weights.  Alternates (cell boundaries = midpoints of adjacent centroids) and
+    (centroid = weighted mean of the bin centres in its cell; an empty cell keeps its centroid) until nothing moves.
+    k-means++ in the paper is a randomised choice of the starting centroids; this reading starts from ``init``
+    (the analytic codebook of the level), which makes the result a function of the data alone.  Distances are taken
+    on the line, also at level 1, as Quant is printed.  Returns (centroids, interior boundaries)."""
+    counts = np.asarray(counts, dtype=np.float64)
+    n_bins = counts.size
+    width = (TWO_PI if level == 1 else HALF_PI) / n_bins
+    centres = (np.arange(n_bins) + 0.5) * width
+    theta = np.array(init, dtype=np.float64)
+    for _ in range(max_iter):
+        beta = 0.5 * (theta[:-1] + theta[1:])
+        cell = np.searchsorted(beta, centres, side="left")      # number of boundaries below the bin centre
+        new = theta.copy()
+        for k in range(theta.size):
+            w = counts[cell == k]
+            if w.sum() > 0:
+                new[k] = float(np.sum(w * centres[cell == k]) / w.sum())
+        if np.array_equal(new, theta):
+            break
+        theta = new
+    return theta, 0.5 * (theta[:-1] + theta[1:])
+
+
+def fit_codebooks_online(x: np.ndarray, S: np.ndarray, bits=DEFAULT_BITS, n_bins: int = 4096) -> Codebooks:
+    """Algorithm 1 line 3 with the "online" codebook of Section 4.1: per level, k-means on the observed angles of
+    this input (binned), started from the analytic codebook."""
+    offline = fit_codebooks(bits)
+    hist = angle_histograms(x, S, len(bits), n_bins)
+    cents, bounds = [], []
+    for level in range(1, len(bits) + 1):
+        c, t = kmeans_on_histogram(hist[level - 1], level, offline.centroids[level - 1])
         cents.append(c)
         bounds.append(t)
     return Codebooks(tuple(bits), tuple(cents), tuple(bounds))

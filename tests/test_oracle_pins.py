@@ -185,6 +185,64 @@ def test_level1_cost_closed_form(cb):
     assert abs(mse - (math.pi / 8) ** 2 / 12) < 1e-14
 
 
+# ---------------------------------------------------------------- online codebook (Section 4.1)
+def test_angle_histograms_count_every_angle_in_its_bin():
+    S = np.eye(4)
+    x = np.array([[3.0, 4.0, -8.0, 6.0], [1.0, 0.0, 0.0, -1.0]])     # level-1 angles: atan2(4,3), atan2(6,-8); 0, 3pi/2
+    h = orc.angle_histograms(x, S, 2, 8)
+    assert h.shape == (2, 8) and h[0].sum() == 4 and h[1].sum() == 2
+    # bins of width pi/4: 0.927 -> 1, 2.498 -> 3, 0 -> 0, 3pi/2 -> 6
+    assert h[0].tolist() == [1, 1, 0, 1, 0, 0, 1, 0]
+    # level 2: atan2(10, 5) = 1.107 and atan2(1, 1) = pi/4, bins of width pi/16: 5 and 4
+    assert h[1].tolist() == [0, 0, 0, 0, 1, 1, 0, 0]
+
+
+def test_kmeans_on_histogram_fixed_point_toy_and_analytic_limit(cb):
+    # two well separated clumps: the centroids are the clumps' weighted means, whatever the start
+    counts = np.zeros(64)
+    counts[[3, 4]] = [10, 30]
+    counts[[40, 41, 42]] = [5, 5, 10]
+    width = (math.pi / 2) / 64
+    theta, beta = orc.kmeans_on_histogram(counts, 2, np.array([0.5, 0.6]))
+    assert np.allclose(theta, [(10 * 3.5 + 30 * 4.5) / 40 * width, (5 * 40.5 + 5 * 41.5 + 10 * 42.5) / 20 * width], atol=1e-15)
+    assert np.allclose(beta, [theta.mean()], atol=1e-15)
+    # a histogram of the analytic density itself: the result is the analytic codebook up to the binning (each of
+    # the n_c stationarity equations holds to half a bin, and the slack adds up along the chain of cells), it is a
+    # fixed point (every centroid is the mean of its cell), and the discrete Eq. 4 cost does not exceed the start's
+    for level in (1, 2, 4):
+        n_bins, n_c = 4096, cb.centroids[level - 1].size
+        hi = 2 * math.pi if level == 1 else math.pi / 2
+        centres = (np.arange(n_bins) + 0.5) * hi / n_bins
+        k = 2 ** (level - 1)
+        dens = np.ones(n_bins) if level == 1 else np.sin(2 * centres) ** (k - 1)
+        counts = np.round(dens / dens.sum() * 5e7)
+        theta, beta = orc.kmeans_on_histogram(counts, level, cb.centroids[level - 1] + 0.01)
+        assert theta.size == n_c and np.allclose(theta, cb.centroids[level - 1], atol=n_c * hi / n_bins)
+        cell = np.searchsorted(beta, centres)
+        for j in range(n_c):
+            assert abs(theta[j] - np.average(centres[cell == j], weights=counts[cell == j])) < 1e-12
+        cost = lambda t: np.sum(counts * np.min((centres[:, None] - t[None, :]) ** 2, axis=1))
+        assert cost(theta) <= cost(cb.centroids[level - 1] + 0.01)
+
+
+def test_online_codebook_follows_the_data():
+    """Gaussian data give back (nearly) the analytic codebook; data that are not isotropic after the rotation move
+    it, and the fitted codebook then encodes those data with a smaller error than the analytic one."""
+    rng = np.random.default_rng(12)
+    d = 16
+    S = orc.make_rotation(d, 1)
+    offline = orc.fit_codebooks()
+    x = rng.normal(size=(20000, d))
+    online = orc.fit_codebooks_online(x, S)
+    for level in range(4):
+        # level 1: 16 cells of width 0.39 on a flat density, where sampling noise moves the optimum most
+        assert np.allclose(online.centroids[level], offline.centroids[level], atol=0.08 if level == 0 else 0.02)
+    skew = x * np.linspace(0.2, 3.0, d)[None, :] @ S.T        # anisotropic in the rotated basis
+    online = orc.fit_codebooks_online(skew, S)
+    err = lambda cbk: np.mean(np.sum((orc.dequant(*orc.encode(skew, S, cbk)[:2], cbk, S) - skew) ** 2, axis=1))
+    assert err(online) < 0.97 * err(offline)
+
+
 # ---------------------------------------------------------------- radii (b_FPN = 16)
 def test_radius_rounding_is_round_to_nearest_even_and_saturates():
     """binary16 spacing in [1, 2) is 2^-10: a value 3/4 of the way up rounds up (truncation would not), exact ties
