@@ -19,6 +19,9 @@ constexpr int kBlockDim = 16;    // coordinates per polar block (L = 4 levels)
 __host__ __device__ constexpr int cen_off(int level) { return level == 1 ? 0 : 16 + 4 * (level - 2); }
 __host__ __device__ constexpr int bnd_off(int level) { return level == 1 ? 0 : 15 + 3 * (level - 2); }
 
+constexpr int kL1Cells = 128;            // cells per octant of the level-1 decision table
+constexpr float kL1CellScale = 127.93f;  // cell = floor(t * kL1CellScale + 1/16): t = 1 still falls in the last cell
+
 // Compiled form of the codebooks (built on the host by pq_build_tables, copied verbatim to
 // the device by the caller).
 struct Tables {
@@ -50,6 +53,11 @@ struct Tables {
   uint2 t1p_hi[256];
   uint2 t1p_lo[256];
   uint32_t reserved[30];
+  // Level-1 decision table for any codebook (see quant_level1_table_push): octant o = (b < 0) << 2 | (a < 0) << 1 |
+  // (|b| > |a|), cell = position of t = min(|a|,|b|) / max(|a|,|b|) in [0, 1].  .x = float bits of tau, the
+  // one boundary value of t the cell decides against (NaN: the cell cannot be decided by one comparison);
+  // .y = code for t < tau in bits 28..31, code for t > tau in bits 24..27.
+  uint2 l1_cells[8][kL1Cells];
 };
 
 constexpr uint32_t kFlagUniformL1 = 1u;

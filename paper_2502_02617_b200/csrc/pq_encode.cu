@@ -204,7 +204,7 @@ __device__ __forceinline__ void store_half_token(uint8_t* tb, int tok, int half,
 
 // Quantise and store the 4 blocks of (row, half) whose rotated coordinates are y[64]; ambiguous
 // decisions go to the fix-up queue.  Returns the ambiguity bits that did not fit (4 x 15 bits).
-__device__ __forceinline__ void quantise_and_store(const EncodeArgs& a, const FastQuant& fq, bool uniform_l1, const float* y,
+__device__ __forceinline__ void quantise_and_store(const EncodeArgs& a, const FastQuant& fq, const float* y,
                                                    float row_norm, int row, int head, int kv, int half, bool valid,
                                                    FixQueue* q, uint32_t* left, int64_t* xoff_out, uint8_t** tb_out,
                                                    int* tok_out) {
@@ -212,9 +212,8 @@ __device__ __forceinline__ void quantise_and_store(const EncodeArgs& a, const Fa
   FastBlock fb[4];
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    if (fq.sym) polar_quant_block_fast<true>(y + 16 * i, rm, fq, &fb[i]);
+    if (fq.analytic) polar_quant_block_fast<true>(y + 16 * i, rm, fq, &fb[i]);
     else polar_quant_block_fast<false>(y + 16 * i, rm, fq, &fb[i]);
-    if (!uniform_l1) fb[i].amb |= 0xFFu;  // other level-1 codebooks: decide every level-1 angle exactly
     left[i] = 0u;
   }
   *tb_out = nullptr;
@@ -330,12 +329,11 @@ __global__ void __launch_bounds__(kFfmaThreads) encode_ffma_kernel(EncodeArgs a)
   rowsq[half * 128 + r] = sq;
   __syncthreads();
   const float row_norm = sqrtf(rowsq[r] + rowsq[128 + r]) * 1.0001f;
-  const bool uniform = (a.tables->flags & kFlagUniformL1) != 0u;
   uint32_t left[4];
   int64_t xoff = 0;
   uint8_t* tb = nullptr;
   int tok = 0;
-  quantise_and_store(a, *fq, uniform, y, row_norm, row0 + r, head, kv, half, row0 + r < a.total_tokens, fixq, left, &xoff,
+  quantise_and_store(a, *fq, y, row_norm, row0 + r, head, kv, half, row0 + r < a.total_tokens, fixq, left, &xoff,
                      &tb, &tok);
   unsigned long long leftbits[1] = {0ull};
   if (tb != nullptr) {
@@ -394,9 +392,8 @@ __global__ void __launch_bounds__(128) encode_vector_kernel(EncodeArgs a) {
     float yb[16];
 #pragma unroll
     for (int i = 0; i < 16; ++i) yb[i] = ys[16 * j + i];
-    if (fq.sym) polar_quant_block_fast<true>(yb, make_row_margins(norm, kRotErr, fq), fq, &fb);
+    if (fq.analytic) polar_quant_block_fast<true>(yb, make_row_margins(norm, kRotErr, fq), fq, &fb);
     else polar_quant_block_fast<false>(yb, make_row_margins(norm, kRotErr, fq), fq, &fb);
-    if ((a.tables->flags & kFlagUniformL1) == 0u) fb.amb |= 0xFFu;
   }
   if (__syncthreads_or(fb.amb != 0u)) {
     double accd[4] = {0.0, 0.0, 0.0, 0.0};

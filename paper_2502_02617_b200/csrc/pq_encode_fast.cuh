@@ -1,4 +1,5 @@
-// Fast encoder for head_dim 128 with the uniform level-1 codebook (included by pq_encode.cu).
+// Fast encoder for head_dim 128 (included by pq_encode.cu): sign tests for the analytic codebooks (uniform level 1,
+// symmetric upper levels), a table-driven level 1 and per-boundary upper levels for any other codebook.
 //
 // The rotation y = x . S is computed with float32-grade accuracy (tensor cores with S split into
 // bf16 terms, or float32 FMAs).  Either way |y - y_exact| <= rot_err * ||x||_2 per coordinate:
@@ -23,21 +24,26 @@ namespace pq {
 constexpr float kRotErr = 1.1f * 7.62939453125e-06f;                                  // 1.1 * 2^-17
 constexpr float kRotErrTc = 1.1f * (3.f * 9.5367431640625e-07f + 1.4901161193847656e-08f);  // 1.1 * (3 * 2^-20 + 2^-26)
 
-// Per-call constants of the fast quantiser (uniform level-1 codebook; levels 2..4 from Tables).
+// Per-call constants of the fast quantiser.
 struct FastQuant {
   float t2[3][3];   // tan^2 of the three boundaries of levels 2, 3, 4
   uint32_t sym;     // the boundaries of every level >= 2 are b, pi/4, pi/2 - b (kFlagSymmetricUpper)
+  uint32_t analytic;       // sym and the uniform level-1 codebook: every decision is a sign test
+  const uint2* l1_cells;   // level-1 decision table of any other codebook (Tables::l1_cells)
 };
 
 __device__ inline void load_fast_quant(const Tables* tb, FastQuant* fq) {
   for (int l = 0; l < 3; ++l)
     for (int k = 0; k < 3; ++k) fq->t2[l][k] = (float)tb->bnd_tan2[3 * l + k];
   fq->sym = (tb->flags & kFlagSymmetricUpper) != 0u;
+  fq->analytic = (tb->flags & (kFlagSymmetricUpper | kFlagUniformL1)) == (kFlagSymmetricUpper | kFlagUniformL1);
+  fq->l1_cells = &tb->l1_cells[0][0];
 }
 
 // Per-row constants of the margins (dy = bound on the error of one rotated coordinate of the row).
 struct RowMargins {
   float dy;       // as given
+  float dy3;      // 3.02 dy: threshold of the table-driven level-1 test
   float dy1;      // level-1 threshold: dy plus the float32 roundings of the level-1 tests
   float c[3];     // 8.4 E^2 for levels 2, 3, 4 (E^2 = 2, 4, 8 dy^2)
   float cs[3];    // the same plus the float32-rounding term of the folded (symmetric) test
@@ -54,6 +60,7 @@ __device__ __forceinline__ RowMargins make_row_margins(float norm, float rot_err
   RowMargins m;
   m.dy = rot_err * norm;
   m.dy1 = fmaf(1.8e-7f, norm, m.dy);
+  m.dy3 = fmaxf(3.02f * m.dy, 1e-30f);  // the floor keeps a certified u in the range where the reciprocal is accurate
   const float e2 = m.dy * m.dy, rr = 6.8e-12f * norm * norm;
 #pragma unroll
   for (int l = 0; l < 3; ++l) {
@@ -141,6 +148,38 @@ __device__ __forceinline__ uint32_t level1_codes(uint32_t raw) {
   return c ^ 0x11111111u;
 }
 
+// Level-1 decision for any codebook, from the table Tables::l1_cells.  With u = max(|a|,|b|), v = min(|a|,|b|) and
+// t = v / u, the octant (signs of b, a and |a| - |b|) and the cell of t select one boundary value tau and the codes
+// on its two sides; the table guarantees that |t - tau| does not exceed the distance from t to any boundary ray,
+// measured in the octant's coordinate t_c = tan(angle from the octant's first edge) continued past both edges.
+// Margin: the exact pair differs from (a, b) by at most dy per coordinate, and in the octant's frame (the
+// coordinates with the computed signs and order) its u changes by at most dy and its signed v by at most dy, so its
+// t_c differs from t by at most dy (u + v) / (u (u - dy)) <= 2 dy / (u - dy).  A decision is certified if
+//   |t - tau| u > 3.02 dy + 6e-7 u:
+// the table keeps |t - tau| <= 1, hence u > 3 dy, hence the bound above is below 3 dy / u; 6e-7 covers the float32
+// roundings of t (reciprocal and product: 1.8e-7), of tau (6e-8) and of this test.  The exact point then lies in the
+// same gap between rays as t, in this octant or past one of its edges, and the code is the gap's.
+// u = 0, a NaN in (a, b) or in the margin, or a cell without a single deciding boundary (tau = NaN) leave the
+// pair uncertified.
+// The function appends the 4 code bits to `l1` and one "certified" bit to `ok`.
+__device__ __forceinline__ void quant_level1_table_push(float a, float b, float dy3, const uint2* __restrict__ cells,
+                                                        uint32_t& l1, uint32_t& ok) {
+  const float ax = fabsf(a), ay = fabsf(b);
+  const float u = fmaxf(ax, ay), v = fminf(ax, ay);
+  float ru;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(ru) : "f"(u));
+  const float t = fminf(v * ru, 1.f);  // u = 0 or denormal (ru = inf): t = 1 and |t - tau| u stays below dy3
+  const uint32_t o = push_sign(push_sign(push_sign(0u, __float_as_uint(b)), __float_as_uint(a)), __float_as_uint(ax - ay));
+  // 2^20 + t * scale: the float's unit in the last place is 1/8, so mantissa bits 3.. hold floor(t * scale + 1/16)
+  const uint32_t cell8 = __float_as_uint(fmaf(t, kL1CellScale, 1048576.f)) & (uint32_t)((kL1Cells - 1) << 3);
+  const uint2 e = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const char*>(cells) + (o * (kL1Cells * 8) + cell8)));
+  const float dd = t - __uint_as_float(e.x);
+  const float slack = fmaf(-fabsf(dd), u, fmaf(6e-7f, u, dy3));  // < 0: certified (NaN: not)
+  const uint32_t code = e.y << (dd > 0.f ? 4 : 0);                // the code in bits 28..31
+  l1 = __funnelshift_l(code, l1, 4);
+  ok = push_sign(ok, __float_as_uint(slack));
+}
+
 // The level >= 2 decision (see quant_upper_fast) for symmetric boundaries (T0, 1, 1/T0), folded onto m = min(sa, sb), M = max(sa, sb):
 // only the diagonal (M - m) and the boundary m = T0 M of the point's own side can be the nearest ones, and the
 // margin of the boundary sb = sa / T0 is the one of m = T0 M after multiplying both sides by T0^2.  Every T
@@ -162,17 +201,19 @@ __device__ __forceinline__ void quant_upper_sym_push(float sa, float sb, float T
 
 // Codes, squared radius and ambiguity mask of one block.  Pairs and nodes are visited from the last to the
 // first, so that the bits that are appended end up in canonical order.
-template <bool kSym>
+// kAnalytic: the analytic codebooks (uniform level 1, symmetric upper levels); otherwise any codebook.
+template <bool kAnalytic>
 __device__ __forceinline__ void polar_quant_block_fast(const float* y, const RowMargins& rm, const FastQuant& fq,
                                                        FastBlock* out) {
   float s1[8], s2[4], s3[2];
   uint32_t l1 = 0, l2 = 0, l3 = 0, l4 = 0, ok1 = 0, ok2 = 0, ok3 = 0, ok4 = 0;
 #pragma unroll
   for (int j = 7; j >= 0; --j) {
-    quant_level1_push(y[2 * j], y[2 * j + 1], rm.dy1, l1, ok1);
+    if (kAnalytic) quant_level1_push(y[2 * j], y[2 * j + 1], rm.dy1, l1, ok1);
+    else quant_level1_table_push(y[2 * j], y[2 * j + 1], rm.dy3, fq.l1_cells, l1, ok1);
     s1[j] = fmaf(y[2 * j], y[2 * j], y[2 * j + 1] * y[2 * j + 1]);
   }
-  if (kSym) {
+  if (kAnalytic) {
 #pragma unroll
     for (int j = 3; j >= 0; --j) {
       quant_upper_sym_push(s1[2 * j], s1[2 * j + 1], fq.t2[0][0], rm.cs[0], rm.base[0], l2, ok2);
@@ -201,7 +242,7 @@ __device__ __forceinline__ void polar_quant_block_fast(const float* y, const Row
     l4 = quant_upper_fast(s3[0], s3[1], fq.t2[2], rm.c[2], rm.base[2], &am);
     ok4 = am ? 0u : 1u;
   }
-  out->l1 = level1_codes(l1);
+  out->l1 = kAnalytic ? level1_codes(l1) : l1;
   out->l2 = l2;
   out->l3 = l3;
   out->l4 = l4;

@@ -295,8 +295,7 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
 
   // ---- tile loop of this slot
   constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock, orad = o4 + 2 * kTokenBlock;
-  const bool uniform = (a.tables->flags & kFlagUniformL1) != 0u;
-  const bool sym = fq->sym != 0u;  // uniform over the grid
+  const bool analytic = fq->analytic != 0u;  // uniform over the grid
   const Layout L = make_layout(128, a.capacity);
   const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + slot * 128;
   const int slot_bar = 1 + slot;
@@ -373,7 +372,7 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
         __syncwarp();
       }
       FastBlock fb0, fb1;
-      if (sym) {
+      if (analytic) {
         polar_quant_block_fast<true>(y, rm, *fq, &fb0);
         polar_quant_block_fast<true>(y + 16, rm, *fq, &fb1);
       } else {
@@ -391,10 +390,6 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
       if (c < 2) l2lo |= l2c << (16 * c);
       else l2hi |= l2c << (16 * (c - 2));
       uint32_t amb0 = fb0.amb, amb1 = fb1.amb;
-      if (!uniform) {  // other level-1 codebooks: decide every level-1 angle exactly
-        amb0 |= 0xFFu;
-        amb1 |= 0xFFu;
-      }
       if (tb != nullptr) {
         if (bad_row) fb0.l1 = fb1.l1 = racc = amb0 = amb1 = 0u;
         *reinterpret_cast<uint2*>(tb + tok * 32 + c * 8) = make_uint2(fb0.l1, fb1.l1);

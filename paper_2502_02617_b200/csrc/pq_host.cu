@@ -49,6 +49,111 @@ inline void cell_moments(int level, double lo, double hi, double* m0, double* m1
   *m1 = s1 * h / 3.0;
 }
 
+// ---- level-1 decision table for an arbitrary codebook ---------------------------------------
+// The plane is cut into octants by the signs of a, b and |b| > |a|; inside octant o the angle is
+// psi = B_o + D_o * phi with phi = atan(t), t = min(|a|,|b|) / max(|a|,|b|) in [0, 1].  The 16 rays that separate
+// the level-1 cells (the 15 boundaries and the ray at 0 = 2 pi between code 15 and code 0) are expressed in the
+// octant's own coordinate continued past its edges, t_c = tan(D_o (beta - B_o)), for every ray within
+// [-pi/4, atan 2] of the octant's first edge: a point whose computed t is off by less than 1 is, in this
+// coordinate, still on the same side of every ray it was not moved across.
+// A cell stores one value tau and two codes such that for EVERY t of the cell
+//   (1) |t - tau| is at most the distance from t to every ray (in t_c), and
+//   (2) the code is `lo` for t < tau and `hi` for t > tau,
+// so the kernel decides with one comparison and certifies with one distance.  A cell that cannot offer both
+// (two rays inside or next to it) stores NaN and every decision in it is taken in float64.
+struct L1Ray {
+  double t;
+  int below, above;  // codes on the sides t_c < t and t_c > t
+};
+
+int l1_code_of_angle(const double* bnd, double psi) {
+  int c = 0;
+  for (int k = 0; k < 15; ++k) c += psi > bnd[k];
+  return c;
+}
+
+bool build_l1_cells(const double* bnd, uint2 (*cells)[pq::kL1Cells]) {
+  const double kHalfPi = 0.5 * kPi;
+  for (int o = 0; o < 8; ++o) {
+    const int sb = (o >> 2) & 1, sa = (o >> 1) & 1, sw = o & 1;
+    double B, D;
+    if (!sa && !sb) { B = sw ? kHalfPi : 0.0; D = sw ? -1.0 : 1.0; }
+    else if (sa && !sb) { B = sw ? kHalfPi : kPi; D = sw ? 1.0 : -1.0; }
+    else if (sa && sb) { B = sw ? 3.0 * kHalfPi : kPi; D = sw ? -1.0 : 1.0; }
+    else { B = sw ? 3.0 * kHalfPi : 2.0 * kPi; D = sw ? 1.0 : -1.0; }
+    std::vector<L1Ray> rays;
+    for (int j = 0; j < 16; ++j) {
+      const double ang = j == 0 ? 0.0 : bnd[j - 1];
+      double phi = std::remainder(D * (ang - B), 2.0 * kPi);  // in [-pi, pi]
+      if (phi < -0.25 * kPi - 0.02 || phi > std::atan(2.0) + 0.02) continue;
+      const int below = (j + 15) & 15, above = j;  // codes at smaller / larger psi
+      rays.push_back({std::tan(phi), D > 0 ? below : above, D > 0 ? above : below});
+    }
+    for (int c = 0; c < pq::kL1Cells; ++c) {
+      // the kernel's cell index is floor(m / 8), m = t * kL1CellScale * 8 rounded to an integer
+      const double scale = (double)pq::kL1CellScale;
+      const double lo = std::fmax(0.0, (c - 1.0 / 16.0) / scale - 1e-6), hi = std::fmin(1.0, (c + 15.0 / 16.0) / scale + 1e-6);
+      const double w = hi - lo;
+      int n_in = 0, in_idx = -1;
+      double dA = 1e30, dB = 1e30;  // distance from the cell to the nearest ray below / above it
+      for (size_t i = 0; i < rays.size(); ++i) {
+        if (rays[i].t >= lo && rays[i].t <= hi) { ++n_in; in_idx = (int)i; }
+        else if (rays[i].t < lo) dA = std::fmin(dA, lo - rays[i].t);
+        else dB = std::fmin(dB, rays[i].t - hi);
+      }
+      float tau;
+      int code_lo, code_hi;
+      if (n_in == 0) {
+        // no ray inside: a virtual tau outside the cell whose distance stays below both neighbours' for every t
+        const double mA = std::fmin(dA, dB - w), mB = std::fmin(dB, dA - w);
+        const double t = mA >= mB ? lo - std::fmin(mA, 1.0) : hi + std::fmin(mB, 1.0);
+        const double mid = 0.5 * (lo + hi);
+        double psi = B + D * std::atan(mid);
+        if (psi >= 2.0 * kPi) psi -= 2.0 * kPi;
+        if (psi < 0.0) psi += 2.0 * kPi;
+        code_lo = code_hi = l1_code_of_angle(bnd, psi);
+        tau = (float)std::fmin(1.0, std::fmax(0.0, t));
+        if ((mA >= mB ? mA : mB) <= 0.0) tau = std::nanf("");  // a ray touches the cell from both sides
+      } else if (n_in == 1) {
+        const double tm = rays[in_idx].t;
+        const double far = std::fmax(tm - lo, hi - tm);  // largest distance from a t of the cell to the ray
+        tau = (dA >= far && dB >= far) ? (float)tm : std::nanf("");
+        code_lo = rays[in_idx].below;
+        code_hi = rays[in_idx].above;
+      } else {
+        tau = std::nanf("");
+        code_lo = code_hi = 0;
+      }
+      uint32_t bits;
+      std::memcpy(&bits, &tau, 4);
+      cells[o][c] = make_uint2(bits, ((uint32_t)code_lo << 28) | ((uint32_t)code_hi << 24));
+    }
+    // Check the two properties on a grid of every cell (the table is small; a wrong entry would be a silent
+    // wrong code).
+    for (int c = 0; c < pq::kL1Cells; ++c) {
+      float tau;
+      std::memcpy(&tau, &cells[o][c].x, 4);
+      if (tau != tau) continue;
+      const double scale = (double)pq::kL1CellScale;
+      const double lo = std::fmax(0.0, (c - 1.0 / 16.0) / scale), hi = std::fmin(1.0, (c + 15.0 / 16.0) / scale);
+      for (int i = 0; i <= 16; ++i) {
+        const double t = lo + (hi - lo) * i / 16.0, dist = std::fabs(t - (double)tau);
+        double nearest = 1e30;
+        for (const L1Ray& r : rays) nearest = std::fmin(nearest, std::fabs(t - r.t));
+        if (dist > nearest + 1e-7) return false;
+        if (dist < 1e-6) continue;
+        double psi = B + D * std::atan(t);
+        if (psi >= 2.0 * kPi) psi -= 2.0 * kPi;
+        if (psi < 0.0) psi += 2.0 * kPi;
+        const int want = l1_code_of_angle(bnd, psi);
+        const int got = (int)((cells[o][c].y >> (t > (double)tau ? 24 : 28)) & 15u);
+        if (want != got) return false;
+      }
+    }
+  }
+  return true;
+}
+
 }  // namespace
 
 namespace pq {
@@ -231,6 +336,7 @@ int32_t pq_build_tables(const double* cen, const double* bnd, void* tables_host)
       const double t3 = (s & 1) ? std::sin(a3) : std::cos(a3);
       split(t4 * t3 * std::cos(a2), t4 * t3 * std::sin(a2), &t.u_tab[s][i].x, &t.u_tab[s][i].y);
     }
+  if (!build_l1_cells(bnd, t.l1_cells)) return PQ_ERR_INVALID_ARG;
   std::memcpy(tables_host, &t, sizeof(t));
   return PQ_OK;
 }

@@ -331,10 +331,61 @@ def _perturbed_codebooks(seed):
     return torch.from_numpy(c), torch.from_numpy(bnd)
 
 
+def _codebooks_with_level1(theta1, upper_shift=0.0):
+    """The analytic codebooks with level 1 replaced by the ascending centroids `theta1` (midpoint boundaries) and
+    the upper levels' centroids moved by `upper_shift` (no longer symmetric about pi/4)."""
+    cen, _ = pq.pq_fit_codebooks()
+    c = cen.numpy().copy()
+    c[:16] = np.asarray(theta1, dtype=np.float64)
+    c[16:] += upper_shift * np.array([1, -0.5, 0.7, -1] * 3)
+    bnd = np.concatenate([0.5 * (c[o:o + n - 1] + c[o + 1:o + n]) for o, n in ((0, 16), (16, 4), (20, 4), (24, 4))])
+    return torch.from_numpy(c), torch.from_numpy(bnd)
+
+
+_UNIFORM16 = (np.arange(16) + 0.5) * np.pi / 8
+_LEVEL1_CASES = {
+    # every boundary a little off the uniform grid: what a fit on observed angles gives
+    "fitted": _UNIFORM16 + np.random.default_rng(1).uniform(-0.06, 0.06, 16),
+    # boundaries exactly on the axes and diagonals of the folding (the uniform grid turned by pi/8 has them all there)
+    "on_axes": np.concatenate(([0.05], np.arange(1, 16) * np.pi / 8 + 1e-9 * np.arange(15))),
+    # two boundaries 0.004 rad apart (one table cell holds both), a gap wider than two octants, centroids next to 0 and 2 pi
+    "clustered": np.array([1e-4, 0.3, 0.304, 0.308, 0.9, 1.2, 1.5702, 1.5712, 1.6, 4.3, 4.6, 5.0, 5.4, 5.9, 6.2, 6.2831]),
+    # boundaries 3e-4 rad on either side of a diagonal (the second lies past the octant's edge), and one 0.02 past the axis at pi
+    "near_edges": np.concatenate(([np.pi / 4 - 6e-4, np.pi / 4, np.pi / 4 + 6e-4, np.pi - 1e-5 + 0.02, np.pi + 1e-5 + 0.02],
+                                  np.linspace(3.5, 6.1, 11))),
+}
+
+
+@pytest.mark.parametrize("case", sorted(_LEVEL1_CASES))
+@pytest.mark.parametrize("n", [40, 700])
+def test_any_level1_codebook_is_decided_in_float32_by_the_table(case, n):
+    """Codebooks other than the analytic ones (data-fitted, Section 4.1) take the table-driven level-1 test and the
+    per-boundary upper-level test: codes equal the oracle's, and float64 decides only a small share of the angles
+    unless the codebook is built to defeat the table (cells holding two boundaries)."""
+    d, Hq, Hkv = 128, 8, 2
+    cbk = _codebooks_with_level1(_LEVEL1_CASES[case], upper_shift=0.03 if case != "on_axes" else 0.0)
+    cache = pq.PolarQuantCache(1, Hq, Hkv, d, capacity=n, seed=21, device=DEV, codebooks=cbk)
+    K, V = synthetic.kv_like(300 + n, n, Hkv, d, torch.bfloat16, DEV)
+    K[3] *= 1e-3   # small and large rows: the margins scale with the row
+    V[5] *= 300.0
+    K[7] = 0       # a zero row: every angle is atan2(0, 0) = 0
+    rep = _encode_and_compare(cache, K, V, [n])
+    st = cache.check_status()
+    decisions = 2 * Hkv * n * 120
+    assert rep["total"] == decisions
+    if case in ("fitted", "on_axes"):
+        assert st[3] < 0.01 * decisions + 200, st   # 120 of the zero row's angles alone
+    ref = _oracle_cache(cache, K, V, [n])
+    q = synthetic.queries(n, 1, Hq, d, torch.bfloat16, DEV)
+    out = cache.attend(q)
+    torch.cuda.synchronize()
+    cache.check_status()
+    assert rel_l2(to_f64(out), ref.attend(to_f64(q), d ** -0.5)) < TOL_ATTENTION
+
+
 @pytest.mark.parametrize("n", [5, 40, 300])
 def test_other_codebooks_fp32_inputs_and_strided_views(n):
-    """Paths beside the bf16 tensor-core encoder: a non-uniform level-1 codebook (every level-1 decision is
-    then taken in float64), float32 inputs (FMA rotation), strided K/V views, and chunks of every size class
+    """Paths beside the bf16 tensor-core encoder: a non-uniform level-1 codebook, float32 inputs (FMA rotation), strided K/V views, and chunks of every size class
     (per-vector kernel < 32 rows, FMA kernel < 128 rows, tensor-core kernel above)."""
     d, Hq, Hkv = 128, 8, 2
     for dtype, cbk in ((torch.bfloat16, _perturbed_codebooks(3)), (torch.float32, None), (torch.bfloat16, None)):
