@@ -15,8 +15,9 @@
  *   - State the library keeps, all of it per process: a call counter that tags the scratch of
  *     pq_decode_attention, a per-device note of which kernels have been configured (and, for
  *     pq_decode_attention_static, the device address of its built-in array, which every GPU
- *     that loads the library carries), the last CUDA error of each host thread, and the test
- *     hook of pq_debug_fail_next_wait.  All of it is updated atomically: host threads may call
+ *     that loads the library carries), the last CUDA error of each host thread, the analytic
+ *     codebook pq_fit_codebooks_from_histograms starts from (computed at its first use), and the
+ *     test hook of pq_debug_fail_next_wait.  All of it is updated atomically: host threads may call
  *     into the library concurrently as long as they do not share output buffers or scratch.
  *   - Device work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
  *     legacy default stream) and the call returns without synchronising.
@@ -62,6 +63,7 @@ extern "C" {
 #define PQ_N_LEVELS 4
 #define PQ_N_CENTROIDS 28  /* 16 + 4 + 4 + 4 */
 #define PQ_N_BOUNDARIES 24 /* 15 + 3 + 3 + 3 */
+#define PQ_HIST_MAX_BINS 1024 /* bins per level of pq_angle_histograms */
 
 /* Human-readable name of a status code (static string, never NULL). */
 const char* pq_status_string(int32_t status);
@@ -100,6 +102,37 @@ int32_t pq_fit_codebooks(const int32_t* bits, double* centroids_host, double* bo
  */
 int64_t pq_tables_bytes(void);
 int32_t pq_build_tables(const double* centroids_host, const double* boundaries_host, void* tables_host);
+
+/*
+ * "Online" codebook (Section 4.1, Eq. 4 on the observed angles of one prompt and layer), in two steps.
+ *
+ * pq_angle_histograms: rotate the rows of K and V by S, take the angles of Algorithm 1's Polar and count them,
+ * per level, in n_bins bins of equal width over the level's range ([0, 2 pi) at level 1, [0, pi/2] above).
+ *   K_dev, V_dev       device, [total_tokens][n_kv_heads][head_dim] of `in_dtype`, strides in elements as for
+ *                      pq_encode_kv (keys and values are counted together: one codebook serves both)
+ *   n_bins             16 .. PQ_HIST_MAX_BINS
+ *   hist_dev           device, uint64[PQ_N_LEVELS][n_bins], 8-byte aligned; counts are ADDED (zero it before the
+ *                      first call; several calls accumulate, e.g. the chunks of one prompt)
+ * Angles are formed in float32: an angle within about 1e-5 rad of a bin edge may be counted in the neighbouring
+ * bin.  A 16-coordinate block with a non-finite rotated coordinate (any non-finite input of the row) is not
+ * counted; the number of such blocks is added to status word 1 and PQ_ERR_NONFINITE is recorded.
+ *
+ * pq_fit_codebooks_from_histograms (host): per level, 1-D k-means (Lloyd's iteration) on the binned sample -- bin
+ * centres weighted by their counts -- until no centroid moves: boundaries are the midpoints of adjacent centroids,
+ * a bin belongs to the cell its centre lies in (a centre on a boundary: the lower cell), a centroid is the weighted
+ * mean of its cell, and an empty cell keeps its centroid.  Distances are taken on the line, also at level 1.  The
+ * paper seeds the clustering with k-means++; here it starts from init_centroids (NULL: the analytic codebook of
+ * pq_fit_codebooks), so the result is a function of the histogram alone.
+ *   hist_host          host, uint64[PQ_N_LEVELS][n_bins]
+ *   init_centroids_host  host, float64[PQ_N_CENTROIDS] ascending per level, or NULL
+ *   centroids_host, boundaries_host   out, as for pq_fit_codebooks; pass them to pq_build_tables
+ * A level without any count keeps its initial centroids.
+ */
+int32_t pq_angle_histograms(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* K_dev,
+                            const void* V_dev, int32_t in_dtype, int64_t token_stride, int64_t head_stride,
+                            int32_t total_tokens, int32_t n_bins, uint64_t* hist_dev, int32_t* status_dev, void* stream);
+int32_t pq_fit_codebooks_from_histograms(const uint64_t* hist_host, int32_t n_bins, const double* init_centroids_host,
+                                         double* centroids_host, double* boundaries_host);
 
 /* Size in bytes of the packed cache for `batch` sequences x n_kv_heads heads x (K and V),
  * each with room for `capacity` tokens (rounded up to whole token-blocks).  At d = 128 a

@@ -22,6 +22,7 @@ ERR_CUDA, ERR_TIMEOUT, ERR_NONFINITE, ERR_EMPTY, ERR_SCRATCH = -5, -6, -7, -8, -
 DTYPE_F32, DTYPE_BF16 = 0, 1
 STATUS_WORDS = 4
 N_CENTROIDS, N_BOUNDARIES = 28, 24
+N_LEVELS, HIST_MAX_BINS = 4, 1024
 DEFAULT_BITS = (4, 2, 2, 2)
 
 # name -> (restype, argtypes); must list every symbol of include/polarquant.h
@@ -31,6 +32,9 @@ _SIGNATURES = {
     "pq_token_block": (c_int32, []),
     "pq_make_rotation": (c_int32, [c_int32, c_uint64, c_void_p]),
     "pq_fit_codebooks": (c_int32, [POINTER(c_int32), POINTER(c_double), POINTER(c_double)]),
+    "pq_angle_histograms": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_int64, c_int64, c_int32,
+                                      c_int32, c_void_p, c_void_p, c_void_p]),
+    "pq_fit_codebooks_from_histograms": (c_int32, [c_void_p, c_int32, c_void_p, c_void_p, c_void_p]),
     "pq_tables_bytes": (c_int64, []),
     "pq_build_tables": (c_int32, [POINTER(c_double), POINTER(c_double), c_void_p]),
     "pq_cache_bytes": (c_int64, [c_int32, c_int32, c_int32, c_int32]),
@@ -125,6 +129,28 @@ def pq_fit_codebooks(bits=DEFAULT_BITS):
     arr = (c_int32 * 4)(*bits)
     _check(lib().pq_fit_codebooks(arr, ctypes.cast(cen.data_ptr(), POINTER(c_double)),
                                   ctypes.cast(bnd.data_ptr(), POINTER(c_double))), "pq_fit_codebooks")
+    return cen, bnd
+
+
+def pq_angle_histograms(S, K, V, hist, status, stream=None):
+    """Add the angles of the rows of K and V [total_tokens, Hkv, d] to hist (int64 device tensor [4, n_bins])."""
+    total, n_kv_heads, d = K.shape
+    assert V.shape == K.shape and V.dtype == K.dtype and K.stride(2) == 1 and V.stride() == K.stride()
+    assert hist.dtype == torch.int64 and hist.is_contiguous() and hist.shape[0] == N_LEVELS
+    _check(lib().pq_angle_histograms(d, n_kv_heads, _ptr(S), _ptr(K), _ptr(V), _dtype_code(K), K.stride(0), K.stride(1),
+                                     total, hist.shape[1], _ptr(hist), _ptr(status), _stream(stream)),
+           "pq_angle_histograms")
+
+
+def pq_fit_codebooks_from_histograms(hist: torch.Tensor, init_centroids: torch.Tensor = None):
+    """k-means on the binned angles (hist: int64 CPU tensor [4, n_bins]): (centroids float64[28], boundaries
+    float64[24]) CPU tensors, started from init_centroids (None: the analytic codebook)."""
+    hist = hist.to(torch.int64).cpu().contiguous()
+    init = None if init_centroids is None else init_centroids.to(torch.float64).cpu().contiguous()
+    cen = torch.empty(N_CENTROIDS, dtype=torch.float64)
+    bnd = torch.empty(N_BOUNDARIES, dtype=torch.float64)
+    _check(lib().pq_fit_codebooks_from_histograms(hist.data_ptr(), hist.shape[1], _ptr(init), cen.data_ptr(),
+                                                  bnd.data_ptr()), "pq_fit_codebooks_from_histograms")
     return cen, bnd
 
 
@@ -248,6 +274,19 @@ class PolarQuantCache:
         self.status = torch.zeros(STATUS_WORDS, dtype=torch.int32, device=self.device)
         self.workspace = torch.empty(pq_workspace_bytes(d, batch, n_q_heads, n_kv_heads, capacity), dtype=torch.uint8,
                                      device=self.device)
+
+    def fit_online_codebooks(self, K, V, n_bins=HIST_MAX_BINS, stream=None):
+        """Replace the codebooks of this cache by the ones clustered on the angles of K, V ([tokens, Hkv, d], the
+        prompt's keys and values): histogram on the device, clustering on the host, new tables.  To be called
+        before anything is encoded (codes already in the cache belong to the previous codebooks)."""
+        hist = torch.zeros((N_LEVELS, n_bins), dtype=torch.int64, device=self.device)
+        pq_angle_histograms(self.S, K, V, hist, self.status, stream)
+        self.set_codebooks(*pq_fit_codebooks_from_histograms(hist.cpu()))
+        return hist
+
+    def set_codebooks(self, centroids, boundaries):
+        self.centroids, self.boundaries = centroids, boundaries
+        self.tables = pq_build_tables(centroids, boundaries).to(self.device)
 
     def encode(self, K, V, cu_seqlens, stream=None):
         pq_encode_kv(self.S, self.tables, K, V, cu_seqlens, self.cache, self.lens, self.capacity, self.status, stream)

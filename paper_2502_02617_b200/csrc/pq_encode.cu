@@ -23,6 +23,9 @@ struct EncodeArgs {
   const int32_t* cache_lens;
   int32_t* status;
   uint32_t debug;  // bit 0: test hook, the first bounded wait of CTA 0 of the tensor-core kernel reports failure
+  // angle histograms (pq_angle_histograms) instead of codes: uint64 [4 levels][n_bins], added to
+  unsigned long long* hist;
+  int n_bins;
 };
 
 __device__ inline float load_elem(const void* base, int dtype, int64_t idx) {
@@ -429,8 +432,54 @@ __global__ void __launch_bounds__(128) encode_vector_kernel(EncodeArgs a) {
 }
 
 }  // namespace pq
+#include "pq_hist.cuh"
 #include "pq_encode_tc.cuh"
 namespace pq {
+
+// Angle histograms of any head_dim (multiple of 16, at most 128) and input type: 128 / head_dim vectors per CTA,
+// thread = rotated coordinate in float32, then one thread per 16-block counts the block's 15 angles into the CTA's
+// shared histogram.  The path of short inputs and of what the tensor-core kernel does not take.
+constexpr int kHistSimpleThreads = 128;
+__global__ void __launch_bounds__(kHistSimpleThreads) hist_simple_kernel(EncodeArgs a, int64_t n_vec, int vec_per_cta_step) {
+  extern __shared__ uint32_t hist_s[];
+  __shared__ float xs[128];
+  __shared__ float ys[128];
+  const int d = a.head_dim, per = 128 / d, j = threadIdx.x, vi = j / d, jj = j % d;
+  for (int i = j; i < 4 * a.n_bins; i += kHistSimpleThreads) hist_s[i] = 0u;
+  const float scale1 = (float)a.n_bins * 0.159154943091895336f, scale_up = (float)a.n_bins * 0.636619772367581343f;
+  int bad = 0;
+  for (int64_t v0 = (int64_t)blockIdx.x * per; v0 < n_vec; v0 += (int64_t)gridDim.x * per) {
+    const int64_t v = v0 + vi;  // vector index: (row * 2 + kv) * n_kv_heads + head
+    const bool valid = vi < per && v < n_vec;
+    __syncthreads();
+    if (valid) {
+      const int head = (int)(v % a.n_kv_heads), kv = (int)((v / a.n_kv_heads) & 1);
+      const int64_t row = v / (2 * a.n_kv_heads);
+      xs[j] = load_elem(kv ? a.V : a.K, a.in_dtype, row * a.token_stride + (int64_t)head * a.head_stride + jj);
+    }
+    __syncthreads();
+    if (valid) {
+      float acc[4] = {0.f, 0.f, 0.f, 0.f};
+      for (int k = 0; k < d; k += 4)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[i] = fmaf(xs[vi * d + k + i], __ldg(a.S + (k + i) * d + jj), acc[i]);
+      ys[j] = (acc[0] + acc[1]) + (acc[2] + acc[3]);
+    }
+    __syncthreads();
+    if (valid && (jj & 15) == 0) {
+      float yb[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) yb[i] = ys[j + i];
+      if (!hist_block(yb, hist_s, a.n_bins, scale1, scale_up)) ++bad;
+    }
+  }
+  if (bad) {
+    atomicAdd(a.status + 1, bad);
+    set_status(a.status, PQ_ERR_NONFINITE);
+  }
+  __syncthreads();
+  hist_flush(hist_s, 4 * a.n_bins, a.hist, j, kHistSimpleThreads);
+}
 
 // lens[b] += rows of sequence b (skipped for sequences that did not fit).
 __global__ void advance_lens_kernel(const int32_t* cu_seqlens, int batch, int capacity, int32_t* lens) {
@@ -528,6 +577,37 @@ int32_t pq_append_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, c
   a.cache = reinterpret_cast<uint8_t*>(cache_dev); a.cache_lens = cache_lens_dev; a.status = status_dev;
   a.debug = 0u;
   return pq::launch_encode(a, cache_lens_dev, reinterpret_cast<cudaStream_t>(stream));
+}
+
+int32_t pq_angle_histograms(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* K_dev,
+                            const void* V_dev, int32_t in_dtype, int64_t token_stride, int64_t head_stride,
+                            int32_t total_tokens, int32_t n_bins, uint64_t* hist_dev, int32_t* status_dev, void* stream) {
+  if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
+  if (n_kv_heads <= 0 || !S_dev || !K_dev || !V_dev || !hist_dev || !status_dev || total_tokens < 0) return PQ_ERR_INVALID_ARG;
+  if (n_bins < 16 || n_bins > PQ_HIST_MAX_BINS) return PQ_ERR_INVALID_ARG;
+  if (in_dtype != PQ_DTYPE_F32 && in_dtype != PQ_DTYPE_BF16) return PQ_ERR_UNSUPPORTED;
+  if (token_stride < 0 || head_stride < 0) return PQ_ERR_INVALID_ARG;
+  if ((int64_t)total_tokens * 2 * n_kv_heads >= (1ll << 31) * 16) return PQ_ERR_UNSUPPORTED;
+  if (((uintptr_t)S_dev & 15) || ((uintptr_t)hist_dev & 7)) return PQ_ERR_ALIGNMENT;
+  if (total_tokens == 0) return PQ_OK;
+  pq::EncodeArgs a;
+  a.K = K_dev; a.V = V_dev; a.in_dtype = in_dtype;
+  a.token_stride = token_stride; a.head_stride = head_stride;
+  a.cu_seqlens = nullptr; a.batch = 0; a.total_tokens = total_tokens;
+  a.n_kv_heads = n_kv_heads; a.head_dim = head_dim; a.capacity = 0;
+  a.S = S_dev; a.tables = nullptr; a.cache = nullptr; a.cache_lens = nullptr; a.status = status_dev;
+  a.debug = 0u;
+  a.hist = reinterpret_cast<unsigned long long*>(hist_dev); a.n_bins = n_bins;
+  cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+  const int32_t tc = pq::try_launch_hist_tc(a, s);
+  if (tc < 0) return tc;
+  if (tc == 1) return pq::launch_status();
+  const int per = 128 / head_dim;
+  const int64_t n_vec = (int64_t)total_tokens * 2 * n_kv_heads;
+  const int64_t want = (n_vec + per - 1) / per;
+  const int grid = (int)(want < 148 * 8 ? want : 148 * 8);
+  pq::hist_simple_kernel<<<grid, pq::kHistSimpleThreads, (size_t)4 * n_bins * sizeof(uint32_t), s>>>(a, n_vec, per);
+  return pq::launch_status();
 }
 
 }  // extern "C"

@@ -48,6 +48,7 @@ constexpr int kTcSpin = 1 << 22;
 static_assert(kTcTerms == 3, "kRotErrTc is the bound for three terms");
 static_assert(sizeof(TcFixQueue) % 16 == 0, "queues are laid out back to back");
 static_assert(kTcSmTotal <= 227 * 1024, "shared memory of one CTA");
+static_assert(4 * PQ_HIST_MAX_BINS * 4 <= kTcSlots * (int)sizeof(TcFixQueue), "the histogram takes the queues' place");
 static_assert(kFixSdBytes <= kTcSmFq, "the float64 copy of S must fit in the operand buffers");
 
 __device__ __forceinline__ uint32_t tc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -156,6 +157,10 @@ __device__ inline int count_nonfinite_bf16(const void* base, int64_t xoff) {
   return bad;
 }
 
+// kHist: the same pipeline up to the rotated coordinates in registers, which are then counted into the angle
+// histograms (pq_hist.cuh) instead of being quantised; the shared memory of the re-decision queues holds the CTA's
+// histogram (4 levels x n_bins 32-bit counters: a CTA would have to take 2^32 / 8192 tiles to overflow one).
+template <bool kHist>
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_tiles) {
   extern __shared__ uint8_t smem_raw[];
@@ -209,9 +214,14 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     for (int it = 0; it < kTcStages; ++it) issue_tma(it);  // the first tiles arrive while S is split
-    load_fast_quant(a.tables, fq);
+    if (!kHist) load_fast_quant(a.tables, fq);
   }
-  if (st < 4) fixq->count[st] = 0;
+  uint32_t* hist_s = reinterpret_cast<uint32_t*>(smem + kTcSmFix);
+  if (kHist) {
+    for (int i = tid; i < 4 * a.n_bins; i += kTcThreads) hist_s[i] = 0u;
+  } else if (st < 4) {
+    fixq->count[st] = 0;
+  }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(sb + kTcSmMisc) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -295,7 +305,9 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
 
   // ---- tile loop of this slot
   constexpr int o2 = 32 * kTokenBlock, o3 = o2 + 8 * kTokenBlock, o4 = o3 + 4 * kTokenBlock, orad = o4 + 2 * kTokenBlock;
-  const bool analytic = fq->analytic != 0u;  // uniform over the grid
+  const bool analytic = kHist || fq->analytic != 0u;  // uniform over the grid
+  const float hist_scale1 = (float)a.n_bins * 0.159154943091895336f, hist_scale_up = (float)a.n_bins * 0.636619772367581343f;
+  int hist_bad = 0;
   const Layout L = make_layout(128, a.capacity);
   const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + slot * 128;
   const int slot_bar = 1 + slot;
@@ -318,6 +330,23 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     float y[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) y[i] = 0.f;
+    if (kHist) {
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        if (ready) tc_ld32(taddr + 32 * c, y);
+        if (c == 3) {  // as below: the accumulator is free for the slot's next tile
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          asm volatile("bar.sync %0, %1;" ::"r"(slot_bar), "n"(kTcSlotThreads) : "memory");
+          if (leader) issue_mmas(it + kTcSlots);
+          __syncwarp();
+        }
+        if (ready && row < a.total_tokens) {
+          hist_bad += !hist_block(y, hist_s, a.n_bins, hist_scale1, hist_scale_up);
+          hist_bad += !hist_block(y + 16, hist_s, a.n_bins, hist_scale1, hist_scale_up);
+        }
+      }
+      continue;
+    }
     // pass 1: squared norm of the row (four partial sums)
     float sq[4] = {0.f, 0.f, 0.f, 0.f};
     if (ready) {
@@ -419,10 +448,17 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  if (kHist) {
+    if (hist_bad) {
+      atomicAdd(a.status + 1, hist_bad);
+      set_status(a.status, PQ_ERR_NONFINITE);
+    }
+    hist_flush(hist_s, 4 * a.n_bins, a.hist, tid, kTcThreads);
+  }
   // Every MMA and copy of this CTA has completed (each was waited for by its slot), so the operand buffers are
   // idle: put a float64 copy of S there (rows permuted, see fix_sd_row) for the queued exact re-decisions.
   double* Sd = reinterpret_cast<double*>(smem + kTcSmS);
-  if (!*abort_flag) {
+  if (!kHist && !*abort_flag) {
     constexpr int kPer = 128 * 128 / kTcThreads;
     float sv[kPer];
 #pragma unroll
@@ -434,8 +470,9 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     }
     __syncthreads();
   }
-  fix_process(fixq - slot, kTcSlots, tid, kTcThreads, a.K, a.V, a.in_dtype, a.S, *abort_flag ? (const double*)nullptr : Sd,
-              *a.tables, a.status);
+  if (!kHist)
+    fix_process(fixq - slot, kTcSlots, tid, kTcThreads, a.K, a.V, a.in_dtype, a.S, *abort_flag ? (const double*)nullptr : Sd,
+                *a.tables, a.status);
   if (*abort_flag && tid < kTcStages && copies_issued[tid] > 0) {
     // gave up somewhere: let the copies that are still in flight land (bounded) before the CTA and its
     // shared memory go away
@@ -477,9 +514,10 @@ static bool make_x_map(EncodeTiledFn fn, CUtensorMap* map, const void* base, int
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Launch the tensor-core encoder if the inputs allow it.  Returns 1 if launched, 0 if not applicable,
-// or a negative status.
-static int32_t try_launch_encode_tc(const EncodeArgs& a, cudaStream_t stream) {
+// Launch the tensor-core encoder (or its histogram form) if the inputs allow it.  Returns 1 if launched, 0 if not
+// applicable, or a negative status.
+template <bool kHist>
+static int32_t try_launch_tc(const EncodeArgs& a, cudaStream_t stream) {
   if (a.head_dim != 128 || a.in_dtype != PQ_DTYPE_BF16 || a.total_tokens < 128) return 0;
   if ((a.token_stride & 7) || (a.head_stride & 7) || a.head_stride < 128 || a.token_stride < 128) return 0;
   if (((uintptr_t)a.K | (uintptr_t)a.V) & 15) return 0;
@@ -489,16 +527,18 @@ static int32_t try_launch_encode_tc(const EncodeArgs& a, cudaStream_t stream) {
   TcMaps maps;
   if (!make_x_map(fn, &maps.k, a.K, a.n_kv_heads, a.total_tokens, a.token_stride, a.head_stride)) return 0;
   if (!make_x_map(fn, &maps.v, a.V, a.n_kv_heads, a.total_tokens, a.token_stride, a.head_stride)) return 0;
-  static DeviceMemo configured;
-  const int n_sm = configure_for_device(encode_tc_kernel, kTcSmTotal, configured);
+  static DeviceMemo configured;  // one per instantiation
+  const int n_sm = configure_for_device(encode_tc_kernel<kHist>, kTcSmTotal, configured);
   if (n_sm == 0) return PQ_ERR_CUDA;
   const int n_row_tiles = (a.total_tokens + 127) / 128;
   const int n_tiles = n_row_tiles * 2 * a.n_kv_heads;
   const int grid = n_tiles < n_sm ? n_tiles : n_sm;
   EncodeArgs args = a;
   if (take_debug_wait_failure(1)) args.debug |= 1u;
-  encode_tc_kernel<<<grid, kTcThreads, kTcSmTotal, stream>>>(args, maps, n_row_tiles);
+  encode_tc_kernel<kHist><<<grid, kTcThreads, kTcSmTotal, stream>>>(args, maps, n_row_tiles);
   return 1;
 }
+static int32_t try_launch_encode_tc(const EncodeArgs& a, cudaStream_t stream) { return try_launch_tc<false>(a, stream); }
+static int32_t try_launch_hist_tc(const EncodeArgs& a, cudaStream_t stream) { return try_launch_tc<true>(a, stream); }
 
 }  // namespace pq

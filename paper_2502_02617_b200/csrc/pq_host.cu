@@ -1,4 +1,5 @@
 // Host-side entry points: rotation generator, Lloyd-Max codebooks, derived tables, size queries.
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstring>
@@ -259,6 +260,70 @@ int32_t pq_fit_codebooks(const int32_t* bits, double* centroids_host, double* bo
         theta[k] = t;
       }
       if (delta < 1e-15) break;
+    }
+    for (int k = 0; k + 1 < n; ++k) beta[k] = 0.5 * (theta[k] + theta[k + 1]);
+  }
+  return PQ_OK;
+}
+
+int32_t pq_fit_codebooks_from_histograms(const uint64_t* hist, int32_t n_bins, const double* init, double* cen,
+                                         double* bnd) {
+  if (hist == nullptr || cen == nullptr || bnd == nullptr || n_bins < 16 || n_bins > PQ_HIST_MAX_BINS) return PQ_ERR_INVALID_ARG;
+  double start[PQ_N_CENTROIDS];
+  if (init == nullptr) {
+    // the analytic codebook costs tens of milliseconds of quadrature: computed once per process
+    struct Analytic {
+      double cen[PQ_N_CENTROIDS], bnd[PQ_N_BOUNDARIES];
+      int32_t status;
+      Analytic() {
+        const int32_t bits[PQ_N_LEVELS] = {4, 2, 2, 2};
+        status = pq_fit_codebooks(bits, cen, bnd);
+      }
+    };
+    static const Analytic analytic;  // thread-safe initialisation
+    if (analytic.status != PQ_OK) return analytic.status;
+    std::memcpy(start, analytic.cen, sizeof(start));
+  } else {
+    std::memcpy(start, init, sizeof(start));
+  }
+  std::vector<double> centre(n_bins), w0(n_bins + 1), w1(n_bins + 1);
+  for (int level = 1; level <= PQ_N_LEVELS; ++level) {
+    const int n = level == 1 ? 16 : 4;
+    const double hi = level == 1 ? 2.0 * kPi : 0.5 * kPi, width = hi / n_bins;
+    const uint64_t* h = hist + (size_t)(level - 1) * n_bins;
+    double* theta = cen + pq::cen_off(level);
+    double* beta = bnd + pq::bnd_off(level);
+    for (int k = 0; k < n; ++k) {
+      theta[k] = start[pq::cen_off(level) + k];
+      if (!(theta[k] >= 0.0 && theta[k] <= hi) || (k > 0 && !(theta[k] > theta[k - 1]))) return PQ_ERR_INVALID_ARG;
+    }
+    // prefix sums of the weights and of weight x centre: a cell's mean is two differences
+    w0[0] = w1[0] = 0.0;
+    for (int i = 0; i < n_bins; ++i) {
+      centre[i] = (i + 0.5) * width;
+      w0[i + 1] = w0[i] + (double)h[i];
+      w1[i + 1] = w1[i] + (double)h[i] * centre[i];
+    }
+    for (int iter = 0; iter < 10000; ++iter) {
+      bool moved = false;
+      int first = 0;  // first bin of cell k
+      double next[16];
+      for (int k = 0; k < n; ++k) {
+        // the cell ends before the first bin whose centre lies above the boundary between k and k + 1
+        int last = n_bins;
+        if (k + 1 < n) {
+          const double b = 0.5 * (theta[k] + theta[k + 1]);
+          last = (int)(std::upper_bound(centre.begin() + first, centre.end(), b) - centre.begin());
+        }
+        const double m0 = w0[last] - w0[first], m1 = w1[last] - w1[first];
+        next[k] = m0 > 0.0 ? m1 / m0 : theta[k];
+        first = last;
+      }
+      for (int k = 0; k < n; ++k) {
+        moved = moved || next[k] != theta[k];
+        theta[k] = next[k];
+      }
+      if (!moved) break;
     }
     for (int k = 0; k + 1 < n; ++k) beta[k] = 0.5 * (theta[k] + theta[k + 1]);
   }

@@ -80,6 +80,50 @@ def test_tables_reject_unsorted_or_out_of_range_codebooks():
         pq.pq_build_tables(cen, bad)
 
 
+def test_level1_decision_table_is_built_for_any_ascending_codebook():
+    """pq_build_tables checks its level-1 cell table against the boundaries it was built from (both guarantees of
+    every cell) and would refuse a codebook whose table fails: random ascending level-1 codebooks, the uniform one
+    turned by small and large angles, boundaries packed closely."""
+    cen, bnd = pq.pq_fit_codebooks()
+    rng = np.random.default_rng(0)
+    cases = [np.sort(rng.uniform(0, 2 * math.pi, 16)) for _ in range(40)]
+    cases += [((np.arange(16) + 0.5) * math.pi / 8 + s) % (2 * math.pi) for s in (1e-9, 1e-4, 0.01, 0.19, 0.2, math.pi / 16)]
+    cases += [np.linspace(1.0, 1.0 + 15e-4, 16), np.linspace(0.0, 2 * math.pi - 1e-7, 16)]
+    for theta in cases:
+        c = cen.clone()
+        c[:16] = torch.from_numpy(np.sort(theta))
+        b = bnd.clone()
+        b[:15] = 0.5 * (c[:15] + c[1:16])
+        assert pq.pq_build_tables(c, b).numel() == pq.lib().pq_tables_bytes()
+
+
+def test_histogram_clustering_matches_the_oracle():
+    """pq_fit_codebooks_from_histograms against the oracle's k-means on the same binned sample: Gaussian and
+    anisotropic rows, 1024 and 256 bins, a level without counts, and a start other than the analytic codebook."""
+    rng = np.random.default_rng(3)
+    S = orc.make_rotation(16, 5)
+    off = orc.fit_codebooks()
+    for n_bins, x in ((1024, rng.normal(size=(3000, 16))), (256, rng.normal(size=(2000, 16)) * np.linspace(0.1, 4, 16))):
+        hist = orc.angle_histograms(x, S, 4, n_bins)
+        cen, bnd = pq.pq_fit_codebooks_from_histograms(torch.from_numpy(hist))
+        for level in range(1, 5):
+            want, want_b = orc.kmeans_on_histogram(hist[level - 1], level, off.centroids[level - 1])
+            o, n = (0, 16) if level == 1 else (16 + 4 * (level - 2), 4)
+            ob = 0 if level == 1 else 15 + 3 * (level - 2)
+            assert np.max(np.abs(cen.numpy()[o:o + n] - want)) < 1e-12
+            assert np.max(np.abs(bnd.numpy()[ob:ob + n - 1] - want_b)) < 1e-12
+        pq.pq_build_tables(cen, bnd)  # a valid codebook
+    hist[2] = 0
+    init = torch.from_numpy(off.flat_centroids() + 0.01)
+    cen, _ = pq.pq_fit_codebooks_from_histograms(torch.from_numpy(hist), init)
+    assert np.array_equal(cen.numpy()[20:24], init.numpy()[20:24])  # nothing observed at level 3
+    want, _ = orc.kmeans_on_histogram(hist[3], 4, init.numpy()[24:28])
+    assert np.max(np.abs(cen.numpy()[24:28] - want)) < 1e-12
+    L = pq.lib()
+    assert L.pq_fit_codebooks_from_histograms(None, 1024, None, cen.data_ptr(), cen.data_ptr()) == pq.ERR_INVALID_ARG
+    assert L.pq_fit_codebooks_from_histograms(cen.data_ptr(), 4096, None, cen.data_ptr(), cen.data_ptr()) == pq.ERR_INVALID_ARG
+
+
 def test_cache_costs_62_bytes_per_token_at_d128():
     T = pq.token_block()
     assert pq.pq_cache_bytes(128, 1, 8, 32768) == 2 * 8 * 32768 * 62
@@ -104,6 +148,10 @@ def test_device_entry_points_validate_before_launching():
     assert L.pq_decode_attention(128, 32, 8, 16, 16, 16, 1, 16, 16, 0, 64, 64, 0.1, 16, 16, 16, nul) == pq.ERR_INVALID_ARG
     assert L.pq_decode_attention(128, 30, 8, 16, 16, 16, 1, 16, 16, 1, 64, 64, 0.1, 16, 16, 16, nul) == pq.ERR_INVALID_ARG
     assert L.pq_decode_attention(128, 32, 8, 16, 16, 8, 1, 16, 16, 1, 64, 64, 0.1, 16, 16, 16, nul) == pq.ERR_ALIGNMENT
+    assert L.pq_angle_histograms(128, 8, 16, 16, 16, 1, 1024, 128, 4, 1024, nul, 16, nul) == pq.ERR_INVALID_ARG
+    assert L.pq_angle_histograms(128, 8, 16, 16, 16, 1, 1024, 128, 4, 2048, 16, 16, nul) == pq.ERR_INVALID_ARG
+    assert L.pq_angle_histograms(48, 8, 16, 16, 16, 1, 1024, 128, 4, 1024, 16, 16, nul) == pq.ERR_UNSUPPORTED
+    assert L.pq_angle_histograms(128, 8, 16, 16, 16, 1, 1024, 128, 4, 1024, 20, 16, nul) == pq.ERR_ALIGNMENT
     assert L.pq_unpack_codes(128, 8, 16, 1, 64, 65, 16, 16, nul) == pq.ERR_INVALID_ARG
     assert L.pq_dequant_kv(128, 8, 16, 16, 16, 1, 64, 0, 16, nul) == pq.ERR_INVALID_ARG
 

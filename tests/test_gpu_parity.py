@@ -383,6 +383,100 @@ def test_any_level1_codebook_is_decided_in_float32_by_the_table(case, n):
     assert rel_l2(to_f64(out), ref.attend(to_f64(q), d ** -0.5)) < TOL_ATTENTION
 
 
+def _hist_close(got, want):
+    """Histograms of the same angles binned in float32 and in float64: the totals agree exactly, an angle may sit in
+    the neighbouring bin (about 1e-5 rad of error against bins of 1.5e-3 rad and more: under 1 % of the angles),
+    and no more than a few angles cross any one bin edge."""
+    assert got.shape == want.shape
+    for level in range(got.shape[0]):
+        n = int(want[level].sum())
+        assert int(got[level].sum()) == n
+        assert np.abs(got[level] - want[level]).sum() <= 0.03 * n + 4
+        assert np.abs(np.cumsum(got[level] - want[level])).max() <= 5 + 3e-4 * n
+
+
+@pytest.mark.parametrize("d,Hkv,n,dtype,n_bins", [(128, 2, 700, torch.bfloat16, 1024), (128, 3, 1000, torch.bfloat16, 256),
+                                                   (128, 2, 40, torch.bfloat16, 1024), (128, 2, 300, torch.float32, 512),
+                                                   (16, 1, 256, torch.float32, 1024), (64, 2, 100, torch.bfloat16, 64)])
+def test_angle_histograms_against_the_oracle(d, Hkv, n, dtype, n_bins):
+    """pq_angle_histograms (tensor-core kernel for long bf16 inputs at d = 128, the per-vector kernel otherwise)
+    against the oracle's histogram of the same rows; a second call adds to the first; a row with a NaN is left out."""
+    S_host = pq.pq_make_rotation(d, 31)
+    S = S_host.to(DEV)
+    status = torch.zeros(pq.STATUS_WORDS, dtype=torch.int32, device=DEV)
+    big_k, big_v = synthetic.kv_like(900 + n, n, Hkv + 1, d + 64, dtype, DEV, n_outliers=4 if d >= 64 else 0)
+    K, V = big_k[:, 1:, 32:32 + d], big_v[:, 1:, 32:32 + d]   # strided views
+    big_k[n // 2, 1, 32 + 5] *= 1e-4
+    hist = torch.zeros((4, n_bins), dtype=torch.int64, device=DEV)
+    pq.pq_angle_histograms(S, K, V, hist, status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist()[:2] == [0, 0]
+    x = np.concatenate([to_f64(K).reshape(-1, d), to_f64(V).reshape(-1, d)])
+    want = orc.angle_histograms(x, S_host.double().numpy(), 4, n_bins)
+    assert want[0].sum() == 2 * n * Hkv * d // 2 and want[3].sum() == 2 * n * Hkv * d // 16
+    _hist_close(hist.cpu().numpy(), want)
+    pq.pq_angle_histograms(S, K, V, hist, status)
+    _hist_close(hist.cpu().numpy(), 2 * want)
+    # one key row with a NaN: its 16-blocks are skipped and reported
+    bk2 = big_k.clone()
+    bk2[n // 3, 1, 32 + 7] = float("nan")
+    K2 = bk2[:, 1:, 32:32 + d]
+    hist.zero_()
+    pq.pq_angle_histograms(S, K2, V, hist, status)
+    torch.cuda.synchronize()
+    st = status.cpu().tolist()
+    assert st[0] == pq.ERR_NONFINITE and st[1] == d // 16
+    keep = np.ones(x.shape[0], dtype=bool)
+    keep[(n // 3) * Hkv + 0] = False
+    _hist_close(hist.cpu().numpy(), orc.angle_histograms(x[keep], S_host.double().numpy(), 4, n_bins))
+
+
+@pytest.mark.parametrize("kind", ["outlier_channels", "anisotropic"])
+def test_online_codebook_fit_then_encode_and_attend(kind):
+    """Section 4.1's online variant end to end: histogram of the prompt's angles on the device, clustering, encode
+    with the fitted codebook.  The codebook is compared with the oracle's own fit on the same rows (two fixed points
+    of the discrete iteration reached from histograms that differ by a few moved angles: close, not equal); the codes
+    are then compared exactly, with the library's codebook given to the oracle as data."""
+    d, Hq, Hkv, n = 128, 8, 2, 1500
+    cache = pq.PolarQuantCache(1, Hq, Hkv, d, capacity=n, seed=13, device=DEV)
+    K, V = synthetic.kv_like(77, n, Hkv, d, torch.bfloat16, DEV)
+    if kind == "anisotropic":   # rows whose rotated coordinates have unequal scales: the angle densities move
+        scales = torch.linspace(0.7, 1.4, d, device=DEV) * torch.tensor([2.0, 0.5], device=DEV).repeat(d // 2)
+        St = cache.S.t().contiguous()
+        K = ((K.float() @ cache.S) * scales @ St).to(torch.bfloat16)
+        V = ((V.float() @ cache.S) * scales.flip(0) @ St).to(torch.bfloat16)
+    analytic = cache.centroids.clone()
+    S = cache.S_host.double().numpy()
+    x = np.concatenate([to_f64(K).reshape(-1, d), to_f64(V).reshape(-1, d)])
+    err_before = None
+    for fitted in (False, True):
+        if fitted:
+            cache.lens.zero_()
+            hist = cache.fit_online_codebooks(K, V)
+            _hist_close(hist.cpu().numpy(), orc.angle_histograms(x, S, 4, pq.HIST_MAX_BINS))
+            want = orc.fit_codebooks_online(x, S, n_bins=pq.HIST_MAX_BINS)
+            for level in range(4):
+                o, k = (0, 16) if level == 0 else (16 + 4 * (level - 1), 4)
+                assert np.max(np.abs(cache.centroids.numpy()[o:o + k] - want.centroids[level])) < (2e-2 if level == 0 else 2e-3)
+            if kind == "anisotropic":
+                assert np.max(np.abs(cache.centroids.numpy() - analytic.numpy())) > 0.02  # the codebook followed the data
+        rep = _encode_and_compare(cache, K, V, [n])
+        st = cache.check_status()
+        assert st[3] < 0.02 * rep["total"], st
+        xh = to_f64(cache.dequant(n))[0]                                   # [Hkv, 2, n, d]
+        got = np.concatenate([xh[:, 0].transpose(1, 0, 2).reshape(-1, d), xh[:, 1].transpose(1, 0, 2).reshape(-1, d)])
+        err = np.sum((got - x) ** 2) / np.sum(x ** 2)
+        if fitted:
+            assert err < err_before * (0.97 if kind == "anisotropic" else 1.0005), (err, err_before)
+        err_before = err
+    ref = _oracle_cache(cache, K, V, [n])
+    q = synthetic.queries(5, 1, Hq, d, torch.bfloat16, DEV)
+    out = cache.attend(q)
+    torch.cuda.synchronize()
+    cache.check_status()
+    assert rel_l2(to_f64(out), ref.attend(to_f64(q), d ** -0.5)) < TOL_ATTENTION
+
+
 @pytest.mark.parametrize("n", [5, 40, 300])
 def test_other_codebooks_fp32_inputs_and_strided_views(n):
     """Paths beside the bf16 tensor-core encoder: a non-uniform level-1 codebook, float32 inputs (FMA rotation), strided K/V views, and chunks of every size class
