@@ -486,6 +486,57 @@ def measure_multi_query(args, pq, synthetic, dev, rank):
                                     "residual and the query likewise (3 products), and PV"}
 
 
+def measure_online_codebook(args, pq, synthetic, dev, rank):
+    """Section 4.1's online codebook on the config-2 chunk (32768 tokens x 8 kv heads, K and V): angle histograms on
+    the device, k-means on the binned angles and the table build on the host, then the encode with the fitted codebook;
+    device times from CUDA events, host times from the wall clock."""
+    cache = pq.PolarQuantCache(1, HQ, HKV, D, CTX, seed=0, device=dev)
+    Ks = [synthetic.kv_like(1000 * rank + 1 + i, CTX, HKV, D, torch.bfloat16, dev) for i in range(2)]
+    cu = torch.tensor([0, CTX], dtype=torch.int32, device=dev)
+    hist = torch.zeros((pq.N_LEVELS, pq.HIST_MAX_BINS), dtype=torch.int64, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, n=20):
+        for i in range(3):
+            fn(i)
+        evs = [(_event(), _event()) for _ in range(n)]
+        for i, (a, b) in enumerate(evs):
+            a.record(stream)
+            fn(i)
+            b.record(stream)
+        torch.cuda.synchronize()
+        return float(np.median([a.elapsed_time(b) for a, b in evs])) * 1e3
+
+    def encode(i):
+        cache.lens.zero_()
+        cache.encode(*Ks[i % 2], cu)
+
+    analytic_us = timed(encode)
+    hist_us = timed(lambda i: pq.pq_angle_histograms(cache.S, *Ks[i % 2], hist, cache.status))
+    hist.zero_()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    pq.pq_angle_histograms(cache.S, *Ks[0], hist, cache.status)
+    h = hist.cpu()
+    t1 = time.perf_counter()
+    cen, bnd = pq.pq_fit_codebooks_from_histograms(h)
+    t2 = time.perf_counter()
+    tables = pq.pq_build_tables(cen, bnd)
+    t3 = time.perf_counter()
+    cache.set_codebooks(cen, bnd)
+    torch.cuda.synchronize()
+    t4 = time.perf_counter()
+    fitted_us = timed(encode)
+    st = cache.check_status()
+    return {"tokens": CTX, "kv_heads": HKV, "bins": pq.HIST_MAX_BINS, "histogram_us": hist_us,
+            "histogram_gbs": 2 * CTX * HKV * D * 2 / (hist_us * 1e-6) / 1e9,
+            "histogram_and_d2h_wall_us": (t1 - t0) * 1e6, "kmeans_host_us": (t2 - t1) * 1e6,
+            "tables_host_us": (t3 - t2) * 1e6, "tables_h2d_wall_us": (t4 - t3) * 1e6 - (t3 - t2) * 1e6,
+            "encode_fitted_codebook_us": fitted_us, "encode_analytic_codebook_us": analytic_us,
+            "max_centroid_shift_rad": float((cen - pq.pq_fit_codebooks()[0]).abs().max()),
+            "float64_decisions": st[3], "rank": rank}
+
+
 def measure_config5(args, pq, synthetic, dev, rank):
     """Config 5: batch 16, ragged contexts in [4096, 65536], prefill in 4096-token chunks, then 128 steps of
     (append one token per sequence, decode attention)."""
@@ -622,6 +673,8 @@ def reduce_and_format(local, steps, warmup, rank, world, dist=None, device="cpu"
         t = red[pos_mq if c5 else pos]
         line["configs"]["multi_query_chunk"] = dict(mq, ms=t, us_per_query=t / mq["n_q"] * 1e3,
                                                     mma_tflops=mq["mma_tflops"] * mq["ms"] / t)
+    if local.get("online"):
+        line["configs"]["online_codebook"] = local["online"]  # this rank's own figures (not reduced over ranks)
     if cpu_baseline is not None:
         line["cpu_baseline"] = cpu_baseline
     return line
@@ -649,6 +702,8 @@ def run_cuda(args):
         local["cfg5"] = measure_config5(args, pq, synthetic, dev, rank)
         torch.cuda.empty_cache()
         local["multi_query"] = measure_multi_query(args, pq, synthetic, dev, rank)
+        torch.cuda.empty_cache()
+        local["online"] = measure_online_codebook(args, pq, synthetic, dev, rank)
         torch.cuda.empty_cache()
     cpu = _oracle_sample_throughput(12.0) if rank == 0 and world == 1 and not args.no_cpu_baseline else None
     line = reduce_and_format(local, args.steps, args.warmup, rank, world, dist, dev, cpu)

@@ -29,7 +29,7 @@ struct FastQuant {
   float t2[3][3];   // tan^2 of the three boundaries of levels 2, 3, 4
   uint32_t sym;     // the boundaries of every level >= 2 are b, pi/4, pi/2 - b (kFlagSymmetricUpper)
   uint32_t analytic;       // sym and the uniform level-1 codebook: every decision is a sign test
-  const uint2* l1_cells;   // level-1 decision table of any other codebook (Tables::l1_cells)
+  const uint2* l1_cells;   // level-1 decision table of any other codebook (Tables::l1_cells or a copy in shared memory)
 };
 
 __device__ inline void load_fast_quant(const Tables* tb, FastQuant* fq) {
@@ -172,7 +172,7 @@ __device__ __forceinline__ void quant_level1_table_push(float a, float b, float 
   const uint32_t o = push_sign(push_sign(push_sign(0u, __float_as_uint(b)), __float_as_uint(a)), __float_as_uint(ax - ay));
   // 2^20 + t * scale: the float's unit in the last place is 1/8, so mantissa bits 3.. hold floor(t * scale + 1/16)
   const uint32_t cell8 = __float_as_uint(fmaf(t, kL1CellScale, 1048576.f)) & (uint32_t)((kL1Cells - 1) << 3);
-  const uint2 e = __ldg(reinterpret_cast<const uint2*>(reinterpret_cast<const char*>(cells) + (o * (kL1Cells * 8) + cell8)));
+  const uint2 e = *reinterpret_cast<const uint2*>(reinterpret_cast<const char*>(cells) + (o * (kL1Cells * 8) + cell8));
   const float dd = t - __uint_as_float(e.x);
   const float slack = fmaf(-fabsf(dd), u, fmaf(6e-7f, u, dy3));  // < 0: certified (NaN: not)
   const uint32_t code = e.y << (dd > 0.f ? 4 : 0);                // the code in bits 28..31

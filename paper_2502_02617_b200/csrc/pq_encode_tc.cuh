@@ -43,7 +43,8 @@ constexpr int kTcSmFq = kTcSmX + kTcStages * kTcXBytes;      // FastQuant (40 B)
 constexpr int kTcSmBar = kTcSmFq + 64;                       // x_full[kTcStages], acc_full[kTcSlots]
 constexpr int kTcSmMisc = kTcSmBar + 64;                     // tmem base, abort flag, copies issued per stage
 constexpr int kTcSmFix = kTcSmMisc + 64;                     // one TcFixQueue per slot
-constexpr int kTcSmTotal = kTcSmFix + kTcSlots * (int)sizeof(TcFixQueue) + 1024;  // + slack for 1024-byte alignment
+constexpr int kTcSmL1 = kTcSmFix + kTcSlots * (int)sizeof(TcFixQueue);  // copy of Tables::l1_cells (codebooks other than the analytic ones)
+constexpr int kTcSmTotal = kTcSmL1 + 8 * kL1Cells * 8 + 1024;             // + slack for 1024-byte alignment
 constexpr int kTcSpin = 1 << 22;
 static_assert(kTcTerms == 3, "kRotErrTc is the bound for three terms");
 static_assert(sizeof(TcFixQueue) % 16 == 0, "queues are laid out back to back");
@@ -214,13 +215,21 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     for (int it = 0; it < kTcStages; ++it) issue_tma(it);  // the first tiles arrive while S is split
-    if (!kHist) load_fast_quant(a.tables, fq);
+    if (!kHist) {
+      load_fast_quant(a.tables, fq);
+      fq->l1_cells = reinterpret_cast<const uint2*>(smem + kTcSmL1);  // the copy made below
+    }
   }
   uint32_t* hist_s = reinterpret_cast<uint32_t*>(smem + kTcSmFix);
   if (kHist) {
     for (int i = tid; i < 4 * a.n_bins; i += kTcThreads) hist_s[i] = 0u;
-  } else if (st < 4) {
-    fixq->count[st] = 0;
+  } else {
+    if (st < 4) fixq->count[st] = 0;
+    if ((a.tables->flags & (kFlagSymmetricUpper | kFlagUniformL1)) != (kFlagSymmetricUpper | kFlagUniformL1)) {
+      const uint2* src = &a.tables->l1_cells[0][0];
+      uint2* dst = reinterpret_cast<uint2*>(smem + kTcSmL1);
+      for (int i = tid; i < 8 * kL1Cells; i += kTcThreads) dst[i] = __ldg(src + i);
+    }
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(sb + kTcSmMisc) : "memory");

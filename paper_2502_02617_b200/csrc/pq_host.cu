@@ -137,8 +137,8 @@ bool build_l1_cells(const double* bnd, uint2 (*cells)[pq::kL1Cells]) {
       if (tau != tau) continue;
       const double scale = (double)pq::kL1CellScale;
       const double lo = std::fmax(0.0, (c - 1.0 / 16.0) / scale), hi = std::fmin(1.0, (c + 15.0 / 16.0) / scale);
-      for (int i = 0; i <= 16; ++i) {
-        const double t = lo + (hi - lo) * i / 16.0, dist = std::fabs(t - (double)tau);
+      for (int i = 0; i <= 4; ++i) {
+        const double t = lo + (hi - lo) * i / 4.0, dist = std::fabs(t - (double)tau);
         double nearest = 1e30;
         for (const L1Ray& r : rays) nearest = std::fmin(nearest, std::fabs(t - r.t));
         if (dist > nearest + 1e-7) return false;
@@ -394,12 +394,17 @@ int32_t pq_build_tables(const double* cen, const double* bnd, void* tables_host)
     t.t1p_hi[e] = make_uint2((ha & 0xFFFFu) | (hb << 16), (ha >> 16) | (hb & 0xFFFF0000u));
     t.t1p_lo[e] = make_uint2((la & 0xFFFFu) | (lb << 16), (la >> 16) | (lb & 0xFFFF0000u));
   }
+  double uc[12], us[12];  // cos / sin of the centroids of levels 2, 3, 4
+  for (int k = 0; k < 12; ++k) {
+    uc[k] = std::cos(cen[16 + k]);
+    us[k] = std::sin(cen[16 + k]);
+  }
   for (int s = 0; s < 4; ++s)
     for (int i = 0; i < 64; ++i) {
-      const double a2 = cen[16 + (i & 3)], a3 = cen[20 + ((i >> 2) & 3)], a4 = cen[24 + (i >> 4)];
-      const double t4 = (s >> 1) ? std::sin(a4) : std::cos(a4);
-      const double t3 = (s & 1) ? std::sin(a3) : std::cos(a3);
-      split(t4 * t3 * std::cos(a2), t4 * t3 * std::sin(a2), &t.u_tab[s][i].x, &t.u_tab[s][i].y);
+      const int k2 = i & 3, k3 = 4 + ((i >> 2) & 3), k4 = 8 + (i >> 4);
+      const double t4 = (s >> 1) ? us[k4] : uc[k4];
+      const double t3 = (s & 1) ? us[k3] : uc[k3];
+      split(t4 * t3 * uc[k2], t4 * t3 * us[k2], &t.u_tab[s][i].x, &t.u_tab[s][i].y);
     }
   if (!build_l1_cells(bnd, t.l1_cells)) return PQ_ERR_INVALID_ARG;
   std::memcpy(tables_host, &t, sizeof(t));
