@@ -538,6 +538,40 @@ def measure_online_codebook(args, pq, synthetic, dev, rank):
             "float64_decisions": st[3], "rank": rank}
 
 
+def measure_paged(args, pq, synthetic, dev, rank):
+    """Config 3 behind a block table: 8 x 32768 tokens in 256-token pages drawn in random order from one pool; the
+    same decode-attention kernel with one table lookup per 128-token stage."""
+    P = 256
+    pages_per_seq = CTX // P
+    n_pages = BATCH * pages_per_seq
+    rng = np.random.default_rng(7 + rank)
+    table = torch.from_numpy(rng.permutation(n_pages).reshape(BATCH, pages_per_seq).astype(np.int32))
+    caches = [pq.PagedPolarQuantCache(BATCH, HQ, HKV, D, P, n_pages, table, seed=0, device=dev) for _ in range(2)]
+    for c, cache in enumerate(caches):
+        for b in range(BATCH):
+            K, V = synthetic.kv_like(1000 * rank + 10 + (b + c) % 2, CTX, HKV, D, torch.bfloat16, dev)
+            cu = torch.zeros(BATCH + 1, dtype=torch.int32, device=dev)
+            cu[b + 1:] = CTX
+            cache.encode(K, V, cu)
+    q = synthetic.queries(3, BATCH, HQ, D, torch.bfloat16, dev)
+    out = torch.empty_like(q)
+    stream = torch.cuda.current_stream()
+    for i in range(4):
+        caches[i % 2].attend(q, out=out)
+    evs = [(_event(), _event()) for _ in range(40)]
+    for i, (a, b) in enumerate(evs):   # the two caches (520 MB) alternate: no block is still in L2 when it is read again
+        a.record(stream)
+        caches[i % 2].attend(q, out=out)
+        b.record(stream)
+    torch.cuda.synchronize()
+    for cache in caches:
+        cache.check_status()
+    t = float(np.median([a.elapsed_time(b) for a, b in evs]))
+    comp = BATCH * HKV * CTX * 124
+    return {"batch": BATCH, "ctx": CTX, "page_tokens": P, "pages": n_pages, "decode_us": t * 1e3,
+            "gbs": comp / (t * 1e-3) / 1e9, "rank": rank}
+
+
 def measure_config5(args, pq, synthetic, dev, rank):
     """Config 5: batch 16, ragged contexts in [4096, 65536], prefill in 4096-token chunks, then 128 steps of
     (append one token per sequence, decode attention)."""
@@ -674,6 +708,8 @@ def reduce_and_format(local, steps, warmup, rank, world, dist=None, device="cpu"
         t = red[pos_mq if c5 else pos]
         line["configs"]["multi_query_chunk"] = dict(mq, ms=t, us_per_query=t / mq["n_q"] * 1e3,
                                                     mma_tflops=mq["mma_tflops"] * mq["ms"] / t)
+    if local.get("paged"):
+        line["configs"]["paged_decode"] = dict(local["paged"], hbm_frac_measured=local["paged"]["gbs"] / peak)
     if local.get("online"):
         line["configs"]["online_codebook"] = local["online"]  # this rank's own figures (not reduced over ranks)
     if cpu_baseline is not None:
@@ -705,6 +741,8 @@ def run_cuda(args):
         local["multi_query"] = measure_multi_query(args, pq, synthetic, dev, rank)
         torch.cuda.empty_cache()
         local["online"] = measure_online_codebook(args, pq, synthetic, dev, rank)
+        torch.cuda.empty_cache()
+        local["paged"] = measure_paged(args, pq, synthetic, dev, rank)
         torch.cuda.empty_cache()
     cpu = _oracle_sample_throughput(12.0) if rank == 0 and world == 1 and not args.no_cpu_baseline else None
     line = reduce_and_format(local, args.steps, args.warmup, rank, world, dist, dev, cpu)

@@ -274,6 +274,54 @@ int32_t pq_dequant_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, 
                       const void* cache_dev, int32_t batch, int32_t capacity, int32_t n_tokens,
                       float* x_hat_dev, void* stream);
 
+/*
+ * Paged cache (the packed layout of Section 4.1 behind a block table, as a serving engine keeps it): the cache is a
+ * pool of n_pages pages; a page holds page_tokens tokens of every kv head -- [kv head][token-block of the page][K | V],
+ * the layout of a contiguous cache of capacity page_tokens -- and sequence b's logical page p (positions
+ * p * page_tokens ..) is physical page page_table[b * pages_per_seq + p].  A sequence may grow to
+ * pages_per_seq * page_tokens tokens; only the table entries of pages it reaches are read.
+ *   page_table_dev   device, int32[batch][pages_per_seq], 4-byte aligned; entries must name distinct pages for
+ *                    distinct (sequence, logical page) -- the library cannot check that -- and lie in [0, n_pages):
+ *                    a row whose page lies outside the pool is not written and its sequence does not grow (encode,
+ *                    append), a reader reads page 0 instead; both record PQ_ERR_INVALID_ARG in the status words
+ *   page_tokens      multiple of the token-block (pq_token_block()), of 128 at head_dim 128
+ * The struct itself is read on the host during the call.  The *_paged entry points below are their contiguous
+ * namesakes with `capacity` replaced by the paging; everything else (arguments, status words, tolerances) is the same,
+ * and the codes, radii and attention outputs are those of a contiguous cache holding the same tokens.
+ */
+typedef struct pq_paging {
+  const int32_t* page_table_dev;
+  int32_t page_tokens;
+  int32_t pages_per_seq;
+  int32_t n_pages;
+} pq_paging;
+
+/* Bytes of a pool of n_pages pages. */
+int64_t pq_paged_cache_bytes(int32_t head_dim, int32_t n_kv_heads, int32_t page_tokens, int32_t n_pages);
+int32_t pq_encode_kv_paged(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                           const void* K_dev, const void* V_dev, int32_t in_dtype, int64_t token_stride,
+                           int64_t head_stride, const int32_t* cu_seqlens_dev, int32_t batch, int32_t total_tokens,
+                           void* cache_dev, int32_t* cache_lens_dev, const pq_paging* paging, int32_t* status_dev,
+                           void* stream);
+int32_t pq_append_kv_paged(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                           const void* k_new_dev, const void* v_new_dev, int32_t in_dtype, int32_t batch,
+                           void* cache_dev, int32_t* cache_lens_dev, const pq_paging* paging, int32_t* status_dev,
+                           void* stream);
+int32_t pq_decode_attention_paged(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                                  const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
+                                  const int32_t* cache_lens_dev, int32_t batch, const pq_paging* paging, int32_t max_len,
+                                  float scale, void* out_dev, void* workspace_dev, int32_t* status_dev, void* stream);
+int32_t pq_multi_query_attention_paged(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                                       const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
+                                       const int32_t* cache_lens_dev, int32_t batch, int32_t n_q, const pq_paging* paging,
+                                       int32_t max_len, float scale, void* out_dev, void* workspace_dev,
+                                       int32_t* status_dev, void* stream);
+int32_t pq_unpack_codes_paged(int32_t head_dim, int32_t n_kv_heads, const void* cache_dev, int32_t batch,
+                              const pq_paging* paging, int32_t n_tokens, uint8_t* codes_dev, void* radii_dev, void* stream);
+int32_t pq_dequant_kv_paged(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                            const void* cache_dev, int32_t batch, const pq_paging* paging, int32_t n_tokens,
+                            float* x_hat_dev, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

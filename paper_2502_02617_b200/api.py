@@ -57,7 +57,31 @@ _SIGNATURES = {
     "pq_unpack_codes": (c_int32, [c_int32, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p]),
     "pq_dequant_kv": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p,
                                 c_void_p]),
+    "pq_paged_cache_bytes": (c_int64, [c_int32, c_int32, c_int32, c_int32]),
+    "pq_encode_kv_paged": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int64, c_int64,
+                                     c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "pq_append_kv_paged": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int32,
+                                     c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "pq_decode_attention_paged": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p,
+                                            c_void_p, c_int32, c_void_p, c_int32, c_float, c_void_p, c_void_p, c_void_p,
+                                            c_void_p]),
+    "pq_multi_query_attention_paged": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p,
+                                                 c_void_p, c_int32, c_int32, c_void_p, c_int32, c_float, c_void_p,
+                                                 c_void_p, c_void_p, c_void_p]),
+    "pq_unpack_codes_paged": (c_int32, [c_int32, c_int32, c_void_p, c_int32, c_void_p, c_int32, c_void_p, c_void_p, c_void_p]),
+    "pq_dequant_kv_paged": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p, c_int32, c_void_p,
+                                      c_void_p]),
 }
+
+
+class Paging(ctypes.Structure):
+    """struct pq_paging of include/polarquant.h."""
+    _fields_ = [("page_table_dev", c_void_p), ("page_tokens", c_int32), ("pages_per_seq", c_int32), ("n_pages", c_int32)]
+
+    @classmethod
+    def of(cls, page_table: torch.Tensor, page_tokens: int, n_pages: int) -> "Paging":
+        assert page_table.dtype == torch.int32 and page_table.is_contiguous() and page_table.dim() == 2
+        return cls(page_table.data_ptr(), page_tokens, page_table.shape[1], n_pages)
 
 _lib = None
 
@@ -259,6 +283,13 @@ def pq_dequant_kv(d, n_kv_heads, S, tables, cache, batch, capacity, n_tokens, st
     return out
 
 
+def pq_paged_cache_bytes(d: int, n_kv_heads: int, page_tokens: int, n_pages: int) -> int:
+    n = int(lib().pq_paged_cache_bytes(d, n_kv_heads, page_tokens, n_pages))
+    if n < 0:
+        raise PolarQuantError(n, "pq_paged_cache_bytes")
+    return n
+
+
 class PolarQuantCache:
     """Convenience owner of the device buffers one (layer's) compressed KV cache needs."""
 
@@ -326,3 +357,91 @@ class PolarQuantCache:
         if st[0] != OK:
             raise PolarQuantError(st[0], "device status")
         return st
+
+
+class PagedPolarQuantCache(PolarQuantCache):
+    """The same cache behind a block table: a pool of `n_pages` pages of `page_tokens` tokens (all kv heads), and
+    page_table int32 [batch, pages_per_seq] naming the physical page of every logical page of every sequence."""
+
+    def __init__(self, batch, n_q_heads, n_kv_heads, d, page_tokens, n_pages, page_table, seed=0, device="cuda", S=None,
+                 codebooks=None):
+        self.batch, self.n_q_heads, self.n_kv_heads, self.d = batch, n_q_heads, n_kv_heads, d
+        self.page_tokens, self.n_pages = page_tokens, n_pages
+        self.device = torch.device(device)
+        self.page_table = page_table.to(torch.int32).to(self.device).contiguous()
+        assert self.page_table.shape[0] == batch
+        self.capacity = page_tokens * self.page_table.shape[1]
+        self.S_host = pq_make_rotation(d, seed) if S is None else S.to(torch.float32).cpu().contiguous()
+        self.centroids, self.boundaries = pq_fit_codebooks() if codebooks is None else codebooks
+        self.S = self.S_host.to(self.device)
+        self.tables = pq_build_tables(self.centroids, self.boundaries).to(self.device)
+        self.cache = torch.empty(pq_paged_cache_bytes(d, n_kv_heads, page_tokens, n_pages), dtype=torch.uint8, device=self.device)
+        self.lens = torch.zeros(batch, dtype=torch.int32, device=self.device)
+        self.status = torch.zeros(STATUS_WORDS, dtype=torch.int32, device=self.device)
+        self.workspace = torch.empty(pq_workspace_bytes(d, batch, n_q_heads, n_kv_heads, self.capacity), dtype=torch.uint8,
+                                     device=self.device)
+
+    def _paging(self):
+        return Paging.of(self.page_table, self.page_tokens, self.n_pages)
+
+    def encode(self, K, V, cu_seqlens, stream=None):
+        total, n_kv_heads, d = K.shape
+        assert V.shape == K.shape and V.dtype == K.dtype and K.stride(2) == 1 and V.stride() == K.stride()
+        pg = self._paging()
+        _check(lib().pq_encode_kv_paged(d, n_kv_heads, _ptr(self.S), _ptr(self.tables), _ptr(K), _ptr(V), _dtype_code(K),
+                                        K.stride(0), K.stride(1), _ptr(cu_seqlens), cu_seqlens.numel() - 1, total,
+                                        _ptr(self.cache), _ptr(self.lens), ctypes.addressof(pg), _ptr(self.status),
+                                        _stream(stream)), "pq_encode_kv_paged")
+
+    def append(self, k_new, v_new, stream=None):
+        batch, n_kv_heads, d = k_new.shape
+        assert k_new.is_contiguous() and v_new.is_contiguous() and v_new.shape == k_new.shape
+        pg = self._paging()
+        _check(lib().pq_append_kv_paged(d, n_kv_heads, _ptr(self.S), _ptr(self.tables), _ptr(k_new), _ptr(v_new),
+                                        _dtype_code(k_new), batch, _ptr(self.cache), _ptr(self.lens), ctypes.addressof(pg),
+                                        _ptr(self.status), _stream(stream)), "pq_append_kv_paged")
+
+    def attend(self, q, out=None, scale=None, max_len=None, stream=None):
+        out = torch.empty_like(q) if out is None else out
+        batch, n_q_heads, d = q.shape
+        assert q.is_contiguous() and out.is_contiguous() and out.shape == q.shape and out.dtype == q.dtype
+        pg = self._paging()
+        _check(lib().pq_decode_attention_paged(d, n_q_heads, self.n_kv_heads, _ptr(self.S), _ptr(self.tables), _ptr(q),
+                                               _dtype_code(q), _ptr(self.cache), _ptr(self.lens), batch,
+                                               ctypes.addressof(pg), self.capacity if max_len is None else max_len,
+                                               float(self.d ** -0.5 if scale is None else scale), _ptr(out),
+                                               _ptr(self.workspace), _ptr(self.status), _stream(stream)),
+               "pq_decode_attention_paged")
+        return out
+
+    def attend_multi(self, q, out=None, scale=None, max_len=None, stream=None):
+        out = torch.empty_like(q) if out is None else out
+        batch, n_q, n_q_heads, d = q.shape
+        assert q.is_contiguous() and out.is_contiguous() and out.shape == q.shape and out.dtype == q.dtype
+        need = pq_workspace_bytes(self.d, self.batch * n_q, self.n_q_heads, self.n_kv_heads, self.capacity)
+        if getattr(self, "_multi_ws", None) is None or self._multi_ws.numel() < need:
+            self._multi_ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        pg = self._paging()
+        _check(lib().pq_multi_query_attention_paged(d, n_q_heads, self.n_kv_heads, _ptr(self.S), _ptr(self.tables), _ptr(q),
+                                                    _dtype_code(q), _ptr(self.cache), _ptr(self.lens), batch, n_q,
+                                                    ctypes.addressof(pg), self.capacity if max_len is None else max_len,
+                                                    float(self.d ** -0.5 if scale is None else scale), _ptr(out),
+                                                    _ptr(self._multi_ws), _ptr(self.status), _stream(stream)),
+               "pq_multi_query_attention_paged")
+        return out
+
+    def unpack(self, n_tokens):
+        codes = torch.zeros((self.batch, self.n_kv_heads, 2, n_tokens, 15 * self.d // 16), dtype=torch.uint8, device=self.device)
+        radii = torch.zeros((self.batch, self.n_kv_heads, 2, n_tokens, self.d // 16), dtype=torch.float16, device=self.device)
+        pg = self._paging()
+        _check(lib().pq_unpack_codes_paged(self.d, self.n_kv_heads, _ptr(self.cache), self.batch, ctypes.addressof(pg),
+                                           n_tokens, _ptr(codes), _ptr(radii), _stream(None)), "pq_unpack_codes_paged")
+        return codes, radii
+
+    def dequant(self, n_tokens):
+        out = torch.zeros((self.batch, self.n_kv_heads, 2, n_tokens, self.d), dtype=torch.float32, device=self.device)
+        pg = self._paging()
+        _check(lib().pq_dequant_kv_paged(self.d, self.n_kv_heads, _ptr(self.S), _ptr(self.tables), _ptr(self.cache),
+                                         self.batch, ctypes.addressof(pg), n_tokens, _ptr(out), _stream(None)),
+               "pq_dequant_kv_paged")
+        return out

@@ -106,8 +106,43 @@ __host__ __device__ inline Layout make_layout(int head_dim, int capacity) {
   return L;
 }
 
-// Start of the token-block that holds position `pos` of (sequence b, head h), K (kv=0) or V (kv=1).
-__host__ __device__ inline int64_t block_offset(const Layout& L, int n_kv_heads, int b, int h, int kv, int pos) {
+// Where the token-blocks of a sequence live.  The cache is a pool of pages; a page holds `page_tokens` tokens of every
+// kv head, head-major: [kv head][token-block of the page][K | V] (Layout::head_bytes per head, with the layout made
+// for page_tokens).  Contiguous cache (table == nullptr): sequence b owns page b, of `capacity` tokens.  Paged cache:
+// logical page p of sequence b is physical page table[b * pages_per_seq + p] of a pool of n_pages.
+struct Paging {
+  const int32_t* table;
+  int page_tokens;    // multiple of kTokenBlock (of 128 at head_dim 128 for the persistent decode kernel) when paged
+  int pages_per_seq;
+  int n_pages;
+};
+__host__ __device__ inline Paging contiguous_paging(int capacity, int batch) {
+  Paging pg;
+  pg.table = nullptr; pg.page_tokens = capacity; pg.pages_per_seq = 1; pg.n_pages = batch;
+  return pg;
+}
+
+// Start of head h's part of the page that holds position `pos` of sequence b; -1 if the table names a page outside
+// the pool.
+__device__ __forceinline__ int64_t head_page_offset(const Layout& L, const Paging& pg, int n_kv_heads, int b, int h, int pos) {
+  int page = b;
+  if (pg.table != nullptr) {
+    page = __ldg(pg.table + (int64_t)b * pg.pages_per_seq + pos / pg.page_tokens);
+    if ((unsigned)page >= (unsigned)pg.n_pages) return -1;
+  }
+  return ((int64_t)page * n_kv_heads + h) * L.head_bytes;
+}
+// Start of the token-block that holds position `pos` of (sequence b, head h), K (kv=0) or V (kv=1); -1: bad page.
+__device__ __forceinline__ int64_t block_offset_paged(int block_bytes, int64_t head_bytes, const int32_t* table, int page_tokens,
+                                                   int pages_per_seq, int n_pages, int n_kv_heads, int b, int h, int kv, int pos) {
+  const int page = __ldg(table + (int64_t)b * pages_per_seq + pos / page_tokens);
+  if ((unsigned)page >= (unsigned)n_pages) return -1;
+  return ((int64_t)page * n_kv_heads + h) * head_bytes + ((int64_t)((pos % page_tokens) / kTokenBlock) * 2 + kv) * block_bytes;
+}
+__device__ __forceinline__ int64_t block_offset(const Layout& L, const Paging& pg, int n_kv_heads, int b, int h, int kv, int pos) {
+  if (pg.table != nullptr)
+    return block_offset_paged(L.block_bytes, L.head_bytes, pg.table, pg.page_tokens, pg.pages_per_seq, pg.n_pages, n_kv_heads, b,
+                              h, kv, pos);
   return ((int64_t)b * n_kv_heads + h) * L.head_bytes + ((int64_t)(pos / kTokenBlock) * 2 + kv) * L.block_bytes;
 }
 
@@ -172,6 +207,7 @@ void note_cuda_error(cudaError_t e);
 // Test hook (pq_debug_fail_next_wait): returns true once after the hook was armed for `which`
 // (1 = tensor-core encoder, 2 = head_dim-128 decode attention) and disarms it.
 bool take_debug_wait_failure(int which);
+int32_t paging_from(const pq_paging* p, int head_dim, Paging* out);
 inline int32_t launch_status() {
   const cudaError_t e = cudaGetLastError();
   if (e == cudaSuccess) return PQ_OK;
@@ -213,6 +249,21 @@ inline int configure_for_device(Kernel kernel, int smem_bytes, DeviceMemo& state
 // Record the first error seen.
 __device__ inline void set_status(int32_t* status, int32_t code) {
   if (status != nullptr) atomicCAS(status, 0, code);
+}
+
+// Readers: offset of the K block of token-block jb of (sequence b, head h); its V block follows it, and so does the
+// next token-block of the same page.  A page outside the pool is reported and page 0 is read instead (the output
+// for that sequence is then meaningless, but no address outside the cache is formed).
+__device__ __forceinline__ int64_t kv_block_pair_offset(const Layout& L, const Paging& pg, int n_kv_heads, int b, int h, int jb,
+                                                        int32_t* status) {
+  if (pg.table == nullptr) return ((int64_t)b * n_kv_heads + h) * L.head_bytes + (int64_t)jb * 2 * L.block_bytes;
+  int64_t off = block_offset_paged(L.block_bytes, L.head_bytes, pg.table, pg.page_tokens, pg.pages_per_seq, pg.n_pages, n_kv_heads,
+                                   b, h, 0, jb * kTokenBlock);
+  if (off < 0) {
+    set_status(status, PQ_ERR_INVALID_ARG);
+    off = (int64_t)h * L.head_bytes;
+  }
+  return off;
 }
 
 }  // namespace pq

@@ -137,6 +137,7 @@ struct DecodeArgs {
   void* out;
   int32_t* status;
   Workspace ws;
+  Paging pg;  // where the cache's token-blocks live
   // Sequence of (sequence, query) pair p, and the cached tokens its query sees: query j of the n_q last positions of
   // a sequence attends to the tokens before and at its own position (Section 4: the i-th query sees i tokens).
   __device__ __forceinline__ int seq_of(int p) const { return n_q == 1 ? p : p / n_q; }
@@ -264,7 +265,7 @@ __device__ void combine_and_store(const DecodeArgs& a, int b, int hk, int g, int
 __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem[];
   const int d = a.d, g = a.n_q_heads / a.n_kv_heads;
-  const Layout L = make_layout(d, a.capacity);
+  const Layout L = make_layout(d, a.pg.page_tokens);
   const int split = blockIdx.x, hk = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
@@ -298,12 +299,12 @@ __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel
   const int per = (nblk_total + a.ws.n_splits - 1) / a.ws.n_splits;
   const int j0 = split * per;
   const int j1 = min(nblk_total, j0 + per);
-  const uint8_t* head_base = a.cache + ((int64_t)a.seq_of(b) * a.n_kv_heads + hk) * L.head_bytes;
+  const int seq = a.seq_of(b);
   __syncthreads();
 
   for (int jb = j0; jb < j1; ++jb) {
     {
-      const uint4* src = reinterpret_cast<const uint4*>(head_base + (int64_t)jb * 2 * L.block_bytes);
+      const uint4* src = reinterpret_cast<const uint4*>(a.cache + kv_block_pair_offset(L, a.pg, a.n_kv_heads, seq, hk, jb, a.status));
       uint4* dst = reinterpret_cast<uint4*>(smem);
       for (int i = tid; i < 2 * L.block_bytes / 16; i += kSimpleThreads) dst[i] = src[i];
     }
@@ -407,9 +408,9 @@ __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel
 namespace pq {
 
 // ---- inspection kernels ----------------------------------------------------------------------
-__global__ void unpack_codes_kernel(int d, int n_kv_heads, const uint8_t* cache, int batch, int capacity,
+__global__ void unpack_codes_kernel(int d, int n_kv_heads, const uint8_t* cache, int batch, Paging pg,
                                     int n_tokens, uint8_t* codes, __half* radii) {
-  const Layout L = make_layout(d, capacity);
+  const Layout L = make_layout(d, pg.page_tokens);
   const int64_t n = (int64_t)batch * n_kv_heads * 2 * n_tokens;
   const int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (v >= n) return;
@@ -417,7 +418,9 @@ __global__ void unpack_codes_kernel(int d, int n_kv_heads, const uint8_t* cache,
   const int kv = (int)((v / n_tokens) & 1);
   const int h = (int)((v / (2 * (int64_t)n_tokens)) % n_kv_heads);
   const int b = (int)(v / (2 * (int64_t)n_tokens * n_kv_heads));
-  const uint8_t* tb = cache + block_offset(L, n_kv_heads, b, h, kv, tok);
+  const int64_t off = block_offset(L, pg, n_kv_heads, b, h, kv, tok);
+  if (off < 0) return;  // a page outside the pool: the outputs of this token keep what they held
+  const uint8_t* tb = cache + off;
   const int t = tok % kTokenBlock;
   const int n_codes = 15 * L.nb;
   uint8_t* out = codes + v * n_codes;
@@ -433,10 +436,10 @@ __global__ void unpack_codes_kernel(int d, int n_kv_heads, const uint8_t* cache,
 }
 
 __global__ void dequant_kernel(int d, int n_kv_heads, const float* S, const Tables* tables, const uint8_t* cache,
-                               int capacity, int n_tokens, float* x_hat) {
+                               Paging pg, int n_tokens, float* x_hat) {
   extern __shared__ float ysm[];
   __shared__ float cc[32], cs[32];
-  const Layout L = make_layout(d, capacity);
+  const Layout L = make_layout(d, pg.page_tokens);
   const int64_t v = blockIdx.x;
   const int j = threadIdx.x;
   for (int i = j; i < PQ_N_CENTROIDS; i += blockDim.x) {
@@ -448,7 +451,9 @@ __global__ void dequant_kernel(int d, int n_kv_heads, const float* S, const Tabl
   const int kv = (int)((v / n_tokens) & 1);
   const int h = (int)((v / (2 * (int64_t)n_tokens)) % n_kv_heads);
   const int b = (int)(v / (2 * (int64_t)n_tokens * n_kv_heads));
-  const uint8_t* tb = cache + block_offset(L, n_kv_heads, b, h, kv, tok);
+  const int64_t off = block_offset(L, pg, n_kv_heads, b, h, kv, tok);
+  if (off < 0) return;  // uniform over the CTA
+  const uint8_t* tb = cache + off;
   if (d == 128) {
     // the fp16 arithmetic of the attention kernel's value path: u = rn(r * U), x = rn(u * t1)
     const int t = tok % kTokenBlock, blk = j >> 4, i = j & 15;
@@ -483,8 +488,9 @@ int64_t pq_workspace_bytes(int32_t head_dim, int32_t batch, int32_t n_q_heads, i
 
 static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
                                 const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
-                                const int32_t* cache_lens_dev, int32_t batch, int32_t n_q, int32_t capacity, int32_t max_len,
-                                float scale, void* out_dev, void* workspace_dev, int32_t* status_dev, void* stream) {
+                                const int32_t* cache_lens_dev, int32_t batch, int32_t n_q, int32_t capacity, const pq::Paging& pg,
+                                int32_t max_len, float scale, void* out_dev, void* workspace_dev, int32_t* status_dev,
+                                void* stream) {
   if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
   if (!S_dev || !tables_dev || !q_dev || !cache_dev || !cache_lens_dev || !out_dev || !workspace_dev || !status_dev)
     return PQ_ERR_INVALID_ARG;
@@ -503,6 +509,7 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
   a.io_dtype = io_dtype; a.scale = scale; a.S = S_dev; a.tables = reinterpret_cast<const pq::Tables*>(tables_dev);
   a.q = q_dev; a.cache = reinterpret_cast<const uint8_t*>(cache_dev); a.lens = cache_lens_dev; a.out = out_dev;
   a.status = status_dev;
+  a.pg = pg;
   a.ws = pq::carve_workspace(workspace_dev, head_dim, (int)pairs, n_q_heads, n_kv_heads, max_len);
   const int g = n_q_heads / n_kv_heads;
   if (head_dim == 128 && n_q * g >= pq::kPfRows) {
@@ -527,19 +534,21 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
     }()};
     a.epoch = call_epoch.fetch_add(0x9E3779B1u, std::memory_order_relaxed) | 0x80000000u;
     a.debug = pq::take_debug_wait_failure(2) ? 1u : 0u;
-    static pq::DeviceMemo configured4, configured8;
-    const int n_sm = g <= 4 ? pq::configure_for_device(pq::decode_attention_fast_kernel<1>, pq::kSmTotal, configured4)
-                            : pq::configure_for_device(pq::decode_attention_fast_kernel<2>, pq::kSmTotal, configured8);
+    static pq::DeviceMemo configured[4];
+    const bool paged = pg.table != nullptr;
+    void (*kernel)(pq::DecodeArgs) =
+        g <= 4 ? (paged ? pq::decode_attention_fast_kernel<1, true> : pq::decode_attention_fast_kernel<1, false>)
+               : (paged ? pq::decode_attention_fast_kernel<2, true> : pq::decode_attention_fast_kernel<2, false>);
+    const int n_sm = pq::configure_for_device(kernel, pq::kSmTotal, configured[(g <= 4 ? 0 : 1) + (paged ? 2 : 0)]);
     if (n_sm == 0) return PQ_ERR_CUDA;
     const int grid = n_sm < pq::kFastMaxGrid ? n_sm : pq::kFastMaxGrid;
-    if (g <= 4) pq::decode_attention_fast_kernel<1><<<grid, pq::kFastThreads, pq::kSmTotal, st>>>(a);
-    else pq::decode_attention_fast_kernel<2><<<grid, pq::kFastThreads, pq::kSmTotal, st>>>(a);
+    kernel<<<grid, pq::kFastThreads, pq::kSmTotal, st>>>(a);
     return pq::launch_status();
   }
   a.epoch = 0u;
   a.debug = 0u;
   pq::rotate_query_kernel<<<(unsigned)pairs * n_q_heads, head_dim, head_dim * sizeof(float), st>>>(a);
-  const pq::Layout L = pq::make_layout(head_dim, capacity);
+  const pq::Layout L = pq::make_layout(head_dim, pg.page_tokens);
   size_t smem = 2 * L.block_bytes + sizeof(float) * ((size_t)g * head_dim + 3 * g * pq::kTokenBlock +
                                                      3 * pq::kMaxGroup + 64);
   const size_t smem_combine = sizeof(float) * pq::combine_smem_floats(g, head_dim, a.ws.n_splits);
@@ -554,7 +563,20 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
                             const int32_t* cache_lens_dev, int32_t batch, int32_t capacity, int32_t max_len,
                             float scale, void* out_dev, void* workspace_dev, int32_t* status_dev, void* stream) {
   return launch_attention(head_dim, n_q_heads, n_kv_heads, S_dev, tables_dev, q_dev, io_dtype, cache_dev, cache_lens_dev,
-                          batch, 1, capacity, max_len, scale, out_dev, workspace_dev, status_dev, stream);
+                          batch, 1, capacity, pq::contiguous_paging(capacity, batch), max_len, scale, out_dev, workspace_dev,
+                          status_dev, stream);
+}
+
+int32_t pq_decode_attention_paged(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                                  const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
+                                  const int32_t* cache_lens_dev, int32_t batch, const pq_paging* paging, int32_t max_len,
+                                  float scale, void* out_dev, void* workspace_dev, int32_t* status_dev, void* stream) {
+  pq::Paging pg;
+  const int32_t st = pq::paging_from(paging, head_dim, &pg);
+  if (st != PQ_OK) return st;
+  return launch_attention(head_dim, n_q_heads, n_kv_heads, S_dev, tables_dev, q_dev, io_dtype, cache_dev, cache_lens_dev,
+                          batch, 1, pg.page_tokens * pg.pages_per_seq, pg, max_len, scale, out_dev, workspace_dev, status_dev,
+                          stream);
 }
 
 int32_t pq_multi_query_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
@@ -563,7 +585,21 @@ int32_t pq_multi_query_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_
                                  int32_t max_len, float scale, void* out_dev, void* workspace_dev, int32_t* status_dev,
                                  void* stream) {
   return launch_attention(head_dim, n_q_heads, n_kv_heads, S_dev, tables_dev, q_dev, io_dtype, cache_dev, cache_lens_dev,
-                          batch, n_q, capacity, max_len, scale, out_dev, workspace_dev, status_dev, stream);
+                          batch, n_q, capacity, pq::contiguous_paging(capacity, batch), max_len, scale, out_dev, workspace_dev,
+                          status_dev, stream);
+}
+
+int32_t pq_multi_query_attention_paged(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                                       const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
+                                       const int32_t* cache_lens_dev, int32_t batch, int32_t n_q, const pq_paging* paging,
+                                       int32_t max_len, float scale, void* out_dev, void* workspace_dev,
+                                       int32_t* status_dev, void* stream) {
+  pq::Paging pg;
+  const int32_t st = pq::paging_from(paging, head_dim, &pg);
+  if (st != PQ_OK) return st;
+  return launch_attention(head_dim, n_q_heads, n_kv_heads, S_dev, tables_dev, q_dev, io_dtype, cache_dev, cache_lens_dev,
+                          batch, n_q, pg.page_tokens * pg.pages_per_seq, pg, max_len, scale, out_dev, workspace_dev, status_dev,
+                          stream);
 }
 
 // ---- decode attention on the library's own scratch ---------------------------------------------
@@ -602,21 +638,36 @@ int32_t pq_decode_attention_static(int32_t head_dim, int32_t n_q_heads, int32_t 
                              cache_lens_dev, batch, capacity, max_len, scale, out_dev, scratch, status_dev, stream);
 }
 
-int32_t pq_unpack_codes(int32_t head_dim, int32_t n_kv_heads, const void* cache_dev, int32_t batch, int32_t capacity,
-                        int32_t n_tokens, uint8_t* codes_dev, void* radii_dev, void* stream) {
+static int32_t unpack_entry(int32_t head_dim, int32_t n_kv_heads, const void* cache_dev, int32_t batch, int32_t capacity,
+                            const pq::Paging& pg, int32_t n_tokens, uint8_t* codes_dev, void* radii_dev, void* stream) {
   if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
   if (!cache_dev || !codes_dev || !radii_dev || batch <= 0 || n_kv_heads <= 0 || n_tokens <= 0 || n_tokens > capacity)
     return PQ_ERR_INVALID_ARG;
   const int64_t n = (int64_t)batch * n_kv_heads * 2 * n_tokens;
   pq::unpack_codes_kernel<<<(unsigned)((n + 127) / 128), 128, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
-      head_dim, n_kv_heads, reinterpret_cast<const uint8_t*>(cache_dev), batch, capacity, n_tokens, codes_dev,
+      head_dim, n_kv_heads, reinterpret_cast<const uint8_t*>(cache_dev), batch, pg, n_tokens, codes_dev,
       reinterpret_cast<__half*>(radii_dev));
   return pq::launch_status();
 }
 
-int32_t pq_dequant_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
-                      const void* cache_dev, int32_t batch, int32_t capacity, int32_t n_tokens, float* x_hat_dev,
-                      void* stream) {
+int32_t pq_unpack_codes(int32_t head_dim, int32_t n_kv_heads, const void* cache_dev, int32_t batch, int32_t capacity,
+                        int32_t n_tokens, uint8_t* codes_dev, void* radii_dev, void* stream) {
+  return unpack_entry(head_dim, n_kv_heads, cache_dev, batch, capacity, pq::contiguous_paging(capacity, batch), n_tokens,
+                      codes_dev, radii_dev, stream);
+}
+
+int32_t pq_unpack_codes_paged(int32_t head_dim, int32_t n_kv_heads, const void* cache_dev, int32_t batch,
+                              const pq_paging* paging, int32_t n_tokens, uint8_t* codes_dev, void* radii_dev, void* stream) {
+  pq::Paging pg;
+  const int32_t st = pq::paging_from(paging, head_dim, &pg);
+  if (st != PQ_OK) return st;
+  return unpack_entry(head_dim, n_kv_heads, cache_dev, batch, pg.page_tokens * pg.pages_per_seq, pg, n_tokens, codes_dev,
+                      radii_dev, stream);
+}
+
+static int32_t dequant_entry(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                             const void* cache_dev, int32_t batch, int32_t capacity, const pq::Paging& pg, int32_t n_tokens,
+                             float* x_hat_dev, void* stream) {
   if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
   if (!S_dev || !tables_dev || !cache_dev || !x_hat_dev || batch <= 0 || n_kv_heads <= 0 || n_tokens <= 0 ||
       n_tokens > capacity)
@@ -625,8 +676,25 @@ int32_t pq_dequant_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, 
   if (n >= (1ll << 31)) return PQ_ERR_UNSUPPORTED;
   pq::dequant_kernel<<<(unsigned)n, head_dim, head_dim * sizeof(float), reinterpret_cast<cudaStream_t>(stream)>>>(
       head_dim, n_kv_heads, S_dev, reinterpret_cast<const pq::Tables*>(tables_dev),
-      reinterpret_cast<const uint8_t*>(cache_dev), capacity, n_tokens, x_hat_dev);
+      reinterpret_cast<const uint8_t*>(cache_dev), pg, n_tokens, x_hat_dev);
   return pq::launch_status();
+}
+
+int32_t pq_dequant_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                      const void* cache_dev, int32_t batch, int32_t capacity, int32_t n_tokens, float* x_hat_dev,
+                      void* stream) {
+  return dequant_entry(head_dim, n_kv_heads, S_dev, tables_dev, cache_dev, batch, capacity,
+                       pq::contiguous_paging(capacity, batch), n_tokens, x_hat_dev, stream);
+}
+
+int32_t pq_dequant_kv_paged(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                            const void* cache_dev, int32_t batch, const pq_paging* paging, int32_t n_tokens,
+                            float* x_hat_dev, void* stream) {
+  pq::Paging pg;
+  const int32_t st = pq::paging_from(paging, head_dim, &pg);
+  if (st != PQ_OK) return st;
+  return dequant_entry(head_dim, n_kv_heads, S_dev, tables_dev, cache_dev, batch, pg.page_tokens * pg.pages_per_seq, pg,
+                       n_tokens, x_hat_dev, stream);
 }
 
 }  // extern "C"

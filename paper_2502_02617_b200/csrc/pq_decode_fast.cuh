@@ -267,7 +267,9 @@ struct Segment {
 };
 
 // kHG = groups of four query heads per kv head (1: up to 4 heads, 2: up to 8).
-template <int kHG>
+// kPaged: the cache lies behind a block table (the contiguous instantiation carries none of that code: the kernel
+// sits at its register limit).
+template <int kHG, bool kPaged>
 __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(DecodeArgs a) {
   extern __shared__ __align__(128) uint8_t smem_raw[];
   uint8_t* smem = smem_raw + ((kSmAlign - (smem_u32(smem_raw) & (kSmAlign - 1))) & (kSmAlign - 1));
@@ -276,7 +278,7 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
   const uint32_t sm_base = smem_u32(smem);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kSmFlags);
   int* is_last = reinterpret_cast<int*>(smem + kSmFlags) + 1;
-  const int64_t head_bytes = make_layout(128, a.capacity).head_bytes;
+  const int64_t head_bytes = make_layout(128, a.pg.page_tokens).head_bytes;
 
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) {
@@ -400,7 +402,8 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     const int b = u / a.n_kv_heads, hk = u - b * a.n_kv_heads;
     const int len = a.visible_len(b);   // b counts (sequence, query) pairs: see DecodeArgs
     const int nblk_total = (len + kTokenBlock - 1) / kTokenBlock;
-    const uint8_t* head_base = a.cache + ((int64_t)a.seq_of(b) * a.n_kv_heads + hk) * head_bytes;
+    const int seq = a.seq_of(b);
+    const uint8_t* head_base = a.cache + ((int64_t)seq * a.n_kv_heads + hk) * head_bytes;  // of a contiguous cache
 
     // per-thread attention state
     // o_acc[hg][S][.]: head c + 4 hg, block g, coordinates 4S, 4S + 2, 4S + 1, 4S + 3 (see the value MMAs)
@@ -428,7 +431,15 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
       const int nblk = min(2, nblk_total - 2 * st);
       const uint32_t bytes = nblk * 2 * kBlockBytes128;
       mbar_expect_tx(sm_base + kSmBar + 8 * s, bytes);
-      bulk_load(sm_base + kSmRing + s * kStageBytes, head_base + (int64_t)st * kStageBytes, bytes, sm_base + kSmBar + 8 * s);
+      // a stage is two token-blocks, K | V | K | V, of one page (page_tokens is a multiple of 128)
+      const uint8_t* src = head_base + (int64_t)st * kStageBytes;
+      if (kPaged) {
+        Layout Lp;  // the two fields the offset needs
+        Lp.block_bytes = kBlockBytes128;
+        Lp.head_bytes = head_bytes;
+        src = a.cache + kv_block_pair_offset(Lp, a.pg, a.n_kv_heads, seq, hk, 2 * st, a.status);
+      }
+      bulk_load(sm_base + kSmRing + s * kStageBytes, src, bytes, sm_base + kSmBar + 8 * s);
       issued = li + 1;
       return true;
     };

@@ -26,6 +26,7 @@ struct EncodeArgs {
   // angle histograms (pq_angle_histograms) instead of codes: uint64 [4 levels][n_bins], added to
   unsigned long long* hist;
   int n_bins;
+  Paging pg;  // where the cache's token-blocks live; `capacity` = pg.pages_per_seq * pg.page_tokens
 };
 
 __device__ inline float load_elem(const void* base, int dtype, int64_t idx) {
@@ -45,6 +46,7 @@ __device__ inline int find_sequence(const int32_t* cu, int batch, int row) {
 
 // Destination of packed row `row`: sequence and cache position, or pos = -1 if the sequence
 // would overflow the capacity (nothing of it is written).
+template <bool kMayBePaged = true>
 __device__ inline void row_destination(const EncodeArgs& a, int row, int* seq, int* pos) {
   int b, first, count;
   if (a.cu_seqlens == nullptr) {
@@ -61,6 +63,12 @@ __device__ inline void row_destination(const EncodeArgs& a, int row, int* seq, i
     *pos = -1;
   } else {
     *pos = start + (row - first);
+    // a page outside the pool: nothing of the row is written
+    if (kMayBePaged && a.pg.table != nullptr && block_offset_paged(0, 0, a.pg.table, a.pg.page_tokens, a.pg.pages_per_seq, a.pg.n_pages, 0, b, 0, 0,
+                                                    *pos) < 0) {
+      set_status(a.status, PQ_ERR_INVALID_ARG);
+      *pos = -1;
+    }
   }
 }
 
@@ -107,7 +115,7 @@ __global__ void __launch_bounds__(kExactThreads) encode_exact_kernel(EncodeArgs 
   const int64_t n_vec = (int64_t)a.total_tokens * 2 * a.n_kv_heads;
   const int64_t v0 = (int64_t)blockIdx.x * vec_per_cta;
   const int tid = threadIdx.x;
-  const Layout L = make_layout(d, a.capacity);
+  const Layout L = make_layout(d, a.pg.page_tokens);
 
   int bad = 0;
   for (int i = tid; i < vec_per_cta * d; i += kExactThreads) {
@@ -169,7 +177,7 @@ __global__ void __launch_bounds__(kExactThreads) encode_exact_kernel(EncodeArgs 
         atomicAdd(a.status + 2, 1);
       }
     }
-    uint8_t* tb_base = a.cache + (valid ? block_offset(L, a.n_kv_heads, seq, head, kv, pos) : 0);
+    uint8_t* tb_base = a.cache + (valid ? block_offset(L, a.pg, a.n_kv_heads, seq, head, kv, pos) : 0);
     store_block(tb_base, L, valid ? pos % kTokenBlock : 0, blk, c, __double2half(radius), valid);
   }
 }
@@ -224,8 +232,8 @@ __device__ __forceinline__ void quantise_and_store(const EncodeArgs& a, const Fa
   int seq, pos;
   row_destination(a, row, &seq, &pos);
   if (pos < 0) return;
-  const Layout L = make_layout(128, a.capacity);
-  uint8_t* tb = a.cache + block_offset(L, a.n_kv_heads, seq, head, kv, pos);
+  const Layout L = make_layout(128, a.pg.page_tokens);
+  uint8_t* tb = a.cache + block_offset(L, a.pg, a.n_kv_heads, seq, head, kv, pos);
   store_half_token(tb, pos % kTokenBlock, half, fb, a.status);
   *xoff_out = (int64_t)row * a.token_stride + (int64_t)head * a.head_stride;
   *tb_out = tb;
@@ -425,9 +433,9 @@ __global__ void __launch_bounds__(128) encode_vector_kernel(EncodeArgs a) {
     rv = 65504.f;
     atomicAdd(a.status + 2, 1);
   }
-  const Layout L = make_layout(128, a.capacity);
+  const Layout L = make_layout(128, a.pg.page_tokens);
   BlockCodes c = {fb.l1, fb.l2, fb.l3, fb.l4};
-  uint8_t* tb = a.cache + (valid ? block_offset(L, a.n_kv_heads, seq, head, kv, pos) : 0);
+  uint8_t* tb = a.cache + (valid ? block_offset(L, a.pg, a.n_kv_heads, seq, head, kv, pos) : 0);
   store_block(tb, L, valid ? pos % kTokenBlock : 0, j & 7, c, __float2half_rn(rv), valid);
 }
 
@@ -481,13 +489,18 @@ __global__ void __launch_bounds__(kHistSimpleThreads) hist_simple_kernel(EncodeA
   hist_flush(hist_s, 4 * a.n_bins, a.hist, j, kHistSimpleThreads);
 }
 
-// lens[b] += rows of sequence b (skipped for sequences that did not fit).
-__global__ void advance_lens_kernel(const int32_t* cu_seqlens, int batch, int capacity, int32_t* lens) {
+// lens[b] += rows of sequence b (skipped for sequences that did not fit, or whose new positions reach a page outside
+// the pool: rows of such a sequence that did land in good pages stay beyond its length).
+__global__ void advance_lens_kernel(const int32_t* cu_seqlens, int batch, int capacity, Paging pg, int32_t* lens) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= batch) return;
   const int count = cu_seqlens ? cu_seqlens[b + 1] - cu_seqlens[b] : 1;
   const int start = lens[b];
-  if (start >= 0 && start + count <= capacity) lens[b] = start + count;
+  if (start < 0 || start + count > capacity || count <= 0) return;
+  if (pg.table != nullptr)
+    for (int p = start / pg.page_tokens; p <= (start + count - 1) / pg.page_tokens; ++p)
+      if ((unsigned)pg.table[(int64_t)b * pg.pages_per_seq + p] >= (unsigned)pg.n_pages) return;
+  lens[b] = start + count;
 }
 
 static int32_t check_common(int head_dim, int n_kv_heads, const void* S, const void* tables, const void* cache,
@@ -506,14 +519,14 @@ static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
     const int32_t tc = try_launch_encode_tc(a, stream);
     if (tc < 0) return tc;
     if (tc == 1) {
-      advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, lens);
+      advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, a.pg, lens);
       return launch_status();
     }
   }
   if (a.head_dim == 128 && a.total_tokens < 32) {
     const int64_t n_vec = (int64_t)a.total_tokens * 2 * a.n_kv_heads;
     encode_vector_kernel<<<(unsigned)n_vec, 128, 0, stream>>>(a);
-    advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, lens);
+    advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, a.pg, lens);
     return launch_status();
   }
   if (a.head_dim == 128 && a.total_tokens >= 32) {
@@ -521,7 +534,7 @@ static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
     if (configure_for_device(encode_ffma_kernel, kFfmaSmem, configured) == 0) return PQ_ERR_CUDA;
     dim3 grid((a.total_tokens + 127) / 128, a.n_kv_heads, 2);
     encode_ffma_kernel<<<grid, kFfmaThreads, kFfmaSmem, stream>>>(a);
-    advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, lens);
+    advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, a.pg, lens);
     return launch_status();
   }
   const int groups = kExactThreads / a.head_dim;
@@ -530,19 +543,17 @@ static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
   const int64_t grid = (n_vec + vec_per_cta - 1) / vec_per_cta;
   const size_t smem = (size_t)2 * vec_per_cta * a.head_dim * sizeof(double);
   encode_exact_kernel<<<(unsigned)grid, kExactThreads, smem, stream>>>(a);
-  advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, lens);
+  advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, a.pg, lens);
   return pq::launch_status();
 }
 
 }  // namespace pq
 
-extern "C" {
-
-int32_t pq_encode_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
-                     const void* K_dev, const void* V_dev, int32_t in_dtype, int64_t token_stride,
-                     int64_t head_stride, const int32_t* cu_seqlens_dev, int32_t batch, int32_t total_tokens,
-                     void* cache_dev, int32_t* cache_lens_dev, int32_t capacity, int32_t* status_dev,
-                     void* stream) {
+static int32_t encode_entry(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                            const void* K_dev, const void* V_dev, int32_t in_dtype, int64_t token_stride,
+                            int64_t head_stride, const int32_t* cu_seqlens_dev, int32_t batch, int32_t total_tokens,
+                            void* cache_dev, int32_t* cache_lens_dev, int32_t capacity, const pq::Paging& pg,
+                            int32_t* status_dev, void* stream) {
   int32_t st = pq::check_common(head_dim, n_kv_heads, S_dev, tables_dev, cache_dev, cache_lens_dev, status_dev);
   if (st != PQ_OK) return st;
   if (!K_dev || !V_dev || !cu_seqlens_dev || batch <= 0 || total_tokens < 0 || capacity <= 0) return PQ_ERR_INVALID_ARG;
@@ -557,13 +568,14 @@ int32_t pq_encode_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, c
   a.S = S_dev; a.tables = reinterpret_cast<const pq::Tables*>(tables_dev);
   a.cache = reinterpret_cast<uint8_t*>(cache_dev); a.cache_lens = cache_lens_dev; a.status = status_dev;
   a.debug = 0u;
+  a.hist = nullptr; a.n_bins = 0; a.pg = pg;
   return pq::launch_encode(a, cache_lens_dev, reinterpret_cast<cudaStream_t>(stream));
 }
 
-int32_t pq_append_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
-                     const void* k_new_dev, const void* v_new_dev, int32_t in_dtype, int32_t batch,
-                     void* cache_dev, int32_t* cache_lens_dev, int32_t capacity, int32_t* status_dev,
-                     void* stream) {
+static int32_t append_entry(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                            const void* k_new_dev, const void* v_new_dev, int32_t in_dtype, int32_t batch,
+                            void* cache_dev, int32_t* cache_lens_dev, int32_t capacity, const pq::Paging& pg,
+                            int32_t* status_dev, void* stream) {
   int32_t st = pq::check_common(head_dim, n_kv_heads, S_dev, tables_dev, cache_dev, cache_lens_dev, status_dev);
   if (st != PQ_OK) return st;
   if (!k_new_dev || !v_new_dev || batch <= 0 || capacity <= 0) return PQ_ERR_INVALID_ARG;
@@ -576,7 +588,52 @@ int32_t pq_append_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, c
   a.S = S_dev; a.tables = reinterpret_cast<const pq::Tables*>(tables_dev);
   a.cache = reinterpret_cast<uint8_t*>(cache_dev); a.cache_lens = cache_lens_dev; a.status = status_dev;
   a.debug = 0u;
+  a.hist = nullptr; a.n_bins = 0; a.pg = pg;
   return pq::launch_encode(a, cache_lens_dev, reinterpret_cast<cudaStream_t>(stream));
+}
+
+extern "C" {
+
+int32_t pq_encode_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                     const void* K_dev, const void* V_dev, int32_t in_dtype, int64_t token_stride,
+                     int64_t head_stride, const int32_t* cu_seqlens_dev, int32_t batch, int32_t total_tokens,
+                     void* cache_dev, int32_t* cache_lens_dev, int32_t capacity, int32_t* status_dev,
+                     void* stream) {
+  return encode_entry(head_dim, n_kv_heads, S_dev, tables_dev, K_dev, V_dev, in_dtype, token_stride, head_stride,
+                      cu_seqlens_dev, batch, total_tokens, cache_dev, cache_lens_dev, capacity,
+                      pq::contiguous_paging(capacity, batch), status_dev, stream);
+}
+
+int32_t pq_encode_kv_paged(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                           const void* K_dev, const void* V_dev, int32_t in_dtype, int64_t token_stride,
+                           int64_t head_stride, const int32_t* cu_seqlens_dev, int32_t batch, int32_t total_tokens,
+                           void* cache_dev, int32_t* cache_lens_dev, const pq_paging* paging, int32_t* status_dev,
+                           void* stream) {
+  pq::Paging pg;
+  const int32_t st = pq::paging_from(paging, head_dim, &pg);
+  if (st != PQ_OK) return st;
+  return encode_entry(head_dim, n_kv_heads, S_dev, tables_dev, K_dev, V_dev, in_dtype, token_stride, head_stride,
+                      cu_seqlens_dev, batch, total_tokens, cache_dev, cache_lens_dev, pg.page_tokens * pg.pages_per_seq, pg,
+                      status_dev, stream);
+}
+
+int32_t pq_append_kv(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                     const void* k_new_dev, const void* v_new_dev, int32_t in_dtype, int32_t batch,
+                     void* cache_dev, int32_t* cache_lens_dev, int32_t capacity, int32_t* status_dev,
+                     void* stream) {
+  return append_entry(head_dim, n_kv_heads, S_dev, tables_dev, k_new_dev, v_new_dev, in_dtype, batch, cache_dev,
+                      cache_lens_dev, capacity, pq::contiguous_paging(capacity, batch), status_dev, stream);
+}
+
+int32_t pq_append_kv_paged(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* tables_dev,
+                           const void* k_new_dev, const void* v_new_dev, int32_t in_dtype, int32_t batch,
+                           void* cache_dev, int32_t* cache_lens_dev, const pq_paging* paging, int32_t* status_dev,
+                           void* stream) {
+  pq::Paging pg;
+  const int32_t st = pq::paging_from(paging, head_dim, &pg);
+  if (st != PQ_OK) return st;
+  return append_entry(head_dim, n_kv_heads, S_dev, tables_dev, k_new_dev, v_new_dev, in_dtype, batch, cache_dev,
+                      cache_lens_dev, pg.page_tokens * pg.pages_per_seq, pg, status_dev, stream);
 }
 
 int32_t pq_angle_histograms(int32_t head_dim, int32_t n_kv_heads, const float* S_dev, const void* K_dev,
@@ -598,6 +655,7 @@ int32_t pq_angle_histograms(int32_t head_dim, int32_t n_kv_heads, const float* S
   a.S = S_dev; a.tables = nullptr; a.cache = nullptr; a.cache_lens = nullptr; a.status = status_dev;
   a.debug = 0u;
   a.hist = reinterpret_cast<unsigned long long*>(hist_dev); a.n_bins = n_bins;
+  a.pg = pq::contiguous_paging(0, 0);
   cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
   const int32_t tc = pq::try_launch_hist_tc(a, s);
   if (tc < 0) return tc;

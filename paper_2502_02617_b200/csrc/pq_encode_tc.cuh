@@ -161,7 +161,8 @@ __device__ inline int count_nonfinite_bf16(const void* base, int64_t xoff) {
 // kHist: the same pipeline up to the rotated coordinates in registers, which are then counted into the angle
 // histograms (pq_hist.cuh) instead of being quantised; the shared memory of the re-decision queues holds the CTA's
 // histogram (4 levels x n_bins 32-bit counters: a CTA would have to take 2^32 / 8192 tiles to overflow one).
-template <bool kHist>
+// kPaged: the cache lies behind a block table (the other instantiations carry none of that code).
+template <bool kHist, bool kPaged>
 __global__ void __launch_bounds__(kTcThreads, 1)
 encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_tiles) {
   extern __shared__ uint8_t smem_raw[];
@@ -317,7 +318,7 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   const bool analytic = kHist || fq->analytic != 0u;  // uniform over the grid
   const float hist_scale1 = (float)a.n_bins * 0.159154943091895336f, hist_scale_up = (float)a.n_bins * 0.636619772367581343f;
   int hist_bad = 0;
-  const Layout L = make_layout(128, a.capacity);
+  const Layout L = make_layout(128, a.pg.page_tokens);
   const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + slot * 128;
   const int slot_bar = 1 + slot;
   int rd_seq = 0, rd_first = 0, rd_count = 0, rd_start = -1;   // destination of the last row looked up
@@ -384,14 +385,15 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
         seq = rd_seq;
         pos = rd_start < 0 ? -1 : rd_start + (row - rd_first);
       } else {
-        row_destination(a, row, &seq, &pos);
+        row_destination<kPaged>(a, row, &seq, &pos);
         rd_seq = seq;
         rd_first = a.cu_seqlens ? a.cu_seqlens[seq] : row;
         rd_count = a.cu_seqlens ? a.cu_seqlens[seq + 1] - rd_first : 1;
         rd_start = pos < 0 ? -1 : pos - (row - rd_first);
       }
       if (pos >= 0) {
-        tb = a.cache + block_offset(L, a.n_kv_heads, seq, head, kv, pos);
+        tb = a.cache + (kPaged ? block_offset(L, a.pg, a.n_kv_heads, seq, head, kv, pos)
+                               : block_offset(L, contiguous_paging(0, 0), a.n_kv_heads, seq, head, kv, pos));
         tok = pos % kTokenBlock;
       }
     }
@@ -525,7 +527,7 @@ static bool make_x_map(EncodeTiledFn fn, CUtensorMap* map, const void* base, int
 
 // Launch the tensor-core encoder (or its histogram form) if the inputs allow it.  Returns 1 if launched, 0 if not
 // applicable, or a negative status.
-template <bool kHist>
+template <bool kHist, bool kPaged>
 static int32_t try_launch_tc(const EncodeArgs& a, cudaStream_t stream) {
   if (a.head_dim != 128 || a.in_dtype != PQ_DTYPE_BF16 || a.total_tokens < 128) return 0;
   if ((a.token_stride & 7) || (a.head_stride & 7) || a.head_stride < 128 || a.token_stride < 128) return 0;
@@ -537,17 +539,19 @@ static int32_t try_launch_tc(const EncodeArgs& a, cudaStream_t stream) {
   if (!make_x_map(fn, &maps.k, a.K, a.n_kv_heads, a.total_tokens, a.token_stride, a.head_stride)) return 0;
   if (!make_x_map(fn, &maps.v, a.V, a.n_kv_heads, a.total_tokens, a.token_stride, a.head_stride)) return 0;
   static DeviceMemo configured;  // one per instantiation
-  const int n_sm = configure_for_device(encode_tc_kernel<kHist>, kTcSmTotal, configured);
+  const int n_sm = configure_for_device(encode_tc_kernel<kHist, kPaged>, kTcSmTotal, configured);
   if (n_sm == 0) return PQ_ERR_CUDA;
   const int n_row_tiles = (a.total_tokens + 127) / 128;
   const int n_tiles = n_row_tiles * 2 * a.n_kv_heads;
   const int grid = n_tiles < n_sm ? n_tiles : n_sm;
   EncodeArgs args = a;
   if (take_debug_wait_failure(1)) args.debug |= 1u;
-  encode_tc_kernel<kHist><<<grid, kTcThreads, kTcSmTotal, stream>>>(args, maps, n_row_tiles);
+  encode_tc_kernel<kHist, kPaged><<<grid, kTcThreads, kTcSmTotal, stream>>>(args, maps, n_row_tiles);
   return 1;
 }
-static int32_t try_launch_encode_tc(const EncodeArgs& a, cudaStream_t stream) { return try_launch_tc<false>(a, stream); }
-static int32_t try_launch_hist_tc(const EncodeArgs& a, cudaStream_t stream) { return try_launch_tc<true>(a, stream); }
+static int32_t try_launch_encode_tc(const EncodeArgs& a, cudaStream_t stream) {
+  return a.pg.table != nullptr ? try_launch_tc<false, true>(a, stream) : try_launch_tc<false, false>(a, stream);
+}
+static int32_t try_launch_hist_tc(const EncodeArgs& a, cudaStream_t stream) { return try_launch_tc<true, false>(a, stream); }
 
 }  // namespace pq

@@ -160,6 +160,18 @@ bool build_l1_cells(const double* bnd, uint2 (*cells)[pq::kL1Cells]) {
 namespace pq {
 static thread_local cudaError_t g_last_cuda_error = cudaSuccess;
 void note_cuda_error(cudaError_t e) { g_last_cuda_error = e; }
+// The kernels' Paging from a caller's pq_paging (validated).
+int32_t paging_from(const pq_paging* p, int head_dim, Paging* out) {
+  if (p == nullptr || p->page_table_dev == nullptr) return PQ_ERR_INVALID_ARG;
+  if (p->page_tokens <= 0 || p->pages_per_seq <= 0 || p->n_pages <= 0) return PQ_ERR_INVALID_ARG;
+  if (p->page_tokens % (head_dim == 128 ? 128 : kTokenBlock)) return PQ_ERR_INVALID_ARG;
+  if ((int64_t)p->page_tokens * p->pages_per_seq >= (1ll << 31)) return PQ_ERR_UNSUPPORTED;
+  if ((uintptr_t)p->page_table_dev & 3) return PQ_ERR_ALIGNMENT;
+  out->table = p->page_table_dev; out->page_tokens = p->page_tokens; out->pages_per_seq = p->pages_per_seq;
+  out->n_pages = p->n_pages;
+  return PQ_OK;
+}
+
 static std::atomic<int> g_debug_wait_failure{0};
 bool take_debug_wait_failure(int which) {
   int armed = which;
@@ -416,6 +428,14 @@ int64_t pq_cache_bytes(int32_t head_dim, int32_t batch, int32_t n_kv_heads, int3
   if (batch <= 0 || n_kv_heads <= 0 || capacity <= 0) return PQ_ERR_INVALID_ARG;
   const pq::Layout L = pq::make_layout(head_dim, capacity);
   return (int64_t)batch * n_kv_heads * L.head_bytes;
+}
+
+int64_t pq_paged_cache_bytes(int32_t head_dim, int32_t n_kv_heads, int32_t page_tokens, int32_t n_pages) {
+  if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
+  if (n_kv_heads <= 0 || page_tokens <= 0 || n_pages <= 0) return PQ_ERR_INVALID_ARG;
+  if (page_tokens % (head_dim == 128 ? 128 : pq::kTokenBlock)) return PQ_ERR_INVALID_ARG;
+  const pq::Layout L = pq::make_layout(head_dim, page_tokens);
+  return (int64_t)n_pages * n_kv_heads * L.head_bytes;
 }
 
 }  // extern "C"

@@ -107,10 +107,9 @@ __global__ void __launch_bounds__(kPfThreads) prefill_attention_kernel(DecodeArg
   }
   const int vis_cta = max(0, len - (n_q - 1 - (q0 + (n_rows - 1) / g)));   // the CTA's last query sees the most
   const int n_blocks = (vis_cta + kTokenBlock - 1) / kTokenBlock;
-  const Layout L = make_layout(128, a.capacity);
-  const uint8_t* head_base = a.cache + ((int64_t)b * a.n_kv_heads + hk) * L.head_bytes;
+  const Layout L = make_layout(128, a.pg.page_tokens);
   auto fetch = [&](int jb) {  // packed K block and V block of token-block jb -> raw buffer jb & 1
-    const uint8_t* src = head_base + (int64_t)jb * kPfRawBytes;
+    const uint8_t* src = a.cache + kv_block_pair_offset(L, a.pg, a.n_kv_heads, b, hk, jb, a.status);
     const uint32_t dst = sb + kPfRaw + (jb & 1) * kPfRawBytes;
     for (int i = tid; i < kPfRawBytes / 16; i += kPfThreads) pf_cp16(dst + 16 * i, src + 16 * i);
     asm volatile("cp.async.commit_group;" ::: "memory");

@@ -153,6 +153,18 @@ def test_device_entry_points_validate_before_launching():
     assert L.pq_angle_histograms(48, 8, 16, 16, 16, 1, 1024, 128, 4, 1024, 16, 16, nul) == pq.ERR_UNSUPPORTED
     assert L.pq_angle_histograms(128, 8, 16, 16, 16, 1, 1024, 128, 4, 1024, 20, 16, nul) == pq.ERR_ALIGNMENT
     assert L.pq_unpack_codes(128, 8, 16, 1, 64, 65, 16, 16, nul) == pq.ERR_INVALID_ARG
+    good = api.Paging(16, 256, 4, 10)
+    for bad in (api.Paging(0, 256, 4, 10), api.Paging(16, 0, 4, 10), api.Paging(16, 192, 4, 10), api.Paging(16, 256, 4, 0)):
+        assert L.pq_decode_attention_paged(128, 32, 8, 16, 16, 16, 1, 16, 16, 1, ctypes.addressof(bad), 64, 0.1, 16, 16, 16,
+                                           nul) == pq.ERR_INVALID_ARG
+        assert L.pq_append_kv_paged(128, 8, 16, 16, 16, 16, 1, 4, 16, 16, ctypes.addressof(bad), 16, nul) == pq.ERR_INVALID_ARG
+    assert L.pq_decode_attention_paged(128, 32, 8, 16, 16, 16, 1, 16, 16, 1, None, 64, 0.1, 16, 16, 16, nul) == pq.ERR_INVALID_ARG
+    assert L.pq_encode_kv_paged(128, 8, 16, 16, 16, 16, 1, 1024, 128, nul, 1, 4, 16, 16, ctypes.addressof(good), 16,
+                                nul) == pq.ERR_INVALID_ARG  # no cu_seqlens
+    assert pq.pq_paged_cache_bytes(128, 8, 256, 10) == 10 * 8 * 256 * 2 * 62
+    assert pq.pq_paged_cache_bytes(64, 2, 64, 3) == 3 * 2 * 64 * 2 * 31
+    with pytest.raises(pq.PolarQuantError):
+        pq.pq_paged_cache_bytes(128, 8, 192, 10)
     assert L.pq_dequant_kv(128, 8, 16, 16, 16, 1, 64, 0, 16, nul) == pq.ERR_INVALID_ARG
 
 
