@@ -572,6 +572,51 @@ def measure_paged(args, pq, synthetic, dev, rank):
             "gbs": comp / (t * 1e-3) / 1e9, "rank": rank}
 
 
+def measure_tail_window(args, pq, synthetic, dev, rank):
+    """Config 3 with the 1024 most recent tokens of every sequence kept in bf16 (Section 5.3's protocol for generated
+    tokens): partial attention over the packed cache with its log-sum-exp, exact attention over the window, merge --
+    three launches, float32 partials."""
+    T = 1024
+    cache = pq.PolarQuantCache(BATCH, HQ, HKV, D, CTX, seed=0, device=dev)
+    for b in range(BATCH):
+        K, V = synthetic.kv_like(1000 * rank + 10 + b % 2, CTX, HKV, D, torch.bfloat16, dev)
+        cu = torch.zeros(BATCH + 1, dtype=torch.int32, device=dev)
+        cu[b + 1:] = CTX
+        cache.encode(K, V, cu)
+    kt, vt = synthetic.kv_like(1000 * rank + 77, BATCH * T, HKV, D, torch.bfloat16, dev, n_outliers=0)
+    kt, vt = kt.view(BATCH, T, HKV, D).contiguous(), vt.view(BATCH, T, HKV, D).contiguous()
+    tail_lens = torch.full((BATCH,), T, dtype=torch.int32, device=dev)
+    q = synthetic.queries(3, BATCH, HQ, D, torch.bfloat16, dev)
+    q32 = q.float()
+    parts_out = torch.empty((2,) + q32.shape, dtype=torch.float32, device=dev)
+    parts_lse = torch.empty((2, BATCH, HQ), dtype=torch.float32, device=dev)
+    out = torch.empty_like(q)
+    stream = torch.cuda.current_stream()
+    scale = D ** -0.5
+
+    def step(evs=None):
+        marks = []
+        for fn in (lambda: pq.pq_decode_attention_lse(cache.S, cache.tables, q32, cache.cache, cache.lens, HKV, CTX, CTX, scale,
+                                                      parts_out[0], parts_lse[0], cache.workspace, cache.status),
+                   lambda: pq.pq_tail_attention(q32, kt, vt, tail_lens, scale, parts_out[1], parts_lse[1], cache.status),
+                   lambda: pq.pq_merge_attention(parts_out, parts_lse, out, cache.status)):
+            a, b = _event(), _event()
+            a.record(stream)
+            fn()
+            b.record(stream)
+            marks.append((a, b))
+        return marks
+
+    for _ in range(3):
+        step()
+    runs = [step() for _ in range(20)]
+    torch.cuda.synchronize()
+    cache.check_status()
+    med = [float(np.median([r[i][0].elapsed_time(r[i][1]) for r in runs])) * 1e3 for i in range(3)]
+    return {"batch": BATCH, "ctx": CTX, "window_tokens": T, "decode_with_lse_us": med[0], "window_attention_us": med[1],
+            "merge_us": med[2], "window_bytes": 2 * BATCH * T * HKV * D * 2, "rank": rank}
+
+
 def measure_config5(args, pq, synthetic, dev, rank):
     """Config 5: batch 16, ragged contexts in [4096, 65536], prefill in 4096-token chunks, then 128 steps of
     (append one token per sequence, decode attention)."""
@@ -710,6 +755,8 @@ def reduce_and_format(local, steps, warmup, rank, world, dist=None, device="cpu"
                                                     mma_tflops=mq["mma_tflops"] * mq["ms"] / t)
     if local.get("paged"):
         line["configs"]["paged_decode"] = dict(local["paged"], hbm_frac_measured=local["paged"]["gbs"] / peak)
+    if local.get("tail"):
+        line["configs"]["tail_window"] = local["tail"]
     if local.get("online"):
         line["configs"]["online_codebook"] = local["online"]  # this rank's own figures (not reduced over ranks)
     if cpu_baseline is not None:
@@ -743,6 +790,8 @@ def run_cuda(args):
         local["online"] = measure_online_codebook(args, pq, synthetic, dev, rank)
         torch.cuda.empty_cache()
         local["paged"] = measure_paged(args, pq, synthetic, dev, rank)
+        torch.cuda.empty_cache()
+        local["tail"] = measure_tail_window(args, pq, synthetic, dev, rank)
         torch.cuda.empty_cache()
     cpu = _oracle_sample_throughput(12.0) if rank == 0 and world == 1 and not args.no_cpu_baseline else None
     line = reduce_and_format(local, args.steps, args.warmup, rank, world, dist, dev, cpu)

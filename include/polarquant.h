@@ -322,6 +322,41 @@ int32_t pq_dequant_kv_paged(int32_t head_dim, int32_t n_kv_heads, const float* S
                             const void* cache_dev, int32_t batch, const pq_paging* paging, int32_t n_tokens,
                             float* x_hat_dev, void* stream);
 
+/*
+ * Partial attentions.  Softmax attention over a union of token sets is the weighted mean of the attentions over
+ * the sets, with weights exp(lse_p - lse), lse_p = log sum_t exp(scale <q, k_t>) over set p (natural logarithm).
+ * Two uses: the cached tokens of a sequence sharded over several GPUs (each GPU attends over its shard, the
+ * (out, lse) pairs are gathered and merged on every GPU), and a cache whose most recent tokens are kept in 16 bits
+ * (Section 5.3 keeps the generated tokens unquantised): compressed part and window are attended separately and merged.
+ *
+ * pq_decode_attention_lse: pq_decode_attention (paging == NULL: contiguous cache of `capacity` tokens; else the
+ * paged cache and `capacity` is ignored) that also writes lse_dev, float32 [batch][n_q_heads].  A sequence of
+ * length 0 yields zeros and lse = -inf and is NOT reported as PQ_ERR_EMPTY (an empty shard is legitimate).
+ *
+ * pq_merge_attention: parts_out_dev [n_parts][batch][n_q_heads][head_dim] of parts_dtype, parts_lse_dev float32
+ * [n_parts][batch][n_q_heads] -> out_dev [batch][n_q_heads][head_dim] of out_dtype and, if not NULL, lse_out_dev.
+ * Parts with lse = -inf are skipped; a row whose parts are all empty yields zeros, -inf and PQ_ERR_EMPTY.  Parts are
+ * added in index order (bit-identical from run to run).  Use float32 parts: a part rounded to bf16 carries its
+ * rounding into the merged output.
+ *
+ * pq_tail_attention: exact attention (Eq. 2) of one query per sequence over an uncompressed window,
+ * k_tail_dev / v_tail_dev [batch][tail_capacity][n_kv_heads][head_dim] of kv_dtype, of which sequence b uses the
+ * first tail_lens_dev[b] rows; out and (if lse_dev is not NULL) lse as above.  With lse_dev == NULL an empty
+ * window records PQ_ERR_EMPTY.  Float32 arithmetic; not a tuned kernel (windows are short).
+ */
+int32_t pq_decode_attention_lse(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                                const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
+                                const int32_t* cache_lens_dev, int32_t batch, int32_t capacity, const pq_paging* paging,
+                                int32_t max_len, float scale, void* out_dev, float* lse_dev, void* workspace_dev,
+                                int32_t* status_dev, void* stream);
+int32_t pq_merge_attention(int32_t head_dim, int32_t n_q_heads, int32_t batch, int32_t n_parts, const void* parts_out_dev,
+                           int32_t parts_dtype, const float* parts_lse_dev, void* out_dev, int32_t out_dtype,
+                           float* lse_out_dev, int32_t* status_dev, void* stream);
+int32_t pq_tail_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const void* q_dev, int32_t io_dtype,
+                          const void* k_tail_dev, const void* v_tail_dev, int32_t kv_dtype, const int32_t* tail_lens_dev,
+                          int32_t batch, int32_t tail_capacity, float scale, void* out_dev, float* lse_dev,
+                          int32_t* status_dev, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

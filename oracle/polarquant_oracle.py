@@ -23,7 +23,8 @@ block radius == block norm, norm preservation under S, Lemma 2 densities against
 incomplete-beta CDF, Lloyd-Max fixed-point equations against independent quadrature,
 the worked d=4 example under tests/golden/, brute force on d=4 and d=16, closed-form
 expected distortion, the len=1 / identical-keys attention special cases, multi-query attention against a
-masked softmax, and the online codebook (histogram counts, k-means fixed point, two-cluster toy, convergence to the
+masked softmax, merging of partial attentions (a split of the tokens gives back the whole; closed forms of the
+log-sum-exp), and the online codebook (histogram counts, k-means fixed point, two-cluster toy, convergence to the
 analytic codebook on samples of the analytic density).
 Parity unpinned: nothing in this file; quality on real model caches is out of scope.
 """
@@ -372,6 +373,54 @@ def multi_query_attention(q, k_codes, k_radii, v_codes, v_radii, lens, cb: Codeb
                 for h in range(hk * group, (hk + 1) * group):
                     out[b, j, h] = softmax_attention(q[b, j, h], K_hat[:visible], V_hat[:visible], scale)
     return out
+
+
+def log_sum_exp_scores(q: np.ndarray, K: np.ndarray, scale: float) -> float:
+    """log of the softmax denominator of Eq. 2 for one query over the rows of K (-inf for no rows)."""
+    if K.shape[0] == 0:
+        return -np.inf
+    s = (K @ q) * scale
+    m = s.max()
+    return float(m + np.log(np.sum(np.exp(s - m))))
+
+
+def merge_attention(outs, lses):
+    """Attention over a union of disjoint token sets from the attentions over the sets: with
+    lse_p = log sum_{t in set p} exp(s_t), softmax over the union gives sum_p exp(lse_p - lse) out_p,
+    lse = log sum_p exp(lse_p) (Eq. 2 with its sum split by set).  outs [P, ..., d], lses [P, ...].
+    Returns (out, lse); rows whose sets are all empty give zeros and -inf."""
+    outs = np.asarray(outs, dtype=np.float64)
+    lses = np.asarray(lses, dtype=np.float64)
+    top = lses.max(axis=0)
+    safe = np.where(np.isfinite(top), top, 0.0)
+    w = np.where(np.isfinite(lses), np.exp(lses - safe), 0.0)
+    tot = w.sum(axis=0)
+    out = np.sum(w[..., None] * np.where(np.isfinite(lses)[..., None], outs, 0.0), axis=0) / np.where(tot > 0, tot, 1.0)[..., None]
+    with np.errstate(divide="ignore"):
+        lse = np.where(tot > 0, safe + np.log(np.where(tot > 0, tot, 1.0)), -np.inf)
+    return out, lse
+
+
+def attention_with_tail(q, k_codes, k_radii, v_codes, v_radii, lens, cb: Codebooks, S, scale, k_tail, v_tail, tail_lens):
+    """Eq. 2 over a cache whose first lens[b] tokens are PolarQuant-compressed and whose last tail_lens[b] tokens are
+    kept as they are (the protocol of Section 5.3 for generated tokens): softmax over the dequantised keys followed
+    by the exact tail keys, values likewise.  k_tail, v_tail [B, T, Hkv, d].  Returns (out [B, Hq, d], lse [B, Hq])."""
+    q = np.asarray(q, dtype=np.float64)
+    B, Hq, d = q.shape
+    Hkv = k_codes.shape[1]
+    group = Hq // Hkv
+    out = np.zeros((B, Hq, d))
+    lse = np.full((B, Hq), -np.inf)
+    for b in range(B):
+        n, t = int(lens[b]), int(tail_lens[b])
+        for hk in range(Hkv):
+            K = np.concatenate([dequant(k_codes[b, hk, :n], k_radii[b, hk, :n], cb, S), np.asarray(k_tail[b, :t, hk], dtype=np.float64)])
+            V = np.concatenate([dequant(v_codes[b, hk, :n], v_radii[b, hk, :n], cb, S), np.asarray(v_tail[b, :t, hk], dtype=np.float64)])
+            for h in range(hk * group, (hk + 1) * group):
+                if n + t > 0:
+                    out[b, h] = softmax_attention(q[b, h], K, V, scale)
+                    lse[b, h] = log_sum_exp_scores(q[b, h], K, scale)
+    return out, lse
 
 
 def exact_attention(q, K, V, lens, scale):

@@ -57,6 +57,13 @@ _SIGNATURES = {
     "pq_unpack_codes": (c_int32, [c_int32, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p]),
     "pq_dequant_kv": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32, c_void_p,
                                 c_void_p]),
+    "pq_decode_attention_lse": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p,
+                                          c_void_p, c_int32, c_int32, c_void_p, c_int32, c_float, c_void_p, c_void_p,
+                                          c_void_p, c_void_p, c_void_p]),
+    "pq_merge_attention": (c_int32, [c_int32, c_int32, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_void_p, c_int32,
+                                     c_void_p, c_void_p, c_void_p]),
+    "pq_tail_attention": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_void_p,
+                                    c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p, c_void_p]),
     "pq_paged_cache_bytes": (c_int64, [c_int32, c_int32, c_int32, c_int32]),
     "pq_encode_kv_paged": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int64, c_int64,
                                      c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -283,6 +290,51 @@ def pq_dequant_kv(d, n_kv_heads, S, tables, cache, batch, capacity, n_tokens, st
     return out
 
 
+def pq_decode_attention_lse(S, tables, q, cache, cache_lens, n_kv_heads, capacity, max_len, scale, out, lse, workspace,
+                            status, paging=None, stream=None):
+    """pq_decode_attention that also writes lse float32 [B, Hq] (log of the softmax denominator); `paging`: a Paging
+    for a paged cache, else the contiguous cache of `capacity` tokens."""
+    batch, n_q_heads, d = q.shape
+    assert q.is_contiguous() and out.is_contiguous() and out.shape == q.shape and out.dtype == q.dtype
+    assert lse.dtype == torch.float32 and lse.is_contiguous() and lse.shape == (batch, n_q_heads)
+    _check(lib().pq_decode_attention_lse(d, n_q_heads, n_kv_heads, _ptr(S), _ptr(tables), _ptr(q), _dtype_code(q),
+                                         _ptr(cache), _ptr(cache_lens), batch, capacity,
+                                         None if paging is None else ctypes.addressof(paging), max_len, float(scale),
+                                         _ptr(out), _ptr(lse), _ptr(workspace), _ptr(status), _stream(stream)),
+           "pq_decode_attention_lse")
+
+
+def pq_merge_attention(parts_out, parts_lse, out, status, lse_out=None, stream=None):
+    """Merge partial attentions: parts_out [P, B, Hq, d] (float32 or bf16), parts_lse float32 [P, B, Hq] -> out [B, Hq, d]."""
+    n_parts, batch, n_q_heads, d = parts_out.shape
+    assert parts_out.is_contiguous() and parts_lse.is_contiguous() and out.is_contiguous()
+    assert parts_lse.shape == (n_parts, batch, n_q_heads) and parts_lse.dtype == torch.float32 and out.shape == parts_out.shape[1:]
+    _check(lib().pq_merge_attention(d, n_q_heads, batch, n_parts, _ptr(parts_out), _dtype_code(parts_out), _ptr(parts_lse),
+                                    _ptr(out), _dtype_code(out), _ptr(lse_out), _ptr(status), _stream(stream)),
+           "pq_merge_attention")
+    return out
+
+
+def pq_tail_attention(q, k_tail, v_tail, tail_lens, scale, out, lse, status, stream=None):
+    """Exact attention of q [B, Hq, d] over an uncompressed window k_tail, v_tail [B, T, Hkv, d] (first tail_lens[b] rows)."""
+    batch, n_q_heads, d = q.shape
+    assert k_tail.is_contiguous() and v_tail.is_contiguous() and k_tail.shape == v_tail.shape and k_tail.dtype == v_tail.dtype
+    assert k_tail.shape[0] == batch and k_tail.shape[3] == d and q.is_contiguous() and out.is_contiguous() and out.dtype == q.dtype
+    _check(lib().pq_tail_attention(d, n_q_heads, k_tail.shape[2], _ptr(q), _dtype_code(q), _ptr(k_tail), _ptr(v_tail),
+                                   _dtype_code(k_tail), _ptr(tail_lens), batch, k_tail.shape[1], float(scale), _ptr(out),
+                                   _ptr(lse), _ptr(status), _stream(stream)), "pq_tail_attention")
+
+
+def sharded_decode_attention(cache, q, dist, group=None, scale=None, stream=None):
+    """Decode attention over a cache whose tokens are sharded over the ranks of `group` (each rank's `cache` holds its
+    own tokens): local partial attention with its log-sum-exp in float32, one all-gather of [B, Hq, d + 1] floats per
+    rank, merge on every rank.  Returns out in q's dtype."""
+    from .sharding import gather_partials
+    out32, lse = cache.attend_lse(q.float(), scale=scale, stream=stream)
+    parts_out, parts_lse = gather_partials(out32, lse, dist, group)
+    return pq_merge_attention(parts_out, parts_lse, torch.empty_like(q), cache.status, stream=stream)
+
+
 def pq_paged_cache_bytes(d: int, n_kv_heads: int, page_tokens: int, n_pages: int) -> int:
     n = int(lib().pq_paged_cache_bytes(d, n_kv_heads, page_tokens, n_pages))
     if n < 0:
@@ -332,6 +384,31 @@ class PolarQuantCache:
                             self.capacity if max_len is None else max_len, scale, out, self.workspace, self.status,
                             stream)
         return out
+
+    def _paging(self):
+        return None
+
+    def attend_lse(self, q, scale=None, max_len=None, stream=None):
+        """Partial attention for merging: (out like q, lse float32 [B, Hq]); an empty sequence gives zeros and -inf."""
+        out = torch.empty_like(q)
+        lse = torch.empty(q.shape[:2], dtype=torch.float32, device=q.device)
+        pq_decode_attention_lse(self.S, self.tables, q, self.cache, self.lens, self.n_kv_heads, self.capacity,
+                                self.capacity if max_len is None else max_len, self.d ** -0.5 if scale is None else scale,
+                                out, lse, self.workspace, self.status, paging=self._paging(), stream=stream)
+        return out, lse
+
+    def attend_with_tail(self, q, k_tail, v_tail, tail_lens, scale=None, stream=None):
+        """Attention over the compressed cache followed by an uncompressed window (k_tail, v_tail [B, T, Hkv, d], the
+        first tail_lens[b] rows): both partial attentions in float32, merged into q's dtype."""
+        scale = self.d ** -0.5 if scale is None else scale
+        q32 = q.float()
+        parts_out = torch.empty((2,) + q32.shape, dtype=torch.float32, device=q.device)
+        parts_lse = torch.empty((2,) + q32.shape[:2], dtype=torch.float32, device=q.device)
+        pq_decode_attention_lse(self.S, self.tables, q32, self.cache, self.lens, self.n_kv_heads, self.capacity, self.capacity,
+                                scale, parts_out[0], parts_lse[0], self.workspace, self.status, paging=self._paging(),
+                                stream=stream)
+        pq_tail_attention(q32, k_tail, v_tail, tail_lens, scale, parts_out[1], parts_lse[1], self.status, stream)
+        return pq_merge_attention(parts_out, parts_lse, torch.empty_like(q), self.status, stream=stream)
 
     def attend_multi(self, q, out=None, scale=None, max_len=None, stream=None):
         """q [B, n_q, Hq, d]: the last n_q positions of every sequence (already in the cache), causal."""

@@ -135,6 +135,8 @@ struct DecodeArgs {
   const uint8_t* cache;
   const int32_t* lens;
   void* out;
+  float* lse;  // optional [batch][n_q_heads]: natural log of the softmax denominator (for merging partial attentions);
+               // with it, a sequence of length 0 is not an error (zeros and -inf)
   int32_t* status;
   Workspace ws;
   Paging pg;  // where the cache's token-blocks live
@@ -201,6 +203,8 @@ __device__ void combine_and_store(const DecodeArgs& a, int b, int hk, int g, int
       Lsum += l_sm[tid * ns + s] * w;
     }
     linv_sm[tid] = Lsum > 0.f ? 1.f / Lsum : 0.f;
+    // scores are kept in the log2 domain: sum_t exp(s_t) = 2^M * Lsum
+    if (a.lse != nullptr) a.lse[h0 + tid] = Lsum > 0.f ? (M + log2f(Lsum)) * 0.693147180559945309f : -CUDART_INF_F;
   }
   __syncthreads();
   for (int idx = tid; idx < g * d; idx += nthr) {
@@ -393,7 +397,7 @@ __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel
     const int t = atomicAdd(a.ws.tickets + b * a.n_kv_heads + hk, 1);
     is_last = (t == a.ws.n_splits - 1);
     if (is_last) a.ws.tickets[b * a.n_kv_heads + hk] = 0;  // leave no small counts behind in scratch that other calls reuse
-    if (is_last && len <= 0) set_status(a.status, PQ_ERR_EMPTY);
+    if (is_last && len <= 0 && a.lse == nullptr) set_status(a.status, PQ_ERR_EMPTY);
   }
   __syncthreads();
   if (is_last) {
@@ -406,6 +410,148 @@ __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel
 #include "pq_decode_fast.cuh"
 #include "pq_prefill.cuh"
 namespace pq {
+
+// ---- partial attentions: merge, and exact attention over an uncompressed window -----------------
+// out = sum_p w_p out_p with w_p = exp(lse_p - lse) and lse = log sum_p exp(lse_p): the attention over the union of
+// the token sets behind the parts (token shards on several GPUs; the packed cache and a 16-bit tail).
+__global__ void merge_attention_kernel(int d, int64_t n_rows, int n_parts, const void* parts_out, int parts_dtype,
+                                       const float* parts_lse, void* out, int out_dtype, float* lse_out, int32_t* status) {
+  const int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (idx >= n_rows * d) return;
+  const int64_t row = idx / d;
+  float mx = -CUDART_INF_F;
+  for (int p = 0; p < n_parts; ++p) mx = fmaxf(mx, parts_lse[(int64_t)p * n_rows + row]);
+  float acc = 0.f, wsum = 0.f;
+  if (mx > -CUDART_INF_F) {
+    for (int p = 0; p < n_parts; ++p) {   // part order: the result does not depend on the launch
+      const float l = parts_lse[(int64_t)p * n_rows + row];
+      if (l == -CUDART_INF_F) continue;   // a part without tokens (its output may hold anything)
+      const float w = __expf(l - mx);
+      const int64_t i = (int64_t)p * n_rows * d + idx;
+      const float v = parts_dtype == PQ_DTYPE_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(parts_out)[i])
+                                                   : reinterpret_cast<const float*>(parts_out)[i];
+      acc = fmaf(w, v, acc);
+      wsum += w;
+    }
+    acc /= wsum;
+  } else if (idx == row * d) {
+    set_status(status, PQ_ERR_EMPTY);
+  }
+  if (out_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(out)[idx] = __float2bfloat16(acc);
+  else reinterpret_cast<float*>(out)[idx] = acc;
+  if (lse_out != nullptr && idx == row * d) lse_out[row] = mx > -CUDART_INF_F ? mx + __logf(wsum) : -CUDART_INF_F;
+}
+
+// Exact softmax attention (Eq. 2) of one query per sequence over an uncompressed window of keys and values (the
+// tokens a serving loop keeps in 16 bits, Section 5.3's protocol for generated tokens).  One CTA per (kv head,
+// sequence); chunks of kTailChunk tokens: scores by a thread per token, running maximum and denominator per head,
+// then a thread per coordinate accumulates P . V.
+constexpr int kTailThreads = 128, kTailChunk = 512;
+struct TailArgs {
+  int d, n_q_heads, n_kv_heads, io_dtype, kv_dtype, capacity;
+  float scale;
+  const void* q;
+  const void* k;
+  const void* v;
+  const int32_t* lens;
+  void* out;
+  float* lse;
+  int32_t* status;
+};
+__device__ __forceinline__ float tail_elem(const void* p, int dtype, int64_t i) {
+  return dtype == PQ_DTYPE_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i])
+                                : reinterpret_cast<const float*>(p)[i];
+}
+__global__ void __launch_bounds__(kTailThreads) tail_attention_kernel(TailArgs a) {
+  extern __shared__ float tsm[];
+  const int d = a.d, g = a.n_q_heads / a.n_kv_heads, hk = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
+  const int lane = tid & 31, warp = tid >> 5;
+  float* qs = tsm;                       // [g][d], times scale * log2(e)
+  float* sc = qs + g * d;                // [g][kTailChunk]
+  float* m_sm = sc + g * kTailChunk;     // [g] running maximum (log2 domain)
+  float* l_sm = m_sm + kMaxGroup;        // [g] running denominator
+  float* corr_sm = l_sm + kMaxGroup;     // [g]
+  for (int i = tid; i < g * d; i += kTailThreads)
+    qs[i] = tail_elem(a.q, a.io_dtype, ((int64_t)b * a.n_q_heads + hk * g) * d + i) * a.scale * 1.4426950408889634f;
+  if (tid < g) {
+    m_sm[tid] = -CUDART_INF_F;
+    l_sm[tid] = 0.f;
+  }
+  int len = a.lens[b];
+  len = len < 0 ? 0 : (len > a.capacity ? a.capacity : len);
+  float acc[kMaxGroup];
+#pragma unroll
+  for (int h = 0; h < kMaxGroup; ++h) acc[h] = 0.f;
+  __syncthreads();
+  for (int c0 = 0; c0 < len; c0 += kTailChunk) {
+    const int n = min(kTailChunk, len - c0);
+    for (int t = tid; t < n; t += kTailThreads) {
+      const int64_t row = (((int64_t)b * a.capacity + c0 + t) * a.n_kv_heads + hk) * d;
+      float s[kMaxGroup];
+#pragma unroll
+      for (int h = 0; h < kMaxGroup; ++h) s[h] = 0.f;
+      for (int i = 0; i < d; ++i) {
+        const float kv = tail_elem(a.k, a.kv_dtype, row + i);
+#pragma unroll
+        for (int h = 0; h < kMaxGroup; ++h)
+          if (h < g) s[h] = fmaf(qs[h * d + i], kv, s[h]);
+      }
+#pragma unroll
+      for (int h = 0; h < kMaxGroup; ++h)
+        if (h < g) sc[h * kTailChunk + t] = s[h];
+    }
+    __syncthreads();
+    for (int h = warp; h < g; h += kTailThreads / 32) {   // a warp per head: maximum, probabilities, their sum
+      float mx = -CUDART_INF_F;
+      for (int t = lane; t < n; t += 32) mx = fmaxf(mx, sc[h * kTailChunk + t]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+      const float m_new = fmaxf(m_sm[h], mx);
+      float sum = 0.f;
+      for (int t = lane; t < n; t += 32) {
+        const float p = exp2f(sc[h * kTailChunk + t] - m_new);
+        sc[h * kTailChunk + t] = p;
+        sum += p;
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      if (lane == 0) {
+        const float corr = exp2f(m_sm[h] - m_new);   // 0 on the first chunk
+        corr_sm[h] = corr;
+        l_sm[h] = l_sm[h] * corr + sum;
+        m_sm[h] = m_new;
+      }
+    }
+    __syncthreads();
+    if (tid < d) {
+#pragma unroll
+      for (int h = 0; h < kMaxGroup; ++h)
+        if (h < g) acc[h] *= corr_sm[h];
+      for (int t = 0; t < n; ++t) {
+        const float vv = tail_elem(a.v, a.kv_dtype, (((int64_t)b * a.capacity + c0 + t) * a.n_kv_heads + hk) * d + tid);
+#pragma unroll
+        for (int h = 0; h < kMaxGroup; ++h)
+          if (h < g) acc[h] = fmaf(sc[h * kTailChunk + t], vv, acc[h]);
+      }
+    }
+    __syncthreads();
+  }
+  if (tid < d) {
+#pragma unroll
+    for (int h = 0; h < kMaxGroup; ++h)
+      if (h < g) {
+        const float o = len > 0 ? acc[h] / l_sm[h] : 0.f;
+        const int64_t oi = ((int64_t)b * a.n_q_heads + hk * g + h) * d + tid;
+        if (a.io_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16(o);
+        else reinterpret_cast<float*>(a.out)[oi] = o;
+      }
+  }
+  if (tid < g) {
+    const int64_t li = (int64_t)b * a.n_q_heads + hk * g + tid;
+    if (a.lse != nullptr) a.lse[li] = len > 0 ? (m_sm[tid] + log2f(l_sm[tid])) * 0.693147180559945309f : -CUDART_INF_F;
+    else if (len <= 0) set_status(a.status, PQ_ERR_EMPTY);
+  }
+}
 
 // ---- inspection kernels ----------------------------------------------------------------------
 __global__ void unpack_codes_kernel(int d, int n_kv_heads, const uint8_t* cache, int batch, Paging pg,
@@ -490,7 +636,7 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
                                 const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
                                 const int32_t* cache_lens_dev, int32_t batch, int32_t n_q, int32_t capacity, const pq::Paging& pg,
                                 int32_t max_len, float scale, void* out_dev, void* workspace_dev, int32_t* status_dev,
-                                void* stream) {
+                                void* stream, float* lse_dev = nullptr) {
   if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
   if (!S_dev || !tables_dev || !q_dev || !cache_dev || !cache_lens_dev || !out_dev || !workspace_dev || !status_dev)
     return PQ_ERR_INVALID_ARG;
@@ -509,9 +655,11 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
   a.io_dtype = io_dtype; a.scale = scale; a.S = S_dev; a.tables = reinterpret_cast<const pq::Tables*>(tables_dev);
   a.q = q_dev; a.cache = reinterpret_cast<const uint8_t*>(cache_dev); a.lens = cache_lens_dev; a.out = out_dev;
   a.status = status_dev;
+  a.lse = lse_dev;
   a.pg = pg;
   a.ws = pq::carve_workspace(workspace_dev, head_dim, (int)pairs, n_q_heads, n_kv_heads, max_len);
   const int g = n_q_heads / n_kv_heads;
+  if (lse_dev != nullptr && n_q != 1) return PQ_ERR_UNSUPPORTED;
   if (head_dim == 128 && n_q * g >= pq::kPfRows) {
     // Many queries per sequence: decode each block of the cache once for 64 (query, head) rows on tensor cores.
     static pq::DeviceMemo configured_pf;
@@ -600,6 +748,58 @@ int32_t pq_multi_query_attention_paged(int32_t head_dim, int32_t n_q_heads, int3
   return launch_attention(head_dim, n_q_heads, n_kv_heads, S_dev, tables_dev, q_dev, io_dtype, cache_dev, cache_lens_dev,
                           batch, n_q, pg.page_tokens * pg.pages_per_seq, pg, max_len, scale, out_dev, workspace_dev, status_dev,
                           stream);
+}
+
+int32_t pq_decode_attention_lse(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                                const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
+                                const int32_t* cache_lens_dev, int32_t batch, int32_t capacity, const pq_paging* paging,
+                                int32_t max_len, float scale, void* out_dev, float* lse_dev, void* workspace_dev,
+                                int32_t* status_dev, void* stream) {
+  if (lse_dev == nullptr || ((uintptr_t)lse_dev & 3)) return lse_dev == nullptr ? PQ_ERR_INVALID_ARG : PQ_ERR_ALIGNMENT;
+  pq::Paging pg = pq::contiguous_paging(capacity, batch);
+  if (paging != nullptr) {
+    const int32_t st = pq::paging_from(paging, head_dim, &pg);
+    if (st != PQ_OK) return st;
+    capacity = pg.page_tokens * pg.pages_per_seq;
+  }
+  return launch_attention(head_dim, n_q_heads, n_kv_heads, S_dev, tables_dev, q_dev, io_dtype, cache_dev, cache_lens_dev,
+                          batch, 1, capacity, pg, max_len, scale, out_dev, workspace_dev, status_dev, stream, lse_dev);
+}
+
+int32_t pq_merge_attention(int32_t head_dim, int32_t n_q_heads, int32_t batch, int32_t n_parts, const void* parts_out_dev,
+                           int32_t parts_dtype, const float* parts_lse_dev, void* out_dev, int32_t out_dtype,
+                           float* lse_out_dev, int32_t* status_dev, void* stream) {
+  if (head_dim <= 0 || n_q_heads <= 0 || batch <= 0 || n_parts <= 0 || n_parts > 1024) return PQ_ERR_INVALID_ARG;
+  if (!parts_out_dev || !parts_lse_dev || !out_dev || !status_dev) return PQ_ERR_INVALID_ARG;
+  if ((parts_dtype != PQ_DTYPE_F32 && parts_dtype != PQ_DTYPE_BF16) || (out_dtype != PQ_DTYPE_F32 && out_dtype != PQ_DTYPE_BF16))
+    return PQ_ERR_UNSUPPORTED;
+  const int64_t n_rows = (int64_t)batch * n_q_heads, n = n_rows * head_dim;
+  if (n * n_parts >= (1ll << 40)) return PQ_ERR_UNSUPPORTED;
+  pq::merge_attention_kernel<<<(unsigned)((n + 255) / 256), 256, 0, reinterpret_cast<cudaStream_t>(stream)>>>(
+      head_dim, n_rows, n_parts, parts_out_dev, parts_dtype, parts_lse_dev, out_dev, out_dtype, lse_out_dev, status_dev);
+  return pq::launch_status();
+}
+
+int32_t pq_tail_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const void* q_dev, int32_t io_dtype,
+                          const void* k_tail_dev, const void* v_tail_dev, int32_t kv_dtype, const int32_t* tail_lens_dev,
+                          int32_t batch, int32_t tail_capacity, float scale, void* out_dev, float* lse_dev,
+                          int32_t* status_dev, void* stream) {
+  if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
+  if (!q_dev || !k_tail_dev || !v_tail_dev || !tail_lens_dev || !out_dev || !status_dev) return PQ_ERR_INVALID_ARG;
+  if (batch <= 0 || batch > 65535 || n_q_heads <= 0 || n_kv_heads <= 0 || tail_capacity <= 0 || n_q_heads % n_kv_heads)
+    return PQ_ERR_INVALID_ARG;
+  if (n_q_heads / n_kv_heads > pq::kMaxGroup) return PQ_ERR_UNSUPPORTED;
+  if ((io_dtype != PQ_DTYPE_F32 && io_dtype != PQ_DTYPE_BF16) || (kv_dtype != PQ_DTYPE_F32 && kv_dtype != PQ_DTYPE_BF16))
+    return PQ_ERR_UNSUPPORTED;
+  pq::TailArgs a;
+  a.d = head_dim; a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads; a.io_dtype = io_dtype; a.kv_dtype = kv_dtype;
+  a.capacity = tail_capacity; a.scale = scale; a.q = q_dev; a.k = k_tail_dev; a.v = v_tail_dev; a.lens = tail_lens_dev;
+  a.out = out_dev; a.lse = lse_dev; a.status = status_dev;
+  const int g = n_q_heads / n_kv_heads;
+  const size_t smem = sizeof(float) * ((size_t)g * head_dim + (size_t)g * pq::kTailChunk + 3 * pq::kMaxGroup);
+  dim3 grid(n_kv_heads, batch);
+  pq::tail_attention_kernel<<<grid, pq::kTailThreads, smem, reinterpret_cast<cudaStream_t>(stream)>>>(a);
+  return pq::launch_status();
 }
 
 // ---- decode attention on the library's own scratch ---------------------------------------------

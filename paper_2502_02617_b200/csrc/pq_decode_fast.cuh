@@ -345,7 +345,10 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
           if (a.io_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[idx] = __float2bfloat16(0.f);
           else reinterpret_cast<float*>(a.out)[idx] = 0.f;
         }
-        set_status(a.status, PQ_ERR_EMPTY);
+        if (a.lse != nullptr)
+          for (int h = 0; h < g_heads; ++h) a.lse[(int64_t)b * a.n_q_heads + hk * g_heads + h] = -CUDART_INF_F;
+        else
+          set_status(a.status, PQ_ERR_EMPTY);
       }
       u_parts[u] = parts;
     }

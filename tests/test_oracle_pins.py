@@ -185,6 +185,59 @@ def test_level1_cost_closed_form(cb):
     assert abs(mse - (math.pi / 8) ** 2 / 12) < 1e-14
 
 
+# ---------------------------------------------------------------- partial attentions
+def test_merged_partial_attentions_equal_the_whole():
+    """Eq. 2 with its sums split over disjoint token sets: any split, merged, gives the attention over all tokens;
+    the log-sum-exp has its closed forms (one token: the score; n identical keys: score + log n; no token: -inf)."""
+    rng = np.random.default_rng(8)
+    d, n = 16, 50
+    q, K, V = rng.normal(size=d), rng.normal(size=(n, d)) * 2, rng.normal(size=(n, d))
+    whole = orc.softmax_attention(q, K, V, 0.3)
+    assert abs(orc.log_sum_exp_scores(q, K[:1], 0.3) - 0.3 * K[0] @ q) < 1e-12
+    same = np.repeat(K[:1], 7, axis=0)
+    assert abs(orc.log_sum_exp_scores(q, same, 0.3) - (0.3 * K[0] @ q + math.log(7))) < 1e-12
+    assert orc.log_sum_exp_scores(q, K[:0], 0.3) == -np.inf
+    brute = math.log(sum(math.exp(0.3 * float(K[t] @ q)) for t in range(n)))
+    assert abs(orc.log_sum_exp_scores(q, K, 0.3) - brute) < 1e-12
+    for cuts in ([0, 50], [0, 1, 50], [0, 13, 13, 40, 50], [0, 0, 25, 50, 50]):      # empty sets included
+        outs, lses = [], []
+        for lo, hi in zip(cuts[:-1], cuts[1:]):
+            outs.append(orc.softmax_attention(q, K[lo:hi], V[lo:hi], 0.3) if hi > lo else np.full(d, np.nan))
+            lses.append(orc.log_sum_exp_scores(q, K[lo:hi], 0.3))
+        out, lse = orc.merge_attention(np.array(outs), np.array(lses))
+        assert np.allclose(out, whole, atol=1e-13) and abs(lse - brute) < 1e-12
+    out, lse = orc.merge_attention(np.zeros((2, 3, d)), np.full((2, 3), -np.inf))
+    assert np.all(out == 0) and np.all(lse == -np.inf)
+    # scores far apart: the weights must not overflow
+    out, lse = orc.merge_attention(np.array([np.ones(d), 3 * np.ones(d)]), np.array([800.0, -800.0]))
+    assert np.allclose(out, 1.0) and lse == 800.0
+
+
+def test_attention_with_an_unquantised_tail_is_attention_over_the_concatenation(cb):
+    rng = np.random.default_rng(9)
+    d, n, t = 16, 20, 6
+    S = orc.make_rotation(d, 2)
+    K, V = rng.normal(size=(n, d)), rng.normal(size=(n, d))
+    kc, kr = orc.encode(K, S, cb)[:2]
+    vc, vr = orc.encode(V, S, cb)[:2]
+    q = rng.normal(size=(1, 2, d))
+    kt, vt = rng.normal(size=(1, t, 1, d)), rng.normal(size=(1, t, 1, d))
+    out, lse = orc.attention_with_tail(q, kc[None, None], kr[None, None], vc[None, None], vr[None, None], [n], cb, S, 0.25, kt, vt, [t])
+    Kall = np.concatenate([orc.dequant(kc, kr, cb, S), kt[0, :, 0]])
+    Vall = np.concatenate([orc.dequant(vc, vr, cb, S), vt[0, :, 0]])
+    for h in range(2):
+        s = Kall @ q[0, h] * 0.25
+        p = np.exp(s - s.max())
+        assert np.allclose(out[0, h], (p / p.sum()) @ Vall, atol=1e-13)
+        assert abs(lse[0, h] - (s.max() + math.log(p.sum()))) < 1e-12
+    # no tail: decode attention; no cache: exact attention over the tail
+    a, _ = orc.attention_with_tail(q, kc[None, None], kr[None, None], vc[None, None], vr[None, None], [n], cb, S, 0.25, kt, vt, [0])
+    assert np.allclose(a, orc.decode_attention(q, kc[None, None], kr[None, None], vc[None, None], vr[None, None], [n], cb, S, 0.25), atol=1e-13)
+    b, _ = orc.attention_with_tail(q, kc[None, None], kr[None, None], vc[None, None], vr[None, None], [0], cb, S, 0.25, kt, vt, [t])
+    for h in range(2):
+        assert np.allclose(b[0, h], orc.softmax_attention(q[0, h], kt[0, :, 0], vt[0, :, 0], 0.25), atol=1e-13)
+
+
 # ---------------------------------------------------------------- online codebook (Section 4.1)
 def test_angle_histograms_count_every_angle_in_its_bin():
     S = np.eye(4)

@@ -121,3 +121,52 @@ def test_two_ranks_shard_sequences_without_data_path_collectives():
     want = caches.attend(q, D ** -0.5)
     assert np.allclose(full, want, atol=1e-13)
     assert slowest == [2.0, 5.0]
+
+
+def _token_shard_worker(rank, world, port, results):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        caches, q = _whole_batch()
+        out = np.zeros((B, HQ, D))
+        lse = np.full((B, HQ), -np.inf)
+        g = HQ // HKV
+        for b in range(B):   # this rank's tokens of every sequence: positions p with (p // 16) % world == rank
+            pos = sharding.shard_positions(int(caches.lens[b]), world, rank, granule=16).numpy()
+            for hk in range(HKV):
+                Kh = orc.dequant(caches.k_codes[b, hk, pos], caches.k_radii[b, hk, pos], caches.cb, caches.S)
+                Vh = orc.dequant(caches.v_codes[b, hk, pos], caches.v_radii[b, hk, pos], caches.cb, caches.S)
+                for h in range(hk * g, (hk + 1) * g):
+                    if len(pos):
+                        out[b, h] = orc.softmax_attention(q[b, h], Kh, Vh, D ** -0.5)
+                        lse[b, h] = orc.log_sum_exp_scores(q[b, h], Kh, D ** -0.5)
+        parts_out, parts_lse = sharding.gather_partials(torch.from_numpy(out), torch.from_numpy(lse), dist)
+        if rank == 0:
+            results.put((parts_out.numpy(), parts_lse.numpy()))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_token_shards_gathered_from_two_ranks_merge_to_the_whole():
+    """Token-sharded decode on CPU: the sharding rule, the all-gather of (out, lse) in rank order, and the merge
+    (here the oracle's; on the GPU pq_merge_attention, tested against it) give the attention over all tokens."""
+    assert sharding.shard_positions(300, 2, 1).tolist() == list(range(128, 256))
+    assert sharding.shard_positions(5, 3, 2).tolist() == []
+    got = sorted(sum((sharding.shard_positions(1000, 3, r, 64).tolist() for r in range(3)), []))
+    assert got == list(range(1000))
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    results = ctx.Queue()
+    procs = [ctx.Process(target=_token_shard_worker, args=(r, 2, port, results)) for r in range(2)]
+    for p in procs:
+        p.start()
+    parts_out, parts_lse = results.get(timeout=120)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert parts_out.shape == (2, B, HQ, D) and parts_lse.shape == (2, B, HQ)
+    caches, q = _whole_batch()
+    merged, _ = orc.merge_attention(parts_out, parts_lse)
+    assert np.allclose(merged, caches.attend(q, D ** -0.5), atol=1e-12)
