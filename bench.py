@@ -588,8 +588,9 @@ def measure_tail_window(args, pq, synthetic, dev, rank):
     tail_lens = torch.full((BATCH,), T, dtype=torch.int32, device=dev)
     q = synthetic.queries(3, BATCH, HQ, D, torch.bfloat16, dev)
     q32 = q.float()
-    parts_out = torch.empty((2,) + q32.shape, dtype=torch.float32, device=dev)
-    parts_lse = torch.empty((2, BATCH, HQ), dtype=torch.float32, device=dev)
+    n_splits = 8
+    parts_out = torch.empty((1 + n_splits,) + q32.shape, dtype=torch.float32, device=dev)
+    parts_lse = torch.empty((1 + n_splits, BATCH, HQ), dtype=torch.float32, device=dev)
     out = torch.empty_like(q)
     stream = torch.cuda.current_stream()
     scale = D ** -0.5
@@ -598,7 +599,7 @@ def measure_tail_window(args, pq, synthetic, dev, rank):
         marks = []
         for fn in (lambda: pq.pq_decode_attention_lse(cache.S, cache.tables, q32, cache.cache, cache.lens, HKV, CTX, CTX, scale,
                                                       parts_out[0], parts_lse[0], cache.workspace, cache.status),
-                   lambda: pq.pq_tail_attention(q32, kt, vt, tail_lens, scale, parts_out[1], parts_lse[1], cache.status),
+                   lambda: pq.pq_tail_attention(q32, kt, vt, tail_lens, scale, parts_out[1:], parts_lse[1:], cache.status, n_splits),
                    lambda: pq.pq_merge_attention(parts_out, parts_lse, out, cache.status)):
             a, b = _event(), _event()
             a.record(stream)
@@ -613,7 +614,7 @@ def measure_tail_window(args, pq, synthetic, dev, rank):
     torch.cuda.synchronize()
     cache.check_status()
     med = [float(np.median([r[i][0].elapsed_time(r[i][1]) for r in runs])) * 1e3 for i in range(3)]
-    return {"batch": BATCH, "ctx": CTX, "window_tokens": T, "decode_with_lse_us": med[0], "window_attention_us": med[1],
+    return {"batch": BATCH, "ctx": CTX, "window_tokens": T, "window_splits": n_splits, "decode_with_lse_us": med[0], "window_attention_us": med[1],
             "merge_us": med[2], "window_bytes": 2 * BATCH * T * HKV * D * 2, "rank": rank}
 
 

@@ -341,8 +341,11 @@ int32_t pq_dequant_kv_paged(int32_t head_dim, int32_t n_kv_heads, const float* S
  *
  * pq_tail_attention: exact attention (Eq. 2) of one query per sequence over an uncompressed window,
  * k_tail_dev / v_tail_dev [batch][tail_capacity][n_kv_heads][head_dim] of kv_dtype, of which sequence b uses the
- * first tail_lens_dev[b] rows; out and (if lse_dev is not NULL) lse as above.  With lse_dev == NULL an empty
- * window records PQ_ERR_EMPTY.  Float32 arithmetic; not a tuned kernel (windows are short).
+ * first tail_lens_dev[b] rows (16-byte aligned).  The window's tokens are cut into n_splits equal ranges, each
+ * attended by its own thread blocks: out_dev holds n_splits parts, [n_splits][batch][n_q_heads][head_dim], and lse_dev
+ * [n_splits][batch][n_q_heads], laid out as pq_merge_attention takes them (so the packed cache's part and the
+ * window's parts can sit in one array and be merged by one call).  n_splits = 1 gives the attention over the whole
+ * window; with lse_dev == NULL (n_splits = 1 only) an empty window records PQ_ERR_EMPTY.  Float32 arithmetic.
  */
 int32_t pq_decode_attention_lse(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
                                 const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
@@ -354,8 +357,8 @@ int32_t pq_merge_attention(int32_t head_dim, int32_t n_q_heads, int32_t batch, i
                            float* lse_out_dev, int32_t* status_dev, void* stream);
 int32_t pq_tail_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const void* q_dev, int32_t io_dtype,
                           const void* k_tail_dev, const void* v_tail_dev, int32_t kv_dtype, const int32_t* tail_lens_dev,
-                          int32_t batch, int32_t tail_capacity, float scale, void* out_dev, float* lse_dev,
-                          int32_t* status_dev, void* stream);
+                          int32_t batch, int32_t tail_capacity, int32_t n_splits, float scale, void* out_dev,
+                          float* lse_dev, int32_t* status_dev, void* stream);
 
 #ifdef __cplusplus
 }

@@ -63,7 +63,7 @@ _SIGNATURES = {
     "pq_merge_attention": (c_int32, [c_int32, c_int32, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_void_p, c_int32,
                                      c_void_p, c_void_p, c_void_p]),
     "pq_tail_attention": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_void_p,
-                                    c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p, c_void_p]),
+                                    c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p, c_void_p]),
     "pq_paged_cache_bytes": (c_int64, [c_int32, c_int32, c_int32, c_int32]),
     "pq_encode_kv_paged": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int64, c_int64,
                                      c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -315,14 +315,16 @@ def pq_merge_attention(parts_out, parts_lse, out, status, lse_out=None, stream=N
     return out
 
 
-def pq_tail_attention(q, k_tail, v_tail, tail_lens, scale, out, lse, status, stream=None):
-    """Exact attention of q [B, Hq, d] over an uncompressed window k_tail, v_tail [B, T, Hkv, d] (first tail_lens[b] rows)."""
+def pq_tail_attention(q, k_tail, v_tail, tail_lens, scale, out, lse, status, n_splits=1, stream=None):
+    """Exact attention of q [B, Hq, d] over an uncompressed window k_tail, v_tail [B, T, Hkv, d] (first tail_lens[b] rows),
+    as n_splits partial attentions: out [n_splits, B, Hq, d] (or [B, Hq, d] for one), lse [n_splits, B, Hq]."""
     batch, n_q_heads, d = q.shape
     assert k_tail.is_contiguous() and v_tail.is_contiguous() and k_tail.shape == v_tail.shape and k_tail.dtype == v_tail.dtype
     assert k_tail.shape[0] == batch and k_tail.shape[3] == d and q.is_contiguous() and out.is_contiguous() and out.dtype == q.dtype
+    assert out.numel() == n_splits * q.numel() and (lse is None or lse.numel() == n_splits * batch * n_q_heads)
     _check(lib().pq_tail_attention(d, n_q_heads, k_tail.shape[2], _ptr(q), _dtype_code(q), _ptr(k_tail), _ptr(v_tail),
-                                   _dtype_code(k_tail), _ptr(tail_lens), batch, k_tail.shape[1], float(scale), _ptr(out),
-                                   _ptr(lse), _ptr(status), _stream(stream)), "pq_tail_attention")
+                                   _dtype_code(k_tail), _ptr(tail_lens), batch, k_tail.shape[1], n_splits, float(scale),
+                                   _ptr(out), _ptr(lse), _ptr(status), _stream(stream)), "pq_tail_attention")
 
 
 def sharded_decode_attention(cache, q, dist, group=None, scale=None, stream=None):
@@ -402,12 +404,13 @@ class PolarQuantCache:
         first tail_lens[b] rows): both partial attentions in float32, merged into q's dtype."""
         scale = self.d ** -0.5 if scale is None else scale
         q32 = q.float()
-        parts_out = torch.empty((2,) + q32.shape, dtype=torch.float32, device=q.device)
-        parts_lse = torch.empty((2,) + q32.shape[:2], dtype=torch.float32, device=q.device)
+        n_splits = max(1, min(16, (k_tail.shape[1] + 127) // 128))   # enough thread blocks for the window
+        parts_out = torch.empty((1 + n_splits,) + q32.shape, dtype=torch.float32, device=q.device)
+        parts_lse = torch.empty((1 + n_splits,) + q32.shape[:2], dtype=torch.float32, device=q.device)
         pq_decode_attention_lse(self.S, self.tables, q32, self.cache, self.lens, self.n_kv_heads, self.capacity, self.capacity,
                                 scale, parts_out[0], parts_lse[0], self.workspace, self.status, paging=self._paging(),
                                 stream=stream)
-        pq_tail_attention(q32, k_tail, v_tail, tail_lens, scale, parts_out[1], parts_lse[1], self.status, stream)
+        pq_tail_attention(q32, k_tail, v_tail, tail_lens, scale, parts_out[1:], parts_lse[1:], self.status, n_splits, stream)
         return pq_merge_attention(parts_out, parts_lse, torch.empty_like(q), self.status, stream=stream)
 
     def attend_multi(self, q, out=None, scale=None, max_len=None, stream=None):

@@ -444,11 +444,12 @@ __global__ void merge_attention_kernel(int d, int64_t n_rows, int n_parts, const
 
 // Exact softmax attention (Eq. 2) of one query per sequence over an uncompressed window of keys and values (the
 // tokens a serving loop keeps in 16 bits, Section 5.3's protocol for generated tokens).  One CTA per (kv head,
-// sequence); chunks of kTailChunk tokens: scores by a thread per token, running maximum and denominator per head,
-// then a thread per coordinate accumulates P . V.
+// sequence, split of the window's tokens); a CTA writes the partial attention of its tokens (part blockIdx.z of the
+// output), to be merged by merge_attention_kernel.  Chunks of kTailChunk tokens: scores by a thread per token (16-byte
+// loads of its key row), running maximum and denominator per head, then a thread per coordinate accumulates P . V.
 constexpr int kTailThreads = 128, kTailChunk = 512;
 struct TailArgs {
-  int d, n_q_heads, n_kv_heads, io_dtype, kv_dtype, capacity;
+  int d, n_q_heads, n_kv_heads, io_dtype, kv_dtype, capacity, batch;
   float scale;
   const void* q;
   const void* k;
@@ -477,8 +478,11 @@ __global__ void __launch_bounds__(kTailThreads) tail_attention_kernel(TailArgs a
     m_sm[tid] = -CUDART_INF_F;
     l_sm[tid] = 0.f;
   }
-  int len = a.lens[b];
-  len = len < 0 ? 0 : (len > a.capacity ? a.capacity : len);
+  int len_all = a.lens[b];
+  len_all = len_all < 0 ? 0 : (len_all > a.capacity ? a.capacity : len_all);
+  const int per = (len_all + (int)gridDim.z - 1) / (int)gridDim.z;
+  const int t_begin = min(len_all, (int)blockIdx.z * per), len = min(len_all, t_begin + per) - t_begin;
+  const int64_t part_rows = (int64_t)blockIdx.z * a.batch * a.n_q_heads;   // this split's part of out and lse
   float acc[kMaxGroup];
 #pragma unroll
   for (int h = 0; h < kMaxGroup; ++h) acc[h] = 0.f;
@@ -486,15 +490,31 @@ __global__ void __launch_bounds__(kTailThreads) tail_attention_kernel(TailArgs a
   for (int c0 = 0; c0 < len; c0 += kTailChunk) {
     const int n = min(kTailChunk, len - c0);
     for (int t = tid; t < n; t += kTailThreads) {
-      const int64_t row = (((int64_t)b * a.capacity + c0 + t) * a.n_kv_heads + hk) * d;
+      const int64_t row = (((int64_t)b * a.capacity + t_begin + c0 + t) * a.n_kv_heads + hk) * d;
       float s[kMaxGroup];
 #pragma unroll
       for (int h = 0; h < kMaxGroup; ++h) s[h] = 0.f;
-      for (int i = 0; i < d; ++i) {
-        const float kv = tail_elem(a.k, a.kv_dtype, row + i);
+      for (int i = 0; i < d; i += 8) {   // d is a multiple of 16 and rows are 16-byte aligned
+        float kv[8];
+        if (a.kv_dtype == PQ_DTYPE_BF16) {
+          const uint4 raw = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.k) + row + i));
+          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            kv[2 * e] = __uint_as_float(w[e] << 16);
+            kv[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
+          }
+        } else {
+          const float4 lo = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(a.k) + row + i));
+          const float4 hi = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(a.k) + row + i + 4));
+          kv[0] = lo.x; kv[1] = lo.y; kv[2] = lo.z; kv[3] = lo.w; kv[4] = hi.x; kv[5] = hi.y; kv[6] = hi.z; kv[7] = hi.w;
+        }
 #pragma unroll
         for (int h = 0; h < kMaxGroup; ++h)
-          if (h < g) s[h] = fmaf(qs[h * d + i], kv, s[h]);
+          if (h < g) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) s[h] = fmaf(qs[h * d + i + e], kv[e], s[h]);
+          }
       }
 #pragma unroll
       for (int h = 0; h < kMaxGroup; ++h)
@@ -528,7 +548,7 @@ __global__ void __launch_bounds__(kTailThreads) tail_attention_kernel(TailArgs a
       for (int h = 0; h < kMaxGroup; ++h)
         if (h < g) acc[h] *= corr_sm[h];
       for (int t = 0; t < n; ++t) {
-        const float vv = tail_elem(a.v, a.kv_dtype, (((int64_t)b * a.capacity + c0 + t) * a.n_kv_heads + hk) * d + tid);
+        const float vv = tail_elem(a.v, a.kv_dtype, (((int64_t)b * a.capacity + t_begin + c0 + t) * a.n_kv_heads + hk) * d + tid);
 #pragma unroll
         for (int h = 0; h < kMaxGroup; ++h)
           if (h < g) acc[h] = fmaf(sc[h * kTailChunk + t], vv, acc[h]);
@@ -541,13 +561,13 @@ __global__ void __launch_bounds__(kTailThreads) tail_attention_kernel(TailArgs a
     for (int h = 0; h < kMaxGroup; ++h)
       if (h < g) {
         const float o = len > 0 ? acc[h] / l_sm[h] : 0.f;
-        const int64_t oi = ((int64_t)b * a.n_q_heads + hk * g + h) * d + tid;
+        const int64_t oi = (part_rows + (int64_t)b * a.n_q_heads + hk * g + h) * d + tid;
         if (a.io_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[oi] = __float2bfloat16(o);
         else reinterpret_cast<float*>(a.out)[oi] = o;
       }
   }
   if (tid < g) {
-    const int64_t li = (int64_t)b * a.n_q_heads + hk * g + tid;
+    const int64_t li = part_rows + (int64_t)b * a.n_q_heads + hk * g + tid;
     if (a.lse != nullptr) a.lse[li] = len > 0 ? (m_sm[tid] + log2f(l_sm[tid])) * 0.693147180559945309f : -CUDART_INF_F;
     else if (len <= 0) set_status(a.status, PQ_ERR_EMPTY);
   }
@@ -782,8 +802,10 @@ int32_t pq_merge_attention(int32_t head_dim, int32_t n_q_heads, int32_t batch, i
 
 int32_t pq_tail_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const void* q_dev, int32_t io_dtype,
                           const void* k_tail_dev, const void* v_tail_dev, int32_t kv_dtype, const int32_t* tail_lens_dev,
-                          int32_t batch, int32_t tail_capacity, float scale, void* out_dev, float* lse_dev,
+                          int32_t batch, int32_t tail_capacity, int32_t n_splits, float scale, void* out_dev, float* lse_dev,
                           int32_t* status_dev, void* stream) {
+  if (n_splits < 1 || n_splits > 1024 || (n_splits > 1 && lse_dev == nullptr)) return PQ_ERR_INVALID_ARG;
+  if (((uintptr_t)k_tail_dev | (uintptr_t)v_tail_dev) & 15) return PQ_ERR_ALIGNMENT;
   if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
   if (!q_dev || !k_tail_dev || !v_tail_dev || !tail_lens_dev || !out_dev || !status_dev) return PQ_ERR_INVALID_ARG;
   if (batch <= 0 || batch > 65535 || n_q_heads <= 0 || n_kv_heads <= 0 || tail_capacity <= 0 || n_q_heads % n_kv_heads)
@@ -793,11 +815,11 @@ int32_t pq_tail_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_head
     return PQ_ERR_UNSUPPORTED;
   pq::TailArgs a;
   a.d = head_dim; a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads; a.io_dtype = io_dtype; a.kv_dtype = kv_dtype;
-  a.capacity = tail_capacity; a.scale = scale; a.q = q_dev; a.k = k_tail_dev; a.v = v_tail_dev; a.lens = tail_lens_dev;
+  a.capacity = tail_capacity; a.batch = batch; a.scale = scale; a.q = q_dev; a.k = k_tail_dev; a.v = v_tail_dev; a.lens = tail_lens_dev;
   a.out = out_dev; a.lse = lse_dev; a.status = status_dev;
   const int g = n_q_heads / n_kv_heads;
   const size_t smem = sizeof(float) * ((size_t)g * head_dim + (size_t)g * pq::kTailChunk + 3 * pq::kMaxGroup);
-  dim3 grid(n_kv_heads, batch);
+  dim3 grid(n_kv_heads, batch, n_splits);
   pq::tail_attention_kernel<<<grid, pq::kTailThreads, smem, reinterpret_cast<cudaStream_t>(stream)>>>(a);
   return pq::launch_status();
 }

@@ -140,3 +140,15 @@ def test_compressed_cache_followed_by_an_unquantised_window(d, Hq, Hkv, dtype):
     pq.pq_tail_attention(q, kt, vt, tail_lens, d ** -0.5, out, None, cache.status)
     torch.cuda.synchronize()
     assert cache.status.cpu().tolist()[0] == pq.ERR_EMPTY
+    # five splits of the window, merged, against the unsplit kernel
+    cache.status.zero_()
+    whole, whole_lse = torch.empty_like(q), torch.empty((B, Hq), dtype=torch.float32, device=DEV)
+    pq.pq_tail_attention(q, kt, vt, tail_lens, d ** -0.5, whole, whole_lse, cache.status)
+    parts, parts_lse = torch.empty((5,) + q.shape, device=DEV), torch.empty((5, B, Hq), device=DEV)
+    pq.pq_tail_attention(q, kt, vt, tail_lens, d ** -0.5, parts, parts_lse, cache.status, n_splits=5)
+    lse5 = torch.empty((B, Hq), device=DEV)
+    merged = pq.pq_merge_attention(parts[:, 1:].contiguous(), parts_lse[:, 1:].contiguous(), torch.empty_like(q[1:]), cache.status, lse_out=lse5[1:])
+    torch.cuda.synchronize()
+    assert cache.check_status()[0] == 0
+    assert torch.allclose(merged, whole[1:], atol=2e-6, rtol=1e-5) and torch.allclose(lse5[1:], whole_lse[1:], atol=1e-5)
+    assert torch.isinf(parts_lse[:, 0]).all() and torch.isinf(parts_lse[3:, 1]).all()   # 3 tokens: splits 3 and 4 are empty
