@@ -779,6 +779,11 @@ def run_cuda(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    extra = {"cfg4": measure_config4, "cfg5": measure_config5, "multi_query": measure_multi_query,
+             "online": measure_online_codebook, "paged": measure_paged, "tail": measure_tail_window}
+    if args.only:   # one of the side measurements by itself (profiling captures): its own figures, this rank's
+        print(json.dumps({"only": args.only, "n_gpus": world, "rank": rank, **extra[args.only](args, pq, synthetic, dev, rank)}))
+        return
     local = {"batch": BATCH, "headline": measure_headline(args, pq, synthetic, dev, rank, barrier)}
     torch.cuda.empty_cache()
     if not args.skip_configs:
@@ -813,6 +818,8 @@ def main():
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiling captures)")
     ap.add_argument("--skip-match", action="store_true", help="skip the sampled oracle checks (profiling captures)")
     ap.add_argument("--skip-configs", action="store_true", help="skip configs 4 and 5 (profiling captures)")
+    ap.add_argument("--only", default="", choices=["", "cfg4", "cfg5", "multi_query", "online", "paged", "tail"],
+                    help="run one of the side measurements alone and print its figures (profiling captures)")
     args = ap.parse_args()
     BATCH = args.batch
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup

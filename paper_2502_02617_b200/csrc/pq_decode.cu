@@ -494,7 +494,8 @@ __global__ void __launch_bounds__(kTailThreads) tail_attention_kernel(TailArgs a
       float s[kMaxGroup];
 #pragma unroll
       for (int h = 0; h < kMaxGroup; ++h) s[h] = 0.f;
-      for (int i = 0; i < d; i += 8) {   // d is a multiple of 16 and rows are 16-byte aligned
+#pragma unroll 4
+      for (int i = 0; i < d; i += 8) {   // d is a multiple of 16 and rows are 16-byte aligned; four loads in flight
         float kv[8];
         if (a.kv_dtype == PQ_DTYPE_BF16) {
           const uint4 raw = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.k) + row + i));
@@ -547,6 +548,7 @@ __global__ void __launch_bounds__(kTailThreads) tail_attention_kernel(TailArgs a
 #pragma unroll
       for (int h = 0; h < kMaxGroup; ++h)
         if (h < g) acc[h] *= corr_sm[h];
+#pragma unroll 8
       for (int t = 0; t < n; ++t) {
         const float vv = tail_elem(a.v, a.kv_dtype, (((int64_t)b * a.capacity + t_begin + c0 + t) * a.n_kv_heads + hk) * d + tid);
 #pragma unroll

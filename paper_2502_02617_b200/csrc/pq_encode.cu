@@ -191,7 +191,7 @@ namespace pq {
 // rows of one (K|V, head); thread (row, half) owns 64 rotated coordinates (4 blocks) of its row.
 // ------------------------------------------------------------------------------------------
 constexpr int kFfmaThreads = 256;
-constexpr int kFfmaSmem = (128 * 129 + 2 * 128) * 4 + 64 + (int)sizeof(FixQueue);
+constexpr int kFfmaSmem = (128 * 129 + 2 * 128) * 4 + kFastQuantBytes + (int)sizeof(FixQueue);
 
 // Write the four blocks [4*half, 4*half+4) of the token at `pos`.
 __device__ __forceinline__ void store_half_token(uint8_t* tb, int tok, int half, const FastBlock* fb, int32_t* status) {
@@ -295,7 +295,7 @@ __global__ void __launch_bounds__(kFfmaThreads) encode_ffma_kernel(EncodeArgs a)
   float* xT = smem_f;                  // [128 k][129]
   float* rowsq = smem_f + 128 * 129;   // [2][128]
   FastQuant* fq = reinterpret_cast<FastQuant*>(rowsq + 256);
-  FixQueue* fixq = reinterpret_cast<FixQueue*>(rowsq + 256 + 16);
+  FixQueue* fixq = reinterpret_cast<FixQueue*>(rowsq + 256 + kFastQuantBytes / 4);
   const int tid = threadIdx.x, head = blockIdx.y, kv = blockIdx.z;
   const int row0 = blockIdx.x * 128;
   const void* xbase = kv ? a.V : a.K;

@@ -28,13 +28,22 @@ constexpr float kRotErrTc = 1.1f * (3.f * 9.5367431640625e-07f + 1.4901161193847
 struct FastQuant {
   float t2[3][3];   // tan^2 of the three boundaries of levels 2, 3, 4
   uint32_t sym;     // the boundaries of every level >= 2 are b, pi/4, pi/2 - b (kFlagSymmetricUpper)
+  float ua[3][3], ub[3][3];  // the boundary lines of levels 2, 3, 4 scaled to max(|A|, |B|) = 1: D_k = A_k sa + B_k sb
   uint32_t analytic;       // sym and the uniform level-1 codebook: every decision is a sign test
   const uint2* l1_cells;   // level-1 decision table of any other codebook (Tables::l1_cells or a copy in shared memory)
 };
 
+constexpr int kFastQuantBytes = 128;  // what the kernels set aside for a FastQuant in shared memory
+static_assert(sizeof(FastQuant) <= kFastQuantBytes, "shared-memory slot of FastQuant");
+
 __device__ inline void load_fast_quant(const Tables* tb, FastQuant* fq) {
   for (int l = 0; l < 3; ++l)
-    for (int k = 0; k < 3; ++k) fq->t2[l][k] = (float)tb->bnd_tan2[3 * l + k];
+    for (int k = 0; k < 3; ++k) {
+      const double T = tb->bnd_tan2[3 * l + k];
+      fq->t2[l][k] = (float)T;
+      fq->ua[l][k] = (float)(T > 1.0 ? -1.0 : -T);      // sb - T sa, divided by max(1, T)
+      fq->ub[l][k] = (float)(T > 1.0 ? 1.0 / T : 1.0);
+    }
   fq->sym = (tb->flags & kFlagSymmetricUpper) != 0u;
   fq->analytic = (tb->flags & (kFlagSymmetricUpper | kFlagUniformL1)) == (kFlagSymmetricUpper | kFlagUniformL1);
   fq->l1_cells = &tb->l1_cells[0][0];
@@ -47,7 +56,8 @@ struct RowMargins {
   float dy1;      // level-1 threshold: dy plus the float32 roundings of the level-1 tests
   float c[3];     // 8.4 E^2 for levels 2, 3, 4 (E^2 = 2, 4, 8 dy^2)
   float cs[3];    // the same plus the float32-rounding term of the folded (symmetric) test
-  float base[3];  // 42 E^4 (1 + T_max)^2
+  float csg[3];   // the same for the scaled-line test of any codebook (quant_upper_lines_push)
+  float base[3];  // 42 E^4 * 4: every tested line has coefficients of at most 1
 };
 // `norm` >= ||y||_2 of the row, `rot_err` = bound on the error of one rotated coordinate relative to it.
 // The float32 roundings of the tests themselves are folded into the constants, using u <= norm and w <= norm^2
@@ -64,42 +74,23 @@ __device__ __forceinline__ RowMargins make_row_margins(float norm, float rot_err
   const float e2 = m.dy * m.dy, rr = 6.8e-12f * norm * norm;
 #pragma unroll
   for (int l = 0; l < 3; ++l) {
-    const float el = (float)(2 << l) * e2, t1 = fq.sym ? 2.f : 1.f + fq.t2[l][2];  // 1 + largest T that is tested
+    const float el = (float)(2 << l) * e2;
     m.c[l] = 8.4f * el;
     m.cs[l] = m.c[l] + rr;
-    m.base[l] = 42.f * el * el * t1 * t1;
+    m.csg[l] = fmaf(1.05e-11f * norm, norm, m.c[l]);
+    m.base[l] = 168.f * el * el;
   }
   return m;
 }
 
-// Level >= 2 decision on squared child radii (sa: cosine side, sb: sine side).
+// Level >= 2 decisions on squared child radii (sa: cosine side, sb: sine side): the common margin.
 //   code = #{k : sb > T_k sa},  T_k = tan^2(beta_k)  (both sides of r_b cos b > r_a sin b are >= 0).
-// Margin: the radii are norms of n-coordinate sub-vectors, so they move by at most E = sqrt(n) * dy.
+// The radii are norms of n-coordinate sub-vectors, so they move by at most E = sqrt(n) * dy.
 // With D = sb - T sa, |D - D_exact| <= 2E(r_b + T r_a) + E^2 (1 + T) + rho (sb + T sa), and
 // (2E(r_b + T r_a))^2 <= 8 E^2 (sb + T^2 sa); with (p+q+z)^2 <= 1.05 p^2 + 21 (q+z)^2 <= 1.05 p^2 + 42 (q^2+z^2)
 // boundary k is certified if D_k^2 > 8.4 E^2 (sb + T_k^2 sa) + 42 E^4 (1+T_k)^2 + 42 rho^2 (sb + T_k sa)^2.
-// A cheap test with the largest T for every k (T_max > 1, so sb + T_max^2 sa bounds both sums)
-// certifies almost all decisions; only its failures run the per-boundary test.
-__device__ __forceinline__ uint32_t quant_upper_fast(float sa, float sb, const float* T, float c, float base,
-                                                     bool* ambiguous) {
-  const float d0 = fmaf(-T[0], sa, sb), d1 = fmaf(-T[1], sa, sb), d2 = fmaf(-T[2], sa, sb);
-  // d0 >= d1 >= d2: the code is the number of positive ones (a zero is ambiguous and decided exactly)
-  const uint32_t neg = (__float_as_uint(d0) >> 31) + (__float_as_uint(d1) >> 31) + (__float_as_uint(d2) >> 31);
-  const float dm = fminf(fminf(fabsf(d0), fabsf(d1)), fabsf(d2));
-  const float w = fmaf(T[2] * T[2], sa, sb);
-  const float rhs = fmaf(4.2e-11f * w, w, fmaf(c, w, base));  // rho = 1e-6 covers the float32 roundings
-  bool amb = !(dm * dm > rhs);  // also true for NaN
-  if (amb) {
-    const float u = fmaf(T[2], sa, sb);
-    const float b2 = fmaf(4.2e-11f * u, u, base);
-    const bool ok0 = d0 * d0 > fmaf(c, fmaf(T[0] * T[0], sa, sb), b2);
-    const bool ok1 = d1 * d1 > fmaf(c, fmaf(T[1] * T[1], sa, sb), b2);
-    const bool ok2 = d2 * d2 > fmaf(c, w, b2);
-    amb = !(ok0 && ok1 && ok2);
-  }
-  *ambiguous = amb;
-  return 3u - neg;
-}
+// Both tests below first bring every line to coefficients of at most 1 (by folding for symmetric boundaries, by
+// scaling otherwise), so that sb + T^2 sa <= sa + sb and (1 + T)^2 <= 4 for all of them.
 
 // Codes, squared radius and ambiguity mask of one 16-coordinate block.
 // Ambiguity bits: 0..7 level-1 pairs, 8..11 level 2, 12..13 level 3, 14 level 4.
@@ -180,7 +171,7 @@ __device__ __forceinline__ void quant_level1_table_push(float a, float b, float 
   ok = push_sign(ok, __float_as_uint(slack));
 }
 
-// The level >= 2 decision (see quant_upper_fast) for symmetric boundaries (T0, 1, 1/T0), folded onto m = min(sa, sb), M = max(sa, sb):
+// The level >= 2 decision (margin: see above) for symmetric boundaries (T0, 1, 1/T0), folded onto m = min(sa, sb), M = max(sa, sb):
 // only the diagonal (M - m) and the boundary m = T0 M of the point's own side can be the nearest ones, and the
 // margin of the boundary sb = sa / T0 is the one of m = T0 M after multiplying both sides by T0^2.  Every T
 // that is tested is <= 1, so sb + T^2 sa <= sa + sb and the caller's `base` uses (1 + T)^2 <= 4.
@@ -196,6 +187,24 @@ __device__ __forceinline__ void quant_upper_sym_push(float sa, float sb, float T
   const float slack = fmaf(-dm, dm, fmaf(cs, w, base));
   const uint32_t hb = __float_as_uint(h);
   lv = push_sign(push_sign(lv, hb), ~(hb ^ __float_as_uint(dout)));
+  ok = push_sign(ok, __float_as_uint(slack));
+}
+
+// The level >= 2 decision for any three ascending boundaries.  Each boundary line sb = T_k sa is scaled by
+// 1 / max(1, T_k): D_k = A_k sa + B_k sb with max(|A_k|, |B_k|) = 1 and the sign of sb - T_k sa, so that one margin
+// serves all three: |D_k - exact| <= 2E(|B_k| r_b + |A_k| r_a) + E^2 (|A_k| + |B_k|) + rho (sa + sb) with
+// (2E(...))^2 <= 8 E^2 (sa + sb), (|A_k| + |B_k|)^2 <= 4 and rho = 5e-7 for the float32 roundings (squared radii
+// 2^-22 + 2^-24, the product and the fma), and as derived above boundary k is certified if
+// D_k^2 > 8.4 E^2 w + 42 * 4 E^4 + 42 rho^2 w^2, w = sa + sb <= norm^2 (the last term is inside csg).
+// D_0 >= D_1 >= D_2 up to those roundings, and the code is the number of positive ones: bit 1 = (D_1 > 0), bit 0 =
+// parity of the three.  The function appends the COMPLEMENTS of the two code bits (the sign bits) to `lv` and one
+// "certified" bit to `ok`; the caller complements `lv` once per block.
+__device__ __forceinline__ void quant_upper_lines_push(float sa, float sb, const float* A, const float* B, float csg, float base,
+                                                       uint32_t& lv, uint32_t& ok) {
+  const float d0 = fmaf(A[0], sa, B[0] * sb), d1 = fmaf(A[1], sa, B[1] * sb), d2 = fmaf(A[2], sa, B[2] * sb);
+  const float dm = fminf(fminf(fabsf(d0), fabsf(d1)), fabsf(d2));
+  const float slack = fmaf(-dm, dm, fmaf(csg, sa + sb, base));  // < 0: certified (NaN: not)
+  lv = push_sign(push_sign(lv, __float_as_uint(d1)), __float_as_uint(d0) ^ __float_as_uint(d1) ^ __float_as_uint(d2));
   ok = push_sign(ok, __float_as_uint(slack));
 }
 
@@ -226,21 +235,20 @@ __device__ __forceinline__ void polar_quant_block_fast(const float* y, const Row
     }
     quant_upper_sym_push(s3[0], s3[1], fq.t2[2][0], rm.cs[2], rm.base[2], l4, ok4);
   } else {
-    bool am;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      l2 |= quant_upper_fast(s1[2 * j], s1[2 * j + 1], fq.t2[0], rm.c[0], rm.base[0], &am) << (2 * j);
-      ok2 |= (am ? 0u : 1u) << j;
+    for (int j = 3; j >= 0; --j) {
+      quant_upper_lines_push(s1[2 * j], s1[2 * j + 1], fq.ua[0], fq.ub[0], rm.csg[0], rm.base[0], l2, ok2);
       s2[j] = s1[2 * j] + s1[2 * j + 1];
     }
 #pragma unroll
-    for (int j = 0; j < 2; ++j) {
-      l3 |= quant_upper_fast(s2[2 * j], s2[2 * j + 1], fq.t2[1], rm.c[1], rm.base[1], &am) << (2 * j);
-      ok3 |= (am ? 0u : 1u) << j;
+    for (int j = 1; j >= 0; --j) {
+      quant_upper_lines_push(s2[2 * j], s2[2 * j + 1], fq.ua[1], fq.ub[1], rm.csg[1], rm.base[1], l3, ok3);
       s3[j] = s2[2 * j] + s2[2 * j + 1];
     }
-    l4 = quant_upper_fast(s3[0], s3[1], fq.t2[2], rm.c[2], rm.base[2], &am);
-    ok4 = am ? 0u : 1u;
+    quant_upper_lines_push(s3[0], s3[1], fq.ua[2], fq.ub[2], rm.csg[2], rm.base[2], l4, ok4);
+    l2 = ~l2 & 0xFFu;   // the sign bits are the complements of the code bits
+    l3 = ~l3 & 0xFu;
+    l4 = ~l4 & 0x3u;
   }
   out->l1 = kAnalytic ? level1_codes(l1) : l1;
   out->l2 = l2;

@@ -39,8 +39,8 @@ constexpr int kTcSBytes = 128 * 128 * 2;   // one bf16 term of S (B operand)
 using TcFixQueue = FixQueueT<256>;
 constexpr int kTcSmS = 0;
 constexpr int kTcSmX = kTcSmS + kTcTerms * kTcSBytes;
-constexpr int kTcSmFq = kTcSmX + kTcStages * kTcXBytes;      // FastQuant (40 B)
-constexpr int kTcSmBar = kTcSmFq + 64;                       // x_full[kTcStages], acc_full[kTcSlots]
+constexpr int kTcSmFq = kTcSmX + kTcStages * kTcXBytes;      // FastQuant
+constexpr int kTcSmBar = kTcSmFq + kFastQuantBytes;                       // x_full[kTcStages], acc_full[kTcSlots]
 constexpr int kTcSmMisc = kTcSmBar + 64;                     // tmem base, abort flag, copies issued per stage
 constexpr int kTcSmFix = kTcSmMisc + 64;                     // one TcFixQueue per slot
 constexpr int kTcSmL1 = kTcSmFix + kTcSlots * (int)sizeof(TcFixQueue);  // copy of Tables::l1_cells (codebooks other than the analytic ones)
