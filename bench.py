@@ -618,6 +618,41 @@ def measure_tail_window(args, pq, synthetic, dev, rank):
             "merge_us": med[2], "window_bytes": 2 * BATCH * T * HKV * D * 2, "rank": rank}
 
 
+def measure_general(args, pq, synthetic, dev, rank):
+    """The general entry points on the full recursion of Section 4 (d = 128, log2 d = 7 levels, 3 bits per angle:
+    16 + 127 x 3 bits per vector): encode of 4096 tokens x 8 kv heads and decode attention over batch 8 x 4096 tokens.
+    Reference-speed kernels (float64 encoder, one thread block per sequence and kv head in attention)."""
+    n, bits = 4096, (3,) * 7
+    cache = pq.GeneralPolarQuantCache(BATCH, HQ, HKV, D, bits, n, seed=0, device=dev)
+    K, V = synthetic.kv_like(1000 * rank + 5, n, HKV, D, torch.bfloat16, dev)
+    stream = torch.cuda.current_stream()
+    enc = []
+    for b in range(BATCH):
+        cu = torch.zeros(BATCH + 1, dtype=torch.int32, device=dev)
+        cu[b + 1:] = n
+        e = (_event(), _event())
+        e[0].record(stream)
+        cache.encode(K, V, cu)
+        e[1].record(stream)
+        enc.append(e)
+    q = synthetic.queries(3, BATCH, HQ, D, torch.bfloat16, dev)
+    out = torch.empty_like(q)
+    cache.attend(q, out=out)
+    dec = [(_event(), _event()) for _ in range(5)]
+    for a, b in dec:
+        a.record(stream)
+        cache.attend(q, out=out)
+        b.record(stream)
+    torch.cuda.synchronize()
+    cache.check_status()
+    t_enc = float(np.median([a.elapsed_time(b) for a, b in enc[1:]]))
+    t_dec = float(np.median([a.elapsed_time(b) for a, b in dec]))
+    comp = BATCH * HKV * n * 2 * cache.row_bytes
+    return {"head_dim": D, "levels": 7, "bits_per_angle": 3, "row_bytes": cache.row_bytes, "tokens": n, "batch": BATCH,
+            "encode_ms": t_enc, "encode_vectors_per_s": 2 * n * HKV / (t_enc * 1e-3), "decode_ms": t_dec,
+            "decode_gbs": comp / (t_dec * 1e-3) / 1e9, "rank": rank}
+
+
 def measure_config5(args, pq, synthetic, dev, rank):
     """Config 5: batch 16, ragged contexts in [4096, 65536], prefill in 4096-token chunks, then 128 steps of
     (append one token per sequence, decode attention)."""
@@ -756,6 +791,8 @@ def reduce_and_format(local, steps, warmup, rank, world, dist=None, device="cpu"
                                                     mma_tflops=mq["mma_tflops"] * mq["ms"] / t)
     if local.get("paged"):
         line["configs"]["paged_decode"] = dict(local["paged"], hbm_frac_measured=local["paged"]["gbs"] / peak)
+    if local.get("general"):
+        line["configs"]["general_full_recursion_3bit"] = local["general"]
     if local.get("tail"):
         line["configs"]["tail_window"] = local["tail"]
     if local.get("online"):
@@ -780,7 +817,7 @@ def run_cuda(args):
         torch.cuda.synchronize()
 
     extra = {"cfg4": measure_config4, "cfg5": measure_config5, "multi_query": measure_multi_query,
-             "online": measure_online_codebook, "paged": measure_paged, "tail": measure_tail_window}
+             "online": measure_online_codebook, "paged": measure_paged, "tail": measure_tail_window, "general": measure_general}
     if args.only:   # one of the side measurements by itself (profiling captures): its own figures, this rank's
         print(json.dumps({"only": args.only, "n_gpus": world, "rank": rank, **extra[args.only](args, pq, synthetic, dev, rank)}))
         return
@@ -798,6 +835,8 @@ def run_cuda(args):
         local["paged"] = measure_paged(args, pq, synthetic, dev, rank)
         torch.cuda.empty_cache()
         local["tail"] = measure_tail_window(args, pq, synthetic, dev, rank)
+        torch.cuda.empty_cache()
+        local["general"] = measure_general(args, pq, synthetic, dev, rank)
         torch.cuda.empty_cache()
     cpu = _oracle_sample_throughput(12.0) if rank == 0 and world == 1 and not args.no_cpu_baseline else None
     line = reduce_and_format(local, args.steps, args.warmup, rank, world, dist, dev, cpu)
@@ -818,7 +857,7 @@ def main():
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer leg (profiling captures)")
     ap.add_argument("--skip-match", action="store_true", help="skip the sampled oracle checks (profiling captures)")
     ap.add_argument("--skip-configs", action="store_true", help="skip configs 4 and 5 (profiling captures)")
-    ap.add_argument("--only", default="", choices=["", "cfg4", "cfg5", "multi_query", "online", "paged", "tail"],
+    ap.add_argument("--only", default="", choices=["", "cfg4", "cfg5", "multi_query", "online", "paged", "tail", "general"],
                     help="run one of the side measurements alone and print its figures (profiling captures)")
     args = ap.parse_args()
     BATCH = args.batch

@@ -64,6 +64,7 @@ extern "C" {
 #define PQ_N_CENTROIDS 28  /* 16 + 4 + 4 + 4 */
 #define PQ_N_BOUNDARIES 24 /* 15 + 3 + 3 + 3 */
 #define PQ_HIST_MAX_BINS 1024 /* bins per level of pq_angle_histograms */
+#define PQ_GENERAL_MAX_LEVELS 8 /* recursion depth of the pq_general_* entry points */
 
 /* Human-readable name of a status code (static string, never NULL). */
 const char* pq_status_string(int32_t status);
@@ -359,6 +360,49 @@ int32_t pq_tail_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_head
                           const void* k_tail_dev, const void* v_tail_dev, int32_t kv_dtype, const int32_t* tail_lens_dev,
                           int32_t batch, int32_t tail_capacity, int32_t n_splits, float scale, void* out_dev,
                           float* lse_dev, int32_t* status_dev, void* stream);
+
+/*
+ * General recursion depth and bit tables.  Definition 1 recurses log2 d times and Section 4 counts
+ * b_FPN + (d - 1) b bits per vector for b bits per angle; Section 4.1 stops at L = 4 with (4,2,2,2) bits, which the
+ * entry points above implement at speed.  The pq_general_* entry points take any head_dim = 2^k <= 256, any
+ * n_levels L with 2^L <= head_dim and any bits[l] in 1..6 for level l + 1 (a block is 2^L coordinates and owns one
+ * fp16 radius), with plain kernels: the encoder works in float64 (codes are those of a float64 evaluation of
+ * Algorithm 1: rotate, atan2, count the boundaries below the angle), attention in float32 with one thread block per
+ * (sequence, kv head).  Reference speed, not the tuned path.
+ *   codebooks      centroids float64[sum_l 2^bits[l]], boundaries float64[sum_l (2^bits[l] - 1)], levels concatenated,
+ *                  ascending; pq_general_fit_codebooks gives the Lloyd-Max codebooks of the analytic densities
+ *                  (Lemma 2); the device entry points take them as device arrays (8-byte aligned)
+ *   cache          [batch][n_kv_heads][K | V][capacity][row_bytes]; a row holds, per level, the level's head_dim / 2^l
+ *                  codes as one bit stream (least significant bit first, padded to a byte), padding to an even offset,
+ *                  then the fp16 radii.  pq_general_sizes reports row_bytes and the counts.
+ *   canonical code order (pq_general_unpack_codes): level 1 codes j = 0 .. d/2 - 1, then level 2, ...; angle j of
+ *                  level l is formed from entries 2j (cosine side) and 2j + 1 of level l - 1
+ * Status words, dtypes, strides, cu_seqlens and cache_lens behave as for pq_encode_kv / pq_decode_attention.
+ */
+typedef struct pq_general_config {
+  int32_t head_dim;
+  int32_t n_levels;
+  int32_t bits[PQ_GENERAL_MAX_LEVELS];
+} pq_general_config;
+
+int32_t pq_general_sizes(const pq_general_config* cfg, int32_t* n_centroids, int32_t* n_boundaries, int32_t* n_codes,
+                         int32_t* n_radii, int32_t* row_bytes);
+int32_t pq_general_fit_codebooks(const pq_general_config* cfg, double* centroids_host, double* boundaries_host);
+int64_t pq_general_cache_bytes(const pq_general_config* cfg, int32_t batch, int32_t n_kv_heads, int32_t capacity);
+int32_t pq_general_encode_kv(const pq_general_config* cfg, int32_t n_kv_heads, const float* S_dev,
+                             const double* boundaries_dev, const void* K_dev, const void* V_dev, int32_t in_dtype,
+                             int64_t token_stride, int64_t head_stride, const int32_t* cu_seqlens_dev, int32_t batch,
+                             int32_t total_tokens, void* cache_dev, int32_t* cache_lens_dev, int32_t capacity,
+                             int32_t* status_dev, void* stream);
+int32_t pq_general_decode_attention(const pq_general_config* cfg, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
+                                    const double* centroids_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
+                                    const int32_t* cache_lens_dev, int32_t batch, int32_t capacity, float scale,
+                                    void* out_dev, int32_t* status_dev, void* stream);
+int32_t pq_general_unpack_codes(const pq_general_config* cfg, int32_t n_kv_heads, const void* cache_dev, int32_t batch,
+                                int32_t capacity, int32_t n_tokens, uint8_t* codes_dev, void* radii_dev, void* stream);
+int32_t pq_general_dequant_kv(const pq_general_config* cfg, int32_t n_kv_heads, const float* S_dev, const double* centroids_dev,
+                              const void* cache_dev, int32_t batch, int32_t capacity, int32_t n_tokens, float* x_hat_dev,
+                              void* stream);
 
 #ifdef __cplusplus
 }

@@ -5,5 +5,5 @@ package does not load the CUDA library; the first API call does, and raises if i
 """
 from . import synthetic  # noqa: F401
 from .api import *  # noqa: F401,F403
-from .api import PagedPolarQuantCache, Paging, PolarQuantCache, PolarQuantError  # noqa: F401
+from .api import GeneralConfig, GeneralPolarQuantCache, PagedPolarQuantCache, Paging, PolarQuantCache, PolarQuantError  # noqa: F401
 from .sharding import gather_partials, shard_positions  # noqa: F401

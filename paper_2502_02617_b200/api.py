@@ -64,6 +64,17 @@ _SIGNATURES = {
                                      c_void_p, c_void_p, c_void_p]),
     "pq_tail_attention": (c_int32, [c_int32, c_int32, c_int32, c_void_p, c_int32, c_void_p, c_void_p, c_int32, c_void_p,
                                     c_int32, c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "pq_general_sizes": (c_int32, [c_void_p, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
+    "pq_general_fit_codebooks": (c_int32, [c_void_p, c_void_p, c_void_p]),
+    "pq_general_cache_bytes": (c_int64, [c_void_p, c_int32, c_int32, c_int32]),
+    "pq_general_encode_kv": (c_int32, [c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int64, c_int64,
+                                       c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_int32, c_void_p, c_void_p]),
+    "pq_general_decode_attention": (c_int32, [c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_void_p,
+                                              c_void_p, c_int32, c_int32, c_float, c_void_p, c_void_p, c_void_p]),
+    "pq_general_unpack_codes": (c_int32, [c_void_p, c_int32, c_void_p, c_int32, c_int32, c_int32, c_void_p, c_void_p,
+                                          c_void_p]),
+    "pq_general_dequant_kv": (c_int32, [c_void_p, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_int32, c_int32,
+                                        c_void_p, c_void_p]),
     "pq_paged_cache_bytes": (c_int64, [c_int32, c_int32, c_int32, c_int32]),
     "pq_encode_kv_paged": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_int32, c_int64, c_int64,
                                      c_void_p, c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_void_p, c_void_p]),
@@ -525,3 +536,88 @@ class PagedPolarQuantCache(PolarQuantCache):
                                          self.batch, ctypes.addressof(pg), n_tokens, _ptr(out), _stream(None)),
                "pq_dequant_kv_paged")
         return out
+
+
+class GeneralConfig(ctypes.Structure):
+    """struct pq_general_config of include/polarquant.h: any recursion depth and bits per level."""
+    _fields_ = [("head_dim", c_int32), ("n_levels", c_int32), ("bits", c_int32 * 8)]
+
+    @classmethod
+    def of(cls, head_dim: int, bits) -> "GeneralConfig":
+        arr = (c_int32 * 8)(*(list(bits) + [0] * (8 - len(bits))))
+        return cls(head_dim, len(bits), arr)
+
+    def sizes(self):
+        """(n_centroids, n_boundaries, n_codes, n_radii, row_bytes)"""
+        out = [c_int32() for _ in range(5)]
+        _check(lib().pq_general_sizes(ctypes.addressof(self), *[ctypes.addressof(o) for o in out]), "pq_general_sizes")
+        return tuple(o.value for o in out)
+
+
+def pq_general_fit_codebooks(cfg: GeneralConfig):
+    """Lloyd-Max codebooks of the analytic densities for every level of `cfg`: (centroids, boundaries) float64 CPU tensors."""
+    n_cen, n_bnd = cfg.sizes()[:2]
+    cen, bnd = torch.empty(n_cen, dtype=torch.float64), torch.empty(n_bnd, dtype=torch.float64)
+    _check(lib().pq_general_fit_codebooks(ctypes.addressof(cfg), cen.data_ptr(), bnd.data_ptr()), "pq_general_fit_codebooks")
+    return cen, bnd
+
+
+class GeneralPolarQuantCache:
+    """A contiguous cache for any recursion depth and bit table (pq_general_*): reference-speed kernels."""
+
+    def __init__(self, batch, n_q_heads, n_kv_heads, d, bits, capacity, seed=0, device="cuda", S=None, codebooks=None):
+        self.batch, self.n_q_heads, self.n_kv_heads, self.d, self.capacity = batch, n_q_heads, n_kv_heads, d, capacity
+        self.bits = tuple(bits)
+        self.cfg = GeneralConfig.of(d, bits)
+        _, _, self.n_codes, self.n_radii, self.row_bytes = self.cfg.sizes()
+        self.device = torch.device(device)
+        self.S_host = pq_make_rotation(d, seed) if S is None else S.to(torch.float32).cpu().contiguous()
+        self.centroids, self.boundaries = pq_general_fit_codebooks(self.cfg) if codebooks is None else codebooks
+        self.S = self.S_host.to(self.device)
+        self.centroids_dev, self.boundaries_dev = self.centroids.to(self.device), self.boundaries.to(self.device)
+        n = int(lib().pq_general_cache_bytes(ctypes.addressof(self.cfg), batch, n_kv_heads, capacity))
+        if n < 0:
+            raise PolarQuantError(n, "pq_general_cache_bytes")
+        self.cache = torch.empty(n, dtype=torch.uint8, device=self.device)
+        self.lens = torch.zeros(batch, dtype=torch.int32, device=self.device)
+        self.status = torch.zeros(STATUS_WORDS, dtype=torch.int32, device=self.device)
+
+    def encode(self, K, V, cu_seqlens, stream=None):
+        total, n_kv_heads, d = K.shape
+        assert V.shape == K.shape and V.dtype == K.dtype and K.stride(2) == 1 and V.stride() == K.stride() and d == self.d
+        _check(lib().pq_general_encode_kv(ctypes.addressof(self.cfg), n_kv_heads, _ptr(self.S), _ptr(self.boundaries_dev), _ptr(K),
+                                          _ptr(V), _dtype_code(K), K.stride(0), K.stride(1), _ptr(cu_seqlens),
+                                          cu_seqlens.numel() - 1, total, _ptr(self.cache), _ptr(self.lens), self.capacity,
+                                          _ptr(self.status), _stream(stream)), "pq_general_encode_kv")
+
+    def attend(self, q, out=None, scale=None, stream=None):
+        out = torch.empty_like(q) if out is None else out
+        batch, n_q_heads, d = q.shape
+        assert q.is_contiguous() and out.is_contiguous() and out.dtype == q.dtype and d == self.d
+        _check(lib().pq_general_decode_attention(ctypes.addressof(self.cfg), n_q_heads, self.n_kv_heads, _ptr(self.S),
+                                                 _ptr(self.centroids_dev), _ptr(q), _dtype_code(q), _ptr(self.cache),
+                                                 _ptr(self.lens), batch, self.capacity,
+                                                 float(self.d ** -0.5 if scale is None else scale), _ptr(out),
+                                                 _ptr(self.status), _stream(stream)), "pq_general_decode_attention")
+        return out
+
+    def unpack(self, n_tokens):
+        codes = torch.empty((self.batch, self.n_kv_heads, 2, n_tokens, self.n_codes), dtype=torch.uint8, device=self.device)
+        radii = torch.empty((self.batch, self.n_kv_heads, 2, n_tokens, self.n_radii), dtype=torch.float16, device=self.device)
+        _check(lib().pq_general_unpack_codes(ctypes.addressof(self.cfg), self.n_kv_heads, _ptr(self.cache), self.batch,
+                                             self.capacity, n_tokens, _ptr(codes), _ptr(radii), _stream(None)),
+               "pq_general_unpack_codes")
+        return codes, radii
+
+    def dequant(self, n_tokens):
+        out = torch.empty((self.batch, self.n_kv_heads, 2, n_tokens, self.d), dtype=torch.float32, device=self.device)
+        _check(lib().pq_general_dequant_kv(ctypes.addressof(self.cfg), self.n_kv_heads, _ptr(self.S), _ptr(self.centroids_dev),
+                                           _ptr(self.cache), self.batch, self.capacity, n_tokens, _ptr(out), _stream(None)),
+               "pq_general_dequant_kv")
+        return out
+
+    def check_status(self):
+        st = self.status.cpu().tolist()
+        if st[0] != OK:
+            raise PolarQuantError(st[0], "device status")
+        return st

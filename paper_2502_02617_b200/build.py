@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libpolarquant.so")
-SOURCES = ["pq_host.cu", "pq_encode.cu", "pq_decode.cu"]
+SOURCES = ["pq_host.cu", "pq_encode.cu", "pq_decode.cu", "pq_general.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared"]
 

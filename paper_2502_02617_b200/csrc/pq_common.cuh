@@ -13,6 +13,7 @@
 namespace pq {
 
 constexpr int kTokenBlock = 64;  // tokens per cache token-block
+constexpr int kMaxGroup = 8;     // query heads per kv head that one thread block of an attention kernel handles
 constexpr int kBlockDim = 16;    // coordinates per polar block (L = 4 levels)
 
 // Offsets of each level inside the concatenated centroid / boundary arrays.

@@ -120,7 +120,6 @@ __host__ inline Workspace carve_workspace(void* base, int d, int batch, int n_q_
   return w;
 }
 
-constexpr int kMaxGroup = 8;  // query heads per kv head handled by one CTA
 
 struct DecodeArgs {
   int d, n_q_heads, n_kv_heads, batch, capacity, io_dtype;

@@ -124,6 +124,27 @@ def test_histogram_clustering_matches_the_oracle():
     assert L.pq_fit_codebooks_from_histograms(cen.data_ptr(), 4096, None, cen.data_ptr(), cen.data_ptr()) == pq.ERR_INVALID_ARG
 
 
+def test_general_configurations_sizes_and_codebooks():
+    """pq_general_*: the row of (4,2,2,2) at d = 128 is the 62 bytes of Section 4.1; the full recursion with 3 bits
+    is Section 4's b_FPN + (d - 1) b bits (padded to bytes per level); codebooks equal the oracle's Lloyd-Max ones."""
+    assert pq.GeneralConfig.of(128, (4, 2, 2, 2)).sizes() == (28, 24, 120, 8, 62)
+    n_cen, n_bnd, n_codes, n_radii, row = pq.GeneralConfig.of(128, (3,) * 7).sizes()
+    assert (n_cen, n_bnd, n_codes, n_radii) == (56, 49, 127, 1)
+    assert row == sum(-(-(128 >> (l + 1)) * 3 // 8) for l in range(7)) + 2 and row * 8 >= 16 + 127 * 3
+    for d, bits in ((64, (4, 3, 2)), (256, (2,) * 8), (16, (2, 2, 2, 2))):
+        cen, bnd = pq.pq_general_fit_codebooks(pq.GeneralConfig.of(d, bits))
+        cb = orc.fit_codebooks(bits)
+        assert np.max(np.abs(cen.numpy() - cb.flat_centroids())) < 1e-10 and np.max(np.abs(bnd.numpy() - cb.flat_boundaries())) < 1e-10
+    for d, bits in ((48, (2, 2)), (16, (2,) * 5), (64, (7, 2)), (512, (2, 2)), (64, ()), (64, (0, 2))):
+        with pytest.raises(pq.PolarQuantError):
+            pq.GeneralConfig.of(d, bits).sizes()
+    cfg = pq.GeneralConfig.of(64, (4, 2))
+    L = pq.lib()
+    assert L.pq_general_cache_bytes(ctypes.addressof(cfg), 2, 3, 10) == 2 * 3 * 2 * 10 * cfg.sizes()[4]
+    assert L.pq_general_encode_kv(ctypes.addressof(cfg), 2, None, 16, 16, 16, 1, 128, 64, 16, 1, 4, 16, 16, 8, 16, None) == pq.ERR_INVALID_ARG
+    assert L.pq_general_decode_attention(ctypes.addressof(cfg), 18, 2, 16, 16, 16, 1, 16, 16, 1, 8, 0.1, 16, 16, None) == pq.ERR_UNSUPPORTED
+
+
 def test_cache_costs_62_bytes_per_token_at_d128():
     T = pq.token_block()
     assert pq.pq_cache_bytes(128, 1, 8, 32768) == 2 * 8 * 32768 * 62
