@@ -130,7 +130,8 @@ def test_general_configurations_sizes_and_codebooks():
     assert pq.GeneralConfig.of(128, (4, 2, 2, 2)).sizes() == (28, 24, 120, 8, 62)
     n_cen, n_bnd, n_codes, n_radii, row = pq.GeneralConfig.of(128, (3,) * 7).sizes()
     assert (n_cen, n_bnd, n_codes, n_radii) == (56, 49, 127, 1)
-    assert row == sum(-(-(128 >> (l + 1)) * 3 // 8) for l in range(7)) + 2 and row * 8 >= 16 + 127 * 3
+    code_bytes = sum(-(-(128 >> (l + 1)) * 3 // 8) for l in range(7))      # 24 + 12 + 6 + 3 + 2 + 1 + 1
+    assert code_bytes == 49 and row == code_bytes + 1 + 2 and row * 8 >= 16 + 127 * 3   # radii start at an even offset
     for d, bits in ((64, (4, 3, 2)), (256, (2,) * 8), (16, (2, 2, 2, 2))):
         cen, bnd = pq.pq_general_fit_codebooks(pq.GeneralConfig.of(d, bits))
         cb = orc.fit_codebooks(bits)
