@@ -255,6 +255,9 @@ int32_t pq_decode_attention_static(int32_t head_dim, int32_t n_q_heads, int32_t 
  * waits for its copies in flight, releases what it holds and records PQ_ERR_TIMEOUT in status word 0;
  * nothing on the device is left waiting and the next call runs normally.  (The paper has no
  * counterpart: it exercises the error handling of Section "General rules" without losing a copy.)
+ * `which` = 3 is of another kind: the next pq_multi_query_attention call at head_dim 128 whose chunk fills
+ * 128 rows runs the register-fragment (mma.sync) kernel instead of the tcgen05 one, so that the two can
+ * be compared on the same inputs.
  */
 int32_t pq_debug_fail_next_wait(int32_t which);
 

@@ -408,6 +408,7 @@ __global__ void __launch_bounds__(kSimpleThreads) decode_attention_simple_kernel
 }  // namespace pq
 #include "pq_decode_fast.cuh"
 #include "pq_prefill.cuh"
+#include "pq_prefill_tc.cuh"
 namespace pq {
 
 // ---- partial attentions: merge, and exact attention over an uncompressed window -----------------
@@ -681,6 +682,15 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
   a.ws = pq::carve_workspace(workspace_dev, head_dim, (int)pairs, n_q_heads, n_kv_heads, max_len);
   const int g = n_q_heads / n_kv_heads;
   if (lse_dev != nullptr && n_q != 1) return PQ_ERR_UNSUPPORTED;
+  if (head_dim == 128 && n_q * g >= pq::kPtRows && !pq::take_debug_wait_failure(3)) {
+    // Chunks that fill 128 rows: the tcgen05 kernel (operands in shared memory, accumulators in tensor memory).
+    static pq::DeviceMemo configured_pt;
+    if (pq::configure_for_device(pq::prefill_tc_kernel, pq::kPtSmTotal, configured_pt) == 0) return PQ_ERR_CUDA;
+    const int qb_rows = pq::kPtRows / g;
+    dim3 grid((n_q + qb_rows - 1) / qb_rows, n_kv_heads, batch);
+    pq::prefill_tc_kernel<<<grid, pq::kPtThreads, pq::kPtSmTotal, st>>>(a, n_q);
+    return pq::launch_status();
+  }
   if (head_dim == 128 && n_q * g >= pq::kPfRows) {
     // Many queries per sequence: decode each block of the cache once for 64 (query, head) rows on tensor cores.
     static pq::DeviceMemo configured_pf;

@@ -27,6 +27,8 @@
 #pragma once
 #include <cuda.h>
 
+#include "pq_tc_common.cuh"
+
 namespace pq {
 
 constexpr int kTcThreads = 512;
@@ -45,97 +47,11 @@ constexpr int kTcSmMisc = kTcSmBar + 64;                     // tmem base, abort
 constexpr int kTcSmFix = kTcSmMisc + 64;                     // one TcFixQueue per slot
 constexpr int kTcSmL1 = kTcSmFix + kTcSlots * (int)sizeof(TcFixQueue);  // copy of Tables::l1_cells (codebooks other than the analytic ones)
 constexpr int kTcSmTotal = kTcSmL1 + 8 * kL1Cells * 8 + 1024;             // + slack for 1024-byte alignment
-constexpr int kTcSpin = 1 << 22;
 static_assert(kTcTerms == 3, "kRotErrTc is the bound for three terms");
 static_assert(sizeof(TcFixQueue) % 16 == 0, "queues are laid out back to back");
 static_assert(kTcSmTotal <= 227 * 1024, "shared memory of one CTA");
 static_assert(4 * PQ_HIST_MAX_BINS * 4 <= kTcSlots * (int)sizeof(TcFixQueue), "the histogram takes the queues' place");
 static_assert(kFixSdBytes <= kTcSmFq, "the float64 copy of S must fit in the operand buffers");
-
-__device__ __forceinline__ uint32_t tc_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void tc_mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void tc_mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool tc_mbar_try(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool tc_mbar_test(uint32_t bar, uint32_t parity) {  // non-blocking probe
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool tc_mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  if (tc_mbar_test(bar, parity)) return true;  // the usual case: completed a tile ago
-  for (int i = 0; i < kTcSpin; ++i) {
-    if (tc_mbar_try(bar, parity)) return true;
-    if (i > 32) {
-      __nanosleep(64);
-      if (*abort_flag) return false;
-    }
-  }
-  *abort_flag = 1;
-  return false;
-}
-
-// K-major, 128-byte-swizzled shared-memory matrix descriptor (rows of 64 bf16 = 128 bytes, groups of
-// 8 rows 1024 bytes apart).
-__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t addr) {
-  uint64_t d = (uint64_t)((addr & 0x3FFFFu) >> 4);
-  d |= (uint64_t)1 << 16;            // leading byte offset (unused with 128-byte swizzle)
-  d |= (uint64_t)(1024 >> 4) << 32;  // stride byte offset: 8 rows
-  d |= (uint64_t)1 << 46;            // descriptor version of this architecture
-  d |= (uint64_t)2 << 61;            // 128-byte swizzle
-  return d;
-}
-// kind::f16 instruction descriptor: D = f32, A = B = bf16, both K-major, N = 128, M = 128.
-constexpr uint32_t kTcIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
-
-__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(kTcIdesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// 32 consecutive columns of this thread's tensor-memory lane (issue only; follow with tc_wait_ld).
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, float* v) {
-  uint32_t r[32];
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-      "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr));
-  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-}
 
 struct TcMaps {
   CUtensorMap k, v;

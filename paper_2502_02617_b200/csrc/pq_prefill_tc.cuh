@@ -1,0 +1,391 @@
+// Multi-query attention over the packed cache on the 5th-generation tensor cores, head_dim 128 (included by
+// pq_decode.cu).  Same computation as pq_prefill.cuh -- the last n_q positions of a sequence attend causally to the
+// cached tokens (Eq. 2 / Eq. 3) -- for chunks that fill 128 rows = (128 / g) queries x the g query heads of a kv head.
+//
+// One CTA of nine warps per (query block, kv head, sequence) loops over the 64-token blocks its queries may see:
+//   * warps 4-7 ("decoders") copy the packed K and V block with cp.async, DeQuant it (Algorithm 1, float32 from
+//     the 28 centroids: a thread decodes half a token) and write the tensor-core operands into shared memory in
+//     the K-major 128-byte-swizzled layout: K_hat as fp16 value + fp16 residual [token][coordinate], V_hat
+//     transposed [coordinate][token]; two stages, so block j + 1 is decoded while block j is multiplied;
+//   * one thread of warp 8 issues the MMAs: S_j = Q' K_hat^T as three products (lo*hi, hi*lo, hi*hi; M = 128,
+//     N = 64, eight k-steps each) into one of two 64-column accumulators in tensor memory, and O += P_j V_hat
+//     (M = 128, N = 128, four k-steps) into a 128-column accumulator; the tensor core reads every operand from
+//     shared memory itself, so no warp re-reads a tile (the register-fragment kernel spends 70 % of the
+//     shared-memory pipe on exactly that);
+//   * warps 0-3 ("row owners": tensor-memory lane = row = thread) read S_j with tcgen05.ld, apply the causal mask
+//     and the online softmax in the log2 domain without any shuffle (a thread owns its whole row), and write P_j
+//     in fp16 as the A operand of the value MMA.  The running maximum is updated lazily: only when a score exceeds
+//     it by more than 8 is the output accumulator rescaled (tcgen05.ld / multiply / tcgen05.st by the row's owner,
+//     after the previous value MMA has completed); otherwise p <= 2^8 stays well inside fp16.
+// Q' = (Q S) * scale * log2 e is formed once per CTA in float32 and kept as fp16 value + residual; the output is
+// normalised and rotated back by S^T in float32 when the CTA ends.  All hand-offs are mbarriers (decoded stage
+// full, scores full / read, P full, value MMA done = stage and P buffer free); every wait is bounded, and a wait
+// that gives up makes every role leave its loop, after which the CTA drains its copies and MMAs, releases tensor
+// memory and records PQ_ERR_TIMEOUT.
+#pragma once
+
+#include "pq_tc_common.cuh"
+
+namespace pq {
+
+constexpr int kPtThreads = 288;
+constexpr int kPtRows = 128;
+constexpr int kPtQBytes = 128 * 128 * 2;            // Q' hi or lo: two k-halves of 128 rows x 128 bytes
+constexpr int kPtKBytes = 64 * 128 * 2;             // K_hat hi or lo of a block: two k-halves of 64 tokens x 128 bytes
+constexpr int kPtVBytes = 128 * 64 * 2;             // V_hat^T of a block: 128 coordinates x 64 tokens
+constexpr int kPtPBytes = 128 * 64 * 2;             // P of a block: 128 rows x 64 tokens
+constexpr int kPtStageBytes = 2 * kPtKBytes + kPtVBytes;
+constexpr int kPtSmQhi = 0, kPtSmQlo = kPtSmQhi + kPtQBytes;
+constexpr int kPtSmKv = kPtSmQlo + kPtQBytes;       // two stages; also q in float32 at the start and O at the end
+constexpr int kPtSmP = kPtSmKv + 2 * kPtStageBytes; // two buffers
+constexpr int kPtSmRaw = kPtSmP + 2 * kPtPBytes;    // two packed (K block, V block) buffers
+constexpr int kPtSmTab = kPtSmRaw + 2 * kPfRawBytes;
+constexpr int kPtSmBar = kPtSmTab + 256;            // kv_full[2], s_full[2], s_free[2], p_full[2], pv_done[2], drain
+constexpr int kPtSmMisc = kPtSmBar + 96;            // tensor-memory base, abort flag
+constexpr int kPtSmTotal = kPtSmMisc + 32 + 1024;   // + slack for 1024-byte alignment
+constexpr int kPtOStride = 132;                     // floats per row of the output staging
+static_assert(kPtSmTotal <= 227 * 1024, "shared memory of one CTA");
+static_assert(128 * kPtOStride * 4 <= 2 * kPtStageBytes && 128 * 128 * 4 <= 2 * kPtStageBytes, "float32 staging fits in the stages");
+static_assert(kPtSmKv % 1024 == 0 && kPtStageBytes % 1024 == 0 && kPtSmP % 1024 == 0, "swizzled tiles start on 1024-byte boundaries");
+
+// acc[r] += sum_k x[r][k0 + k] * w[k] for 64 rows of a float32 tile in shared memory (the same address in every thread)
+__device__ __forceinline__ void pt_rank4(float (&acc)[64], const float* x, int ld, int k0, float4 w) {
+#pragma unroll
+  for (int r = 0; r < 64; ++r) {
+    const float4 v = *reinterpret_cast<const float4*>(x + r * ld + k0);
+    acc[r] = fmaf(v.x, w.x, fmaf(v.y, w.y, fmaf(v.z, w.z, fmaf(v.w, w.w, acc[r]))));
+  }
+}
+
+// Named-barrier OR over `n_threads` threads (also a barrier).
+__device__ __forceinline__ bool pt_bar_or(int bar_id, int n_threads, bool v) {
+  uint32_t out;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.or.pred p, %2, %3, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(out)
+      : "r"((uint32_t)v), "r"(bar_id), "r"(n_threads)
+      : "memory");
+  return out != 0;
+}
+
+__global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a, int n_q) {
+  extern __shared__ uint8_t pt_smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(pt_smem_raw) + 1023) & ~(uintptr_t)1023);
+  const uint32_t sb = tc_smem_u32(smem);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int g = a.n_q_heads / a.n_kv_heads;
+  const int qb_rows = kPtRows / g;                      // queries of a CTA
+  const int q0 = blockIdx.x * qb_rows, hk = blockIdx.y, b = blockIdx.z;
+  const int n_rows = min(qb_rows, n_q - q0) * g;        // rows in use; row r = (query q0 + r / g, head hk * g + r % g)
+  const int len = a.lens[b];
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kPtSmMisc + 4);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kPtSmMisc);
+  float* cen_cos = reinterpret_cast<float*>(smem + kPtSmTab);
+  float* cen_sin = cen_cos + 32;
+  const uint32_t bar_kv = sb + kPtSmBar, bar_sfull = bar_kv + 16, bar_sfree = bar_kv + 32, bar_pfull = bar_kv + 48,
+                 bar_pv = bar_kv + 64, bar_drain = bar_kv + 80;
+  auto row_index = [&](int r) -> int64_t {               // offset of row r in q / out ([batch][n_q][n_q_heads][128])
+    return (((int64_t)b * n_q + q0 + r / g) * a.n_q_heads + hk * g + r % g) * 128;
+  };
+  if (tid == 0) {
+    for (int i = 0; i < 2; ++i) {
+      tc_mbar_init(bar_kv + 8 * i, 4);      // one arrival per decoder warp
+      tc_mbar_init(bar_sfull + 8 * i, 1);   // tcgen05.commit
+      tc_mbar_init(bar_sfree + 8 * i, 4);   // one arrival per row-owner warp
+      tc_mbar_init(bar_pfull + 8 * i, 4);
+      tc_mbar_init(bar_pv + 8 * i, 1);
+    }
+    tc_mbar_init(bar_drain, 1);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (tid < PQ_N_CENTROIDS) {
+    cen_cos[tid] = a.tables->cen_cos[tid];
+    cen_sin[tid] = a.tables->cen_sin[tid];
+  }
+  if (warp == 8) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(sb + kPtSmMisc) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // ---- Q' = (Q S) * scale * log2(e) as fp16 value + residual in the A-operand layout (threads 0..255: column, half of the rows)
+  {
+    float* qs = reinterpret_cast<float*>(smem + kPtSmKv);
+    for (int i = tid; i < kPtRows * 128; i += kPtThreads) {
+      const int r = i >> 7, k = i & 127;
+      float v = 0.f;
+      if (r < n_rows)
+        v = a.io_dtype == PQ_DTYPE_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(a.q)[row_index(r) + k])
+                                        : reinterpret_cast<const float*>(a.q)[row_index(r) + k];
+      qs[i] = v;
+    }
+    __syncthreads();
+    if (tid < 256) {
+      const int j = tid & 127, rh = tid >> 7;
+      float acc[64];
+#pragma unroll
+      for (int r = 0; r < 64; ++r) acc[r] = 0.f;
+      for (int k0 = 0; k0 < 128; k0 += 4) {
+        const float4 w = make_float4(__ldg(a.S + (k0 + 0) * 128 + j), __ldg(a.S + (k0 + 1) * 128 + j),
+                                     __ldg(a.S + (k0 + 2) * 128 + j), __ldg(a.S + (k0 + 3) * 128 + j));
+        pt_rank4(acc, qs + rh * 64 * 128, 128, k0, w);
+      }
+      const float f = a.scale * 1.4426950408889634f;
+      const uint32_t col = (uint32_t)(j >> 6) * 16384u + (uint32_t)(j & 7) * 2u, chunk = (uint32_t)(j & 63) >> 3;
+#pragma unroll
+      for (int r = 0; r < 64; ++r) {
+        const int row = rh * 64 + r;
+        const float v = acc[r] * f;
+        const __half h = __float2half_rn(v);
+        const uint32_t off = col + (uint32_t)row * 128u + ((chunk ^ (uint32_t)(row & 7)) << 4);
+        *reinterpret_cast<__half*>(smem + kPtSmQlo + off) = __float2half_rn(v - __half2float(h));
+        *reinterpret_cast<__half*>(smem + kPtSmQhi + off) = h;
+      }
+    }
+  }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // Q' (generic-proxy writes) -> visible to the MMA unit
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();   // Q' is complete, the float32 copy of q is dead (the stages may be written), tensor memory is allocated
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+  const int vis_cta = max(0, len - (n_q - 1 - (q0 + (n_rows - 1) / g)));   // the CTA's last query sees the most
+  const int n_blocks = (vis_cta + kTokenBlock - 1) / kTokenBlock;
+  const Layout L = make_layout(128, a.pg.page_tokens);
+
+  float l_run = 0.f;   // row owners: denominator of this thread's row
+  if (warp < 4) {
+    // ================= row owners: softmax of row `tid` =================
+    const int r = tid;
+    const int vis = r < n_rows ? max(0, len - (n_q - 1 - (q0 + r / g))) : 0;
+    const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
+    float m_run = -CUDART_INF_F;
+    for (int jb = 0; jb < n_blocks; ++jb) {
+      const int t = jb & 1;
+      const uint32_t ph = (uint32_t)(jb >> 1) & 1u;
+      bool ok = __all_sync(0xffffffffu, tc_mbar_wait(bar_sfull + 8 * t, ph, abort_flag));
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      float s[64];
+      tc_ld32(trow + t * 64, s);
+      tc_ld32(trow + t * 64 + 32, s + 32);
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) tc_mbar_arrive(bar_sfree + 8 * t);   // the scores are in registers: the accumulator may be overwritten
+      float mx = -CUDART_INF_F;
+#pragma unroll
+      for (int i = 0; i < 64; ++i) {
+        s[i] = jb * kTokenBlock + i < vis ? s[i] : -CUDART_INF_F;
+        mx = fmaxf(mx, s[i]);
+      }
+      // lazy reference: move it only when some score exceeds it by more than 8 (p <= 2^8 otherwise)
+      const bool grow = mx > m_run + 8.f || (m_run == -CUDART_INF_F && mx > -CUDART_INF_F);
+      if (__any_sync(0xffffffffu, grow)) {
+        const float m_new = grow ? mx : m_run;
+        const float corr = m_run == -CUDART_INF_F ? 1.f : fast_exp2(m_run - m_new);   // nothing accumulated yet: nothing to scale
+        if (jb > 0) {
+          // the value MMAs up to block jb - 1 must have completed before the accumulator is touched
+          ok = __all_sync(0xffffffffu, tc_mbar_wait(bar_pv + 8 * ((jb - 1) & 1), (uint32_t)((jb - 1) >> 1) & 1u, abort_flag));
+          if (!ok) break;
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+#pragma unroll 1
+          for (int c = 0; c < 4; ++c) {
+            float o[32];
+            tc_ld32(trow + 128 + 32 * c, o);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) o[i] *= corr;
+            tc_st32(trow + 128 + 32 * c, o);
+          }
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        }
+        l_run *= corr;
+        m_run = m_new;
+      }
+      const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;   // nothing visible yet: every p is 0
+      // P buffer t is free once the value MMA of block jb - 2 has completed
+      if (jb >= 2) {
+        ok = __all_sync(0xffffffffu, tc_mbar_wait(bar_pv + 8 * t, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag));
+        if (!ok) break;
+      }
+      uint8_t* prow = smem + kPtSmP + t * kPtPBytes + r * 128;
+      float sum = 0.f;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const __half2 p2 = __floats2half2_rn(fast_exp2(s[8 * c + 2 * e] - m_use), fast_exp2(s[8 * c + 2 * e + 1] - m_use));
+          sum += __low2float(p2) + __high2float(p2);   // the denominator of what the MMA will see
+          w[e] = as_u32(p2);
+        }
+        *reinterpret_cast<uint4*>(prow + ((c ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      l_run += sum;
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) tc_mbar_arrive(bar_pfull + 8 * t);
+    }
+  } else if (warp < 8) {
+    // ================= decoders: packed block -> K_hat hi / lo, V_hat^T =================
+    const int dt = tid - 128, tok = dt & 63, half = dt >> 6;
+    auto fetch = [&](int jb) {  // packed K block and V block of token-block jb -> raw buffer jb & 1
+      const uint8_t* src = a.cache + kv_block_pair_offset(L, a.pg, a.n_kv_heads, b, hk, jb, a.status);
+      const uint32_t dst = sb + kPtSmRaw + (jb & 1) * kPfRawBytes;
+      for (int i = dt; i < kPfRawBytes / 16; i += 128) pf_cp16(dst + 16 * i, src + 16 * i);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    if (n_blocks > 0) fetch(0);
+    for (int jb = 0; jb < n_blocks; ++jb) {
+      const int st = jb & 1;
+      if (jb + 1 < n_blocks) {
+        fetch(jb + 1);
+        asm volatile("cp.async.wait_group 1;" ::: "memory");
+      } else {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+      }
+      // stage st is free once the value MMA of block jb - 2 has completed (it also covers that block's score MMAs)
+      bool ok = true;
+      if (jb >= 2) ok = tc_mbar_wait(bar_pv + 8 * st, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag);
+      // the raw block has landed for all 128 threads; the decision to go on is taken together
+      if (pt_bar_or(1, 128, !ok)) break;
+      const uint8_t* kraw = smem + kPtSmRaw + st * kPfRawBytes;
+      const uint8_t* vraw = kraw + 62 * kTokenBlock;
+      const bool live = jb * kTokenBlock + tok < len;   // stale bytes past the sequence end must not reach the MMAs
+      uint8_t* stage = smem + kPtSmKv + st * kPtStageBytes;
+      uint8_t* khi = stage + half * 8192 + tok * 128;
+      uint8_t* klo = khi + kPtKBytes;
+      uint8_t* vt = stage + 2 * kPtKBytes + (tok & 7) * 2;   // V_hat^T: row = coordinate, the token is the k index
+#pragma unroll 1
+      for (int bi = 0; bi < 4; ++bi) {
+        float y[16];
+        __align__(16) __half h[16], lo[16];
+        decode_block(kraw, L, tok, half * 4 + bi, cen_cos, cen_sin, y);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float v = live ? y[i] : 0.f;
+          h[i] = __float2half_rn(v);
+          lo[i] = __float2half_rn(v - __half2float(h[i]));
+        }
+        const int c0 = ((2 * bi) ^ (tok & 7)) << 4, c1 = ((2 * bi + 1) ^ (tok & 7)) << 4;
+        *reinterpret_cast<uint4*>(khi + c0) = *reinterpret_cast<const uint4*>(h);
+        *reinterpret_cast<uint4*>(khi + c1) = *reinterpret_cast<const uint4*>(h + 8);
+        *reinterpret_cast<uint4*>(klo + c0) = *reinterpret_cast<const uint4*>(lo);
+        *reinterpret_cast<uint4*>(klo + c1) = *reinterpret_cast<const uint4*>(lo + 8);
+        decode_block(vraw, L, tok, half * 4 + bi, cen_cos, cen_sin, y);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int coord = half * 64 + bi * 16 + i;
+          *reinterpret_cast<__half*>(vt + coord * 128 + (((tok >> 3) ^ (coord & 7)) << 4)) = __float2half_rn(live ? y[i] : 0.f);
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) tc_mbar_arrive(bar_kv + 8 * st);
+      // the next iteration starts the copy of block jb + 2 into this iteration's raw buffer: every thread must have
+      // finished reading it
+      asm volatile("bar.sync 2, 128;" ::: "memory");
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+  } else if (tid == 256) {
+    // ================= MMA issuer =================
+    constexpr uint32_t idesc_qk = tc_idesc(false, 128, 64), idesc_pv = tc_idesc(false, 128, 128);
+    const uint64_t desc_hi = tc_smem_desc(0u) & 0xFFFFFFFF00000000ull;
+    const uint32_t qhi_lo = (uint32_t)tc_smem_desc(sb + kPtSmQhi), qlo_lo = (uint32_t)tc_smem_desc(sb + kPtSmQlo);
+    auto issue_pv = [&](int jb) -> bool {   // O (+)= P_jb V_hat_jb
+      const int t = jb & 1;
+      if (!tc_mbar_wait(bar_pfull + 8 * t, (uint32_t)(jb >> 1) & 1u, abort_flag)) return false;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t p_lo = (uint32_t)tc_smem_desc(sb + kPtSmP + t * kPtPBytes);
+      const uint32_t v_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + t * kPtStageBytes + 2 * kPtKBytes);
+#pragma unroll
+      for (int kk = 0; kk < 4; ++kk)
+        tc_mma_idesc(tmem_base + 128, desc_hi | (p_lo + 2 * kk), desc_hi | (v_lo + 2 * kk), idesc_pv, (jb > 0 || kk > 0) ? 1u : 0u);
+      tc_commit(bar_pv + 8 * t);
+      return true;
+    };
+    bool ok = true;
+    for (int jb = 0; jb < n_blocks && ok; ++jb) {
+      const int t = jb & 1;
+      ok = tc_mbar_wait(bar_kv + 8 * t, (uint32_t)(jb >> 1) & 1u, abort_flag);
+      if (ok && jb >= 2) ok = tc_mbar_wait(bar_sfree + 8 * t, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag);
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t khi_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + t * kPtStageBytes);
+      const uint32_t klo_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + t * kPtStageBytes + kPtKBytes);
+      // S = Q'lo K_hi^T + Q'hi K_lo^T + Q'hi K_hi^T (small terms first); k-step ks: half ks >> 2, 32 bytes per step
+#pragma unroll
+      for (int term = 0; term < 3; ++term) {
+        const uint32_t qa = term == 0 ? qlo_lo : qhi_lo, kb = term == 1 ? klo_lo : khi_lo;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+          const uint32_t qoff = (uint32_t)((ks >> 2) * 16384 + (ks & 3) * 32) >> 4, koff = (uint32_t)((ks >> 2) * 8192 + (ks & 3) * 32) >> 4;
+          tc_mma_idesc(tmem_base + t * 64, desc_hi | (qa + qoff), desc_hi | (kb + koff), idesc_qk, (term | ks) ? 1u : 0u);
+        }
+      }
+      tc_commit(bar_sfull + 8 * t);
+      if (jb >= 1) ok = issue_pv(jb - 1);
+    }
+    if (ok && n_blocks > 0) ok = issue_pv(n_blocks - 1);
+    // every MMA issued above has completed when this commit arrives
+    tc_commit(bar_drain);
+    bool drained = false;
+    for (int i = 0; i < (1 << 20) && !drained; ++i) {
+      drained = tc_mbar_try(bar_drain, 0);
+      if (!drained) __nanosleep(32);
+    }
+    if (!drained) *abort_flag = 1;
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();   // all MMAs have completed (the issuer waited for its last commit), the stages are idle
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const bool aborted = *abort_flag != 0;
+  // ---- normalise, un-rotate by S^T, store
+  float* osm = reinterpret_cast<float*>(smem + kPtSmKv);
+  if (warp < 4) {
+    const int r = tid;
+    const float inv = (!aborted && l_run > 0.f) ? 1.f / l_run : 0.f;
+    const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {
+      float o[32];
+      if (n_blocks > 0 && !aborted) {
+        tc_ld32(trow + 128 + 32 * c, o);
+      } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = 0.f;
+      }
+#pragma unroll
+      for (int i = 0; i < 32; i += 4)
+        *reinterpret_cast<float4*>(osm + r * kPtOStride + 32 * c + i) = make_float4(o[i] * inv, o[i + 1] * inv, o[i + 2] * inv, o[i + 3] * inv);
+    }
+    if (r < n_rows && l_run <= 0.f && !aborted) set_status(a.status, PQ_ERR_EMPTY);   // a query that sees no token: zeros
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  }
+  __syncthreads();
+  if (warp == 8) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem_base) : "memory");
+  }
+  if (tid == 0 && aborted) set_status(a.status, PQ_ERR_TIMEOUT);
+  if (tid < 256 && !aborted) {
+    const int i = tid & 127, rh = tid >> 7;   // x_hat_i = sum_j y_hat_j S[i][j]: thread = i, half of the rows
+    float acc[64];
+#pragma unroll
+    for (int r = 0; r < 64; ++r) acc[r] = 0.f;
+    const float4* srow = reinterpret_cast<const float4*>(a.S + i * 128);
+    for (int j0 = 0; j0 < 128; j0 += 4) pt_rank4(acc, osm + rh * 64 * kPtOStride, kPtOStride, j0, __ldg(srow + (j0 >> 2)));
+#pragma unroll 1
+    for (int r = 0; r < 64; ++r) {
+      const int row = rh * 64 + r;
+      if (row < n_rows) {
+        const int64_t o = row_index(row) + i;
+        if (a.io_dtype == PQ_DTYPE_BF16) reinterpret_cast<__nv_bfloat16*>(a.out)[o] = __float2bfloat16(acc[r]);
+        else reinterpret_cast<float*>(a.out)[o] = acc[r];
+      }
+    }
+  }
+}
+
+}  // namespace pq

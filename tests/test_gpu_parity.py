@@ -183,7 +183,9 @@ def test_attention_special_cases_len1_and_identical_keys():
 
 
 @pytest.mark.parametrize("d,Hq,Hkv,n_q", [(128, 8, 2, 5), (128, 8, 1, 3), (16, 4, 2, 4),            # one decode per query
-                                           (128, 8, 2, 40), (128, 8, 1, 9), (128, 6, 2, 22), (128, 2, 2, 70)])  # tensor-core kernel
+                                           (128, 8, 1, 9), (128, 6, 2, 22), (128, 2, 2, 70),      # register-fragment MMA kernel (64..127 rows)
+                                           (128, 8, 2, 40), (128, 8, 1, 20), (128, 6, 2, 50), (128, 2, 2, 150),   # tcgen05 kernel (>= 128 rows)
+                                           (128, 10, 2, 70)])
 def test_multi_query_attention_is_causal_over_the_last_positions(d, Hq, Hkv, n_q):
     """The last n_q positions of every sequence attend at once; query j sees the tokens up to its own position.
     Float32 I/O against the oracle per query, and n_q = 1 equals decode attention bit for bit."""
@@ -213,6 +215,12 @@ def test_multi_query_attention_is_causal_over_the_last_positions(d, Hq, Hkv, n_q
     assert torch.equal(one[:, 0], cache.attend(q[:, -1].contiguous()))
     qb = q.to(torch.bfloat16)
     assert rel_l2(to_f64(cache.attend_multi(qb))[:2], want_bf16(orc, ref, qb, d)[:2]) < TOL_ATTENTION
+    if d == 128 and n_q * (Hq // Hkv) >= 128:
+        # the two tensor-core kernels on the same inputs: the register-fragment one on request
+        pq.pq_debug_fail_next_wait(3)
+        legacy = cache.attend_multi(q)
+        torch.cuda.synchronize()
+        assert rel_l2(to_f64(legacy), got) < 5e-4 and not torch.equal(legacy, out)   # different kernels, same answer
 
 
 def want_bf16(orc, ref, qb, d):
