@@ -2,12 +2,15 @@
 // pq_decode.cu).  Same computation as pq_prefill.cuh -- the last n_q positions of a sequence attend causally to the
 // cached tokens (Eq. 2 / Eq. 3) -- for chunks that fill 128 rows = (128 / g) queries x the g query heads of a kv head.
 //
-// One CTA of nine warps per (query block, kv head, sequence) loops over the 64-token blocks its queries may see:
-//   * warps 4-7 ("decoders") copy the packed K and V block with cp.async, DeQuant it (Algorithm 1, float32 from
-//     the 28 centroids: a thread decodes half a token) and write the tensor-core operands into shared memory in
-//     the K-major 128-byte-swizzled layout: K_hat as fp16 value + fp16 residual [token][coordinate], V_hat
-//     transposed [coordinate][token]; two stages, so block j + 1 is decoded while block j is multiplied;
-//   * one thread of warp 8 issues the MMAs: S_j = Q' K_hat^T as three products (lo*hi, hi*lo, hi*hi; M = 128,
+// One CTA of thirteen warps per (query block, kv head, sequence) loops over the 64-token blocks its queries may see:
+//   * warps 4-11 ("decoders") copy the packed K and V block with cp.async, DeQuant it (Algorithm 1 by the table
+//     lookups of the decode kernel: per 4-coordinate sub-block one entry for levels 4-2 and one for the two level-1
+//     pairs, fp16 with error-free residuals; a thread decodes a quarter of a token) and write the tensor-core operands into
+//     shared memory in the K-major 128-byte-swizzled layout: K_hat as fp16 value + fp16 residual
+//     [token][coordinate], V_hat transposed [coordinate][token]; two stages, so block j + 1 is decoded while block j
+//     is multiplied.  The lookups deliver coordinates (4s, 4s+2 | 4s+1, 4s+3); K_hat keeps that order and Q' is stored
+//     in the same one (the contraction does not care), V_hat^T has the coordinate as its row index and needs none;
+//   * one thread of warp 12 issues the MMAs: S_j = Q' K_hat^T as three products (lo*hi, hi*lo, hi*hi; M = 128,
 //     N = 64, eight k-steps each) into one of two 64-column accumulators in tensor memory, and O += P_j V_hat
 //     (M = 128, N = 128, four k-steps) into a 128-column accumulator; the tensor core reads every operand from
 //     shared memory itself, so no warp re-reads a tile (the register-fragment kernel spends 70 % of the
@@ -28,7 +31,8 @@
 
 namespace pq {
 
-constexpr int kPtThreads = 288;
+constexpr int kPtThreads = 416;   // warps 0-3 row owners, 4-11 decoders, 12 the MMA issuer
+constexpr int kPtDecoders = 256;
 constexpr int kPtRows = 128;
 constexpr int kPtQBytes = 128 * 128 * 2;            // Q' hi or lo: two k-halves of 128 rows x 128 bytes
 constexpr int kPtKBytes = 64 * 128 * 2;             // K_hat hi or lo of a block: two k-halves of 64 tokens x 128 bytes
@@ -39,8 +43,8 @@ constexpr int kPtSmQhi = 0, kPtSmQlo = kPtSmQhi + kPtQBytes;
 constexpr int kPtSmKv = kPtSmQlo + kPtQBytes;       // two stages; also q in float32 at the start and O at the end
 constexpr int kPtSmP = kPtSmKv + 2 * kPtStageBytes; // two buffers
 constexpr int kPtSmRaw = kPtSmP + 2 * kPtPBytes;    // two packed (K block, V block) buffers
-constexpr int kPtSmTab = kPtSmRaw + 2 * kPfRawBytes;
-constexpr int kPtSmBar = kPtSmTab + 256;            // kv_full[2], s_full[2], s_free[2], p_full[2], pv_done[2], drain
+constexpr int kPtSmTab = kPtSmRaw + 2 * kPfRawBytes;   // u_tab[4][64], t1p_hi[256], t1p_lo[256] of Tables (8 bytes per entry)
+constexpr int kPtSmBar = kPtSmTab + 6144;           // kv_full[2], s_full[2], s_free[2], p_full[2], pv_done[2], drain
 constexpr int kPtSmMisc = kPtSmBar + 96;            // tensor-memory base, abort flag
 constexpr int kPtSmTotal = kPtSmMisc + 32 + 1024;   // + slack for 1024-byte alignment
 constexpr int kPtOStride = 132;                     // floats per row of the output staging
@@ -83,8 +87,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
   const int len = a.lens[b];
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kPtSmMisc + 4);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kPtSmMisc);
-  float* cen_cos = reinterpret_cast<float*>(smem + kPtSmTab);
-  float* cen_sin = cen_cos + 32;
+  uint2* tab = reinterpret_cast<uint2*>(smem + kPtSmTab);
   const uint32_t bar_kv = sb + kPtSmBar, bar_sfull = bar_kv + 16, bar_sfree = bar_kv + 32, bar_pfull = bar_kv + 48,
                  bar_pv = bar_kv + 64, bar_drain = bar_kv + 80;
   auto row_index = [&](int r) -> int64_t {               // offset of row r in q / out ([batch][n_q][n_q_heads][128])
@@ -92,7 +95,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
   };
   if (tid == 0) {
     for (int i = 0; i < 2; ++i) {
-      tc_mbar_init(bar_kv + 8 * i, 4);      // one arrival per decoder warp
+      tc_mbar_init(bar_kv + 8 * i, kPtDecoders / 32);   // one arrival per decoder warp
       tc_mbar_init(bar_sfull + 8 * i, 1);   // tcgen05.commit
       tc_mbar_init(bar_sfree + 8 * i, 4);   // one arrival per row-owner warp
       tc_mbar_init(bar_pfull + 8 * i, 4);
@@ -102,11 +105,9 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (tid < PQ_N_CENTROIDS) {
-    cen_cos[tid] = a.tables->cen_cos[tid];
-    cen_sin[tid] = a.tables->cen_sin[tid];
-  }
-  if (warp == 8) {
+  for (int i = tid; i < 768; i += kPtThreads)
+    tab[i] = i < 256 ? a.tables->u_tab[i >> 6][i & 63] : (i < 512 ? a.tables->t1p_hi[i - 256] : a.tables->t1p_lo[i - 512]);
+  if (warp == 12) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(sb + kPtSmMisc) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -133,7 +134,9 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
         pt_rank4(acc, qs + rh * 64 * 128, 128, k0, w);
       }
       const float f = a.scale * 1.4426950408889634f;
-      const uint32_t col = (uint32_t)(j >> 6) * 16384u + (uint32_t)(j & 7) * 2u, chunk = (uint32_t)(j & 63) >> 3;
+      // coordinate j sits at position (j & ~3) | (0, 2, 1, 3)[j & 3] of the contraction index: the order the decoders write
+      const int jp = (j & ~3) | ((j & 1) << 1) | ((j >> 1) & 1);
+      const uint32_t col = (uint32_t)(jp >> 6) * 16384u + (uint32_t)(jp & 7) * 2u, chunk = (uint32_t)(jp & 63) >> 3;
 #pragma unroll
       for (int r = 0; r < 64; ++r) {
         const int row = rh * 64 + r;
@@ -227,13 +230,13 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       __syncwarp();
       if (lane == 0) tc_mbar_arrive(bar_pfull + 8 * t);
     }
-  } else if (warp < 8) {
+  } else if (warp < 12) {
     // ================= decoders: packed block -> K_hat hi / lo, V_hat^T =================
-    const int dt = tid - 128, tok = dt & 63, half = dt >> 6;
+    const int dt = tid - 128, tok = dt & 63, quarter = dt >> 6, half = quarter >> 1;
     auto fetch = [&](int jb) {  // packed K block and V block of token-block jb -> raw buffer jb & 1
       const uint8_t* src = a.cache + kv_block_pair_offset(L, a.pg, a.n_kv_heads, b, hk, jb, a.status);
       const uint32_t dst = sb + kPtSmRaw + (jb & 1) * kPfRawBytes;
-      for (int i = dt; i < kPfRawBytes / 16; i += 128) pf_cp16(dst + 16 * i, src + 16 * i);
+      for (int i = dt; i < kPfRawBytes / 16; i += kPtDecoders) pf_cp16(dst + 16 * i, src + 16 * i);
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
     if (n_blocks > 0) fetch(0);
@@ -248,8 +251,8 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       // stage st is free once the value MMA of block jb - 2 has completed (it also covers that block's score MMAs)
       bool ok = true;
       if (jb >= 2) ok = tc_mbar_wait(bar_pv + 8 * st, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag);
-      // the raw block has landed for all 128 threads; the decision to go on is taken together
-      if (pt_bar_or(1, 128, !ok)) break;
+      // the raw block has landed for all decoder threads; the decision to go on is taken together
+      if (pt_bar_or(1, kPtDecoders, !ok)) break;
       const uint8_t* kraw = smem + kPtSmRaw + st * kPfRawBytes;
       const uint8_t* vraw = kraw + 62 * kTokenBlock;
       const bool live = jb * kTokenBlock + tok < len;   // stale bytes past the sequence end must not reach the MMAs
@@ -257,27 +260,57 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       uint8_t* khi = stage + half * 8192 + tok * 128;
       uint8_t* klo = khi + kPtKBytes;
       uint8_t* vt = stage + 2 * kPtKBytes + (tok & 7) * 2;   // V_hat^T: row = coordinate, the token is the k index
+      const uint2* utab = tab;
+      const uint2* t1hi = tab + 256;
+      const uint2* t1lo = tab + 512;
 #pragma unroll 1
-      for (int bi = 0; bi < 4; ++bi) {
-        float y[16];
-        __align__(16) __half h[16], lo[16];
-        decode_block(kraw, L, tok, half * 4 + bi, cen_cos, cen_sin, y);
+      for (int bi = 2 * (quarter & 1); bi < 2 * (quarter & 1) + 2; ++bi) {   // block half * 4 + bi of the token
+        const int blk = half * 4 + bi;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const float v = live ? y[i] : 0.f;
-          h[i] = __float2half_rn(v);
-          lo[i] = __float2half_rn(v - __half2float(h[i]));
-        }
-        const int c0 = ((2 * bi) ^ (tok & 7)) << 4, c1 = ((2 * bi + 1) ^ (tok & 7)) << 4;
-        *reinterpret_cast<uint4*>(khi + c0) = *reinterpret_cast<const uint4*>(h);
-        *reinterpret_cast<uint4*>(khi + c1) = *reinterpret_cast<const uint4*>(h + 8);
-        *reinterpret_cast<uint4*>(klo + c0) = *reinterpret_cast<const uint4*>(lo);
-        *reinterpret_cast<uint4*>(klo + c1) = *reinterpret_cast<const uint4*>(lo + 8);
-        decode_block(vraw, L, tok, half * 4 + bi, cen_cos, cen_sin, y);
+        for (int kv = 0; kv < 2; ++kv) {
+          const uint8_t* raw = kv ? vraw : kraw;
+          const uint32_t l1 = *reinterpret_cast<const uint32_t*>(raw + tok * 32 + blk * 4);
+          const uint32_t c2 = raw[kO2 + tok * 8 + blk];
+          const uint32_t c3 = (uint32_t)raw[kO3 + tok * 4 + (blk >> 1)] >> (4 * (blk & 1));
+          const uint32_t c4 = ((uint32_t)*reinterpret_cast<const uint16_t*>(raw + kO4 + tok * 2) >> (2 * blk)) & 3u;
+          const uint32_t rbits = live ? (uint32_t)*reinterpret_cast<const uint16_t*>(raw + kORad + tok * 16 + blk * 2) : 0u;
+          const __half2 r2 = as_h2(rbits | (rbits << 16));
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int coord = half * 64 + bi * 16 + i;
-          *reinterpret_cast<__half*>(vt + coord * 128 + (((tok >> 3) ^ (coord & 7)) << 4)) = __float2half_rn(live ? y[i] : 0.f);
+          for (int sp = 0; sp < 2; ++sp) {   // two sub-blocks = eight coordinates = one 16-byte chunk of the key row
+            uint32_t hw[4], lw[4];
+#pragma unroll
+            for (int q = 0; q < 2; ++q) {
+              const int sb4 = 2 * sp + q;    // sub-block: coordinates 4 sb4 .. 4 sb4 + 3 of the block
+              const uint32_t iu = ((c2 >> (2 * sb4)) & 3u) | (((c3 >> (2 * sp)) & 3u) << 2) | (c4 << 4);
+              const uint2 uu = utab[sb4 * 64 + iu];
+              const uint32_t e = (l1 >> (8 * sb4)) & 0xFFu;
+              const uint2 th = t1hi[e];
+              const __half2 u_hi = __hmul2(r2, as_h2(uu.x));
+              const __half2 xh = __hmul2(u_hi, as_h2(th.x)), yh = __hmul2(u_hi, as_h2(th.y));   // coordinates (4s, 4s+2), (4s+1, 4s+3)
+              if (kv == 0) {
+                // the key as an unevaluated sum hi + lo (fp16 fused multiply-adds return the exact residual of a product)
+                const uint2 tl = t1lo[e];
+                const __half2 u_lo = __hfma2(r2, as_h2(uu.y), __hfma2(r2, as_h2(uu.x), __hneg2(u_hi)));
+                hw[2 * q] = as_u32(xh);
+                hw[2 * q + 1] = as_u32(yh);
+                lw[2 * q] = as_u32(__hfma2(u_hi, as_h2(tl.x), __hfma2(u_lo, as_h2(th.x), __hfma2(u_hi, as_h2(th.x), __hneg2(xh)))));
+                lw[2 * q + 1] = as_u32(__hfma2(u_hi, as_h2(tl.y), __hfma2(u_lo, as_h2(th.y), __hfma2(u_hi, as_h2(th.y), __hneg2(yh)))));
+              } else {
+                const int coord = half * 64 + bi * 16 + 4 * sb4;
+                uint8_t* vrow = vt + coord * 128;
+                const int ch = tok >> 3;
+                *reinterpret_cast<__half*>(vrow + ((ch ^ (coord & 7)) << 4)) = __low2half(xh);
+                *reinterpret_cast<__half*>(vrow + 128 + ((ch ^ ((coord + 1) & 7)) << 4)) = __low2half(yh);
+                *reinterpret_cast<__half*>(vrow + 256 + ((ch ^ ((coord + 2) & 7)) << 4)) = __high2half(xh);
+                *reinterpret_cast<__half*>(vrow + 384 + ((ch ^ ((coord + 3) & 7)) << 4)) = __high2half(yh);
+              }
+            }
+            if (kv == 0) {
+              const int c = ((2 * bi + sp) ^ (tok & 7)) << 4;
+              *reinterpret_cast<uint4*>(khi + c) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
+              *reinterpret_cast<uint4*>(klo + c) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+            }
+          }
         }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -285,10 +318,10 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       if (lane == 0) tc_mbar_arrive(bar_kv + 8 * st);
       // the next iteration starts the copy of block jb + 2 into this iteration's raw buffer: every thread must have
       // finished reading it
-      asm volatile("bar.sync 2, 128;" ::: "memory");
+      asm volatile("bar.sync 2, %0;" ::"n"(kPtDecoders) : "memory");
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-  } else if (tid == 256) {
+  } else if (tid == 384) {
     // ================= MMA issuer =================
     constexpr uint32_t idesc_qk = tc_idesc(false, 128, 64), idesc_pv = tc_idesc(false, 128, 128);
     const uint64_t desc_hi = tc_smem_desc(0u) & 0xFFFFFFFF00000000ull;
@@ -308,6 +341,15 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     bool ok = true;
     for (int jb = 0; jb < n_blocks && ok; ++jb) {
       const int t = jb & 1;
+      // The value MMA of the previous block frees its stage for the decoders: it goes first if its P is ready, so that
+      // it does not queue behind this block's score MMAs; otherwise the score MMAs go first and keep the tensor
+      // core busy while the softmax of the previous block finishes.
+      bool pv_issued = jb == 0;
+      if (!pv_issued && tc_mbar_test(bar_pfull + 8 * ((jb - 1) & 1), (uint32_t)((jb - 1) >> 1) & 1u)) {
+        ok = issue_pv(jb - 1);
+        pv_issued = true;
+        if (!ok) break;
+      }
       ok = tc_mbar_wait(bar_kv + 8 * t, (uint32_t)(jb >> 1) & 1u, abort_flag);
       if (ok && jb >= 2) ok = tc_mbar_wait(bar_sfree + 8 * t, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag);
       if (!ok) break;
@@ -325,17 +367,19 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
         }
       }
       tc_commit(bar_sfull + 8 * t);
-      if (jb >= 1) ok = issue_pv(jb - 1);
+      if (!pv_issued) ok = issue_pv(jb - 1);
     }
     if (ok && n_blocks > 0) ok = issue_pv(n_blocks - 1);
-    // every MMA issued above has completed when this commit arrives
-    tc_commit(bar_drain);
-    bool drained = false;
-    for (int i = 0; i < (1 << 20) && !drained; ++i) {
-      drained = tc_mbar_try(bar_drain, 0);
-      if (!drained) __nanosleep(32);
+    if (n_blocks > 0) {
+      // every MMA issued above has completed when this commit arrives (nothing was issued without blocks: no commit)
+      tc_commit(bar_drain);
+      bool drained = false;
+      for (int i = 0; i < (1 << 20) && !drained; ++i) {
+        drained = tc_mbar_try(bar_drain, 0);
+        if (!drained) __nanosleep(32);
+      }
+      if (!drained) *abort_flag = 1;
     }
-    if (!drained) *abort_flag = 1;
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();   // all MMAs have completed (the issuer waited for its last commit), the stages are idle
@@ -364,7 +408,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
   __syncthreads();
-  if (warp == 8) {
+  if (warp == 12) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem_base) : "memory");
   }
@@ -376,7 +420,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     for (int r = 0; r < 64; ++r) acc[r] = 0.f;
     const float4* srow = reinterpret_cast<const float4*>(a.S + i * 128);
     for (int j0 = 0; j0 < 128; j0 += 4) pt_rank4(acc, osm + rh * 64 * kPtOStride, kPtOStride, j0, __ldg(srow + (j0 >> 2)));
-#pragma unroll 1
+#pragma unroll
     for (int r = 0; r < 64; ++r) {
       const int row = rh * 64 + r;
       if (row < n_rows) {
