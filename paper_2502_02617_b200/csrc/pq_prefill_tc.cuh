@@ -12,12 +12,13 @@
 //     in the same one (the contraction does not care), V_hat^T has the coordinate as its row index and needs none;
 //   * one thread of warp 12 issues the MMAs: S_j = Q' K_hat^T as three products (lo*hi, hi*lo, hi*hi; M = 128,
 //     N = 64, eight k-steps each) into one of two 64-column accumulators in tensor memory, and O += P_j V_hat
-//     (M = 128, N = 128, four k-steps) into a 128-column accumulator; the tensor core reads every operand from
-//     shared memory itself, so no warp re-reads a tile (the register-fragment kernel spends 70 % of the
-//     shared-memory pipe on exactly that);
+//     (M = 128, N = 128, four k-steps) into a 128-column accumulator.  The A operands live in tensor memory too
+//     (Q' hi and lo, written once; P_j, written by the row owners), the B operands are read from shared memory by
+//     the tensor core itself: no warp re-reads a tile (the register-fragment kernel spends 70 % of the
+//     shared-memory pipe on exactly that), and shared memory is left for a ring of four decoded stages;
 //   * warps 0-3 ("row owners": tensor-memory lane = row = thread) read S_j with tcgen05.ld, apply the causal mask
 //     and the online softmax in the log2 domain without any shuffle (a thread owns its whole row), and write P_j
-//     in fp16 as the A operand of the value MMA.  The running maximum is updated lazily: only when a score exceeds
+//     in fp16 into tensor memory as the A operand of the value MMA.  The running maximum is updated lazily: only when a score exceeds
 //     it by more than 8 is the output accumulator rescaled (tcgen05.ld / multiply / tcgen05.st by the row's owner,
 //     after the previous value MMA has completed); otherwise p <= 2^8 stays well inside fp16.
 // Q' = (Q S) * scale * log2 e is formed once per CTA in float32 and kept as fp16 value + residual; the output is
@@ -34,23 +35,24 @@ namespace pq {
 constexpr int kPtThreads = 416;   // warps 0-3 row owners, 4-11 decoders, 12 the MMA issuer
 constexpr int kPtDecoders = 256;
 constexpr int kPtRows = 128;
-constexpr int kPtQBytes = 128 * 128 * 2;            // Q' hi or lo: two k-halves of 128 rows x 128 bytes
+constexpr int kPtStages = 4;                        // decoded (K_hat hi, K_hat lo, V_hat^T) blocks in flight
 constexpr int kPtKBytes = 64 * 128 * 2;             // K_hat hi or lo of a block: two k-halves of 64 tokens x 128 bytes
 constexpr int kPtVBytes = 128 * 64 * 2;             // V_hat^T of a block: 128 coordinates x 64 tokens
-constexpr int kPtPBytes = 128 * 64 * 2;             // P of a block: 128 rows x 64 tokens
 constexpr int kPtStageBytes = 2 * kPtKBytes + kPtVBytes;
-constexpr int kPtSmQhi = 0, kPtSmQlo = kPtSmQhi + kPtQBytes;
-constexpr int kPtSmKv = kPtSmQlo + kPtQBytes;       // two stages; also q in float32 at the start and O at the end
-constexpr int kPtSmP = kPtSmKv + 2 * kPtStageBytes; // two buffers
-constexpr int kPtSmRaw = kPtSmP + 2 * kPtPBytes;    // two packed (K block, V block) buffers
+constexpr int kPtSmKv = 0;                          // the stages; also q, Q' at the start and O at the end
+constexpr int kPtSmRaw = kPtSmKv + kPtStages * kPtStageBytes;   // two packed (K block, V block) buffers
 constexpr int kPtSmTab = kPtSmRaw + 2 * kPfRawBytes;   // u_tab[4][64], t1p_hi[256], t1p_lo[256] of Tables (8 bytes per entry)
-constexpr int kPtSmBar = kPtSmTab + 6144;           // kv_full[2], s_full[2], s_free[2], p_full[2], pv_done[2], drain
-constexpr int kPtSmMisc = kPtSmBar + 96;            // tensor-memory base, abort flag
+constexpr int kPtSmBar = kPtSmTab + 6144;           // kv_full[S], pv_done[S], s_full[2], s_free[2], p_full[2], p_free[2], drain
+constexpr int kPtSmMisc = kPtSmBar + 16 * kPtStages + 80;   // tensor-memory base, abort flag
 constexpr int kPtSmTotal = kPtSmMisc + 32 + 1024;   // + slack for 1024-byte alignment
 constexpr int kPtOStride = 132;                     // floats per row of the output staging
+constexpr int kPtQStride = 136;                     // halves per row of the Q' staging (rows 16 bytes apart mod 128)
+// tensor-memory columns: two score accumulators, the output accumulator, Q' hi and lo (two fp16 per column), two P buffers
+constexpr uint32_t kPtTmS = 0, kPtTmO = 128, kPtTmQhi = 256, kPtTmQlo = 320, kPtTmP = 384;
 static_assert(kPtSmTotal <= 227 * 1024, "shared memory of one CTA");
-static_assert(128 * kPtOStride * 4 <= 2 * kPtStageBytes && 128 * 128 * 4 <= 2 * kPtStageBytes, "float32 staging fits in the stages");
-static_assert(kPtSmKv % 1024 == 0 && kPtStageBytes % 1024 == 0 && kPtSmP % 1024 == 0, "swizzled tiles start on 1024-byte boundaries");
+static_assert(128 * kPtOStride * 4 <= kPtStages * kPtStageBytes, "float32 output staging fits in the stages");
+static_assert(128 * 128 * 4 + 2 * 128 * kPtQStride * 2 <= kPtStages * kPtStageBytes, "q and Q' staging fit in the stages");
+static_assert(kPtStageBytes % 1024 == 0, "swizzled tiles start on 1024-byte boundaries");
 
 // acc[r] += sum_k x[r][k0 + k] * w[k] for 64 rows of a float32 tile in shared memory (the same address in every thread)
 __device__ __forceinline__ void pt_rank4(float (&acc)[64], const float* x, int ld, int k0, float4 w) {
@@ -88,18 +90,21 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kPtSmMisc + 4);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kPtSmMisc);
   uint2* tab = reinterpret_cast<uint2*>(smem + kPtSmTab);
-  const uint32_t bar_kv = sb + kPtSmBar, bar_sfull = bar_kv + 16, bar_sfree = bar_kv + 32, bar_pfull = bar_kv + 48,
-                 bar_pv = bar_kv + 64, bar_drain = bar_kv + 80;
+  const uint32_t bar_kv = sb + kPtSmBar, bar_pv = bar_kv + 8 * kPtStages, bar_sfull = bar_pv + 8 * kPtStages,
+                 bar_sfree = bar_sfull + 16, bar_pfull = bar_sfree + 16, bar_pfree = bar_pfull + 16, bar_drain = bar_pfree + 16;
   auto row_index = [&](int r) -> int64_t {               // offset of row r in q / out ([batch][n_q][n_q_heads][128])
     return (((int64_t)b * n_q + q0 + r / g) * a.n_q_heads + hk * g + r % g) * 128;
   };
   if (tid == 0) {
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < kPtStages; ++i) {
       tc_mbar_init(bar_kv + 8 * i, kPtDecoders / 32);   // one arrival per decoder warp
+      tc_mbar_init(bar_pv + 8 * i, 1);                  // tcgen05.commit after the value MMA that read the stage
+    }
+    for (int i = 0; i < 2; ++i) {
       tc_mbar_init(bar_sfull + 8 * i, 1);   // tcgen05.commit
       tc_mbar_init(bar_sfree + 8 * i, 4);   // one arrival per row-owner warp
       tc_mbar_init(bar_pfull + 8 * i, 4);
-      tc_mbar_init(bar_pv + 8 * i, 1);
+      tc_mbar_init(bar_pfree + 8 * i, 1);   // tcgen05.commit after the value MMA that read the P buffer
     }
     tc_mbar_init(bar_drain, 1);
     *abort_flag = 0;
@@ -108,10 +113,13 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
   for (int i = tid; i < 768; i += kPtThreads)
     tab[i] = i < 256 ? a.tables->u_tab[i >> 6][i & 63] : (i < 512 ? a.tables->t1p_hi[i - 256] : a.tables->t1p_lo[i - 512]);
   if (warp == 12) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 256;" ::"r"(sb + kPtSmMisc) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(sb + kPtSmMisc) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // ---- Q' = (Q S) * scale * log2(e) as fp16 value + residual in the A-operand layout (threads 0..255: column, half of the rows)
+  // ---- Q' = (Q S) * scale * log2(e) as fp16 value + residual (threads 0..255: column, half of the rows), staged in shared
+  // memory and then written to tensor memory by the row owners (lane = row, two k values per column)
+  __half* qhi_s = reinterpret_cast<__half*>(smem + kPtSmKv + 128 * 128 * 4);
+  __half* qlo_s = qhi_s + 128 * kPtQStride;
   {
     float* qs = reinterpret_cast<float*>(smem + kPtSmKv);
     for (int i = tid; i < kPtRows * 128; i += kPtThreads) {
@@ -136,23 +144,37 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       const float f = a.scale * 1.4426950408889634f;
       // coordinate j sits at position (j & ~3) | (0, 2, 1, 3)[j & 3] of the contraction index: the order the decoders write
       const int jp = (j & ~3) | ((j & 1) << 1) | ((j >> 1) & 1);
-      const uint32_t col = (uint32_t)(jp >> 6) * 16384u + (uint32_t)(jp & 7) * 2u, chunk = (uint32_t)(jp & 63) >> 3;
 #pragma unroll
       for (int r = 0; r < 64; ++r) {
         const int row = rh * 64 + r;
         const float v = acc[r] * f;
         const __half h = __float2half_rn(v);
-        const uint32_t off = col + (uint32_t)row * 128u + ((chunk ^ (uint32_t)(row & 7)) << 4);
-        *reinterpret_cast<__half*>(smem + kPtSmQlo + off) = __float2half_rn(v - __half2float(h));
-        *reinterpret_cast<__half*>(smem + kPtSmQhi + off) = h;
+        qhi_s[row * kPtQStride + jp] = h;
+        qlo_s[row * kPtQStride + jp] = __float2half_rn(v - __half2float(h));
       }
     }
   }
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // Q' (generic-proxy writes) -> visible to the MMA unit
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();   // Q' is complete, the float32 copy of q is dead (the stages may be written), tensor memory is allocated
+  __syncthreads();   // Q' is staged, tensor memory is allocated
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
+  if (warp < 4) {
+    const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
+#pragma unroll 1
+    for (int c = 0; c < 4; ++c) {   // hi columns 0..31, 32..63, then lo
+      const uint4* src = reinterpret_cast<const uint4*>((c < 2 ? qhi_s : qlo_s) + tid * kPtQStride + 64 * (c & 1));
+      uint32_t v[32];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const uint4 w = src[i];
+        v[4 * i] = w.x; v[4 * i + 1] = w.y; v[4 * i + 2] = w.z; v[4 * i + 3] = w.w;
+      }
+      tc_st32u(trow + (c < 2 ? kPtTmQhi : kPtTmQlo) + 32 * (c & 1), v);
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  }
+  __syncthreads();   // Q' is in tensor memory; the staging is dead: the stages may be written
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const int vis_cta = max(0, len - (n_q - 1 - (q0 + (n_rows - 1) / g)));   // the CTA's last query sees the most
   const int n_blocks = (vis_cta + kTokenBlock - 1) / kTokenBlock;
   const Layout L = make_layout(128, a.pg.page_tokens);
@@ -189,16 +211,16 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
         const float corr = m_run == -CUDART_INF_F ? 1.f : fast_exp2(m_run - m_new);   // nothing accumulated yet: nothing to scale
         if (jb > 0) {
           // the value MMAs up to block jb - 1 must have completed before the accumulator is touched
-          ok = __all_sync(0xffffffffu, tc_mbar_wait(bar_pv + 8 * ((jb - 1) & 1), (uint32_t)((jb - 1) >> 1) & 1u, abort_flag));
+          ok = __all_sync(0xffffffffu, tc_mbar_wait(bar_pfree + 8 * ((jb - 1) & 1), (uint32_t)((jb - 1) >> 1) & 1u, abort_flag));
           if (!ok) break;
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
 #pragma unroll 1
           for (int c = 0; c < 4; ++c) {
             float o[32];
-            tc_ld32(trow + 128 + 32 * c, o);
+            tc_ld32(trow + kPtTmO + 32 * c, o);
 #pragma unroll
             for (int i = 0; i < 32; ++i) o[i] *= corr;
-            tc_st32(trow + 128 + 32 * c, o);
+            tc_st32(trow + kPtTmO + 32 * c, o);
           }
           asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
         }
@@ -208,24 +230,19 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;   // nothing visible yet: every p is 0
       // P buffer t is free once the value MMA of block jb - 2 has completed
       if (jb >= 2) {
-        ok = __all_sync(0xffffffffu, tc_mbar_wait(bar_pv + 8 * t, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag));
+        ok = __all_sync(0xffffffffu, tc_mbar_wait(bar_pfree + 8 * t, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag));
         if (!ok) break;
       }
-      uint8_t* prow = smem + kPtSmP + t * kPtPBytes + r * 128;
       float sum = 0.f;
+      uint32_t pw[32];
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
-        uint32_t w[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const __half2 p2 = __floats2half2_rn(fast_exp2(s[8 * c + 2 * e] - m_use), fast_exp2(s[8 * c + 2 * e + 1] - m_use));
-          sum += __low2float(p2) + __high2float(p2);   // the denominator of what the MMA will see
-          w[e] = as_u32(p2);
-        }
-        *reinterpret_cast<uint4*>(prow + ((c ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+      for (int e = 0; e < 32; ++e) {
+        const __half2 p2 = __floats2half2_rn(fast_exp2(s[2 * e] - m_use), fast_exp2(s[2 * e + 1] - m_use));
+        sum += __low2float(p2) + __high2float(p2);   // the denominator of what the MMA will see
+        pw[e] = as_u32(p2);
       }
       l_run += sum;
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      tc_st32u(trow + kPtTmP + 32 * t, pw);
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) tc_mbar_arrive(bar_pfull + 8 * t);
@@ -241,19 +258,19 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     };
     if (n_blocks > 0) fetch(0);
     for (int jb = 0; jb < n_blocks; ++jb) {
-      const int st = jb & 1;
+      const int st = jb % kPtStages;
       if (jb + 1 < n_blocks) {
         fetch(jb + 1);
         asm volatile("cp.async.wait_group 1;" ::: "memory");
       } else {
         asm volatile("cp.async.wait_group 0;" ::: "memory");
       }
-      // stage st is free once the value MMA of block jb - 2 has completed (it also covers that block's score MMAs)
+      // stage st is free once the value MMA of block jb - kPtStages has completed (it also covers that block's score MMAs)
       bool ok = true;
-      if (jb >= 2) ok = tc_mbar_wait(bar_pv + 8 * st, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag);
+      if (jb >= kPtStages) ok = tc_mbar_wait(bar_pv + 8 * st, (uint32_t)(jb / kPtStages - 1) & 1u, abort_flag);
       // the raw block has landed for all decoder threads; the decision to go on is taken together
       if (pt_bar_or(1, kPtDecoders, !ok)) break;
-      const uint8_t* kraw = smem + kPtSmRaw + st * kPfRawBytes;
+      const uint8_t* kraw = smem + kPtSmRaw + (jb & 1) * kPfRawBytes;
       const uint8_t* vraw = kraw + 62 * kTokenBlock;
       const bool live = jb * kTokenBlock + tok < len;   // stale bytes past the sequence end must not reach the MMAs
       uint8_t* stage = smem + kPtSmKv + st * kPtStageBytes;
@@ -325,17 +342,16 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     // ================= MMA issuer =================
     constexpr uint32_t idesc_qk = tc_idesc(false, 128, 64), idesc_pv = tc_idesc(false, 128, 128);
     const uint64_t desc_hi = tc_smem_desc(0u) & 0xFFFFFFFF00000000ull;
-    const uint32_t qhi_lo = (uint32_t)tc_smem_desc(sb + kPtSmQhi), qlo_lo = (uint32_t)tc_smem_desc(sb + kPtSmQlo);
     auto issue_pv = [&](int jb) -> bool {   // O (+)= P_jb V_hat_jb
-      const int t = jb & 1;
+      const int t = jb & 1, st = jb % kPtStages;
       if (!tc_mbar_wait(bar_pfull + 8 * t, (uint32_t)(jb >> 1) & 1u, abort_flag)) return false;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t p_lo = (uint32_t)tc_smem_desc(sb + kPtSmP + t * kPtPBytes);
-      const uint32_t v_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + t * kPtStageBytes + 2 * kPtKBytes);
+      const uint32_t v_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + st * kPtStageBytes + 2 * kPtKBytes);
 #pragma unroll
-      for (int kk = 0; kk < 4; ++kk)
-        tc_mma_idesc(tmem_base + 128, desc_hi | (p_lo + 2 * kk), desc_hi | (v_lo + 2 * kk), idesc_pv, (jb > 0 || kk > 0) ? 1u : 0u);
-      tc_commit(bar_pv + 8 * t);
+      for (int kk = 0; kk < 4; ++kk)   // 16 tokens = 8 columns of P per step
+        tc_mma_ts(tmem_base + kPtTmO, tmem_base + kPtTmP + 32 * t + 8 * kk, desc_hi | (v_lo + 2 * kk), idesc_pv, (jb > 0 || kk > 0) ? 1u : 0u);
+      tc_commit(bar_pv + 8 * st);     // the stage is free
+      tc_commit(bar_pfree + 8 * t);   // and so is the P buffer; the output accumulator holds block jb
       return true;
     };
     bool ok = true;
@@ -350,20 +366,21 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
         pv_issued = true;
         if (!ok) break;
       }
-      ok = tc_mbar_wait(bar_kv + 8 * t, (uint32_t)(jb >> 1) & 1u, abort_flag);
+      const int st = jb % kPtStages;
+      ok = tc_mbar_wait(bar_kv + 8 * st, (uint32_t)(jb / kPtStages) & 1u, abort_flag);
       if (ok && jb >= 2) ok = tc_mbar_wait(bar_sfree + 8 * t, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag);
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t khi_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + t * kPtStageBytes);
-      const uint32_t klo_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + t * kPtStageBytes + kPtKBytes);
+      const uint32_t khi_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + st * kPtStageBytes);
+      const uint32_t klo_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + st * kPtStageBytes + kPtKBytes);
       // S = Q'lo K_hi^T + Q'hi K_lo^T + Q'hi K_hi^T (small terms first); k-step ks: half ks >> 2, 32 bytes per step
 #pragma unroll
       for (int term = 0; term < 3; ++term) {
-        const uint32_t qa = term == 0 ? qlo_lo : qhi_lo, kb = term == 1 ? klo_lo : khi_lo;
+        const uint32_t qa = tmem_base + (term == 0 ? kPtTmQlo : kPtTmQhi), kb = term == 1 ? klo_lo : khi_lo;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint32_t qoff = (uint32_t)((ks >> 2) * 16384 + (ks & 3) * 32) >> 4, koff = (uint32_t)((ks >> 2) * 8192 + (ks & 3) * 32) >> 4;
-          tc_mma_idesc(tmem_base + t * 64, desc_hi | (qa + qoff), desc_hi | (kb + koff), idesc_qk, (term | ks) ? 1u : 0u);
+        for (int ks = 0; ks < 8; ++ks) {   // 16 k values = 8 columns of Q' per step
+          const uint32_t koff = (uint32_t)((ks >> 2) * 8192 + (ks & 3) * 32) >> 4;
+          tc_mma_ts(tmem_base + kPtTmS + t * 64, qa + 8 * ks, desc_hi | (kb + koff), idesc_qk, (term | ks) ? 1u : 0u);
         }
       }
       tc_commit(bar_sfull + 8 * t);
@@ -395,7 +412,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     for (int c = 0; c < 4; ++c) {
       float o[32];
       if (n_blocks > 0 && !aborted) {
-        tc_ld32(trow + 128 + 32 * c, o);
+        tc_ld32(trow + kPtTmO + 32 * c, o);
       } else {
 #pragma unroll
         for (int i = 0; i < 32; ++i) o[i] = 0.f;
@@ -410,7 +427,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
   __syncthreads();
   if (warp == 12) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 256;" ::"r"(tmem_base) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
   }
   if (tid == 0 && aborted) set_status(a.status, PQ_ERR_TIMEOUT);
   if (tid < 256 && !aborted) {
