@@ -2,15 +2,15 @@
 // pq_decode.cu).  Same computation as pq_prefill.cuh -- the last n_q positions of a sequence attend causally to the
 // cached tokens (Eq. 2 / Eq. 3) -- for chunks that fill 128 rows = (128 / g) queries x the g query heads of a kv head.
 //
-// One CTA of thirteen warps per (query block, kv head, sequence) loops over the 64-token blocks its queries may see:
-//   * warps 4-11 ("decoders") copy the packed K and V block with cp.async, DeQuant it (Algorithm 1 by the table
+// One CTA of sixteen warps per (query block, kv head, sequence) loops over the 64-token blocks its queries may see:
+//   * warps 4-14 ("decoders") copy the packed K and V block with cp.async, DeQuant it (Algorithm 1 by the table
 //     lookups of the decode kernel: per 4-coordinate sub-block one entry for levels 4-2 and one for the two level-1
-//     pairs, fp16 with error-free residuals; a thread decodes a quarter of a token) and write the tensor-core operands into
+//     pairs, fp16 with error-free residuals; the 1024 (K | V, 16-block, token) items of a block go round the 352 threads) and write the tensor-core operands into
 //     shared memory in the K-major 128-byte-swizzled layout: K_hat as fp16 value + fp16 residual
 //     [token][coordinate], V_hat transposed [coordinate][token]; two stages, so block j + 1 is decoded while block j
 //     is multiplied.  The lookups deliver coordinates (4s, 4s+2 | 4s+1, 4s+3); K_hat keeps that order and Q' is stored
 //     in the same one (the contraction does not care), V_hat^T has the coordinate as its row index and needs none;
-//   * one thread of warp 12 issues the MMAs: S_j = Q' K_hat^T as three products (lo*hi, hi*lo, hi*hi; M = 128,
+//   * one thread of warp 15 issues the MMAs: S_j = Q' K_hat^T as three products (lo*hi, hi*lo, hi*hi; M = 128,
 //     N = 64, eight k-steps each) into one of two 64-column accumulators in tensor memory, and O += P_j V_hat
 //     (M = 128, N = 128, four k-steps) into a 128-column accumulator.  The A operands live in tensor memory too
 //     (Q' hi and lo, written once; P_j, written by the row owners), the B operands are read from shared memory by
@@ -32,16 +32,17 @@
 
 namespace pq {
 
-constexpr int kPtThreads = 416;   // warps 0-3 row owners, 4-11 decoders, 12 the MMA issuer
-constexpr int kPtDecoders = 256;
+constexpr int kPtThreads = 512;   // warps 0-3 row owners, 4-14 decoders, 15 the MMA issuer (registers are allocated per four warps)
+constexpr int kPtDecoders = 352;
+constexpr int kPtRawBufs = 3;
 constexpr int kPtRows = 128;
 constexpr int kPtStages = 4;                        // decoded (K_hat hi, K_hat lo, V_hat^T) blocks in flight
 constexpr int kPtKBytes = 64 * 128 * 2;             // K_hat hi or lo of a block: two k-halves of 64 tokens x 128 bytes
 constexpr int kPtVBytes = 128 * 64 * 2;             // V_hat^T of a block: 128 coordinates x 64 tokens
 constexpr int kPtStageBytes = 2 * kPtKBytes + kPtVBytes;
 constexpr int kPtSmKv = 0;                          // the stages; also q, Q' at the start and O at the end
-constexpr int kPtSmRaw = kPtSmKv + kPtStages * kPtStageBytes;   // two packed (K block, V block) buffers
-constexpr int kPtSmTab = kPtSmRaw + 2 * kPfRawBytes;   // u_tab[4][64], t1p_hi[256], t1p_lo[256] of Tables (8 bytes per entry)
+constexpr int kPtSmRaw = kPtSmKv + kPtStages * kPtStageBytes;   // three packed (K block, V block) buffers
+constexpr int kPtSmTab = kPtSmRaw + kPtRawBufs * kPfRawBytes;   // u_tab[4][64], t1p_hi[256], t1p_lo[256] of Tables (8 bytes per entry)
 constexpr int kPtSmBar = kPtSmTab + 6144;           // kv_full[S], pv_done[S], s_full[2], s_free[2], p_full[2], p_free[2], drain
 constexpr int kPtSmMisc = kPtSmBar + 16 * kPtStages + 80;   // tensor-memory base, abort flag
 constexpr int kPtSmTotal = kPtSmMisc + 32 + 1024;   // + slack for 1024-byte alignment
@@ -112,7 +113,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
   }
   for (int i = tid; i < 768; i += kPtThreads)
     tab[i] = i < 256 ? a.tables->u_tab[i >> 6][i & 63] : (i < 512 ? a.tables->t1p_hi[i - 256] : a.tables->t1p_lo[i - 512]);
-  if (warp == 12) {
+  if (warp == 15) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(sb + kPtSmMisc) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -247,12 +248,12 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       __syncwarp();
       if (lane == 0) tc_mbar_arrive(bar_pfull + 8 * t);
     }
-  } else if (warp < 12) {
+  } else if (warp < 15) {
     // ================= decoders: packed block -> K_hat hi / lo, V_hat^T =================
-    const int dt = tid - 128, tok = dt & 63, quarter = dt >> 6, half = quarter >> 1;
-    auto fetch = [&](int jb) {  // packed K block and V block of token-block jb -> raw buffer jb & 1
+    const int dt = tid - 128;
+    auto fetch = [&](int jb) {  // packed K block and V block of token-block jb -> raw buffer jb % 3
       const uint8_t* src = a.cache + kv_block_pair_offset(L, a.pg, a.n_kv_heads, b, hk, jb, a.status);
-      const uint32_t dst = sb + kPtSmRaw + (jb & 1) * kPfRawBytes;
+      const uint32_t dst = sb + kPtSmRaw + (jb % kPtRawBufs) * kPfRawBytes;
       for (int i = dt; i < kPfRawBytes / 16; i += kPtDecoders) pf_cp16(dst + 16 * i, src + 16 * i);
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
@@ -268,24 +269,25 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       // stage st is free once the value MMA of block jb - kPtStages has completed (it also covers that block's score MMAs)
       bool ok = true;
       if (jb >= kPtStages) ok = tc_mbar_wait(bar_pv + 8 * st, (uint32_t)(jb / kPtStages - 1) & 1u, abort_flag);
-      // the raw block has landed for all decoder threads; the decision to go on is taken together
+      // The raw block has landed for all decoder threads, and all of them have finished the previous block (the copy
+      // that the next iteration starts goes into the buffer that block was read from); the decision to go on is
+      // taken together.
       if (pt_bar_or(1, kPtDecoders, !ok)) break;
-      const uint8_t* kraw = smem + kPtSmRaw + (jb & 1) * kPfRawBytes;
-      const uint8_t* vraw = kraw + 62 * kTokenBlock;
-      const bool live = jb * kTokenBlock + tok < len;   // stale bytes past the sequence end must not reach the MMAs
+      const uint8_t* kraw = smem + kPtSmRaw + (jb % kPtRawBufs) * kPfRawBytes;
       uint8_t* stage = smem + kPtSmKv + st * kPtStageBytes;
-      uint8_t* khi = stage + half * 8192 + tok * 128;
-      uint8_t* klo = khi + kPtKBytes;
-      uint8_t* vt = stage + 2 * kPtKBytes + (tok & 7) * 2;   // V_hat^T: row = coordinate, the token is the k index
       const uint2* utab = tab;
       const uint2* t1hi = tab + 256;
       const uint2* t1lo = tab + 512;
-#pragma unroll 1
-      for (int bi = 2 * (quarter & 1); bi < 2 * (quarter & 1) + 2; ++bi) {   // block half * 4 + bi of the token
-        const int blk = half * 4 + bi;
+      // item = (K | V) * 512 + block * 64 + token: the 32 items of a warp share K | V and the block
 #pragma unroll
-        for (int kv = 0; kv < 2; ++kv) {
-          const uint8_t* raw = kv ? vraw : kraw;
+      for (int item = dt; item < 1024; item += kPtDecoders) {
+        const int kv = item >> 9, blk = (item >> 6) & 7, tok = item & 63, half = blk >> 2, bi = blk & 3;
+        const bool live = jb * kTokenBlock + tok < len;   // stale bytes past the sequence end must not reach the MMAs
+        uint8_t* khi = stage + half * 8192 + tok * 128;
+        uint8_t* klo = khi + kPtKBytes;
+        uint8_t* vt = stage + 2 * kPtKBytes + (tok & 7) * 2;   // V_hat^T: row = coordinate, the token is the k index
+        {
+          const uint8_t* raw = kraw + kv * 62 * kTokenBlock;
           const uint32_t l1 = *reinterpret_cast<const uint32_t*>(raw + tok * 32 + blk * 4);
           const uint32_t c2 = raw[kO2 + tok * 8 + blk];
           const uint32_t c3 = (uint32_t)raw[kO3 + tok * 4 + (blk >> 1)] >> (4 * (blk & 1));
@@ -333,12 +335,9 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) tc_mbar_arrive(bar_kv + 8 * st);
-      // the next iteration starts the copy of block jb + 2 into this iteration's raw buffer: every thread must have
-      // finished reading it
-      asm volatile("bar.sync 2, %0;" ::"n"(kPtDecoders) : "memory");
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-  } else if (tid == 384) {
+  } else if (tid == 480) {
     // ================= MMA issuer =================
     constexpr uint32_t idesc_qk = tc_idesc(false, 128, 64), idesc_pv = tc_idesc(false, 128, 128);
     const uint64_t desc_hi = tc_smem_desc(0u) & 0xFFFFFFFF00000000ull;
@@ -425,7 +424,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
   __syncthreads();
-  if (warp == 12) {
+  if (warp == 15) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
   }
