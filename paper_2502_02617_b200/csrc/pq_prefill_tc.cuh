@@ -64,6 +64,13 @@ __device__ __forceinline__ void pt_rank4(float (&acc)[64], const float* x, int l
   }
 }
 
+__device__ __forceinline__ void pt_sts128(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
+  asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ void pt_sts16(uint32_t addr, __half v) {
+  asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(__half_as_ushort(v)) : "memory");
+}
+
 // Named-barrier OR over `n_threads` threads (also a barrier).
 __device__ __forceinline__ bool pt_bar_or(int bar_id, int n_threads, bool v) {
   uint32_t out;
@@ -273,61 +280,60 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       // that the next iteration starts goes into the buffer that block was read from); the decision to go on is
       // taken together.
       if (pt_bar_or(1, kPtDecoders, !ok)) break;
-      const uint8_t* kraw = smem + kPtSmRaw + (jb % kPtRawBufs) * kPfRawBytes;
-      uint8_t* stage = smem + kPtSmKv + st * kPtStageBytes;
-      const uint2* utab = tab;
-      const uint2* t1hi = tab + 256;
-      const uint2* t1lo = tab + 512;
+      // all accesses below are shared-memory instructions on 32-bit addresses
+      const uint32_t kraw = sb + kPtSmRaw + (jb % kPtRawBufs) * kPfRawBytes;
+      const uint32_t stage = sb + kPtSmKv + st * kPtStageBytes;
+      const uint32_t utab = sb + kPtSmTab, t1hi = utab + 2048, t1lo = utab + 4096;
       // item = (K | V) * 512 + block * 64 + token: the 32 items of a warp share K | V and the block
 #pragma unroll
       for (int item = dt; item < 1024; item += kPtDecoders) {
         const int kv = item >> 9, blk = (item >> 6) & 7, tok = item & 63, half = blk >> 2, bi = blk & 3;
         const bool live = jb * kTokenBlock + tok < len;   // stale bytes past the sequence end must not reach the MMAs
-        uint8_t* khi = stage + half * 8192 + tok * 128;
-        uint8_t* klo = khi + kPtKBytes;
-        uint8_t* vt = stage + 2 * kPtKBytes + (tok & 7) * 2;   // V_hat^T: row = coordinate, the token is the k index
+        const uint32_t khi = stage + half * 8192 + tok * 128, klo = khi + kPtKBytes;
+        const uint32_t vt = stage + 2 * kPtKBytes + (tok & 7) * 2;   // V_hat^T: row = coordinate, the token is the k index
         {
-          const uint8_t* raw = kraw + kv * 62 * kTokenBlock;
-          const uint32_t l1 = *reinterpret_cast<const uint32_t*>(raw + tok * 32 + blk * 4);
-          const uint32_t c2 = raw[kO2 + tok * 8 + blk];
-          const uint32_t c3 = (uint32_t)raw[kO3 + tok * 4 + (blk >> 1)] >> (4 * (blk & 1));
-          const uint32_t c4 = ((uint32_t)*reinterpret_cast<const uint16_t*>(raw + kO4 + tok * 2) >> (2 * blk)) & 3u;
-          const uint32_t rbits = live ? (uint32_t)*reinterpret_cast<const uint16_t*>(raw + kORad + tok * 16 + blk * 2) : 0u;
+          const uint32_t raw = kraw + kv * 62 * kTokenBlock;
+          const uint32_t l1 = lds32(raw + tok * 32 + blk * 4);
+          const uint32_t c2 = lds8(raw + kO2 + tok * 8 + blk);
+          const uint32_t c3 = lds8(raw + kO3 + tok * 4 + (blk >> 1)) >> (4 * (blk & 1));
+          const uint32_t c4 = (lds16(raw + kO4 + tok * 2) >> (2 * blk)) & 3u;
+          const uint32_t rbits = live ? lds16(raw + kORad + tok * 16 + blk * 2) : 0u;
           const __half2 r2 = as_h2(rbits | (rbits << 16));
 #pragma unroll
           for (int sp = 0; sp < 2; ++sp) {   // two sub-blocks = eight coordinates = one 16-byte chunk of the key row
             uint32_t hw[4], lw[4];
+            const uint32_t c34 = (((c3 >> (2 * sp)) & 3u) << 2) | (c4 << 4);
 #pragma unroll
             for (int q = 0; q < 2; ++q) {
               const int sb4 = 2 * sp + q;    // sub-block: coordinates 4 sb4 .. 4 sb4 + 3 of the block
-              const uint32_t iu = ((c2 >> (2 * sb4)) & 3u) | (((c3 >> (2 * sp)) & 3u) << 2) | (c4 << 4);
-              const uint2 uu = utab[sb4 * 64 + iu];
-              const uint32_t e = (l1 >> (8 * sb4)) & 0xFFu;
-              const uint2 th = t1hi[e];
+              const uint32_t iu = ((c2 >> (2 * sb4)) & 3u) | c34;
+              const uint2 uu = lds64(utab + (sb4 * 64 + iu) * 8);
+              const uint32_t e = ((l1 >> (8 * sb4)) & 0xFFu) * 8;
+              const uint2 th = lds64(t1hi + e);
               const __half2 u_hi = __hmul2(r2, as_h2(uu.x));
               const __half2 xh = __hmul2(u_hi, as_h2(th.x)), yh = __hmul2(u_hi, as_h2(th.y));   // coordinates (4s, 4s+2), (4s+1, 4s+3)
               if (kv == 0) {
                 // the key as an unevaluated sum hi + lo (fp16 fused multiply-adds return the exact residual of a product)
-                const uint2 tl = t1lo[e];
+                const uint2 tl = lds64(t1lo + e);
                 const __half2 u_lo = __hfma2(r2, as_h2(uu.y), __hfma2(r2, as_h2(uu.x), __hneg2(u_hi)));
                 hw[2 * q] = as_u32(xh);
                 hw[2 * q + 1] = as_u32(yh);
                 lw[2 * q] = as_u32(__hfma2(u_hi, as_h2(tl.x), __hfma2(u_lo, as_h2(th.x), __hfma2(u_hi, as_h2(th.x), __hneg2(xh)))));
                 lw[2 * q + 1] = as_u32(__hfma2(u_hi, as_h2(tl.y), __hfma2(u_lo, as_h2(th.y), __hfma2(u_hi, as_h2(th.y), __hneg2(yh)))));
               } else {
-                const int coord = half * 64 + bi * 16 + 4 * sb4;
-                uint8_t* vrow = vt + coord * 128;
-                const int ch = tok >> 3;
-                *reinterpret_cast<__half*>(vrow + ((ch ^ (coord & 7)) << 4)) = __low2half(xh);
-                *reinterpret_cast<__half*>(vrow + 128 + ((ch ^ ((coord + 1) & 7)) << 4)) = __low2half(yh);
-                *reinterpret_cast<__half*>(vrow + 256 + ((ch ^ ((coord + 2) & 7)) << 4)) = __high2half(xh);
-                *reinterpret_cast<__half*>(vrow + 384 + ((ch ^ ((coord + 3) & 7)) << 4)) = __high2half(yh);
+                // rows blk * 16 + 4 sb4 + {0, 1, 2, 3}: the row's low three bits are those of 4 sb4 + k
+                const uint32_t vrow = vt + (uint32_t)(blk * 16 + 4 * sb4) * 128u;
+                const uint32_t ch = (uint32_t)tok >> 3;
+                pt_sts16(vrow + ((ch ^ ((4 * sb4) & 7)) << 4), __low2half(xh));
+                pt_sts16(vrow + 128 + ((ch ^ ((4 * sb4 + 1) & 7)) << 4), __low2half(yh));
+                pt_sts16(vrow + 256 + ((ch ^ ((4 * sb4 + 2) & 7)) << 4), __high2half(xh));
+                pt_sts16(vrow + 384 + ((ch ^ ((4 * sb4 + 3) & 7)) << 4), __high2half(yh));
               }
             }
             if (kv == 0) {
               const int c = ((2 * bi + sp) ^ (tok & 7)) << 4;
-              *reinterpret_cast<uint4*>(khi + c) = make_uint4(hw[0], hw[1], hw[2], hw[3]);
-              *reinterpret_cast<uint4*>(klo + c) = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+              pt_sts128(khi + c, hw[0], hw[1], hw[2], hw[3]);
+              pt_sts128(klo + c, lw[0], lw[1], lw[2], lw[3]);
             }
           }
         }
