@@ -249,7 +249,9 @@ int32_t pq_decode_attention_static(int32_t head_dim, int32_t n_q_heads, int32_t 
 /*
  * Test support: make the next launch of one kernel run its give-up path.  `which` = 1 arms the
  * tensor-core encoder behind pq_encode_kv (head_dim 128, bf16, >= 128 rows), 2 arms the head_dim-128
- * kernel behind pq_decode_attention, 0 disarms.  In the armed launch the first bounded wait of one CTA
+ * kernel behind pq_decode_attention, 4 the tcgen05 kernel behind pq_multi_query_attention (head_dim 128,
+ * chunks of 128 rows and more: its MMA-issuing thread gives up after two blocks, the other warps of the
+ * CTA follow, the rows of that CTA are not written), 0 disarms.  In the armed launch the first bounded wait of one CTA
  * (the one that starts the first tile / the first non-empty sequence) is reported as failed although
  * what it waited for arrived: the CTA abandons its share of the work,
  * waits for its copies in flight, releases what it holds and records PQ_ERR_TIMEOUT in status word 0;

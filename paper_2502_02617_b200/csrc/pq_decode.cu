@@ -127,7 +127,9 @@ struct DecodeArgs {
             // [batch][n_q_heads][d] with pair p = sequence * n_q + query; `lens` and the cache are per sequence.
   float scale;
   uint32_t epoch;  // differs from call to call (top bit set): tags the split tickets of the persistent kernel
-  uint32_t debug;  // bit 0: test hook, the first bounded wait of CTA 0 of the persistent kernel reports failure
+  uint32_t debug;  // test hooks.  bit 0: the first bounded wait of CTA 0 of the persistent kernel reports failure;
+                   // bit 1: the MMA thread of CTA (0, 0, 0) of the tcgen05 multi-query kernel reports its wait for the
+                   // third decoded block (the last one of a shorter sequence) as failed
   const float* S;
   const Tables* tables;
   const void* q;
@@ -688,6 +690,8 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
     if (pq::configure_for_device(pq::prefill_tc_kernel, pq::kPtSmTotal, configured_pt) == 0) return PQ_ERR_CUDA;
     const int qb_rows = pq::kPtRows / g;
     dim3 grid((n_q + qb_rows - 1) / qb_rows, n_kv_heads, batch);
+    a.epoch = 0u;
+    a.debug = pq::take_debug_wait_failure(4) ? 2u : 0u;
     pq::prefill_tc_kernel<<<grid, pq::kPtThreads, pq::kPtSmTotal, st>>>(a, n_q);
     return pq::launch_status();
   }

@@ -204,7 +204,7 @@ const char* pq_status_string(int32_t status) {
 int32_t pq_token_block(void) { return pq::kTokenBlock; }
 
 int32_t pq_debug_fail_next_wait(int32_t which) {
-  if (which < 0 || which > 3) return PQ_ERR_INVALID_ARG;
+  if (which < 0 || which > 4) return PQ_ERR_INVALID_ARG;
   pq::g_debug_wait_failure.store(which);
   return PQ_OK;
 }

@@ -374,6 +374,10 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       const int st = jb % kPtStages;
       ok = tc_mbar_wait(bar_kv + 8 * st, (uint32_t)(jb / kPtStages) & 1u, abort_flag);
       if (ok && jb >= 2) ok = tc_mbar_wait(bar_sfree + 8 * t, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag);
+      if (ok && (a.debug & 2u) && (blockIdx.x | blockIdx.y | blockIdx.z) == 0 && jb == min(2, n_blocks - 1)) {
+        *abort_flag = 1;   // test hook: this wait counts as failed (what it waited for has arrived)
+        ok = false;
+      }
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t khi_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + st * kPtStageBytes);

@@ -313,6 +313,33 @@ def test_wait_that_gives_up_in_decode_attention_is_reported_and_the_next_call_is
     pq.pq_debug_fail_next_wait(0)
 
 
+def test_wait_that_gives_up_in_the_tcgen05_multi_query_kernel_is_reported_and_the_next_call_is_clean():
+    """The MMA-issuing thread of one CTA gives up after two blocks: the decoder and row-owner warps of that CTA see the
+    abort flag at their next waits, the CTA drains its copies and MMAs, frees tensor memory and reports PQ_ERR_TIMEOUT;
+    the other CTAs finish, nothing stays behind and the next call is normal."""
+    d, Hq, Hkv, n, n_q = 128, 8, 2, 1000, 70
+    cache = pq.PolarQuantCache(2, Hq, Hkv, d, capacity=n, seed=4, device=DEV)
+    K, V = synthetic.kv_like(6, 2 * n, Hkv, d, torch.bfloat16, DEV)
+    cache.encode(K, V, torch.tensor([0, n, 2 * n], dtype=torch.int32, device=DEV))
+    g = torch.Generator(device=DEV)
+    g.manual_seed(5)
+    q = torch.randn((2, n_q, Hq, d), generator=g, device=DEV, dtype=torch.float32)
+    want = cache.attend_multi(q)
+    torch.cuda.synchronize()
+    cache.check_status()
+    pq.pq_debug_fail_next_wait(4)
+    got = cache.attend_multi(q)
+    torch.cuda.synchronize()
+    assert cache.status.cpu().tolist()[0] == pq.ERR_TIMEOUT
+    assert torch.equal(got[1], want[1])          # the other sequence's CTAs are untouched
+    cache.status.zero_()
+    again = cache.attend_multi(q)
+    torch.cuda.synchronize()
+    cache.check_status()
+    assert torch.equal(again, want)
+    pq.pq_debug_fail_next_wait(0)
+
+
 def test_mid_size_llama_shape_codes_with_window_accounting():
     """8 kv heads x 2048 tokens x d = 128 (the encode config's shape, shortened): ~3.9 M codes."""
     d, Hkv, n = 128, 8, 2048
