@@ -6,10 +6,11 @@
 //   * warps 4-14 ("decoders") copy the packed K and V block with cp.async, DeQuant it (Algorithm 1 by the table
 //     lookups of the decode kernel: per 4-coordinate sub-block one entry for levels 4-2 and one for the two level-1
 //     pairs, fp16 with error-free residuals; the 1024 (K | V, 16-block, token) items of a block go round the 352 threads) and write the tensor-core operands into
-//     shared memory in the K-major 128-byte-swizzled layout: K_hat as fp16 value + fp16 residual
-//     [token][coordinate], V_hat transposed [coordinate][token]; two stages, so block j + 1 is decoded while block j
-//     is multiplied.  The lookups deliver coordinates (4s, 4s+2 | 4s+1, 4s+3); K_hat keeps that order and Q' is stored
-//     in the same one (the contraction does not care), V_hat^T has the coordinate as its row index and needs none;
+//     shared memory as 128-byte-swizzled tiles [token][64 coordinates] x two coordinate halves: K_hat as fp16 value
+//     + fp16 residual (a K-major B operand: the contraction runs over the coordinates), V_hat as fp16 value (an
+//     MN-major B operand: the contraction runs over the tokens); four stages, so the decoders run ahead of the MMAs.
+//     The lookups deliver coordinates (4s, 4s+2 | 4s+1, 4s+3); K_hat keeps that order and Q' is stored in the same
+//     one (the contraction does not care), V_hat is put back in natural order by two byte permutes per sub-block;
 //   * one thread of warp 15 issues the MMAs: S_j = Q' K_hat^T as three products (lo*hi, hi*lo, hi*hi; M = 128,
 //     N = 64, eight k-steps each) into one of two 64-column accumulators in tensor memory, and O += P_j V_hat
 //     (M = 128, N = 128, four k-steps) into a 128-column accumulator.  The A operands live in tensor memory too
@@ -38,7 +39,7 @@ constexpr int kPtRawBufs = 3;
 constexpr int kPtRows = 128;
 constexpr int kPtStages = 4;                        // decoded (K_hat hi, K_hat lo, V_hat^T) blocks in flight
 constexpr int kPtKBytes = 64 * 128 * 2;             // K_hat hi or lo of a block: two k-halves of 64 tokens x 128 bytes
-constexpr int kPtVBytes = 128 * 64 * 2;             // V_hat^T of a block: 128 coordinates x 64 tokens
+constexpr int kPtVBytes = 64 * 128 * 2;             // V_hat of a block: two coordinate halves of 64 tokens x 128 bytes
 constexpr int kPtStageBytes = 2 * kPtKBytes + kPtVBytes;
 constexpr int kPtSmKv = 0;                          // the stages; also q, Q' at the start and O at the end
 constexpr int kPtSmRaw = kPtSmKv + kPtStages * kPtStageBytes;   // three packed (K block, V block) buffers
@@ -290,7 +291,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
         const int kv = item >> 9, blk = (item >> 6) & 7, tok = item & 63, half = blk >> 2, bi = blk & 3;
         const bool live = jb * kTokenBlock + tok < len;   // stale bytes past the sequence end must not reach the MMAs
         const uint32_t khi = stage + half * 8192 + tok * 128, klo = khi + kPtKBytes;
-        const uint32_t vt = stage + 2 * kPtKBytes + (tok & 7) * 2;   // V_hat^T: row = coordinate, the token is the k index
+        const uint32_t vrow = stage + 2 * kPtKBytes + half * 8192 + tok * 128;   // V_hat: [coordinate half][token][64 coordinates]
         {
           const uint32_t raw = kraw + kv * 62 * kTokenBlock;
           const uint32_t l1 = lds32(raw + tok * 32 + blk * 4);
@@ -321,19 +322,17 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
                 lw[2 * q] = as_u32(__hfma2(u_hi, as_h2(tl.x), __hfma2(u_lo, as_h2(th.x), __hfma2(u_hi, as_h2(th.x), __hneg2(xh)))));
                 lw[2 * q + 1] = as_u32(__hfma2(u_hi, as_h2(tl.y), __hfma2(u_lo, as_h2(th.y), __hfma2(u_hi, as_h2(th.y), __hneg2(yh)))));
               } else {
-                // rows blk * 16 + 4 sb4 + {0, 1, 2, 3}: the row's low three bits are those of 4 sb4 + k
-                const uint32_t vrow = vt + (uint32_t)(blk * 16 + 4 * sb4) * 128u;
-                const uint32_t ch = (uint32_t)tok >> 3;
-                pt_sts16(vrow + ((ch ^ ((4 * sb4) & 7)) << 4), __low2half(xh));
-                pt_sts16(vrow + 128 + ((ch ^ ((4 * sb4 + 1) & 7)) << 4), __low2half(yh));
-                pt_sts16(vrow + 256 + ((ch ^ ((4 * sb4 + 2) & 7)) << 4), __high2half(xh));
-                pt_sts16(vrow + 384 + ((ch ^ ((4 * sb4 + 3) & 7)) << 4), __high2half(yh));
+                // coordinates in natural order: (4s, 4s+1) = (x.lo, y.lo), (4s+2, 4s+3) = (x.hi, y.hi)
+                hw[2 * q] = __byte_perm(as_u32(xh), as_u32(yh), 0x5410);
+                hw[2 * q + 1] = __byte_perm(as_u32(xh), as_u32(yh), 0x7632);
               }
             }
+            const int c = ((2 * bi + sp) ^ (tok & 7)) << 4;
             if (kv == 0) {
-              const int c = ((2 * bi + sp) ^ (tok & 7)) << 4;
               pt_sts128(khi + c, hw[0], hw[1], hw[2], hw[3]);
               pt_sts128(klo + c, lw[0], lw[1], lw[2], lw[3]);
+            } else {
+              pt_sts128(vrow + c, hw[0], hw[1], hw[2], hw[3]);
             }
           }
         }
@@ -345,16 +344,21 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     asm volatile("cp.async.wait_group 0;" ::: "memory");
   } else if (tid == 480) {
     // ================= MMA issuer =================
-    constexpr uint32_t idesc_qk = tc_idesc(false, 128, 64), idesc_pv = tc_idesc(false, 128, 128);
+    // the value operand is MN-major: [token][coordinate] rows of 64 coordinates, the two coordinate halves 8192 bytes apart
+    constexpr uint32_t idesc_qk = tc_idesc(false, 128, 64), idesc_pv = tc_idesc(false, 128, 128) | (1u << 16);
+    uint64_t vdesc_hi = (uint64_t)(1024 >> 4) << 32;   // stride between groups of 8 tokens
+    vdesc_hi |= (uint64_t)1 << 46;
+    vdesc_hi |= (uint64_t)2 << 61;
+    const uint32_t vdesc_lbo = (8192u >> 4) << 16;     // leading-dimension offset: the next 64 coordinates
     const uint64_t desc_hi = tc_smem_desc(0u) & 0xFFFFFFFF00000000ull;
     auto issue_pv = [&](int jb) -> bool {   // O (+)= P_jb V_hat_jb
       const int t = jb & 1, st = jb % kPtStages;
       if (!tc_mbar_wait(bar_pfull + 8 * t, (uint32_t)(jb >> 1) & 1u, abort_flag)) return false;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t v_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + st * kPtStageBytes + 2 * kPtKBytes);
+      const uint32_t v_lo = (((sb + kPtSmKv + st * kPtStageBytes + 2 * kPtKBytes) & 0x3FFFFu) >> 4) | vdesc_lbo;
 #pragma unroll
-      for (int kk = 0; kk < 4; ++kk)   // 16 tokens = 8 columns of P per step
-        tc_mma_ts(tmem_base + kPtTmO, tmem_base + kPtTmP + 32 * t + 8 * kk, desc_hi | (v_lo + 2 * kk), idesc_pv, (jb > 0 || kk > 0) ? 1u : 0u);
+      for (int kk = 0; kk < 4; ++kk)   // 16 tokens = 8 columns of P = 16 rows of 128 bytes of V_hat per step
+        tc_mma_ts(tmem_base + kPtTmO, tmem_base + kPtTmP + 32 * t + 8 * kk, vdesc_hi | (v_lo + 128 * kk), idesc_pv, (jb > 0 || kk > 0) ? 1u : 0u);
       tc_commit(bar_pv + 8 * st);     // the stage is free
       tc_commit(bar_pfree + 8 * t);   // and so is the P buffer; the output accumulator holds block jb
       return true;
