@@ -686,13 +686,36 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
   if (lse_dev != nullptr && n_q != 1) return PQ_ERR_UNSUPPORTED;
   if (head_dim == 128 && n_q * g >= pq::kPtRows && !pq::take_debug_wait_failure(3)) {
     // Chunks that fill 128 rows: the tcgen05 kernel (operands in shared memory, accumulators in tensor memory).
-    static pq::DeviceMemo configured_pt;
-    if (pq::configure_for_device(pq::prefill_tc_kernel, pq::kPtSmTotal, configured_pt) == 0) return PQ_ERR_CUDA;
+    static pq::DeviceMemo configured_pt, configured_pt2;
+    if (pq::configure_for_device(pq::prefill_tc_kernel<false>, pq::kPtSmTotal, configured_pt) == 0) return PQ_ERR_CUDA;
+    if (pq::configure_for_device(pq::prefill_tc_kernel<true>, pq::kPtSmTotal, configured_pt2) == 0) return PQ_ERR_CUDA;
     const int qb_rows = pq::kPtRows / g;
-    dim3 grid((n_q + qb_rows - 1) / qb_rows, n_kv_heads, batch);
+    const int q_blocks = (n_q + qb_rows - 1) / qb_rows;
     a.epoch = 0u;
     a.debug = pq::take_debug_wait_failure(4) ? 2u : 0u;
-    pq::prefill_tc_kernel<<<grid, pq::kPtThreads, pq::kPtSmTotal, st>>>(a, n_q);
+    if (q_blocks >= 2) {
+      // Two query blocks of one (kv head, sequence) per cluster: one 256-row MMA per step, each CTA decodes half of
+      // every block.  An odd count is completed by a CTA without rows.
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((q_blocks + 1) & ~1, n_kv_heads, batch);
+      cfg.blockDim = dim3(pq::kPtThreads);
+      cfg.dynamicSmemBytes = pq::kPtSmTotal;
+      cfg.stream = st;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = 2;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      if (cudaLaunchKernelEx(&cfg, pq::prefill_tc_kernel<true>, a, (int)n_q) != cudaSuccess) {
+        cudaGetLastError();
+        return PQ_ERR_CUDA;
+      }
+      return pq::launch_status();
+    }
+    dim3 grid(q_blocks, n_kv_heads, batch);
+    pq::prefill_tc_kernel<false><<<grid, pq::kPtThreads, pq::kPtSmTotal, st>>>(a, n_q);
     return pq::launch_status();
   }
   if (head_dim == 128 && n_q * g >= pq::kPfRows) {

@@ -33,6 +33,7 @@
 
 namespace pq {
 
+
 constexpr int kPtThreads = 512;   // warps 0-3 row owners, 4-14 decoders, 15 the MMA issuer (registers are allocated per four warps)
 constexpr int kPtDecoders = 352;
 constexpr int kPtRawBufs = 3;
@@ -72,6 +73,21 @@ __device__ __forceinline__ void pt_sts16(uint32_t addr, __half v) {
   asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"(__half_as_ushort(v)) : "memory");
 }
 
+__device__ __forceinline__ uint32_t pt_mapa(uint32_t addr, uint32_t cta_rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(cta_rank));
+  return r;
+}
+__device__ __forceinline__ void pt_cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// Arrival on a barrier of the even CTA of the pair (`bar` = its shared::cluster address, from mapa), ordered after this
+// thread's earlier writes at cluster scope.
+__device__ __forceinline__ void pt_arrive_cluster(uint32_t bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
 // Named-barrier OR over `n_threads` threads (also a barrier).
 __device__ __forceinline__ bool pt_bar_or(int bar_id, int n_threads, bool v) {
   uint32_t out;
@@ -86,6 +102,13 @@ __device__ __forceinline__ bool pt_bar_or(int bar_id, int n_threads, bool v) {
   return out != 0;
 }
 
+// kPair: the CTAs of two consecutive query blocks of one (kv head, sequence) form a cluster and run ONE 256-row MMA per
+// step (cta_group::2, issued by a thread of the even CTA): every CTA keeps its own 128 rows of Q', S, P and O in its own
+// tensor memory and supplies half of each B operand from its own shared memory -- the keys of 32 of the block's 64
+// tokens, the values of 64 of the 128 coordinates -- so a CTA decodes half a block per block and no decoded data
+// crosses between the CTAs.  The even CTA's barriers collect the arrivals of both CTAs' decoder and row-owner warps;
+// its commits are multicast to both CTAs' barriers.
+template <bool kPair>
 __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a, int n_q) {
   extern __shared__ uint8_t pt_smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(pt_smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -94,7 +117,19 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
   const int g = a.n_q_heads / a.n_kv_heads;
   const int qb_rows = kPtRows / g;                      // queries of a CTA
   const int q0 = blockIdx.x * qb_rows, hk = blockIdx.y, b = blockIdx.z;
-  const int n_rows = min(qb_rows, n_q - q0) * g;        // rows in use; row r = (query q0 + r / g, head hk * g + r % g)
+  const int n_rows = max(0, min(qb_rows, n_q - q0)) * g;   // rows in use; row r = (query q0 + r / g, head hk * g + r % g);
+                                                           // none in the CTA that only completes a pair
+  uint32_t crank = 0;
+  if (kPair) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
+  const bool leader = crank == 0;   // the CTA whose thread issues the MMAs and whose barriers collect the arrivals
+  // per-CTA shapes of the B operands: keys of kKTok tokens (two coordinate halves), values of 64 tokens x kVHalves x 64 coordinates
+  constexpr int kKTok = kPair ? 32 : 64, kKHalf = kKTok * 128, kKTile = 2 * kKHalf, kVHalves = kPair ? 1 : 2;
+  constexpr int kStage = 2 * kKTile + kVHalves * 8192;
+  // packed blocks in flight: the copy of block jb + kRawBufs - 1 starts when block jb is decoded.  A pair's stages are
+  // half as large: its packed buffers follow them inside the stage area.
+  constexpr int kRawBufs = kPair ? 6 : kPtRawBufs;
+  constexpr int kSmRaw = kPair ? kPtSmKv + kPtStages * kStage : kPtSmRaw;
+  static_assert(!kPair || kSmRaw + kRawBufs * kPfRawBytes <= kPtSmRaw, "a pair's packed buffers fit behind its stages");
   const int len = a.lens[b];
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + kPtSmMisc + 4);
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kPtSmMisc);
@@ -106,13 +141,13 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
   };
   if (tid == 0) {
     for (int i = 0; i < kPtStages; ++i) {
-      tc_mbar_init(bar_kv + 8 * i, kPtDecoders / 32);   // one arrival per decoder warp
+      tc_mbar_init(bar_kv + 8 * i, (kPair ? 2 : 1) * kPtDecoders / 32);   // one arrival per decoder warp (of both CTAs)
       tc_mbar_init(bar_pv + 8 * i, 1);                  // tcgen05.commit after the value MMA that read the stage
     }
     for (int i = 0; i < 2; ++i) {
       tc_mbar_init(bar_sfull + 8 * i, 1);   // tcgen05.commit
-      tc_mbar_init(bar_sfree + 8 * i, 4);   // one arrival per row-owner warp
-      tc_mbar_init(bar_pfull + 8 * i, 4);
+      tc_mbar_init(bar_sfree + 8 * i, kPair ? 8 : 4);   // one arrival per row-owner warp (of both CTAs)
+      tc_mbar_init(bar_pfull + 8 * i, kPair ? 8 : 4);
       tc_mbar_init(bar_pfree + 8 * i, 1);   // tcgen05.commit after the value MMA that read the P buffer
     }
     tc_mbar_init(bar_drain, 1);
@@ -121,9 +156,14 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
   }
   for (int i = tid; i < 768; i += kPtThreads)
     tab[i] = i < 256 ? a.tables->u_tab[i >> 6][i & 63] : (i < 512 ? a.tables->t1p_hi[i - 256] : a.tables->t1p_lo[i - 512]);
-  if (warp == 15) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(sb + kPtSmMisc) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (warp == 15) {   // in a pair: the same warp of both CTAs, the same destination offset
+    if (kPair) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(sb + kPtSmMisc) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(sb + kPtSmMisc) : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   // ---- Q' = (Q S) * scale * log2(e) as fp16 value + residual (threads 0..255: column, half of the rows), staged in shared
   // memory and then written to tensor memory by the row owners (lane = row, two k values per column)
@@ -183,9 +223,14 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
   __syncthreads();   // Q' is in tensor memory; the staging is dead: the stages may be written
+  if (kPair) pt_cluster_sync();   // both CTAs' barriers are initialised and both halves of Q' are in place
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const int vis_cta = max(0, len - (n_q - 1 - (q0 + (n_rows - 1) / g)));   // the CTA's last query sees the most
+  // the last query of the CTA (of the pair) sees the most
+  const int q_last = min(n_q, ((kPair ? (int)(blockIdx.x | 1u) : (int)blockIdx.x) + 1) * qb_rows) - 1;
+  const int vis_cta = max(0, len - (n_q - 1 - q_last));
   const int n_blocks = (vis_cta + kTokenBlock - 1) / kTokenBlock;
+  // where this CTA's warps announce themselves: the barriers of the even CTA
+  const uint32_t to_leader = kPair ? pt_mapa(sb, 0u) - sb : 0u;   // + a local shared address: that place in the even CTA (cluster window)
   const Layout L = make_layout(128, a.pg.page_tokens);
 
   float l_run = 0.f;   // row owners: denominator of this thread's row
@@ -195,6 +240,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     const int vis = r < n_rows ? max(0, len - (n_q - 1 - (q0 + r / g))) : 0;
     const uint32_t trow = tmem_base + ((uint32_t)(warp * 32) << 16);
     float m_run = -CUDART_INF_F;
+    const int vis_min = __reduce_min_sync(0xffffffffu, vis);
     for (int jb = 0; jb < n_blocks; ++jb) {
       const int t = jb & 1;
       const uint32_t ph = (uint32_t)(jb >> 1) & 1u;
@@ -206,13 +252,22 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       tc_ld32(trow + t * 64 + 32, s + 32);
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
-      if (lane == 0) tc_mbar_arrive(bar_sfree + 8 * t);   // the scores are in registers: the accumulator may be overwritten
-      float mx = -CUDART_INF_F;
-#pragma unroll
-      for (int i = 0; i < 64; ++i) {
-        s[i] = jb * kTokenBlock + i < vis ? s[i] : -CUDART_INF_F;
-        mx = fmaxf(mx, s[i]);
+      if (lane == 0) {   // the scores are in registers: the accumulator may be overwritten
+        if (kPair) pt_arrive_cluster(bar_sfree + 8 * t + to_leader);
+        else tc_mbar_arrive(bar_sfree + 8 * t);
       }
+      // the causal mask touches only the last blocks of a row: one uniform test per warp skips it elsewhere
+      if ((jb + 1) * kTokenBlock > vis_min) {
+#pragma unroll
+        for (int i = 0; i < 64; ++i) s[i] = jb * kTokenBlock + i < vis ? s[i] : -CUDART_INF_F;
+      }
+      float mx4[4] = {-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F};   // four chains: no 64-long dependency
+#pragma unroll
+      for (int i = 0; i < 64; i += 8) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) mx4[c] = fmaxf(mx4[c], fmaxf(s[i + 2 * c], s[i + 2 * c + 1]));
+      }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       // lazy reference: move it only when some score exceeds it by more than 8 (p <= 2^8 otherwise)
       const bool grow = mx > m_run + 8.f || (m_run == -CUDART_INF_F && mx > -CUDART_INF_F);
       if (__any_sync(0xffffffffu, grow)) {
@@ -242,38 +297,43 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
         ok = __all_sync(0xffffffffu, tc_mbar_wait(bar_pfree + 8 * t, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag));
         if (!ok) break;
       }
-      float sum = 0.f;
-      uint32_t pw[32];
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int e = 0; e < 32; ++e) {
-        const __half2 p2 = __floats2half2_rn(fast_exp2(s[2 * e] - m_use), fast_exp2(s[2 * e + 1] - m_use));
-        sum += __low2float(p2) + __high2float(p2);   // the denominator of what the MMA will see
-        pw[e] = as_u32(p2);
+      for (int hf = 0; hf < 2; ++hf) {   // the store of the first half runs while the second half is computed
+        uint32_t pw[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const int i = 32 * hf + 2 * e;
+          const __half2 p2 = __floats2half2_rn(fast_exp2(s[i] - m_use), fast_exp2(s[i + 1] - m_use));
+          sum4[e & 3] += __low2float(p2) + __high2float(p2);   // the denominator of what the MMA will see
+          pw[e] = as_u32(p2);
+        }
+        tc_st16u_nowait(trow + kPtTmP + 32 * t + 16 * hf, pw);
       }
-      l_run += sum;
-      tc_st32u(trow + kPtTmP + 32 * t, pw);
+      l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
-      if (lane == 0) tc_mbar_arrive(bar_pfull + 8 * t);
+      if (lane == 0) {
+        if (kPair) pt_arrive_cluster(bar_pfull + 8 * t + to_leader);
+        else tc_mbar_arrive(bar_pfull + 8 * t);
+      }
     }
   } else if (warp < 15) {
     // ================= decoders: packed block -> K_hat hi / lo, V_hat^T =================
     const int dt = tid - 128;
-    auto fetch = [&](int jb) {  // packed K block and V block of token-block jb -> raw buffer jb % 3
-      const uint8_t* src = a.cache + kv_block_pair_offset(L, a.pg, a.n_kv_heads, b, hk, jb, a.status);
-      const uint32_t dst = sb + kPtSmRaw + (jb % kPtRawBufs) * kPfRawBytes;
-      for (int i = dt; i < kPfRawBytes / 16; i += kPtDecoders) pf_cp16(dst + 16 * i, src + 16 * i);
+    auto fetch = [&](int jb) {  // packed K block and V block of token-block jb -> raw buffer jb % kRawBufs (one group per call)
+      if (jb < n_blocks) {
+        const uint8_t* src = a.cache + kv_block_pair_offset(L, a.pg, a.n_kv_heads, b, hk, jb, a.status);
+        const uint32_t dst = sb + kSmRaw + (jb % kRawBufs) * kPfRawBytes;
+        for (int i = dt; i < kPfRawBytes / 16; i += kPtDecoders) pf_cp16(dst + 16 * i, src + 16 * i);
+      }
       asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    if (n_blocks > 0) fetch(0);
+    for (int i = 0; i < kRawBufs - 1; ++i) fetch(i);
     for (int jb = 0; jb < n_blocks; ++jb) {
       const int st = jb % kPtStages;
-      if (jb + 1 < n_blocks) {
-        fetch(jb + 1);
-        asm volatile("cp.async.wait_group 1;" ::: "memory");
-      } else {
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-      }
+      asm volatile("cp.async.wait_group %0;" ::"n"(kRawBufs - 2) : "memory");   // this thread's part of block jb has landed
       // stage st is free once the value MMA of block jb - kPtStages has completed (it also covers that block's score MMAs)
       bool ok = true;
       if (jb >= kPtStages) ok = tc_mbar_wait(bar_pv + 8 * st, (uint32_t)(jb / kPtStages - 1) & 1u, abort_flag);
@@ -281,71 +341,95 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       // that the next iteration starts goes into the buffer that block was read from); the decision to go on is
       // taken together.
       if (pt_bar_or(1, kPtDecoders, !ok)) break;
+      fetch(jb + kRawBufs - 1);   // into the buffer of block jb - 1
       // all accesses below are shared-memory instructions on 32-bit addresses
-      const uint32_t kraw = sb + kPtSmRaw + (jb % kPtRawBufs) * kPfRawBytes;
-      const uint32_t stage = sb + kPtSmKv + st * kPtStageBytes;
+      const uint32_t kraw = sb + kSmRaw + (jb % kRawBufs) * kPfRawBytes;
+      const uint32_t stage = sb + kPtSmKv + st * kStage;
       const uint32_t utab = sb + kPtSmTab, t1hi = utab + 2048, t1lo = utab + 4096;
-      // item = (K | V) * 512 + block * 64 + token: the 32 items of a warp share K | V and the block
+      // An item is one 16-byte chunk of an operand row: (K | V, 16-block, half of the block, token); the 32 items of
+      // a warp share all but the token.  A CTA of a pair takes the keys of tokens 32 rank .. 32 rank + 31 and the
+      // values of blocks 4 rank .. 4 rank + 3 (coordinates 64 rank .. 64 rank + 63) of all 64 tokens.
+      constexpr int kItems = kPair ? 1024 : 2048;
 #pragma unroll
-      for (int item = dt; item < 1024; item += kPtDecoders) {
-        const int kv = item >> 9, blk = (item >> 6) & 7, tok = item & 63, half = blk >> 2, bi = blk & 3;
+      for (int item = dt; item < kItems; item += kPtDecoders) {
+        int kv, blk, sp, tok;
+        if (kPair) {
+          kv = item >> 9;
+          if (kv == 0) { blk = (item >> 6) & 7; sp = (item >> 5) & 1; tok = (item & 31) + 32 * (int)crank; }
+          else { blk = ((item >> 7) & 3) + 4 * (int)crank; sp = (item >> 6) & 1; tok = item & 63; }
+        } else {
+          kv = item >> 10; blk = (item >> 7) & 7; sp = (item >> 6) & 1; tok = item & 63;
+        }
+        const int half = blk >> 2, bi = blk & 3;
         const bool live = jb * kTokenBlock + tok < len;   // stale bytes past the sequence end must not reach the MMAs
-        const uint32_t khi = stage + half * 8192 + tok * 128, klo = khi + kPtKBytes;
-        const uint32_t vrow = stage + 2 * kPtKBytes + half * 8192 + tok * 128;   // V_hat: [coordinate half][token][64 coordinates]
-        {
-          const uint32_t raw = kraw + kv * 62 * kTokenBlock;
-          const uint32_t l1 = lds32(raw + tok * 32 + blk * 4);
-          const uint32_t c2 = lds8(raw + kO2 + tok * 8 + blk);
-          const uint32_t c3 = lds8(raw + kO3 + tok * 4 + (blk >> 1)) >> (4 * (blk & 1));
-          const uint32_t c4 = (lds16(raw + kO4 + tok * 2) >> (2 * blk)) & 3u;
-          const uint32_t rbits = live ? lds16(raw + kORad + tok * 16 + blk * 2) : 0u;
-          const __half2 r2 = as_h2(rbits | (rbits << 16));
+        const uint32_t raw = kraw + kv * 62 * kTokenBlock;
+        const uint32_t l1 = lds16(raw + tok * 32 + blk * 4 + sp * 2);               // the two level-1 bytes of this half
+        const uint32_t c2 = lds8(raw + kO2 + tok * 8 + blk) >> (4 * sp);
+        const uint32_t c3 = lds8(raw + kO3 + tok * 4 + (blk >> 1)) >> (4 * (blk & 1) + 2 * sp);
+        const uint32_t c4 = (lds16(raw + kO4 + tok * 2) >> (2 * blk)) & 3u;
+        const uint32_t rbits = live ? lds16(raw + kORad + tok * 16 + blk * 2) : 0u;
+        const __half2 r2 = as_h2(rbits | (rbits << 16));
+        const uint32_t c34 = ((c3 & 3u) << 2) | (c4 << 4);
+        uint32_t hw[4], lw[4];
 #pragma unroll
-          for (int sp = 0; sp < 2; ++sp) {   // two sub-blocks = eight coordinates = one 16-byte chunk of the key row
-            uint32_t hw[4], lw[4];
-            const uint32_t c34 = (((c3 >> (2 * sp)) & 3u) << 2) | (c4 << 4);
-#pragma unroll
-            for (int q = 0; q < 2; ++q) {
-              const int sb4 = 2 * sp + q;    // sub-block: coordinates 4 sb4 .. 4 sb4 + 3 of the block
-              const uint32_t iu = ((c2 >> (2 * sb4)) & 3u) | c34;
-              const uint2 uu = lds64(utab + (sb4 * 64 + iu) * 8);
-              const uint32_t e = ((l1 >> (8 * sb4)) & 0xFFu) * 8;
-              const uint2 th = lds64(t1hi + e);
-              const __half2 u_hi = __hmul2(r2, as_h2(uu.x));
-              const __half2 xh = __hmul2(u_hi, as_h2(th.x)), yh = __hmul2(u_hi, as_h2(th.y));   // coordinates (4s, 4s+2), (4s+1, 4s+3)
-              if (kv == 0) {
-                // the key as an unevaluated sum hi + lo (fp16 fused multiply-adds return the exact residual of a product)
-                const uint2 tl = lds64(t1lo + e);
-                const __half2 u_lo = __hfma2(r2, as_h2(uu.y), __hfma2(r2, as_h2(uu.x), __hneg2(u_hi)));
-                hw[2 * q] = as_u32(xh);
-                hw[2 * q + 1] = as_u32(yh);
-                lw[2 * q] = as_u32(__hfma2(u_hi, as_h2(tl.x), __hfma2(u_lo, as_h2(th.x), __hfma2(u_hi, as_h2(th.x), __hneg2(xh)))));
-                lw[2 * q + 1] = as_u32(__hfma2(u_hi, as_h2(tl.y), __hfma2(u_lo, as_h2(th.y), __hfma2(u_hi, as_h2(th.y), __hneg2(yh)))));
-              } else {
-                // coordinates in natural order: (4s, 4s+1) = (x.lo, y.lo), (4s+2, 4s+3) = (x.hi, y.hi)
-                hw[2 * q] = __byte_perm(as_u32(xh), as_u32(yh), 0x5410);
-                hw[2 * q + 1] = __byte_perm(as_u32(xh), as_u32(yh), 0x7632);
-              }
-            }
-            const int c = ((2 * bi + sp) ^ (tok & 7)) << 4;
-            if (kv == 0) {
-              pt_sts128(khi + c, hw[0], hw[1], hw[2], hw[3]);
-              pt_sts128(klo + c, lw[0], lw[1], lw[2], lw[3]);
-            } else {
-              pt_sts128(vrow + c, hw[0], hw[1], hw[2], hw[3]);
-            }
+        for (int q = 0; q < 2; ++q) {   // sub-block 2 sp + q: coordinates 4 (2 sp + q) .. + 3 of the block
+          const uint32_t iu = ((c2 >> (2 * q)) & 3u) | c34;
+          const uint2 uu = lds64(utab + (uint32_t)(2 * sp + q) * 512u + iu * 8u);
+          const uint32_t e = ((l1 >> (8 * q)) & 0xFFu) * 8u;
+          const uint2 th = lds64(t1hi + e);
+          const __half2 u_hi = __hmul2(r2, as_h2(uu.x));
+          const __half2 xh = __hmul2(u_hi, as_h2(th.x)), yh = __hmul2(u_hi, as_h2(th.y));   // coordinates (4s, 4s+2), (4s+1, 4s+3)
+          if (kv == 0) {
+            // the key as an unevaluated sum hi + lo (fp16 fused multiply-adds return the exact residual of a product)
+            const uint2 tl = lds64(t1lo + e);
+            const __half2 u_lo = __hfma2(r2, as_h2(uu.y), __hfma2(r2, as_h2(uu.x), __hneg2(u_hi)));
+            hw[2 * q] = as_u32(xh);
+            hw[2 * q + 1] = as_u32(yh);
+            lw[2 * q] = as_u32(__hfma2(u_hi, as_h2(tl.x), __hfma2(u_lo, as_h2(th.x), __hfma2(u_hi, as_h2(th.x), __hneg2(xh)))));
+            lw[2 * q + 1] = as_u32(__hfma2(u_hi, as_h2(tl.y), __hfma2(u_lo, as_h2(th.y), __hfma2(u_hi, as_h2(th.y), __hneg2(yh)))));
+          } else {
+            // coordinates in natural order: (4s, 4s+1) = (x.lo, y.lo), (4s+2, 4s+3) = (x.hi, y.hi)
+            hw[2 * q] = __byte_perm(as_u32(xh), as_u32(yh), 0x5410);
+            hw[2 * q + 1] = __byte_perm(as_u32(xh), as_u32(yh), 0x7632);
           }
+        }
+        // chunk 2 bi + sp of the row's 64-coordinate half, swizzled by the row
+        if (kv == 0) {
+          const int row = tok & (kKTok - 1);
+          const uint32_t dst = stage + half * kKHalf + row * 128 + (((2 * bi + sp) ^ (row & 7)) << 4);
+          pt_sts128(dst, hw[0], hw[1], hw[2], hw[3]);
+          pt_sts128(dst + kKTile, lw[0], lw[1], lw[2], lw[3]);
+        } else {
+          const uint32_t dst = stage + 2 * kKTile + (kPair ? 0 : half * 8192) + tok * 128 + (((2 * bi + sp) ^ (tok & 7)) << 4);
+          pt_sts128(dst, hw[0], hw[1], hw[2], hw[3]);
         }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0) tc_mbar_arrive(bar_kv + 8 * st);
+      if (lane == 0) {
+        if (kPair) pt_arrive_cluster(bar_kv + 8 * st + to_leader);
+        else tc_mbar_arrive(bar_kv + 8 * st);
+      }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
-  } else if (tid == 480) {
+  } else if (tid == 480 && leader) {
     // ================= MMA issuer =================
     // the value operand is MN-major: [token][coordinate] rows of 64 coordinates, the two coordinate halves 8192 bytes apart
-    constexpr uint32_t idesc_qk = tc_idesc(false, 128, 64), idesc_pv = tc_idesc(false, 128, 128) | (1u << 16);
+    // (in a pair: one half per CTA)
+    constexpr uint32_t kM = kPair ? 256 : 128;
+    constexpr uint32_t idesc_qk = tc_idesc(false, kM, 64);
+    constexpr uint32_t idesc_pv = tc_idesc(false, kM, 128) | (1u << 16);
+    auto mma = [&](uint32_t d, uint32_t a_t, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+      if (kPair) tc_mma_ts_pair(d, a_t, bdesc, idesc, acc);
+      else tc_mma_ts(d, a_t, bdesc, idesc, acc);
+    };
+    auto commit = [&](uint32_t bar) {   // in a pair: arrives on both CTAs' barriers
+      if (kPair) tc_commit_pair(bar);
+      else tc_commit(bar);
+    };
+    auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {   // barriers that warps of both CTAs arrive on
+      return kPair ? tc_mbar_wait_cluster(bar, parity, abort_flag) : tc_mbar_wait(bar, parity, abort_flag);
+    };
     uint64_t vdesc_hi = (uint64_t)(1024 >> 4) << 32;   // stride between groups of 8 tokens
     vdesc_hi |= (uint64_t)1 << 46;
     vdesc_hi |= (uint64_t)2 << 61;
@@ -353,14 +437,14 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     const uint64_t desc_hi = tc_smem_desc(0u) & 0xFFFFFFFF00000000ull;
     auto issue_pv = [&](int jb) -> bool {   // O (+)= P_jb V_hat_jb
       const int t = jb & 1, st = jb % kPtStages;
-      if (!tc_mbar_wait(bar_pfull + 8 * t, (uint32_t)(jb >> 1) & 1u, abort_flag)) return false;
+      if (!wait_all(bar_pfull + 8 * t, (uint32_t)(jb >> 1) & 1u)) return false;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t v_lo = (((sb + kPtSmKv + st * kPtStageBytes + 2 * kPtKBytes) & 0x3FFFFu) >> 4) | vdesc_lbo;
+      const uint32_t v_lo = (((sb + kPtSmKv + st * kStage + 2 * kKTile) & 0x3FFFFu) >> 4) | vdesc_lbo;
 #pragma unroll
       for (int kk = 0; kk < 4; ++kk)   // 16 tokens = 8 columns of P = 16 rows of 128 bytes of V_hat per step
-        tc_mma_ts(tmem_base + kPtTmO, tmem_base + kPtTmP + 32 * t + 8 * kk, vdesc_hi | (v_lo + 128 * kk), idesc_pv, (jb > 0 || kk > 0) ? 1u : 0u);
-      tc_commit(bar_pv + 8 * st);     // the stage is free
-      tc_commit(bar_pfree + 8 * t);   // and so is the P buffer; the output accumulator holds block jb
+        mma(tmem_base + kPtTmO, tmem_base + kPtTmP + 32 * t + 8 * kk, vdesc_hi | (v_lo + 128 * kk), idesc_pv, (jb > 0 || kk > 0) ? 1u : 0u);
+      commit(bar_pv + 8 * st);     // the stage is free
+      commit(bar_pfree + 8 * t);   // and so is the P buffer; the output accumulator holds block jb
       return true;
     };
     bool ok = true;
@@ -376,37 +460,49 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
         if (!ok) break;
       }
       const int st = jb % kPtStages;
-      ok = tc_mbar_wait(bar_kv + 8 * st, (uint32_t)(jb / kPtStages) & 1u, abort_flag);
-      if (ok && jb >= 2) ok = tc_mbar_wait(bar_sfree + 8 * t, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag);
+      ok = wait_all(bar_kv + 8 * st, (uint32_t)(jb / kPtStages) & 1u);
+      if (ok && jb >= 2) ok = wait_all(bar_sfree + 8 * t, (uint32_t)((jb - 2) >> 1) & 1u);
       if (ok && (a.debug & 2u) && (blockIdx.x | blockIdx.y | blockIdx.z) == 0 && jb == min(2, n_blocks - 1)) {
         *abort_flag = 1;   // test hook: this wait counts as failed (what it waited for has arrived)
         ok = false;
       }
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t khi_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + st * kPtStageBytes);
-      const uint32_t klo_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + st * kPtStageBytes + kPtKBytes);
+      const uint32_t khi_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + st * kStage);
+      const uint32_t klo_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + st * kStage + kKTile);
       // S = Q'lo K_hi^T + Q'hi K_lo^T + Q'hi K_hi^T (small terms first); k-step ks: half ks >> 2, 32 bytes per step
 #pragma unroll
       for (int term = 0; term < 3; ++term) {
         const uint32_t qa = tmem_base + (term == 0 ? kPtTmQlo : kPtTmQhi), kb = term == 1 ? klo_lo : khi_lo;
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {   // 16 k values = 8 columns of Q' per step
-          const uint32_t koff = (uint32_t)((ks >> 2) * 8192 + (ks & 3) * 32) >> 4;
-          tc_mma_ts(tmem_base + kPtTmS + t * 64, qa + 8 * ks, desc_hi | (kb + koff), idesc_qk, (term | ks) ? 1u : 0u);
+          const uint32_t koff = (uint32_t)((ks >> 2) * kKHalf + (ks & 3) * 32) >> 4;
+          mma(tmem_base + kPtTmS + t * 64, qa + 8 * ks, desc_hi | (kb + koff), idesc_qk, (term | ks) ? 1u : 0u);
         }
       }
-      tc_commit(bar_sfull + 8 * t);
+      commit(bar_sfull + 8 * t);
       if (!pv_issued) ok = issue_pv(jb - 1);
     }
     if (ok && n_blocks > 0) ok = issue_pv(n_blocks - 1);
     if (n_blocks > 0) {
       // every MMA issued above has completed when this commit arrives (nothing was issued without blocks: no commit)
-      tc_commit(bar_drain);
+      commit(bar_drain);
       bool drained = false;
       for (int i = 0; i < (1 << 20) && !drained; ++i) {
         drained = tc_mbar_try(bar_drain, 0);
         if (!drained) __nanosleep(32);
+      }
+      if (!drained) *abort_flag = 1;
+    }
+    if (kPair && *abort_flag)   // tell the other CTA, whose warps wait for commits that will not come
+      asm volatile("st.relaxed.cluster.shared::cluster.u32 [%0], %1;" ::"r"(sb + kPtSmMisc + 4 + (pt_mapa(sb, 1u) - sb)), "r"(1u) : "memory");
+  } else if (kPair && tid == 480) {
+    // the odd CTA of a pair: its operands are read until the even CTA's last commit arrives here too
+    if (n_blocks > 0) {
+      bool drained = false;
+      for (int i = 0; i < kTcSpin && !drained && !*abort_flag; ++i) {
+        drained = tc_mbar_try(bar_drain, 0);
+        if (!drained) __nanosleep(64);
       }
       if (!drained) *abort_flag = 1;
     }
@@ -438,9 +534,13 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
   __syncthreads();
+  // In a pair neither CTA may release tensor memory or leave while the other may still arrive on its barriers or
+  // have its operands read: both have drained here.
+  if (kPair) pt_cluster_sync();
   if (warp == 15) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    if (kPair) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
   }
   if (tid == 0 && aborted) set_status(a.status, PQ_ERR_TIMEOUT);
   if (tid < 256 && !aborted) {

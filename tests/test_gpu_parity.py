@@ -184,8 +184,9 @@ def test_attention_special_cases_len1_and_identical_keys():
 
 @pytest.mark.parametrize("d,Hq,Hkv,n_q", [(128, 8, 2, 5), (128, 8, 1, 3), (16, 4, 2, 4),            # one decode per query
                                            (128, 8, 1, 9), (128, 6, 2, 22), (128, 2, 2, 70),      # register-fragment MMA kernel (64..127 rows)
-                                           (128, 8, 2, 40), (128, 8, 1, 20), (128, 6, 2, 50), (128, 2, 2, 150),   # tcgen05 kernel (>= 128 rows)
-                                           (128, 10, 2, 70)])
+                                           (128, 8, 2, 32), (128, 8, 1, 16),                      # tcgen05 kernel, one query block: single CTAs
+                                           (128, 8, 2, 40), (128, 8, 1, 20), (128, 6, 2, 50), (128, 2, 2, 150),   # two query blocks: a CTA pair
+                                           (128, 10, 2, 70), (128, 8, 2, 140)])                   # odd block counts: a pair completed by an idle CTA
 def test_multi_query_attention_is_causal_over_the_last_positions(d, Hq, Hkv, n_q):
     """The last n_q positions of every sequence attend at once; query j sees the tokens up to its own position.
     Float32 I/O against the oracle per query, and n_q = 1 equals decode attention bit for bit."""
