@@ -82,10 +82,11 @@ __device__ __forceinline__ void pt_cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
-// Arrival on a barrier of the even CTA of the pair (`bar` = its shared::cluster address, from mapa), ordered after this
-// thread's earlier writes at cluster scope.
+// Arrival on a barrier of the even CTA of the pair (`bar` = its shared::cluster address, from mapa).  What the arriving
+// warp wrote before is read by its own SM's tensor core (operands in shared memory after fence.proxy.async, P in
+// tensor memory after tcgen05.wait::st), which the even CTA's MMA triggers after it has seen the arrival.
 __device__ __forceinline__ void pt_arrive_cluster(uint32_t bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
 // Named-barrier OR over `n_threads` threads (also a barrier).
@@ -428,7 +429,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       else tc_commit(bar);
     };
     auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {   // barriers that warps of both CTAs arrive on
-      return kPair ? tc_mbar_wait_cluster(bar, parity, abort_flag) : tc_mbar_wait(bar, parity, abort_flag);
+      return tc_mbar_wait(bar, parity, abort_flag);
     };
     uint64_t vdesc_hi = (uint64_t)(1024 >> 4) << 32;   // stride between groups of 8 tokens
     vdesc_hi |= (uint64_t)1 << 46;

@@ -107,29 +107,6 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
                "h"((uint16_t)3)
                : "memory");
 }
-// Probe with acquire semantics at cluster scope (arrivals from the other CTA of a cluster).
-__device__ __forceinline__ bool tc_mbar_try_cluster(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ bool tc_mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (int i = 0; i < kTcSpin; ++i) {
-    if (tc_mbar_try_cluster(bar, parity)) return true;
-    if (i > 32) {
-      __nanosleep(64);
-      if (*abort_flag) return false;
-    }
-  }
-  *abort_flag = 1;
-  return false;
-}
 // Write 32 consecutive columns of this thread's tensor-memory lane.
 __device__ __forceinline__ void tc_st32(uint32_t taddr, const float* v) {
   asm volatile(
