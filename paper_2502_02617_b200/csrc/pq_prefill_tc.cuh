@@ -50,8 +50,9 @@ constexpr int kPtSmMisc = kPtSmBar + 16 * kPtStages + 80;   // tensor-memory bas
 constexpr int kPtSmTotal = kPtSmMisc + 32 + 1024;   // + slack for 1024-byte alignment
 constexpr int kPtOStride = 132;                     // floats per row of the output staging
 constexpr int kPtQStride = 136;                     // halves per row of the Q' staging (rows 16 bytes apart mod 128)
-// tensor-memory columns: two score accumulators, the output accumulator, Q' hi and lo (two fp16 per column), two P buffers
-constexpr uint32_t kPtTmS = 0, kPtTmO = 128, kPtTmQhi = 256, kPtTmQlo = 320, kPtTmP = 384;
+// tensor-memory columns: two score accumulators of 128 (64 tokens x key value and residual; P_j, two fp16 per column,
+// later takes the first 32 columns of the accumulator it came from), the output accumulator, Q' hi and lo
+constexpr uint32_t kPtTmS = 0, kPtTmO = 256, kPtTmQhi = 384, kPtTmQlo = 448;
 static_assert(kPtSmTotal <= 227 * 1024, "shared memory of one CTA");
 static_assert(128 * kPtOStride * 4 <= kPtStages * kPtStageBytes, "float32 output staging fits in the stages");
 static_assert(128 * 128 * 4 + 2 * 128 * kPtQStride * 2 <= kPtStages * kPtStageBytes, "q and Q' staging fit in the stages");
@@ -124,8 +125,14 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
   if (kPair) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
   const bool leader = crank == 0;   // the CTA whose thread issues the MMAs and whose barriers collect the arrivals
   // per-CTA shapes of the B operands: keys of kKTok tokens (two coordinate halves), values of 64 tokens x kVHalves x 64 coordinates
-  constexpr int kKTok = kPair ? 32 : 64, kKHalf = kKTok * 128, kKTile = 2 * kKHalf, kVHalves = kPair ? 1 : 2;
-  constexpr int kStage = 2 * kKTile + kVHalves * 8192;
+  // A key tile holds, for each half of the coordinates, the fp16 values of the kKTok tokens followed by their residuals:
+  // one B operand of 2 kKTok rows, so one MMA gives the products with both.
+  constexpr int kKTok = kPair ? 32 : 64, kKLo = kKTok * 128, kKHalf = 2 * kKLo, kKTile = 2 * kKHalf, kVHalves = kPair ? 1 : 2;
+  constexpr int kStage = kKTile + kVHalves * 8192;
+  // columns of a score accumulator: tokens [32 c, 32 c + 32) times the values at kColHi(c), times the residuals at kColLo(c)
+  // (a pair's accumulator columns follow the two CTAs' operand rows)
+  auto col_hi = [](int c) -> uint32_t { return kPair ? 64u * c : 32u * c; };
+  auto col_lo = [](int c) -> uint32_t { return kPair ? 64u * c + 32u : 64u + 32u * c; };
   // packed blocks in flight: the copy of block jb + kRawBufs - 1 starts when block jb is decoded.  A pair's stages are
   // half as large: its packed buffers follow them inside the stage area.
   constexpr int kRawBufs = kPair ? 6 : kPtRawBufs;
@@ -147,9 +154,8 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     }
     for (int i = 0; i < 2; ++i) {
       tc_mbar_init(bar_sfull + 8 * i, 1);   // tcgen05.commit
-      tc_mbar_init(bar_sfree + 8 * i, kPair ? 8 : 4);   // one arrival per row-owner warp (of both CTAs)
       tc_mbar_init(bar_pfull + 8 * i, kPair ? 8 : 4);
-      tc_mbar_init(bar_pfree + 8 * i, 1);   // tcgen05.commit after the value MMA that read the P buffer
+      tc_mbar_init(bar_pfree + 8 * i, 1);   // tcgen05.commit after the value MMA: the output accumulator holds the block
     }
     tc_mbar_init(bar_drain, 1);
     *abort_flag = 0;
@@ -249,13 +255,13 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       float s[64];
-      tc_ld32(trow + t * 64, s);
-      tc_ld32(trow + t * 64 + 32, s + 32);
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) {   // the scores are in registers: the accumulator may be overwritten
-        if (kPair) pt_arrive_cluster(bar_sfree + 8 * t + to_leader);
-        else tc_mbar_arrive(bar_sfree + 8 * t);
+#pragma unroll
+      for (int c = 0; c < 2; ++c) {   // Q' K_hi^T + Q' K_lo^T
+        float lo[32];
+        tc_ld32(trow + t * 128 + col_hi(c), s + 32 * c);
+        tc_ld32(trow + t * 128 + col_lo(c), lo);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) s[32 * c + i] += lo[i];
       }
       // the causal mask touches only the last blocks of a row: one uniform test per warp skips it elsewhere
       if ((jb + 1) * kTokenBlock > vis_min) {
@@ -293,11 +299,8 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
         m_run = m_new;
       }
       const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;   // nothing visible yet: every p is 0
-      // P buffer t is free once the value MMA of block jb - 2 has completed
-      if (jb >= 2) {
-        ok = __all_sync(0xffffffffu, tc_mbar_wait(bar_pfree + 8 * t, (uint32_t)((jb - 2) >> 1) & 1u, abort_flag));
-        if (!ok) break;
-      }
+      // P_jb takes the first 32 columns of the accumulator it was computed from (all of it is in registers): the value
+      // MMA of block jb - 2, which read them last, was issued before the score MMAs that s_full reported
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {   // the store of the first half runs while the second half is computed
@@ -309,7 +312,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
           sum4[e & 3] += __low2float(p2) + __high2float(p2);   // the denominator of what the MMA will see
           pw[e] = as_u32(p2);
         }
-        tc_st16u_nowait(trow + kPtTmP + 32 * t + 16 * hf, pw);
+        tc_st16u_nowait(trow + kPtTmS + 128 * t + 16 * hf, pw);
       }
       l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
@@ -399,9 +402,9 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
           const int row = tok & (kKTok - 1);
           const uint32_t dst = stage + half * kKHalf + row * 128 + (((2 * bi + sp) ^ (row & 7)) << 4);
           pt_sts128(dst, hw[0], hw[1], hw[2], hw[3]);
-          pt_sts128(dst + kKTile, lw[0], lw[1], lw[2], lw[3]);
+          pt_sts128(dst + kKLo, lw[0], lw[1], lw[2], lw[3]);
         } else {
-          const uint32_t dst = stage + 2 * kKTile + (kPair ? 0 : half * 8192) + tok * 128 + (((2 * bi + sp) ^ (tok & 7)) << 4);
+          const uint32_t dst = stage + kKTile + (kPair ? 0 : half * 8192) + tok * 128 + (((2 * bi + sp) ^ (tok & 7)) << 4);
           pt_sts128(dst, hw[0], hw[1], hw[2], hw[3]);
         }
       }
@@ -418,7 +421,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     // the value operand is MN-major: [token][coordinate] rows of 64 coordinates, the two coordinate halves 8192 bytes apart
     // (in a pair: one half per CTA)
     constexpr uint32_t kM = kPair ? 256 : 128;
-    constexpr uint32_t idesc_qk = tc_idesc(false, kM, 64);
+    constexpr uint32_t idesc_qk = tc_idesc(false, kM, 128);   // 64 tokens x (value, residual)
     constexpr uint32_t idesc_pv = tc_idesc(false, kM, 128) | (1u << 16);
     auto mma = [&](uint32_t d, uint32_t a_t, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
       if (kPair) tc_mma_ts_pair(d, a_t, bdesc, idesc, acc);
@@ -440,12 +443,12 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       const int t = jb & 1, st = jb % kPtStages;
       if (!wait_all(bar_pfull + 8 * t, (uint32_t)(jb >> 1) & 1u)) return false;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t v_lo = (((sb + kPtSmKv + st * kStage + 2 * kKTile) & 0x3FFFFu) >> 4) | vdesc_lbo;
+      const uint32_t v_lo = (((sb + kPtSmKv + st * kStage + kKTile) & 0x3FFFFu) >> 4) | vdesc_lbo;
 #pragma unroll
       for (int kk = 0; kk < 4; ++kk)   // 16 tokens = 8 columns of P = 16 rows of 128 bytes of V_hat per step
-        mma(tmem_base + kPtTmO, tmem_base + kPtTmP + 32 * t + 8 * kk, vdesc_hi | (v_lo + 128 * kk), idesc_pv, (jb > 0 || kk > 0) ? 1u : 0u);
+        mma(tmem_base + kPtTmO, tmem_base + kPtTmS + 128 * t + 8 * kk, vdesc_hi | (v_lo + 128 * kk), idesc_pv, (jb > 0 || kk > 0) ? 1u : 0u);
       commit(bar_pv + 8 * st);     // the stage is free
-      commit(bar_pfree + 8 * t);   // and so is the P buffer; the output accumulator holds block jb
+      commit(bar_pfree + 8 * t);   // the output accumulator holds block jb
       return true;
     };
     bool ok = true;
@@ -462,23 +465,24 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       }
       const int st = jb % kPtStages;
       ok = wait_all(bar_kv + 8 * st, (uint32_t)(jb / kPtStages) & 1u);
-      if (ok && jb >= 2) ok = wait_all(bar_sfree + 8 * t, (uint32_t)((jb - 2) >> 1) & 1u);
+      // accumulator t is free: its scores were read before P_{jb-2} was announced, and the value MMA that read
+      // P_{jb-2} from its columns was issued in the previous iteration (MMAs of one thread execute in order)
       if (ok && (a.debug & 2u) && (blockIdx.x | blockIdx.y | blockIdx.z) == 0 && jb == min(2, n_blocks - 1)) {
         *abort_flag = 1;   // test hook: this wait counts as failed (what it waited for has arrived)
         ok = false;
       }
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t khi_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + st * kStage);
-      const uint32_t klo_lo = (uint32_t)tc_smem_desc(sb + kPtSmKv + st * kStage + kKTile);
-      // S = Q'lo K_hi^T + Q'hi K_lo^T + Q'hi K_hi^T (small terms first); k-step ks: half ks >> 2, 32 bytes per step
+      const uint32_t kb = (uint32_t)tc_smem_desc(sb + kPtSmKv + st * kStage);
+      // [Q' K_hi^T | Q' K_lo^T] = (Q'lo + Q'hi) [K_hi | K_lo]^T, the small term first (its product with K_lo is
+      // below float32 resolution and rides along); k-step ks: half ks >> 2, 32 bytes per step
 #pragma unroll
-      for (int term = 0; term < 3; ++term) {
-        const uint32_t qa = tmem_base + (term == 0 ? kPtTmQlo : kPtTmQhi), kb = term == 1 ? klo_lo : khi_lo;
+      for (int term = 0; term < 2; ++term) {
+        const uint32_t qa = tmem_base + (term == 0 ? kPtTmQlo : kPtTmQhi);
 #pragma unroll
         for (int ks = 0; ks < 8; ++ks) {   // 16 k values = 8 columns of Q' per step
           const uint32_t koff = (uint32_t)((ks >> 2) * kKHalf + (ks & 3) * 32) >> 4;
-          mma(tmem_base + kPtTmS + t * 64, qa + 8 * ks, desc_hi | (kb + koff), idesc_qk, (term | ks) ? 1u : 0u);
+          mma(tmem_base + kPtTmS + t * 128, qa + 8 * ks, desc_hi | (kb + koff), idesc_qk, (term | ks) ? 1u : 0u);
         }
       }
       commit(bar_sfull + 8 * t);
