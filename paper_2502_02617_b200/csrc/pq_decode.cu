@@ -687,15 +687,17 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
   if (head_dim == 128 && n_q * g >= pq::kPtRows && !pq::take_debug_wait_failure(3)) {
     // Chunks that fill 128 rows: the tcgen05 kernel (operands in shared memory, accumulators in tensor memory).
     static pq::DeviceMemo configured_pt, configured_pt2;
-    if (pq::configure_for_device(pq::prefill_tc_kernel<false>, pq::kPtSmTotal, configured_pt) == 0) return PQ_ERR_CUDA;
+    const int n_sm = pq::configure_for_device(pq::prefill_tc_kernel<false>, pq::kPtSmTotal, configured_pt);
+    if (n_sm == 0) return PQ_ERR_CUDA;
     if (pq::configure_for_device(pq::prefill_tc_kernel<true>, pq::kPtSmTotal, configured_pt2) == 0) return PQ_ERR_CUDA;
     const int qb_rows = pq::kPtRows / g;
     const int q_blocks = (n_q + qb_rows - 1) / qb_rows;
     a.epoch = 0u;
     a.debug = pq::take_debug_wait_failure(4) ? 2u : 0u;
-    if (q_blocks >= 2) {
+    if (q_blocks >= 2 || 2 * (int64_t)n_kv_heads * batch <= n_sm) {
       // Two query blocks of one (kv head, sequence) per cluster: one 256-row MMA per step, each CTA decodes half of
-      // every block.  An odd count is completed by a CTA without rows.
+      // every block.  An odd count is completed by a CTA without rows -- also a single block when the pairs still fit
+      // on the device at once: the second CTA then only shares the decoding (the kernel is bound by it).
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3((q_blocks + 1) & ~1, n_kv_heads, batch);
       cfg.blockDim = dim3(pq::kPtThreads);

@@ -224,6 +224,38 @@ def test_multi_query_attention_is_causal_over_the_last_positions(d, Hq, Hkv, n_q
         assert rel_l2(to_f64(legacy), got) < 5e-4 and not torch.equal(legacy, out)   # different kernels, same answer
 
 
+def test_multi_query_single_block_on_a_full_device_runs_unpaired_ctas():
+    """One query block per (kv head, sequence) and more units than half the SMs: the tcgen05 kernel runs one CTA per
+    unit, each decoding whole blocks (with fewer units a second CTA shares the decoding).  Against the oracle on the
+    first and last sequence, against the register-fragment kernel everywhere."""
+    d, Hq, Hkv, n_q, B, n = 128, 8, 2, 32, 80, 130
+    lens_list = [n - (b % 3) for b in range(B)]
+    cache = pq.PolarQuantCache(B, Hq, Hkv, d, capacity=n, seed=31, device=DEV)
+    K, V = synthetic.kv_like(32, sum(lens_list), Hkv, d, torch.bfloat16, DEV)
+    cu = torch.tensor(np.concatenate(([0], np.cumsum(lens_list))), dtype=torch.int32, device=DEV)
+    cache.encode(K, V, cu)
+    g = torch.Generator(device=DEV)
+    g.manual_seed(33)
+    q = torch.randn((B, n_q, Hq, d), generator=g, device=DEV, dtype=torch.float32)
+    out = cache.attend_multi(q)
+    torch.cuda.synchronize()
+    cache.check_status()
+    pq.pq_debug_fail_next_wait(3)
+    legacy = cache.attend_multi(q)
+    torch.cuda.synchronize()
+    assert rel_l2(to_f64(legacy), to_f64(out)) < 5e-4 and not torch.equal(legacy, out)
+    cb = oracle_codebooks(cache)
+    S = cache.S_host.double().numpy()
+    Kc, Vc = to_f64(K), to_f64(V)
+    for b in (0, B - 1):
+        ref = orc.OracleCache(1, Hkv, n, d, cb, S)
+        row = int(cu[b])
+        ref.encode_chunk(0, Kc[row:row + lens_list[b]], Vc[row:row + lens_list[b]])
+        want = orc.multi_query_attention(to_f64(q[b:b + 1]), ref.k_codes, ref.k_radii, ref.v_codes, ref.v_radii, ref.lens, ref.cb,
+                                         ref.S, d ** -0.5)
+        assert rel_l2(to_f64(out[b:b + 1]), want) < TOL_ATTENTION_F32_IO, b
+
+
 def want_bf16(orc, ref, qb, d):
     return orc.multi_query_attention(to_f64(qb), ref.k_codes, ref.k_radii, ref.v_codes, ref.v_radii, ref.lens, ref.cb, ref.S,
                                      d ** -0.5)
