@@ -350,21 +350,25 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       const uint32_t kraw = sb + kSmRaw + (jb % kRawBufs) * kPfRawBytes;
       const uint32_t stage = sb + kPtSmKv + st * kStage;
       const uint32_t utab = sb + kPtSmTab, t1hi = utab + 2048, t1lo = utab + 4096;
-      // An item is one 16-byte chunk of an operand row: (K | V, 16-block, half of the block, token); the 32 items of
-      // a warp share all but the token.  A CTA of a pair takes the keys of tokens 32 rank .. 32 rank + 31 and the
-      // values of blocks 4 rank .. 4 rank + 3 (coordinates 64 rank .. 64 rank + 63) of all 64 tokens.
+      // An item is one 16-byte chunk of an operand row: (K | V, 16-block, half of the block, token).  The 32 items of a
+      // warp are 8 tokens x the 4 blocks of one coordinate half: the code words of a warp then sit in few shared-
+      // memory rows (the level-1 plane is 32 bytes per token: 32 tokens with one block would be an 8-way bank
+      // conflict, this is 2-way), and 8 lanes with one block and 8 tokens still store to 8 distinct swizzled
+      // positions.  A CTA of a pair takes the keys of tokens 32 rank .. 32 rank + 31 and the values of blocks
+      // 4 rank .. 4 rank + 3 (coordinates 64 rank .. 64 rank + 63) of all 64 tokens.
       constexpr int kItems = kPair ? 1024 : 2048;
 #pragma unroll
       for (int item = dt; item < kItems; item += kPtDecoders) {
-        int kv, blk, sp, tok;
+        const int iw = item >> 5;   // the warp's item group
+        int kv, half, sp, tg;
         if (kPair) {
-          kv = item >> 9;
-          if (kv == 0) { blk = (item >> 6) & 7; sp = (item >> 5) & 1; tok = (item & 31) + 32 * (int)crank; }
-          else { blk = ((item >> 7) & 3) + 4 * (int)crank; sp = (item >> 6) & 1; tok = item & 63; }
+          kv = iw >> 4;
+          if (kv == 0) { half = (iw >> 3) & 1; sp = (iw >> 2) & 1; tg = (iw & 3) + 4 * (int)crank; }
+          else { half = (int)crank; sp = (iw >> 3) & 1; tg = iw & 7; }
         } else {
-          kv = item >> 10; blk = (item >> 7) & 7; sp = (item >> 6) & 1; tok = item & 63;
+          kv = iw >> 5; half = (iw >> 4) & 1; sp = (iw >> 3) & 1; tg = iw & 7;
         }
-        const int half = blk >> 2, bi = blk & 3;
+        const int blk = 4 * half + (lane >> 3), tok = 8 * tg + (lane & 7), bi = blk & 3;
         const bool live = jb * kTokenBlock + tok < len;   // stale bytes past the sequence end must not reach the MMAs
         const uint32_t raw = kraw + kv * 62 * kTokenBlock;
         const uint32_t l1 = lds16(raw + tok * 32 + blk * 4 + sp * 2);               // the two level-1 bytes of this half
