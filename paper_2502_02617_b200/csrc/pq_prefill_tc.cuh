@@ -2,31 +2,33 @@
 // pq_decode.cu).  Same computation as pq_prefill.cuh -- the last n_q positions of a sequence attend causally to the
 // cached tokens (Eq. 2 / Eq. 3) -- for chunks that fill 128 rows = (128 / g) queries x the g query heads of a kv head.
 //
-// One CTA of sixteen warps per (query block, kv head, sequence) loops over the 64-token blocks its queries may see:
+// A CTA of sixteen warps owns 128 rows of one (kv head, sequence) and loops over the 64-token blocks its queries may
+// see; two CTAs with consecutive query blocks run as a pair on one 256-row MMA (see prefill_tc_kernel):
 //   * warps 4-14 ("decoders") copy the packed K and V block with cp.async, DeQuant it (Algorithm 1 by the table
 //     lookups of the decode kernel: per 4-coordinate sub-block one entry for levels 4-2 and one for the two level-1
-//     pairs, fp16 with error-free residuals; the 1024 (K | V, 16-block, token) items of a block go round the 352 threads) and write the tensor-core operands into
-//     shared memory as 128-byte-swizzled tiles [token][64 coordinates] x two coordinate halves: K_hat as fp16 value
-//     + fp16 residual (a K-major B operand: the contraction runs over the coordinates), V_hat as fp16 value (an
-//     MN-major B operand: the contraction runs over the tokens); four stages, so the decoders run ahead of the MMAs.
+//     pairs, fp16 with error-free residuals) and write the tensor-core operands into shared memory as
+//     128-byte-swizzled tiles of 64-coordinate rows: per coordinate half the fp16 values of the tokens followed by
+//     their fp16 residuals (ONE K-major B operand: the contraction runs over the coordinates, the rows are
+//     (value | residual, token)), and V_hat as fp16 values [token][64 coordinates] x two halves (an MN-major B
+//     operand: the contraction runs over the tokens); four stages, so the decoders run ahead of the MMAs.
 //     The lookups deliver coordinates (4s, 4s+2 | 4s+1, 4s+3); K_hat keeps that order and Q' is stored in the same
 //     one (the contraction does not care), V_hat is put back in natural order by two byte permutes per sub-block;
-//   * one thread of warp 15 issues the MMAs: S_j = Q' K_hat^T as three products (lo*hi, hi*lo, hi*hi; M = 128,
-//     N = 64, eight k-steps each) into one of two 64-column accumulators in tensor memory, and O += P_j V_hat
-//     (M = 128, N = 128, four k-steps) into a 128-column accumulator.  The A operands live in tensor memory too
-//     (Q' hi and lo, written once; P_j, written by the row owners), the B operands are read from shared memory by
-//     the tensor core itself: no warp re-reads a tile (the register-fragment kernel spends 70 % of the
-//     shared-memory pipe on exactly that), and shared memory is left for a ring of four decoded stages;
-//   * warps 0-3 ("row owners": tensor-memory lane = row = thread) read S_j with tcgen05.ld, apply the causal mask
-//     and the online softmax in the log2 domain without any shuffle (a thread owns its whole row), and write P_j
-//     in fp16 into tensor memory as the A operand of the value MMA.  The running maximum is updated lazily: only when a score exceeds
-//     it by more than 8 is the output accumulator rescaled (tcgen05.ld / multiply / tcgen05.st by the row's owner,
-//     after the previous value MMA has completed); otherwise p <= 2^8 stays well inside fp16.
-// Q' = (Q S) * scale * log2 e is formed once per CTA in float32 and kept as fp16 value + residual; the output is
+//   * one thread of warp 15 issues the MMAs: [Q' K_hi^T | Q' K_lo^T] = (Q'lo + Q'hi) [K_hi | K_lo]^T (N = 128, eight
+//     k-steps per term) into one of two 128-column accumulators in tensor memory, and O += P_j V_hat (N = 128, four
+//     k-steps) into a 128-column accumulator.  The A operands live in tensor memory too (Q' hi and lo, written
+//     once; P_j, written by the row owners), the B operands are read from shared memory by the tensor core itself:
+//     no warp re-reads a tile (the register-fragment kernel spends 70 % of the shared-memory pipe on exactly that);
+//   * warps 0-3 ("row owners": tensor-memory lane = row = thread) read the scores with tcgen05.ld, add the value and
+//     residual halves, apply the causal mask and the online softmax in the log2 domain without any shuffle (a thread
+//     owns its whole row), and write P_j in fp16 over the first columns of the accumulator the scores came from, as
+//     the A operand of the value MMA.  The running maximum is updated lazily: only when a score exceeds it by more
+//     than 8 is the output accumulator rescaled (tcgen05.ld / multiply / tcgen05.st by the row's owner, after the
+//     previous value MMA has completed); otherwise p <= 2^8 stays well inside fp16.
+// Q' = (Q S) * scale * log2(e) is formed once per CTA in float32 and kept as fp16 value + residual; the output is
 // normalised and rotated back by S^T in float32 when the CTA ends.  All hand-offs are mbarriers (decoded stage
-// full, scores full / read, P full, value MMA done = stage and P buffer free); every wait is bounded, and a wait
-// that gives up makes every role leave its loop, after which the CTA drains its copies and MMAs, releases tensor
-// memory and records PQ_ERR_TIMEOUT.
+// full, scores full, P full, value MMA done = stage free); every wait is bounded, and a wait that gives up makes
+// every role leave its loop, after which the CTA (the pair) drains its copies and MMAs, releases tensor memory and
+// records PQ_ERR_TIMEOUT.
 #pragma once
 
 #include "pq_tc_common.cuh"
@@ -45,7 +47,7 @@ constexpr int kPtStageBytes = 2 * kPtKBytes + kPtVBytes;
 constexpr int kPtSmKv = 0;                          // the stages; also q, Q' at the start and O at the end
 constexpr int kPtSmRaw = kPtSmKv + kPtStages * kPtStageBytes;   // three packed (K block, V block) buffers
 constexpr int kPtSmTab = kPtSmRaw + kPtRawBufs * kPfRawBytes;   // u_tab[4][64], t1p_hi[256], t1p_lo[256] of Tables (8 bytes per entry)
-constexpr int kPtSmBar = kPtSmTab + 6144;           // kv_full[S], pv_done[S], s_full[2], s_free[2], p_full[2], p_free[2], drain
+constexpr int kPtSmBar = kPtSmTab + 6144;           // kv_full[S], pv_done[S], s_full[2], (unused)[2], p_full[2], p_free[2], drain
 constexpr int kPtSmMisc = kPtSmBar + 16 * kPtStages + 80;   // tensor-memory base, abort flag
 constexpr int kPtSmTotal = kPtSmMisc + 32 + 1024;   // + slack for 1024-byte alignment
 constexpr int kPtOStride = 132;                     // floats per row of the output staging
@@ -143,7 +145,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + kPtSmMisc);
   uint2* tab = reinterpret_cast<uint2*>(smem + kPtSmTab);
   const uint32_t bar_kv = sb + kPtSmBar, bar_pv = bar_kv + 8 * kPtStages, bar_sfull = bar_pv + 8 * kPtStages,
-                 bar_sfree = bar_sfull + 16, bar_pfull = bar_sfree + 16, bar_pfree = bar_pfull + 16, bar_drain = bar_pfree + 16;
+                 bar_pfull = bar_sfull + 32, bar_pfree = bar_pfull + 16, bar_drain = bar_pfree + 16;
   auto row_index = [&](int r) -> int64_t {               // offset of row r in q / out ([batch][n_q][n_q_heads][128])
     return (((int64_t)b * n_q + q0 + r / g) * a.n_q_heads + hk * g + r % g) * 128;
   };
