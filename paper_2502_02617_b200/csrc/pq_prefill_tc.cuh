@@ -92,6 +92,17 @@ __device__ __forceinline__ void pt_arrive_cluster(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
+// (a0, a1) + (b0, b1) as one packed float32 instruction
+__device__ __forceinline__ void pt_add2(float a0, float a1, float b0, float b1, float& c0, float& c1) {
+  asm("{\n\t.reg .b64 a, b, c;\n\t"
+      "mov.b64 a, {%2, %3};\n\t"
+      "mov.b64 b, {%4, %5};\n\t"
+      "add.rn.f32x2 c, a, b;\n\t"
+      "mov.b64 {%0, %1}, c;\n\t}"
+      : "=f"(c0), "=f"(c1)
+      : "f"(a0), "f"(a1), "f"(b0), "f"(b1));
+}
+
 // Named-barrier OR over `n_threads` threads (also a barrier).
 __device__ __forceinline__ bool pt_bar_or(int bar_id, int n_threads, bool v) {
   uint32_t out;
@@ -263,7 +274,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
         tc_ld32(trow + t * 128 + col_hi(c), s + 32 * c);
         tc_ld32(trow + t * 128 + col_lo(c), lo);
 #pragma unroll
-        for (int i = 0; i < 32; ++i) s[32 * c + i] += lo[i];
+        for (int i = 0; i < 32; i += 2) pt_add2(s[32 * c + i], s[32 * c + i + 1], lo[i], lo[i + 1], s[32 * c + i], s[32 * c + i + 1]);
       }
       // the causal mask touches only the last blocks of a row: one uniform test per warp skips it elsewhere
       if ((jb + 1) * kTokenBlock > vis_min) {
@@ -303,20 +314,23 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       const float m_use = m_run == -CUDART_INF_F ? 0.f : m_run;   // nothing visible yet: every p is 0
       // P_jb takes the first 32 columns of the accumulator it was computed from (all of it is in registers): the value
       // MMA of block jb - 2, which read them last, was issued before the score MMAs that s_full reported
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      float sum8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int hf = 0; hf < 2; ++hf) {   // the store of the first half runs while the second half is computed
         uint32_t pw[16];
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
           const int i = 32 * hf + 2 * e;
-          const __half2 p2 = __floats2half2_rn(fast_exp2(s[i] - m_use), fast_exp2(s[i + 1] - m_use));
-          sum4[e & 3] += __low2float(p2) + __high2float(p2);   // the denominator of what the MMA will see
+          float x0, x1;
+          pt_add2(s[i], s[i + 1], -m_use, -m_use, x0, x1);
+          const __half2 p2 = __floats2half2_rn(fast_exp2(x0), fast_exp2(x1));
+          const float2 pf = __half22float2(p2);   // the denominator of what the MMA will see
+          pt_add2(sum8[2 * (e & 3)], sum8[2 * (e & 3) + 1], pf.x, pf.y, sum8[2 * (e & 3)], sum8[2 * (e & 3) + 1]);
           pw[e] = as_u32(p2);
         }
         tc_st16u_nowait(trow + kPtTmS + 128 * t + 16 * hf, pw);
       }
-      l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+      l_run += ((sum8[0] + sum8[1]) + (sum8[2] + sum8[3])) + ((sum8[4] + sum8[5]) + (sum8[6] + sum8[7]));
       asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
