@@ -492,6 +492,9 @@ __global__ void __launch_bounds__(kHistSimpleThreads) hist_simple_kernel(EncodeA
 // lens[b] += rows of sequence b (skipped for sequences that did not fit, or whose new positions reach a page outside
 // the pool: rows of such a sequence that did land in good pages stay beyond its length).
 __global__ void advance_lens_kernel(const int32_t* cu_seqlens, int batch, int capacity, Paging pg, int32_t* lens) {
+  // After a tensor-core encode this grid is launched ahead of time: wait for the encode grid (which reads the
+  // lengths) to complete.  Without such a predecessor the instruction does nothing.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= batch) return;
   const int count = cu_seqlens ? cu_seqlens[b + 1] - cu_seqlens[b] : 1;
@@ -519,7 +522,20 @@ static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
     const int32_t tc = try_launch_encode_tc(a, stream);
     if (tc < 0) return tc;
     if (tc == 1) {
-      advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, a.pg, lens);
+      // programmatic dependent launch: set up while the encode grid runs, starts when that grid has completed
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((a.batch + 127) / 128);
+      cfg.blockDim = dim3(128);
+      cfg.stream = stream;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      if (cudaLaunchKernelEx(&cfg, advance_lens_kernel, a.cu_seqlens, a.batch, a.capacity, a.pg, lens) != cudaSuccess) {
+        cudaGetLastError();
+        return PQ_ERR_CUDA;
+      }
       return launch_status();
     }
   }

@@ -85,6 +85,9 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
   const uint32_t sb = tc_smem_u32(smem);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  // The kernel that advances the lengths may be set up now; it waits (griddepcontrol.wait) until this grid has
+  // completed and its writes are visible, so only its launch latency is hidden.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int quarter = warp & 3;            // tensor-memory lanes this warp may read: rows 32 * quarter ..
   const int slot = warp >> 2;              // accumulator and tile sequence of this group of four warps
   const int st = quarter * 32 + lane;      // thread index inside the slot = row of the tile
