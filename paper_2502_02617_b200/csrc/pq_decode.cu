@@ -447,9 +447,19 @@ __global__ void merge_attention_kernel(int d, int64_t n_rows, int n_parts, const
 // Exact softmax attention (Eq. 2) of one query per sequence over an uncompressed window of keys and values (the
 // tokens a serving loop keeps in 16 bits, Section 5.3's protocol for generated tokens).  One CTA per (kv head,
 // sequence, split of the window's tokens); a CTA writes the partial attention of its tokens (part blockIdx.z of the
-// output), to be merged by merge_attention_kernel.  Chunks of kTailChunk tokens: scores by a thread per token (16-byte
-// loads of its key row), running maximum and denominator per head, then a thread per coordinate accumulates P . V.
-constexpr int kTailThreads = 128, kTailChunk = 512;
+// output), to be merged by merge_attention_kernel.  Steps of kTailStage tokens (half as many for a float32 window): the
+// key and value rows are copied to shared memory with coalesced 16-byte cp.async (all of a step's loads in flight at
+// once), then scores by a thread per token (key rows 16 bytes apart modulo 128: conflict-free 16-byte reads), running
+// maximum and denominator per head, then a thread per coordinate accumulates P . V.
+constexpr int kTailThreads = 128, kTailStage = 64;
+static_assert(2 * kTailStage <= kTailThreads, "two threads per staged token");
+constexpr int kTailSmemMax = 80 * 1024;
+__host__ __device__ inline int tail_stage_tokens(int kv_dtype) { return kv_dtype == PQ_DTYPE_BF16 ? kTailStage : kTailStage / 2; }
+__host__ __device__ inline size_t tail_smem_bytes(int d, int g, int kv_dtype) {
+  const int T = tail_stage_tokens(kv_dtype), row = d * (kv_dtype == PQ_DTYPE_BF16 ? 2 : 4);
+  const int h = 4 * ((g + 3) / 4);
+  return (size_t)4 * (h * d + h * kTailStage + 3 * kMaxGroup + 4) + (size_t)T * (row + 16) + (size_t)T * row;
+}
 struct TailArgs {
   int d, n_q_heads, n_kv_heads, io_dtype, kv_dtype, capacity, batch;
   float scale;
@@ -465,18 +475,27 @@ __device__ __forceinline__ float tail_elem(const void* p, int dtype, int64_t i) 
   return dtype == PQ_DTYPE_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(p)[i])
                                 : reinterpret_cast<const float*>(p)[i];
 }
+// kHG = groups of four query heads per kv head (heads past the group read q' = 0 and are not stored).
+template <int kHG>
 __global__ void __launch_bounds__(kTailThreads) tail_attention_kernel(TailArgs a) {
+  constexpr int kH = 4 * kHG;
   extern __shared__ float tsm[];
   const int d = a.d, g = a.n_q_heads / a.n_kv_heads, hk = blockIdx.x, b = blockIdx.y, tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
-  float* qs = tsm;                       // [g][d], times scale * log2(e)
-  float* sc = qs + g * d;                // [g][kTailChunk]
-  float* m_sm = sc + g * kTailChunk;     // [g] running maximum (log2 domain)
-  float* l_sm = m_sm + kMaxGroup;        // [g] running denominator
-  float* corr_sm = l_sm + kMaxGroup;     // [g]
-  for (int i = tid; i < g * d; i += kTailThreads)
-    qs[i] = tail_elem(a.q, a.io_dtype, ((int64_t)b * a.n_q_heads + hk * g) * d + i) * a.scale * 1.4426950408889634f;
-  if (tid < g) {
+  float* qs = tsm;                       // [d][kH]: q' = q * scale * log2(e), the heads of a coordinate side by side
+  float* sc = qs + kH * d;               // [kTailStage][kH]: scores, then probabilities, of a step
+  float* m_sm = sc + kH * kTailStage;    // [kH] running maximum (log2 domain)
+  float* l_sm = m_sm + kMaxGroup;        // [kH] running denominator
+  float* corr_sm = l_sm + kMaxGroup;     // [kH]
+  const int esz = a.kv_dtype == PQ_DTYPE_BF16 ? 2 : 4, row_bytes = d * esz, krow = row_bytes + 16;
+  const int T = tail_stage_tokens(a.kv_dtype);
+  uint8_t* ks = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(corr_sm + kMaxGroup) + 15) & ~(uintptr_t)15);   // [T][krow]
+  uint8_t* vs = ks + (size_t)T * krow;                                                                          // [T][row_bytes]
+  for (int i = tid; i < kH * d; i += kTailThreads) {
+    const int c = i / kH, h = i - c * kH;
+    qs[i] = h < g ? tail_elem(a.q, a.io_dtype, ((int64_t)b * a.n_q_heads + hk * g + h) * d + c) * a.scale * 1.4426950408889634f : 0.f;
+  }
+  if (tid < kH) {
     m_sm[tid] = -CUDART_INF_F;
     l_sm[tid] = 0.f;
   }
@@ -485,22 +504,36 @@ __global__ void __launch_bounds__(kTailThreads) tail_attention_kernel(TailArgs a
   const int per = (len_all + (int)gridDim.z - 1) / (int)gridDim.z;
   const int t_begin = min(len_all, (int)blockIdx.z * per), len = min(len_all, t_begin + per) - t_begin;
   const int64_t part_rows = (int64_t)blockIdx.z * a.batch * a.n_q_heads;   // this split's part of out and lse
-  float acc[kMaxGroup];
+  float acc[kH];
 #pragma unroll
-  for (int h = 0; h < kMaxGroup; ++h) acc[h] = 0.f;
-  __syncthreads();
-  for (int c0 = 0; c0 < len; c0 += kTailChunk) {
-    const int n = min(kTailChunk, len - c0);
-    for (int t = tid; t < n; t += kTailThreads) {
-      const int64_t row = (((int64_t)b * a.capacity + t_begin + c0 + t) * a.n_kv_heads + hk) * d;
-      float s[kMaxGroup];
+  for (int h = 0; h < kH; ++h) acc[h] = 0.f;
+  const uint32_t ks_s = (uint32_t)__cvta_generic_to_shared(ks), vs_s = (uint32_t)__cvta_generic_to_shared(vs);
+  const int gr_shift = 31 - __clz(row_bytes >> 4);   // 16-byte pieces of a row: a power of two
+  const int64_t row_stride = (int64_t)a.n_kv_heads * row_bytes;
+  const int64_t base = (((int64_t)b * a.capacity + t_begin) * a.n_kv_heads + hk) * row_bytes;
+  for (int c0 = 0; c0 < len; c0 += T) {
+    const int n = min(T, len - c0);
+    __syncthreads();   // the previous step's rows and probabilities have been used (first step: q', m, l are set)
+    for (int i = tid; i < (n << gr_shift); i += kTailThreads) {
+      const int t = i >> gr_shift, piece = i - (t << gr_shift);
+      const int64_t off = base + (c0 + t) * row_stride + 16 * piece;
+      pf_cp16(ks_s + t * krow + 16 * piece, reinterpret_cast<const uint8_t*>(a.k) + off);
+      pf_cp16(vs_s + t * row_bytes + 16 * piece, reinterpret_cast<const uint8_t*>(a.v) + off);
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    {   // scores: two threads per token, each over half of the coordinates (a stage holds at most 64 tokens)
+      const int t = tid >> 1, i0 = (tid & 1) * (d >> 1);
+      const uint8_t* row = ks + t * krow;
+      float s[kH];
 #pragma unroll
-      for (int h = 0; h < kMaxGroup; ++h) s[h] = 0.f;
-#pragma unroll 4
-      for (int i = 0; i < d; i += 8) {   // d is a multiple of 16 and rows are 16-byte aligned; four loads in flight
+      for (int h = 0; h < kH; ++h) s[h] = 0.f;
+#pragma unroll 2
+      for (int i = i0; i < i0 + (d >> 1) && t < n; i += 8) {   // d is a multiple of 16
         float kv[8];
         if (a.kv_dtype == PQ_DTYPE_BF16) {
-          const uint4 raw = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(a.k) + row + i));
+          const uint4 raw = *reinterpret_cast<const uint4*>(row + 2 * i);
           const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
@@ -508,38 +541,47 @@ __global__ void __launch_bounds__(kTailThreads) tail_attention_kernel(TailArgs a
             kv[2 * e + 1] = __uint_as_float(w[e] & 0xFFFF0000u);
           }
         } else {
-          const float4 lo = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(a.k) + row + i));
-          const float4 hi = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(a.k) + row + i + 4));
+          const float4 lo = *reinterpret_cast<const float4*>(row + 4 * i);
+          const float4 hi = *reinterpret_cast<const float4*>(row + 4 * i + 16);
           kv[0] = lo.x; kv[1] = lo.y; kv[2] = lo.z; kv[3] = lo.w; kv[4] = hi.x; kv[5] = hi.y; kv[6] = hi.z; kv[7] = hi.w;
         }
 #pragma unroll
-        for (int h = 0; h < kMaxGroup; ++h)
-          if (h < g) {
+        for (int e = 0; e < 8; ++e) {
 #pragma unroll
-            for (int e = 0; e < 8; ++e) s[h] = fmaf(qs[h * d + i + e], kv[e], s[h]);
+          for (int hg = 0; hg < kHG; ++hg) {   // one 16-byte broadcast read gives q' of four heads
+            const float4 q4 = *reinterpret_cast<const float4*>(qs + (i + e) * kH + 4 * hg);
+            s[4 * hg] = fmaf(q4.x, kv[e], s[4 * hg]);
+            s[4 * hg + 1] = fmaf(q4.y, kv[e], s[4 * hg + 1]);
+            s[4 * hg + 2] = fmaf(q4.z, kv[e], s[4 * hg + 2]);
+            s[4 * hg + 3] = fmaf(q4.w, kv[e], s[4 * hg + 3]);
           }
+        }
       }
 #pragma unroll
-      for (int h = 0; h < kMaxGroup; ++h)
-        if (h < g) sc[h * kTailChunk + t] = s[h];
+      for (int h = 0; h < kH; ++h) s[h] += __shfl_xor_sync(0xffffffffu, s[h], 1);
+      if (t < n && (tid & 1) == 0) {
+#pragma unroll
+        for (int hg = 0; hg < kHG; ++hg)
+          *reinterpret_cast<float4*>(sc + t * kH + 4 * hg) = make_float4(s[4 * hg], s[4 * hg + 1], s[4 * hg + 2], s[4 * hg + 3]);
+      }
     }
     __syncthreads();
     for (int h = warp; h < g; h += kTailThreads / 32) {   // a warp per head: maximum, probabilities, their sum
       float mx = -CUDART_INF_F;
-      for (int t = lane; t < n; t += 32) mx = fmaxf(mx, sc[h * kTailChunk + t]);
+      for (int t = lane; t < n; t += 32) mx = fmaxf(mx, sc[t * kH + h]);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
       const float m_new = fmaxf(m_sm[h], mx);
       float sum = 0.f;
       for (int t = lane; t < n; t += 32) {
-        const float p = exp2f(sc[h * kTailChunk + t] - m_new);
-        sc[h * kTailChunk + t] = p;
+        const float p = exp2f(sc[t * kH + h] - m_new);
+        sc[t * kH + h] = p;
         sum += p;
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
       if (lane == 0) {
-        const float corr = exp2f(m_sm[h] - m_new);   // 0 on the first chunk
+        const float corr = exp2f(m_sm[h] - m_new);   // 0 on the first step
         corr_sm[h] = corr;
         l_sm[h] = l_sm[h] * corr + sum;
         m_sm[h] = m_new;
@@ -548,21 +590,26 @@ __global__ void __launch_bounds__(kTailThreads) tail_attention_kernel(TailArgs a
     __syncthreads();
     if (tid < d) {
 #pragma unroll
-      for (int h = 0; h < kMaxGroup; ++h)
-        if (h < g) acc[h] *= corr_sm[h];
+      for (int h = 0; h < kH; ++h) acc[h] *= h < g ? corr_sm[h] : 0.f;
 #pragma unroll 8
       for (int t = 0; t < n; ++t) {
-        const float vv = tail_elem(a.v, a.kv_dtype, (((int64_t)b * a.capacity + t_begin + c0 + t) * a.n_kv_heads + hk) * d + tid);
+        const float vv = a.kv_dtype == PQ_DTYPE_BF16 ? __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(vs + t * row_bytes)[tid])
+                                                     : reinterpret_cast<const float*>(vs + t * row_bytes)[tid];
 #pragma unroll
-        for (int h = 0; h < kMaxGroup; ++h)
-          if (h < g) acc[h] = fmaf(sc[h * kTailChunk + t], vv, acc[h]);
+        for (int hg = 0; hg < kHG; ++hg) {
+          const float4 p4 = *reinterpret_cast<const float4*>(sc + t * kH + 4 * hg);
+          acc[4 * hg] = fmaf(p4.x, vv, acc[4 * hg]);
+          acc[4 * hg + 1] = fmaf(p4.y, vv, acc[4 * hg + 1]);
+          acc[4 * hg + 2] = fmaf(p4.z, vv, acc[4 * hg + 2]);
+          acc[4 * hg + 3] = fmaf(p4.w, vv, acc[4 * hg + 3]);
+        }
       }
     }
-    __syncthreads();
   }
+  __syncthreads();
   if (tid < d) {
 #pragma unroll
-    for (int h = 0; h < kMaxGroup; ++h)
+    for (int h = 0; h < kH; ++h)
       if (h < g) {
         const float o = len > 0 ? acc[h] / l_sm[h] : 0.f;
         const int64_t oi = (part_rows + (int64_t)b * a.n_q_heads + hk * g + h) * d + tid;
@@ -858,9 +905,14 @@ int32_t pq_tail_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_head
   a.capacity = tail_capacity; a.batch = batch; a.scale = scale; a.q = q_dev; a.k = k_tail_dev; a.v = v_tail_dev; a.lens = tail_lens_dev;
   a.out = out_dev; a.lse = lse_dev; a.status = status_dev;
   const int g = n_q_heads / n_kv_heads;
-  const size_t smem = sizeof(float) * ((size_t)g * head_dim + (size_t)g * pq::kTailChunk + 3 * pq::kMaxGroup);
+  const size_t smem = pq::tail_smem_bytes(head_dim, g, kv_dtype);
+  static pq::DeviceMemo configured1, configured2;
+  if (smem > (size_t)pq::kTailSmemMax) return PQ_ERR_UNSUPPORTED;
+  if (pq::configure_for_device(pq::tail_attention_kernel<1>, pq::kTailSmemMax, configured1) == 0) return PQ_ERR_CUDA;
+  if (pq::configure_for_device(pq::tail_attention_kernel<2>, pq::kTailSmemMax, configured2) == 0) return PQ_ERR_CUDA;
   dim3 grid(n_kv_heads, batch, n_splits);
-  pq::tail_attention_kernel<<<grid, pq::kTailThreads, smem, reinterpret_cast<cudaStream_t>(stream)>>>(a);
+  if (g <= 4) pq::tail_attention_kernel<1><<<grid, pq::kTailThreads, smem, reinterpret_cast<cudaStream_t>(stream)>>>(a);
+  else pq::tail_attention_kernel<2><<<grid, pq::kTailThreads, smem, reinterpret_cast<cudaStream_t>(stream)>>>(a);
   return pq::launch_status();
 }
 
