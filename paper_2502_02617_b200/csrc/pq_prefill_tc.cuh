@@ -137,8 +137,8 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
   uint32_t crank = 0;
   if (kPair) asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(crank));
   const bool leader = crank == 0;   // the CTA whose thread issues the MMAs and whose barriers collect the arrivals
-  // per-CTA shapes of the B operands: keys of kKTok tokens (two coordinate halves), values of 64 tokens x kVHalves x 64 coordinates
-  // A key tile holds, for each half of the coordinates, the fp16 values of the kKTok tokens followed by their residuals:
+  // Per-CTA shapes of the B operands: keys of kKTok tokens (two coordinate halves), values of 64 tokens x kVHalves x 64
+  // coordinates.  A key tile holds, for each half of the coordinates, the fp16 values of the kKTok tokens followed by their residuals:
   // one B operand of 2 kKTok rows, so one MMA gives the products with both.
   constexpr int kKTok = kPair ? 32 : 64, kKLo = kKTok * 128, kKHalf = 2 * kKLo, kKTile = 2 * kKHalf, kVHalves = kPair ? 1 : 2;
   constexpr int kStage = kKTile + kVHalves * 8192;
@@ -451,9 +451,6 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
       if (kPair) tc_commit_pair(bar);
       else tc_commit(bar);
     };
-    auto wait_all = [&](uint32_t bar, uint32_t parity) -> bool {   // barriers that warps of both CTAs arrive on
-      return tc_mbar_wait(bar, parity, abort_flag);
-    };
     uint64_t vdesc_hi = (uint64_t)(1024 >> 4) << 32;   // stride between groups of 8 tokens
     vdesc_hi |= (uint64_t)1 << 46;
     vdesc_hi |= (uint64_t)2 << 61;
@@ -461,7 +458,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
     const uint64_t desc_hi = tc_smem_desc(0u) & 0xFFFFFFFF00000000ull;
     auto issue_pv = [&](int jb) -> bool {   // O (+)= P_jb V_hat_jb
       const int t = jb & 1, st = jb % kPtStages;
-      if (!wait_all(bar_pfull + 8 * t, (uint32_t)(jb >> 1) & 1u)) return false;
+      if (!tc_mbar_wait(bar_pfull + 8 * t, (uint32_t)(jb >> 1) & 1u, abort_flag)) return false;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const uint32_t v_lo = (((sb + kPtSmKv + st * kStage + kKTile) & 0x3FFFFu) >> 4) | vdesc_lbo;
 #pragma unroll
@@ -484,7 +481,7 @@ __global__ void __launch_bounds__(kPtThreads, 1) prefill_tc_kernel(DecodeArgs a,
         if (!ok) break;
       }
       const int st = jb % kPtStages;
-      ok = wait_all(bar_kv + 8 * st, (uint32_t)(jb / kPtStages) & 1u);
+      ok = tc_mbar_wait(bar_kv + 8 * st, (uint32_t)(jb / kPtStages) & 1u, abort_flag);
       // accumulator t is free: its scores were read before P_{jb-2} was announced, and the value MMA that read
       // P_{jb-2} from its columns was issued in the previous iteration (MMAs of one thread execute in order)
       if (ok && (a.debug & 2u) && (blockIdx.x | blockIdx.y | blockIdx.z) == 0 && jb == min(2, n_blocks - 1)) {
