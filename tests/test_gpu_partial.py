@@ -98,10 +98,11 @@ def test_merge_reports_rows_without_any_token():
 
 
 @pytest.mark.parametrize("d,Hq,Hkv,dtype", [(128, 8, 2, torch.bfloat16), (128, 32, 8, torch.bfloat16), (64, 4, 4, torch.bfloat16),
-                                             (16, 2, 1, torch.float32)])
+                                             (16, 2, 1, torch.float32),
+                                             (128, 8, 1, torch.bfloat16), (128, 4, 2, torch.float32)])   # eight heads per kv head; float32 rows
 def test_compressed_cache_followed_by_an_unquantised_window(d, Hq, Hkv, dtype):
     """Section 5.3's protocol: prompt tokens compressed, generated tokens kept in 16 bits.  Windows of 0, 3 and 600
-    tokens (more than one chunk of the window kernel), one sequence with an empty compressed part."""
+    tokens (more than one step of the window kernel), one sequence with an empty compressed part."""
     lens, tails, T = [300, 0, 64], [0, 3, 600], 640
     B = len(lens)
     cache = pq.PolarQuantCache(B, Hq, Hkv, d, capacity=320, seed=8, device=DEV)
