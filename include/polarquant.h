@@ -206,9 +206,11 @@ int32_t pq_decode_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_he
  *   q_dev, out_dev   [batch][n_q][n_q_heads][head_dim] of `io_dtype`
  *   workspace_dev    pq_workspace_bytes(head_dim, batch * n_q, n_q_heads, n_kv_heads, max_len) bytes
  * A query that sees no token (lens[b] < n_q - j) yields zeros and records PQ_ERR_EMPTY.  At head_dim 128, chunks
- * of at least 64 / (n_q_heads / n_kv_heads) queries run on a kernel that decodes every block of the cache once for 64
- * (query, head) rows and contracts on tensor cores (no workspace is touched); shorter chunks and other head_dims
- * decode the cache once per query (the cost is n_q decode attentions).  batch * n_q must not exceed 65535.
+ * of at least 128 rows (queries x query heads per kv head) run on a kernel that decodes every block of the cache
+ * once for 128 -- two CTAs together: 256 -- rows and contracts on the tensor cores (no workspace is touched); so do
+ * chunks of 32 to 127 rows when that is estimated to be faster (large batches, see pq_debug_fail_next_wait); shorter
+ * chunks and other head_dims decode the cache once per query (the cost is n_q decode attentions).  batch * n_q
+ * must not exceed 65535.
  */
 int32_t pq_multi_query_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_kv_heads, const float* S_dev,
                                  const void* tables_dev, const void* q_dev, int32_t io_dtype, const void* cache_dev,
@@ -250,16 +252,19 @@ int32_t pq_decode_attention_static(int32_t head_dim, int32_t n_q_heads, int32_t 
  * Test support: make the next launch of one kernel run its give-up path.  `which` = 1 arms the
  * tensor-core encoder behind pq_encode_kv (head_dim 128, bf16, >= 128 rows), 2 arms the head_dim-128
  * kernel behind pq_decode_attention, 4 the tcgen05 kernel behind pq_multi_query_attention (head_dim 128,
- * chunks of 128 rows and more: its MMA-issuing thread gives up after two blocks, the other warps of the
- * CTA follow, the rows of that CTA are not written), 0 disarms.  In the armed launch the first bounded wait of one CTA
+ * chunks that take that kernel, see below: its MMA-issuing thread gives up after two blocks, the other warps of
+ * the CTA -- of the CTA pair -- follow, their rows are not written), 0 disarms.  In the armed launch the first bounded wait of one CTA
  * (the one that starts the first tile / the first non-empty sequence) is reported as failed although
  * what it waited for arrived: the CTA abandons its share of the work,
  * waits for its copies in flight, releases what it holds and records PQ_ERR_TIMEOUT in status word 0;
  * nothing on the device is left waiting and the next call runs normally.  (The paper has no
  * counterpart: it exercises the error handling of Section "General rules" without losing a copy.)
- * `which` = 3 is of another kind: the next pq_multi_query_attention call at head_dim 128 whose chunk fills
- * 128 rows runs the register-fragment (mma.sync) kernel instead of the tcgen05 one, so that the two can
- * be compared on the same inputs.
+ * `which` = 3 is of another kind: the next pq_multi_query_attention call at head_dim 128 whose chunk has
+ * 64 or more rows (queries x query heads per kv head) runs the register-fragment (mma.sync) kernel, which
+ * no call reaches otherwise, so that it can be compared with the product path on the same inputs.  (The
+ * tcgen05 kernel takes chunks of 128 rows and more, and chunks of 32 to 127 rows when its estimated time
+ * -- kv heads x sequences CTA pairs walking max_len / 64 blocks -- is below that of one decode attention
+ * per query; everything else runs the decode kernels with one (sequence, query) pair per unit.)
  */
 int32_t pq_debug_fail_next_wait(int32_t which);
 

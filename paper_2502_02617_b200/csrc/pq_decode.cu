@@ -1,5 +1,6 @@
 // Decode attention over the packed cache (Eq. 3) and the inspection kernels.
 #include <atomic>
+#include <cmath>
 #include <chrono>
 #include <math_constants.h>
 
@@ -731,17 +732,42 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
   a.ws = pq::carve_workspace(workspace_dev, head_dim, (int)pairs, n_q_heads, n_kv_heads, max_len);
   const int g = n_q_heads / n_kv_heads;
   if (lse_dev != nullptr && n_q != 1) return PQ_ERR_UNSUPPORTED;
-  if (head_dim == 128 && n_q * g >= pq::kPtRows && !pq::take_debug_wait_failure(3)) {
-    // Chunks that fill 128 rows: the tcgen05 kernel (operands in shared memory, accumulators in tensor memory).
+  // Chunks of 32 or more rows (queries x heads of a group), d = 128: the tcgen05 kernel (operands in shared memory,
+  // accumulators in tensor memory) decodes every block once for all rows; below 128 rows it is taken when that is
+  // estimated to be faster than one decode attention per query, which spreads over all SMs whatever the batch.
+  // The register-fragment kernel is only reached through the test hook (it is the slower of the two at every size).
+  const int rows = n_q * g;
+  bool use_tc = false, use_fragment_kernel = false;
+  int n_sm = 0, q_blocks = 0;
+  bool pair = false;
+  if (head_dim == 128 && rows >= 32) {
     static pq::DeviceMemo configured_pt, configured_pt2;
-    const int n_sm = pq::configure_for_device(pq::prefill_tc_kernel<false>, pq::kPtSmTotal, configured_pt);
+    n_sm = pq::configure_for_device(pq::prefill_tc_kernel<false>, pq::kPtSmTotal, configured_pt);
     if (n_sm == 0) return PQ_ERR_CUDA;
     if (pq::configure_for_device(pq::prefill_tc_kernel<true>, pq::kPtSmTotal, configured_pt2) == 0) return PQ_ERR_CUDA;
     const int qb_rows = pq::kPtRows / g;
-    const int q_blocks = (n_q + qb_rows - 1) / qb_rows;
+    q_blocks = (n_q + qb_rows - 1) / qb_rows;
+    // Two query blocks of one (kv head, sequence) per cluster: one 256-row MMA per step, each CTA decodes half of
+    // every block.  An odd count is completed by a CTA without rows -- also a single block when the pairs still fit
+    // on the device at once: the second CTA then only shares the decoding (the kernel is bound by it).
+    pair = q_blocks >= 2 || 2 * (int64_t)n_kv_heads * batch <= n_sm;
+    if (rows >= pq::kPfRows && pq::take_debug_wait_failure(3)) {
+      use_fragment_kernel = true;
+    } else if (rows >= pq::kPtRows) {
+      use_tc = true;
+    } else {
+      // measured on B200: 1.25 us (pair) or 2.4 us per 64-token block and CTA; decode attention at 1.7 TB/s of packed bytes
+      const double ctas = (double)n_kv_heads * batch * (pair ? 2.0 : 1.0);
+      const double waves = std::ceil(ctas / n_sm);
+      const double t_tc = waves * std::ceil(max_len / 64.0) * (pair ? 1.25 : 2.4) + 10.0;
+      const double t_decode = (double)pairs * n_kv_heads * max_len * 124.0 / 1.7e6 + 10.0;
+      use_tc = t_tc < t_decode || pairs * n_kv_heads > pq::kFastMaxUnits;
+    }
+  }
+  if (use_tc) {
     a.epoch = 0u;
     a.debug = pq::take_debug_wait_failure(4) ? 2u : 0u;
-    if (q_blocks >= 2 || 2 * (int64_t)n_kv_heads * batch <= n_sm) {
+    if (pair) {
       // Two query blocks of one (kv head, sequence) per cluster: one 256-row MMA per step, each CTA decodes half of
       // every block.  An odd count is completed by a CTA without rows -- also a single block when the pairs still fit
       // on the device at once: the second CTA then only shares the decoding (the kernel is bound by it).
@@ -767,8 +793,8 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
     pq::prefill_tc_kernel<false><<<grid, pq::kPtThreads, pq::kPtSmTotal, st>>>(a, n_q);
     return pq::launch_status();
   }
-  if (head_dim == 128 && n_q * g >= pq::kPfRows) {
-    // Many queries per sequence: decode each block of the cache once for 64 (query, head) rows on tensor cores.
+  if (use_fragment_kernel) {
+    // decode each block of the cache once for 64 (query, head) rows, mma.sync on register fragments
     static pq::DeviceMemo configured_pf;
     if (pq::configure_for_device(pq::prefill_attention_kernel, pq::kPfTotal, configured_pf) == 0) return PQ_ERR_CUDA;
     const int qb_rows = pq::kPfRows / g;

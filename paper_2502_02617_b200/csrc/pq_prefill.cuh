@@ -9,8 +9,10 @@
 // on tensor cores (mma.sync m16n8k16 fed by ldmatrix; a warp owns 16 rows).  The queries are rotated by S
 // once when the CTA starts (Q' = Q S * scale * log2 e, kept as fp16 value + residual) and the output by S^T
 // once when it ends, as in decode attention.  There is no split over the tokens: the grid is
-// (query blocks, kv heads, sequences), which fills the GPU for chunks of a prefill; chunks that do not fill the 64
-// rows of a CTA go through the decode kernel instead (one decode per query).
+// (query blocks, kv heads, sequences), which fills the GPU for chunks of a prefill.
+// This is the first implementation of the path.  The tcgen05 kernel (pq_prefill_tc.cuh) is faster at every size and
+// takes every chunk this one could; the dispatch reaches this kernel only through the test hook, for chunks of 64
+// rows and more, so that two independent implementations can be compared on the same inputs.
 #pragma once
 
 namespace pq {
