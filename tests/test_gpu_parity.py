@@ -262,6 +262,43 @@ def test_multi_query_single_block_on_a_full_device(n_q, B):
         assert rel_l2(to_f64(out[b:b + 1]), want) < TOL_ATTENTION_F32_IO, b
 
 
+def test_multi_query_random_shapes_agree_with_the_other_paths_and_repeat_bit_for_bit():
+    """Seeded random (group size, kv heads, batch, capacity, chunk length, ragged lengths): whatever kernel the dispatch
+    picks, the result repeats bit for bit and agrees with another path -- the register-fragment kernel for chunks of
+    64 rows and more, one decode attention per query over the tokens that query sees for shorter ones."""
+    rng = np.random.default_rng(5)
+    for it in range(24):
+        g, Hkv = int(rng.choice([1, 2, 3, 4, 5, 8])), int(rng.choice([1, 2, 4, 8]))
+        B, cap = int(rng.choice([1, 2, 3, 8, 20, 40])), int(rng.choice([70, 200, 700, 2100]))
+        n_q = max(1, min(int(rng.choice([32, 64, 100, 128, 160, 256, 300, 520])) // g, cap))
+        lens = [cap] + [int(rng.integers(0, cap + 1)) for _ in range(B - 1)]
+        cache = pq.PolarQuantCache(B, g * Hkv, Hkv, 128, capacity=cap, seed=it, device=DEV)
+        K, V = synthetic.kv_like(it, sum(lens), Hkv, 128, torch.bfloat16, DEV)
+        cache.encode(K, V, torch.tensor(np.concatenate(([0], np.cumsum(lens))), dtype=torch.int32, device=DEV))
+        gen = torch.Generator(device=DEV)
+        gen.manual_seed(it)
+        q = torch.randn((B, n_q, g * Hkv, 128), generator=gen, device=DEV, dtype=torch.float32)
+        out = cache.attend_multi(q).clone()
+        again = cache.attend_multi(q)
+        torch.cuda.synchronize()
+        assert cache.status.cpu().tolist()[0] in (pq.OK, pq.ERR_EMPTY)
+        assert torch.equal(out, again) and bool(torch.isfinite(out).all()), (it, g, Hkv, B, cap, n_q)
+        cache.status.zero_()
+        if n_q * g >= 64:
+            pq.pq_debug_fail_next_wait(3)
+            other = cache.attend_multi(q)
+        else:
+            held, parts = cache.lens.clone(), []
+            for j in range(n_q):
+                cache.lens.copy_((held - (n_q - 1 - j)).clamp(min=0))
+                parts.append(cache.attend(q[:, j].contiguous()).clone())
+            cache.lens.copy_(held)
+            other = torch.stack(parts, dim=1)
+        torch.cuda.synchronize()
+        assert rel_l2(to_f64(out), to_f64(other)) < 6e-4, (it, g, Hkv, B, cap, n_q)
+    pq.pq_debug_fail_next_wait(0)
+
+
 def want_bf16(orc, ref, qb, d):
     return orc.multi_query_attention(to_f64(qb), ref.k_codes, ref.k_radii, ref.v_codes, ref.v_radii, ref.lens, ref.cb, ref.S,
                                      d ** -0.5)
