@@ -291,6 +291,7 @@ __device__ inline void fix_rounds(const EncodeArgs& a, Q* q, unsigned long long 
 }
 
 __global__ void __launch_bounds__(kFfmaThreads) encode_ffma_kernel(EncodeArgs a) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the length update may be set up (it waits for this grid)
   extern __shared__ __align__(16) float smem_f[];
   float* xT = smem_f;                  // [128 k][129]
   float* rowsq = smem_f + 128 * 129;   // [2][128]
@@ -365,6 +366,7 @@ __global__ void __launch_bounds__(kFfmaThreads) encode_ffma_kernel(EncodeArgs a)
 // decided exactly.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128) encode_vector_kernel(EncodeArgs a) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the length update may be set up (it waits for this grid)
   __shared__ float xs[128];
   __shared__ float ys[128];
   __shared__ double yd[128];
@@ -492,8 +494,7 @@ __global__ void __launch_bounds__(kHistSimpleThreads) hist_simple_kernel(EncodeA
 // lens[b] += rows of sequence b (skipped for sequences that did not fit, or whose new positions reach a page outside
 // the pool: rows of such a sequence that did land in good pages stay beyond its length).
 __global__ void advance_lens_kernel(const int32_t* cu_seqlens, int batch, int capacity, Paging pg, int32_t* lens) {
-  // After a tensor-core encode this grid is launched ahead of time: wait for the encode grid (which reads the
-  // lengths) to complete.  Without such a predecessor the instruction does nothing.
+  // This grid is launched ahead of time: wait for the encode grid (which reads the lengths) to complete.
   asm volatile("griddepcontrol.wait;" ::: "memory");
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= batch) return;
@@ -516,42 +517,43 @@ static int32_t check_common(int head_dim, int n_kv_heads, const void* S, const v
   return PQ_OK;
 }
 
+// The length update as a programmatic dependent launch of the encode kernel before it (which allows it with
+// griddepcontrol.launch_dependents): set up while that grid runs, started when it has completed.
+static int32_t launch_advance_lens(const EncodeArgs& a, int32_t* lens, cudaStream_t stream) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((a.batch + 127) / 128);
+  cfg.blockDim = dim3(128);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, advance_lens_kernel, a.cu_seqlens, a.batch, a.capacity, a.pg, lens) != cudaSuccess) {
+    cudaGetLastError();
+    return PQ_ERR_CUDA;
+  }
+  return launch_status();
+}
+
 static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
   if (a.total_tokens == 0) return PQ_OK;
   {
     const int32_t tc = try_launch_encode_tc(a, stream);
     if (tc < 0) return tc;
-    if (tc == 1) {
-      // programmatic dependent launch: set up while the encode grid runs, starts when that grid has completed
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3((a.batch + 127) / 128);
-      cfg.blockDim = dim3(128);
-      cfg.stream = stream;
-      cudaLaunchAttribute attr[1];
-      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-      attr[0].val.programmaticStreamSerializationAllowed = 1;
-      cfg.attrs = attr;
-      cfg.numAttrs = 1;
-      if (cudaLaunchKernelEx(&cfg, advance_lens_kernel, a.cu_seqlens, a.batch, a.capacity, a.pg, lens) != cudaSuccess) {
-        cudaGetLastError();
-        return PQ_ERR_CUDA;
-      }
-      return launch_status();
-    }
+    if (tc == 1) return launch_advance_lens(a, lens, stream);
   }
   if (a.head_dim == 128 && a.total_tokens < 32) {
     const int64_t n_vec = (int64_t)a.total_tokens * 2 * a.n_kv_heads;
     encode_vector_kernel<<<(unsigned)n_vec, 128, 0, stream>>>(a);
-    advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, a.pg, lens);
-    return launch_status();
+    return launch_advance_lens(a, lens, stream);
   }
   if (a.head_dim == 128 && a.total_tokens >= 32) {
     static DeviceMemo configured;
     if (configure_for_device(encode_ffma_kernel, kFfmaSmem, configured) == 0) return PQ_ERR_CUDA;
     dim3 grid((a.total_tokens + 127) / 128, a.n_kv_heads, 2);
     encode_ffma_kernel<<<grid, kFfmaThreads, kFfmaSmem, stream>>>(a);
-    advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, a.pg, lens);
-    return launch_status();
+    return launch_advance_lens(a, lens, stream);
   }
   const int groups = kExactThreads / a.head_dim;
   const int vec_per_cta = kExactVecPerGroup * groups;
@@ -559,8 +561,7 @@ static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
   const int64_t grid = (n_vec + vec_per_cta - 1) / vec_per_cta;
   const size_t smem = (size_t)2 * vec_per_cta * a.head_dim * sizeof(double);
   encode_exact_kernel<<<(unsigned)grid, kExactThreads, smem, stream>>>(a);
-  advance_lens_kernel<<<(a.batch + 127) / 128, 128, 0, stream>>>(a.cu_seqlens, a.batch, a.capacity, a.pg, lens);
-  return pq::launch_status();
+  return launch_advance_lens(a, lens, stream);
 }
 
 }  // namespace pq
