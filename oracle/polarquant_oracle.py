@@ -19,7 +19,8 @@ Conventions (the paper is 1-indexed, this file is 0-indexed):
 * Level 1 angles live in [0, 2*pi), higher levels in [0, pi/2] (Definition 1).
 
 Pins (tests/test_oracle_*.py): exact invertibility of the unquantised transform,
-block radius == block norm, norm preservation under S, Lemma 2 densities against the
+block radius == block norm, norm preservation under S, the structured preconditioners against the closed form of
+the Sylvester matrix and the fast Walsh-Hadamard butterfly, Lemma 2 densities against the
 incomplete-beta CDF, Lloyd-Max fixed-point equations against independent quadrature,
 the worked d=4 example under tests/golden/, brute force on d=4 and d=16, closed-form
 expected distortion, the len=1 / identical-keys attention special cases, multi-query attention against a
@@ -52,6 +53,25 @@ def make_rotation(d: int, seed: int) -> np.ndarray:
     q, r = np.linalg.qr(g)
     sign = np.where(np.diag(r) < 0.0, -1.0, 1.0)
     return q * sign[None, :]
+
+
+def make_structured_rotation(d: int, kind: str, signs=None) -> np.ndarray:
+    """Preconditioners without a dense random matrix.  Section 3.2 only asks for an orthogonal S that spreads a vector
+    over its coordinates (the footnote's fast transforms), and Section 5's rows named "PolarQuant" (without "-R") use
+    none at all.  kind "identity": S = I.  kind "hadamard": S = diag(signs) H_d / sqrt(d), with H_d the Sylvester
+    Hadamard matrix of a power-of-two order, H_1 = [1], H_2n = [[H_n, H_n], [H_n, -H_n]], and signs in {+1, -1}
+    drawn by the caller (y = x . S flips the signs of x, then transforms)."""
+    if kind == "identity":
+        return np.eye(d, dtype=np.float64)
+    if kind != "hadamard" or d < 1 or d & (d - 1):
+        raise ValueError("kind must be 'identity' or 'hadamard' (power-of-two order)")
+    H = np.ones((1, 1), dtype=np.float64)
+    while H.shape[0] < d:
+        H = np.block([[H, H], [H, -H]])
+    sg = np.asarray(signs, dtype=np.float64)
+    if sg.shape != (d,) or not np.all(np.abs(sg) == 1.0):
+        raise ValueError("signs must be d entries of +1 or -1")
+    return sg[:, None] * H / np.sqrt(float(d))
 
 
 def rotate(x: np.ndarray, S: np.ndarray) -> np.ndarray:

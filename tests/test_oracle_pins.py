@@ -83,6 +83,33 @@ def test_rotation_is_orthogonal_and_preserves_geometry(d):
     assert np.array_equal(orc.make_rotation(d, seed=7), S)  # and is reproducible
 
 
+@pytest.mark.parametrize("d", [2, 16, 128])
+def test_structured_preconditioners_are_what_their_definitions_say(d):
+    """Section 3.2 / Section 5 ("PolarQuant" without "-R"): the identity, and diag(signs) H / sqrt(d) with the Sylvester
+    matrix.  Pinned by the closed form H[i][j] = (-1)^popcount(i & j), by H H^T = d I in exact integers, by the
+    fast Walsh-Hadamard butterfly applied to a vector, and by the order-2 matrix written out."""
+    rng = np.random.default_rng(d)
+    signs = rng.choice([-1.0, 1.0], size=d)
+    S = orc.make_structured_rotation(d, "hadamard", signs)
+    H = np.rint(S * np.sqrt(d) * signs[:, None]).astype(np.int64)      # undo the scaling and the row signs
+    assert np.array_equal(H, [[(-1) ** bin(i & j).count("1") for j in range(d)] for i in range(d)])
+    assert np.array_equal(H @ H.T, d * np.eye(d, dtype=np.int64))
+    assert np.allclose(S @ S.T, np.eye(d), atol=1e-14) and np.allclose(np.abs(S), d ** -0.5, atol=1e-16)
+    x = rng.standard_normal(d)
+    y = x * signs                      # y = x . S: sign flips, butterflies, scaling
+    h = 1
+    while h < d:
+        y = y.reshape(-1, 2, h)
+        y = np.stack([y[:, 0] + y[:, 1], y[:, 0] - y[:, 1]], axis=1).reshape(-1)
+        h *= 2
+    assert np.allclose(orc.rotate(x[None], S)[0], y / np.sqrt(d), atol=1e-12)
+    if d == 2:
+        assert np.allclose(orc.make_structured_rotation(2, "hadamard", [1, -1]), np.array([[1, 1], [-1, 1]]) / np.sqrt(2))
+    assert np.array_equal(orc.make_structured_rotation(d, "identity"), np.eye(d))
+    with pytest.raises(ValueError):
+        orc.make_structured_rotation(12, "hadamard", np.ones(12))
+
+
 # ---------------------------------------------------------------- densities (Lemma 2)
 def _cdf(level, psi):
     """sin^2(psi) ~ Beta(2^(l-2), 2^(l-2)): Lemma 2's density after a change of variable."""
