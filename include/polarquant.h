@@ -85,6 +85,21 @@ int32_t pq_token_block(void);
 int32_t pq_make_rotation(int32_t head_dim, uint64_t seed, float* S_host);
 
 /*
+ * Preconditioners without a dense random matrix (Section 3.2 asks only for an orthogonal S; its footnote
+ * names fast transforms; Section 5's rows called "PolarQuant" without "-R" use none).  Written to
+ * S_host[d*d] like pq_make_rotation; every entry point takes the result like any other S.
+ *   kind = PQ_ROTATION_IDENTITY   S = I (signs_host is ignored and may be NULL)
+ *   kind = PQ_ROTATION_HADAMARD   S = diag(signs) . H_d / sqrt(d), H_d the Sylvester Hadamard matrix
+ *                                 (H_1 = [1], H_2n = [[H_n, H_n], [H_n, -H_n]]; head_dim a power of two);
+ *                                 signs_host[d] holds +1 / -1 drawn by the caller
+ * Returns PQ_ERR_INVALID_ARG for a NULL output, an unknown kind, a sign other than +1 / -1 or a missing sign
+ * array, PQ_ERR_UNSUPPORTED for a head_dim that is not a power of two (Hadamard) or above 4096.
+ */
+#define PQ_ROTATION_IDENTITY 0
+#define PQ_ROTATION_HADAMARD 1
+int32_t pq_make_structured_rotation(int32_t head_dim, int32_t kind, const int8_t* signs_host, float* S_host);
+
+/*
  * Angle codebooks (Algorithm 1 line 3, Eq. 4) for the analytic densities of Lemma 2:
  * level 1 uniform on [0, 2pi), level l >= 2 proportional to sin^(2^(l-1)-1)(2 psi) on
  * [0, pi/2].  Lloyd-Max iteration in float64 on the host.

@@ -31,6 +31,7 @@ _SIGNATURES = {
     "pq_last_cuda_error": (c_char_p, []),
     "pq_token_block": (c_int32, []),
     "pq_make_rotation": (c_int32, [c_int32, c_uint64, c_void_p]),
+    "pq_make_structured_rotation": (c_int32, [c_int32, c_int32, c_void_p, c_void_p]),
     "pq_fit_codebooks": (c_int32, [POINTER(c_int32), POINTER(c_double), POINTER(c_double)]),
     "pq_angle_histograms": (c_int32, [c_int32, c_int32, c_void_p, c_void_p, c_void_p, c_int32, c_int64, c_int64, c_int32,
                                       c_int32, c_void_p, c_void_p, c_void_p]),
@@ -163,6 +164,19 @@ def pq_make_rotation(d: int, seed: int) -> torch.Tensor:
     _check(lib().pq_make_rotation(d, seed, S.data_ptr()), "pq_make_rotation")
     return S
 
+
+
+ROTATION_IDENTITY, ROTATION_HADAMARD = 0, 1
+
+
+def pq_make_structured_rotation(d: int, kind: int, signs=None) -> torch.Tensor:
+    """S = I, or diag(signs) . H_d / sqrt(d) with the Sylvester Hadamard matrix; `signs`: d values of +1 / -1 (int8)."""
+    S = torch.empty((d, d), dtype=torch.float32)
+    sg = None if signs is None else torch.as_tensor(signs).to(torch.int8).contiguous()
+    if sg is not None and sg.numel() != d:
+        raise ValueError("signs must have head_dim entries")
+    _check(lib().pq_make_structured_rotation(d, kind, 0 if sg is None else sg.data_ptr(), S.data_ptr()), "pq_make_structured_rotation")
+    return S
 
 def pq_fit_codebooks(bits=DEFAULT_BITS):
     """Analytic Lloyd-Max codebooks: (centroids float64[28], boundaries float64[24]) CPU tensors."""

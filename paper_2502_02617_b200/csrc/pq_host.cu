@@ -209,6 +209,31 @@ int32_t pq_debug_fail_next_wait(int32_t which) {
   return PQ_OK;
 }
 
+int32_t pq_make_structured_rotation(int32_t d, int32_t kind, const int8_t* signs_host, float* S_host) {
+  if (S_host == nullptr || d <= 0) return PQ_ERR_INVALID_ARG;
+  if (kind != PQ_ROTATION_IDENTITY && kind != PQ_ROTATION_HADAMARD) return PQ_ERR_INVALID_ARG;
+  if (d > 4096) return PQ_ERR_UNSUPPORTED;
+  if (kind == PQ_ROTATION_IDENTITY) {
+    for (int i = 0; i < d; ++i)
+      for (int j = 0; j < d; ++j) S_host[(size_t)i * d + j] = i == j ? 1.f : 0.f;
+    return PQ_OK;
+  }
+  if (d & (d - 1)) return PQ_ERR_UNSUPPORTED;
+  if (signs_host == nullptr) return PQ_ERR_INVALID_ARG;
+  for (int i = 0; i < d; ++i)
+    if (signs_host[i] != 1 && signs_host[i] != -1) return PQ_ERR_INVALID_ARG;
+  // entry (i, j) of the Sylvester matrix: -1 to the number of bit positions set in both indices
+  const double c = 1.0 / std::sqrt((double)d);
+  for (int i = 0; i < d; ++i)
+    for (int j = 0; j < d; ++j) {
+      unsigned both = (unsigned)i & (unsigned)j;
+      int odd = 0;
+      for (; both; both &= both - 1) odd ^= 1;
+      S_host[(size_t)i * d + j] = (float)((odd ? -c : c) * (double)signs_host[i]);
+    }
+  return PQ_OK;
+}
+
 int32_t pq_make_rotation(int32_t d, uint64_t seed, float* S_host) {
   if (S_host == nullptr || d <= 0) return PQ_ERR_INVALID_ARG;
   if (d > 4096) return PQ_ERR_UNSUPPORTED;

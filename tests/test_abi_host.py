@@ -52,6 +52,27 @@ def test_rotation_is_orthogonal_seeded_and_gaussianising(d):
     assert 0.5 < np.mean(row ** 2) < 1.5 and np.max(np.abs(row)) < 6.0
 
 
+@pytest.mark.parametrize("d", [16, 64, 128, 256])
+def test_structured_preconditioners_equal_the_oracle(d):
+    """Identity and sign-flipped Sylvester-Hadamard (Section 3.2's fast transforms; Section 5's rows without R): the
+    library's closed form against the oracle's recursion, entry by entry after rounding to float32."""
+    signs = np.random.default_rng(d).choice([-1, 1], size=d).astype(np.int8)
+    S = pq.pq_make_structured_rotation(d, pq.ROTATION_HADAMARD, signs).numpy()
+    want = orc.make_structured_rotation(d, "hadamard", signs.astype(np.float64))
+    assert np.array_equal(S, want.astype(np.float32))
+    assert np.max(np.abs(S.astype(np.float64).T @ S.astype(np.float64) - np.eye(d))) < 1e-6
+    assert np.array_equal(pq.pq_make_structured_rotation(d, pq.ROTATION_IDENTITY).numpy(), np.eye(d, dtype=np.float32))
+    bad = signs.copy()
+    bad[3] = 0
+    out = np.empty((d, d), dtype=np.float32)
+    f = pq.lib().pq_make_structured_rotation
+    assert f(d, pq.ROTATION_HADAMARD, bad.ctypes.data, out.ctypes.data) == pq.ERR_INVALID_ARG
+    assert f(d, pq.ROTATION_HADAMARD, None, out.ctypes.data) == pq.ERR_INVALID_ARG
+    assert f(d, 7, signs.ctypes.data, out.ctypes.data) == pq.ERR_INVALID_ARG
+    assert f(d, pq.ROTATION_IDENTITY, None, None) == pq.ERR_INVALID_ARG
+    assert f(48, pq.ROTATION_HADAMARD, signs.ctypes.data, out.ctypes.data) == pq.ERR_UNSUPPORTED
+
+
 def test_rotation_rejects_bad_arguments():
     assert pq.lib().pq_make_rotation(0, 1, None) == pq.ERR_INVALID_ARG
     assert pq.lib().pq_make_rotation(16, 1, None) == pq.ERR_INVALID_ARG

@@ -304,6 +304,39 @@ def want_bf16(orc, ref, qb, d):
                                      d ** -0.5)
 
 
+@pytest.mark.parametrize("kind,d,dtype", [("hadamard", 128, torch.bfloat16), ("hadamard", 64, torch.float32),
+                                           ("identity", 128, torch.bfloat16), ("identity", 16, torch.float32)])
+def test_structured_preconditioners_encode_and_attend_like_the_oracle(kind, d, dtype):
+    """S = sign-flipped Hadamard / sqrt(d) and S = I (the paper's rows without preconditioning) through the same entry
+    points as a random S.  Without mixing, bf16 coordinates tie exactly (a = b puts a level-1 angle on a boundary of the
+    uniform codebook): the float64 re-decision must break those ties like the oracle."""
+    Hq, Hkv, lens_list = 8, 2, [300, 70]
+    signs = np.random.default_rng(3).choice([-1, 1], size=d).astype(np.int8)
+    S = pq.pq_make_structured_rotation(d, pq.ROTATION_HADAMARD if kind == "hadamard" else pq.ROTATION_IDENTITY, signs)
+    cache = pq.PolarQuantCache(len(lens_list), Hq, Hkv, d, capacity=320, seed=0, device=DEV, S=S)
+    K, V = synthetic.kv_like(41, sum(lens_list), Hkv, d, dtype, DEV, n_outliers=4 if d >= 64 else 0)
+    _encode_and_compare(cache, K, V, lens_list)
+    ref = _oracle_cache(cache, K, V, lens_list)
+    q = synthetic.queries(42, len(lens_list), Hq, d, torch.float32, DEV)
+    out = cache.attend(q)
+    torch.cuda.synchronize()
+    cache.check_status()
+    want = ref.attend(to_f64(q), d ** -0.5)
+    for b in range(len(lens_list)):
+        assert rel_l2(to_f64(out[b]), want[b]) < TOL_ATTENTION_F32_IO, b
+    if d == 128:
+        n_q = 40   # 160 rows: the tcgen05 multi-query kernel rotates by the same S
+        g = torch.Generator(device=DEV)
+        g.manual_seed(43)
+        qm = torch.randn((len(lens_list), n_q, Hq, d), generator=g, device=DEV, dtype=torch.float32)
+        got = to_f64(cache.attend_multi(qm))
+        torch.cuda.synchronize()
+        wantm = orc.multi_query_attention(to_f64(qm), ref.k_codes, ref.k_radii, ref.v_codes, ref.v_radii, ref.lens, ref.cb,
+                                          ref.S, d ** -0.5)
+        for b in range(len(lens_list)):
+            assert rel_l2(got[b], wantm[b]) < TOL_ATTENTION_F32_IO, b
+
+
 def test_capacity_overflow_and_empty_sequence_are_reported_not_faulted():
     d, Hq, Hkv = 128, 4, 1
     cache = pq.PolarQuantCache(2, Hq, Hkv, d, capacity=64, seed=7, device=DEV)
