@@ -27,6 +27,8 @@
  *       [0] first error code seen (0 = none)      [1] non-finite input elements seen
  *       [2] radii that saturated at the fp16 max  [3] 16-coordinate blocks that were
  *                                                     re-encoded by the float64 path
+ *   - pq_make_rotation, pq_fit_codebooks, the encode / append calls and the attention calls open an NVTX
+ *     range for the duration of the host call (a no-op unless a profiler is attached).
  *   - Row-vector convention of Algorithm 1: y = x . S, x_hat = y_hat . S^T; S is stored
  *     row-major [head_dim][head_dim] in float32.
  *   - Shapes: head_dim d in {16, 32, 64, 128}; L = 4 levels; bits (4,2,2,2) (Section 4.1);

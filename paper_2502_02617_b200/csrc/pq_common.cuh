@@ -8,9 +8,20 @@
 
 #include <atomic>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/polarquant.h"
 
 namespace pq {
+
+// NVTX range around a C-ABI call (shows the call in a timeline next to its kernels; a no-op without a profiler).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+  NvtxRange(const NvtxRange&) = delete;
+  NvtxRange& operator=(const NvtxRange&) = delete;
+};
+
 
 constexpr int kTokenBlock = 64;  // tokens per cache token-block
 constexpr int kMaxGroup = 8;     // query heads per kv head that one thread block of an attention kernel handles

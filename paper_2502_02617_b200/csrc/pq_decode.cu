@@ -709,6 +709,7 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
                                 const int32_t* cache_lens_dev, int32_t batch, int32_t n_q, int32_t capacity, const pq::Paging& pg,
                                 int32_t max_len, float scale, void* out_dev, void* workspace_dev, int32_t* status_dev,
                                 void* stream, float* lse_dev = nullptr) {
+  pq::NvtxRange nvtx_range("pq attention");
   if (!(head_dim == 16 || head_dim == 32 || head_dim == 64 || head_dim == 128)) return PQ_ERR_UNSUPPORTED;
   if (!S_dev || !tables_dev || !q_dev || !cache_dev || !cache_lens_dev || !out_dev || !workspace_dev || !status_dev)
     return PQ_ERR_INVALID_ARG;

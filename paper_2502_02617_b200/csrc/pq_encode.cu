@@ -571,6 +571,7 @@ static int32_t encode_entry(int32_t head_dim, int32_t n_kv_heads, const float* S
                             int64_t head_stride, const int32_t* cu_seqlens_dev, int32_t batch, int32_t total_tokens,
                             void* cache_dev, int32_t* cache_lens_dev, int32_t capacity, const pq::Paging& pg,
                             int32_t* status_dev, void* stream) {
+  pq::NvtxRange nvtx_range("pq_encode_kv");
   int32_t st = pq::check_common(head_dim, n_kv_heads, S_dev, tables_dev, cache_dev, cache_lens_dev, status_dev);
   if (st != PQ_OK) return st;
   if (!K_dev || !V_dev || !cu_seqlens_dev || batch <= 0 || total_tokens < 0 || capacity <= 0) return PQ_ERR_INVALID_ARG;
@@ -593,6 +594,7 @@ static int32_t append_entry(int32_t head_dim, int32_t n_kv_heads, const float* S
                             const void* k_new_dev, const void* v_new_dev, int32_t in_dtype, int32_t batch,
                             void* cache_dev, int32_t* cache_lens_dev, int32_t capacity, const pq::Paging& pg,
                             int32_t* status_dev, void* stream) {
+  pq::NvtxRange nvtx_range("pq_append_kv");
   int32_t st = pq::check_common(head_dim, n_kv_heads, S_dev, tables_dev, cache_dev, cache_lens_dev, status_dev);
   if (st != PQ_OK) return st;
   if (!k_new_dev || !v_new_dev || batch <= 0 || capacity <= 0) return PQ_ERR_INVALID_ARG;

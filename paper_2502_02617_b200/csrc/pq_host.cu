@@ -235,6 +235,7 @@ int32_t pq_make_structured_rotation(int32_t d, int32_t kind, const int8_t* signs
 }
 
 int32_t pq_make_rotation(int32_t d, uint64_t seed, float* S_host) {
+  pq::NvtxRange nvtx_range("pq_make_rotation");
   if (S_host == nullptr || d <= 0) return PQ_ERR_INVALID_ARG;
   if (d > 4096) return PQ_ERR_UNSUPPORTED;
   std::vector<double> A((size_t)d * d), Q((size_t)d * d, 0.0), v(d), w(d), rdiag(d);
@@ -277,6 +278,7 @@ int32_t pq_make_rotation(int32_t d, uint64_t seed, float* S_host) {
 }
 
 int32_t pq_fit_codebooks(const int32_t* bits, double* centroids_host, double* boundaries_host) {
+  pq::NvtxRange nvtx_range("pq_fit_codebooks");
   if (bits == nullptr || centroids_host == nullptr || boundaries_host == nullptr) return PQ_ERR_INVALID_ARG;
   if (bits[0] != 4 || bits[1] != 2 || bits[2] != 2 || bits[3] != 2) return PQ_ERR_UNSUPPORTED;
   for (int level = 1; level <= PQ_N_LEVELS; ++level) {
