@@ -371,6 +371,7 @@ __global__ void __launch_bounds__(128) encode_vector_kernel(EncodeArgs a) {
   __shared__ float ys[128];
   __shared__ double yd[128];
   __shared__ float red[4];
+  __shared__ uint32_t amb_blocks;   // bit b: block b has a decision that float32 cannot certify
   __shared__ FastQuant fq;
   const int j = threadIdx.x;
   const int64_t v = blockIdx.x;  // vector index: (row * 2 + kv) * n_kv_heads + head
@@ -383,7 +384,10 @@ __global__ void __launch_bounds__(128) encode_vector_kernel(EncodeArgs a) {
     set_status(a.status, PQ_ERR_NONFINITE);
   }
   xs[j] = xv;
-  if (j == 0) load_fast_quant(a.tables, &fq);
+  if (j == 0) {
+    load_fast_quant(a.tables, &fq);
+    amb_blocks = 0u;
+  }
   __syncthreads();
   float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 8
@@ -408,13 +412,16 @@ __global__ void __launch_bounds__(128) encode_vector_kernel(EncodeArgs a) {
     if (fq.analytic) polar_quant_block_fast<true>(yb, make_row_margins(norm, kRotErr, fq), fq, &fb);
     else polar_quant_block_fast<false>(yb, make_row_margins(norm, kRotErr, fq), fq, &fb);
   }
+  if (fb.amb != 0u) atomicOr(&amb_blocks, 1u << j);
   if (__syncthreads_or(fb.amb != 0u)) {
-    double accd[4] = {0.0, 0.0, 0.0, 0.0};
-    for (int k = 0; k < 128; k += 4) {
+    if ((amb_blocks >> (j >> 4)) & 1u) {   // only the coordinates of the blocks in question (half-warps: the float64 pipe is slow)
+      double accd[4] = {0.0, 0.0, 0.0, 0.0};
+      for (int k = 0; k < 128; k += 4) {
 #pragma unroll
-      for (int i = 0; i < 4; ++i) accd[i] = fma((double)xs[k + i], (double)__ldg(a.S + (k + i) * 128 + j), accd[i]);
+        for (int i = 0; i < 4; ++i) accd[i] = fma((double)xs[k + i], (double)__ldg(a.S + (k + i) * 128 + j), accd[i]);
+      }
+      yd[j] = (accd[0] + accd[1]) + (accd[2] + accd[3]);
     }
-    yd[j] = (accd[0] + accd[1]) + (accd[2] + accd[3]);
     __syncthreads();
     if (j < 8 && fb.amb != 0u) {
       double yb[16];
