@@ -824,7 +824,20 @@ static int32_t launch_attention(int32_t head_dim, int32_t n_q_heads, int32_t n_k
     const int n_sm = pq::configure_for_device(kernel, pq::kSmTotal, configured[(g <= 4 ? 0 : 1) + (paged ? 2 : 0)]);
     if (n_sm == 0) return PQ_ERR_CUDA;
     const int grid = n_sm < pq::kFastMaxGrid ? n_sm : pq::kFastMaxGrid;
-    kernel<<<grid, pq::kFastThreads, pq::kSmTotal, st>>>(a);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(pq::kFastThreads);
+    cfg.dynamicSmemBytes = pq::kSmTotal;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];   // may be set up while the kernel before it in the stream finishes (it waits inside)
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kernel, a) != cudaSuccess) {
+      cudaGetLastError();
+      return PQ_ERR_CUDA;
+    }
     return pq::launch_status();
   }
   a.epoch = 0u;

@@ -288,6 +288,12 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // Launched as a programmatic dependent of the kernel before it in the stream: everything up to here may run
+  // while that kernel finishes; its results (lengths, cache, queries, workspace) are read only after this wait.
+  // The kernel after this one may be set up as soon as this grid has started.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  build_fast_tables(smem, a.tables);   // from the caller's tables, which no kernel writes
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   __syncthreads();
 
   // ---- persistent work split: the 128-token stages of all units, in unit order, are cut into
@@ -449,9 +455,6 @@ __global__ void __launch_bounds__(kFastThreads, 1) decode_attention_fast_kernel(
     const bool producer = (tid & 255) == 0;
     if (producer && n_li > 0) issue_copy(0);
     __syncwarp();
-    // The lookup tables are filled once, with the CTA's first copies already on their way (the barriers
-    // of the query rotation below order the fill before the first lookup).
-    if (sg == 0 && batch_no == 0) build_fast_tables(smem, a.tables);
     // q' = (q S) * scale * log2(e) for the unit's query heads, as an fp16 value plus an fp16 residual.
     // The first stages of the segment are already on their way while this runs.
     {
