@@ -58,13 +58,17 @@ __device__ __forceinline__ bool hist_block(const float* y, uint32_t* h, int n_bi
   s3[0] = s2[0] + s2[1];
   s3[1] = s2[2] + s2[3];
   if (!(s3[0] + s3[1] < CUDART_INF_F)) return false;
+  // all fifteen bins first (independent dependency chains that overlap), then the fifteen counts
+  int bin[15];
 #pragma unroll
-  for (int j = 0; j < 8; ++j) atomicAdd(h + hist_bin_level1(y[2 * j], y[2 * j + 1], scale1, n_bins), 1u);
+  for (int j = 0; j < 8; ++j) bin[j] = hist_bin_level1(y[2 * j], y[2 * j + 1], scale1, n_bins);
 #pragma unroll
-  for (int j = 0; j < 4; ++j) atomicAdd(h + n_bins + hist_bin_upper(s1[2 * j], s1[2 * j + 1], scale_up, n_bins), 1u);
+  for (int j = 0; j < 4; ++j) bin[8 + j] = n_bins + hist_bin_upper(s1[2 * j], s1[2 * j + 1], scale_up, n_bins);
 #pragma unroll
-  for (int j = 0; j < 2; ++j) atomicAdd(h + 2 * n_bins + hist_bin_upper(s2[2 * j], s2[2 * j + 1], scale_up, n_bins), 1u);
-  atomicAdd(h + 3 * n_bins + hist_bin_upper(s3[0], s3[1], scale_up, n_bins), 1u);
+  for (int j = 0; j < 2; ++j) bin[12 + j] = 2 * n_bins + hist_bin_upper(s2[2 * j], s2[2 * j + 1], scale_up, n_bins);
+  bin[14] = 3 * n_bins + hist_bin_upper(s3[0], s3[1], scale_up, n_bins);
+#pragma unroll
+  for (int j = 0; j < 15; ++j) atomicAdd(h + bin[j], 1u);
   return true;
 }
 
