@@ -134,6 +134,9 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     for (int i = 0; i < kTcSlots; ++i) tc_mbar_init(bar_acc + 8 * i, 1);   // one commit by the slot's issuing thread
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // Launched as a programmatic dependent of the kernel before it in the stream (which may have produced K and V):
+    // its results are read only after this wait; the set-up around it overlaps that kernel's tail.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int it = 0; it < kTcStages; ++it) issue_tma(it);  // the first tiles arrive while S is split
     if (!kHist) {
       load_fast_quant(a.tables, fq);
@@ -190,6 +193,7 @@ encode_tc_kernel(EncodeArgs a, const __grid_constant__ TcMaps maps, int n_row_ti
     }
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the MMA unit
+  asm volatile("griddepcontrol.wait;" ::: "memory");            // every thread reads lengths and writes the cache below
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -465,7 +469,20 @@ static int32_t try_launch_tc(const EncodeArgs& a, cudaStream_t stream) {
   const int grid = n_tiles < n_sm ? n_tiles : n_sm;
   EncodeArgs args = a;
   if (take_debug_wait_failure(1)) args.debug |= 1u;
-  encode_tc_kernel<kHist, kPaged><<<grid, kTcThreads, kTcSmTotal, stream>>>(args, maps, n_row_tiles);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = kTcSmTotal;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];   // may be set up while the kernel before it in the stream finishes (it waits inside)
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (cudaLaunchKernelEx(&cfg, encode_tc_kernel<kHist, kPaged>, args, maps, n_row_tiles) != cudaSuccess) {
+    cudaGetLastError();
+    return PQ_ERR_CUDA;
+  }
   return 1;
 }
 static int32_t try_launch_encode_tc(const EncodeArgs& a, cudaStream_t stream) {
