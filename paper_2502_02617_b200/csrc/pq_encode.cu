@@ -366,7 +366,10 @@ __global__ void __launch_bounds__(kFfmaThreads) encode_ffma_kernel(EncodeArgs a)
 // decided exactly.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128) encode_vector_kernel(EncodeArgs a) {
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the length update may be set up (it waits for this grid)
+  // a programmatic dependent of the kernel before it (which may have produced the vectors, or still reads the lengths):
+  // nothing of the stream is read before the wait; the length update after this grid may be set up at once
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   __shared__ float xs[128];
   __shared__ float ys[128];
   __shared__ double yd[128];
@@ -552,7 +555,19 @@ static int32_t launch_encode(EncodeArgs a, int32_t* lens, cudaStream_t stream) {
   }
   if (a.head_dim == 128 && a.total_tokens < 32) {
     const int64_t n_vec = (int64_t)a.total_tokens * 2 * a.n_kv_heads;
-    encode_vector_kernel<<<(unsigned)n_vec, 128, 0, stream>>>(a);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)n_vec);
+    cfg.blockDim = dim3(128);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];   // may be set up while the kernel before it in the stream finishes (it waits inside)
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, encode_vector_kernel, a) != cudaSuccess) {
+      cudaGetLastError();
+      return PQ_ERR_CUDA;
+    }
     return launch_advance_lens(a, lens, stream);
   }
   if (a.head_dim == 128 && a.total_tokens >= 32) {
