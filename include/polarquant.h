@@ -20,7 +20,11 @@
  *     test hook of pq_debug_fail_next_wait.  All of it is updated atomically: host threads may call
  *     into the library concurrently as long as they do not share output buffers or scratch.
  *   - Device work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
- *     legacy default stream) and the call returns without synchronising.
+ *     legacy default stream) and the call returns without synchronising.  The encode, append and
+ *     decode-attention kernels are launched as programmatic dependents of whatever kernel precedes
+ *     them in the stream: they may set up (barriers, tables from the caller's constant inputs) while
+ *     that kernel finishes, and read K, V, q, the cache, the lengths and the workspace only after it
+ *     has completed, so stream order holds for everything a caller can observe.
  *   - Problems that only the device can see (a sequence that would exceed `capacity`,
  *     an empty sequence in attention, non-finite inputs) are written to the caller's
  *     status words `status_dev` (int32[PQ_STATUS_WORDS], zero it before the first call):
