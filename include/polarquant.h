@@ -24,7 +24,10 @@
  *     decode-attention kernels are launched as programmatic dependents of whatever kernel precedes
  *     them in the stream: they may set up (barriers, tables from the caller's constant inputs) while
  *     that kernel finishes, and read K, V, q, the cache, the lengths and the workspace only after it
- *     has completed, so stream order holds for everything a caller can observe.
+ *     has completed, so stream order holds for everything a caller can observe.  S_dev and
+ *     tables_dev are the exception: they are read during that set-up, so they must not be written
+ *     by the kernel that directly precedes the call in the stream (a copy, as in the binding, or any
+ *     other operation in between is fine).
  *   - Problems that only the device can see (a sequence that would exceed `capacity`,
  *     an empty sequence in attention, non-finite inputs) are written to the caller's
  *     status words `status_dev` (int32[PQ_STATUS_WORDS], zero it before the first call):
